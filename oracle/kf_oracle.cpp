@@ -1,0 +1,207 @@
+// kf_oracle.cpp -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+//
+// Plain, slow, fp64 CPU restatement of the fused operator chains that the
+// "Kernel Foundry" paper's search produces kernels for.  Every function here is the
+// chain's textbook definition written out as loops; nothing is blocked, fused or
+// reordered beyond what the definition states.  Only tests, the smoke check and the
+// benchmark's cpu_baseline / reference arm may load this file; the CUDA library never
+// does, and the two share no code, headers, tables or helpers.
+//
+// Passages followed:
+//   * "Operator Fusion ... (e.g. matmul + relu)" and "Algorithmic Optimization ...
+//     online softmax" (Appendix A, allowed optimisation strategies 2 and 3): the chains
+//     are a contraction followed by elementwise and reduction operators, and the fused
+//     kernel must keep "full functional equivalence" with the PyTorch chain (Appendix A,
+//     output requirement 1; Section 4.1 "numerical equivalence to PyTorch").
+//   * Softmax: the three-pass definition printed in Appendix C.1 (row max, sum of
+//     exp(x - max), quotient), and expert recommendation "Correctness 1" (normalise
+//     before exponentiation, high-precision accumulators).
+//   * Activations: Appendix C.2 listing formulas -- sigmoid(x)*x (swish), tanh written as
+//     (e^{2s}-1)/(e^{2s}+1), GELU in its erf form t*0.5*(1+erf(t/sqrt 2)), hardtanh as
+//     clamp to [-1,1].  GELU-tanh is the usual PyTorch approximate='tanh' definition.
+//   * Convolution / GroupNorm: Table 2 "Conv-centered" chains; PyTorch semantics
+//     (cross-correlation, zero padding, biased variance, eps inside the root).
+//
+// Pins (tests/test_oracle_*.py): closed forms, fixed activation values, invariants
+// (softmax rows sum to 1, shift invariance, sigmoid antisymmetry, GroupNorm moments),
+// brute force with exact rational arithmetic on tiny shapes.  No function here is
+// "parity unpinned".
+//
+// Storage dtypes: 0 = fp32, 1 = bf16 (uint16 bit patterns).  All arithmetic is fp64 on
+// the widened stored values; outputs are fp64 and never rounded.
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <vector>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+namespace {
+
+enum { DT_F32 = 0, DT_BF16 = 1 };
+enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SIGMOID = 3, ACT_GELU_ERF = 4,
+       ACT_SWISH = 5, ACT_TANH = 6, ACT_HARDTANH = 7, ACT_CHAIN95 = 8 };
+enum { RED_SOFTMAX = 0, RED_SUM = 1 };
+
+int g_threads = 0;  // 0 = OpenMP default
+
+inline double widen(const void* p, int dt, int64_t i) {
+  if (dt == DT_F32) return (double)((const float*)p)[i];
+  uint32_t bits = (uint32_t)((const uint16_t*)p)[i] << 16;  // bf16 = top half of an fp32
+  float f;
+  std::memcpy(&f, &bits, 4);
+  return (double)f;
+}
+
+inline double sigmoid(double z) { return 1.0 / (1.0 + std::exp(-z)); }
+
+double act_apply(int act, double z) {
+  switch (act) {
+    case ACT_NONE: return z;
+    case ACT_RELU: return z > 0.0 ? z : 0.0;
+    case ACT_GELU_TANH: {
+      const double c = 0.7978845608028654;  // sqrt(2/pi)
+      return 0.5 * z * (1.0 + std::tanh(c * (z + 0.044715 * z * z * z)));
+    }
+    case ACT_SIGMOID: return sigmoid(z);
+    case ACT_GELU_ERF: return z * 0.5 * (1.0 + std::erf(z * 0.7071067811865475));
+    case ACT_SWISH: return sigmoid(z) * z;
+    case ACT_TANH: return std::tanh(z);
+    case ACT_HARDTANH: return std::fmin(std::fmax(z, -1.0), 1.0);
+    case ACT_CHAIN95: {
+      // Appendix C.2: swish -> tanh -> GELU(erf) -> hardtanh, applied after the addend.
+      double s = sigmoid(z) * z;
+      double e = std::exp(2.0 * s);
+      double t = std::isinf(e) ? 1.0 : (e - 1.0) / (e + 1.0);
+      double g = t * 0.5 * (1.0 + std::erf(t * 0.7071067811865475));
+      return std::fmin(std::fmax(g, -1.0), 1.0);
+    }
+  }
+  return NAN;
+}
+
+inline int nthreads() {
+#ifdef _OPENMP
+  return g_threads > 0 ? g_threads : omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+}  // namespace
+
+extern "C" {
+
+void oracle_set_threads(int n) { g_threads = n; }
+int oracle_get_threads(void) { return nthreads(); }
+
+double oracle_act(int act, double z) { return act_apply(act, z); }
+
+// Z[m,n] = sum_k X[m,k] * W[n,k] + bias[n]   (torch Linear: W is [out,in])
+// Y[m,n] = scale * act(Z[m,n]) + R[m,n]      order: bias, activation, scale, residual
+// bias, R may be null.  Y is fp64 [M,N], dense.
+int oracle_gemm_epilogue(int64_t M, int64_t N, int64_t K, int dt, const void* X, int64_t ldx,
+                         const void* W, int64_t ldw, const void* bias, int act, double scale,
+                         const void* R, int64_t ldr, double* Y) {
+#pragma omp parallel for schedule(static) num_threads(nthreads())
+  for (int64_t m = 0; m < M; ++m) {
+    for (int64_t n = 0; n < N; ++n) {
+      double z = 0.0;
+      for (int64_t k = 0; k < K; ++k) z += widen(X, dt, m * ldx + k) * widen(W, dt, n * ldw + k);
+      if (bias) z += widen(bias, dt, n);
+      double y = scale * act_apply(act, z);
+      if (R) y += widen(R, dt, m * ldr + n);
+      Y[m * N + n] = y;
+    }
+  }
+  return 0;
+}
+
+// A[m,n] = pre_act(sum_k X[m,k] W[n,k] + bias[n])
+// red = SOFTMAX: out[m,n] = exp(A[m,n]-max_n A[m,:]) / sum_n exp(A[m,n]-max)   (out is [M,N])
+// red = SUM:     out[m]   = sum_n A[m,n]                                        (out is [M])
+int oracle_gemm_rowreduce(int64_t M, int64_t N, int64_t K, int dt, const void* X, int64_t ldx,
+                          const void* W, int64_t ldw, const void* bias, int pre_act, int red,
+                          double* out) {
+#pragma omp parallel for schedule(static) num_threads(nthreads())
+  for (int64_t m = 0; m < M; ++m) {
+    std::vector<double> a((size_t)N);
+    for (int64_t n = 0; n < N; ++n) {
+      double z = 0.0;
+      for (int64_t k = 0; k < K; ++k) z += widen(X, dt, m * ldx + k) * widen(W, dt, n * ldw + k);
+      if (bias) z += widen(bias, dt, n);
+      a[(size_t)n] = act_apply(pre_act, z);
+    }
+    if (red == RED_SOFTMAX) {
+      double mx = -INFINITY;
+      for (int64_t n = 0; n < N; ++n) mx = std::fmax(mx, a[(size_t)n]);
+      double s = 0.0;
+      for (int64_t n = 0; n < N; ++n) s += std::exp(a[(size_t)n] - mx);
+      for (int64_t n = 0; n < N; ++n) out[m * N + n] = std::exp(a[(size_t)n] - mx) / s;
+    } else {
+      double s = 0.0;
+      for (int64_t n = 0; n < N; ++n) s += a[(size_t)n];
+      out[m] = s;
+    }
+  }
+  return 0;
+}
+
+// c[n,o,h,w] = bias[o] + sum_{c,r,s} x[n,c,h+r-1,w+s-1] * wt[o,c,r,s]   zero padding, stride 1
+// a = act(c)
+// groups > 0: per (n,g), channels [g*Cout/groups, (g+1)*Cout/groups):
+//   mu = mean(a), var = mean((a-mu)^2) (biased), y = (a-mu)/sqrt(var+eps)*gamma[o]+beta[o]
+// groups == 0: y = a.   gamma/beta null => 1/0.   y is fp64 NCHW.
+int oracle_conv3x3_gn(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout, int dt,
+                      const void* x, const void* wt, const void* bias, int act, int groups,
+                      double eps, const void* gamma, const void* beta, double* y) {
+  if (groups > 0 && Cout % groups != 0) return 1;
+#pragma omp parallel for schedule(dynamic) num_threads(nthreads())
+  for (int64_t n = 0; n < Nb; ++n) {
+    for (int64_t o = 0; o < Cout; ++o) {
+      for (int64_t h = 0; h < H; ++h) {
+        for (int64_t w = 0; w < Wd; ++w) {
+          double acc = bias ? widen(bias, dt, o) : 0.0;
+          for (int64_t c = 0; c < Cin; ++c) {
+            for (int r = 0; r < 3; ++r) {
+              int64_t hh = h + r - 1;
+              if (hh < 0 || hh >= H) continue;
+              for (int s = 0; s < 3; ++s) {
+                int64_t ww = w + s - 1;
+                if (ww < 0 || ww >= Wd) continue;
+                acc += widen(x, dt, ((n * Cin + c) * H + hh) * Wd + ww) *
+                       widen(wt, dt, ((o * Cin + c) * 3 + r) * 3 + s);
+              }
+            }
+          }
+          y[((n * Cout + o) * H + h) * Wd + w] = act_apply(act, acc);
+        }
+      }
+    }
+    if (groups > 0) {
+      int64_t cpg = Cout / groups;
+      int64_t cnt = cpg * H * Wd;
+      for (int64_t g = 0; g < groups; ++g) {
+        double* blk = y + (n * Cout + g * cpg) * H * Wd;  // channels of a group are contiguous
+        double mu = 0.0;
+        for (int64_t i = 0; i < cnt; ++i) mu += blk[i];
+        mu /= (double)cnt;
+        double var = 0.0;
+        for (int64_t i = 0; i < cnt; ++i) var += (blk[i] - mu) * (blk[i] - mu);
+        var /= (double)cnt;
+        double rstd = 1.0 / std::sqrt(var + eps);
+        for (int64_t i = 0; i < cnt; ++i) {
+          int64_t o = g * cpg + i / (H * Wd);
+          double ga = gamma ? widen(gamma, dt, o) : 1.0;
+          double be = beta ? widen(beta, dt, o) : 0.0;
+          blk[i] = (blk[i] - mu) * rstd * ga + be;
+        }
+      }
+    }
+  }
+  return 0;
+}
+
+}  // extern "C"

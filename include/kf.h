@@ -1,0 +1,138 @@
+/* kf.h -- C ABI of the fused-operator-chain library for NVIDIA B200 (sm_100a).
+ *
+ * The library executes, as one hand-written CUDA kernel per chain (plus a streaming second
+ * pass where a reduction spans tiles), the operator chains the Kernel Foundry paper's search
+ * targets: a dense contraction followed by its elementwise and reduction epilogue.  The
+ * problem statement mirrored here is the paper's own (Section 3.1 and Appendix A, output
+ * requirement 1): a given PyTorch operator chain in, a kernel with "full functional
+ * equivalence" out, with every operator computed inside the kernel rather than by an
+ * external library call (Section 3.2.2, anti-cheating rule).
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers on the current CUDA device.  The caller owns
+ *     every buffer, including the workspace; the library allocates no device memory.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Calls only enqueue work on that stream and return; nothing synchronises.
+ *   - Matrices are row-major with a leading dimension in ELEMENTS (ld >= row length).
+ *   - dtype KF_F32 = IEEE fp32, KF_BF16 = bfloat16.  bf16 chains accumulate in fp32 on the
+ *     tensor cores, apply the epilogue in fp32 and round once (nearest-even) on store.
+ *     fp32 chains use fp32 FMA throughout (no TF32).
+ *   - bias / gamma / beta vectors have the chain's io dtype.
+ *   - Errors are return codes; nothing throws, aborts or prints.  On any code other than
+ *     KF_OK no kernel was launched by that call.  Inputs must be finite.
+ *   - The workspace must be 256-byte aligned and at least the size the matching
+ *     *_workspace_bytes() query returns (which may be 0, in which case NULL is accepted).
+ *     Its contents need not be initialised and are undefined afterwards.  Two calls that
+ *     share a workspace must be ordered on one stream.
+ *   - There is no CPU fallback: without a CUDA device the calls return KF_ERR_CUDA.
+ */
+#ifndef KF_H_
+#define KF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  KF_OK = 0,
+  KF_ERR_INVALID_ARG = 1, /* null/misaligned pointer, non-positive size, ld too small, bad enum */
+  KF_ERR_UNSUPPORTED = 2, /* a valid request this build has no kernel for */
+  KF_ERR_WORKSPACE = 3,   /* workspace null, misaligned or too small */
+  KF_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed (no device, launch error) */
+  KF_ERR_TIMEOUT = 5      /* a device-side bounded wait ran out (reported by kf_device_status) */
+} kf_status;
+
+typedef enum { KF_F32 = 0, KF_BF16 = 1 } kf_dtype;
+
+/* Activations.  0..3 are the benchmark chains' (the paper's "matmul + relu" class,
+ * Appendix A strategy 2); 4..8 are the operators of the paper's worked chain (Appendix C.2):
+ * erf-form GELU t*0.5*(1+erf(t/sqrt 2)), swish sigmoid(x)*x, tanh, hardtanh clamp[-1,1], and
+ * KF_ACT_CHAIN95 = hardtanh(gelu_erf(tanh(swish(z)))) applied to z = XW^T + bias. */
+typedef enum {
+  KF_ACT_NONE = 0,
+  KF_ACT_RELU = 1,
+  KF_ACT_GELU_TANH = 2,
+  KF_ACT_SIGMOID = 3,
+  KF_ACT_GELU_ERF = 4,
+  KF_ACT_SWISH = 5,
+  KF_ACT_TANH = 6,
+  KF_ACT_HARDTANH = 7,
+  KF_ACT_CHAIN95 = 8
+} kf_act;
+
+typedef enum { KF_RED_SOFTMAX = 0, KF_RED_SUM = 1 } kf_rowred;
+
+/* GEMM + elementwise epilogue (Appendix A, "Operator Fusion": matmul + activation class;
+ * Table 2 "Matmul-centered").
+ *   Y[m,n] = scale * act( sum_k X[m,k]*W[n,k] + bias[n] ) + residual[m,n]
+ * in that order: bias, activation, scale, residual.  X is [M,K] (ldx), W is [N,K] (ldw) as in
+ * torch.nn.Linear, residual and Y are [M,N] (ldr, ldy).  bias and residual may be NULL.
+ * Y must not alias X or W; Y may alias residual only if ldr == ldy (same element, same place).
+ * Shapes: any M,N,K >= 1.  bf16 problems with K % 8 == 0, ldx % 8 == 0, ldw % 8 == 0 and
+ * 16-byte aligned X, W take the tensor-core kernel; everything else takes a scalar kernel. */
+kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
+                           const void* X, int64_t ldx, const void* W, int64_t ldw,
+                           const void* bias, kf_act act, float scale,
+                           const void* residual, int64_t ldr, void* Y, int64_t ldy,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* GEMM + row reduction over N (Appendix A, "Algorithmic Optimization": online softmax;
+ * Appendix C.1 prints the three-pass softmax definition; Table 2 "Mixed reduction" and
+ * "Reduction-dominated").  With A[m,n] = pre_act( sum_k X[m,k]*W[n,k] + bias[n] ):
+ *   KF_RED_SOFTMAX: out[m,n] = exp(A[m,n]-max_n A[m,:]) / sum_n exp(A[m,n]-max_n A[m,:]),
+ *                   out is [M,N] with leading dimension ldo, dtype out_dtype.
+ *   KF_RED_SUM:     out[m] = sum_n A[m,n], out is [M] fp32 (out_dtype must be KF_F32, ldo
+ *                   ignored).
+ * The reduction is deterministic (no floating-point atomics): repeated calls give identical
+ * bits.  The workspace holds per-tile partial statistics. */
+kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype,
+                            const void* X, int64_t ldx, const void* W, int64_t ldw,
+                            const void* bias, kf_act pre_act, kf_rowred red,
+                            void* out, int64_t ldo, kf_dtype out_dtype,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* 3x3 convolution (pad 1, stride 1, cross-correlation as in torch.nn.Conv2d) + activation +
+ * optional GroupNorm (Table 2 "Conv-centered" chains).
+ *   c[n,o,h,w] = bias[o] + sum_{c,r,s} x[n,c,h+r-1,w+s-1] * w[o,c,r,s]      (zero padding)
+ *   a = act(c)
+ *   groups > 0: per image n and group g (channels [g*Cout/groups,(g+1)*Cout/groups)):
+ *       mu = mean(a), var = mean((a-mu)^2) (biased), y = (a-mu)/sqrt(var+eps)*gamma[o]+beta[o]
+ *   groups == 0: y = a.
+ * x is NCHW [Nb,Cin,H,Wd], w is OIHW [Cout,Cin,3,3], y is NCHW [Nb,Cout,H,Wd], all dense, of
+ * io_dtype.  bias, gamma, beta may be NULL (0, 1, 0).  y must not alias x.
+ * bf16 problems with Cin % 64 == 0, Cout % 16 == 0, Cout <= 256, Wd in {8,16,32,64,128} and
+ * (H*Wd) % 128 == 0 take the implicit-GEMM tensor-core kernel; everything else takes a
+ * scalar kernel.  groups must divide Cout. */
+kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                              kf_dtype io_dtype, const void* x, const void* w, const void* bias,
+                              kf_act act, int groups, float eps, const void* gamma,
+                              const void* beta, void* y,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Workspace sizes in bytes for the calls above with the same arguments (0 = none needed).
+ * Pure host arithmetic; no CUDA call is made. */
+size_t kf_gemm_epilogue_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype);
+size_t kf_gemm_rowreduce_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype,
+                                         kf_rowred red);
+size_t kf_conv3x3_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                                  kf_dtype io_dtype, int groups);
+
+/* Every wait inside the kernels (on an mbarrier) is bounded; a wait that runs out sets a
+ * device-side status word and the kernel drains and returns.  This call synchronises the
+ * current device, reads that word, clears it, and returns KF_OK, KF_ERR_TIMEOUT or
+ * KF_ERR_CUDA.  It is not needed for correct runs; tests call it after each launch. */
+kf_status kf_device_status(void);
+
+/* Number of kernels the library has launched from this process since load (all streams). */
+int64_t kf_launch_count(void);
+
+const char* kf_status_string(kf_status s);
+int kf_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KF_H_ */

@@ -1,0 +1,240 @@
+"""Fused operator chains for NVIDIA B200 (sm_100a): Python binding of the C-ABI library.
+
+The binding only marshals arguments: every step of every chain runs in the library's own
+CUDA kernels.  PyTorch is used for device memory and streams.  There is no CPU fallback;
+importing works without a GPU, calling does not.
+
+Raw entry points (same names and argument order as include/kf.h, pointers as ints):
+    kf_gemm_epilogue, kf_gemm_rowreduce, kf_conv3x3_epilogue, kf_*_workspace_bytes,
+    kf_device_status, kf_launch_count, kf_status_string, kf_version
+Tensor-level helpers:
+    gemm_epilogue(X, W, bias, act, scale, residual) -> Y
+    gemm_rowreduce(X, W, bias, pre_act, red, out_dtype) -> out
+    conv3x3_epilogue(x, w, bias, act, groups, eps, gamma, beta) -> y
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libkf.so")
+
+KF_OK, KF_ERR_INVALID_ARG, KF_ERR_UNSUPPORTED, KF_ERR_WORKSPACE, KF_ERR_CUDA, KF_ERR_TIMEOUT = range(6)
+KF_F32, KF_BF16 = 0, 1
+ACT = {"none": 0, "relu": 1, "gelu_tanh": 2, "sigmoid": 3, "gelu_erf": 4, "swish": 5, "tanh": 6,
+       "hardtanh": 7, "chain95": 8}
+RED = {"softmax": 0, "sum": 1}
+
+EXPORTS = ["kf_gemm_epilogue", "kf_gemm_rowreduce", "kf_conv3x3_epilogue",
+           "kf_gemm_epilogue_workspace_bytes", "kf_gemm_rowreduce_workspace_bytes",
+           "kf_conv3x3_workspace_bytes", "kf_device_status", "kf_launch_count",
+           "kf_status_string", "kf_version"]
+
+
+class KfError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (kf_status %d)" % (where, status_string(status), status))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libkf.so; raises if it has not been built (python -m paper_2605_30359_b200.build)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError("%s is missing: build it with `python -m paper_2605_30359_b200.build` "
+                          "(there is no fallback path)" % LIB_PATH)
+    L = ctypes.CDLL(LIB_PATH)
+    i64, vp, ci, f32, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    L.kf_gemm_epilogue.restype = ci
+    L.kf_gemm_epilogue.argtypes = [i64, i64, i64, ci, vp, i64, vp, i64, vp, ci, f32, vp, i64, vp,
+                                   i64, vp, sz, vp]
+    L.kf_gemm_rowreduce.restype = ci
+    L.kf_gemm_rowreduce.argtypes = [i64, i64, i64, ci, vp, i64, vp, i64, vp, ci, ci, vp, i64, ci,
+                                    vp, sz, vp]
+    L.kf_conv3x3_epilogue.restype = ci
+    L.kf_conv3x3_epilogue.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, ci, f32, vp, vp,
+                                      vp, vp, sz, vp]
+    L.kf_gemm_epilogue_workspace_bytes.restype = sz
+    L.kf_gemm_epilogue_workspace_bytes.argtypes = [i64, i64, i64, ci]
+    L.kf_gemm_rowreduce_workspace_bytes.restype = sz
+    L.kf_gemm_rowreduce_workspace_bytes.argtypes = [i64, i64, i64, ci, ci]
+    L.kf_conv3x3_workspace_bytes.restype = sz
+    L.kf_conv3x3_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, ci, ci]
+    L.kf_device_status.restype = ci
+    L.kf_device_status.argtypes = []
+    L.kf_launch_count.restype = i64
+    L.kf_launch_count.argtypes = []
+    L.kf_status_string.restype = ctypes.c_char_p
+    L.kf_status_string.argtypes = [ci]
+    L.kf_version.restype = ci
+    L.kf_version.argtypes = []
+    _lib = L
+    return L
+
+
+# ------------------------------------------------------------------ raw entry points
+def kf_gemm_epilogue(M, N, K, io_dtype, X, ldx, W, ldw, bias, act, scale, residual, ldr, Y, ldy,
+                     workspace, workspace_bytes, stream) -> int:
+    return lib().kf_gemm_epilogue(M, N, K, io_dtype, X, ldx, W, ldw, bias, act, scale, residual,
+                                  ldr, Y, ldy, workspace, workspace_bytes, stream)
+
+
+def kf_gemm_rowreduce(M, N, K, in_dtype, X, ldx, W, ldw, bias, pre_act, red, out, ldo, out_dtype,
+                      workspace, workspace_bytes, stream) -> int:
+    return lib().kf_gemm_rowreduce(M, N, K, in_dtype, X, ldx, W, ldw, bias, pre_act, red, out, ldo,
+                                   out_dtype, workspace, workspace_bytes, stream)
+
+
+def kf_conv3x3_epilogue(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, groups, eps, gamma, beta,
+                        y, workspace, workspace_bytes, stream) -> int:
+    return lib().kf_conv3x3_epilogue(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, groups, eps,
+                                     gamma, beta, y, workspace, workspace_bytes, stream)
+
+
+def kf_gemm_epilogue_workspace_bytes(M, N, K, io_dtype) -> int:
+    return lib().kf_gemm_epilogue_workspace_bytes(M, N, K, io_dtype)
+
+
+def kf_gemm_rowreduce_workspace_bytes(M, N, K, in_dtype, red) -> int:
+    return lib().kf_gemm_rowreduce_workspace_bytes(M, N, K, in_dtype, red)
+
+
+def kf_conv3x3_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype, groups) -> int:
+    return lib().kf_conv3x3_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype, groups)
+
+
+def kf_device_status() -> int:
+    return lib().kf_device_status()
+
+
+def kf_launch_count() -> int:
+    return lib().kf_launch_count()
+
+
+def status_string(status: int) -> str:
+    return lib().kf_status_string(status).decode()
+
+
+def kf_version() -> int:
+    return lib().kf_version()
+
+
+# ------------------------------------------------------------------ tensor-level helpers
+def _torch():
+    import torch
+    return torch
+
+
+def _kf_dtype(t) -> int:
+    torch = _torch()
+    if t.dtype == torch.float32:
+        return KF_F32
+    if t.dtype == torch.bfloat16:
+        return KF_BF16
+    raise TypeError("kf chains take float32 or bfloat16 tensors, got %s" % t.dtype)
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _check_cuda(*ts):
+    for t in ts:
+        if t is not None and not t.is_cuda:
+            raise ValueError("kf chains run on CUDA tensors only (no CPU fallback)")
+
+
+_workspaces = {}
+
+
+def workspace(nbytes: int, device):
+    """A cached, 256-byte aligned device scratch buffer of at least nbytes (None for 0)."""
+    if nbytes == 0:
+        return None
+    torch = _torch()
+    key = (device.type, device.index)
+    buf = _workspaces.get(key)
+    if buf is None or buf.numel() < nbytes:
+        buf = torch.empty(max(nbytes, 1 << 20), dtype=torch.uint8, device=device)
+        _workspaces[key] = buf
+    return buf
+
+
+def _stream_ptr(stream):
+    torch = _torch()
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def gemm_epilogue(X, W, bias=None, act="none", scale=1.0, residual=None, out=None, stream=None):
+    """Y = scale*act(X @ W.T + bias) + residual in one kernel.  X [M,K], W [N,K], row-major."""
+    torch = _torch()
+    _check_cuda(X, W, bias, residual, out)
+    M, K = X.shape
+    N = W.shape[0]
+    dt = _kf_dtype(X)
+    if out is None:
+        out = torch.empty((M, N), dtype=X.dtype, device=X.device)
+    nb = kf_gemm_epilogue_workspace_bytes(M, N, K, dt)
+    ws = workspace(nb, X.device)
+    st = kf_gemm_epilogue(M, N, K, dt, _ptr(X), X.stride(0), _ptr(W), W.stride(0), _ptr(bias),
+                          ACT[act], float(scale), _ptr(residual),
+                          residual.stride(0) if residual is not None else 0, _ptr(out),
+                          out.stride(0), _ptr(ws), nb, _stream_ptr(stream))
+    if st != KF_OK:
+        raise KfError(st, "kf_gemm_epilogue")
+    return out
+
+
+def gemm_rowreduce(X, W, bias=None, pre_act="none", red="softmax", out_dtype=None, out=None,
+                   stream=None):
+    """softmax: out[M,N] = softmax_n(pre_act(X @ W.T + bias)); sum: out[M] fp32 = row sums."""
+    torch = _torch()
+    _check_cuda(X, W, bias, out)
+    M, K = X.shape
+    N = W.shape[0]
+    dt = _kf_dtype(X)
+    if red == "sum":
+        if out is None:
+            out = torch.empty((M,), dtype=torch.float32, device=X.device)
+        odt, ldo = KF_F32, 1
+    else:
+        if out is None:
+            out = torch.empty((M, N), dtype=out_dtype or X.dtype, device=X.device)
+        odt, ldo = _kf_dtype(out), out.stride(0)
+    nb = kf_gemm_rowreduce_workspace_bytes(M, N, K, dt, RED[red])
+    ws = workspace(nb, X.device)
+    st = kf_gemm_rowreduce(M, N, K, dt, _ptr(X), X.stride(0), _ptr(W), W.stride(0), _ptr(bias),
+                           ACT[pre_act], RED[red], _ptr(out), ldo, odt, _ptr(ws), nb,
+                           _stream_ptr(stream))
+    if st != KF_OK:
+        raise KfError(st, "kf_gemm_rowreduce")
+    return out
+
+
+def conv3x3_epilogue(x, w, bias=None, act="none", groups=0, eps=1e-5, gamma=None, beta=None,
+                     out=None, stream=None):
+    """y = GroupNorm(act(conv3x3_pad1(x, w) + bias)); x NCHW, w OIHW, contiguous."""
+    torch = _torch()
+    _check_cuda(x, w, bias, gamma, beta, out)
+    if not (x.is_contiguous() and w.is_contiguous()):
+        raise ValueError("conv3x3_epilogue takes contiguous NCHW / OIHW tensors")
+    Nb, Cin, H, Wd = x.shape
+    Cout = w.shape[0]
+    dt = _kf_dtype(x)
+    if out is None:
+        out = torch.empty((Nb, Cout, H, Wd), dtype=x.dtype, device=x.device)
+    nb = kf_conv3x3_workspace_bytes(Nb, Cin, H, Wd, Cout, dt, groups)
+    ws = workspace(nb, x.device)
+    st = kf_conv3x3_epilogue(Nb, Cin, H, Wd, Cout, dt, _ptr(x), _ptr(w), _ptr(bias), ACT[act],
+                             int(groups), float(eps), _ptr(gamma), _ptr(beta), _ptr(out), _ptr(ws),
+                             nb, _stream_ptr(stream))
+    if st != KF_OK:
+        raise KfError(st, "kf_conv3x3_epilogue")
+    return out

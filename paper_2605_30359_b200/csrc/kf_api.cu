@@ -1,0 +1,367 @@
+// kf_api.cu -- the C ABI: argument validation, kernel selection, tensor-map encoding and the
+// launches.  See include/kf.h for the contract of every entry point.
+#include <atomic>
+#include <cstring>
+#include <mutex>
+
+#include "../../include/kf.h"
+#include "kf_internal.h"
+
+namespace {
+
+using namespace kf;
+
+std::atomic<int64_t> g_launches{0};
+
+// One status word per device, in static device memory (no allocation on any call path).
+__device__ uint32_t g_dev_status_word;
+
+struct DeviceInfo {
+  bool ready = false;
+  int sm_count = 0;
+  uint32_t* status = nullptr;
+};
+std::mutex g_mu;
+DeviceInfo g_dev[64];
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+bool device_info(DeviceInfo** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+  std::lock_guard<std::mutex> lk(g_mu);
+  DeviceInfo& d = g_dev[dev];
+  if (!d.ready) {
+    if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return false;
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_dev_status_word) != cudaSuccess) return false;
+    d.status = static_cast<uint32_t*>(p);
+    if (g_encode == nullptr) {
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult q;
+      if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) !=
+              cudaSuccess || q != cudaDriverEntryPointSuccess || fn == nullptr)
+        return false;
+      g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    d.ready = true;
+  }
+  *out = &d;
+  return true;
+}
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline size_t esize(int dt) { return dt == DT_F32 ? 4 : 2; }
+inline size_t round256(size_t b) { return (b + 255) & ~static_cast<size_t>(255); }
+inline bool valid_dtype(int dt) { return dt == DT_F32 || dt == DT_BF16; }
+inline bool valid_act(int a) { return a >= 0 && a < ACT_COUNT; }
+constexpr int64_t kMaxDim = 2147483647ll;
+
+// bf16 row-major [rows, cols] with leading dimension ld -> tiles of box_rows x 64 columns,
+// 128-byte swizzle, zero fill outside the tensor.
+bool encode_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld,
+               int box_rows) {
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBK), static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1, 1};
+  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides,
+                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+         CUDA_SUCCESS;
+}
+
+// NHWC bf16 activations [Nb,H,W,C] -> boxes of 64 channels x W pixels x rows image rows.
+bool encode_nhwc(CUtensorMap* tm, const void* base, int64_t Nb, int64_t H, int64_t Wd, int64_t C,
+                 int rows) {
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(Wd),
+                              static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(Nb)};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(C) * 2,
+                                 static_cast<cuuint64_t>(Wd) * C * 2,
+                                 static_cast<cuuint64_t>(H) * Wd * C * 2};
+  const cuuint32_t box[4] = {static_cast<cuuint32_t>(kBK), static_cast<cuuint32_t>(Wd),
+                             static_cast<cuuint32_t>(rows), 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides,
+                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+         CUDA_SUCCESS;
+}
+
+// Can the tensor-core GEMM take these operands?  (TMA: 16-byte aligned base and row pitch.)
+bool umma_gemm_ok(int dt, int64_t K, const void* X, int64_t ldx, const void* W, int64_t ldw) {
+  return dt == DT_BF16 && K % 8 == 0 && ldx % 8 == 0 && ldw % 8 == 0 && aligned(X, 16) &&
+         aligned(W, 16);
+}
+
+bool conv_umma_shape_ok(int dt, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout) {
+  const bool w_ok = Wd == 8 || Wd == 16 || Wd == 32 || Wd == 64 || Wd == 128;
+  return dt == DT_BF16 && Cin % 64 == 0 && Cout % 16 == 0 && Cout <= 256 && w_ok &&
+         (H * Wd) % 128 == 0;
+}
+
+kf_status check_gemm_common(int64_t M, int64_t N, int64_t K, int dt, const void* X, int64_t ldx,
+                            const void* W, int64_t ldw, const void* bias) {
+  if (M < 1 || N < 1 || K < 1 || M > kMaxDim || N > kMaxDim || K > kMaxDim) return KF_ERR_INVALID_ARG;
+  if (!valid_dtype(dt)) return KF_ERR_INVALID_ARG;
+  if (X == nullptr || W == nullptr) return KF_ERR_INVALID_ARG;
+  if (ldx < K || ldw < K) return KF_ERR_INVALID_ARG;
+  const size_t es = esize(dt);
+  if (!aligned(X, es) || !aligned(W, es) || !aligned(bias, es)) return KF_ERR_INVALID_ARG;
+  return KF_OK;
+}
+
+kf_status check_workspace(const void* ws, size_t have, size_t need) {
+  if (need == 0) return KF_OK;
+  if (ws == nullptr || !aligned(ws, 256) || have < need) return KF_ERR_WORKSPACE;
+  return KF_OK;
+}
+
+size_t rowreduce_umma_ws(int64_t M, int64_t N, int red) {
+  const int64_t tiles_n = (N + kRowReduceBN - 1) / kRowReduceBN;
+  return round256(static_cast<size_t>(M) * tiles_n * (red == RED_SOFTMAX ? 8 : 4));
+}
+size_t rowreduce_simt_ws(int64_t M, int64_t N) { return round256(static_cast<size_t>(M) * N * 4); }
+
+}  // namespace
+
+extern "C" {
+
+const char* kf_status_string(kf_status s) {
+  switch (s) {
+    case KF_OK: return "ok";
+    case KF_ERR_INVALID_ARG: return "invalid argument";
+    case KF_ERR_UNSUPPORTED: return "unsupported";
+    case KF_ERR_WORKSPACE: return "workspace null, misaligned or too small";
+    case KF_ERR_CUDA: return "CUDA error";
+    case KF_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+int kf_version(void) { return 100; }
+
+int64_t kf_launch_count(void) { return g_launches.load(); }
+
+kf_status kf_device_status(void) {
+  DeviceInfo* d = nullptr;
+  if (!device_info(&d)) return KF_ERR_CUDA;
+  if (cudaDeviceSynchronize() != cudaSuccess) return KF_ERR_CUDA;
+  uint32_t w = 0;
+  if (cudaMemcpy(&w, d->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return KF_ERR_CUDA;
+  if (w != 0) {
+    if (cudaMemset(d->status, 0, 4) != cudaSuccess) return KF_ERR_CUDA;
+    return KF_ERR_TIMEOUT;
+  }
+  return KF_OK;
+}
+
+size_t kf_gemm_epilogue_workspace_bytes(int64_t, int64_t, int64_t, kf_dtype) { return 0; }
+
+size_t kf_gemm_rowreduce_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype,
+                                         kf_rowred red) {
+  if (M < 1 || N < 1 || K < 1) return 0;
+  if (in_dtype == KF_BF16 && K % 8 == 0) return rowreduce_umma_ws(M, N, red);
+  return rowreduce_simt_ws(M, N);
+}
+
+size_t kf_conv3x3_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                                  kf_dtype io_dtype, int groups) {
+  (void)groups;
+  if (Nb < 1 || Cin < 1 || H < 1 || Wd < 1 || Cout < 1) return 0;
+  if (!conv_umma_shape_ok(io_dtype, Cin, H, Wd, Cout)) return 0;
+  return round256(static_cast<size_t>(Nb) * H * Wd * Cin * 2) +
+         round256(static_cast<size_t>(9) * Cout * Cin * 2);
+}
+
+kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, const void* X,
+                           int64_t ldx, const void* W, int64_t ldw, const void* bias, kf_act act,
+                           float scale, const void* residual, int64_t ldr, void* Y, int64_t ldy,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  (void)workspace; (void)workspace_bytes;
+  kf_status vs = check_gemm_common(M, N, K, io_dtype, X, ldx, W, ldw, bias);
+  if (vs != KF_OK) return vs;
+  if (!valid_act(act) || Y == nullptr || ldy < N) return KF_ERR_INVALID_ARG;
+  if (residual != nullptr && ldr < N) return KF_ERR_INVALID_ARG;
+  const size_t es = esize(io_dtype);
+  if (!aligned(Y, es) || !aligned(residual, es)) return KF_ERR_INVALID_ARG;
+  if (Y == X || Y == W) return KF_ERR_INVALID_ARG;
+  if (residual == Y && ldr != ldy) return KF_ERR_INVALID_ARG;
+  DeviceInfo* d = nullptr;
+  if (!device_info(&d)) return KF_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+  if (umma_gemm_ok(io_dtype, K, X, ldx, W, ldw)) {
+    const int bn = N <= 128 ? 128 : 256;
+    CUtensorMap ta, tb;
+    if (!encode_2d(&ta, X, M, K, ldx, kBM) || !encode_2d(&tb, W, N, K, ldw, bn)) return KF_ERR_CUDA;
+    UmmaParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+    p.tiles_m = static_cast<int>((M + kBM - 1) / kBM);
+    p.tiles_n = static_cast<int>((N + bn - 1) / bn);
+    if (static_cast<int64_t>(p.tiles_m) * p.tiles_n > kMaxDim) return KF_ERR_UNSUPPORTED;
+    p.num_tiles = p.tiles_m * p.tiles_n;
+    p.k_blocks = static_cast<int>((K + kBK - 1) / kBK);
+    p.bias = static_cast<const __nv_bfloat16*>(bias);
+    p.R = static_cast<const __nv_bfloat16*>(residual);
+    p.ldr = ldr; p.out = Y; p.ldo = ldy; p.scale = scale;
+    p.vec_ok = (ldy % 8 == 0 && aligned(Y, 16) &&
+                (residual == nullptr || (ldr % 8 == 0 && aligned(residual, 16)))) ? 1 : 0;
+    p.status = d->status;
+    const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
+    if (launch_umma_elementwise(bn, act, ta, tb, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
+    g_launches += 1;
+    return KF_OK;
+  }
+  if (launch_simt_gemm(io_dtype, 0, act, static_cast<int>(M), static_cast<int>(N),
+                       static_cast<int>(K), X, ldx, W, ldw, bias, scale, residual, ldr, Y, ldy,
+                       st) != cudaSuccess)
+    return KF_ERR_CUDA;
+  g_launches += 1;
+  return KF_OK;
+}
+
+kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, const void* X,
+                            int64_t ldx, const void* W, int64_t ldw, const void* bias,
+                            kf_act pre_act, kf_rowred red, void* out, int64_t ldo,
+                            kf_dtype out_dtype, void* workspace, size_t workspace_bytes,
+                            void* cuda_stream) {
+  kf_status vs = check_gemm_common(M, N, K, in_dtype, X, ldx, W, ldw, bias);
+  if (vs != KF_OK) return vs;
+  if (!valid_act(pre_act) || out == nullptr || !valid_dtype(out_dtype)) return KF_ERR_INVALID_ARG;
+  if (red != KF_RED_SOFTMAX && red != KF_RED_SUM) return KF_ERR_INVALID_ARG;
+  if (red == KF_RED_SUM && out_dtype != KF_F32) return KF_ERR_INVALID_ARG;
+  if (red == KF_RED_SOFTMAX && ldo < N) return KF_ERR_INVALID_ARG;
+  if (!aligned(out, esize(out_dtype))) return KF_ERR_INVALID_ARG;
+  if (out == X || out == W) return KF_ERR_INVALID_ARG;
+  DeviceInfo* d = nullptr;
+  if (!device_info(&d)) return KF_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int Mi = static_cast<int>(M), Ni = static_cast<int>(N), Ki = static_cast<int>(K);
+
+  const int64_t tiles_n64 = (N + kRowReduceBN - 1) / kRowReduceBN;
+  if (umma_gemm_ok(in_dtype, K, X, ldx, W, ldw) && tiles_n64 <= 8192) {
+    vs = check_workspace(workspace, workspace_bytes, rowreduce_umma_ws(M, N, red));
+    if (vs != KF_OK) return vs;
+    CUtensorMap ta, tb;
+    if (!encode_2d(&ta, X, M, K, ldx, kBM) || !encode_2d(&tb, W, N, K, ldw, kRowReduceBN))
+      return KF_ERR_CUDA;
+    UmmaParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.M = Mi; p.N = Ni; p.K = Ki;
+    p.tiles_m = static_cast<int>((M + kBM - 1) / kBM);
+    p.tiles_n = static_cast<int>(tiles_n64);
+    if (static_cast<int64_t>(p.tiles_m) * p.tiles_n > kMaxDim) return KF_ERR_UNSUPPORTED;
+    p.num_tiles = p.tiles_m * p.tiles_n;
+    p.k_blocks = static_cast<int>((K + kBK - 1) / kBK);
+    p.bias = static_cast<const __nv_bfloat16*>(bias);
+    p.out = out; p.ldo = ldo; p.scale = 1.0f;
+    p.partial = static_cast<float*>(workspace);
+    p.vec_ok = (red == KF_RED_SOFTMAX && (ldo * esize(out_dtype)) % 16 == 0 && aligned(out, 16)) ? 1 : 0;
+    p.status = d->status;
+    const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
+    if (red == KF_RED_SOFTMAX) {
+      if (launch_umma_softmax(pre_act, out_dtype, ta, tb, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
+      if (launch_softmax_finalize(out_dtype, Mi, Ni, p.tiles_n, p.partial, out, ldo, p.vec_ok, st) !=
+          cudaSuccess)
+        return KF_ERR_CUDA;
+    } else {
+      if (launch_umma_rowsum(pre_act, ta, tb, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
+      if (launch_rowsum_finalize(Mi, p.tiles_n, p.partial, static_cast<float*>(out), st) != cudaSuccess)
+        return KF_ERR_CUDA;
+    }
+    g_launches += 2;
+    return KF_OK;
+  }
+  // scalar path: pre-reduction values in fp32, then one CTA per row
+  vs = check_workspace(workspace, workspace_bytes, rowreduce_simt_ws(M, N));
+  if (vs != KF_OK) return vs;
+  float* A = static_cast<float*>(workspace);
+  if (launch_simt_gemm(in_dtype, 1, pre_act, Mi, Ni, Ki, X, ldx, W, ldw, bias, 1.0f, nullptr, 0, A,
+                       N, st) != cudaSuccess)
+    return KF_ERR_CUDA;
+  cudaError_t e = red == KF_RED_SOFTMAX ? launch_row_softmax(out_dtype, Mi, Ni, A, N, out, ldo, st)
+                                        : launch_row_sum(Mi, Ni, A, N, static_cast<float*>(out), st);
+  if (e != cudaSuccess) return KF_ERR_CUDA;
+  g_launches += 2;
+  return KF_OK;
+}
+
+kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                              kf_dtype io_dtype, const void* x, const void* w, const void* bias,
+                              kf_act act, int groups, float eps, const void* gamma,
+                              const void* beta, void* y, void* workspace, size_t workspace_bytes,
+                              void* cuda_stream) {
+  if (Nb < 1 || Cin < 1 || H < 1 || Wd < 1 || Cout < 1) return KF_ERR_INVALID_ARG;
+  if (Nb > kMaxDim || Cin > kMaxDim || H > kMaxDim || Wd > kMaxDim || Cout > kMaxDim) return KF_ERR_INVALID_ARG;
+  if (!valid_dtype(io_dtype) || !valid_act(act)) return KF_ERR_INVALID_ARG;
+  if (x == nullptr || w == nullptr || y == nullptr || y == x) return KF_ERR_INVALID_ARG;
+  if (groups < 0 || (groups > 0 && Cout % groups != 0)) return KF_ERR_INVALID_ARG;
+  if (groups > 0 && !(eps >= 0.0f)) return KF_ERR_INVALID_ARG;
+  const size_t es = esize(io_dtype);
+  if (!aligned(x, es) || !aligned(w, es) || !aligned(bias, es) || !aligned(y, es) ||
+      !aligned(gamma, es) || !aligned(beta, es))
+    return KF_ERR_INVALID_ARG;
+  const int64_t hw = H * Wd;
+  if (hw > kMaxDim || Nb * hw > kMaxDim) return KF_ERR_UNSUPPORTED;
+  DeviceInfo* d = nullptr;
+  if (!device_info(&d)) return KF_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int launches = 0;
+
+  if (conv_umma_shape_ok(io_dtype, Cin, H, Wd, Cout) && aligned(x, 16)) {
+    const size_t xt_bytes = round256(static_cast<size_t>(Nb) * hw * Cin * 2);
+    const size_t wr_bytes = round256(static_cast<size_t>(9) * Cout * Cin * 2);
+    kf_status vs = check_workspace(workspace, workspace_bytes, xt_bytes + wr_bytes);
+    if (vs != KF_OK) return vs;
+    void* xt = workspace;
+    void* wr = static_cast<uint8_t*>(workspace) + xt_bytes;
+    if (launch_conv_prep(static_cast<int>(Nb), static_cast<int>(Cin), static_cast<int>(H),
+                         static_cast<int>(Wd), static_cast<int>(Cout), x, w, xt, wr, st) != cudaSuccess)
+      return KF_ERR_CUDA;
+    ++launches;
+    const int bn = Cout <= 64 ? 64 : (Cout <= 128 ? 128 : 256);
+    const int rows = static_cast<int>(kBM / Wd);
+    CUtensorMap ta, tb;
+    if (!encode_nhwc(&ta, xt, Nb, H, Wd, Cin, rows) || !encode_2d(&tb, wr, 9 * Cout, Cin, Cin, bn))
+      return KF_ERR_CUDA;
+    UmmaParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.M = static_cast<int>(Nb * hw); p.N = static_cast<int>(Cout); p.K = static_cast<int>(9 * Cin);
+    p.tiles_per_image = static_cast<int>(hw / kBM);
+    p.tiles_m = static_cast<int>(Nb) * p.tiles_per_image; p.tiles_n = 1;
+    p.num_tiles = p.tiles_m;
+    p.kb_per_tap = static_cast<int>(Cin / kBK);
+    p.k_blocks = 9 * p.kb_per_tap;
+    p.bias = static_cast<const __nv_bfloat16*>(bias);
+    p.out = y; p.scale = 1.0f;
+    p.status = d->status;
+    p.H = static_cast<int>(H); p.Wd = static_cast<int>(Wd); p.Cin = static_cast<int>(Cin);
+    p.rows_per_tile = rows;
+    const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
+    if (launch_umma_conv(bn, act, ta, tb, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
+    ++launches;
+  } else {
+    if (launch_conv_direct(io_dtype, act, static_cast<int>(Nb), static_cast<int>(Cin),
+                           static_cast<int>(H), static_cast<int>(Wd), static_cast<int>(Cout), x, w,
+                           bias, y, st) != cudaSuccess)
+      return KF_ERR_CUDA;
+    ++launches;
+  }
+  if (groups > 0) {
+    if (launch_groupnorm(io_dtype, static_cast<int>(Nb), static_cast<int>(Cout), groups, hw, eps,
+                         gamma, beta, y, st) != cudaSuccess)
+      return KF_ERR_CUDA;
+    ++launches;
+  }
+  g_launches += launches;
+  return KF_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,61 @@
+// kf_internal.h -- host-side launcher interface between the C ABI (kf_api.cu) and the files
+// that instantiate the kernels.  Every launcher enqueues on `st` and returns the launch's
+// cudaError_t; none synchronises.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "kf_umma.cuh"
+
+namespace kf {
+
+// tensor-core chains (bf16)
+cudaError_t launch_umma_elementwise(int bn, int act, const CUtensorMap& a, const CUtensorMap& b,
+                                    const UmmaParams& p, int grid, cudaStream_t st);
+cudaError_t launch_umma_softmax(int act, int out_dt, const CUtensorMap& a, const CUtensorMap& b,
+                                const UmmaParams& p, int grid, cudaStream_t st);
+cudaError_t launch_umma_rowsum(int act, const CUtensorMap& a, const CUtensorMap& b,
+                               const UmmaParams& p, int grid, cudaStream_t st);
+cudaError_t launch_umma_conv(int bn, int act, const CUtensorMap& a, const CUtensorMap& b,
+                             const UmmaParams& p, int grid, cudaStream_t st);
+constexpr int kRowReduceBN = 256;   // tile width of the row-reduce first pass
+
+// second passes of the tensor-core row reductions
+cudaError_t launch_softmax_finalize(int out_dt, int M, int N, int tiles_n, const float* partial,
+                                    void* out, long long ldo, int vec_ok, cudaStream_t st);
+cudaError_t launch_rowsum_finalize(int M, int tiles_n, const float* partial, float* out,
+                                   cudaStream_t st);
+
+// scalar chains (fp32, and bf16 shapes the tensor-core kernels do not take)
+cudaError_t launch_simt_gemm(int dt, int mode, int act, int M, int N, int K, const void* X,
+                             long long ldx, const void* W, long long ldw, const void* bias,
+                             float scale, const void* R, long long ldr, void* out, long long ldo,
+                             cudaStream_t st);
+cudaError_t launch_row_softmax(int out_dt, int M, int N, const float* A, long long lda, void* out,
+                               long long ldo, cudaStream_t st);
+cudaError_t launch_row_sum(int M, int N, const float* A, long long lda, float* out,
+                           cudaStream_t st);
+
+// convolution helpers
+cudaError_t launch_conv_prep(int Nb, int Cin, int H, int Wd, int Cout, const void* x,
+                             const void* w, void* xt, void* wr, cudaStream_t st);
+cudaError_t launch_conv_direct(int dt, int act, int Nb, int Cin, int H, int Wd, int Cout,
+                               const void* x, const void* w, const void* bias, void* y,
+                               cudaStream_t st);
+cudaError_t launch_groupnorm(int dt, int Nb, int Cout, int groups, long long hw, float eps,
+                             const void* gamma, const void* beta, void* y, cudaStream_t st);
+
+// Generic launcher for one instantiation of the tensor-core kernel.
+template <int BN, int EPI, int ACT, typename OutT>
+inline cudaError_t launch_umma_instance(const CUtensorMap& a, const CUtensorMap& b,
+                                        const UmmaParams& p, int grid, cudaStream_t st) {
+  auto kern = umma_chain_kernel<BN, EPI, ACT, OutT>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       UmmaSmem<BN>::kTotal);
+  if (e != cudaSuccess) return e;
+  kern<<<grid, kNumThreads, UmmaSmem<BN>::kTotal, st>>>(a, b, p);
+  return cudaGetLastError();
+}
+
+}  // namespace kf

@@ -1,0 +1,119 @@
+// Launchers for the CUDA-core kernels.
+#include "kf_internal.h"
+#include "kf_simt.cuh"
+
+namespace kf {
+
+template <typename T>
+static cudaError_t simt_gemm_t(int mode, int act, int M, int N, int K, const void* X,
+                               long long ldx, const void* W, long long ldw, const void* bias,
+                               float scale, const void* R, long long ldr, void* out, long long ldo,
+                               cudaStream_t st) {
+  const dim3 grid((N + 31) / 32, (M + 31) / 32), block(256);
+  bool ok = dispatch_act(act, [&](auto A) {
+    constexpr int ACT = decltype(A)::value;
+    if (mode == 0)
+      simt_gemm_kernel<T, 0, ACT><<<grid, block, 0, st>>>(
+          M, N, K, static_cast<const T*>(X), ldx, static_cast<const T*>(W), ldw,
+          static_cast<const T*>(bias), scale, static_cast<const T*>(R), ldr, out, ldo);
+    else
+      simt_gemm_kernel<T, 1, ACT><<<grid, block, 0, st>>>(
+          M, N, K, static_cast<const T*>(X), ldx, static_cast<const T*>(W), ldw,
+          static_cast<const T*>(bias), scale, static_cast<const T*>(R), ldr, out, ldo);
+  });
+  return ok ? cudaGetLastError() : cudaErrorInvalidValue;
+}
+
+cudaError_t launch_simt_gemm(int dt, int mode, int act, int M, int N, int K, const void* X,
+                             long long ldx, const void* W, long long ldw, const void* bias,
+                             float scale, const void* R, long long ldr, void* out, long long ldo,
+                             cudaStream_t st) {
+  if (dt == DT_F32)
+    return simt_gemm_t<float>(mode, act, M, N, K, X, ldx, W, ldw, bias, scale, R, ldr, out, ldo, st);
+  return simt_gemm_t<__nv_bfloat16>(mode, act, M, N, K, X, ldx, W, ldw, bias, scale, R, ldr, out, ldo, st);
+}
+
+cudaError_t launch_row_softmax(int out_dt, int M, int N, const float* A, long long lda, void* out,
+                               long long ldo, cudaStream_t st) {
+  if (out_dt == DT_F32)
+    row_softmax_kernel<float><<<M, 256, 0, st>>>(N, A, lda, static_cast<float*>(out), ldo);
+  else
+    row_softmax_kernel<__nv_bfloat16><<<M, 256, 0, st>>>(N, A, lda, static_cast<__nv_bfloat16*>(out), ldo);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_row_sum(int M, int N, const float* A, long long lda, float* out,
+                           cudaStream_t st) {
+  row_sum_kernel<<<M, 256, 0, st>>>(N, A, lda, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_softmax_finalize(int out_dt, int M, int N, int tiles_n, const float* partial,
+                                    void* out, long long ldo, int vec_ok, cudaStream_t st) {
+  const size_t smem = static_cast<size_t>(tiles_n) * sizeof(float);
+  const float2* part = reinterpret_cast<const float2*>(partial);
+  if (out_dt == DT_F32)
+    softmax_finalize_kernel<float, kRowReduceBN><<<M, 256, smem, st>>>(
+        N, tiles_n, part, static_cast<float*>(out), ldo, vec_ok);
+  else
+    softmax_finalize_kernel<__nv_bfloat16, kRowReduceBN><<<M, 256, smem, st>>>(
+        N, tiles_n, part, static_cast<__nv_bfloat16*>(out), ldo, vec_ok);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rowsum_finalize(int M, int tiles_n, const float* partial, float* out,
+                                   cudaStream_t st) {
+  rowsum_finalize_kernel<<<(M + 255) / 256, 256, 0, st>>>(M, tiles_n, partial, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_conv_prep(int Nb, int Cin, int H, int Wd, int Cout, const void* x,
+                             const void* w, void* xt, void* wr, cudaStream_t st) {
+  const long long x_blocks = static_cast<long long>(Nb) * H * (Cin / 8) * (Wd / 8);
+  const long long total = x_blocks + 9ll * Cout * Cin;
+  const long long grid = (total + 255) / 256;
+  conv_prep_kernel<<<static_cast<unsigned>(grid), 256, 0, st>>>(
+      Nb, Cin, H, Wd, Cout, static_cast<const __nv_bfloat16*>(x),
+      static_cast<const __nv_bfloat16*>(w), static_cast<__nv_bfloat16*>(xt),
+      static_cast<__nv_bfloat16*>(wr), x_blocks);
+  return cudaGetLastError();
+}
+
+template <typename T>
+static cudaError_t conv_direct_t(int act, int Nb, int Cin, int H, int Wd, int Cout, const void* x,
+                                 const void* w, const void* bias, void* y, cudaStream_t st) {
+  const long long total = static_cast<long long>(Nb) * Cout * H * Wd;
+  const unsigned grid = static_cast<unsigned>((total + 255) / 256);
+  bool ok = dispatch_act(act, [&](auto A) {
+    constexpr int ACT = decltype(A)::value;
+    conv_direct_kernel<T, ACT><<<grid, 256, 0, st>>>(Nb, Cin, H, Wd, Cout, static_cast<const T*>(x),
+                                                     static_cast<const T*>(w),
+                                                     static_cast<const T*>(bias),
+                                                     static_cast<T*>(y));
+  });
+  return ok ? cudaGetLastError() : cudaErrorInvalidValue;
+}
+
+cudaError_t launch_conv_direct(int dt, int act, int Nb, int Cin, int H, int Wd, int Cout,
+                               const void* x, const void* w, const void* bias, void* y,
+                               cudaStream_t st) {
+  if (dt == DT_F32) return conv_direct_t<float>(act, Nb, Cin, H, Wd, Cout, x, w, bias, y, st);
+  return conv_direct_t<__nv_bfloat16>(act, Nb, Cin, H, Wd, Cout, x, w, bias, y, st);
+}
+
+cudaError_t launch_groupnorm(int dt, int Nb, int Cout, int groups, long long hw, float eps,
+                             const void* gamma, const void* beta, void* y, cudaStream_t st) {
+  const unsigned grid = static_cast<unsigned>(Nb) * static_cast<unsigned>(groups);
+  if (dt == DT_F32)
+    groupnorm_kernel<float><<<grid, 512, 0, st>>>(Cout, groups, hw, eps,
+                                                  static_cast<const float*>(gamma),
+                                                  static_cast<const float*>(beta),
+                                                  static_cast<float*>(y));
+  else
+    groupnorm_kernel<__nv_bfloat16><<<grid, 512, 0, st>>>(
+        Cout, groups, hw, eps, static_cast<const __nv_bfloat16*>(gamma),
+        static_cast<const __nv_bfloat16*>(beta), static_cast<__nv_bfloat16*>(y));
+  return cudaGetLastError();
+}
+
+}  // namespace kf

@@ -1,0 +1,353 @@
+// kf_simt.cuh -- CUDA-core kernels: the fp32 chains (plain FMA, no TF32), the bf16 chains on
+// shapes the tensor-core kernel does not take, the streaming second passes of the row
+// reductions, the convolution's layout prepass and GroupNorm.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include "kf_act.cuh"
+
+namespace kf {
+
+// ---------------------------------------------------------------- block reductions
+// Fixed tree order: results are bit-identical from run to run.
+template <bool IS_MAX>
+__device__ __forceinline__ float block_reduce(float v, float* scratch /*[32]*/) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (blockDim.x + 31) >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float u = __shfl_xor_sync(0xffffffffu, v, o);
+    v = IS_MAX ? fmaxf(v, u) : v + u;
+  }
+  __syncthreads();                 // scratch may still be read from a previous reduction
+  if (lane == 0) scratch[warp] = v;
+  __syncthreads();
+  float r = IS_MAX ? -INFINITY : 0.0f;
+  if (lane < nwarps) r = scratch[lane];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float u = __shfl_xor_sync(0xffffffffu, r, o);
+    r = IS_MAX ? fmaxf(r, u) : r + u;
+  }
+  return r;                        // every thread holds the result
+}
+
+// ---------------------------------------------------------------- scalar GEMM + epilogue
+// 32x32 output tile per CTA of 16x16 threads, 2x2 outputs per thread, K in slabs of 32 through
+// shared memory.  fp32 FMA accumulation in increasing k.
+//   MODE 0: out = T,     Y[m,n] = scale*act(z+b) + R[m,n]
+//   MODE 1: out = float, A[m,n] = act(z+b) (pre-reduction values for the row kernels)
+template <typename T, int MODE, int ACT>
+__global__ void __launch_bounds__(256)
+simt_gemm_kernel(int M, int N, int K, const T* __restrict__ X, long long ldx,
+                 const T* __restrict__ W, long long ldw, const T* __restrict__ bias, float scale,
+                 const T* R, long long ldr, void* out, long long ldo) {
+  __shared__ float As[32][33];
+  __shared__ float Bs[32][33];
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int m0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+  float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+  const int lr = threadIdx.x >> 5, lc = threadIdx.x & 31;
+  for (int k0 = 0; k0 < K; k0 += 32) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int r = lr + 8 * i;
+      const int k = k0 + lc;
+      const long long m = m0 + r, n = n0 + r;
+      As[r][lc] = (m < M && k < K) ? to_f32(X[m * ldx + k]) : 0.0f;
+      Bs[r][lc] = (n < N && k < K) ? to_f32(W[n * ldw + k]) : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 32; ++kk) {
+      const float a0 = As[ty][kk], a1 = As[ty + 16][kk];
+      const float b0 = Bs[tx][kk], b1 = Bs[tx + 16][kk];
+      acc[0][0] = fmaf(a0, b0, acc[0][0]); acc[0][1] = fmaf(a0, b1, acc[0][1]);
+      acc[1][0] = fmaf(a1, b0, acc[1][0]); acc[1][1] = fmaf(a1, b1, acc[1][1]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const long long m = m0 + ty + 16 * i;
+      const int n = n0 + tx + 16 * j;
+      if (m < M && n < N) {
+        float z = acc[i][j];
+        if (bias != nullptr) z += to_f32(bias[n]);
+        if constexpr (MODE == 0) {
+          float y = scale * act_f<ACT, false>(z);
+          if (R != nullptr) y += to_f32(R[m * ldr + n]);
+          reinterpret_cast<T*>(out)[m * ldo + n] = from_f32<T>(y);
+        } else {
+          reinterpret_cast<float*>(out)[m * ldo + n] = act_f<ACT, false>(z);
+        }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------- row kernels, scalar path
+// One CTA per row over fp32 pre-reduction values A[M,N]: the three-pass softmax (max, sum of
+// exp(a-max), quotient) or the plain sum.
+template <typename OutT>
+__global__ void __launch_bounds__(256)
+row_softmax_kernel(int N, const float* __restrict__ A, long long lda, OutT* out, long long ldo) {
+  __shared__ float scratch[32];
+  const float* a = A + static_cast<long long>(blockIdx.x) * lda;
+  OutT* o = out + static_cast<long long>(blockIdx.x) * ldo;
+  float mx = -INFINITY;
+  for (int n = threadIdx.x; n < N; n += blockDim.x) mx = fmaxf(mx, a[n]);
+  mx = block_reduce<true>(mx, scratch);
+  float s = 0.0f;
+  for (int n = threadIdx.x; n < N; n += blockDim.x) s += expf(a[n] - mx);
+  s = block_reduce<false>(s, scratch);
+  for (int n = threadIdx.x; n < N; n += blockDim.x) o[n] = from_f32<OutT>(expf(a[n] - mx) / s);
+}
+
+__global__ void __launch_bounds__(256)
+row_sum_kernel(int N, const float* __restrict__ A, long long lda, float* out) {
+  __shared__ float scratch[32];
+  const float* a = A + static_cast<long long>(blockIdx.x) * lda;
+  float s = 0.0f;
+  for (int n = threadIdx.x; n < N; n += blockDim.x) s += a[n];
+  s = block_reduce<false>(s, scratch);
+  if (threadIdx.x == 0) out[blockIdx.x] = s;
+}
+
+// ---------------------------------------------------------------- second passes, tensor path
+// Softmax: the first pass left e[m,n] = exp(a[m,n] - mx_t) in `out` and (mx_t, sum_t) per
+// 256-column tile t in `partial`.  Row maximum mx = max_t mx_t, denominator
+// S = sum_t sum_t*exp(mx_t - mx); the output is e * exp(mx_t - mx) / S, in place.
+template <typename OutT, int BN>
+__global__ void __launch_bounds__(256)
+softmax_finalize_kernel(int N, int tiles_n, const float2* __restrict__ partial, OutT* out,
+                        long long ldo, int vec_ok) {
+  extern __shared__ float fac[];   // [tiles_n]
+  __shared__ float scratch[32];
+  const long long m = blockIdx.x;
+  const float2* part = partial + m * tiles_n;
+  float mx = -INFINITY;
+  for (int t = threadIdx.x; t < tiles_n; t += blockDim.x) mx = fmaxf(mx, part[t].x);
+  mx = block_reduce<true>(mx, scratch);
+  float s = 0.0f;
+  for (int t = threadIdx.x; t < tiles_n; t += blockDim.x) {
+    const float2 pt = part[t];
+    const float f = __expf(pt.x - mx);
+    fac[t] = f;
+    s += pt.y * f;
+  }
+  s = block_reduce<false>(s, scratch);   // contains the __syncthreads that publishes fac[]
+  const float inv = 1.0f / s;
+  OutT* o = out + m * ldo;
+  if (vec_ok && (N % 8) == 0) {
+    constexpr int V = 16 / sizeof(OutT);               // elements per 16-byte vector
+    const int nvec = N / V;
+    uint4* ov = reinterpret_cast<uint4*>(o);
+    for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
+      const float f = fac[(i * V) / BN] * inv;
+      uint4 w = ov[i];
+      if constexpr (sizeof(OutT) == 2) {
+        w.x = pack_bf16x2(bf16_lo(w.x) * f, bf16_hi(w.x) * f);
+        w.y = pack_bf16x2(bf16_lo(w.y) * f, bf16_hi(w.y) * f);
+        w.z = pack_bf16x2(bf16_lo(w.z) * f, bf16_hi(w.z) * f);
+        w.w = pack_bf16x2(bf16_lo(w.w) * f, bf16_hi(w.w) * f);
+      } else {
+        w.x = __float_as_uint(__uint_as_float(w.x) * f);
+        w.y = __float_as_uint(__uint_as_float(w.y) * f);
+        w.z = __float_as_uint(__uint_as_float(w.z) * f);
+        w.w = __float_as_uint(__uint_as_float(w.w) * f);
+      }
+      ov[i] = w;
+    }
+  } else {
+    for (int n = threadIdx.x; n < N; n += blockDim.x)
+      o[n] = from_f32<OutT>(to_f32(o[n]) * fac[n / BN] * inv);
+  }
+}
+
+// Row sum: out[m] = sum_t partial[m,t] in increasing t.
+__global__ void __launch_bounds__(256)
+rowsum_finalize_kernel(int M, int tiles_n, const float* __restrict__ partial, float* out) {
+  const long long m = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (m >= M) return;
+  float s = 0.0f;
+  for (int t = 0; t < tiles_n; ++t) s += partial[m * tiles_n + t];
+  out[m] = s;
+}
+
+// ---------------------------------------------------------------- conv: layout prepass
+// x NCHW bf16 -> xt NHWC bf16 (so a pixel's channels are one contiguous, K-major row for the
+// implicit GEMM), and w OIHW -> wr[tap][o][c].  Each thread moves an 8-channel x 8-pixel block:
+// eight 16-byte reads along w, an in-register transpose, eight 16-byte writes along c.
+// Requires Cin % 8 == 0 and Wd % 8 == 0.
+__global__ void __launch_bounds__(256)
+conv_prep_kernel(int Nb, int Cin, int H, int Wd, int Cout, const __nv_bfloat16* __restrict__ x,
+                 const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ xt,
+                 __nv_bfloat16* __restrict__ wr, long long x_blocks) {
+  const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int wb = Wd / 8, cbk = Cin / 8;
+  if (gid < x_blocks) {
+    // gid -> (n, h, cblk, wblk) with wblk fastest: neighbouring lanes read one row of x
+    const int wblk = static_cast<int>(gid % wb);
+    long long t = gid / wb;
+    const int cblk = static_cast<int>(t % cbk); t /= cbk;
+    const int h = static_cast<int>(t % H);
+    const long long n = t / H;
+    const long long hw = static_cast<long long>(H) * Wd;
+    const __nv_bfloat16* src = x + ((n * Cin + cblk * 8) * H + h) * Wd + wblk * 8;
+    uint4 rows[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) rows[i] = __ldg(reinterpret_cast<const uint4*>(src + i * hw));
+    const unsigned short* e = reinterpret_cast<const unsigned short*>(rows);   // e[c*8 + p]
+    __nv_bfloat16* dst = xt + ((n * H + h) * Wd + wblk * 8) * Cin + cblk * 8;
+#pragma unroll
+    for (int p = 0; p < 8; ++p) {
+      uint4 o;
+      o.x = static_cast<uint32_t>(e[0 * 8 + p]) | (static_cast<uint32_t>(e[1 * 8 + p]) << 16);
+      o.y = static_cast<uint32_t>(e[2 * 8 + p]) | (static_cast<uint32_t>(e[3 * 8 + p]) << 16);
+      o.z = static_cast<uint32_t>(e[4 * 8 + p]) | (static_cast<uint32_t>(e[5 * 8 + p]) << 16);
+      o.w = static_cast<uint32_t>(e[6 * 8 + p]) | (static_cast<uint32_t>(e[7 * 8 + p]) << 16);
+      *reinterpret_cast<uint4*>(dst + static_cast<long long>(p) * Cin) = o;
+    }
+  } else {
+    const long long i = gid - x_blocks;                 // index into wr[tap][o][c]
+    const long long total = 9ll * Cout * Cin;
+    if (i < total) {
+      const int c = static_cast<int>(i % Cin);
+      const int o = static_cast<int>((i / Cin) % Cout);
+      const int tap = static_cast<int>(i / (static_cast<long long>(Cin) * Cout));
+      wr[i] = w[(static_cast<long long>(o) * Cin + c) * 9 + tap];
+    }
+  }
+}
+
+// ---------------------------------------------------------------- conv: scalar path
+// One thread per output element, taps with an explicit bounds test; stores act(c) in T.
+template <typename T, int ACT>
+__global__ void __launch_bounds__(256)
+conv_direct_kernel(int Nb, int Cin, int H, int Wd, int Cout, const T* __restrict__ x,
+                   const T* __restrict__ w, const T* __restrict__ bias, T* __restrict__ y) {
+  const long long total = static_cast<long long>(Nb) * Cout * H * Wd;
+  const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (gid >= total) return;
+  const int wq = static_cast<int>(gid % Wd);
+  const int h = static_cast<int>((gid / Wd) % H);
+  const int o = static_cast<int>((gid / (static_cast<long long>(Wd) * H)) % Cout);
+  const long long n = gid / (static_cast<long long>(Wd) * H * Cout);
+  float acc = bias != nullptr ? to_f32(bias[o]) : 0.0f;
+  for (int c = 0; c < Cin; ++c) {
+    const T* xp = x + (n * Cin + c) * H * Wd;
+    const T* wp = w + (static_cast<long long>(o) * Cin + c) * 9;
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+      const int hh = h + r - 1;
+      if (hh < 0 || hh >= H) continue;
+#pragma unroll
+      for (int s = 0; s < 3; ++s) {
+        const int ww = wq + s - 1;
+        if (ww < 0 || ww >= Wd) continue;
+        acc = fmaf(to_f32(xp[hh * Wd + ww]), to_f32(wp[r * 3 + s]), acc);
+      }
+    }
+  }
+  y[gid] = from_f32<T>(act_f<ACT, false>(acc));
+}
+
+// ---------------------------------------------------------------- GroupNorm, in place
+// One CTA per (image, group): the group's cpg*H*W activations are contiguous in NCHW.  Mean,
+// then the biased variance about that mean (two passes: no cancellation), then
+// y = (a-mu)*rstd*gamma[o]+beta[o].  The group is re-read from cache, not from HBM, when it
+// fits (32 KB for the benchmark's groups).
+template <typename T>
+__global__ void __launch_bounds__(512)
+groupnorm_kernel(int Cout, int groups, long long hw, float eps, const T* __restrict__ gamma,
+                 const T* __restrict__ beta, T* y) {
+  __shared__ float scratch[32];
+  const int cpg = Cout / groups;
+  const long long cnt = static_cast<long long>(cpg) * hw;
+  const int g = blockIdx.x % groups;
+  const long long n = blockIdx.x / groups;
+  T* blk = y + (n * Cout + static_cast<long long>(g) * cpg) * hw;
+  constexpr int V = 16 / sizeof(T);
+  const bool vec = (cnt % V) == 0 && (hw % V) == 0 &&
+                   (reinterpret_cast<uintptr_t>(blk) & 15u) == 0;
+  float s = 0.0f;
+  if (vec) {
+    const uint4* bv = reinterpret_cast<const uint4*>(blk);
+    for (long long i = threadIdx.x; i < cnt / V; i += blockDim.x) {
+      const uint4 w = bv[i];
+      if constexpr (sizeof(T) == 2) {
+        s += (bf16_lo(w.x) + bf16_hi(w.x)) + (bf16_lo(w.y) + bf16_hi(w.y)) +
+             (bf16_lo(w.z) + bf16_hi(w.z)) + (bf16_lo(w.w) + bf16_hi(w.w));
+      } else {
+        s += (__uint_as_float(w.x) + __uint_as_float(w.y)) +
+             (__uint_as_float(w.z) + __uint_as_float(w.w));
+      }
+    }
+  } else {
+    for (long long i = threadIdx.x; i < cnt; i += blockDim.x) s += to_f32(blk[i]);
+  }
+  const float mu = block_reduce<false>(s, scratch) / static_cast<float>(cnt);
+  float q = 0.0f;
+  if (vec) {
+    const uint4* bv = reinterpret_cast<const uint4*>(blk);
+    for (long long i = threadIdx.x; i < cnt / V; i += blockDim.x) {
+      const uint4 w = bv[i];
+      float d[8];
+      int nv;
+      if constexpr (sizeof(T) == 2) {
+        d[0] = bf16_lo(w.x); d[1] = bf16_hi(w.x); d[2] = bf16_lo(w.y); d[3] = bf16_hi(w.y);
+        d[4] = bf16_lo(w.z); d[5] = bf16_hi(w.z); d[6] = bf16_lo(w.w); d[7] = bf16_hi(w.w);
+        nv = 8;
+      } else {
+        d[0] = __uint_as_float(w.x); d[1] = __uint_as_float(w.y);
+        d[2] = __uint_as_float(w.z); d[3] = __uint_as_float(w.w);
+        nv = 4;
+      }
+      float part = 0.0f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) if (j < nv) part = fmaf(d[j] - mu, d[j] - mu, part);
+      q += part;
+    }
+  } else {
+    for (long long i = threadIdx.x; i < cnt; i += blockDim.x) {
+      const float d = to_f32(blk[i]) - mu;
+      q = fmaf(d, d, q);
+    }
+  }
+  const float var = block_reduce<false>(q, scratch) / static_cast<float>(cnt);
+  const float rstd = rsqrtf(var + eps);
+  if (vec) {
+    uint4* bv = reinterpret_cast<uint4*>(blk);
+    for (long long i = threadIdx.x; i < cnt / V; i += blockDim.x) {
+      const int o = g * cpg + static_cast<int>((i * V) / hw);   // a vector never straddles channels
+      const float ga = gamma != nullptr ? to_f32(gamma[o]) : 1.0f;
+      const float be = beta != nullptr ? to_f32(beta[o]) : 0.0f;
+      const float a = rstd * ga, b = fmaf(-mu, rstd * ga, be);
+      uint4 w = bv[i];
+      if constexpr (sizeof(T) == 2) {
+        w.x = pack_bf16x2(fmaf(bf16_lo(w.x), a, b), fmaf(bf16_hi(w.x), a, b));
+        w.y = pack_bf16x2(fmaf(bf16_lo(w.y), a, b), fmaf(bf16_hi(w.y), a, b));
+        w.z = pack_bf16x2(fmaf(bf16_lo(w.z), a, b), fmaf(bf16_hi(w.z), a, b));
+        w.w = pack_bf16x2(fmaf(bf16_lo(w.w), a, b), fmaf(bf16_hi(w.w), a, b));
+      } else {
+        w.x = __float_as_uint(fmaf(__uint_as_float(w.x), a, b));
+        w.y = __float_as_uint(fmaf(__uint_as_float(w.y), a, b));
+        w.z = __float_as_uint(fmaf(__uint_as_float(w.z), a, b));
+        w.w = __float_as_uint(fmaf(__uint_as_float(w.w), a, b));
+      }
+      bv[i] = w;
+    }
+  } else {
+    for (long long i = threadIdx.x; i < cnt; i += blockDim.x) {
+      const int o = g * cpg + static_cast<int>(i / hw);
+      const float ga = gamma != nullptr ? to_f32(gamma[o]) : 1.0f;
+      const float be = beta != nullptr ? to_f32(beta[o]) : 0.0f;
+      blk[i] = from_f32<T>((to_f32(blk[i]) - mu) * rstd * ga + be);
+    }
+  }
+}
+
+}  // namespace kf

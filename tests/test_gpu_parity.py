@@ -1,0 +1,327 @@
+"""GPU parity: the CUDA chains (called through the C ABI) against the fp64 CPU oracle, element by
+element on the same seeded inputs.  Sizes span several tiles and ragged tails; the full-size
+benchmark configurations are checked on sampled rows / images in test_gpu_fullsize.py."""
+import math
+
+import numpy as np
+import pytest
+
+import kf_inputs as ki
+import oracle
+from gpu_util import assert_close, check_status, to_dev, to_f64, tol_for
+
+pytestmark = pytest.mark.gpu
+
+ACTS = ["none", "relu", "gelu_tanh", "sigmoid", "gelu_erf", "swish", "tanh", "hardtanh", "chain95"]
+
+
+@pytest.fixture(scope="module")
+def kf():
+    import paper_2605_30359_b200 as kf
+    kf.lib()
+    return kf
+
+
+def run_gemm(kf, d, act, scale=1.0, use_bias=True, use_res=True):
+    X, W = to_dev(d["X"]), to_dev(d["W"])
+    b = to_dev(d["b"]) if use_bias else None
+    R = to_dev(d["R"]) if (use_res and d["R"] is not None) else None
+    Y = kf.gemm_epilogue(X, W, b, act, scale, R)
+    check_status()
+    ref = oracle.gemm_epilogue(d["X"], d["W"], d["b"] if use_bias else None, act, scale,
+                               d["R"] if (use_res and d["R"] is not None) else None)
+    return to_f64(Y), ref
+
+
+# ------------------------------------------------------------------ config 1 (fp32), full size
+def test_c1_fp32_linear_bias_relu(kf):
+    d = ki.gemm_inputs("c1", seed=0)
+    got, ref = run_gemm(kf, d, "relu")
+    assert_close(got, ref, 1e-4, 1e-4, "c1")
+    assert ((got == 0) == (ref <= 0)).mean() > 0.999
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 1), (3, 5, 7), (33, 65, 31), (100, 37, 129), (64, 64, 64)])
+@pytest.mark.parametrize("act", ["none", "gelu_tanh", "sigmoid", "chain95"])
+def test_fp32_ragged_shapes(kf, shape, act):
+    M, N, K = shape
+    d = ki.gemm_inputs("c2", seed=3, M=M, N=N, K=K, dtype="f32")
+    got, ref = run_gemm(kf, d, act, 0.5)
+    assert_close(got, ref, 1e-4, 1e-4, "fp32 %s %s" % (shape, act))
+
+
+def test_fp32_gelu_variant_is_the_tanh_one(kf):
+    # X = 0, b = -3: the two GELUs differ by 4.1e-4 there, four times the fp32 tolerance
+    X = np.zeros((4, 8), np.float32); W = np.zeros((8, 8), np.float32)
+    b = np.full(8, -3.0, np.float32)
+    Y = kf.gemm_epilogue(to_dev(X), to_dev(W), to_dev(b), "gelu_tanh")
+    assert_close(to_f64(Y), np.full((4, 8), oracle.act("gelu_tanh", -3.0)), 1e-4, 1e-4, "gelu fixed point")
+    assert abs(to_f64(Y)[0, 0] - oracle.act("gelu_erf", -3.0)) > 3e-4
+
+
+# ------------------------------------------------------------------ bf16 tensor-core GEMM
+def test_bf16_layout_pins_onehot_and_permutation(kf):
+    """Products by 0/1 are exact, so any mismatch is a layout / swizzle / descriptor bug."""
+    M, N, K = 256, 512, 192
+    r = np.random.default_rng(5)
+    Wv = (r.integers(-64, 65, size=(N, K)) / 64.0)
+    ks = r.integers(0, K, size=M)
+    Xf = np.zeros((M, K)); Xf[np.arange(M), ks] = 1.0
+    Y = kf.gemm_epilogue(to_dev(ki.store(Xf, "bf16")), to_dev(ki.store(Wv, "bf16")))
+    check_status()
+    assert_close(to_f64(Y), Wv[:, ks].T, 0.0, 0.0, "one-hot X rows")
+    K2 = 512
+    Xv = (r.integers(-64, 65, size=(M, K2)) / 64.0)
+    perm = r.permutation(K2)
+    Wp = np.zeros((K2, K2)); Wp[np.arange(K2), perm] = 1.0
+    Y = kf.gemm_epilogue(to_dev(ki.store(Xv, "bf16")), to_dev(ki.store(Wp, "bf16")))
+    check_status()
+    assert_close(to_f64(Y), Xv[:, perm], 0.0, 0.0, "permutation W")
+
+
+@pytest.mark.parametrize("act", ACTS)
+def test_bf16_gemm_epilogue_all_activations(kf, act):
+    d = ki.gemm_inputs("c2", seed=1, M=300, N=520, K=200)       # 3x3 tiles, ragged in M, N and K
+    got, ref = run_gemm(kf, d, act, 0.5)
+    assert_close(got, ref, 2e-2, 2e-2, "bf16 %s" % act)
+
+
+@pytest.mark.parametrize("shape", [(128, 256, 64), (1, 8, 8), (129, 264, 72), (640, 128, 1024),
+                                   (257, 1000, 136), (130, 100, 64)])
+def test_bf16_gemm_shapes(kf, shape):
+    M, N, K = shape
+    d = ki.gemm_inputs("c2", seed=2, M=M, N=N, K=K)
+    got, ref = run_gemm(kf, d, "gelu_tanh", 0.5)
+    assert_close(got, ref, 2e-2, 2e-2, "bf16 %s" % (shape,))
+
+
+@pytest.mark.parametrize("shape", [(5, 7, 3), (17, 9, 13), (40, 33, 20)])
+def test_bf16_unaligned_shapes_take_the_scalar_kernel(kf, shape):
+    M, N, K = shape
+    d = ki.gemm_inputs("c2", seed=4, M=M, N=N, K=K)
+    got, ref = run_gemm(kf, d, "gelu_tanh", 0.5)
+    assert_close(got, ref, 2e-2, 2e-2, "bf16 scalar %s" % (shape,))
+
+
+def test_bf16_zero_inputs_return_residual_bit_exact(kf):
+    d = ki.gemm_inputs("c2", seed=6, M=256, N=256, K=128)
+    Z = np.zeros_like(d["X"])
+    zb = np.zeros_like(d["b"])
+    Y = kf.gemm_epilogue(to_dev(Z), to_dev(d["W"]), to_dev(zb), "gelu_tanh", 0.5, to_dev(d["R"]))
+    assert np.array_equal(to_f64(Y), ki.widen(d["R"]))
+    # X = 0, b = value: every row equals scale*act(b) + R
+    Y = kf.gemm_epilogue(to_dev(Z), to_dev(d["W"]), to_dev(d["b"]), "relu", 2.0, None)
+    want = 2.0 * np.maximum(ki.widen(d["b"]), 0.0)
+    assert_close(to_f64(Y), np.broadcast_to(want, (256, 256)), 2e-2, 2e-2, "X=0")
+
+
+def test_bf16_no_bias_no_residual_and_strided_operands(kf):
+    import torch
+    d = ki.gemm_inputs("c2", seed=7, M=200, N=264, K=128)
+    got, ref = run_gemm(kf, d, "relu", 1.0, use_bias=False, use_res=False)
+    assert_close(got, ref, 2e-2, 2e-2, "no bias")
+    # leading dimensions larger than the row length
+    Xp = torch.zeros(200, 160, dtype=torch.bfloat16, device="cuda"); Xp[:, :128] = to_dev(d["X"])
+    Yp = torch.full((200, 272), 7.0, dtype=torch.bfloat16, device="cuda")
+    kf.gemm_epilogue(Xp[:, :128], to_dev(d["W"]), to_dev(d["b"]), "relu", 1.0, None, out=Yp[:, :264])
+    check_status()
+    ref = oracle.gemm_epilogue(d["X"], d["W"], d["b"], "relu")
+    assert_close(to_f64(Yp[:, :264]), ref, 2e-2, 2e-2, "strided")
+    assert (Yp[:, 264:] == 7.0).all()                          # padding columns untouched
+
+
+def test_repeat_runs_are_bit_identical(kf):
+    d = ki.gemm_inputs("c3", seed=8, M=300, N=1100, K=256)
+    X, W, b = to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"])
+    a1 = kf.gemm_rowreduce(X, W, b, "none", "softmax").clone()
+    s1 = kf.gemm_rowreduce(X, W, b, "sigmoid", "sum").clone()
+    for _ in range(3):
+        assert (kf.gemm_rowreduce(X, W, b, "none", "softmax") == a1).all()
+        assert (kf.gemm_rowreduce(X, W, b, "sigmoid", "sum") == s1).all()
+
+
+# ------------------------------------------------------------------ row reductions
+def softmax_gates(got, ref, what):
+    assert_close(got, ref, 2e-2, 2e-2, what)                     # the official (weak) tolerance
+    assert_close(got, ref, 1e-7, 2e-2, what + " relative")       # elementwise relative error
+    assert np.abs(got.sum(axis=1) - 1.0).max() < 4e-3, what
+
+
+@pytest.mark.parametrize("shape", [(200, 1000, 136), (128, 256, 64), (300, 2056, 512), (1, 8, 8)])
+def test_bf16_softmax(kf, shape):
+    M, N, K = shape
+    d = ki.gemm_inputs("c3", seed=1, M=M, N=N, K=K)
+    P = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "none", "softmax")
+    check_status()
+    softmax_gates(to_f64(P), oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "none", "softmax"),
+                  "softmax %s" % (shape,))
+
+
+def test_bf16_softmax_fp32_output_and_closed_forms(kf):
+    import torch
+    N, K = 1024, 64
+    X = np.zeros((130, K)); W = ki.normal(1, 2, (N, K))
+    b = np.full(N, 0.75)
+    P = kf.gemm_rowreduce(to_dev(ki.store(X, "bf16")), to_dev(ki.store(W, "bf16")),
+                          to_dev(ki.store(b, "bf16")), "none", "softmax", out_dtype=torch.float32)
+    check_status()
+    assert_close(to_f64(P), np.full((130, N), 1.0 / N), 0.0, 1e-6, "constant row")
+    # one logit far above the rest: one-hot, no overflow
+    b2 = np.zeros(N); b2[700] = 120.0
+    P = kf.gemm_rowreduce(to_dev(ki.store(X, "bf16")), to_dev(ki.store(W, "bf16")),
+                          to_dev(ki.store(b2, "bf16")), "none", "softmax", out_dtype=torch.float32)
+    got = to_f64(P)
+    assert not np.isnan(got).any() and (got[:, 700] == 1.0).all() and got.sum() == 130.0
+    d = ki.gemm_inputs("c3", seed=2, M=150, N=1024, K=128)
+    P = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "none", "softmax",
+                          out_dtype=torch.float32)
+    ref = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "none", "softmax")
+    assert_close(to_f64(P), ref, 1e-7, 1e-3, "softmax fp32 out")
+
+
+@pytest.mark.parametrize("shape", [(200, 1000, 136), (128, 256, 64), (513, 1024, 256)])
+def test_bf16_sigmoid_rowsum(kf, shape):
+    M, N, K = shape
+    d = ki.gemm_inputs("c4", seed=1, M=M, N=N, K=K)
+    S = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "sigmoid", "sum")
+    check_status()
+    ref = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "sigmoid", "sum")
+    assert_close(to_f64(S), ref, 2e-2, 2e-2, "rowsum %s" % (shape,))
+    assert_close(to_f64(S), ref, 0.0, 1e-3, "rowsum relative %s" % (shape,))
+
+
+def test_rowsum_closed_forms(kf):
+    N, K = 1024, 128
+    d = ki.gemm_inputs("c4", seed=3, M=256, N=N, K=K)
+    zX = np.zeros_like(d["X"]); zb = np.zeros_like(d["b"])
+    S = kf.gemm_rowreduce(to_dev(zX), to_dev(d["W"]), to_dev(zb), "sigmoid", "sum")
+    assert_close(to_f64(S), np.full(256, N / 2), 0.0, 1e-6, "X=0,b=0")
+    # sigmoid(z)+sigmoid(-z)=1: stacking W with -W and b with -b gives N per row for any X
+    W2 = np.concatenate([ki.widen(d["W"])[:512], -ki.widen(d["W"])[:512]])
+    b2 = np.concatenate([ki.widen(d["b"])[:512], -ki.widen(d["b"])[:512]])
+    S = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(ki.store(W2, "bf16")), to_dev(ki.store(b2, "bf16")),
+                          "sigmoid", "sum")
+    assert_close(to_f64(S), np.full(256, 512.0), 0.0, 1e-4, "antisymmetry")
+
+
+@pytest.mark.parametrize("red,act", [("softmax", "none"), ("sum", "sigmoid"), ("softmax", "relu")])
+@pytest.mark.parametrize("dtype,shape", [("f32", (33, 70, 31)), ("f32", (128, 256, 512)), ("bf16", (9, 21, 13))])
+def test_scalar_path_row_reductions(kf, red, act, dtype, shape):
+    M, N, K = shape
+    d = ki.gemm_inputs("c3", seed=4, M=M, N=N, K=K, dtype=dtype)
+    out = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), act, red)
+    check_status()
+    ref = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], act, red)
+    atol, rtol = tol_for(dtype)
+    assert_close(to_f64(out), ref, atol, rtol, "scalar %s %s %s" % (red, dtype, shape))
+    if red == "softmax":
+        assert_close(to_f64(out), ref, 1e-7, 2e-4 if dtype == "f32" else 2e-2, "relative")
+
+
+# ------------------------------------------------------------------ convolution + GroupNorm
+def run_conv(kf, d, act="relu", groups=None, gamma=None, beta=None, use_bias=True):
+    groups = d["groups"] if groups is None else groups
+    y = kf.conv3x3_epilogue(to_dev(d["x"]), to_dev(d["w"]), to_dev(d["bias"]) if use_bias else None,
+                            act, groups, d["eps"], to_dev(gamma), to_dev(beta))
+    check_status()
+    ref = oracle.conv3x3_gn(d["x"], d["w"], d["bias"] if use_bias else None, act, groups, d["eps"],
+                            gamma, beta)
+    return to_f64(y), ref
+
+
+@pytest.mark.parametrize("cfg", [
+    dict(Nb=2, Cin=64, H=8, W=64, Cout=128, groups=32),      # benchmark geometry, small
+    dict(Nb=3, Cin=128, H=16, W=32, Cout=64, groups=4),      # two channel blocks per tap, 4 rows per tile
+    dict(Nb=1, Cin=64, H=16, W=8, Cout=256, groups=0),       # 16 rows per tile, widest N tile, no norm
+    dict(Nb=2, Cin=64, H=2, W=128, Cout=48, groups=3),       # one row per tile, Cout below the tile width
+])
+def test_bf16_conv_tensor_core_path(kf, cfg):
+    d = ki.conv_inputs(seed=1, **cfg)
+    got, ref = run_conv(kf, d)
+    assert_close(got, ref, 2e-2, 2e-2, "conv %s" % cfg)
+
+
+def test_bf16_conv_position_pins(kf):
+    """Delta kernels and all-ones inputs: exact results that pin tap orientation and padding."""
+    Nb, C, H, W = 2, 64, 8, 64
+    r = np.random.default_rng(2)
+    xv = r.integers(-32, 33, size=(Nb, C, H, W)) / 32.0
+    for (rr, ss) in [(1, 1), (0, 0), (2, 1), (1, 2), (0, 2)]:
+        wt = np.zeros((C, C, 3, 3)); wt[np.arange(C), np.arange(C), rr, ss] = 1.0
+        d = dict(x=ki.store(xv, "bf16"), w=ki.store(wt, "bf16"), bias=None, groups=0, eps=1e-5)
+        got, ref = run_conv(kf, d, act="none", use_bias=False)
+        assert_close(got, ref, 0.0, 0.0, "delta tap (%d,%d)" % (rr, ss))
+    d = dict(x=ki.store(np.ones((1, C, H, W)), "bf16"), w=ki.store(np.ones((16, C, 3, 3)), "bf16"),
+             bias=None, groups=0, eps=1e-5)
+    got, _ = run_conv(kf, d, act="none", use_bias=False)
+    assert got[0, 0, 3, 5] == 9 * C and got[0, 3, 0, 5] == 6 * C and got[0, 15, H - 1, W - 1] == 4 * C
+
+
+def test_bf16_conv_groupnorm_moments_and_affine(kf):
+    d = ki.conv_inputs(seed=3, Nb=2, Cin=64, H=16, W=64, Cout=128, groups=32)
+    got, ref = run_conv(kf, d)
+    blk = got.reshape(2, 32, -1)
+    assert np.abs(blk.mean(axis=2)).max() < 2e-3
+    assert np.abs(blk.var(axis=2) - 1.0).max() < 1e-2
+    gamma = ki.store(ki.uniform(3, 7, (128,), 0.5, 1.5), "bf16")
+    beta = ki.store(ki.uniform(3, 8, (128,), -1.0, 1.0), "bf16")
+    got, ref = run_conv(kf, d, gamma=gamma, beta=beta)
+    assert_close(got, ref, 2e-2, 2e-2, "affine")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("cfg", [dict(Nb=1, Cin=2, H=1, W=1, Cout=4, groups=2),
+                                 dict(Nb=2, Cin=3, H=5, W=7, Cout=6, groups=3),
+                                 dict(Nb=2, Cin=4, H=9, W=4, Cout=8, groups=0)])
+def test_conv_scalar_path(kf, dtype, cfg):
+    d = ki.conv_inputs(seed=4, dtype=dtype, **cfg)
+    got, ref = run_conv(kf, d)
+    atol, rtol = tol_for(dtype)
+    if dtype == "f32" and d["groups"] > 0:
+        atol, rtol = 5e-4, 5e-4      # rsqrt of a small-sample variance amplifies fp32 rounding
+    assert_close(got, ref, atol, rtol, "conv scalar %s %s" % (dtype, cfg))
+
+
+def test_groupnorm_biased_variance_on_gpu(kf):
+    # 1x1 image, four channels per group, x = 0 so the activations are the biases {1,2,3,4}/4
+    bias = np.array([0.25, 0.5, 0.75, 1.0, 2.0, 2.0, 2.0, 2.0], np.float32)
+    d = dict(x=np.zeros((1, 2, 1, 1), np.float32), w=np.zeros((8, 2, 3, 3), np.float32), bias=bias,
+             groups=2, eps=0.0)
+    got, ref = run_conv(kf, d)
+    v = np.array([0.25, 0.5, 0.75, 1.0])
+    assert_close(got[0, :4, 0, 0], (v - 0.625) / math.sqrt(5.0 / 64), 1e-5, 1e-5, "biased variance")
+    d["eps"] = 1e-5
+    got, _ = run_conv(kf, d)
+    assert (got[0, 4:, 0, 0] == 0).all()
+
+
+# ------------------------------------------------------------------ error handling on the device box
+def test_workspace_errors(kf):
+    import torch
+    d = ki.gemm_inputs("c3", seed=1, M=128, N=512, K=64)
+    X, W = to_dev(d["X"]), to_dev(d["W"])
+    out = torch.empty(128, 512, dtype=torch.bfloat16, device="cuda")
+    before = kf.kf_launch_count()
+    st = kf.kf_gemm_rowreduce(128, 512, 64, kf.KF_BF16, X.data_ptr(), 64, W.data_ptr(), 64, None, 0, 0,
+                              out.data_ptr(), 512, kf.KF_BF16, None, 0, None)
+    assert st == kf.KF_ERR_WORKSPACE
+    ws = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    st = kf.kf_gemm_rowreduce(128, 512, 64, kf.KF_BF16, X.data_ptr(), 64, W.data_ptr(), 64, None, 0, 0,
+                              out.data_ptr(), 512, kf.KF_BF16, ws.data_ptr() + 8, 4088, None)
+    assert st == kf.KF_ERR_WORKSPACE
+    assert kf.kf_launch_count() == before
+    with pytest.raises(kf.KfError):
+        kf.gemm_epilogue(X, W, act="none", out=X)
+
+
+def test_calls_on_a_side_stream(kf):
+    import torch
+    d = ki.gemm_inputs("c2", seed=9, M=256, N=256, K=128)
+    s = torch.cuda.Stream()
+    X, W, b, R = to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), to_dev(d["R"])
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s):
+        Y = kf.gemm_epilogue(X, W, b, "gelu_tanh", 0.5, R, stream=s)
+    s.synchronize()
+    ref = oracle.gemm_epilogue(d["X"], d["W"], d["b"], "gelu_tanh", 0.5, d["R"])
+    assert_close(to_f64(Y), ref, 2e-2, 2e-2, "side stream")

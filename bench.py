@@ -1,0 +1,439 @@
+#!/usr/bin/env python
+"""Benchmark of the fused operator chains on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extras]
+
+One step = one pass of the headline chain over one batch of synthetic input: config 2,
+bf16 Y = 0.5*GELU_tanh(X W^T + b) + R with X[8192,4096], W[4096,4096] (fp32 accumulate, bf16 out),
+through the C-ABI call kf_gemm_epilogue.  The metric is fused-chain TFLOP/s (2*M*N*K per call).
+With N > 1 (torchrun) every rank runs the same shape on its own batch (rows are independent:
+weak scaling, no collective on the data path); the value is the aggregate over ranks and the
+time is the maximum over ranks.
+
+Prints ONE JSON line with the metric, the roofline of the dominant kernel, the CPU oracle
+timed on a bounded sample (rank 0, N = 1), the end-to-end figure with host buffers, and, as
+context, every other benchmark chain next to the same chain as separate torch ops.
+
+--impl reference times the fp64 CPU oracle on the host cores instead (a deliberately slow
+program: a reported baseline, not a target).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import kf_inputs as ki  # noqa: E402
+
+WORKLOAD = "c2"
+M2, N2, K2 = 8192, 4096, 4096
+FLOPS_C2 = 2.0 * M2 * N2 * K2
+ALG_BYTES_C2 = 2 * (M2 * K2 + N2 * K2 + N2 + 2 * M2 * N2)   # X, W, b, R read once, Y written once
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            d["_source"] = "measured"
+            return d
+        except Exception:
+            pass
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+def load_traffic():
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if any."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        return json.load(open(p))
+    except Exception:
+        return {}
+
+
+# ------------------------------------------------------------------ clocks during the timed region
+class ClockSampler:
+    """Polls NVML (read-only) for SM clock and throttle reasons while a timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ helpers
+def to_dev(a, device):
+    import torch
+    if a is None:
+        return None
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).to(device)
+    return torch.from_numpy(a).to(device)
+
+
+def to_pinned(a):
+    import torch
+    if a.dtype == np.uint16:
+        t = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
+    else:
+        t = torch.from_numpy(a)
+    return t.pin_memory()
+
+
+def time_calls(fn, iters, warmup, graph_batch=0):
+    """Average device time of fn() in microseconds (CUDA events on the current stream).
+
+    graph_batch > 0 captures that many calls into a CUDA graph first, so that launch-bound
+    chains are timed on the device rather than at the host's launch rate."""
+    import torch
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    runner, per = fn, 1
+    if graph_batch > 0:
+        try:
+            g = torch.cuda.CUDAGraph()
+            s = torch.cuda.Stream()
+            s.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(s):
+                fn()
+                with torch.cuda.graph(g, stream=s):
+                    for _ in range(graph_batch):
+                        fn()
+            torch.cuda.current_stream().wait_stream(s)
+            torch.cuda.synchronize()
+            runner, per = g.replay, graph_batch
+            runner()
+            torch.cuda.synchronize()
+        except Exception:
+            runner, per = fn, 1
+    reps = max(1, iters // per)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        runner()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / (reps * per)
+
+
+# ------------------------------------------------------------------ the CPU oracle as a baseline
+def oracle_sample_c2(d, target_seconds=12.0):
+    """Time the fp64 oracle on the first rows of the workload; returns (rows, seconds, cores)."""
+    import oracle
+    cores = oracle.get_threads()
+    probe = 128
+    t0 = time.perf_counter()
+    oracle.gemm_epilogue(d["X"][:probe], d["W"], d["b"], "gelu_tanh", 0.5, d["R"][:probe])
+    dt = time.perf_counter() - t0
+    rows = int(min(d["X"].shape[0], max(probe, (target_seconds / dt) * probe)))
+    rows -= rows % 128
+    t0 = time.perf_counter()
+    oracle.gemm_epilogue(d["X"][:rows], d["W"], d["b"], "gelu_tanh", 0.5, d["R"][:rows])
+    return rows, time.perf_counter() - t0, cores
+
+
+def run_reference(args):
+    """--impl reference: the oracle, as it stands, on the host cores; rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    d = ki.gemm_inputs(WORKLOAD, seed=0)
+    cores = oracle.get_threads()
+    # size one step at ~6 s of CPU work so that warmup + steps end within a few minutes
+    probe = 128
+    t0 = time.perf_counter()
+    oracle.gemm_epilogue(d["X"][:probe], d["W"], d["b"], "gelu_tanh", 0.5, d["R"][:probe])
+    dt = time.perf_counter() - t0
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    rows = int(min(M2, max(probe, (min(6.0, budget) / dt) * probe)))
+    rows -= rows % 128
+    step = lambda: oracle.gemm_epilogue(d["X"][:rows], d["W"], d["b"], "gelu_tanh", 0.5, d["R"][:rows])
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    secs = time.perf_counter() - t0
+    flops = 2.0 * rows * N2 * K2 * args.steps
+    val = flops / secs / 1e12
+    sample = "rows [0,%d) of X/R per step, all of W (%.3g of the workload's FLOPs)" % (rows, rows / M2)
+    line = {
+        "impl": "reference", "metric": "fused_chain_tflops", "value": val, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": secs * 1e3 / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "c2: bf16 Linear+bias+GELU(tanh)*0.5+residual, X[8192,4096] W[4096,4096]",
+                   "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------ context: the other chains
+def torch_unfused(name, t):
+    """The same chain as separate eager torch ops (the paper's speedup denominator)."""
+    import torch
+    import torch.nn.functional as F
+    if name == "c1":
+        return lambda: torch.relu(F.linear(t["X"], t["W"], t["b"]))
+    if name == "c2":
+        return lambda: F.gelu(F.linear(t["X"], t["W"], t["b"]), approximate="tanh") * 0.5 + t["R"]
+    if name == "c3":
+        return lambda: torch.softmax(F.linear(t["X"], t["W"], t["b"]), dim=1)
+    if name == "c4":
+        return lambda: torch.sigmoid(F.linear(t["X"], t["W"], t["b"])).sum(dim=1, dtype=torch.float32)
+    return lambda: F.group_norm(torch.relu(F.conv2d(t["x"], t["w"], t["bias"], padding=1)), 32, eps=1e-5)
+
+
+def chain_table(kf, device, peaks, c2_tensors, c2_us):
+    """us/call, TFLOP/s and roofline fractions of every benchmark chain + unfused torch."""
+    import torch
+    torch.backends.cuda.matmul.allow_tf32 = False
+    torch.backends.cudnn.allow_tf32 = False
+    out = {}
+    specs = {
+        "c1": dict(flops=2.0 * 128 * 256 * 512, bytes=4 * (128 * 512 + 256 * 512 + 256 + 128 * 256)),
+        "c2": dict(flops=FLOPS_C2, bytes=ALG_BYTES_C2),
+        "c3": dict(flops=2.0 * 4096 * 8192 * 2048, bytes=2 * (4096 * 2048 + 8192 * 2048 + 8192 + 4096 * 8192)),
+        "c4": dict(flops=2.0 * 16384 * 1024 * 1024, bytes=2 * (16384 * 1024 + 1024 * 1024 + 1024) + 4 * 16384),
+        "c5": dict(flops=2.0 * 128 * 64 * 64 * 128 * 576,
+                   bytes=2 * (128 * 64 * 64 * 64 + 128 * 64 * 9 + 128 + 128 * 128 * 64 * 64)),
+    }
+    for name in ("c1", "c2", "c3", "c4", "c5"):
+        if name == "c2":
+            t = c2_tensors
+        elif name == "c5":
+            d = ki.conv_inputs("c5", seed=0)
+            t = {k: to_dev(d[k], device) for k in ("x", "w", "bias")}
+        else:
+            d = ki.gemm_inputs(name, seed=0)
+            t = {k: to_dev(d[k], device) for k in ("X", "W", "b")}
+        if name == "c1":
+            fn = lambda: kf.gemm_epilogue(t["X"], t["W"], t["b"], "relu")
+        elif name == "c2":
+            fn = None
+        elif name == "c3":
+            o3 = torch.empty(4096, 8192, dtype=torch.bfloat16, device=device)
+            fn = lambda: kf.gemm_rowreduce(t["X"], t["W"], t["b"], "none", "softmax", out=o3)
+        elif name == "c4":
+            o4 = torch.empty(16384, dtype=torch.float32, device=device)
+            fn = lambda: kf.gemm_rowreduce(t["X"], t["W"], t["b"], "sigmoid", "sum", out=o4)
+        else:
+            o5 = torch.empty(128, 128, 64, 64, dtype=torch.bfloat16, device=device)
+            fn = lambda: kf.conv3x3_epilogue(t["x"], t["w"], t["bias"], "relu", 32, 1e-5, out=o5)
+        small = name in ("c1", "c4")
+        us = c2_us if fn is None else time_calls(fn, 200 if small else 40, 5, graph_batch=20 if small else 0)
+        us_torch = time_calls(torch_unfused(name, t), 200 if small else 20, 5, graph_batch=20 if small else 0)
+        s = specs[name]
+        tf = s["flops"] / us / 1e6
+        gbs = s["bytes"] / us / 1e3
+        out[name] = {
+            "us_per_call": round(us, 3), "tflops": round(tf, 2),
+            "frac_tensor_peak_measured_burst": round(tf / peaks["bf16_tflops"], 4),
+            "frac_tensor_peak_nominal_2250": round(tf / 2250.0, 4),
+            "algorithmic_gbs": round(gbs, 1), "frac_hbm_measured": round(gbs / peaks["hbm_gbs"], 4),
+            "unfused_torch_us": round(us_torch, 3), "speedup_vs_unfused_torch": round(us_torch / us, 3),
+        }
+        del t
+    return out
+
+
+# ------------------------------------------------------------------ main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the context table and baselines")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the chains have no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    import paper_2605_30359_b200 as kf   # raises if libkf.so is missing
+    kf.lib()
+    peaks = load_peaks()
+
+    # inputs: rank r works on its own batch (seed r); resident in HBM before the timed region
+    d = ki.gemm_inputs(WORKLOAD, seed=rank)
+    t = {k: to_dev(d[k], device) for k in ("X", "W", "b", "R")}
+    Y = torch.empty(M2, N2, dtype=torch.bfloat16, device=device)
+    step = lambda: kf.gemm_epilogue(t["X"], t["W"], t["b"], "gelu_tanh", 0.5, t["R"], out=Y)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = kf.kf_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = kf.kf_launch_count() - launches0
+    clocks = sampler.stop()
+    if kf.kf_device_status() != kf.KF_OK:
+        raise SystemExit("device status reports a timed-out wait: the run is invalid")
+    if world > 1:
+        tt = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt.item())
+    ms_per_step = ms / args.steps
+    value = FLOPS_C2 * world / (ms_per_step * 1e-3) / 1e12
+    kernel_tflops = FLOPS_C2 / (ms_per_step * 1e-3) / 1e12          # one launch per step per rank
+
+    # end to end: pinned host buffers in, host buffer out, copies inside the timed region
+    hX, hW, hb, hR = (to_pinned(d[k]) for k in ("X", "W", "b", "R"))
+    hY = torch.empty(M2, N2, dtype=torch.bfloat16).pin_memory()
+    e2e_steps = max(3, min(args.steps, 10))
+
+    def e2e_step():
+        return kf.gemm_epilogue_host(hX, hW, hb, "gelu_tanh", 0.5, hR, out_host=hY, device=device)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        tt = torch.tensor([e2e_ms], dtype=torch.float64, device=device)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item())
+    e2e_val = FLOPS_C2 * world / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    h2d = sum(x.numel() * x.element_size() for x in (hX, hW, hb, hR))
+    d2h = hY.numel() * hY.element_size()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    traffic = load_traffic().get("umma_chain_kernel_c2_bytes_per_launch")
+    line = {
+        "metric": "fused_chain_tflops", "value": round(value, 2), "unit": "TFLOP/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": round(ms_per_step, 5), "us_per_call": round(ms_per_step * 1e3, 2),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": "c2: bf16 Linear+bias+GELU(tanh)*0.5+residual, X[8192,4096] W[4096,4096] "
+                               "b[4096] R[8192,4096], fp32 accumulate, bf16 out",
+                   "flops_per_step_per_gpu": FLOPS_C2, "l2": "inputs larger than L2 (235 MB per step)",
+                   "parallelism": "replicas: each rank its own batch, no collective",
+                   "peaks": peaks["_source"]},
+        "clocks": clocks,
+        "e2e": {"value": round(e2e_val, 2), "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "kernel": "umma_chain_kernel<256,elementwise,gelu_tanh>",
+                     "achieved": round(kernel_tflops, 2), "peak": peaks["bf16_tflops"],
+                     "unit": "TFLOP/s", "frac": round(kernel_tflops / peaks["bf16_tflops"], 4),
+                     "frac_of_sustained_peak": round(kernel_tflops / peaks["bf16_tflops_sustained"], 4),
+                     "frac_of_nominal_2250": round(kernel_tflops / 2250.0, 4),
+                     "peak_source": peaks["_source"] + " cuBLAS bf16 burst",
+                     "traffic": traffic},
+    }
+    if world == 1 and not args.no_extras:
+        rows, secs, cores = oracle_sample_c2(d)
+        line["cpu_baseline"] = {
+            "value": round(2.0 * rows * N2 * K2 / secs / 1e12, 6), "unit": "TFLOP/s", "cores": cores,
+            "kind": "oracle", "seconds": round(secs, 2),
+            "sample": "rows [0,%d) of X/R, all of W (%.3g of one step's FLOPs)" % (rows, rows / M2)}
+        line["chains"] = chain_table(kf, device, peaks, t, ms_per_step * 1e3)
+        line["paper_context"] = {"hardware": "RTX 5090", "matmul_centered_avg_speedup": 1.16,
+                                 "conv_centered_avg_speedup": 1.33, "mixed_reduction_avg_speedup": 1.23,
+                                 "reduction_dominated_avg_speedup": 6.56}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -238,3 +238,42 @@ def conv3x3_epilogue(x, w, bias=None, act="none", groups=0, eps=1e-5, gamma=None
     if st != KF_OK:
         raise KfError(st, "kf_conv3x3_epilogue")
     return out
+
+
+# ------------------------------------------------------------------ host-buffer front end
+_staging = {}
+
+
+def _stage(name, host, device):
+    """Device staging buffer matching a host tensor (cached: repeated calls allocate nothing)."""
+    torch = _torch()
+    key = (name, tuple(host.shape), host.dtype, device.index)
+    buf = _staging.get(key)
+    if buf is None:
+        buf = torch.empty(host.shape, dtype=host.dtype, device=device)
+        _staging[key] = buf
+    return buf
+
+
+def gemm_epilogue_host(X, W, bias=None, act="none", scale=1.0, residual=None, out_host=None,
+                       device=None, stream=None):
+    """gemm_epilogue for HOST tensors (pinned memory recommended): copies the inputs to the
+    device, runs the fused kernel, copies Y back into out_host.  Everything is enqueued on one
+    stream; synchronise that stream before reading out_host."""
+    torch = _torch()
+    device = device or torch.device("cuda", torch.cuda.current_device())
+    s = stream if stream is not None else torch.cuda.current_stream(device)
+    with torch.cuda.stream(s):
+        dX = _stage("X", X, device); dX.copy_(X, non_blocking=True)
+        dW = _stage("W", W, device); dW.copy_(W, non_blocking=True)
+        db = dR = None
+        if bias is not None:
+            db = _stage("b", bias, device); db.copy_(bias, non_blocking=True)
+        if residual is not None:
+            dR = _stage("R", residual, device); dR.copy_(residual, non_blocking=True)
+        if out_host is None:
+            out_host = torch.empty((X.shape[0], W.shape[0]), dtype=X.dtype).pin_memory()
+        dY = _stage("Y", out_host, device)
+        gemm_epilogue(dX, dW, db, act, scale, dR, out=dY, stream=s)
+        out_host.copy_(dY, non_blocking=True)
+    return out_host

@@ -94,6 +94,34 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype,
                             void* out, int64_t ldo, kf_dtype out_dtype,
                             void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Row reduction for callers that cannot allocate device memory (no counterpart in the paper:
+ * this is a packaging variant of kf_gemm_rowreduce, not another chain).
+ *
+ * Who needs it: anything that calls from a place where cudaMalloc is forbidden or bound to
+ * fail -- inside an inference runtime's enqueue hook, in a process whose own allocator
+ * already owns all device memory, or in a serving loop that must not allocate after
+ * start-up -- and that therefore has no workspace to pass.
+ *
+ * Same arguments, results and error codes as kf_gemm_rowreduce, minus the workspace: the
+ * per-tile partial statistics go to a fixed KF_STATIC_SCRATCH_BYTES array that is part of the
+ * library image (each GPU that loads the library holds those bytes until the process exits).
+ * The call allocates nothing: no cudaMalloc/cudaFree, no allocating library routine.
+ *   - Limit: a problem whose kf_gemm_rowreduce_workspace_bytes() exceeds
+ *     KF_STATIC_SCRATCH_BYTES is refused with KF_ERR_WORKSPACE and nothing is launched
+ *     (bf16, K % 8 == 0: M * ceil(N/256) * 8 bytes for softmax, * 4 for sum; otherwise M*N*4).
+ *   - The first call on each device looks up the array's device address (a one-time host-side
+ *     query, made with that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the last call wrote.
+ *     No entry has to start at zero (every entry read was written earlier in the same call),
+ *     but two calls that may overlap on the GPU -- different streams without an ordering
+ *     between them -- race on it.  Keep calls to this function ordered on one stream. */
+#define KF_STATIC_SCRATCH_BYTES (2u << 20)
+kf_status kf_gemm_rowreduce_static(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype,
+                                   const void* X, int64_t ldx, const void* W, int64_t ldw,
+                                   const void* bias, kf_act pre_act, kf_rowred red,
+                                   void* out, int64_t ldo, kf_dtype out_dtype,
+                                   void* cuda_stream);
+
 /* 3x3 convolution (pad 1, stride 1, cross-correlation as in torch.nn.Conv2d) + activation +
  * optional GroupNorm (Table 2 "Conv-centered" chains).
  *   c[n,o,h,w] = bias[o] + sum_{c,r,s} x[n,c,h+r-1,w+s-1] * w[o,c,r,s]      (zero padding)

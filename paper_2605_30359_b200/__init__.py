@@ -26,7 +26,8 @@ ACT = {"none": 0, "relu": 1, "gelu_tanh": 2, "sigmoid": 3, "gelu_erf": 4, "swish
        "hardtanh": 7, "chain95": 8}
 RED = {"softmax": 0, "sum": 1}
 
-EXPORTS = ["kf_gemm_epilogue", "kf_gemm_rowreduce", "kf_conv3x3_epilogue",
+EXPORTS = ["kf_gemm_epilogue", "kf_gemm_rowreduce", "kf_gemm_rowreduce_static",
+           "kf_conv3x3_epilogue",
            "kf_gemm_epilogue_workspace_bytes", "kf_gemm_rowreduce_workspace_bytes",
            "kf_conv3x3_workspace_bytes", "kf_device_status", "kf_launch_count",
            "kf_status_string", "kf_version"]
@@ -57,6 +58,9 @@ def lib() -> ctypes.CDLL:
     L.kf_gemm_rowreduce.restype = ci
     L.kf_gemm_rowreduce.argtypes = [i64, i64, i64, ci, vp, i64, vp, i64, vp, ci, ci, vp, i64, ci,
                                     vp, sz, vp]
+    L.kf_gemm_rowreduce_static.restype = ci
+    L.kf_gemm_rowreduce_static.argtypes = [i64, i64, i64, ci, vp, i64, vp, i64, vp, ci, ci, vp, i64,
+                                           ci, vp]
     L.kf_conv3x3_epilogue.restype = ci
     L.kf_conv3x3_epilogue.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, ci, f32, vp, vp,
                                       vp, vp, sz, vp]
@@ -89,6 +93,17 @@ def kf_gemm_rowreduce(M, N, K, in_dtype, X, ldx, W, ldw, bias, pre_act, red, out
                       workspace, workspace_bytes, stream) -> int:
     return lib().kf_gemm_rowreduce(M, N, K, in_dtype, X, ldx, W, ldw, bias, pre_act, red, out, ldo,
                                    out_dtype, workspace, workspace_bytes, stream)
+
+
+KF_STATIC_SCRATCH_BYTES = 2 << 20
+
+
+def kf_gemm_rowreduce_static(M, N, K, in_dtype, X, ldx, W, ldw, bias, pre_act, red, out, ldo,
+                             out_dtype, stream) -> int:
+    """kf_gemm_rowreduce for callers that cannot allocate: no workspace argument, the partial
+    statistics go to a fixed array inside the library (at most KF_STATIC_SCRATCH_BYTES)."""
+    return lib().kf_gemm_rowreduce_static(M, N, K, in_dtype, X, ldx, W, ldw, bias, pre_act, red,
+                                          out, ldo, out_dtype, stream)
 
 
 def kf_conv3x3_epilogue(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, groups, eps, gamma, beta,

@@ -365,3 +365,62 @@ kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Row reduction without any allocation.
+//
+// Some callers have no way to hand the library a scratch buffer, because they cannot allocate
+// device memory at the point where they call: plug-ins of an inference runtime whose enqueue
+// hook must not allocate, services whose allocator has already claimed the whole device so that
+// a further cudaMalloc simply fails, and latency-critical loops that forbid allocation after
+// start-up.
+// For them the per-tile partial statistics of kf_gemm_rowreduce live in the fixed array below,
+// which is part of the loaded library image: every GPU that loads the library carries these
+// bytes until the process exits, whether or not the entry point is ever used.
+//
+// g_static_scratch names the array for DEVICE code.  In host code the same name is only a
+// host-side handle: handing it to a kernel as if it were an address would make the kernel
+// fault, or quietly use unrelated memory on systems where the GPU can reach host memory.  The
+// real device address is asked for once per device, with that device current, through
+// cudaGetSymbolAddress, and only that address is passed on.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+static __device__ __align__(256) unsigned char g_static_scratch[KF_STATIC_SCRATCH_BYTES];
+
+std::mutex g_static_mu;
+void* g_static_scratch_addr[64];   // per device, filled on first use
+
+// Device address of this device's copy of the array; nullptr on failure.
+void* static_scratch_address() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lk(g_static_mu);
+  if (g_static_scratch_addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_scratch) != cudaSuccess)
+      return nullptr;
+    g_static_scratch_addr[dev] = ptr;
+  }
+  return g_static_scratch_addr[dev];
+}
+
+}  // namespace
+
+extern "C" kf_status kf_gemm_rowreduce_static(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype,
+                                              const void* X, int64_t ldx, const void* W,
+                                              int64_t ldw, const void* bias, kf_act pre_act,
+                                              kf_rowred red, void* out, int64_t ldo,
+                                              kf_dtype out_dtype, void* cuda_stream) {
+  // Refuse, before touching the device, any problem whose partial statistics do not fit.
+  if (M >= 1 && N >= 1 && K >= 1 && (red == KF_RED_SOFTMAX || red == KF_RED_SUM) &&
+      (in_dtype == KF_F32 || in_dtype == KF_BF16) &&
+      kf_gemm_rowreduce_workspace_bytes(M, N, K, in_dtype, red) > KF_STATIC_SCRATCH_BYTES)
+    return KF_ERR_WORKSPACE;
+  void* scratch = static_scratch_address();
+  if (scratch == nullptr) return KF_ERR_CUDA;
+  // Nothing in the scratch has to start at zero: the first pass writes every (row, tile) entry
+  // the second pass reads, so whatever an earlier call left behind is never observed.
+  return kf_gemm_rowreduce(M, N, K, in_dtype, X, ldx, W, ldw, bias, pre_act, red, out, ldo,
+                           out_dtype, scratch, KF_STATIC_SCRATCH_BYTES, cuda_stream);
+}

@@ -297,6 +297,43 @@ def chain_table(kf, device, peaks, c2_tensors, c2_us):
     return out
 
 
+def run_single_workload(args, kf, device, peaks):
+    """--workload cN: time one chain alone (used for profiling); prints a reduced JSON line."""
+    import torch
+    name = args.workload
+    specs = {
+        "c1": (2.0 * 128 * 256 * 512, 4 * (128 * 512 + 256 * 512 + 256 + 128 * 256)),
+        "c3": (2.0 * 4096 * 8192 * 2048, 2 * (4096 * 2048 + 8192 * 2048 + 8192 + 4096 * 8192)),
+        "c4": (2.0 * 16384 * 1024 * 1024, 2 * (16384 * 1024 + 1024 * 1024 + 1024) + 4 * 16384),
+        "c5": (2.0 * 128 * 64 * 64 * 128 * 576, 2 * (128 * 64 * 64 * 64 + 128 * 64 * 9 + 128 + 128 * 128 * 64 * 64)),
+    }
+    flops, nbytes = specs[name]
+    if name == "c5":
+        d = ki.conv_inputs("c5", seed=0)
+        t = {k: to_dev(d[k], device) for k in ("x", "w", "bias")}
+        o = torch.empty(128, 128, 64, 64, dtype=torch.bfloat16, device=device)
+        fn = lambda: kf.conv3x3_epilogue(t["x"], t["w"], t["bias"], "relu", 32, 1e-5, out=o)
+    else:
+        d = ki.gemm_inputs(name, seed=0)
+        t = {k: to_dev(d[k], device) for k in ("X", "W", "b")}
+        if name == "c1":
+            fn = lambda: kf.gemm_epilogue(t["X"], t["W"], t["b"], "relu")
+        elif name == "c3":
+            o = torch.empty(4096, 8192, dtype=torch.bfloat16, device=device)
+            fn = lambda: kf.gemm_rowreduce(t["X"], t["W"], t["b"], "none", "softmax", out=o)
+        else:
+            o = torch.empty(16384, dtype=torch.float32, device=device)
+            fn = lambda: kf.gemm_rowreduce(t["X"], t["W"], t["b"], "sigmoid", "sum", out=o)
+    l0 = kf.kf_launch_count()
+    us = time_calls(fn, args.steps, max(3, args.warmup), graph_batch=0)
+    tf = flops / us / 1e6
+    print(json.dumps({"metric": "fused_chain_tflops", "value": round(tf, 3), "unit": "TFLOP/s",
+                      "us_per_call": round(us, 3), "steps": args.steps, "warmup": max(3, args.warmup),
+                      "algorithmic_gbs": round(nbytes / us / 1e3, 1),
+                      "gpu_launches": int(kf.kf_launch_count() - l0),
+                      "config": {"workload": name}, "data": "synthetic"}))
+
+
 # ------------------------------------------------------------------ main
 def main():
     ap = argparse.ArgumentParser()
@@ -305,6 +342,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the context table and baselines")
+    ap.add_argument("--workload", default=WORKLOAD, choices=["c1", "c2", "c3", "c4", "c5"],
+                    help="c2 is the headline; the others print a reduced line (profiling aid)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -328,6 +367,10 @@ def main():
     import paper_2605_30359_b200 as kf   # raises if libkf.so is missing
     kf.lib()
     peaks = load_peaks()
+    if args.workload != WORKLOAD:
+        if rank == 0:
+            run_single_workload(args, kf, device, peaks)
+        return
 
     # inputs: rank r works on its own batch (seed r); resident in HBM before the timed region
     d = ki.gemm_inputs(WORKLOAD, seed=rank)

@@ -131,9 +131,9 @@ kf_status kf_gemm_rowreduce_static(int64_t M, int64_t N, int64_t K, kf_dtype in_
  *   groups == 0: y = a.
  * x is NCHW [Nb,Cin,H,Wd], w is OIHW [Cout,Cin,3,3], y is NCHW [Nb,Cout,H,Wd], all dense, of
  * io_dtype.  bias, gamma, beta may be NULL (0, 1, 0).  y must not alias x.
- * bf16 problems with Cin % 64 == 0, Cout % 16 == 0, Cout <= 256, Wd in {8,16,32,64,128} and
- * (H*Wd) % 128 == 0 take the implicit-GEMM tensor-core kernel; everything else takes a
- * scalar kernel.  groups must divide Cout. */
+ * bf16 problems with Cin % 64 == 0, Wd in {8,16,32,64,128}, (H*Wd) % 128 == 0 and a 16-byte
+ * aligned x take the implicit-GEMM tensor-core kernel; everything else takes a scalar kernel.
+ * groups must divide Cout. */
 kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
                               kf_dtype io_dtype, const void* x, const void* w, const void* bias,
                               kf_act act, int groups, float eps, const void* gamma,

@@ -23,7 +23,7 @@ LIB = os.path.join(PKG, "libkf.so")
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"),
-]
+] + os.environ.get("KF_NVCC_EXTRA", "").split()
 
 
 def _nvcc() -> str:

@@ -62,18 +62,23 @@ inline bool valid_dtype(int dt) { return dt == DT_F32 || dt == DT_BF16; }
 inline bool valid_act(int a) { return a >= 0 && a < ACT_COUNT; }
 constexpr int64_t kMaxDim = 2147483647ll;
 
-// bf16 row-major [rows, cols] with leading dimension ld -> tiles of box_rows x 64 columns,
-// 128-byte swizzle, zero fill outside the tensor.
+// bf16 row-major [rows, cols] with leading dimension ld -> boxes of box_rows x box_cols,
+// zero fill outside the tensor on loads, clipping on stores.  Operand tiles use 64 columns with
+// the 128-byte swizzle; epilogue pieces use 32 columns with the 64-byte swizzle.
 bool encode_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld,
-               int box_rows) {
+               int box_rows, int box_cols = kBK,
+               CUtensorMapSwizzle swz = CU_TENSOR_MAP_SWIZZLE_128B) {
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
   const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBK), static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
   const cuuint32_t estr[2] = {1, 1};
   return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides,
-                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
          CUDA_SUCCESS;
+}
+bool encode_piece(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld) {
+  return encode_2d(tm, base, rows, cols, ld, kBM, kPieceCols, CU_TENSOR_MAP_SWIZZLE_64B);
 }
 
 // NHWC bf16 activations [Nb,H,W,C] -> boxes of 64 channels x W pixels x rows image rows.
@@ -93,6 +98,21 @@ bool encode_nhwc(CUtensorMap* tm, const void* base, int64_t Nb, int64_t H, int64
          CUDA_SUCCESS;
 }
 
+// NCHW bf16 output seen as [Nb][C][H*W] -> store boxes of 32 pixels x 128 channels of one image
+// (64-byte swizzle like every epilogue piece); channels past C are clipped.
+bool encode_nchw_out(CUtensorMap* tm, const void* base, int64_t Nb, int64_t C, int64_t hw) {
+  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(hw), static_cast<cuuint64_t>(C),
+                              static_cast<cuuint64_t>(Nb)};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(hw) * 2,
+                                 static_cast<cuuint64_t>(C) * hw * 2};
+  const cuuint32_t box[3] = {static_cast<cuuint32_t>(kPieceCols), static_cast<cuuint32_t>(kBM), 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides,
+                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+         CUDA_SUCCESS;
+}
+
 // Can the tensor-core GEMM take these operands?  (TMA: 16-byte aligned base and row pitch.)
 bool umma_gemm_ok(int dt, int64_t K, const void* X, int64_t ldx, const void* W, int64_t ldw) {
   return dt == DT_BF16 && K % 8 == 0 && ldx % 8 == 0 && ldw % 8 == 0 && aligned(X, 16) &&
@@ -100,9 +120,14 @@ bool umma_gemm_ok(int dt, int64_t K, const void* X, int64_t ldx, const void* W, 
 }
 
 bool conv_umma_shape_ok(int dt, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout) {
+  (void)Cout;
   const bool w_ok = Wd == 8 || Wd == 16 || Wd == 32 || Wd == 64 || Wd == 128;
-  return dt == DT_BF16 && Cin % 64 == 0 && Cout % 16 == 0 && Cout <= 256 && w_ok &&
-         (H * Wd) % 128 == 0;
+  return dt == DT_BF16 && Cin % 64 == 0 && w_ok && (H * Wd) % 128 == 0;
+}
+// pixels per tile: 256 when whole tiles of 256 pixels cover the image, else 128
+int conv_tile_pixels(int64_t H, int64_t Wd) { return (H * Wd) % 256 == 0 ? 256 : 128; }
+size_t conv_stats_bytes(int64_t Nb, int64_t H, int64_t Wd, int64_t Cout) {
+  return round256(static_cast<size_t>(Nb) * ((H * Wd) / conv_tile_pixels(H, Wd)) * Cout * 8);
 }
 
 kf_status check_gemm_common(int64_t M, int64_t N, int64_t K, int dt, const void* X, int64_t ldx,
@@ -176,7 +201,7 @@ size_t kf_conv3x3_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd
   if (Nb < 1 || Cin < 1 || H < 1 || Wd < 1 || Cout < 1) return 0;
   if (!conv_umma_shape_ok(io_dtype, Cin, H, Wd, Cout)) return 0;
   return round256(static_cast<size_t>(Nb) * H * Wd * Cin * 2) +
-         round256(static_cast<size_t>(9) * Cout * Cin * 2);
+         round256(static_cast<size_t>(9) * Cout * Cin * 2) + conv_stats_bytes(Nb, H, Wd, Cout);
 }
 
 kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, const void* X,
@@ -198,8 +223,8 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
 
   if (umma_gemm_ok(io_dtype, K, X, ldx, W, ldw)) {
     const int bn = N <= 128 ? 128 : 256;
-    CUtensorMap ta, tb;
-    if (!encode_2d(&ta, X, M, K, ldx, kBM) || !encode_2d(&tb, W, N, K, ldw, bn)) return KF_ERR_CUDA;
+    UmmaMaps tm;
+    if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, bn)) return KF_ERR_CUDA;
     UmmaParams p;
     std::memset(&p, 0, sizeof(p));
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
@@ -213,9 +238,17 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
     p.ldr = ldr; p.out = Y; p.ldo = ldy; p.scale = scale;
     p.vec_ok = (ldy % 8 == 0 && aligned(Y, 16) &&
                 (residual == nullptr || (ldr % 8 == 0 && aligned(residual, 16)))) ? 1 : 0;
+    p.bias_vec = aligned(bias, 16) ? 1 : 0;
+    // aligned output (and residual): epilogue pieces travel by TMA through shared memory
+    p.staged = p.vec_ok;
+    tm.r = tm.a; tm.y = tm.a;
+    if (p.staged) {
+      if (!encode_piece(&tm.y, Y, M, N, ldy)) return KF_ERR_CUDA;
+      if (residual != nullptr && !encode_piece(&tm.r, residual, M, N, ldr)) return KF_ERR_CUDA;
+    }
     p.status = d->status;
     const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
-    if (launch_umma_elementwise(bn, act, ta, tb, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
+    if (launch_umma_elementwise(bn, act, tm, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
     g_launches += 1;
     return KF_OK;
   }
@@ -249,9 +282,10 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
   if (umma_gemm_ok(in_dtype, K, X, ldx, W, ldw) && tiles_n64 <= 8192) {
     vs = check_workspace(workspace, workspace_bytes, rowreduce_umma_ws(M, N, red));
     if (vs != KF_OK) return vs;
-    CUtensorMap ta, tb;
-    if (!encode_2d(&ta, X, M, K, ldx, kBM) || !encode_2d(&tb, W, N, K, ldw, kRowReduceBN))
+    UmmaMaps tm;
+    if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, kRowReduceBN))
       return KF_ERR_CUDA;
+    tm.r = tm.a; tm.y = tm.a;
     UmmaParams p;
     std::memset(&p, 0, sizeof(p));
     p.M = Mi; p.N = Ni; p.K = Ki;
@@ -264,15 +298,18 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
     p.out = out; p.ldo = ldo; p.scale = 1.0f;
     p.partial = static_cast<float*>(workspace);
     p.vec_ok = (red == KF_RED_SOFTMAX && (ldo * esize(out_dtype)) % 16 == 0 && aligned(out, 16)) ? 1 : 0;
+    p.bias_vec = aligned(bias, 16) ? 1 : 0;
+    p.staged = (p.vec_ok && out_dtype == KF_BF16) ? 1 : 0;
+    if (p.staged && !encode_piece(&tm.y, out, M, N, ldo)) return KF_ERR_CUDA;
     p.status = d->status;
     const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
     if (red == KF_RED_SOFTMAX) {
-      if (launch_umma_softmax(pre_act, out_dtype, ta, tb, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
+      if (launch_umma_softmax(pre_act, out_dtype, tm, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
       if (launch_softmax_finalize(out_dtype, Mi, Ni, p.tiles_n, p.partial, out, ldo, p.vec_ok, st) !=
           cudaSuccess)
         return KF_ERR_CUDA;
     } else {
-      if (launch_umma_rowsum(pre_act, ta, tb, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
+      if (launch_umma_rowsum(pre_act, tm, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
       if (launch_rowsum_finalize(Mi, p.tiles_n, p.partial, static_cast<float*>(out), st) != cudaSuccess)
         return KF_ERR_CUDA;
     }
@@ -318,47 +355,62 @@ kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
   if (conv_umma_shape_ok(io_dtype, Cin, H, Wd, Cout) && aligned(x, 16)) {
     const size_t xt_bytes = round256(static_cast<size_t>(Nb) * hw * Cin * 2);
     const size_t wr_bytes = round256(static_cast<size_t>(9) * Cout * Cin * 2);
-    kf_status vs = check_workspace(workspace, workspace_bytes, xt_bytes + wr_bytes);
+    const size_t st_bytes = conv_stats_bytes(Nb, H, Wd, Cout);
+    kf_status vs = check_workspace(workspace, workspace_bytes, xt_bytes + wr_bytes + st_bytes);
     if (vs != KF_OK) return vs;
     void* xt = workspace;
     void* wr = static_cast<uint8_t*>(workspace) + xt_bytes;
+    float* stats = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + xt_bytes + wr_bytes);
     if (launch_conv_prep(static_cast<int>(Nb), static_cast<int>(Cin), static_cast<int>(H),
                          static_cast<int>(Wd), static_cast<int>(Cout), x, w, xt, wr, st) != cudaSuccess)
       return KF_ERR_CUDA;
     ++launches;
-    const int bn = Cout <= 64 ? 64 : (Cout <= 128 ? 128 : 256);
-    const int rows = static_cast<int>(kBM / Wd);
-    CUtensorMap ta, tb;
-    if (!encode_nhwc(&ta, xt, Nb, H, Wd, Cin, rows) || !encode_2d(&tb, wr, 9 * Cout, Cin, Cin, bn))
+    const int bn = conv_tile_pixels(H, Wd);            // pixels per tile = UMMA N
+    const int rows = static_cast<int>(bn / Wd);        // image rows per tile
+    UmmaMaps tm;
+    // A: weights [9*Cout, Cin], 128 output channels per tile; B: NHWC activations
+    if (!encode_2d(&tm.a, wr, 9 * Cout, Cin, Cin, kBM) || !encode_nhwc(&tm.b, xt, Nb, H, Wd, Cin, rows))
       return KF_ERR_CUDA;
+    tm.r = tm.a; tm.y = tm.a;
     UmmaParams p;
     std::memset(&p, 0, sizeof(p));
     p.M = static_cast<int>(Nb * hw); p.N = static_cast<int>(Cout); p.K = static_cast<int>(9 * Cin);
-    p.tiles_per_image = static_cast<int>(hw / kBM);
-    p.tiles_m = static_cast<int>(Nb) * p.tiles_per_image; p.tiles_n = 1;
-    p.num_tiles = p.tiles_m;
+    p.tiles_per_image = static_cast<int>(hw / bn);
+    p.tiles_m = static_cast<int>((Cout + kBM - 1) / kBM);              // output-channel tiles
+    p.tiles_n = static_cast<int>(Nb) * p.tiles_per_image;              // pixel tiles
+    if (static_cast<int64_t>(p.tiles_m) * p.tiles_n > kMaxDim) return KF_ERR_UNSUPPORTED;
+    p.num_tiles = p.tiles_m * p.tiles_n;
     p.kb_per_tap = static_cast<int>(Cin / kBK);
     p.k_blocks = 9 * p.kb_per_tap;
     p.bias = static_cast<const __nv_bfloat16*>(bias);
     p.out = y; p.scale = 1.0f;
+    p.partial = groups > 0 ? stats : nullptr;
     p.status = d->status;
     p.H = static_cast<int>(H); p.Wd = static_cast<int>(Wd); p.Cin = static_cast<int>(Cin);
     p.rows_per_tile = rows;
+    p.staged = aligned(y, 16) ? 1 : 0;
+    if (p.staged && !encode_nchw_out(&tm.y, y, Nb, Cout, hw)) return KF_ERR_CUDA;
     const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
-    if (launch_umma_conv(bn, act, ta, tb, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
+    if (launch_umma_conv(bn, act, tm, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
     ++launches;
+    if (groups > 0) {
+      if (launch_groupnorm_apply(static_cast<int>(Nb), static_cast<int>(Cout), groups, hw,
+                                 p.tiles_per_image, eps, stats, gamma, beta, y, st) != cudaSuccess)
+        return KF_ERR_CUDA;
+      ++launches;
+    }
   } else {
     if (launch_conv_direct(io_dtype, act, static_cast<int>(Nb), static_cast<int>(Cin),
                            static_cast<int>(H), static_cast<int>(Wd), static_cast<int>(Cout), x, w,
                            bias, y, st) != cudaSuccess)
       return KF_ERR_CUDA;
     ++launches;
-  }
-  if (groups > 0) {
-    if (launch_groupnorm(io_dtype, static_cast<int>(Nb), static_cast<int>(Cout), groups, hw, eps,
-                         gamma, beta, y, st) != cudaSuccess)
-      return KF_ERR_CUDA;
-    ++launches;
+    if (groups > 0) {
+      if (launch_groupnorm(io_dtype, static_cast<int>(Nb), static_cast<int>(Cout), groups, hw, eps,
+                           gamma, beta, y, st) != cudaSuccess)
+        return KF_ERR_CUDA;
+      ++launches;
+    }
   }
   g_launches += launches;
   return KF_OK;

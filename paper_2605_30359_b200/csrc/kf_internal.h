@@ -10,15 +10,21 @@
 
 namespace kf {
 
+// The four tensor maps of one tensor-core launch: A and B operands, residual in, output out
+// (unused ones are copies of a valid map; the kernel never touches them).
+struct UmmaMaps {
+  CUtensorMap a, b, r, y;
+};
+
 // tensor-core chains (bf16)
-cudaError_t launch_umma_elementwise(int bn, int act, const CUtensorMap& a, const CUtensorMap& b,
-                                    const UmmaParams& p, int grid, cudaStream_t st);
-cudaError_t launch_umma_softmax(int act, int out_dt, const CUtensorMap& a, const CUtensorMap& b,
-                                const UmmaParams& p, int grid, cudaStream_t st);
-cudaError_t launch_umma_rowsum(int act, const CUtensorMap& a, const CUtensorMap& b,
-                               const UmmaParams& p, int grid, cudaStream_t st);
-cudaError_t launch_umma_conv(int bn, int act, const CUtensorMap& a, const CUtensorMap& b,
-                             const UmmaParams& p, int grid, cudaStream_t st);
+cudaError_t launch_umma_elementwise(int bn, int act, const UmmaMaps& tm, const UmmaParams& p,
+                                    int grid, cudaStream_t st);
+cudaError_t launch_umma_softmax(int act, int out_dt, const UmmaMaps& tm, const UmmaParams& p,
+                                int grid, cudaStream_t st);
+cudaError_t launch_umma_rowsum(int act, const UmmaMaps& tm, const UmmaParams& p, int grid,
+                               cudaStream_t st);
+cudaError_t launch_umma_conv(int bn, int act, const UmmaMaps& tm, const UmmaParams& p, int grid,
+                             cudaStream_t st);
 constexpr int kRowReduceBN = 256;   // tile width of the row-reduce first pass
 
 // second passes of the tensor-core row reductions
@@ -45,16 +51,22 @@ cudaError_t launch_conv_direct(int dt, int act, int Nb, int Cin, int H, int Wd, 
                                cudaStream_t st);
 cudaError_t launch_groupnorm(int dt, int Nb, int Cout, int groups, long long hw, float eps,
                              const void* gamma, const void* beta, void* y, cudaStream_t st);
+// GroupNorm from the per-tile channel statistics the convolution epilogue wrote (bf16 only)
+cudaError_t launch_groupnorm_apply(int Nb, int Cout, int groups, long long hw, int tiles_per_image,
+                                   float eps, const float* stats, const void* gamma,
+                                   const void* beta, void* y, cudaStream_t st);
 
 // Generic launcher for one instantiation of the tensor-core kernel.
 template <int BN, int EPI, int ACT, typename OutT>
-inline cudaError_t launch_umma_instance(const CUtensorMap& a, const CUtensorMap& b,
-                                        const UmmaParams& p, int grid, cudaStream_t st) {
+inline cudaError_t launch_umma_instance(const UmmaMaps& tm, const UmmaParams& p, int grid,
+                                        cudaStream_t st) {
+  using C = UmmaCfg<BN, EPI>;
+  constexpr int smem = C::kTotal;
+  static_assert(smem <= kMaxDynSmem, "shared-memory plan exceeds the per-CTA limit");
   auto kern = umma_chain_kernel<BN, EPI, ACT, OutT>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       UmmaSmem<BN>::kTotal);
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  kern<<<grid, kNumThreads, UmmaSmem<BN>::kTotal, st>>>(a, b, p);
+  kern<<<grid, kNumThreads, smem, st>>>(tm.a, tm.b, tm.r, tm.y, p);
   return cudaGetLastError();
 }
 

@@ -116,4 +116,15 @@ cudaError_t launch_groupnorm(int dt, int Nb, int Cout, int groups, long long hw,
   return cudaGetLastError();
 }
 
+cudaError_t launch_groupnorm_apply(int Nb, int Cout, int groups, long long hw, int tiles_per_image,
+                                   float eps, const float* stats, const void* gamma,
+                                   const void* beta, void* y, cudaStream_t st) {
+  const unsigned grid = static_cast<unsigned>(Nb) * static_cast<unsigned>(groups);
+  groupnorm_apply_kernel<<<grid, 512, 0, st>>>(
+      Cout, groups, hw, tiles_per_image, eps, reinterpret_cast<const float2*>(stats),
+      static_cast<const __nv_bfloat16*>(gamma), static_cast<const __nv_bfloat16*>(beta),
+      static_cast<__nv_bfloat16*>(y));
+  return cudaGetLastError();
+}
+
 }  // namespace kf

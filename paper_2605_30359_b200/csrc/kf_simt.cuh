@@ -118,7 +118,7 @@ row_sum_kernel(int N, const float* __restrict__ A, long long lda, float* out) {
 
 // ---------------------------------------------------------------- second passes, tensor path
 // Softmax: the first pass left e[m,n] = exp(a[m,n] - mx_t) in `out` and (mx_t, sum_t) per
-// 256-column tile t in `partial`.  Row maximum mx = max_t mx_t, denominator
+// BN-column slice t (half an MMA tile) in `partial`.  Row maximum mx = max_t mx_t, denominator
 // S = sum_t sum_t*exp(mx_t - mx); the output is e * exp(mx_t - mx) / S, in place.
 template <typename OutT, int BN>
 __global__ void __launch_bounds__(256)
@@ -346,6 +346,57 @@ groupnorm_kernel(int Cout, int groups, long long hw, float eps, const T* __restr
       const float ga = gamma != nullptr ? to_f32(gamma[o]) : 1.0f;
       const float be = beta != nullptr ? to_f32(beta[o]) : 0.0f;
       blk[i] = from_f32<T>((to_f32(blk[i]) - mu) * rstd * ga + be);
+    }
+  }
+}
+
+// ---------------------------------------------------------------- GroupNorm from tile statistics
+// The convolution epilogue left, per pixel tile t and channel c, stats[t][c] = (sum, sum of
+// squares) of the stored activations.  One CTA per (image, group): add the group's entries in a
+// fixed order, mean = S1/cnt, var = S2/cnt - mean^2 (biased), then normalise the group's
+// contiguous NCHW block in place: one read and one write of the activations.
+__global__ void __launch_bounds__(512)
+groupnorm_apply_kernel(int Cout, int groups, long long hw, int tiles_per_image, float eps,
+                       const float2* __restrict__ stats, const __nv_bfloat16* __restrict__ gamma,
+                       const __nv_bfloat16* __restrict__ beta, __nv_bfloat16* y) {
+  __shared__ float scratch[32];
+  const int cpg = Cout / groups;
+  const long long cnt = static_cast<long long>(cpg) * hw;
+  const int g = blockIdx.x % groups;
+  const long long n = blockIdx.x / groups;
+  float s1 = 0.0f, s2 = 0.0f;
+  for (int i = threadIdx.x; i < tiles_per_image * cpg; i += blockDim.x) {
+    const int t = i / cpg, c = g * cpg + i % cpg;
+    const float2 v = stats[(n * tiles_per_image + t) * Cout + c];
+    s1 += v.x;
+    s2 += v.y;
+  }
+  s1 = block_reduce<false>(s1, scratch);
+  s2 = block_reduce<false>(s2, scratch);
+  const float mu = s1 / static_cast<float>(cnt);
+  const float var = fmaxf(s2 / static_cast<float>(cnt) - mu * mu, 0.0f);
+  const float rstd = rsqrtf(var + eps);
+  __nv_bfloat16* blk = y + (n * Cout + static_cast<long long>(g) * cpg) * hw;
+  if ((hw % 8) == 0 && (reinterpret_cast<uintptr_t>(blk) & 15u) == 0) {
+    uint4* bv = reinterpret_cast<uint4*>(blk);
+    for (long long i = threadIdx.x; i < cnt / 8; i += blockDim.x) {
+      const int o = g * cpg + static_cast<int>((i * 8) / hw);
+      const float ga = gamma != nullptr ? to_f32(gamma[o]) : 1.0f;
+      const float be = beta != nullptr ? to_f32(beta[o]) : 0.0f;
+      const float a = rstd * ga, b = fmaf(-mu, rstd * ga, be);
+      uint4 w = bv[i];
+      w.x = pack_bf16x2(fmaf(bf16_lo(w.x), a, b), fmaf(bf16_hi(w.x), a, b));
+      w.y = pack_bf16x2(fmaf(bf16_lo(w.y), a, b), fmaf(bf16_hi(w.y), a, b));
+      w.z = pack_bf16x2(fmaf(bf16_lo(w.z), a, b), fmaf(bf16_hi(w.z), a, b));
+      w.w = pack_bf16x2(fmaf(bf16_lo(w.w), a, b), fmaf(bf16_hi(w.w), a, b));
+      bv[i] = w;
+    }
+  } else {
+    for (long long i = threadIdx.x; i < cnt; i += blockDim.x) {
+      const int o = g * cpg + static_cast<int>(i / hw);
+      const float ga = gamma != nullptr ? to_f32(gamma[o]) : 1.0f;
+      const float be = beta != nullptr ? to_f32(beta[o]) : 0.0f;
+      blk[i] = __float2bfloat16_rn((to_f32(blk[i]) - mu) * rstd * ga + be);
     }
   }
 }

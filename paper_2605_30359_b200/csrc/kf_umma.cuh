@@ -2,13 +2,21 @@
 //
 // One persistent CTA per SM walks output tiles of 128 rows x BN columns.  Warp roles:
 //   warp 0 (one lane)  TMA producer: fills a ring of shared-memory stages (A 128x64, B BNx64
-//                      bf16, 128-byte swizzle) and signals `full[s]` by transaction bytes.
+//                      bf16, 128-byte swizzle) and signals `full[s]` by transaction bytes.  For
+//                      the convolution A is the weight tile of one tap (rows = output channels)
+//                      and B the shifted window of BN pixels, so that the accumulator comes out
+//                      channel-major like the NCHW output.
 //   warp 1 (one lane)  UMMA issuer: four tcgen05.mma (K=16 each) per stage into one of two
 //                      TMEM accumulators, tcgen05.commit to `empty[s]` (stage free) and, after
 //                      the last K block, to `tmem_full[a]`.
 //   warps 2..5         epilogue: tcgen05.ld the accumulator (thread = one row of the tile),
-//                      apply the chain's epilogue in fp32 registers, store, then release the
-//                      accumulator through `tmem_empty[a]` so the next tile's MMAs overlap.
+//                      apply the chain's epilogue in fp32 registers and release the accumulator
+//                      through `tmem_empty[a]` so the next tile's MMAs overlap.  Results leave
+//                      through shared-memory staging and TMA stores (the residual arrives the
+//                      same way, by TMA loads issued two pieces ahead): a row-per-lane global
+//                      access touches 32 cache lines per instruction and was measured to cost
+//                      the mainloop 10-15 % of its speed; a direct path remains for operands
+//                      whose alignment TMA cannot take.
 // Every wait is bounded (mbar_wait); a wait that runs out raises the CTA's abort flag, all
 // roles leave their loops, in-flight copies are given time to land, TMEM is freed.
 #pragma once
@@ -20,11 +28,14 @@ namespace kf {
 
 enum : int { EPI_ELEMENTWISE = 0, EPI_SOFTMAX = 1, EPI_ROWSUM = 2, EPI_CONV = 3 };
 
-constexpr int kBM = 128;         // tile rows = UMMA M = TMEM lanes
-constexpr int kBK = 64;          // K per stage: 64 bf16 = one 128-byte swizzled row
-constexpr int kUmmaK = 16;       // K per tcgen05.mma for 16-bit inputs
-constexpr int kNumThreads = 192; // 6 warps
-constexpr int kEpiThreads = 128; // warps 2..5
+constexpr int kBM = 128;          // tile rows = UMMA M = TMEM lanes
+constexpr int kBK = 64;           // K per stage: 64 bf16 = one 128-byte swizzled row
+constexpr int kUmmaK = 16;        // K per tcgen05.mma for 16-bit inputs
+constexpr int kEpiThreads = 128;  // warps 2..5
+constexpr int kNumThreads = 192;  // 6 warps
+constexpr int kPieceCols = 32;    // epilogue piece: 128 rows x 32 columns
+constexpr int kPieceBytes = kBM * kPieceCols * 2;   // 8 KB of bf16
+constexpr int kMaxDynSmem = 232448;                 // 227 KB opt-in limit per CTA
 
 struct UmmaParams {
   int M, N, K;                 // GEMM view (conv: M = Nb*H*W pixels, N = Cout, K = 9*Cin)
@@ -36,40 +47,77 @@ struct UmmaParams {
   long long ldo;
   float* partial;              // row-reduce partial statistics
   float scale;
-  int vec_ok;                  // rows of out (and R) are 16-byte aligned
+  int vec_ok;                  // rows of out (and R) are 16-byte aligned (direct path vectors)
+  int staged;                  // out (and R) go through shared memory and TMA
+  int bias_vec;                // bias is 16-byte aligned
   uint32_t* status;            // device status word
   // conv only
   int H, Wd, Cin, rows_per_tile, tiles_per_image, kb_per_tap;
 };
 
-template <int BN>
-struct UmmaSmem {
+template <int BN, int EPI>
+struct UmmaCfg {
   static constexpr int kStageA = kBM * kBK * 2;
   static constexpr int kStageB = BN * kBK * 2;
   static constexpr int kStage = kStageA + kStageB;
-  static constexpr int kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+  // staging: elementwise = 2 output + 2 residual pieces; softmax / conv = 2 output pieces
+  static constexpr int kStaging =
+      EPI == EPI_ELEMENTWISE ? 4 * kPieceBytes : (EPI == EPI_ROWSUM ? 0 : 2 * kPieceBytes);
+  static constexpr int kBarBytes = 256;
+  static constexpr int kFit = (kMaxDynSmem - 1024 - kStaging - kBarBytes) / kStage;
+  static constexpr int kStages = kFit > 8 ? 8 : kFit;
   static constexpr int kRing = kStage * kStages;
-  static constexpr int kBiasBytes = 2 * BN * 4;
-  static constexpr int kBarBytes = 8 * (2 * kStages + 4) + 16;
-  static constexpr int kTotal = 1024 /*alignment slack*/ + kRing + kBiasBytes + kBarBytes;
+  static constexpr int kTotal = 1024 /*alignment slack*/ + kRing + kStaging + kBarBytes;
 };
+
+// 32 consecutive bias values as fp32 (zeros past N or without a bias).  All lanes read the same
+// addresses, so each load is one broadcast transaction.
+__device__ __forceinline__ void load_bias32(const UmmaParams& p, int n0, float (&b)[32]) {
+  if (p.bias == nullptr) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) b[j] = 0.0f;
+  } else if (p.bias_vec && n0 + 32 <= p.N) {
+    const uint4* bp = reinterpret_cast<const uint4*>(p.bias + n0);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint4 w = __ldg(bp + q);
+      b[8 * q + 0] = bf16_lo(w.x); b[8 * q + 1] = bf16_hi(w.x);
+      b[8 * q + 2] = bf16_lo(w.y); b[8 * q + 3] = bf16_hi(w.y);
+      b[8 * q + 4] = bf16_lo(w.z); b[8 * q + 5] = bf16_hi(w.z);
+      b[8 * q + 6] = bf16_lo(w.w); b[8 * q + 7] = bf16_hi(w.w);
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      b[j] = (n0 + j < p.N) ? __bfloat162float(p.bias[n0 + j]) : 0.0f;
+  }
+}
+
+// Byte offset of 16-byte chunk j (0..3) of row r in a 128-row x 64-byte piece laid out the way
+// TMA's SWIZZLE_64B expects it (address bits 4..5 xor bits 7..8): conflict-free for a warp
+// whose lanes are consecutive rows.
+__device__ __forceinline__ uint32_t piece_off(int r, int j) {
+  return static_cast<uint32_t>(r * 64 + ((j ^ ((r >> 1) & 3)) << 4));
+}
 
 template <int BN, int EPI, int ACT, typename OutT>
 __global__ void __launch_bounds__(kNumThreads, 1)
 umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmY,
                   const UmmaParams p) {
-  using S = UmmaSmem<BN>;
-  constexpr int kStages = S::kStages;
+  using C = UmmaCfg<BN, EPI>;
+  constexpr int kStages = C::kStages;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
   uint8_t* ring = smem;
-  float* sbias = reinterpret_cast<float*>(smem + S::kRing);              // [2][BN]
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + S::kRing + S::kBiasBytes);
+  uint8_t* stg = smem + C::kRing;                                    // epilogue staging
+  uint64_t* full = reinterpret_cast<uint64_t*>(stg + C::kStaging);
   uint64_t* empty = full + kStages;
   uint64_t* tmem_full = empty + kStages;
   uint64_t* tmem_empty = tmem_full + 2;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+  uint64_t* r_full = tmem_empty + 2;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(r_full + 2);
   volatile uint32_t* abort_flag = tmem_holder + 1;
 
   const int warp = threadIdx.x >> 5;
@@ -77,7 +125,11 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], kEpiThreads); }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&tmem_full[a], 1);
+      mbar_init(&tmem_empty[a], kEpiThreads / 32);
+      mbar_init(&r_full[a], 1);
+    }
     *abort_flag = 0;
     mbar_init_fence();
     tma_prefetch_desc(&tmA);
@@ -99,9 +151,9 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
         int tm, tn, img = 0, h0 = 0;
         if constexpr (EPI == EPI_CONV) {
-          tm = tile; tn = 0;
-          img = tile / p.tiles_per_image;
-          h0 = (tile % p.tiles_per_image) * p.rows_per_tile;
+          tm = tile % p.tiles_m; tn = tile / p.tiles_m;        // output-channel tile, pixel tile
+          img = tn / p.tiles_per_image;
+          h0 = (tn % p.tiles_per_image) * p.rows_per_tile;
         } else {
           tm = tile / p.tiles_n; tn = tile % p.tiles_n;
         }
@@ -109,15 +161,16 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           ok = mbar_wait(&empty[s], ph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_PRODUCER);
           if (!ok) break;
-          uint8_t* sa = ring + s * S::kStage;
-          uint8_t* sb = sa + S::kStageA;
-          mbar_expect_tx(&full[s], S::kStage);
+          uint8_t* sa = ring + s * C::kStage;
+          uint8_t* sb = sa + C::kStageA;
+          mbar_expect_tx(&full[s], C::kStage);
           if constexpr (EPI == EPI_CONV) {
             const int tap = kb / p.kb_per_tap, cb = kb % p.kb_per_tap;
             const int r = tap / 3, sx = tap % 3;
-            // A: 128 pixels x 64 channels of the shifted window; out-of-image taps read zeros.
-            tma_load_4d(sa, &tmA, &full[s], cb * kBK, sx - 1, h0 + r - 1, img);
-            tma_load_2d(sb, &tmB, &full[s], cb * kBK, tap * p.N);
+            // A: this tap's weights for 128 output channels.  B: BN pixels x 64 input channels
+            // of the window shifted by the tap; out-of-image pixels read zeros (the padding).
+            tma_load_2d(sa, &tmA, &full[s], cb * kBK, tap * p.N + tm * kBM);
+            tma_load_4d(sb, &tmB, &full[s], cb * kBK, sx - 1, h0 + r - 1, img);
           } else {
             tma_load_2d(sa, &tmA, &full[s], kb * kBK, tm * kBM);
             tma_load_2d(sb, &tmB, &full[s], kb * kBK, tn * BN);
@@ -133,8 +186,9 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16_f32(kBM, BN);
       int s = 0; uint32_t ph = 0; int a = 0; uint32_t aph = 0;
-      for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
-        bool ok = mbar_wait(&tmem_empty[a], aph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+        ok = mbar_wait(&tmem_empty[a], aph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(a * BN);
@@ -142,9 +196,9 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           ok = mbar_wait(&full[s], ph, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t sa = smem_u32(ring + s * S::kStage);
+          const uint32_t sa = smem_u32(ring + s * C::kStage);
           const uint64_t adesc = smem_desc_kmajor_sw128(sa);
-          const uint64_t bdesc = smem_desc_kmajor_sw128(sa + S::kStageA);
+          const uint64_t bdesc = smem_desc_kmajor_sw128(sa + C::kStageA);
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
             // +32 bytes per K step inside the 128-byte swizzled row = +2 in the address field
@@ -161,108 +215,224 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     __syncwarp();
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5)
+    constexpr int PIECES = BN / kPieceCols;
     const int quad = warp & 3;                 // TMEM lane quarter this warp may read
     const int row = quad * 32 + lane;          // row of the tile = TMEM lane
     const int et = threadIdx.x - 64;           // 0..127 among epilogue threads
+    const bool leader = et == 0;               // issues the epilogue's TMA loads and stores
     const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
-    int a = 0; uint32_t aph = 0;
-    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
-      int tm, tn;
-      if constexpr (EPI == EPI_CONV) { tm = tile; tn = 0; }
-      else { tm = tile / p.tiles_n; tn = tile % p.tiles_n; }
-      // stage this tile's bias slice as fp32 (zeros past N or without a bias)
-      float* sb = sbias + a * BN;
-      for (int j = et; j < BN; j += kEpiThreads) {
-        const int n = tn * BN + j;
-        sb[j] = (p.bias != nullptr && n < p.N) ? __bfloat162float(p.bias[n]) : 0.0f;
+    [[maybe_unused]] uint8_t* ybuf = stg;      // [2][kPieceBytes] output pieces
+    [[maybe_unused]] uint8_t* rbuf = stg + 2 * kPieceBytes;   // [2][kPieceBytes] residual pieces
+    const bool staged = p.staged != 0;
+    [[maybe_unused]] const bool has_r = EPI == EPI_ELEMENTWISE && p.R != nullptr;
+    const int my_tiles = (p.num_tiles - static_cast<int>(blockIdx.x) +
+                          static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+    [[maybe_unused]] const long long total_pieces = static_cast<long long>(my_tiles) * PIECES;
+    [[maybe_unused]] long long g = 0;          // running piece index of this CTA
+
+    // residual piece gi -> rbuf[gi & 1] (leader only)
+    [[maybe_unused]] auto issue_r = [&](long long gi) {
+      const int ti = static_cast<int>(gi / PIECES), c = static_cast<int>(gi % PIECES);
+      const int tile = blockIdx.x + ti * gridDim.x;
+      const int b = static_cast<int>(gi & 1);
+      mbar_expect_tx(&r_full[b], kPieceBytes);
+      tma_load_2d(rbuf + b * kPieceBytes, &tmR, &r_full[b],
+                  (tile % p.tiles_n) * BN + c * kPieceCols, (tile / p.tiles_n) * kBM);
+    };
+    if constexpr (EPI == EPI_ELEMENTWISE) {
+      if (staged && has_r && leader) {
+        if (total_pieces > 0) issue_r(0);
+        if (total_pieces > 1) issue_r(1);
       }
-      bool ok = mbar_wait(&tmem_full[a], aph, abort_flag, p.status, KF_DEV_TIMEOUT_EPILOGUE);
-      // one uniform go/no-go for all four epilogue warps; also publishes the bias slice
+    }
+
+    int a = 0; uint32_t aph = 0;
+    bool alive = true;
+    for (int tile = blockIdx.x; alive && tile < p.num_tiles; tile += gridDim.x) {
+      int tm, tn;
+      if constexpr (EPI == EPI_CONV) { tm = tile % p.tiles_m; tn = tile / p.tiles_m; }
+      else { tm = tile / p.tiles_n; tn = tile % p.tiles_n; }
+      const long long m = static_cast<long long>(tm) * kBM + row;
+      [[maybe_unused]] const bool row_ok = m < p.M;
+      [[maybe_unused]] const int n_tile = tn * BN;
+      [[maybe_unused]] const int n_valid = min(BN, p.N - n_tile);   // valid columns in this tile
+
+      // One thread polls the accumulator barrier; the rest block in hardware at the named
+      // barrier, which hands every epilogue warp the same go/no-go.
+      bool ok = true;
+      if (leader)
+        ok = mbar_wait(&tmem_full[a], aph, abort_flag, p.status, KF_DEV_TIMEOUT_EPILOGUE);
       ok = named_barrier_and(1, kEpiThreads, ok);
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t t_acc = tmem_base + static_cast<uint32_t>(a * BN) + lane_off;
-      const long long m = static_cast<long long>(tm) * kBM + row;
-      const bool row_ok = m < p.M;
-      const int n_tile = tn * BN;
-      const int n_valid = min(BN, p.N - n_tile);          // valid columns in this tile (>0)
+      // hand the accumulator back to the UMMA issuer (one arrival per warp)
+      auto release_acc = [&]() {
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tmem_empty[a]);
+      };
 
       if constexpr (EPI == EPI_ELEMENTWISE) {
         __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(p.out);
+        if (staged) {
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          if (c * 32 >= n_valid) break;
-          uint32_t v[32];
-          tmem_ld_32x32(t_acc + c * 32, v);
-          tmem_ld_wait();
-          float f[32];
+          for (int c = 0; c < PIECES; ++c, ++g) {
+            const int b = static_cast<int>(g & 1);
+            uint4 rv[4];
+            bool rok = true;
+            if (has_r) {
+              rok = mbar_wait(&r_full[b], static_cast<uint32_t>((g >> 1) & 1), abort_flag, p.status,
+                              KF_DEV_TIMEOUT_EPILOGUE);
+              const uint8_t* rb = rbuf + b * kPieceBytes;
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            f[j] = p.scale * act_f<ACT, true>(__uint_as_float(v[j]) + sb[c * 32 + j]);
-          if (row_ok) {
-            const int n0 = n_tile + c * 32;
-            if (p.vec_ok && c * 32 + 32 <= n_valid) {
-              if (p.R != nullptr) {
-                const uint4* rp = reinterpret_cast<const uint4*>(p.R + m * p.ldr + n0);
+              for (int q = 0; q < 4; ++q)
+                rv[q] = *reinterpret_cast<const uint4*>(rb + piece_off(row, q));
+            }
+            // ybuf[b] is free once the store issued two pieces ago has read it
+            if (leader) bulk_wait_group_read<1>();
+            rok = named_barrier_and(2, kEpiThreads, rok);   // all have consumed rbuf[b]
+            if (!rok) { alive = false; break; }
+            if (has_r && leader && g + 2 < total_pieces) issue_r(g + 2);
+            uint32_t v[32];
+            tmem_ld_32x32(t_acc + c * kPieceCols, v);
+            float bs[32];
+            load_bias32(p, n_tile + c * kPieceCols, bs);
+            tmem_ld_wait();
+            if (c == PIECES - 1) release_acc();
+            float f[32];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                  const uint4 r4 = __ldg(rp + q);
-                  f[8 * q + 0] += bf16_lo(r4.x); f[8 * q + 1] += bf16_hi(r4.x);
-                  f[8 * q + 2] += bf16_lo(r4.y); f[8 * q + 3] += bf16_hi(r4.y);
-                  f[8 * q + 4] += bf16_lo(r4.z); f[8 * q + 5] += bf16_hi(r4.z);
-                  f[8 * q + 6] += bf16_lo(r4.w); f[8 * q + 7] += bf16_hi(r4.w);
-                }
-              }
-              uint4* yp = reinterpret_cast<uint4*>(Y + m * p.ldo + n0);
+            for (int j = 0; j < 32; ++j)
+              f[j] = p.scale * act_f<ACT, true>(__uint_as_float(v[j]) + bs[j]);
+            if (has_r) {
 #pragma unroll
               for (int q = 0; q < 4; ++q) {
-                yp[q] = make_uint4(pack_bf16x2(f[8 * q + 0], f[8 * q + 1]),
-                                   pack_bf16x2(f[8 * q + 2], f[8 * q + 3]),
-                                   pack_bf16x2(f[8 * q + 4], f[8 * q + 5]),
-                                   pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
+                f[8 * q + 0] += bf16_lo(rv[q].x); f[8 * q + 1] += bf16_hi(rv[q].x);
+                f[8 * q + 2] += bf16_lo(rv[q].y); f[8 * q + 3] += bf16_hi(rv[q].y);
+                f[8 * q + 4] += bf16_lo(rv[q].z); f[8 * q + 5] += bf16_hi(rv[q].z);
+                f[8 * q + 6] += bf16_lo(rv[q].w); f[8 * q + 7] += bf16_hi(rv[q].w);
               }
-            } else {
+            }
+            uint8_t* yb = ybuf + b * kPieceBytes;
 #pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                if (c * 32 + j < n_valid) {
-                  float y = f[j];
-                  if (p.R != nullptr) y += __bfloat162float(p.R[m * p.ldr + n0 + j]);
-                  Y[m * p.ldo + n0 + j] = __float2bfloat16_rn(y);
+            for (int q = 0; q < 4; ++q)
+              *reinterpret_cast<uint4*>(yb + piece_off(row, q)) =
+                  make_uint4(pack_bf16x2(f[8 * q + 0], f[8 * q + 1]),
+                             pack_bf16x2(f[8 * q + 2], f[8 * q + 3]),
+                             pack_bf16x2(f[8 * q + 4], f[8 * q + 5]),
+                             pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
+            fence_proxy_async_smem();
+            named_barrier_sync(3, kEpiThreads);
+            if (leader) {
+              tma_store_2d(&tmY, yb, n_tile + c * kPieceCols, tm * kBM);   // clipped at M, N
+              bulk_commit_group();
+            }
+          }
+        } else {
+#pragma unroll 1
+          for (int c = 0; c < PIECES; ++c) {
+            if (c * 32 >= n_valid) break;
+            uint32_t v[32];
+            tmem_ld_32x32(t_acc + c * 32, v);
+            float bs[32];
+            load_bias32(p, n_tile + c * 32, bs);
+            tmem_ld_wait();
+            float f[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              f[j] = p.scale * act_f<ACT, true>(__uint_as_float(v[j]) + bs[j]);
+            if (row_ok) {
+              const int n0 = n_tile + c * 32;
+              if (p.vec_ok && c * 32 + 32 <= n_valid) {
+                if (p.R != nullptr) {
+                  const uint4* rp = reinterpret_cast<const uint4*>(p.R + m * p.ldr + n0);
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    const uint4 r4 = __ldg(rp + q);
+                    f[8 * q + 0] += bf16_lo(r4.x); f[8 * q + 1] += bf16_hi(r4.x);
+                    f[8 * q + 2] += bf16_lo(r4.y); f[8 * q + 3] += bf16_hi(r4.y);
+                    f[8 * q + 4] += bf16_lo(r4.z); f[8 * q + 5] += bf16_hi(r4.z);
+                    f[8 * q + 6] += bf16_lo(r4.w); f[8 * q + 7] += bf16_hi(r4.w);
+                  }
+                }
+                uint4* yp = reinterpret_cast<uint4*>(Y + m * p.ldo + n0);
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                  yp[q] = make_uint4(pack_bf16x2(f[8 * q + 0], f[8 * q + 1]),
+                                     pack_bf16x2(f[8 * q + 2], f[8 * q + 3]),
+                                     pack_bf16x2(f[8 * q + 4], f[8 * q + 5]),
+                                     pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                  if (c * 32 + j < n_valid) {
+                    float y = f[j];
+                    if (p.R != nullptr) y += __bfloat162float(p.R[m * p.ldr + n0 + j]);
+                    Y[m * p.ldo + n0 + j] = __float2bfloat16_rn(y);
+                  }
                 }
               }
             }
           }
+          release_acc();
         }
       } else if constexpr (EPI == EPI_SOFTMAX) {
         // pass 1: tile maximum of a = pre_act(z + b) over the valid columns of this row
         float mx = -INFINITY;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = 0; c < PIECES; ++c) {
           if (c * 32 >= n_valid) break;
           uint32_t v[32];
           tmem_ld_32x32(t_acc + c * 32, v);
+          float bs[32];
+          load_bias32(p, n_tile + c * 32, bs);
           tmem_ld_wait();
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + sb[c * 32 + j]);
+            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j]);
             if (c * 32 + j < n_valid) mx = fmaxf(mx, z);
           }
         }
-        // pass 2: numerators e = exp(a - mx), their fp32 sum, store e in the output dtype
+        // pass 2: numerators e = exp(a - mx), their fp32 sum, e stored in the output dtype
         OutT* P = reinterpret_cast<OutT*>(p.out);
         float sum = 0.0f;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          if (c * 32 >= n_valid) break;
+        for (int c = 0; c < PIECES; ++c, ++g) {
+          if (!staged && c * 32 >= n_valid) break;
           uint32_t v[32];
           tmem_ld_32x32(t_acc + c * 32, v);
+          float bs[32];
+          load_bias32(p, n_tile + c * 32, bs);
           tmem_ld_wait();
+          if (staged && c == PIECES - 1) release_acc();
           float f[32];
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + sb[c * 32 + j]);
+            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j]);
             f[j] = __expf(z - mx);
             if (c * 32 + j < n_valid) sum += f[j];
+          }
+          if constexpr (sizeof(OutT) == 2) {
+            if (staged) {
+              const int b = static_cast<int>(g & 1);
+              if (leader) bulk_wait_group_read<1>();
+              named_barrier_sync(2, kEpiThreads);
+              uint8_t* yb = ybuf + b * kPieceBytes;
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                *reinterpret_cast<uint4*>(yb + piece_off(row, q)) =
+                    make_uint4(pack_bf16x2(f[8 * q + 0], f[8 * q + 1]),
+                               pack_bf16x2(f[8 * q + 2], f[8 * q + 3]),
+                               pack_bf16x2(f[8 * q + 4], f[8 * q + 5]),
+                               pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
+              fence_proxy_async_smem();
+              named_barrier_sync(3, kEpiThreads);
+              if (leader) {
+                tma_store_2d(&tmY, yb, n_tile + c * kPieceCols, tm * kBM);
+                bulk_commit_group();
+              }
+              continue;
+            }
           }
           if (row_ok) {
             const int n0 = n_tile + c * 32;
@@ -288,6 +458,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
           }
         }
+        if (!staged) release_acc();
         if (row_ok) {
           float2* part = reinterpret_cast<float2*>(p.partial);
           part[m * p.tiles_n + tn] = make_float2(mx, sum);
@@ -295,48 +466,85 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       } else if constexpr (EPI == EPI_ROWSUM) {
         float sum = 0.0f;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = 0; c < PIECES; ++c) {
           if (c * 32 >= n_valid) break;
           uint32_t v[32];
           tmem_ld_32x32(t_acc + c * 32, v);
+          float bs[32];
+          load_bias32(p, n_tile + c * 32, bs);
           tmem_ld_wait();
           float part = 0.0f;
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + sb[c * 32 + j]);
+            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j]);
             if (c * 32 + j < n_valid) part += z;
           }
           sum += part;
         }
+        release_acc();
         if (row_ok) p.partial[m * p.tiles_n + tn] = sum;
-      } else {  // EPI_CONV: a = act(z + b) stored NCHW; thread = pixel, column = output channel
-        OutT* Yc = reinterpret_cast<OutT*>(p.out);
+      } else {
+        // EPI_CONV: rows = output channels, columns = BN consecutive pixels of one image, so a
+        // thread's 32-column chunk is 64 contiguous bytes of the NCHW output.  a = act(z + b) is
+        // rounded to bf16 and stored; the per-channel sum and sum of squares of the stored
+        // values over this tile go to `partial` for the GroupNorm that follows.
+        const int ch = tm * kBM + row;                      // output channel of this thread
+        const bool ch_ok = ch < p.N;
+        const int img = tn / p.tiles_per_image;
+        const int pt = tn % p.tiles_per_image;              // pixel tile inside the image
+        const float bias_v = (p.bias != nullptr && ch_ok) ? __bfloat162float(p.bias[ch]) : 0.0f;
         const long long hw = static_cast<long long>(p.H) * p.Wd;
-        const long long img = m / hw;
-        const long long pix = m - img * hw;
-        OutT* base = Yc + img * p.N * hw + pix;
+        float s1 = 0.0f, s2 = 0.0f;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          if (c * 32 >= n_valid) break;
+        for (int c = 0; c < PIECES; ++c, ++g) {
           uint32_t v[32];
           tmem_ld_32x32(t_acc + c * 32, v);
           tmem_ld_wait();
-          if (row_ok) {
+          if (c == PIECES - 1) release_acc();
+          uint32_t w[16];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              if (c * 32 + j < n_valid) {
-                const float y = act_f<ACT, true>(__uint_as_float(v[j]) + sb[c * 32 + j]);
-                base[static_cast<long long>(c * 32 + j) * hw] = from_f32<OutT>(y);
-              }
+          for (int j = 0; j < 16; ++j) {
+            const float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + bias_v);
+            const float y1 = act_f<ACT, true>(__uint_as_float(v[2 * j + 1]) + bias_v);
+            w[j] = pack_bf16x2(y0, y1);
+            const float r0 = bf16_lo(w[j]), r1 = bf16_hi(w[j]);
+            s1 += r0 + r1;
+            s2 = fmaf(r0, r0, fmaf(r1, r1, s2));
+          }
+          if (staged) {
+            const int b = static_cast<int>(g & 1);
+            if (leader) bulk_wait_group_read<1>();
+            named_barrier_sync(2, kEpiThreads);
+            uint8_t* yb = ybuf + b * kPieceBytes;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              *reinterpret_cast<uint4*>(yb + piece_off(row, q)) =
+                  make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+            fence_proxy_async_smem();
+            named_barrier_sync(3, kEpiThreads);
+            if (leader) {
+              // box = 32 pixels x 128 channels of image img; channels past Cout are clipped
+              tma_store_3d(&tmY, yb, pt * BN + c * 32, tm * kBM, img);
+              bulk_commit_group();
+            }
+          } else if (ch_ok) {
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) +
+                                 (static_cast<long long>(img) * p.N + ch) * hw + pt * BN + c * 32;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {       // the output may be only 2-byte aligned here
+              dst[2 * j] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j] & 0xFFFFu));
+              dst[2 * j + 1] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j] >> 16));
             }
           }
         }
+        if (p.partial != nullptr && ch_ok) {
+          float2* part = reinterpret_cast<float2*>(p.partial);
+          part[static_cast<long long>(tn) * p.N + ch] = make_float2(s1, s2);
+        }
       }
-      // accumulator drained: hand it back to the UMMA issuer
-      tc_fence_before_sync();
-      mbar_arrive(&tmem_empty[a]);
       if (++a == 2) { a = 0; aph ^= 1u; }
     }
+    if (leader) bulk_wait_group<0>();          // every output store has completed
   }
 
   // ---------------------------------------------------------------- teardown

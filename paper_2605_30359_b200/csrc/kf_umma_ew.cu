@@ -4,13 +4,13 @@
 
 namespace kf {
 
-cudaError_t launch_umma_elementwise(int bn, int act, const CUtensorMap& a, const CUtensorMap& b,
-                                    const UmmaParams& p, int grid, cudaStream_t st) {
+cudaError_t launch_umma_elementwise(int bn, int act, const UmmaMaps& tm, const UmmaParams& p,
+                                    int grid, cudaStream_t st) {
   cudaError_t e = cudaErrorInvalidValue;
   dispatch_act(act, [&](auto A) {
     constexpr int ACT = decltype(A)::value;
-    if (bn == 256) e = launch_umma_instance<256, EPI_ELEMENTWISE, ACT, __nv_bfloat16>(a, b, p, grid, st);
-    else if (bn == 128) e = launch_umma_instance<128, EPI_ELEMENTWISE, ACT, __nv_bfloat16>(a, b, p, grid, st);
+    if (bn == 256) e = launch_umma_instance<256, EPI_ELEMENTWISE, ACT, __nv_bfloat16>(tm, p, grid, st);
+    else if (bn == 128) e = launch_umma_instance<128, EPI_ELEMENTWISE, ACT, __nv_bfloat16>(tm, p, grid, st);
   });
   return e;
 }

@@ -4,23 +4,23 @@
 
 namespace kf {
 
-cudaError_t launch_umma_softmax(int act, int out_dt, const CUtensorMap& a, const CUtensorMap& b,
-                                const UmmaParams& p, int grid, cudaStream_t st) {
+cudaError_t launch_umma_softmax(int act, int out_dt, const UmmaMaps& tm, const UmmaParams& p,
+                                int grid, cudaStream_t st) {
   cudaError_t e = cudaErrorInvalidValue;
   dispatch_act(act, [&](auto A) {
     constexpr int ACT = decltype(A)::value;
-    if (out_dt == DT_BF16) e = launch_umma_instance<kRowReduceBN, EPI_SOFTMAX, ACT, __nv_bfloat16>(a, b, p, grid, st);
-    else e = launch_umma_instance<kRowReduceBN, EPI_SOFTMAX, ACT, float>(a, b, p, grid, st);
+    if (out_dt == DT_BF16) e = launch_umma_instance<kRowReduceBN, EPI_SOFTMAX, ACT, __nv_bfloat16>(tm, p, grid, st);
+    else e = launch_umma_instance<kRowReduceBN, EPI_SOFTMAX, ACT, float>(tm, p, grid, st);
   });
   return e;
 }
 
-cudaError_t launch_umma_rowsum(int act, const CUtensorMap& a, const CUtensorMap& b,
-                               const UmmaParams& p, int grid, cudaStream_t st) {
+cudaError_t launch_umma_rowsum(int act, const UmmaMaps& tm, const UmmaParams& p, int grid,
+                               cudaStream_t st) {
   cudaError_t e = cudaErrorInvalidValue;
   dispatch_act(act, [&](auto A) {
     constexpr int ACT = decltype(A)::value;
-    e = launch_umma_instance<kRowReduceBN, EPI_ROWSUM, ACT, float>(a, b, p, grid, st);
+    e = launch_umma_instance<kRowReduceBN, EPI_ROWSUM, ACT, float>(tm, p, grid, st);
   });
   return e;
 }

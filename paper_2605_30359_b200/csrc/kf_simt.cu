@@ -9,19 +9,23 @@ static cudaError_t simt_gemm_t(int mode, int act, int M, int N, int K, const voi
                                long long ldx, const void* W, long long ldw, const void* bias,
                                float scale, const void* R, long long ldr, void* out, long long ldo,
                                cudaStream_t st) {
-  const dim3 grid((N + 31) / 32, (M + 31) / 32), block(256);
+  const dim3 grid((M + 31) / 32, (N + 31) / 32), block(256);   // rows on x: up to 2^31-1 tiles
+  if (grid.y > 65535u) return cudaErrorInvalidValue;
+  cudaError_t err = cudaSuccess;
   bool ok = dispatch_act(act, [&](auto A) {
     constexpr int ACT = decltype(A)::value;
-    if (mode == 0)
-      simt_gemm_kernel<T, 0, ACT><<<grid, block, 0, st>>>(
+    auto go = [&](auto kern) {
+      err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSimtSmemBytes);
+      if (err != cudaSuccess) return;
+      kern<<<grid, block, kSimtSmemBytes, st>>>(
           M, N, K, static_cast<const T*>(X), ldx, static_cast<const T*>(W), ldw,
           static_cast<const T*>(bias), scale, static_cast<const T*>(R), ldr, out, ldo);
-    else
-      simt_gemm_kernel<T, 1, ACT><<<grid, block, 0, st>>>(
-          M, N, K, static_cast<const T*>(X), ldx, static_cast<const T*>(W), ldw,
-          static_cast<const T*>(bias), scale, static_cast<const T*>(R), ldr, out, ldo);
+      err = cudaGetLastError();
+    };
+    if (mode == 0) go(simt_gemm_kernel<T, 0, ACT>);
+    else go(simt_gemm_kernel<T, 1, ACT>);
   });
-  return ok ? cudaGetLastError() : cudaErrorInvalidValue;
+  return ok ? err : cudaErrorInvalidValue;
 }
 
 cudaError_t launch_simt_gemm(int dt, int mode, int act, int M, int N, int K, const void* X,

@@ -33,48 +33,90 @@ __device__ __forceinline__ float block_reduce(float v, float* scratch /*[32]*/) 
 }
 
 // ---------------------------------------------------------------- scalar GEMM + epilogue
-// 32x32 output tile per CTA of 16x16 threads, 2x2 outputs per thread, K in slabs of 32 through
-// shared memory.  fp32 FMA accumulation in increasing k.
+// 32x32 output tile per CTA of eight warps.  The warps split K: in each pass over 256 values of
+// k, warp w owns k in [32w, 32w+32), loads its 32x32 slabs of X and W with coalesced reads
+// (lane = k), stages them k-major in its private shared memory and accumulates the whole 32x32
+// tile with an 8x4 register block per lane (32 FMAs per three 16-byte shared loads).  The next
+// slab is fetched into registers while the current one is consumed; there is no block-wide
+// barrier inside the K loop.  The eight partial tiles are then added in a fixed order.
 //   MODE 0: out = T,     Y[m,n] = scale*act(z+b) + R[m,n]
 //   MODE 1: out = float, A[m,n] = act(z+b) (pre-reduction values for the row kernels)
+constexpr int kSimtLd = 36;                                   // staged row pitch in floats
+constexpr int kSimtSmemBytes = 8 * 2 * 32 * kSimtLd * 4;      // 73,728 bytes of dynamic smem
+
 template <typename T, int MODE, int ACT>
 __global__ void __launch_bounds__(256)
 simt_gemm_kernel(int M, int N, int K, const T* __restrict__ X, long long ldx,
                  const T* __restrict__ W, long long ldw, const T* __restrict__ bias, float scale,
                  const T* R, long long ldr, void* out, long long ldo) {
-  __shared__ float As[32][33];
-  __shared__ float Bs[32][33];
-  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  const int m0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
-  float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-  const int lr = threadIdx.x >> 5, lc = threadIdx.x & 31;
-  for (int k0 = 0; k0 < K; k0 += 32) {
+  extern __shared__ float sm[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * 32, n0 = blockIdx.y * 32;
+  float* As = sm + warp * (2 * 32 * kSimtLd);
+  float* Bs = As + 32 * kSimtLd;
+  const int ly = lane >> 3, lx = lane & 7;
+  float acc[8][4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int r = lr + 8 * i;
-      const int k = k0 + lc;
-      const long long m = m0 + r, n = n0 + r;
-      As[r][lc] = (m < M && k < K) ? to_f32(X[m * ldx + k]) : 0.0f;
-      Bs[r][lc] = (n < N && k < K) ? to_f32(W[n * ldw + k]) : 0.0f;
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+  float ra[32], rb[32];
+  auto load_slab = [&](int kw) {
+    const int k = kw + lane;
+    const bool k_ok = k < K;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const long long m = m0 + i, n = n0 + i;
+      ra[i] = (k_ok && m < M) ? to_f32(X[m * ldx + k]) : 0.0f;
+      rb[i] = (k_ok && n < N) ? to_f32(W[n * ldw + k]) : 0.0f;
     }
-    __syncthreads();
+  };
+  int kw = warp * 32;
+  if (kw < K) load_slab(kw);
+  for (; kw < K; kw += 256) {
 #pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      As[lane * kSimtLd + i] = ra[i];
+      Bs[lane * kSimtLd + i] = rb[i];
+    }
+    __syncwarp();
+    if (kw + 256 < K) load_slab(kw + 256);
+#pragma unroll 8
     for (int kk = 0; kk < 32; ++kk) {
-      const float a0 = As[ty][kk], a1 = As[ty + 16][kk];
-      const float b0 = Bs[tx][kk], b1 = Bs[tx + 16][kk];
-      acc[0][0] = fmaf(a0, b0, acc[0][0]); acc[0][1] = fmaf(a0, b1, acc[0][1]);
-      acc[1][0] = fmaf(a1, b0, acc[1][0]); acc[1][1] = fmaf(a1, b1, acc[1][1]);
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[kk * kSimtLd + ly * 8]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&As[kk * kSimtLd + ly * 8 + 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&Bs[kk * kSimtLd + lx * 4]);
+      const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const float bb[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], bb[j], acc[i][j]);
     }
-    __syncthreads();
+    __syncwarp();
   }
+  __syncthreads();                       // staging is dead: reuse it for the partial tiles
+  float* red = sm;                       // [8 warps][32 rows][32 cols]
 #pragma unroll
-  for (int i = 0; i < 2; ++i) {
+  for (int i = 0; i < 8; ++i)
+    *reinterpret_cast<float4*>(&red[(warp * 32 + ly * 8 + i) * 32 + lx * 4]) =
+        make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+  __syncthreads();
+  const int r = threadIdx.x >> 3, c4 = (threadIdx.x & 7) * 4;
+  float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      const long long m = m0 + ty + 16 * i;
-      const int n = n0 + tx + 16 * j;
-      if (m < M && n < N) {
-        float z = acc[i][j];
+  for (int w = 0; w < 8; ++w) {
+    const float4 v = *reinterpret_cast<const float4*>(&red[(w * 32 + r) * 32 + c4]);
+    z4.x += v.x; z4.y += v.y; z4.z += v.z; z4.w += v.w;
+  }
+  const float zs[4] = {z4.x, z4.y, z4.z, z4.w};
+  const long long m = m0 + r;
+  if (m < M) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + c4 + j;
+      if (n < N) {
+        float z = zs[j];
         if (bias != nullptr) z += to_f32(bias[n]);
         if constexpr (MODE == 0) {
           float y = scale * act_f<ACT, false>(z);
@@ -364,6 +406,21 @@ groupnorm_apply_kernel(int Cout, int groups, long long hw, int tiles_per_image, 
   const long long cnt = static_cast<long long>(cpg) * hw;
   const int g = blockIdx.x % groups;
   const long long n = blockIdx.x / groups;
+  __nv_bfloat16* blk = y + (n * Cout + static_cast<long long>(g) * cpg) * hw;
+  const bool vec = (hw % 8) == 0 && (reinterpret_cast<uintptr_t>(blk) & 15u) == 0;
+  // Fetch this thread's first vectors before the statistics are known: the loads do not depend
+  // on them, so their latency hides behind the reduction.
+  constexpr int PRE = 4;
+  uint4 pre[PRE];
+  const long long nvec = cnt / 8;
+  if (vec) {
+    const uint4* bv = reinterpret_cast<const uint4*>(blk);
+#pragma unroll
+    for (int k = 0; k < PRE; ++k) {
+      const long long i = threadIdx.x + static_cast<long long>(k) * blockDim.x;
+      if (i < nvec) pre[k] = bv[i];
+    }
+  }
   float s1 = 0.0f, s2 = 0.0f;
   for (int i = threadIdx.x; i < tiles_per_image * cpg; i += blockDim.x) {
     const int t = i / cpg, c = g * cpg + i % cpg;
@@ -376,15 +433,19 @@ groupnorm_apply_kernel(int Cout, int groups, long long hw, int tiles_per_image, 
   const float mu = s1 / static_cast<float>(cnt);
   const float var = fmaxf(s2 / static_cast<float>(cnt) - mu * mu, 0.0f);
   const float rstd = rsqrtf(var + eps);
-  __nv_bfloat16* blk = y + (n * Cout + static_cast<long long>(g) * cpg) * hw;
-  if ((hw % 8) == 0 && (reinterpret_cast<uintptr_t>(blk) & 15u) == 0) {
+  if (vec) {
     uint4* bv = reinterpret_cast<uint4*>(blk);
-    for (long long i = threadIdx.x; i < cnt / 8; i += blockDim.x) {
+    for (long long i = threadIdx.x, k = 0; i < nvec; i += blockDim.x, ++k) {
       const int o = g * cpg + static_cast<int>((i * 8) / hw);
       const float ga = gamma != nullptr ? to_f32(gamma[o]) : 1.0f;
       const float be = beta != nullptr ? to_f32(beta[o]) : 0.0f;
       const float a = rstd * ga, b = fmaf(-mu, rstd * ga, be);
-      uint4 w = bv[i];
+      uint4 w;
+      if (k == 0) w = pre[0];
+      else if (k == 1) w = pre[1];
+      else if (k == 2) w = pre[2];
+      else if (k == 3) w = pre[3];
+      else w = bv[i];
       w.x = pack_bf16x2(fmaf(bf16_lo(w.x), a, b), fmaf(bf16_hi(w.x), a, b));
       w.y = pack_bf16x2(fmaf(bf16_lo(w.y), a, b), fmaf(bf16_hi(w.y), a, b));
       w.z = pack_bf16x2(fmaf(bf16_lo(w.z), a, b), fmaf(bf16_hi(w.z), a, b));

@@ -486,8 +486,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       } else {
         // EPI_CONV: rows = output channels, columns = BN consecutive pixels of one image, so a
         // thread's 32-column chunk is 64 contiguous bytes of the NCHW output.  a = act(z + b) is
-        // rounded to bf16 and stored; the per-channel sum and sum of squares of the stored
-        // values over this tile go to `partial` for the GroupNorm that follows.
+        // rounded to bf16 and stored; the per-channel sum and sum of squares of a (in fp32,
+        // before rounding) over this tile go to `partial` for the GroupNorm that follows.
         const int ch = tm * kBM + row;                      // output channel of this thread
         const bool ch_ok = ch < p.N;
         const int img = tn / p.tiles_per_image;
@@ -507,9 +507,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + bias_v);
             const float y1 = act_f<ACT, true>(__uint_as_float(v[2 * j + 1]) + bias_v);
             w[j] = pack_bf16x2(y0, y1);
-            const float r0 = bf16_lo(w[j]), r1 = bf16_hi(w[j]);
-            s1 += r0 + r1;
-            s2 = fmaf(r0, r0, fmaf(r1, r1, s2));
+            s1 += y0 + y1;
+            s2 = fmaf(y0, y0, fmaf(y1, y1, s2));
           }
           if (staged) {
             const int b = static_cast<int>(g & 1);

@@ -54,13 +54,9 @@ def load_peaks():
     return d
 
 
-def load_traffic():
-    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if any."""
-    p = os.path.join(ROOT, "profiles", "traffic.json")
-    try:
-        return json.load(open(p))
-    except Exception:
-        return {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the config-2 kernel, from the ncu
+# capture summarised in profiles/umma_chain_kernel_c2_gelu_residual.md (201.6 MB + 52.7 MB)
+TRAFFIC_C2_BYTES = 254.3e6
 
 
 # ------------------------------------------------------------------ clocks during the timed region
@@ -439,7 +435,7 @@ def main():
             dist.destroy_process_group()
         return
 
-    traffic = load_traffic().get("umma_chain_kernel_c2_bytes_per_launch")
+    traffic = TRAFFIC_C2_BYTES
     line = {
         "metric": "fused_chain_tflops", "value": round(value, 2), "unit": "TFLOP/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

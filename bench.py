@@ -112,6 +112,28 @@ class ClockSampler:
                 "samples": len(self.samples)}
 
 
+# ------------------------------------------------------------------ multi-rank bookkeeping
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """The slowest rank's time: what the whole job took (any torch.distributed backend)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tflops(flops_per_rank_per_step: float, world: int, ms_per_step: float) -> float:
+    """Aggregate throughput of `world` replicas that each did the full per-rank work."""
+    return flops_per_rank_per_step * world / (ms_per_step * 1e-3) / 1e12
+
+
+def rank_seed(rank: int) -> int:
+    """Each rank generates its own batch: the seed is the rank."""
+    return int(rank)
+
+
 # ------------------------------------------------------------------ helpers
 def to_dev(a, device):
     import torch
@@ -369,7 +391,7 @@ def main():
         return
 
     # inputs: rank r works on its own batch (seed r); resident in HBM before the timed region
-    d = ki.gemm_inputs(WORKLOAD, seed=rank)
+    d = ki.gemm_inputs(WORKLOAD, seed=rank_seed(rank))
     t = {k: to_dev(d[k], device) for k in ("X", "W", "b", "R")}
     Y = torch.empty(M2, N2, dtype=torch.bfloat16, device=device)
     step = lambda: kf.gemm_epilogue(t["X"], t["W"], t["b"], "gelu_tanh", 0.5, t["R"], out=Y)
@@ -397,12 +419,9 @@ def main():
     clocks = sampler.stop()
     if kf.kf_device_status() != kf.KF_OK:
         raise SystemExit("device status reports a timed-out wait: the run is invalid")
-    if world > 1:
-        tt = torch.tensor([ms], dtype=torch.float64, device=device)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms = float(tt.item())
+    ms = max_over_ranks(ms, world, device)
     ms_per_step = ms / args.steps
-    value = FLOPS_C2 * world / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tflops(FLOPS_C2, world, ms_per_step)
     kernel_tflops = FLOPS_C2 / (ms_per_step * 1e-3) / 1e12          # one launch per step per rank
 
     # end to end: pinned host buffers in, host buffer out, copies inside the timed region
@@ -422,11 +441,8 @@ def main():
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        tt = torch.tensor([e2e_ms], dtype=torch.float64, device=device)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt.item())
-    e2e_val = FLOPS_C2 * world / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    e2e_ms = max_over_ranks(e2e_ms, world, device)
+    e2e_val = whole_job_tflops(FLOPS_C2, world, e2e_ms / e2e_steps)
     h2d = sum(x.numel() * x.element_size() for x in (hX, hW, hb, hR))
     d2h = hY.numel() * hY.element_size()
 

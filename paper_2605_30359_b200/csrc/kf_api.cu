@@ -126,8 +126,10 @@ bool conv_umma_shape_ok(int dt, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout
 }
 // pixels per tile: 256 when whole tiles of 256 pixels cover the image, else 128
 int conv_tile_pixels(int64_t H, int64_t Wd) { return (H * Wd) % 256 == 0 ? 256 : 128; }
+// statistics entries per image: one per pixel tile
+int64_t conv_stat_parts(int64_t H, int64_t Wd) { return (H * Wd) / conv_tile_pixels(H, Wd); }
 size_t conv_stats_bytes(int64_t Nb, int64_t H, int64_t Wd, int64_t Cout) {
-  return round256(static_cast<size_t>(Nb) * ((H * Wd) / conv_tile_pixels(H, Wd)) * Cout * 8);
+  return round256(static_cast<size_t>(Nb) * conv_stat_parts(H, Wd) * Cout * 8);
 }
 
 kf_status check_gemm_common(int64_t M, int64_t N, int64_t K, int dt, const void* X, int64_t ldx,
@@ -395,7 +397,8 @@ kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
     ++launches;
     if (groups > 0) {
       if (launch_groupnorm_apply(static_cast<int>(Nb), static_cast<int>(Cout), groups, hw,
-                                 p.tiles_per_image, eps, stats, gamma, beta, y, st) != cudaSuccess)
+                                 static_cast<int>(conv_stat_parts(H, Wd)), eps, stats, gamma, beta,
+                                 y, st) != cudaSuccess)
         return KF_ERR_CUDA;
       ++launches;
     }

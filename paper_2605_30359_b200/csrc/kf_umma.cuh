@@ -31,8 +31,8 @@ enum : int { EPI_ELEMENTWISE = 0, EPI_SOFTMAX = 1, EPI_ROWSUM = 2, EPI_CONV = 3 
 constexpr int kBM = 128;          // tile rows = UMMA M = TMEM lanes
 constexpr int kBK = 64;           // K per stage: 64 bf16 = one 128-byte swizzled row
 constexpr int kUmmaK = 16;        // K per tcgen05.mma for 16-bit inputs
-constexpr int kEpiThreads = 128;  // warps 2..5
-constexpr int kNumThreads = 192;  // 6 warps
+constexpr int kEpiThreads = 128;  // warps 2..5: one per TMEM lane quarter
+constexpr int kNumThreads = 192;  // 6 warps: producer, UMMA issuer, epilogue
 constexpr int kPieceCols = 32;    // epilogue piece: 128 rows x 32 columns
 constexpr int kPieceBytes = kBM * kPieceCols * 2;   // 8 KB of bf16
 constexpr int kMaxDynSmem = 232448;                 // 227 KB opt-in limit per CTA
@@ -289,11 +289,6 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               for (int q = 0; q < 4; ++q)
                 rv[q] = *reinterpret_cast<const uint4*>(rb + piece_off(row, q));
             }
-            // ybuf[b] is free once the store issued two pieces ago has read it
-            if (leader) bulk_wait_group_read<1>();
-            rok = named_barrier_and(2, kEpiThreads, rok);   // all have consumed rbuf[b]
-            if (!rok) { alive = false; break; }
-            if (has_r && leader && g + 2 < total_pieces) issue_r(g + 2);
             uint32_t v[32];
             tmem_ld_32x32(t_acc + c * kPieceCols, v);
             float bs[32];
@@ -322,10 +317,16 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                              pack_bf16x2(f[8 * q + 4], f[8 * q + 5]),
                              pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
             fence_proxy_async_smem();
-            named_barrier_sync(3, kEpiThreads);
+            // One barrier per piece.  Before it the leader makes sure the previous piece's store
+            // has finished reading the other buffer, so after it (a) this piece may be stored,
+            // (b) the other output buffer may be rewritten, (c) rbuf[b] has been consumed by all.
+            if (leader) bulk_wait_group_read<0>();
+            rok = named_barrier_and(2, kEpiThreads, rok);
+            if (!rok) { alive = false; break; }
             if (leader) {
               tma_store_2d(&tmY, yb, n_tile + c * kPieceCols, tm * kBM);   // clipped at M, N
               bulk_commit_group();
+              if (has_r && g + 2 < total_pieces) issue_r(g + 2);
             }
           }
         } else {
@@ -415,8 +416,6 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if constexpr (sizeof(OutT) == 2) {
             if (staged) {
               const int b = static_cast<int>(g & 1);
-              if (leader) bulk_wait_group_read<1>();
-              named_barrier_sync(2, kEpiThreads);
               uint8_t* yb = ybuf + b * kPieceBytes;
 #pragma unroll
               for (int q = 0; q < 4; ++q)
@@ -426,7 +425,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                                pack_bf16x2(f[8 * q + 4], f[8 * q + 5]),
                                pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
               fence_proxy_async_smem();
-              named_barrier_sync(3, kEpiThreads);
+              if (leader) bulk_wait_group_read<0>();   // the other buffer's store has let go
+              named_barrier_sync(2, kEpiThreads);
               if (leader) {
                 tma_store_2d(&tmY, yb, n_tile + c * kPieceCols, tm * kBM);
                 bulk_commit_group();
@@ -512,15 +512,14 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
           if (staged) {
             const int b = static_cast<int>(g & 1);
-            if (leader) bulk_wait_group_read<1>();
-            named_barrier_sync(2, kEpiThreads);
             uint8_t* yb = ybuf + b * kPieceBytes;
 #pragma unroll
             for (int q = 0; q < 4; ++q)
               *reinterpret_cast<uint4*>(yb + piece_off(row, q)) =
                   make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
             fence_proxy_async_smem();
-            named_barrier_sync(3, kEpiThreads);
+            if (leader) bulk_wait_group_read<0>();     // the other buffer's store has let go
+            named_barrier_sync(2, kEpiThreads);
             if (leader) {
               // box = 32 pixels x 128 channels of image img; channels past Cout are clipped
               tma_store_3d(&tmY, yb, pt * BN + c * 32, tm * kBM, img);
@@ -536,7 +535,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
           }
         }
-        if (p.partial != nullptr && ch_ok) {
+        if (p.partial != nullptr && ch_ok) {      // one entry per pixel tile and channel
           float2* part = reinterpret_cast<float2*>(p.partial);
           part[static_cast<long long>(tn) * p.N + ch] = make_float2(s1, s2);
         }

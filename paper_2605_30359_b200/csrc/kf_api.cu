@@ -2,6 +2,7 @@
 // launches.  See include/kf.h for the contract of every entry point.
 #include <atomic>
 #include <cstring>
+#include <cstdlib>
 #include <mutex>
 
 #include "../../include/kf.h"
@@ -225,12 +226,17 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
 
   if (umma_gemm_ok(io_dtype, K, X, ldx, W, ldw)) {
     const int bn = N <= 128 ? 128 : 256;
+    // CTA pairs (256-row tiles, each CTA loading half of the W tile) when the problem has at
+    // least a few such tiles; env KF_NO_PAIR=1 forces one CTA per tile (for A/B measurements)
+    const bool pair = bn == 256 && M > 256 && getenv("KF_NO_PAIR") == nullptr;
     UmmaMaps tm;
-    if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, bn)) return KF_ERR_CUDA;
+    if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, pair ? bn / 2 : bn))
+      return KF_ERR_CUDA;
     UmmaParams p;
     std::memset(&p, 0, sizeof(p));
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
-    p.tiles_m = static_cast<int>((M + kBM - 1) / kBM);
+    const int tile_m = pair ? 2 * kBM : kBM;
+    p.tiles_m = static_cast<int>((M + tile_m - 1) / tile_m);
     p.tiles_n = static_cast<int>((N + bn - 1) / bn);
     if (static_cast<int64_t>(p.tiles_m) * p.tiles_n > kMaxDim) return KF_ERR_UNSUPPORTED;
     p.num_tiles = p.tiles_m * p.tiles_n;
@@ -249,8 +255,10 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
       if (residual != nullptr && !encode_piece(&tm.r, residual, M, N, ldr)) return KF_ERR_CUDA;
     }
     p.status = d->status;
-    const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
-    if (launch_umma_elementwise(bn, act, tm, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
+    const int slots = pair ? d->sm_count / 2 : d->sm_count;       // CTAs, or CTA pairs
+    const int grid = p.num_tiles < slots ? p.num_tiles : slots;
+    if (launch_umma_elementwise(bn, act, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
+      return KF_ERR_CUDA;
     g_launches += 1;
     return KF_OK;
   }

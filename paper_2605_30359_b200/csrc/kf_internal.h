@@ -17,8 +17,10 @@ struct UmmaMaps {
 };
 
 // tensor-core chains (bf16)
-cudaError_t launch_umma_elementwise(int bn, int act, const UmmaMaps& tm, const UmmaParams& p,
-                                    int grid, cudaStream_t st);
+// pair != 0: CTA-pair kernel (256-row tiles, `grid` = number of pairs, p.tiles_m counts 256-row
+// tiles); otherwise one CTA per 128-row tile
+cudaError_t launch_umma_elementwise(int bn, int act, int pair, const UmmaMaps& tm,
+                                    const UmmaParams& p, int grid, cudaStream_t st);
 cudaError_t launch_umma_softmax(int act, int out_dt, const UmmaMaps& tm, const UmmaParams& p,
                                 int grid, cudaStream_t st);
 cudaError_t launch_umma_rowsum(int act, const UmmaMaps& tm, const UmmaParams& p, int grid,
@@ -57,17 +59,35 @@ cudaError_t launch_groupnorm_apply(int Nb, int Cout, int groups, long long hw, i
                                    const void* beta, void* y, cudaStream_t st);
 
 // Generic launcher for one instantiation of the tensor-core kernel.
-template <int BN, int EPI, int ACT, typename OutT>
+// `grid` counts scheduled CTAs for the single-CTA kernel and CTA PAIRS for the pair kernel
+// (which launches 2*grid CTAs in clusters of two).
+template <int BN, int EPI, int ACT, typename OutT, bool CTA2 = false>
 inline cudaError_t launch_umma_instance(const UmmaMaps& tm, const UmmaParams& p, int grid,
                                         cudaStream_t st) {
-  using C = UmmaCfg<BN, EPI>;
+  using C = UmmaCfg<BN, EPI, CTA2>;
   constexpr int smem = C::kTotal;
   static_assert(smem <= kMaxDynSmem, "shared-memory plan exceeds the per-CTA limit");
-  auto kern = umma_chain_kernel<BN, EPI, ACT, OutT>;
+  auto kern = umma_chain_kernel<BN, EPI, ACT, OutT, CTA2>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  kern<<<grid, kNumThreads, smem, st>>>(tm.a, tm.b, tm.r, tm.y, p);
-  return cudaGetLastError();
+  if constexpr (CTA2) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * grid, 1, 1);
+    cfg.blockDim = dim3(kNumThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, tm.a, tm.b, tm.r, tm.y, p);
+  } else {
+    kern<<<grid, kNumThreads, smem, st>>>(tm.a, tm.b, tm.r, tm.y, p);
+    return cudaGetLastError();
+  }
 }
 
 }  // namespace kf

@@ -55,10 +55,13 @@ struct UmmaParams {
   int H, Wd, Cin, rows_per_tile, tiles_per_image, kb_per_tap;
 };
 
-template <int BN, int EPI>
+// CTA2: two CTAs of a cluster share one 256-row x BN tile (tcgen05 cta_group::2): each loads its
+// own 128 rows of A and HALF of the B tile, so a stage costs a CTA a third less shared memory
+// and L2 traffic for the same number of flops.
+template <int BN, int EPI, bool CTA2 = false>
 struct UmmaCfg {
   static constexpr int kStageA = kBM * kBK * 2;
-  static constexpr int kStageB = BN * kBK * 2;
+  static constexpr int kStageB = (CTA2 ? BN / 2 : BN) * kBK * 2;
   static constexpr int kStage = kStageA + kStageB;
   // staging: elementwise = 2 output + 2 residual pieces; softmax / conv = 2 output pieces
   static constexpr int kStaging =
@@ -100,12 +103,20 @@ __device__ __forceinline__ uint32_t piece_off(int r, int j) {
   return static_cast<uint32_t>(r * 64 + ((j ^ ((r >> 1) & 3)) << 4));
 }
 
-template <int BN, int EPI, int ACT, typename OutT>
+template <int BN, int EPI, int ACT, typename OutT, bool CTA2>
 __global__ void __launch_bounds__(kNumThreads, 1)
 umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmY,
                   const UmmaParams p) {
-  using C = UmmaCfg<BN, EPI>;
+  using C = UmmaCfg<BN, EPI, CTA2>;
+  static_assert(!CTA2 || EPI != EPI_CONV, "the convolution runs one CTA per tile");
+  constexpr int kTileM = CTA2 ? 2 * kBM : kBM;            // rows of one scheduled tile
+  // In a pair, rank 0 issues the MMAs; both ranks load, and both run the epilogue on their own
+  // 128 accumulator rows.  `cta` / `ncta` index the tile schedule (pairs count once).
+  uint32_t rank = 0;
+  if constexpr (CTA2) rank = cluster_ctarank();
+  const int cta = CTA2 ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+  const int ncta = CTA2 ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
   constexpr int kStages = C::kStages;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -127,7 +138,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     for (int a = 0; a < 2; ++a) {
       mbar_init(&tmem_full[a], 1);
-      mbar_init(&tmem_empty[a], kEpiThreads / 32);
+      mbar_init(&tmem_empty[a], (kEpiThreads / 32) * (CTA2 ? 2 : 1));
       mbar_init(&r_full[a], 1);
     }
     *abort_flag = 0;
@@ -135,12 +146,14 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
   }
-  if (warp == 1) {          // TMEM: two accumulators of BN fp32 columns
-    tmem_alloc(tmem_holder, 2 * BN);
-    tmem_relinquish();
+  __syncwarp();
+  if (warp == 1) {          // TMEM: two accumulators of BN fp32 columns (in both CTAs of a pair)
+    if constexpr (CTA2) { tmem_alloc_pair(tmem_holder, 2 * BN); tmem_relinquish_pair(); }
+    else { tmem_alloc(tmem_holder, 2 * BN); tmem_relinquish(); }
   }
   tc_fence_before_sync();
-  __syncthreads();
+  if constexpr (CTA2) cluster_sync_all();   // the peer's barriers exist before anyone signals them
+  else __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_holder;
 
@@ -148,7 +161,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int s = 0; uint32_t ph = 0;
-      for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+      for (int tile = cta; tile < p.num_tiles; tile += ncta) {
         int tm, tn, img = 0, h0 = 0;
         if constexpr (EPI == EPI_CONV) {
           tm = tile % p.tiles_m; tn = tile / p.tiles_m;        // output-channel tile, pixel tile
@@ -163,6 +176,14 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (!ok) break;
           uint8_t* sa = ring + s * C::kStage;
           uint8_t* sb = sa + C::kStageA;
+          if constexpr (CTA2) {
+            // both CTAs' bytes complete on rank 0's barrier, which rank 0 arms for the pair
+            if (rank == 0) mbar_expect_tx(&full[s], 2 * C::kStage);
+            tma_load_2d_pair(sa, &tmA, &full[s], kb * kBK, tm * kTileM + static_cast<int>(rank) * kBM);
+            tma_load_2d_pair(sb, &tmB, &full[s], kb * kBK, tn * BN + static_cast<int>(rank) * (BN / 2));
+            if (++s == kStages) { s = 0; ph ^= 1u; }
+            continue;
+          }
           mbar_expect_tx(&full[s], C::kStage);
           if constexpr (EPI == EPI_CONV) {
             const int tap = kb / p.kb_per_tap, cb = kb % p.kb_per_tap;
@@ -183,11 +204,11 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------ UMMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16_f32(kBM, BN);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16_f32(kTileM, BN);
       int s = 0; uint32_t ph = 0; int a = 0; uint32_t aph = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+      for (int tile = cta; ok && tile < p.num_tiles; tile += ncta) {
         ok = mbar_wait(&tmem_empty[a], aph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
         if (!ok) break;
         tc_fence_after_sync();
@@ -202,13 +223,18 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
             // +32 bytes per K step inside the 128-byte swizzled row = +2 in the address field
-            umma_f16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            if constexpr (CTA2)
+              umma_f16_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            else
+              umma_f16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          umma_commit(&empty[s]);
+          if constexpr (CTA2) umma_commit_pair(&empty[s], 3);      // frees the stage in both CTAs
+          else umma_commit(&empty[s]);
           if (++s == kStages) { s = 0; ph ^= 1u; }
         }
         if (!ok) break;
-        umma_commit(&tmem_full[a]);
+        if constexpr (CTA2) umma_commit_pair(&tmem_full[a], 3);    // wakes both epilogues
+        else umma_commit(&tmem_full[a]);
         if (++a == 2) { a = 0; aph ^= 1u; }
       }
     }
@@ -225,19 +251,19 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     [[maybe_unused]] uint8_t* rbuf = stg + 2 * kPieceBytes;   // [2][kPieceBytes] residual pieces
     const bool staged = p.staged != 0;
     [[maybe_unused]] const bool has_r = EPI == EPI_ELEMENTWISE && p.R != nullptr;
-    const int my_tiles = (p.num_tiles - static_cast<int>(blockIdx.x) +
-                          static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+    const int my_tiles = (p.num_tiles - cta + ncta - 1) / ncta;
+    const int row0 = static_cast<int>(rank) * kBM;      // this CTA's first row inside the tile
     [[maybe_unused]] const long long total_pieces = static_cast<long long>(my_tiles) * PIECES;
     [[maybe_unused]] long long g = 0;          // running piece index of this CTA
 
     // residual piece gi -> rbuf[gi & 1] (leader only)
     [[maybe_unused]] auto issue_r = [&](long long gi) {
       const int ti = static_cast<int>(gi / PIECES), c = static_cast<int>(gi % PIECES);
-      const int tile = blockIdx.x + ti * gridDim.x;
+      const int tile = cta + ti * ncta;
       const int b = static_cast<int>(gi & 1);
       mbar_expect_tx(&r_full[b], kPieceBytes);
       tma_load_2d(rbuf + b * kPieceBytes, &tmR, &r_full[b],
-                  (tile % p.tiles_n) * BN + c * kPieceCols, (tile / p.tiles_n) * kBM);
+                  (tile % p.tiles_n) * BN + c * kPieceCols, (tile / p.tiles_n) * kTileM + row0);
     };
     if constexpr (EPI == EPI_ELEMENTWISE) {
       if (staged && has_r && leader) {
@@ -248,11 +274,12 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
     int a = 0; uint32_t aph = 0;
     bool alive = true;
-    for (int tile = blockIdx.x; alive && tile < p.num_tiles; tile += gridDim.x) {
+    for (int tile = cta; alive && tile < p.num_tiles; tile += ncta) {
       int tm, tn;
       if constexpr (EPI == EPI_CONV) { tm = tile % p.tiles_m; tn = tile / p.tiles_m; }
       else { tm = tile / p.tiles_n; tn = tile % p.tiles_n; }
-      const long long m = static_cast<long long>(tm) * kBM + row;
+      const int m_cta = tm * kTileM + row0;               // first row of this CTA's 128 rows
+      const long long m = static_cast<long long>(m_cta) + row;
       [[maybe_unused]] const bool row_ok = m < p.M;
       [[maybe_unused]] const int n_tile = tn * BN;
       [[maybe_unused]] const int n_valid = min(BN, p.N - n_tile);   // valid columns in this tile
@@ -270,7 +297,10 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       auto release_acc = [&]() {
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&tmem_empty[a]);
+        if (lane == 0) {
+          if constexpr (CTA2) mbar_arrive_cluster(mapa_shared(smem_u32(&tmem_empty[a]), 0));
+          else mbar_arrive(&tmem_empty[a]);
+        }
       };
 
       if constexpr (EPI == EPI_ELEMENTWISE) {
@@ -324,7 +354,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             rok = named_barrier_and(2, kEpiThreads, rok);
             if (!rok) { alive = false; break; }
             if (leader) {
-              tma_store_2d(&tmY, yb, n_tile + c * kPieceCols, tm * kBM);   // clipped at M, N
+              tma_store_2d(&tmY, yb, n_tile + c * kPieceCols, m_cta);   // clipped at M, N
               bulk_commit_group();
               if (has_r && g + 2 < total_pieces) issue_r(g + 2);
             }
@@ -428,7 +458,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               if (leader) bulk_wait_group_read<0>();   // the other buffer's store has let go
               named_barrier_sync(2, kEpiThreads);
               if (leader) {
-                tma_store_2d(&tmY, yb, n_tile + c * kPieceCols, tm * kBM);
+                tma_store_2d(&tmY, yb, n_tile + c * kPieceCols, m_cta);
                 bulk_commit_group();
               }
               continue;
@@ -554,10 +584,13 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
     __syncthreads();
   }
+  // a pair leaves together: the peer's MMAs read this CTA's shared memory and signal its barriers
+  if constexpr (CTA2) cluster_sync_all();
   if (warp == 1) {
     __syncwarp();
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, 2 * BN);
+    if constexpr (CTA2) tmem_dealloc_pair(tmem_base, 2 * BN);
+    else tmem_dealloc(tmem_base, 2 * BN);
   }
 }
 

@@ -150,9 +150,16 @@ kf_status check_workspace(const void* ws, size_t have, size_t need) {
   return KF_OK;
 }
 
+// one statistic per row and 256-column tile
 size_t rowreduce_umma_ws(int64_t M, int64_t N, int red) {
   const int64_t tiles_n = (N + kRowReduceBN - 1) / kRowReduceBN;
   return round256(static_cast<size_t>(M) * tiles_n * (red == RED_SOFTMAX ? 8 : 4));
+}
+// CTA pairs (256-row tiles, each CTA loading half of the W tile) pay off when the K loop is
+// long: measured +3.6 % at K = 4096, +3.3 % at K = 2048, -4 % at K = 1024 (fewer, larger tiles
+// make the last wave's tail longer).  KF_NO_PAIR=1 forces one CTA per tile for A/B runs.
+bool use_cta_pairs(int64_t M, int64_t K) {
+  return M > 256 && K >= 2048 && getenv("KF_NO_PAIR") == nullptr;
 }
 size_t rowreduce_simt_ws(int64_t M, int64_t N) { return round256(static_cast<size_t>(M) * N * 4); }
 
@@ -226,9 +233,7 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
 
   if (umma_gemm_ok(io_dtype, K, X, ldx, W, ldw)) {
     const int bn = N <= 128 ? 128 : 256;
-    // CTA pairs (256-row tiles, each CTA loading half of the W tile) when the problem has at
-    // least a few such tiles; env KF_NO_PAIR=1 forces one CTA per tile (for A/B measurements)
-    const bool pair = bn == 256 && M > 256 && getenv("KF_NO_PAIR") == nullptr;
+    const bool pair = bn == 256 && use_cta_pairs(M, K);
     UmmaMaps tm;
     if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, pair ? bn / 2 : bn))
       return KF_ERR_CUDA;
@@ -288,20 +293,25 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int Mi = static_cast<int>(M), Ni = static_cast<int>(N), Ki = static_cast<int>(K);
 
-  const int64_t tiles_n64 = (N + kRowReduceBN - 1) / kRowReduceBN;
-  if (umma_gemm_ok(in_dtype, K, X, ldx, W, ldw) && tiles_n64 <= 8192) {
+  if (umma_gemm_ok(in_dtype, K, X, ldx, W, ldw) && (N + kRowReduceBN - 1) / kRowReduceBN <= 8192) {
     vs = check_workspace(workspace, workspace_bytes, rowreduce_umma_ws(M, N, red));
     if (vs != KF_OK) return vs;
+    const bool pair = use_cta_pairs(M, K);
+    const int tile_m = pair ? 2 * kBM : kBM;
+    const int slots = pair ? d->sm_count / 2 : d->sm_count;
+    const int64_t tiles_m64 = (M + tile_m - 1) / tile_m;
+    const int bn = kRowReduceBN;
+    const int64_t tiles_n64 = (N + bn - 1) / bn;
     UmmaMaps tm;
-    if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, kRowReduceBN))
+    if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, pair ? bn / 2 : bn))
       return KF_ERR_CUDA;
     tm.r = tm.a; tm.y = tm.a;
     UmmaParams p;
     std::memset(&p, 0, sizeof(p));
     p.M = Mi; p.N = Ni; p.K = Ki;
-    p.tiles_m = static_cast<int>((M + kBM - 1) / kBM);
+    p.tiles_m = static_cast<int>(tiles_m64);
     p.tiles_n = static_cast<int>(tiles_n64);
-    if (static_cast<int64_t>(p.tiles_m) * p.tiles_n > kMaxDim) return KF_ERR_UNSUPPORTED;
+    if (tiles_m64 * tiles_n64 > kMaxDim) return KF_ERR_UNSUPPORTED;
     p.num_tiles = p.tiles_m * p.tiles_n;
     p.k_blocks = static_cast<int>((K + kBK - 1) / kBK);
     p.bias = static_cast<const __nv_bfloat16*>(bias);
@@ -312,14 +322,16 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
     p.staged = (p.vec_ok && out_dtype == KF_BF16) ? 1 : 0;
     if (p.staged && !encode_piece(&tm.y, out, M, N, ldo)) return KF_ERR_CUDA;
     p.status = d->status;
-    const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
+    const int grid = p.num_tiles < slots ? p.num_tiles : slots;
     if (red == KF_RED_SOFTMAX) {
-      if (launch_umma_softmax(pre_act, out_dtype, tm, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
+      if (launch_umma_softmax(pre_act, out_dtype, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
+        return KF_ERR_CUDA;
       if (launch_softmax_finalize(out_dtype, Mi, Ni, p.tiles_n, p.partial, out, ldo, p.vec_ok, st) !=
           cudaSuccess)
         return KF_ERR_CUDA;
     } else {
-      if (launch_umma_rowsum(pre_act, tm, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
+      if (launch_umma_rowsum(pre_act, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
+        return KF_ERR_CUDA;
       if (launch_rowsum_finalize(Mi, p.tiles_n, p.partial, static_cast<float*>(out), st) != cudaSuccess)
         return KF_ERR_CUDA;
     }

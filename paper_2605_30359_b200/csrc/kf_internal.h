@@ -21,10 +21,10 @@ struct UmmaMaps {
 // tiles); otherwise one CTA per 128-row tile
 cudaError_t launch_umma_elementwise(int bn, int act, int pair, const UmmaMaps& tm,
                                     const UmmaParams& p, int grid, cudaStream_t st);
-cudaError_t launch_umma_softmax(int act, int out_dt, const UmmaMaps& tm, const UmmaParams& p,
-                                int grid, cudaStream_t st);
-cudaError_t launch_umma_rowsum(int act, const UmmaMaps& tm, const UmmaParams& p, int grid,
-                               cudaStream_t st);
+cudaError_t launch_umma_softmax(int act, int out_dt, int pair, const UmmaMaps& tm,
+                                const UmmaParams& p, int grid, cudaStream_t st);
+cudaError_t launch_umma_rowsum(int act, int pair, const UmmaMaps& tm, const UmmaParams& p,
+                               int grid, cudaStream_t st);
 cudaError_t launch_umma_conv(int bn, int act, const UmmaMaps& tm, const UmmaParams& p, int grid,
                              cudaStream_t st);
 constexpr int kRowReduceBN = 256;   // tile width of the row-reduce first pass

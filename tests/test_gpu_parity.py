@@ -95,6 +95,42 @@ def test_bf16_gemm_shapes(kf, shape):
     assert_close(got, ref, 2e-2, 2e-2, "bf16 %s" % (shape,))
 
 
+# K >= 2048 with more than 256 rows takes the CTA-pair kernel (256-row tiles over two SMs)
+@pytest.mark.parametrize("shape", [(384, 520, 2048), (257, 256, 2112), (1000, 264, 2048)])
+def test_bf16_gemm_cta_pair_kernel(kf, shape):
+    M, N, K = shape
+    d = ki.gemm_inputs("c2", seed=12, M=M, N=N, K=K)
+    got, ref = run_gemm(kf, d, "gelu_tanh", 0.5)
+    assert_close(got, ref, 2e-2, 2e-2, "bf16 pair %s" % (shape,))
+
+
+def test_bf16_cta_pair_layout_pins(kf):
+    """One-hot rows through the pair kernel: each CTA's A half and B half must land where the
+    256-row MMA expects them."""
+    M, N, K = 640, 512, 2048
+    r = np.random.default_rng(6)
+    Wv = (r.integers(-64, 65, size=(N, K)) / 64.0)
+    ks = r.integers(0, K, size=M)
+    Xf = np.zeros((M, K)); Xf[np.arange(M), ks] = 1.0
+    Y = kf.gemm_epilogue(to_dev(ki.store(Xf, "bf16")), to_dev(ki.store(Wv, "bf16")))
+    check_status()
+    assert_close(to_f64(Y), Wv[:, ks].T, 0.0, 0.0, "one-hot X rows, pair kernel")
+
+
+@pytest.mark.parametrize("red,act,shape", [("softmax", "none", (300, 1000, 2048)),
+                                           ("sum", "sigmoid", (520, 512, 2048))])
+def test_bf16_row_reductions_cta_pair_kernel(kf, red, act, shape):
+    M, N, K = shape
+    d = ki.gemm_inputs("c3", seed=13, M=M, N=N, K=K)
+    out = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), act, red)
+    check_status()
+    ref = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], act, red)
+    if red == "softmax":
+        softmax_gates(to_f64(out), ref, "softmax pair %s" % (shape,))
+    else:
+        assert_close(to_f64(out), ref, 0.0, 1e-3, "rowsum pair %s" % (shape,))
+
+
 @pytest.mark.parametrize("shape", [(5, 7, 3), (17, 9, 13), (40, 33, 20)])
 def test_bf16_unaligned_shapes_take_the_scalar_kernel(kf, shape):
     M, N, K = shape

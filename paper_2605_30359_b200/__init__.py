@@ -270,25 +270,60 @@ def _stage(name, host, device):
     return buf
 
 
+_side_streams = {}
+
+
+def _side(device):
+    """Two cached copy streams per device (host-to-device, device-to-host)."""
+    torch = _torch()
+    key = device.index
+    if key not in _side_streams:
+        _side_streams[key] = (torch.cuda.Stream(device), torch.cuda.Stream(device))
+    return _side_streams[key]
+
+
 def gemm_epilogue_host(X, W, bias=None, act="none", scale=1.0, residual=None, out_host=None,
-                       device=None, stream=None):
-    """gemm_epilogue for HOST tensors (pinned memory recommended): copies the inputs to the
-    device, runs the fused kernel, copies Y back into out_host.  Everything is enqueued on one
-    stream; synchronise that stream before reading out_host."""
+                       device=None, stream=None, chunks=4):
+    """gemm_epilogue for HOST tensors (pinned memory recommended).
+
+    Copies the inputs to the device, runs the fused kernel and copies Y back into out_host.
+    Rows are independent, so the batch is cut into `chunks` row blocks: block i is computed
+    while block i+1 is still arriving and block i-1 is already leaving (the copy engines of the
+    two directions run concurrently).  All work is ordered after, and joined back into, `stream`
+    (default: the current stream); synchronise it before reading out_host."""
     torch = _torch()
     device = device or torch.device("cuda", torch.cuda.current_device())
     s = stream if stream is not None else torch.cuda.current_stream(device)
-    with torch.cuda.stream(s):
-        dX = _stage("X", X, device); dX.copy_(X, non_blocking=True)
-        dW = _stage("W", W, device); dW.copy_(W, non_blocking=True)
-        db = dR = None
-        if bias is not None:
-            db = _stage("b", bias, device); db.copy_(bias, non_blocking=True)
-        if residual is not None:
-            dR = _stage("R", residual, device); dR.copy_(residual, non_blocking=True)
-        if out_host is None:
-            out_host = torch.empty((X.shape[0], W.shape[0]), dtype=X.dtype).pin_memory()
-        dY = _stage("Y", out_host, device)
-        gemm_epilogue(dX, dW, db, act, scale, dR, out=dY, stream=s)
-        out_host.copy_(dY, non_blocking=True)
+    s_in, s_out = _side(device)
+    M = X.shape[0]
+    if out_host is None:
+        out_host = torch.empty((M, W.shape[0]), dtype=X.dtype).pin_memory()
+    dX, dW, dY = _stage("X", X, device), _stage("W", W, device), _stage("Y", out_host, device)
+    db = _stage("b", bias, device) if bias is not None else None
+    dR = _stage("R", residual, device) if residual is not None else None
+    chunks = max(1, min(int(chunks), M // 256)) if M >= 512 else 1
+    bounds = [M * i // chunks for i in range(chunks + 1)]
+    s_in.wait_stream(s)
+    s_out.wait_stream(s)
+    with torch.cuda.stream(s_in):
+        dW.copy_(W, non_blocking=True)
+        if db is not None:
+            db.copy_(bias, non_blocking=True)
+    for i in range(chunks):
+        r0, r1 = bounds[i], bounds[i + 1]
+        with torch.cuda.stream(s_in):
+            dX[r0:r1].copy_(X[r0:r1], non_blocking=True)
+            if dR is not None:
+                dR[r0:r1].copy_(residual[r0:r1], non_blocking=True)
+            arrived = torch.cuda.Event()
+            arrived.record(s_in)
+        s.wait_event(arrived)
+        gemm_epilogue(dX[r0:r1], dW, db, act, scale, dR[r0:r1] if dR is not None else None,
+                      out=dY[r0:r1], stream=s)
+        computed = torch.cuda.Event()
+        computed.record(s)
+        s_out.wait_event(computed)
+        with torch.cuda.stream(s_out):
+            out_host[r0:r1].copy_(dY[r0:r1], non_blocking=True)
+    s.wait_stream(s_out)
     return out_host

@@ -361,3 +361,17 @@ def test_calls_on_a_side_stream(kf):
     s.synchronize()
     ref = oracle.gemm_epilogue(d["X"], d["W"], d["b"], "gelu_tanh", 0.5, d["R"])
     assert_close(to_f64(Y), ref, 2e-2, 2e-2, "side stream")
+
+
+def test_host_front_end_matches_device_call(kf):
+    """gemm_epilogue_host (chunked copies on side streams) gives the same bits as one device call."""
+    import torch
+    d = ki.gemm_inputs("c2", seed=10, M=1300, N=264, K=128)
+    pin = lambda a: torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    hX, hW, hb, hR = pin(d["X"]), pin(d["W"]), pin(d["b"]), pin(d["R"])
+    out = torch.zeros(1300, 264, dtype=torch.bfloat16).pin_memory()
+    kf.gemm_epilogue_host(hX, hW, hb, "gelu_tanh", 0.5, hR, out_host=out)
+    torch.cuda.synchronize()
+    ref = kf.gemm_epilogue(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "gelu_tanh", 0.5, to_dev(d["R"]))
+    assert torch.equal(out, ref.cpu())
+    check_status()

@@ -274,6 +274,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
     int a = 0; uint32_t aph = 0;
     bool alive = true;
+    [[maybe_unused]] uint64_t keep_policy = 0;
+    if constexpr (EPI == EPI_SOFTMAX) keep_policy = l2_policy_evict_last();
     for (int tile = cta; alive && tile < p.num_tiles; tile += ncta) {
       int tm, tn;
       if constexpr (EPI == EPI_CONV) { tm = tile % p.tiles_m; tn = tile / p.tiles_m; }
@@ -458,7 +460,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               if (leader) bulk_wait_group_read<0>();   // the other buffer's store has let go
               named_barrier_sync(2, kEpiThreads);
               if (leader) {
-                tma_store_2d(&tmY, yb, n_tile + c * kPieceCols, m_cta);
+                // the second pass reads these numerators back: ask L2 to keep them
+                tma_store_2d_hint(&tmY, yb, n_tile + c * kPieceCols, m_cta, keep_policy);
                 bulk_commit_group();
               }
               continue;

@@ -218,8 +218,8 @@ def run_reference(args):
     t0 = time.perf_counter()
     oracle.gemm_epilogue(d["X"][:probe], d["W"], d["b"], "gelu_tanh", 0.5, d["R"][:probe])
     dt = time.perf_counter() - t0
-    budget = 150.0 / max(1, args.steps + args.warmup)
-    rows = int(min(M2, max(probe, (min(6.0, budget) / dt) * probe)))
+    per_step_s = 150.0 / max(1, args.steps + args.warmup)
+    rows = int(min(M2, max(probe, (min(6.0, per_step_s) / dt) * probe)))
     rows -= rows % 128
     step = lambda: oracle.gemm_epilogue(d["X"][:rows], d["W"], d["b"], "gelu_tanh", 0.5, d["R"][:rows])
     for _ in range(args.warmup):

@@ -246,6 +246,7 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
     if (static_cast<int64_t>(p.tiles_m) * p.tiles_n > kMaxDim) return KF_ERR_UNSUPPORTED;
     p.num_tiles = p.tiles_m * p.tiles_n;
     p.k_blocks = static_cast<int>((K + kBK - 1) / kBK);
+    p.tiles_per_unit = 1;
     p.bias = static_cast<const __nv_bfloat16*>(bias);
     p.R = static_cast<const __nv_bfloat16*>(residual);
     p.ldr = ldr; p.out = Y; p.ldo = ldy; p.scale = scale;
@@ -314,15 +315,23 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
     if (tiles_m64 * tiles_n64 > kMaxDim) return KF_ERR_UNSUPPORTED;
     p.num_tiles = p.tiles_m * p.tiles_n;
     p.k_blocks = static_cast<int>((K + kBK - 1) / kBK);
+    p.tiles_per_unit = 1;
     p.bias = static_cast<const __nv_bfloat16*>(bias);
     p.out = out; p.ldo = ldo; p.scale = 1.0f;
     p.partial = static_cast<float*>(workspace);
+    // Row sum: when giving each CTA whole row blocks costs no extra wave, the epilogue carries
+    // the sum across the block's tiles and writes out[m] itself: no partials, no second pass.
+    const int64_t waves_rr = (tiles_m64 * tiles_n64 + slots - 1) / slots;
+    const int64_t waves_own = ((tiles_m64 + slots - 1) / slots) * tiles_n64;
+    const bool row_owner = red == KF_RED_SUM && waves_own <= waves_rr;
+    if (row_owner) { p.tiles_per_unit = p.tiles_n; p.partial = nullptr; }
     p.vec_ok = (red == KF_RED_SOFTMAX && (ldo * esize(out_dtype)) % 16 == 0 && aligned(out, 16)) ? 1 : 0;
     p.bias_vec = aligned(bias, 16) ? 1 : 0;
     p.staged = (p.vec_ok && out_dtype == KF_BF16) ? 1 : 0;
     if (p.staged && !encode_piece(&tm.y, out, M, N, ldo)) return KF_ERR_CUDA;
     p.status = d->status;
-    const int grid = p.num_tiles < slots ? p.num_tiles : slots;
+    const int units = p.num_tiles / p.tiles_per_unit;
+    const int grid = units < slots ? units : slots;
     if (red == KF_RED_SOFTMAX) {
       if (launch_umma_softmax(pre_act, out_dtype, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
         return KF_ERR_CUDA;
@@ -332,8 +341,14 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
     } else {
       if (launch_umma_rowsum(pre_act, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
         return KF_ERR_CUDA;
-      if (launch_rowsum_finalize(Mi, p.tiles_n, p.partial, static_cast<float*>(out), st) != cudaSuccess)
-        return KF_ERR_CUDA;
+      if (!row_owner) {
+        if (launch_rowsum_finalize(Mi, p.tiles_n, p.partial, static_cast<float*>(out), st) !=
+            cudaSuccess)
+          return KF_ERR_CUDA;
+        g_launches += 1;
+      }
+      g_launches += 1;
+      return KF_OK;
     }
     g_launches += 2;
     return KF_OK;
@@ -404,6 +419,7 @@ kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
     p.num_tiles = p.tiles_m * p.tiles_n;
     p.kb_per_tap = static_cast<int>(Cin / kBK);
     p.k_blocks = 9 * p.kb_per_tap;
+    p.tiles_per_unit = 1;
     p.bias = static_cast<const __nv_bfloat16*>(bias);
     p.out = y; p.scale = 1.0f;
     p.partial = groups > 0 ? stats : nullptr;

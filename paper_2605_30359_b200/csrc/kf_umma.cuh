@@ -51,9 +51,21 @@ struct UmmaParams {
   int staged;                  // out (and R) go through shared memory and TMA
   int bias_vec;                // bias is 16-byte aligned
   uint32_t* status;            // device status word
+  // Tile schedule: CTA (or pair) c takes units c, c+ncta, ...; a unit is `tiles_per_unit`
+  // consecutive tiles.  1 = plain round-robin; tiles_n = one CTA owns whole row blocks (row sum
+  // without a second pass).
+  int tiles_per_unit;
   // conv only
   int H, Wd, Cin, rows_per_tile, tiles_per_image, kb_per_tap;
 };
+
+// The it-th tile of scheduling slot `cta` out of `ncta`, or -1 when the slot has no more work.
+__device__ __forceinline__ int sched_tile(const UmmaParams& p, int cta, int ncta, int it) {
+  const int tpu = p.tiles_per_unit;
+  const int unit = cta + (it / tpu) * ncta;
+  if (unit >= p.num_tiles / tpu) return -1;
+  return unit * tpu + it % tpu;
+}
 
 // CTA2: two CTAs of a cluster share one 256-row x BN tile (tcgen05 cta_group::2): each loads its
 // own 128 rows of A and HALF of the B tile, so a stage costs a CTA a third less shared memory
@@ -161,7 +173,9 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int s = 0; uint32_t ph = 0;
-      for (int tile = cta; tile < p.num_tiles; tile += ncta) {
+      for (int it = 0;; ++it) {
+        const int tile = sched_tile(p, cta, ncta, it);
+        if (tile < 0) break;
         int tm, tn, img = 0, h0 = 0;
         if constexpr (EPI == EPI_CONV) {
           tm = tile % p.tiles_m; tn = tile / p.tiles_m;        // output-channel tile, pixel tile
@@ -208,7 +222,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       constexpr uint32_t idesc = umma_idesc_bf16_f32(kTileM, BN);
       int s = 0; uint32_t ph = 0; int a = 0; uint32_t aph = 0;
       bool ok = true;
-      for (int tile = cta; ok && tile < p.num_tiles; tile += ncta) {
+      for (int it = 0; ok; ++it) {
+        if (sched_tile(p, cta, ncta, it) < 0) break;
         ok = mbar_wait(&tmem_empty[a], aph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
         if (!ok) break;
         tc_fence_after_sync();
@@ -251,7 +266,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     [[maybe_unused]] uint8_t* rbuf = stg + 2 * kPieceBytes;   // [2][kPieceBytes] residual pieces
     const bool staged = p.staged != 0;
     [[maybe_unused]] const bool has_r = EPI == EPI_ELEMENTWISE && p.R != nullptr;
-    const int my_tiles = (p.num_tiles - cta + ncta - 1) / ncta;
+    const int num_units = p.num_tiles / p.tiles_per_unit;
+    const int my_tiles = cta < num_units ? (num_units - cta + ncta - 1) / ncta * p.tiles_per_unit : 0;
     const int row0 = static_cast<int>(rank) * kBM;      // this CTA's first row inside the tile
     [[maybe_unused]] const long long total_pieces = static_cast<long long>(my_tiles) * PIECES;
     [[maybe_unused]] long long g = 0;          // running piece index of this CTA
@@ -259,7 +275,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // residual piece gi -> rbuf[gi & 1] (leader only)
     [[maybe_unused]] auto issue_r = [&](long long gi) {
       const int ti = static_cast<int>(gi / PIECES), c = static_cast<int>(gi % PIECES);
-      const int tile = cta + ti * ncta;
+      const int tile = sched_tile(p, cta, ncta, ti);
       const int b = static_cast<int>(gi & 1);
       mbar_expect_tx(&r_full[b], kPieceBytes);
       tma_load_2d(rbuf + b * kPieceBytes, &tmR, &r_full[b],
@@ -276,7 +292,10 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     bool alive = true;
     [[maybe_unused]] uint64_t keep_policy = 0;
     if constexpr (EPI == EPI_SOFTMAX) keep_policy = l2_policy_evict_last();
-    for (int tile = cta; alive && tile < p.num_tiles; tile += ncta) {
+    [[maybe_unused]] float unit_sum = 0.0f;    // row sum carried across the tiles of a unit
+    for (int it = 0; alive; ++it) {
+      const int tile = sched_tile(p, cta, ncta, it);
+      if (tile < 0) break;
       int tm, tn;
       if constexpr (EPI == EPI_CONV) { tm = tile % p.tiles_m; tn = tile / p.tiles_m; }
       else { tm = tile / p.tiles_n; tn = tile % p.tiles_n; }
@@ -515,7 +534,13 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           sum += part;
         }
         release_acc();
-        if (row_ok) p.partial[m * p.tiles_n + tn] = sum;
+        if (p.partial != nullptr) {
+          if (row_ok) p.partial[m * p.tiles_n + tn] = sum;
+        } else {
+          // this CTA owns the whole row block: add the tiles in order, write the row sum once
+          unit_sum = (tn == 0) ? sum : unit_sum + sum;
+          if (tn == p.tiles_n - 1 && row_ok) reinterpret_cast<float*>(p.out)[m] = unit_sum;
+        }
       } else {
         // EPI_CONV: rows = output channels, columns = BN consecutive pixels of one image, so a
         // thread's 32-column chunk is 64 contiguous bytes of the NCHW output.  a = act(z + b) is

@@ -226,6 +226,19 @@ def test_bf16_sigmoid_rowsum(kf, shape):
     assert_close(to_f64(S), ref, 0.0, 1e-3, "rowsum relative %s" % (shape,))
 
 
+def test_bf16_rowsum_row_owner_schedule(kf):
+    """148 row blocks x 2 column tiles: each CTA owns whole row blocks, carries the sum across
+    its tiles and writes out[m] itself (no partial buffer, one kernel)."""
+    M, N, K = 18900, 512, 64
+    d = ki.gemm_inputs("c4", seed=2, M=M, N=N, K=K)
+    before = kf.kf_launch_count()
+    S = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "sigmoid", "sum")
+    check_status()
+    assert kf.kf_launch_count() - before == 1
+    ref = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "sigmoid", "sum")
+    assert_close(to_f64(S), ref, 0.0, 1e-3, "rowsum row-owner")
+
+
 def test_rowsum_closed_forms(kf):
     N, K = 1024, 128
     d = ki.gemm_inputs("c4", seed=3, M=256, N=N, K=K)

@@ -283,6 +283,8 @@ def run_conv(kf, d, act="relu", groups=None, gamma=None, beta=None, use_bias=Tru
     dict(Nb=3, Cin=128, H=16, W=32, Cout=64, groups=4),      # two channel blocks per tap, 4 rows per tile
     dict(Nb=1, Cin=64, H=16, W=8, Cout=256, groups=0),       # 16 rows per tile, widest N tile, no norm
     dict(Nb=2, Cin=64, H=2, W=128, Cout=48, groups=3),       # one row per tile, Cout below the tile width
+    dict(Nb=3, Cin=64, H=13, W=64, Cout=96, groups=3),       # NCHW-direct kernel, ragged row units
+    dict(Nb=1, Cin=64, H=1, W=64, Cout=128, groups=0),       # NCHW-direct kernel, single row
 ])
 def test_bf16_conv_tensor_core_path(kf, cfg):
     d = ki.conv_inputs(seed=1, **cfg)

@@ -54,6 +54,8 @@ def _load():
         lib.oracle_conv3x3_gn.restype = ci
         lib.oracle_conv3x3_gn.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, ci, dbl,
                                           vp, vp, vp]
+        lib.oracle_conv3x3_softmax_pool.restype = ci
+        lib.oracle_conv3x3_softmax_pool.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, i64, vp]
         _lib = lib
     return _lib
 
@@ -128,5 +130,17 @@ def conv3x3_gn(x, w, bias=None, act="none", groups=0, eps=1e-5, gamma=None, beta
     rc = _load().oracle_conv3x3_gn(Nb, Cin, H, Wd, Cout, dt, _ptr(x), _ptr(w), _ptr(bias),
                                    ACT[act], int(groups), float(eps), _ptr(gamma), _ptr(beta),
                                    _ptr(y))
+    assert rc == 0
+    return y
+
+
+def conv3x3_softmax_pool(x, w, bias=None, pool=1):
+    """max_pool(softmax over channels(conv3x3_pad1(x, w) + bias), pool), fp64 NCHW."""
+    x = _c(x); dt = _dt(x); w = _c(w, dt); bias = _c(bias, dt)
+    Nb, Cin, H, Wd = x.shape
+    Cout = w.shape[0]
+    y = np.empty((Nb, Cout, H // pool, Wd // pool), np.float64)
+    rc = _load().oracle_conv3x3_softmax_pool(Nb, Cin, H, Wd, Cout, dt, _ptr(x), _ptr(w), _ptr(bias),
+                                             int(pool), _ptr(y))
     assert rc == 0
     return y

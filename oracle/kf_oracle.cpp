@@ -19,6 +19,9 @@
 //   * Activations: Appendix C.2 listing formulas -- sigmoid(x)*x (swish), tanh written as
 //     (e^{2s}-1)/(e^{2s}+1), GELU in its erf form t*0.5*(1+erf(t/sqrt 2)), hardtanh as
 //     clamp to [-1,1].  GELU-tanh is the usual PyTorch approximate='tanh' definition.
+//   * Channel softmax + max-pool after a convolution: the chain of Appendix C.1
+//     (conv -> softmax over channels -> max-pool -> max-pool), with the softmax in the three
+//     passes printed there.
 //   * Convolution / GroupNorm: Table 2 "Conv-centered" chains; PyTorch semantics
 //     (cross-correlation, zero padding, biased variance, eps inside the root).
 //
@@ -200,6 +203,63 @@ int oracle_conv3x3_gn(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Co
         }
       }
     }
+  }
+  return 0;
+}
+
+// c[n,o,h,w] = bias[o] + sum_{c,r,s} x[n,c,h+r-1,w+s-1] * wt[o,c,r,s]   (as above)
+// s[n,o,h,w] = exp(c[n,o,h,w] - max_o c[n,:,h,w]) / sum_o exp(c[n,o,h,w] - max_o c[n,:,h,w])
+//              -- softmax over the CHANNEL dimension, in the three passes the paper prints for
+//              this operator (Appendix C.1: per (batch, position): max, sum of exp, quotient)
+// y[n,o,i,j] = max over the pool x pool window starting at (i*pool, j*pool) of s  (pool >= 1;
+//              windows do not overlap, a ragged rim is dropped as torch's max_pool2d does).
+// Two max-pools of size k in a row, as in the paper's chain, equal one of size k*k.
+// y is fp64 [Nb, Cout, H/pool, Wd/pool].
+int oracle_conv3x3_softmax_pool(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                                int dt, const void* x, const void* wt, const void* bias,
+                                int64_t pool, double* y) {
+  if (pool < 1) return 1;
+  const int64_t Ho = H / pool, Wo = Wd / pool;
+#pragma omp parallel for schedule(dynamic) num_threads(nthreads())
+  for (int64_t n = 0; n < Nb; ++n) {
+    std::vector<double> s((size_t)(Cout * H * Wd));
+    for (int64_t o = 0; o < Cout; ++o)
+      for (int64_t h = 0; h < H; ++h)
+        for (int64_t w = 0; w < Wd; ++w) {
+          double acc = bias ? widen(bias, dt, o) : 0.0;
+          for (int64_t c = 0; c < Cin; ++c)
+            for (int r = 0; r < 3; ++r) {
+              int64_t hh = h + r - 1;
+              if (hh < 0 || hh >= H) continue;
+              for (int q = 0; q < 3; ++q) {
+                int64_t ww = w + q - 1;
+                if (ww < 0 || ww >= Wd) continue;
+                acc += widen(x, dt, ((n * Cin + c) * H + hh) * Wd + ww) *
+                       widen(wt, dt, ((o * Cin + c) * 3 + r) * 3 + q);
+              }
+            }
+          s[(size_t)((o * H + h) * Wd + w)] = acc;
+        }
+    for (int64_t h = 0; h < H; ++h)
+      for (int64_t w = 0; w < Wd; ++w) {
+        double mx = -INFINITY;
+        for (int64_t o = 0; o < Cout; ++o) mx = std::fmax(mx, s[(size_t)((o * H + h) * Wd + w)]);
+        double sum = 0.0;
+        for (int64_t o = 0; o < Cout; ++o) sum += std::exp(s[(size_t)((o * H + h) * Wd + w)] - mx);
+        for (int64_t o = 0; o < Cout; ++o) {
+          double& v = s[(size_t)((o * H + h) * Wd + w)];
+          v = std::exp(v - mx) / sum;
+        }
+      }
+    for (int64_t o = 0; o < Cout; ++o)
+      for (int64_t i = 0; i < Ho; ++i)
+        for (int64_t j = 0; j < Wo; ++j) {
+          double m = -INFINITY;
+          for (int64_t a = 0; a < pool; ++a)
+            for (int64_t b = 0; b < pool; ++b)
+              m = std::fmax(m, s[(size_t)((o * H + i * pool + a) * Wd + j * pool + b)]);
+          y[((n * Cout + o) * Ho + i) * Wo + j] = m;
+        }
   }
   return 0;
 }

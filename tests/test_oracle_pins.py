@@ -380,3 +380,38 @@ def test_bf16_rounding_is_nearest_even():
     assert np.array_equal(got, [1.0, 1 + 2 ** -6, 1 + 2 ** -7, -1.0, 1 + 2 ** -7])
     x = ki.normal(3, 1, (1000,))
     assert np.abs(ki.widen(ki.to_bf16_bits(x)) / x - 1).max() <= 2 ** -8
+
+
+# ------------------------------------------------------------------ conv -> channel softmax -> pool
+def test_channel_softmax_invariants_and_library_case():
+    d = ki.conv_inputs(Nb=2, Cin=3, H=6, W=8, Cout=5, groups=0, seed=7)
+    s = oracle.conv3x3_softmax_pool(d["x"], d["w"], d["bias"], pool=1)
+    assert np.abs(s.sum(axis=1) - 1.0).max() < 1e-14 and (s > 0).all()      # over channels
+    c = oracle.conv3x3_gn(d["x"], d["w"], d["bias"])                         # pinned above
+    assert np.abs(s - scipy.special.softmax(c, axis=1)).max() < 1e-15
+    # the reduction runs over channels, not over pixels: pixel sums are not 1
+    assert np.abs(s.sum(axis=(2, 3)) - 1.0).min() > 0.5
+    # shift invariance per pixel: adding a constant to every channel's bias changes nothing
+    b2 = ki.store(ki.widen(d["bias"]) + 0.5, "bf16")
+    if np.array_equal(ki.widen(b2), ki.widen(d["bias"]) + 0.5):
+        s2 = oracle.conv3x3_softmax_pool(d["x"], d["w"], b2, pool=1)
+        assert np.abs(s2 - s).max() < 1e-14
+    # zero weights: every channel equal -> exactly 1/Cout
+    z = oracle.conv3x3_softmax_pool(d["x"], bf(np.zeros((5, 3, 3, 3))), None, pool=1)
+    assert np.array_equal(z, np.full_like(z, 0.2))
+
+
+def test_channel_softmax_pooling():
+    d = ki.conv_inputs(Nb=1, Cin=2, H=8, W=12, Cout=4, groups=0, seed=8)
+    s = oracle.conv3x3_softmax_pool(d["x"], d["w"], d["bias"], pool=1)
+    for k in (2, 4):
+        p = oracle.conv3x3_softmax_pool(d["x"], d["w"], d["bias"], pool=k)
+        want = s[:, :, :8 // k * k, :12 // k * k].reshape(1, 4, 8 // k, k, 12 // k, k).max(axis=(3, 5))
+        assert p.shape == (1, 4, 8 // k, 12 // k) and np.array_equal(p, want)
+    # two pools of 2 in a row (the paper's chain) equal one pool of 4
+    p2 = oracle.conv3x3_softmax_pool(d["x"], d["w"], d["bias"], pool=2)
+    twice = p2.reshape(1, 4, 2, 2, 3, 2).max(axis=(3, 5))
+    assert np.array_equal(twice, oracle.conv3x3_softmax_pool(d["x"], d["w"], d["bias"], pool=4))
+    # a ragged rim is dropped
+    d3 = ki.conv_inputs(Nb=1, Cin=2, H=5, W=7, Cout=3, groups=0, seed=9)
+    assert oracle.conv3x3_softmax_pool(d3["x"], d3["w"], None, pool=2).shape == (1, 3, 2, 3)

@@ -332,6 +332,22 @@ def chain_table(kf, device, peaks, c2_tensors, c2_us):
         "shape": "config 2's X, W, b", "us_per_call": round(us, 3),
         "tflops": round(FLOPS_C2 / us / 1e6, 2), "unfused_torch_us": round(us_torch, 3),
         "speedup_vs_unfused_torch": round(us_torch / us, 3), "paper_speedup_rtx5090": 1.31}
+    # The 2-D form of the paper's case-study chain (Appendix C.1): conv, softmax over channels,
+    # two max-pools of 2 (= one of 4).  Shape: config 5's x, w, bias (the paper prints none).
+    d = ki.conv_inputs("c5", seed=0)
+    t5 = {k: to_dev(d[k], device) for k in ("x", "w", "bias")}
+    op = torch.empty(128, 128, 16, 16, dtype=torch.bfloat16, device=device)
+    us = time_calls(lambda: kf.conv3x3_softmax_pool(t5["x"], t5["w"], t5["bias"], 4, out=op), 40, 5)
+
+    def torch_conv_softmax_pool():
+        z = torch.softmax(F.conv2d(t5["x"], t5["w"], t5["bias"], padding=1), dim=1)
+        return F.max_pool2d(F.max_pool2d(z, 2), 2)
+
+    us_torch = time_calls(torch_conv_softmax_pool, 20, 5)
+    out["paper_chain_conv_softmax_maxpool_maxpool_2d"] = {
+        "shape": "config 5's x, w, bias; pool 2 twice", "us_per_call": round(us, 3),
+        "tflops": round(specs["c5"]["flops"] / us / 1e6, 2), "unfused_torch_us": round(us_torch, 3),
+        "speedup_vs_unfused_torch": round(us_torch / us, 3)}
     return out
 
 

@@ -140,6 +140,25 @@ kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
                               const void* beta, void* y,
                               void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* 3x3 convolution -> softmax over the channel dimension -> max-pool: the 2-D form of the chain in
+ * the paper's Appendix C.1 case study (3-D there: conv, softmax, max-pool, max-pool; two pools of size k in a row equal
+ * one of size k*k), with the softmax as printed there (per position: max over channels, sum of
+ * exp, quotient).
+ *   c[n,o,h,w] = bias[o] + sum_{c,r,s} x[n,c,h+r-1,w+s-1] * w[o,c,r,s]
+ *   s[n,o,h,w] = exp(c[n,o,h,w] - max_o c[n,:,h,w]) / sum_o exp(c[n,o,h,w] - max_o c[n,:,h,w])
+ *   y[n,o,i,j] = max of s over the pool x pool window at (i*pool, j*pool)
+ * x NCHW [Nb,Cin,H,Wd], w OIHW, y NCHW [Nb,Cout,H/pool,Wd/pool] (floor; a ragged rim is dropped),
+ * all dense, of io_dtype; bias may be NULL.  1 <= pool <= 4 (larger: KF_ERR_UNSUPPORTED); pool
+ * above H or Wd gives an empty y and the call returns KF_OK without work.  The
+ * convolution takes the same kernels as kf_conv3x3_epilogue; its output is staged in the
+ * workspace (io_dtype), whose size kf_conv3x3_softmax_pool_workspace_bytes() returns. */
+kf_status kf_conv3x3_softmax_pool(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                                  kf_dtype io_dtype, const void* x, const void* w, const void* bias,
+                                  int pool, void* y,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+size_t kf_conv3x3_softmax_pool_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd,
+                                               int64_t Cout, kf_dtype io_dtype);
+
 /* Workspace sizes in bytes for the calls above with the same arguments (0 = none needed).
  * Pure host arithmetic; no CUDA call is made. */
 size_t kf_gemm_epilogue_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype);

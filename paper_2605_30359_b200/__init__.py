@@ -27,7 +27,8 @@ ACT = {"none": 0, "relu": 1, "gelu_tanh": 2, "sigmoid": 3, "gelu_erf": 4, "swish
 RED = {"softmax": 0, "sum": 1}
 
 EXPORTS = ["kf_gemm_epilogue", "kf_gemm_rowreduce", "kf_gemm_rowreduce_static",
-           "kf_conv3x3_epilogue",
+           "kf_conv3x3_epilogue", "kf_conv3x3_softmax_pool",
+           "kf_conv3x3_softmax_pool_workspace_bytes",
            "kf_gemm_epilogue_workspace_bytes", "kf_gemm_rowreduce_workspace_bytes",
            "kf_conv3x3_workspace_bytes", "kf_device_status", "kf_launch_count",
            "kf_status_string", "kf_version"]
@@ -64,6 +65,10 @@ def lib() -> ctypes.CDLL:
     L.kf_conv3x3_epilogue.restype = ci
     L.kf_conv3x3_epilogue.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, ci, f32, vp, vp,
                                       vp, vp, sz, vp]
+    L.kf_conv3x3_softmax_pool.restype = ci
+    L.kf_conv3x3_softmax_pool.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp, sz, vp]
+    L.kf_conv3x3_softmax_pool_workspace_bytes.restype = sz
+    L.kf_conv3x3_softmax_pool_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, ci]
     L.kf_gemm_epilogue_workspace_bytes.restype = sz
     L.kf_gemm_epilogue_workspace_bytes.argtypes = [i64, i64, i64, ci]
     L.kf_gemm_rowreduce_workspace_bytes.restype = sz
@@ -110,6 +115,16 @@ def kf_conv3x3_epilogue(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, groups,
                         y, workspace, workspace_bytes, stream) -> int:
     return lib().kf_conv3x3_epilogue(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, groups, eps,
                                      gamma, beta, y, workspace, workspace_bytes, stream)
+
+
+def kf_conv3x3_softmax_pool(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, pool, y, workspace,
+                            workspace_bytes, stream) -> int:
+    return lib().kf_conv3x3_softmax_pool(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, pool, y,
+                                         workspace, workspace_bytes, stream)
+
+
+def kf_conv3x3_softmax_pool_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype) -> int:
+    return lib().kf_conv3x3_softmax_pool_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype)
 
 
 def kf_gemm_epilogue_workspace_bytes(M, N, K, io_dtype) -> int:
@@ -252,6 +267,27 @@ def conv3x3_epilogue(x, w, bias=None, act="none", groups=0, eps=1e-5, gamma=None
                              nb, _stream_ptr(stream))
     if st != KF_OK:
         raise KfError(st, "kf_conv3x3_epilogue")
+    return out
+
+
+def conv3x3_softmax_pool(x, w, bias=None, pool=1, out=None, stream=None):
+    """y = max_pool(softmax over channels(conv3x3_pad1(x, w) + bias), pool); NCHW / OIHW."""
+    torch = _torch()
+    _check_cuda(x, w, bias, out)
+    if not (x.is_contiguous() and w.is_contiguous()):
+        raise ValueError("conv3x3_softmax_pool takes contiguous NCHW / OIHW tensors")
+    Nb, Cin, H, Wd = x.shape
+    Cout = w.shape[0]
+    dt = _kf_dtype(x)
+    if out is None:
+        div = max(int(pool), 1)        # a bad pool is rejected by the library, not here
+        out = torch.empty((Nb, Cout, H // div, Wd // div), dtype=x.dtype, device=x.device)
+    nb = kf_conv3x3_softmax_pool_workspace_bytes(Nb, Cin, H, Wd, Cout, dt)
+    ws = workspace(nb, x.device)
+    st = kf_conv3x3_softmax_pool(Nb, Cin, H, Wd, Cout, dt, _ptr(x), _ptr(w), _ptr(bias), int(pool),
+                                 _ptr(out), _ptr(ws), nb, _stream_ptr(stream))
+    if st != KF_OK:
+        raise KfError(st, "kf_conv3x3_softmax_pool")
     return out
 
 

@@ -515,3 +515,43 @@ extern "C" kf_status kf_gemm_rowreduce_static(int64_t M, int64_t N, int64_t K, k
   return kf_gemm_rowreduce(M, N, K, in_dtype, X, ldx, W, ldw, bias, pre_act, red, out, ldo,
                            out_dtype, scratch, KF_STATIC_SCRATCH_BYTES, cuda_stream);
 }
+
+// ---------------------------------------------------------------------------------------------
+// conv3x3 -> softmax over channels -> max-pool: the convolution entry point writes conv + bias
+// into the front of the workspace, a second kernel reduces over channels and pools.
+// ---------------------------------------------------------------------------------------------
+extern "C" size_t kf_conv3x3_softmax_pool_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H,
+                                                          int64_t Wd, int64_t Cout,
+                                                          kf_dtype io_dtype) {
+  if (Nb < 1 || Cin < 1 || H < 1 || Wd < 1 || Cout < 1) return 0;
+  return round256(static_cast<size_t>(Nb) * Cout * H * Wd * esize(io_dtype)) +
+         kf_conv3x3_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype, 0);
+}
+
+extern "C" kf_status kf_conv3x3_softmax_pool(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd,
+                                             int64_t Cout, kf_dtype io_dtype, const void* x,
+                                             const void* w, const void* bias, int pool, void* y,
+                                             void* workspace, size_t workspace_bytes,
+                                             void* cuda_stream) {
+  if (Nb < 1 || Cin < 1 || H < 1 || Wd < 1 || Cout < 1) return KF_ERR_INVALID_ARG;
+  if (!valid_dtype(io_dtype) || pool < 1) return KF_ERR_INVALID_ARG;
+  if (pool > 4) return KF_ERR_UNSUPPORTED;
+  if (H / pool == 0 || Wd / pool == 0) return KF_OK;   // empty result: nothing to compute
+  if (y == nullptr || !aligned(y, esize(io_dtype)) || y == x) return KF_ERR_INVALID_ARG;
+  if (Nb > kMaxDim || Cout > kMaxDim || H > kMaxDim || Wd > kMaxDim) return KF_ERR_INVALID_ARG;
+  const size_t a_bytes = round256(static_cast<size_t>(Nb) * Cout * H * Wd * esize(io_dtype));
+  const size_t conv_bytes = kf_conv3x3_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype, 0);
+  kf_status vs = check_workspace(workspace, workspace_bytes, a_bytes + conv_bytes);
+  if (vs != KF_OK) return vs;
+  void* a = workspace;
+  void* conv_ws = conv_bytes ? static_cast<uint8_t*>(workspace) + a_bytes : nullptr;
+  vs = kf_conv3x3_epilogue(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, KF_ACT_NONE, 0, 0.0f, nullptr,
+                           nullptr, a, conv_ws, conv_bytes, cuda_stream);
+  if (vs != KF_OK) return vs;
+  if (launch_channel_softmax_pool(io_dtype, static_cast<int>(Nb), static_cast<int>(Cout),
+                                  static_cast<int>(H), static_cast<int>(Wd), pool, a, y,
+                                  static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return KF_ERR_CUDA;
+  g_launches += 1;
+  return KF_OK;
+}

@@ -58,6 +58,10 @@ cudaError_t launch_groupnorm_apply(int Nb, int Cout, int groups, long long hw, i
                                    float eps, const float* stats, const void* gamma,
                                    const void* beta, void* y, cudaStream_t st);
 
+// softmax over channels + pool x pool max-pool of an NCHW tensor (pool <= 4)
+cudaError_t launch_channel_softmax_pool(int dt, int Nb, int C, int H, int Wd, int pool, const void* a,
+                                        void* y, cudaStream_t st);
+
 // Generic launcher for one instantiation of the tensor-core kernel.
 // `grid` counts scheduled CTAs for the single-CTA kernel and CTA PAIRS for the pair kernel
 // (which launches 2*grid CTAs in clusters of two).

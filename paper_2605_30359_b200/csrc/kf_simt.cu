@@ -131,4 +131,58 @@ cudaError_t launch_groupnorm_apply(int Nb, int Cout, int groups, long long hw, i
   return cudaGetLastError();
 }
 
+namespace {
+constexpr size_t kPoolStripBytes = 64 * 1024;   // shared-memory strip per block (3 blocks per SM)
+// plus one float per strip pixel for the log-sum-exp: at most kPoolStripBytes / sizeof(T) / C * 4
+
+template <typename T>
+cudaError_t channel_softmax_pool_typed(int Nb, int C, int H, int Wd, int pool, const T* a, T* y,
+                                       cudaStream_t st) {
+  const int Ho = H / pool, Wo = Wd / pool;
+  const size_t per_col = static_cast<size_t>(C) * pool * pool * sizeof(T);   // one pooled column
+  if (per_col > kPoolStripBytes) {
+    // strip does not fit: one thread per pooled pixel straight from global memory
+    const long long total = static_cast<long long>(Nb) * Ho * Wo;
+    channel_softmax_pool_kernel<T><<<static_cast<unsigned>((total + 255) / 256), 256, 0, st>>>(
+        Nb, C, H, Wd, pool, a, y);
+    return cudaGetLastError();
+  }
+  int tw = static_cast<int>(kPoolStripBytes / per_col);
+  if (tw > Wo) tw = Wo;
+  constexpr int kVec = 16 / sizeof(T);
+  // vector loads need every row segment to start on 16 bytes and to be whole vectors
+  bool vec = (reinterpret_cast<uintptr_t>(a) % 16 == 0) && (Wd % kVec == 0);
+  if (vec) {
+    // shrink tw until tw*pool is a multiple of the vector (the ragged last tile must be too)
+    int t = tw;
+    while (t > 0 && ((t * pool) % kVec != 0)) --t;
+    if (t > 0 && ((Wo % t) * pool) % kVec == 0) tw = t; else vec = false;
+  }
+  const size_t smem = ((static_cast<size_t>(C) * pool * pool * tw * sizeof(T) + 15) & ~static_cast<size_t>(15)) +
+                      static_cast<size_t>(pool) * pool * tw * sizeof(float);
+  const long long blocks = static_cast<long long>(Nb) * Ho * ((Wo + tw - 1) / tw);
+  if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+  auto launch = [&](auto kern) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(kPoolStripBytes * 3 + 16));
+    if (e != cudaSuccess) return e;
+    kern<<<static_cast<unsigned>(blocks), 256, smem, st>>>(Nb, C, H, Wd, pool, tw, a, y);
+    return cudaGetLastError();
+  };
+  return vec ? launch(channel_softmax_pool_tiled_kernel<T, kVec>)
+             : launch(channel_softmax_pool_tiled_kernel<T, 1>);
+}
+}  // namespace
+
+cudaError_t launch_channel_softmax_pool(int dt, int Nb, int C, int H, int Wd, int pool, const void* a,
+                                        void* y, cudaStream_t st) {
+  if (static_cast<long long>(Nb) * (H / pool) * (Wd / pool) == 0) return cudaSuccess;
+  if (dt == DT_F32)
+    return channel_softmax_pool_typed<float>(Nb, C, H, Wd, pool, static_cast<const float*>(a),
+                                             static_cast<float*>(y), st);
+  return channel_softmax_pool_typed<__nv_bfloat16>(Nb, C, H, Wd, pool,
+                                                   static_cast<const __nv_bfloat16*>(a),
+                                                   static_cast<__nv_bfloat16*>(y), st);
+}
+
 }  // namespace kf

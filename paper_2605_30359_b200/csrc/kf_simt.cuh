@@ -462,4 +462,121 @@ groupnorm_apply_kernel(int Cout, int groups, long long hw, int tiles_per_image, 
   }
 }
 
+// ---------------------------------------------------------------- channel softmax + max-pool
+// Second pass of conv -> softmax over channels -> max-pool.  `a` holds the convolution output
+// NCHW.  One thread per pooled output pixel: for each of the pool x pool input pixels the
+// three-pass softmax over the channel dimension (max, sum of exp, quotient), then per channel
+// the maximum of the window's probabilities.  pool <= 4 (the window's statistics live in
+// registers); the second and third reads of `a` come from cache.
+template <typename T>
+__global__ void __launch_bounds__(256)
+channel_softmax_pool_kernel(int Nb, int C, int H, int Wd, int pool, const T* __restrict__ a,
+                            T* __restrict__ y) {
+  const int Ho = H / pool, Wo = Wd / pool;
+  const long long total = static_cast<long long>(Nb) * Ho * Wo;
+  const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (gid >= total) return;
+  const int j = static_cast<int>(gid % Wo);
+  const int i = static_cast<int>((gid / Wo) % Ho);
+  const long long n = gid / (static_cast<long long>(Wo) * Ho);
+  const long long hw = static_cast<long long>(H) * Wd;
+  const T* an = a + n * C * hw;
+  const int pp = pool * pool;
+  float mx[16], inv[16];
+  for (int q = 0; q < pp; ++q) {
+    const T* px = an + static_cast<long long>(i * pool + q / pool) * Wd + (j * pool + q % pool);
+    float m = -INFINITY;
+    for (int c = 0; c < C; ++c) m = fmaxf(m, to_f32(px[c * hw]));
+    float s = 0.0f;
+    for (int c = 0; c < C; ++c) s += expf(to_f32(px[c * hw]) - m);
+    mx[q] = m;
+    inv[q] = 1.0f / s;
+  }
+  T* yo = y + (n * C * Ho + i) * Wo + j;
+  for (int c = 0; c < C; ++c) {
+    float best = 0.0f;
+    for (int q = 0; q < pp; ++q) {
+      const float v = to_f32(an[c * hw + static_cast<long long>(i * pool + q / pool) * Wd +
+                                (j * pool + q % pool)]);
+      best = fmaxf(best, expf(v - mx[q]) * inv[q]);
+    }
+    yo[static_cast<long long>(c) * Ho * Wo] = from_f32<T>(best);
+  }
+}
+
+// Tiled form of the same pass: one block owns, for one image, one pooled output row and `tw`
+// pooled columns, i.e. a strip of pool rows x tw*pool columns x C channels, held in shared
+// memory as s[c][p] (p = row*tw*pool + column, storage type T).  Phase 1 loads the strip with
+// VEC-element vectors (coalesced along w); phase 2 has one thread per pixel compute the
+// log-sum-exp L over c (max pass, then sum of exp); phase 3 has one thread per (c, pooled
+// column) take the window maximum of z - L and store its exponential: softmax = exp(z - L) and
+// exp is monotone, so one exponential per OUTPUT replaces one per input of the third softmax
+// pass.  The intermediate is read from DRAM exactly once.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256)
+channel_softmax_pool_tiled_kernel(int Nb, int C, int H, int Wd, int pool, int tw,
+                                  const T* __restrict__ a, T* __restrict__ y) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  T* s = reinterpret_cast<T*>(smem_raw);
+  const int Ho = H / pool, Wo = Wd / pool;
+  const int col_tiles = (Wo + tw - 1) / tw;
+  long long b = blockIdx.x;
+  const int jt = static_cast<int>(b % col_tiles); b /= col_tiles;
+  const int i = static_cast<int>(b % Ho);
+  const long long n = b / Ho;
+  const int j0 = jt * tw;
+  const int twb = min(tw, Wo - j0);          // pooled columns this block owns
+  const int rowlen = tw * pool;              // shared-memory row pitch (elements)
+  const int cols = twb * pool;               // valid input columns
+  const int P = pool * rowlen;
+  const long long hw = static_cast<long long>(H) * Wd;
+  const T* src = a + n * C * hw + static_cast<long long>(i) * pool * Wd + static_cast<long long>(j0) * pool;
+
+  // phase 1: strip -> shared memory
+  {
+    const int vrow = cols / VEC;             // VEC divides cols when VEC > 1 (checked by the host)
+    const int per_c = pool * vrow;
+    const int total = C * per_c;
+    for (int idx = threadIdx.x; idx < total; idx += blockDim.x) {
+      const int c = idx / per_c;
+      const int rem = idx - c * per_c;
+      const int r = rem / vrow;
+      const int v = rem - r * vrow;
+      const T* g = src + c * hw + static_cast<long long>(r) * Wd + v * VEC;
+      T* d = s + c * P + r * rowlen + v * VEC;
+      if constexpr (VEC * sizeof(T) == 16) {
+        *reinterpret_cast<uint4*>(d) = __ldg(reinterpret_cast<const uint4*>(g));
+      } else {
+        *d = *g;
+      }
+    }
+  }
+  __syncthreads();
+  // phase 2: per pixel, L = max_c z + log(sum_c exp(z - max)), kept behind the strip
+  float* lse = reinterpret_cast<float*>(
+      smem_raw + ((static_cast<size_t>(C) * P * sizeof(T) + 15) & ~static_cast<size_t>(15)));
+  for (int p = threadIdx.x; p < P; p += blockDim.x) {
+    if (p % rowlen >= cols) continue;
+    float m = -INFINITY;
+    for (int c = 0; c < C; ++c) m = fmaxf(m, to_f32(s[c * P + p]));
+    float sum = 0.0f;
+    for (int c = 0; c < C; ++c) sum += __expf(to_f32(s[c * P + p]) - m);
+    lse[p] = m + __logf(sum);
+  }
+  __syncthreads();
+  // phase 3: exp is monotone, so the window maximum of exp(z - L) is exp(max(z - L))
+  T* yo = y + (n * C * Ho + i) * Wo + j0;
+  for (int idx = threadIdx.x; idx < C * twb; idx += blockDim.x) {
+    const int c = idx / twb;
+    const int jo = idx - c * twb;
+    float best = -INFINITY;
+    for (int r = 0; r < pool; ++r)
+      for (int q = 0; q < pool; ++q) {
+        const int p = r * rowlen + jo * pool + q;
+        best = fmaxf(best, to_f32(s[c * P + p]) - lse[p]);
+      }
+    yo[static_cast<long long>(c) * Ho * Wo + jo] = from_f32<T>(__expf(best));
+  }
+}
+
 }  // namespace kf

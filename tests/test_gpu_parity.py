@@ -346,6 +346,73 @@ def test_groupnorm_biased_variance_on_gpu(kf):
     assert (got[0, 4:, 0, 0] == 0).all()
 
 
+# ------------------------------------------------------------------ conv -> channel softmax -> max-pool
+def run_conv_softmax_pool(kf, d, pool, use_bias=True):
+    bias = d["bias"] if use_bias else None
+    y = kf.conv3x3_softmax_pool(to_dev(d["x"]), to_dev(d["w"]), to_dev(bias), pool)
+    check_status()
+    return to_f64(y), oracle.conv3x3_softmax_pool(d["x"], d["w"], bias, pool)
+
+
+@pytest.mark.parametrize("pool", [1, 2, 4])
+@pytest.mark.parametrize("cfg", [
+    dict(Nb=2, Cin=64, H=8, W=64, Cout=128),       # tensor-core convolution, benchmark geometry
+    dict(Nb=1, Cin=64, H=13, W=64, Cout=96),       # ragged rows: 13 = 3*4 + 1, the rim is dropped
+    dict(Nb=3, Cin=128, H=16, W=32, Cout=16),      # the case study's 16 output channels
+])
+def test_bf16_conv_softmax_pool(kf, cfg, pool):
+    d = ki.conv_inputs(seed=11, groups=0, **cfg)
+    got, ref = run_conv_softmax_pool(kf, d, pool)
+    assert got.shape == (cfg["Nb"], cfg["Cout"], cfg["H"] // pool, cfg["W"] // pool)
+    assert_close(got, ref, 2e-2, 2e-2, "conv softmax pool %s pool %d" % (cfg, pool))
+    # probabilities are ~1/Cout, far below the absolute tolerance: gate them relatively as well
+    # (bf16 staging of the logits and of the result, 2^-9 each)
+    assert_close(got, ref, 1e-6, 2e-2, "relative gate %s pool %d" % (cfg, pool))
+
+
+def test_bf16_conv_softmax_pool_peaked(kf):
+    """Weights x16 make the softmax peaked: winners near 1 and losers near 0 in one image."""
+    d = ki.conv_inputs(seed=12, Nb=2, Cin=64, H=8, W=64, Cout=32, groups=0)
+    d["w"] = ki.store(ki.widen(d["w"]) * 16.0, "bf16")        # exact: a power of two
+    got, ref = run_conv_softmax_pool(kf, d, 2)
+    assert ref.max() > 0.9 and ref.min() < 1e-3
+    assert_close(got, ref, 2e-2, 2e-2, "peaked softmax, official tolerance")
+    # The logits are staged in bf16: each carries a relative rounding of 2^-9, so a probability
+    # (a ratio of exponentials of two logits) moves by up to 2 * 2^-9 * max|logit| relatively,
+    # plus 2^-9 for its own rounding.
+    zmax = np.abs(oracle.conv3x3_gn(d["x"], d["w"], d["bias"], "none", 0)).max()
+    assert_close(got, ref, 1e-6, 2.0 ** -8 * (zmax + 1.0), "peaked softmax, derived relative gate")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("cfg,pool", [(dict(Nb=2, Cin=3, H=5, W=7, Cout=6), 2),
+                                      (dict(Nb=1, Cin=2, H=4, W=9, Cout=1), 3),
+                                      (dict(Nb=2, Cin=4, H=9, W=4, Cout=8), 1),
+                                      (dict(Nb=1, Cin=2, H=3, W=3, Cout=5), 4),    # empty result
+                                      (dict(Nb=1, Cin=2, H=4, W=200, Cout=64), 2),  # two column tiles, ragged
+                                      (dict(Nb=1, Cin=1, H=4, W=8, Cout=2100), 4)])  # strip too big for smem
+def test_conv_softmax_pool_scalar_path(kf, dtype, cfg, pool):
+    d = ki.conv_inputs(seed=13, dtype=dtype, groups=0, **cfg)
+    got, ref = run_conv_softmax_pool(kf, d, pool, use_bias=(cfg["Cout"] != 8))
+    atol, rtol = tol_for(dtype)
+    assert_close(got, ref, atol, rtol, "scalar conv softmax pool %s %s" % (dtype, cfg))
+    if dtype == "f32":
+        assert_close(got, ref, 1e-7, 1e-4, "relative gate")
+    if cfg["Cout"] == 1 and got.size:
+        assert (got == 1.0).all()          # one channel: every probability is exactly 1
+
+
+def test_conv_softmax_pool_errors(kf):
+    import torch
+    x = torch.zeros((1, 2, 8, 8), device="cuda"); w = torch.zeros((2, 2, 3, 3), device="cuda")
+    with pytest.raises(kf.KfError) as e:
+        kf.conv3x3_softmax_pool(x, w, None, 5)
+    assert e.value.status == kf.KF_ERR_UNSUPPORTED
+    with pytest.raises(kf.KfError) as e:
+        kf.conv3x3_softmax_pool(x, w, None, 0)
+    assert e.value.status == kf.KF_ERR_INVALID_ARG
+
+
 # ------------------------------------------------------------------ error handling on the device box
 def test_workspace_errors(kf):
     import torch

@@ -1,4 +1,5 @@
 // Launchers for the CUDA-core kernels.
+#include <type_traits>
 #include "kf_internal.h"
 #include "kf_simt.cuh"
 
@@ -132,7 +133,7 @@ cudaError_t launch_groupnorm_apply(int Nb, int Cout, int groups, long long hw, i
 }
 
 namespace {
-constexpr size_t kPoolStripBytes = 64 * 1024;   // shared-memory strip per block (3 blocks per SM)
+constexpr size_t kPoolStripBytes = 32 * 1024;   // shared-memory strip per block (6 blocks per SM)
 // plus one float per strip pixel for the log-sum-exp: at most kPoolStripBytes / sizeof(T) / C * 4
 
 template <typename T>
@@ -158,19 +159,29 @@ cudaError_t channel_softmax_pool_typed(int Nb, int C, int H, int Wd, int pool, c
     while (t > 0 && ((t * pool) % kVec != 0)) --t;
     if (t > 0 && ((Wo % t) * pool) % kVec == 0) tw = t; else vec = false;
   }
-  const size_t smem = ((static_cast<size_t>(C) * pool * pool * tw * sizeof(T) + 15) & ~static_cast<size_t>(15)) +
-                      static_cast<size_t>(pool) * pool * tw * sizeof(float);
+  const size_t px = static_cast<size_t>(pool) * pool * tw;
+  const size_t smem = ((static_cast<size_t>(C) * px * sizeof(T) + 15) & ~static_cast<size_t>(15)) +
+                      ((px + 3) & ~static_cast<size_t>(3)) * sizeof(float) +
+                      kPoolPartials * sizeof(float2);
   const long long blocks = static_cast<long long>(Nb) * Ho * ((Wo + tw - 1) / tw);
   if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
   auto launch = [&](auto kern) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(kPoolStripBytes * 3 + 16));
+                                         static_cast<int>(kPoolStripBytes * 3 + 8192));
     if (e != cudaSuccess) return e;
-    kern<<<static_cast<unsigned>(blocks), 256, smem, st>>>(Nb, C, H, Wd, pool, tw, a, y);
+    kern<<<static_cast<unsigned>(blocks), 256, smem, st>>>(Nb, C, H, Wd, tw, a, y);
     return cudaGetLastError();
   };
-  return vec ? launch(channel_softmax_pool_tiled_kernel<T, kVec>)
-             : launch(channel_softmax_pool_tiled_kernel<T, 1>);
+  auto by_pool = [&](auto vec_tag) -> cudaError_t {
+    constexpr int V = decltype(vec_tag)::value;
+    switch (pool) {
+      case 1: return launch(channel_softmax_pool_tiled_kernel<T, V, 1>);
+      case 2: return launch(channel_softmax_pool_tiled_kernel<T, V, 2>);
+      case 3: return launch(channel_softmax_pool_tiled_kernel<T, V, 3>);
+      default: return launch(channel_softmax_pool_tiled_kernel<T, V, 4>);
+    }
+  };
+  return vec ? by_pool(std::integral_constant<int, kVec>{}) : by_pool(std::integral_constant<int, 1>{});
 }
 }  // namespace
 

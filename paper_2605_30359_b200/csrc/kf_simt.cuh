@@ -504,21 +504,64 @@ channel_softmax_pool_kernel(int Nb, int C, int H, int Wd, int pool, const T* __r
   }
 }
 
+// 2^x in one MUFU op (relative error about 2^-22; flushes results below 2^-126 to zero).
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Helpers of the tiled pass: N adjacent elements of shared memory as floats, with the widest
+// load the alignment allows (the caller guarantees alignment to N * sizeof(T) when that is a
+// power of two).
+template <int N>
+__device__ __forceinline__ void ld_row(const float* p, float (&o)[N]) {
+  if constexpr (N == 4) {
+    const float4 v = *reinterpret_cast<const float4*>(p);
+    o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+  } else if constexpr (N == 2) {
+    const float2 v = *reinterpret_cast<const float2*>(p);
+    o[0] = v.x; o[1] = v.y;
+  } else {
+#pragma unroll
+    for (int i = 0; i < N; ++i) o[i] = p[i];
+  }
+}
+template <int N>
+__device__ __forceinline__ void ld_row(const __nv_bfloat16* p, float (&o)[N]) {
+  if constexpr (N == 4) {
+    const uint2 v = *reinterpret_cast<const uint2*>(p);
+    o[0] = __uint_as_float(v.x << 16); o[1] = __uint_as_float(v.x & 0xffff0000u);
+    o[2] = __uint_as_float(v.y << 16); o[3] = __uint_as_float(v.y & 0xffff0000u);
+  } else if constexpr (N == 2) {
+    const uint32_t v = *reinterpret_cast<const uint32_t*>(p);
+    o[0] = __uint_as_float(v << 16); o[1] = __uint_as_float(v & 0xffff0000u);
+  } else {
+#pragma unroll
+    for (int i = 0; i < N; ++i) o[i] = __bfloat162float(p[i]);
+  }
+}
+
 // Tiled form of the same pass: one block owns, for one image, one pooled output row and `tw`
-// pooled columns, i.e. a strip of pool rows x tw*pool columns x C channels, held in shared
-// memory as s[c][p] (p = row*tw*pool + column, storage type T).  Phase 1 loads the strip with
-// VEC-element vectors (coalesced along w); phase 2 has one thread per pixel compute the
-// log-sum-exp L over c (max pass, then sum of exp); phase 3 has one thread per (c, pooled
-// column) take the window maximum of z - L and store its exponential: softmax = exp(z - L) and
-// exp is monotone, so one exponential per OUTPUT replaces one per input of the third softmax
-// pass.  The intermediate is read from DRAM exactly once.
-template <typename T, int VEC>
+// pooled columns, i.e. a strip of POOL rows x tw*POOL columns x C channels, held in shared
+// memory as s[c][p] (p = row*tw*POOL + column, storage type T).
+//   phase 1  loads the strip with VEC-element vectors (coalesced along w);
+//   phase 2  computes per pixel the log-sum-exp L over c: a thread owns two adjacent pixels and
+//            a slice of the channels (max pass, then sum of exp2), slices are merged through
+//            shared memory; strips with an odd row pitch take one thread per pixel instead;
+//   phase 3  has one thread per (c, pooled column) take the window maximum of z - L and store
+//            its exponential: softmax = exp(z - L) and exp is monotone, so one exponential per
+//            OUTPUT replaces one per input of the third softmax pass.
+// The intermediate is read from DRAM exactly once.  Shared memory: the strip, P floats of L,
+// and up to 512 float2 of per-slice partials.
+constexpr int kPoolPartials = 512;
+template <typename T, int VEC, int POOL>
 __global__ void __launch_bounds__(256)
-channel_softmax_pool_tiled_kernel(int Nb, int C, int H, int Wd, int pool, int tw,
-                                  const T* __restrict__ a, T* __restrict__ y) {
+channel_softmax_pool_tiled_kernel(int Nb, int C, int H, int Wd, int tw, const T* __restrict__ a,
+                                  T* __restrict__ y) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   T* s = reinterpret_cast<T*>(smem_raw);
-  const int Ho = H / pool, Wo = Wd / pool;
+  const int Ho = H / POOL, Wo = Wd / POOL;
   const int col_tiles = (Wo + tw - 1) / tw;
   long long b = blockIdx.x;
   const int jt = static_cast<int>(b % col_tiles); b /= col_tiles;
@@ -526,56 +569,156 @@ channel_softmax_pool_tiled_kernel(int Nb, int C, int H, int Wd, int pool, int tw
   const long long n = b / Ho;
   const int j0 = jt * tw;
   const int twb = min(tw, Wo - j0);          // pooled columns this block owns
-  const int rowlen = tw * pool;              // shared-memory row pitch (elements)
-  const int cols = twb * pool;               // valid input columns
-  const int P = pool * rowlen;
+  const int rowlen = tw * POOL;              // shared-memory row pitch (elements)
+  const int cols = twb * POOL;               // valid input columns
+  const int P = POOL * rowlen;
   const long long hw = static_cast<long long>(H) * Wd;
-  const T* src = a + n * C * hw + static_cast<long long>(i) * pool * Wd + static_cast<long long>(j0) * pool;
+  const T* src = a + n * C * hw + static_cast<long long>(i) * POOL * Wd + static_cast<long long>(j0) * POOL;
+  float* lse = reinterpret_cast<float*>(
+      smem_raw + ((static_cast<size_t>(C) * P * sizeof(T) + 15) & ~static_cast<size_t>(15)));
+  float2* part = reinterpret_cast<float2*>(lse + ((P + 3) & ~3));
+  const int tid = threadIdx.x;
 
-  // phase 1: strip -> shared memory
+  // phase 1: strip -> shared memory.  When one channel's POOL row segments take at most 256
+  // vectors, a thread keeps its (row, vector) slot and strides over channels: one load, one
+  // store and two pointer bumps per vector.  Otherwise threads form a (rows x vectors) grid.
   {
     const int vrow = cols / VEC;             // VEC divides cols when VEC > 1 (checked by the host)
-    const int per_c = pool * vrow;
-    const int total = C * per_c;
-    for (int idx = threadIdx.x; idx < total; idx += blockDim.x) {
-      const int c = idx / per_c;
-      const int rem = idx - c * per_c;
-      const int r = rem / vrow;
-      const int v = rem - r * vrow;
-      const T* g = src + c * hw + static_cast<long long>(r) * Wd + v * VEC;
-      T* d = s + c * P + r * rowlen + v * VEC;
-      if constexpr (VEC * sizeof(T) == 16) {
-        *reinterpret_cast<uint4*>(d) = __ldg(reinterpret_cast<const uint4*>(g));
-      } else {
-        *d = *g;
+    const int per_c = POOL * vrow;
+    if (per_c <= 256) {
+      const int cstep = 256 / per_c;
+      const int c_first = tid / per_c;
+      const int rv = tid - c_first * per_c;
+      const int r = rv / vrow, v = rv - r * vrow;
+      if (c_first < cstep) {
+        const T* g = src + c_first * hw + static_cast<long long>(r) * Wd + v * VEC;
+        T* d = s + c_first * P + r * rowlen + v * VEC;
+        const long long gstep = cstep * hw;
+        const int dstep = cstep * P;
+#pragma unroll 4
+        for (int c = c_first; c < C; c += cstep, g += gstep, d += dstep) {
+          if constexpr (VEC * sizeof(T) == 16) {
+            *reinterpret_cast<uint4*>(d) = __ldg(reinterpret_cast<const uint4*>(g));
+          } else {
+            *d = *g;
+          }
+        }
+      }
+    } else {
+      int vl = 1;
+      while (vl < vrow && vl < 256) vl <<= 1;
+      const int v0 = tid & (vl - 1);
+      const int rstep = 256 / vl;
+      for (int row = tid / vl; row < C * POOL; row += rstep) {
+        const int c = row / POOL, r = row - c * POOL;
+        const T* g = src + c * hw + static_cast<long long>(r) * Wd;
+        T* d = s + c * P + r * rowlen;
+        for (int v = v0; v < vrow; v += vl) {
+          if constexpr (VEC * sizeof(T) == 16) {
+            *reinterpret_cast<uint4*>(d + v * VEC) = __ldg(reinterpret_cast<const uint4*>(g + v * VEC));
+          } else {
+            d[v] = g[v];
+          }
+        }
       }
     }
   }
   __syncthreads();
-  // phase 2: per pixel, L = max_c z + log(sum_c exp(z - max)), kept behind the strip
-  float* lse = reinterpret_cast<float*>(
-      smem_raw + ((static_cast<size_t>(C) * P * sizeof(T) + 15) & ~static_cast<size_t>(15)));
-  for (int p = threadIdx.x; p < P; p += blockDim.x) {
-    if (p % rowlen >= cols) continue;
-    float m = -INFINITY;
-    for (int c = 0; c < C; ++c) m = fmaxf(m, to_f32(s[c * P + p]));
-    float sum = 0.0f;
-    for (int c = 0; c < C; ++c) sum += __expf(to_f32(s[c * P + p]) - m);
-    lse[p] = m + __logf(sum);
+
+  // phase 2: L[p] = max_c z + log(sum_c exp(z - max))
+  constexpr float kLog2e = 1.4426950408889634f;
+  if ((rowlen & 1) == 0) {
+    const int NP = P / 2;
+    const int slices = NP >= 256 ? 1 : 256 / NP;
+    const int cs = (C + slices - 1) / slices;
+    for (int wi = tid; wi < NP * slices; wi += 256) {
+      const int slice = wi / NP;
+      const int p = 2 * (wi - slice * NP);
+      const int c0 = slice * cs, c1 = min(C, c0 + cs);
+      const T* col = s + p;
+      float m0 = -INFINITY, m1 = -INFINITY;
+      if constexpr (sizeof(T) == 2) {
+        __nv_bfloat162 mm = __floats2bfloat162_rn(-INFINITY, -INFINITY);
+#pragma unroll 8
+        for (int c = c0; c < c1; ++c)
+          mm = __hmax2(mm, *reinterpret_cast<const __nv_bfloat162*>(col + c * P));
+        m0 = __low2float(mm); m1 = __high2float(mm);
+      } else {
+#pragma unroll 8
+        for (int c = c0; c < c1; ++c) {
+          float v[2];
+          ld_row<2>(col + c * P, v);
+          m0 = fmaxf(m0, v[0]); m1 = fmaxf(m1, v[1]);
+        }
+      }
+      const float b0 = -m0 * kLog2e, b1 = -m1 * kLog2e;
+      float s0 = 0.0f, s1 = 0.0f;
+#pragma unroll 8
+      for (int c = c0; c < c1; ++c) {
+        float v[2];
+        ld_row<2>(col + c * P, v);
+        s0 += ex2_approx(fmaf(v[0], kLog2e, b0));
+        s1 += ex2_approx(fmaf(v[1], kLog2e, b1));
+      }
+      if (slices == 1) {
+        lse[p] = m0 + __logf(s0);
+        lse[p + 1] = m1 + __logf(s1);
+      } else {
+        part[slice * P + p] = make_float2(m0, s0);
+        part[slice * P + p + 1] = make_float2(m1, s1);
+      }
+    }
+    if (slices > 1) {
+      __syncthreads();
+      for (int p = tid; p < P; p += 256) {
+        float m = -INFINITY;
+        for (int k = 0; k < slices; ++k) m = fmaxf(m, part[k * P + p].x);
+        float sum = 0.0f;
+        for (int k = 0; k < slices; ++k) {
+          const float2 q = part[k * P + p];
+          sum += q.y * ex2_approx((q.x - m) * kLog2e);     // an empty slice holds (-inf, 0): adds 0
+        }
+        lse[p] = m + __logf(sum);
+      }
+    }
+  } else {
+    for (int p = tid; p < P; p += 256) {
+      if (p % rowlen >= cols) continue;
+      float m = -INFINITY;
+      for (int c = 0; c < C; ++c) m = fmaxf(m, to_f32(s[c * P + p]));
+      float sum = 0.0f;
+      for (int c = 0; c < C; ++c) sum += ex2_approx((to_f32(s[c * P + p]) - m) * kLog2e);
+      lse[p] = m + __logf(sum);
+    }
   }
   __syncthreads();
-  // phase 3: exp is monotone, so the window maximum of exp(z - L) is exp(max(z - L))
-  T* yo = y + (n * C * Ho + i) * Wo + j0;
-  for (int idx = threadIdx.x; idx < C * twb; idx += blockDim.x) {
-    const int c = idx / twb;
-    const int jo = idx - c * twb;
-    float best = -INFINITY;
-    for (int r = 0; r < pool; ++r)
-      for (int q = 0; q < pool; ++q) {
-        const int p = r * rowlen + jo * pool + q;
-        best = fmaxf(best, to_f32(s[c * P + p]) - lse[p]);
+
+  // phase 3: window maxima of z - L, one exponential per output.  A thread keeps one pooled
+  // column (its window's L values stay in registers) and strides over channels; the column
+  // extent of the thread grid is the power of two covering twb, so no index needs a division.
+  {
+    int tl = 1;
+    while (tl < twb && tl < 256) tl <<= 1;
+    const int cstep = 256 / tl;
+    T* yo = y + (n * C * Ho + i) * Wo + j0;
+    for (int jo = tid & (tl - 1); jo < twb; jo += tl) {
+      float l[POOL][POOL];
+#pragma unroll
+      for (int r = 0; r < POOL; ++r) ld_row<POOL>(lse + r * rowlen + jo * POOL, l[r]);
+      const T* zc = s + jo * POOL;
+#pragma unroll 2
+      for (int c = tid / tl; c < C; c += cstep) {
+        float best = -INFINITY;
+#pragma unroll
+        for (int r = 0; r < POOL; ++r) {
+          float z[POOL];
+          ld_row<POOL>(zc + c * P + r * rowlen, z);
+#pragma unroll
+          for (int q = 0; q < POOL; ++q) best = fmaxf(best, z[q] - l[r][q]);
+        }
+        yo[static_cast<long long>(c) * Ho * Wo + jo] = from_f32<T>(ex2_approx(best * kLog2e));
       }
-    yo[static_cast<long long>(c) * Ho * Wo + jo] = from_f32<T>(__expf(best));
+    }
   }
 }
 

@@ -361,8 +361,14 @@ def run_single_workload(args, kf, device, peaks):
         "c4": (2.0 * 16384 * 1024 * 1024, 2 * (16384 * 1024 + 1024 * 1024 + 1024) + 4 * 16384),
         "c5": (2.0 * 128 * 64 * 64 * 128 * 576, 2 * (128 * 64 * 64 * 64 + 128 * 64 * 9 + 128 + 128 * 128 * 64 * 64)),
     }
+    specs["pool"] = (specs["c5"][0], 2 * (128 * 64 * 64 * 64 + 128 * 64 * 9 + 128 + 128 * 128 * 16 * 16))
     flops, nbytes = specs[name]
-    if name == "c5":
+    if name == "pool":      # conv3x3 -> channel softmax -> max-pool 4 on config 5's tensors
+        d = ki.conv_inputs("c5", seed=0)
+        t = {k: to_dev(d[k], device) for k in ("x", "w", "bias")}
+        o = torch.empty(128, 128, 16, 16, dtype=torch.bfloat16, device=device)
+        fn = lambda: kf.conv3x3_softmax_pool(t["x"], t["w"], t["bias"], 4, out=o)
+    elif name == "c5":
         d = ki.conv_inputs("c5", seed=0)
         t = {k: to_dev(d[k], device) for k in ("x", "w", "bias")}
         o = torch.empty(128, 128, 64, 64, dtype=torch.bfloat16, device=device)
@@ -396,8 +402,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the context table and baselines")
-    ap.add_argument("--workload", default=WORKLOAD, choices=["c1", "c2", "c3", "c4", "c5"],
-                    help="c2 is the headline; the others print a reduced line (profiling aid)")
+    ap.add_argument("--workload", default=WORKLOAD, choices=["c1", "c2", "c3", "c4", "c5", "pool"],
+                    help="c2 is the headline; the others print a reduced line (profiling aid); "
+                         "pool = conv3x3 -> channel softmax -> max-pool on config 5's tensors")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 

@@ -394,6 +394,120 @@ def run_single_workload(args, kf, device, peaks):
                       "config": {"workload": name}, "data": "synthetic"}))
 
 
+# ------------------------------------------------------------------ shape sweep (the paper's metrics)
+# Synthetic shapes in the four categories of the paper's Table 2 (matmul-centered, mixed
+# reduction, reduction-dominated, conv-centered); none is an item of the paper's benchmark suite.
+SWEEP_GEMM = [  # (dtype, M, N, K, act, scale, residual)
+    ("bf16", 128, 1024, 1024, "relu", 1.0, False), ("bf16", 512, 512, 512, "gelu_tanh", 1.0, False),
+    ("bf16", 1024, 4096, 1024, "swish", 1.0, True), ("bf16", 2048, 2048, 2048, "gelu_erf", 0.5, True),
+    ("bf16", 4096, 4096, 4096, "sigmoid", 1.0, False), ("bf16", 8192, 1024, 8192, "tanh", 2.0, False),
+    ("bf16", 16384, 512, 512, "relu", 1.0, True), ("bf16", 1000, 1000, 1000, "gelu_tanh", 1.0, False),
+    ("bf16", 4096, 11008, 4096, "swish", 1.0, False), ("bf16", 333, 777, 520, "hardtanh", 1.0, True),
+    ("bf16", 8192, 4096, 4096, "chain95", 1.0, False), ("bf16", 64, 8192, 8192, "none", 1.0, False),
+    ("f32", 128, 256, 512, "relu", 1.0, False), ("f32", 64, 64, 64, "gelu_tanh", 1.0, False),
+    ("f32", 512, 512, 256, "sigmoid", 1.0, True),
+]
+SWEEP_ROWRED = [  # (M, N, K, pre_act, red)
+    (1024, 1024, 1024, "none", "softmax"), (4096, 8192, 2048, "none", "softmax"),
+    (512, 32000, 1024, "none", "softmax"), (8192, 512, 512, "relu", "softmax"),
+    (100, 1000, 304, "none", "softmax"),
+    (16384, 1024, 1024, "sigmoid", "sum"), (4096, 4096, 1024, "gelu_tanh", "sum"),
+    (1024, 512, 2048, "sigmoid", "sum"), (65536, 256, 256, "relu", "sum"),
+]
+SWEEP_CONV = [  # (Nb, Cin, H, W, Cout, groups [GroupNorm] or -pool [softmax + max-pool])
+    (16, 64, 32, 32, 64, 8), (128, 64, 64, 64, 128, 32), (32, 128, 32, 32, 128, 16),
+    (8, 64, 128, 128, 64, 4), (64, 64, 16, 16, 256, 32), (10, 3, 30, 30, 16, 4),
+    (128, 64, 64, 64, 128, -4), (16, 64, 32, 32, 16, -2),
+]
+
+
+def _torch_act(name):
+    import torch
+    import torch.nn.functional as F
+    return {"none": lambda z: z, "relu": torch.relu, "gelu_tanh": lambda z: F.gelu(z, approximate="tanh"),
+            "gelu_erf": F.gelu, "sigmoid": torch.sigmoid, "swish": lambda z: torch.sigmoid(z) * z,
+            "tanh": torch.tanh, "hardtanh": lambda z: F.hardtanh(z, -1.0, 1.0),
+            "chain95": lambda z: F.hardtanh(F.gelu(torch.tanh(torch.sigmoid(z) * z)), -1.0, 1.0)}[name]
+
+
+def run_sweep(kf, device):
+    """Speedup of every sweep shape over the same chain as separate eager torch ops, and the
+    paper's summary metrics (Section 4.1): fast_1 = share of shapes with speedup > 1, average
+    and geometric-mean speedup.  Timing only; parity of these kernels is the tests' job."""
+    import torch
+    import torch.nn.functional as F
+    torch.backends.cuda.matmul.allow_tf32 = False
+    torch.backends.cudnn.allow_tf32 = False
+    g = torch.Generator(device=device).manual_seed(0)
+    rnd = lambda shape, dt, sc=1.0: (torch.randn(shape, generator=g, device=device) * sc).to(dt)
+    rows = []
+
+    def record(cat, name, fn, ref, flops):
+        big = flops > 2e9
+        us = time_calls(fn, 30 if big else 200, 5, graph_batch=0 if big else 20)
+        ut = time_calls(ref, 20 if big else 200, 5, graph_batch=0 if big else 20)
+        rows.append({"category": cat, "shape": name, "us": round(us, 2), "torch_us": round(ut, 2),
+                     "speedup": round(ut / us, 3), "tflops": round(flops / us / 1e6, 1)})
+
+    for dtn, M, N, K, act, scale, res in SWEEP_GEMM:
+        dt = torch.bfloat16 if dtn == "bf16" else torch.float32
+        X, W, b = rnd((M, K), dt), rnd((N, K), dt, K ** -0.5), rnd((N,), dt, K ** -0.5)
+        R = rnd((M, N), dt) if res else None
+        out = torch.empty((M, N), dtype=dt, device=device)
+        ta = _torch_act(act)
+
+        def ref(X=X, W=W, b=b, R=R, ta=ta, scale=scale):
+            y = ta(F.linear(X, W, b))
+            if scale != 1.0:
+                y = y * scale
+            return y + R if R is not None else y
+
+        record("matmul-centered", "%s %dx%dx%d %s%s%s" % (dtn, M, N, K, act, "*s" if scale != 1.0 else "",
+                                                           "+R" if res else ""),
+               lambda X=X, W=W, b=b, R=R, out=out, act=act, scale=scale:
+               kf.gemm_epilogue(X, W, b, act, scale, R, out=out), ref, 2.0 * M * N * K)
+        del X, W, b, R, out
+    for M, N, K, pre, red in SWEEP_ROWRED:
+        dt = torch.bfloat16
+        X, W, b = rnd((M, K), dt), rnd((N, K), dt, K ** -0.5), rnd((N,), dt, K ** -0.5)
+        ta = _torch_act(pre)
+        if red == "softmax":
+            out = torch.empty((M, N), dtype=dt, device=device)
+            ref = lambda X=X, W=W, b=b, ta=ta: torch.softmax(ta(F.linear(X, W, b)), dim=1)
+            cat = "mixed-reduction"
+        else:
+            out = torch.empty((M,), dtype=torch.float32, device=device)
+            ref = lambda X=X, W=W, b=b, ta=ta: ta(F.linear(X, W, b)).sum(dim=1, dtype=torch.float32)
+            cat = "reduction-dominated"
+        record(cat, "bf16 %dx%dx%d %s->%s" % (M, N, K, pre, red),
+               lambda X=X, W=W, b=b, out=out, pre=pre, red=red: kf.gemm_rowreduce(X, W, b, pre, red, out=out),
+               ref, 2.0 * M * N * K)
+        del X, W, b, out
+    for Nb, Cin, H, Wd, Cout, gp in SWEEP_CONV:
+        dt = torch.bfloat16
+        x, w, b = rnd((Nb, Cin, H, Wd), dt), rnd((Cout, Cin, 3, 3), dt, (9 * Cin) ** -0.5), rnd((Cout,), dt, 0.1)
+        flops = 2.0 * Nb * H * Wd * Cout * Cin * 9
+        if gp > 0:
+            out = torch.empty((Nb, Cout, H, Wd), dtype=dt, device=device)
+            record("conv-centered", "bf16 conv %dx%dx%dx%d->%d relu GN%d" % (Nb, Cin, H, Wd, Cout, gp),
+                   lambda x=x, w=w, b=b, out=out, gp=gp: kf.conv3x3_epilogue(x, w, b, "relu", gp, 1e-5, out=out),
+                   lambda x=x, w=w, b=b, gp=gp: F.group_norm(torch.relu(F.conv2d(x, w, b, padding=1)), gp, eps=1e-5),
+                   flops)
+        else:
+            pool = -gp
+            out = torch.empty((Nb, Cout, H // pool, Wd // pool), dtype=dt, device=device)
+            record("conv-centered", "bf16 conv %dx%dx%dx%d->%d softmax pool%d" % (Nb, Cin, H, Wd, Cout, pool),
+                   lambda x=x, w=w, b=b, out=out, pool=pool: kf.conv3x3_softmax_pool(x, w, b, pool, out=out),
+                   lambda x=x, w=w, b=b, pool=pool: F.max_pool2d(torch.softmax(F.conv2d(x, w, b, padding=1), dim=1), pool),
+                   flops)
+        del x, w, b, out
+    sp = np.array([r["speedup"] for r in rows])
+    summary = {"shapes": len(rows), "fast_1": round(float((sp > 1.0).mean()), 3),
+               "avg_speedup": round(float(sp.mean()), 3),
+               "geomean_speedup": round(float(np.exp(np.log(sp).mean())), 3), "min_speedup": float(sp.min())}
+    print(json.dumps({"metric": "speedup_over_unfused_torch", "summary": summary, "rows": rows,
+                      "data": "synthetic", "config": {"workload": "sweep"}}))
+
 # ------------------------------------------------------------------ main
 def main():
     ap = argparse.ArgumentParser()
@@ -405,6 +519,8 @@ def main():
     ap.add_argument("--workload", default=WORKLOAD, choices=["c1", "c2", "c3", "c4", "c5", "pool"],
                     help="c2 is the headline; the others print a reduced line (profiling aid); "
                          "pool = conv3x3 -> channel softmax -> max-pool on config 5's tensors")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time every sweep shape against unfused torch; prints fast_1 / avg / geomean")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -428,6 +544,10 @@ def main():
     import paper_2605_30359_b200 as kf   # raises if libkf.so is missing
     kf.lib()
     peaks = load_peaks()
+    if args.sweep:
+        if rank == 0:
+            run_sweep(kf, device)
+        return
     if args.workload != WORKLOAD:
         if rank == 0:
             run_single_workload(args, kf, device, peaks)

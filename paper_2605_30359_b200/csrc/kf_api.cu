@@ -158,6 +158,19 @@ size_t rowreduce_umma_ws(int64_t M, int64_t N, int red) {
 // CTA pairs (256-row tiles, each CTA loading half of the W tile) pay off when the K loop is
 // long: measured +3.6 % at K = 4096, +3.3 % at K = 2048, -4 % at K = 1024 (fewer, larger tiles
 // make the last wave's tail longer).  KF_NO_PAIR=1 forces one CTA per tile for A/B runs.
+// Tile width of the elementwise chain.  Problems of more than one wave take the widest tile
+// that N fills (the cost of a tcgen05.mma hardly falls with N, so wide tiles feed the tensor
+// pipe best); problems that fit in one wave take the narrowest tile that still fits in one
+// wave, which spreads them over the most SMs.
+int pick_tile_n(int64_t M, int64_t N, int sm_count) {
+  const int64_t tm = (M + kBM - 1) / kBM;
+  const int cover = N <= 32 ? 32 : (N <= 64 ? 64 : (N <= 128 ? 128 : 256));
+  if (tm * ((N + 255) / 256) > sm_count) return cover;
+  for (int bn = 32; bn < cover; bn *= 2)
+    if (tm * ((N + bn - 1) / bn) <= sm_count) return bn;
+  return cover;
+}
+
 bool use_cta_pairs(int64_t M, int64_t K) {
   return M > 256 && K >= 2048 && getenv("KF_NO_PAIR") == nullptr;
 }
@@ -232,7 +245,7 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
   if (umma_gemm_ok(io_dtype, K, X, ldx, W, ldw)) {
-    const int bn = N <= 128 ? 128 : 256;
+    const int bn = pick_tile_n(M, N, d->sm_count);
     const bool pair = bn == 256 && use_cta_pairs(M, K);
     UmmaMaps tm;
     if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, pair ? bn / 2 : bn))

@@ -381,50 +381,64 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
           }
         } else {
+          // Output (or residual) rows that do not start on 16 bytes: no TMA.  Pieces still go
+          // through shared memory so that global accesses run along rows: a warp moves 32 rows,
+          // its lanes one bf16 column each (64 contiguous bytes per row and instruction).
+          const int er = et >> 5;                      // this warp's row group in the copy loops
 #pragma unroll 1
           for (int c = 0; c < PIECES; ++c) {
             if (c * 32 >= n_valid) break;
+            const int n0 = n_tile + c * 32;
+            const bool col_ok = n0 + lane < p.N;
+            uint8_t* rb = rbuf;
+            uint8_t* yb = ybuf;
+            if (has_r) {
+#pragma unroll 4
+              for (int i = 0; i < 32; ++i) {
+                const int r = i * 4 + er;
+                const long long mr = static_cast<long long>(m_cta) + r;
+                __nv_bfloat16 rv = __float2bfloat16_rn(0.0f);
+                if (col_ok && mr < p.M) rv = p.R[mr * p.ldr + n0 + lane];
+                *reinterpret_cast<__nv_bfloat16*>(rb + piece_off(r, lane >> 3) + (lane & 7) * 2) = rv;
+              }
+              named_barrier_sync(2, kEpiThreads);
+            }
             uint32_t v[32];
             tmem_ld_32x32(t_acc + c * 32, v);
             float bs[32];
-            load_bias32(p, n_tile + c * 32, bs);
+            load_bias32(p, n0, bs);
             tmem_ld_wait();
             float f[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j)
               f[j] = p.scale * act_f<ACT, true>(__uint_as_float(v[j]) + bs[j]);
-            if (row_ok) {
-              const int n0 = n_tile + c * 32;
-              if (p.vec_ok && c * 32 + 32 <= n_valid) {
-                if (p.R != nullptr) {
-                  const uint4* rp = reinterpret_cast<const uint4*>(p.R + m * p.ldr + n0);
+            if (has_r) {
 #pragma unroll
-                  for (int q = 0; q < 4; ++q) {
-                    const uint4 r4 = __ldg(rp + q);
-                    f[8 * q + 0] += bf16_lo(r4.x); f[8 * q + 1] += bf16_hi(r4.x);
-                    f[8 * q + 2] += bf16_lo(r4.y); f[8 * q + 3] += bf16_hi(r4.y);
-                    f[8 * q + 4] += bf16_lo(r4.z); f[8 * q + 5] += bf16_hi(r4.z);
-                    f[8 * q + 6] += bf16_lo(r4.w); f[8 * q + 7] += bf16_hi(r4.w);
-                  }
-                }
-                uint4* yp = reinterpret_cast<uint4*>(Y + m * p.ldo + n0);
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                  yp[q] = make_uint4(pack_bf16x2(f[8 * q + 0], f[8 * q + 1]),
-                                     pack_bf16x2(f[8 * q + 2], f[8 * q + 3]),
-                                     pack_bf16x2(f[8 * q + 4], f[8 * q + 5]),
-                                     pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
-              } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                  if (c * 32 + j < n_valid) {
-                    float y = f[j];
-                    if (p.R != nullptr) y += __bfloat162float(p.R[m * p.ldr + n0 + j]);
-                    Y[m * p.ldo + n0 + j] = __float2bfloat16_rn(y);
-                  }
-                }
+              for (int q = 0; q < 4; ++q) {
+                const uint4 r4 = *reinterpret_cast<const uint4*>(rb + piece_off(row, q));
+                f[8 * q + 0] += bf16_lo(r4.x); f[8 * q + 1] += bf16_hi(r4.x);
+                f[8 * q + 2] += bf16_lo(r4.y); f[8 * q + 3] += bf16_hi(r4.y);
+                f[8 * q + 4] += bf16_lo(r4.z); f[8 * q + 5] += bf16_hi(r4.z);
+                f[8 * q + 6] += bf16_lo(r4.w); f[8 * q + 7] += bf16_hi(r4.w);
               }
             }
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              *reinterpret_cast<uint4*>(yb + piece_off(row, q)) =
+                  make_uint4(pack_bf16x2(f[8 * q + 0], f[8 * q + 1]),
+                             pack_bf16x2(f[8 * q + 2], f[8 * q + 3]),
+                             pack_bf16x2(f[8 * q + 4], f[8 * q + 5]),
+                             pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
+            named_barrier_sync(2, kEpiThreads);
+#pragma unroll 4
+            for (int i = 0; i < 32; ++i) {
+              const int r = i * 4 + er;
+              const long long mr = static_cast<long long>(m_cta) + r;
+              if (col_ok && mr < p.M)
+                Y[mr * p.ldo + n0 + lane] =
+                    *reinterpret_cast<const __nv_bfloat16*>(yb + piece_off(r, lane >> 3) + (lane & 7) * 2);
+            }
+            named_barrier_sync(2, kEpiThreads);        // buffers free for the next piece
           }
           release_acc();
         }

@@ -14,6 +14,8 @@ cudaError_t launch_umma_elementwise(int bn, int act, int pair, const UmmaMaps& t
     } else {
       if (bn == 256) e = launch_umma_instance<256, EPI_ELEMENTWISE, ACT, __nv_bfloat16>(tm, p, grid, st);
       else if (bn == 128) e = launch_umma_instance<128, EPI_ELEMENTWISE, ACT, __nv_bfloat16>(tm, p, grid, st);
+      else if (bn == 64) e = launch_umma_instance<64, EPI_ELEMENTWISE, ACT, __nv_bfloat16>(tm, p, grid, st);
+      else if (bn == 32) e = launch_umma_instance<32, EPI_ELEMENTWISE, ACT, __nv_bfloat16>(tm, p, grid, st);
     }
   });
   return e;

@@ -95,6 +95,22 @@ def test_bf16_gemm_shapes(kf, shape):
     assert_close(got, ref, 2e-2, 2e-2, "bf16 %s" % (shape,))
 
 
+# One-wave problems take the narrowest tile that keeps them in one wave (32, 64, 128 or 256
+# columns); rows of Y / R that do not start on 16 bytes take the epilogue without TMA.
+@pytest.mark.parametrize("shape", [(1024, 1000, 64),      # 64-column tiles
+                                   (2048, 777, 72),       # 128-column tiles, unaligned rows
+                                   (2304, 1030, 64),      # 256-column tiles, unaligned rows
+                                   (333, 777, 520),       # 32-column tiles, unaligned rows
+                                   (128, 33, 8)])         # one tile, one ragged piece + 1 column
+def test_bf16_gemm_tile_widths_and_unaligned_rows(kf, shape):
+    M, N, K = shape
+    d = ki.gemm_inputs("c2", seed=21, M=M, N=N, K=K)
+    got, ref = run_gemm(kf, d, "swish", 2.0)
+    assert_close(got, ref, 2e-2, 2e-2, "bf16 %s" % (shape,))
+    got, ref = run_gemm(kf, d, "none", 1.0, use_bias=False, use_res=False)
+    assert_close(got, ref, 2e-2, 2e-2, "bf16 bare %s" % (shape,))
+
+
 # K >= 2048 with more than 256 rows takes the CTA-pair kernel (256-row tiles over two SMs)
 @pytest.mark.parametrize("shape", [(384, 520, 2048), (257, 256, 2112), (1000, 264, 2048)])
 def test_bf16_gemm_cta_pair_kernel(kf, shape):

@@ -171,6 +171,22 @@ int pick_tile_n(int64_t M, int64_t N, int sm_count) {
   return cover;
 }
 
+// Cluster size of the split-K kernel, or 0.  Measured on B200: a narrow-tile CTA spends about
+// 0.28 us per K block whatever the tile width, the cluster exchange costs about 4 us, so
+// splitting pays from about 24 K blocks; clusters of 8 schedule well only while there are few
+// of them (16 clusters of 8 already ran in two waves).
+int pick_split_k(int64_t M, int64_t N, int64_t K, int sm_count, int* bn_out) {
+  if (getenv("KF_NO_SPLITK") != nullptr) return 0;
+  const int bn = N <= 128 ? 128 : 256;
+  const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + bn - 1) / bn);
+  const int64_t kb = (K + kBK - 1) / kBK;
+  *bn_out = bn;
+  if (kb < 24) return 0;
+  if (bn == 256 && kb >= 32 && tiles * 8 <= 64) return 8;
+  if (tiles * 4 <= sm_count - sm_count % 4) return 4;
+  return 0;
+}
+
 bool use_cta_pairs(int64_t M, int64_t K) {
   return M > 256 && K >= 2048 && getenv("KF_NO_PAIR") == nullptr;
 }
@@ -244,6 +260,33 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
   if (!device_info(&d)) return KF_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
+  int bn_split = 0;
+  const int split = umma_gemm_ok(io_dtype, K, X, ldx, W, ldw)
+                        ? pick_split_k(M, N, K, d->sm_count, &bn_split) : 0;
+  if (split > 0) {
+    UmmaMaps tm;
+    if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, bn_split))
+      return KF_ERR_CUDA;
+    tm.r = tm.a; tm.y = tm.a;
+    UmmaParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+    p.tiles_m = static_cast<int>((M + kBM - 1) / kBM);
+    p.tiles_n = static_cast<int>((N + bn_split - 1) / bn_split);
+    p.num_tiles = p.tiles_m * p.tiles_n;
+    p.k_blocks = static_cast<int>((K + kBK - 1) / kBK);
+    p.tiles_per_unit = 1;
+    p.bias = static_cast<const __nv_bfloat16*>(bias);
+    p.R = static_cast<const __nv_bfloat16*>(residual);
+    p.ldr = ldr; p.out = Y; p.ldo = ldy; p.scale = scale;
+    p.vec_ok = (ldy % 8 == 0 && aligned(Y, 16) &&
+                (residual == nullptr || (ldr % 8 == 0 && aligned(residual, 16)))) ? 1 : 0;
+    p.bias_vec = aligned(bias, 16) ? 1 : 0;
+    p.status = d->status;
+    if (launch_umma_splitk(bn_split, split, act, tm, p, st) != cudaSuccess) return KF_ERR_CUDA;
+    g_launches += 1;
+    return KF_OK;
+  }
   if (umma_gemm_ok(io_dtype, K, X, ldx, W, ldw)) {
     const int bn = pick_tile_n(M, N, d->sm_count);
     const bool pair = bn == 256 && use_cta_pairs(M, K);

@@ -58,6 +58,10 @@ cudaError_t launch_groupnorm_apply(int Nb, int Cout, int groups, long long hw, i
                                    float eps, const float* stats, const void* gamma,
                                    const void* beta, void* y, cudaStream_t st);
 
+// split-K cluster kernel of the elementwise chain: bn in {128, 256}, s CTAs per tile
+cudaError_t launch_umma_splitk(int bn, int s, int act, const UmmaMaps& tm, const UmmaParams& p,
+                               cudaStream_t st);
+
 // softmax over channels + pool x pool max-pool of an NCHW tensor (pool <= 4)
 cudaError_t launch_channel_softmax_pool(int dt, int Nb, int C, int H, int Wd, int pool, const void* a,
                                         void* y, cudaStream_t st);

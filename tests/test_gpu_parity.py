@@ -111,6 +111,41 @@ def test_bf16_gemm_tile_widths_and_unaligned_rows(kf, shape):
     assert_close(got, ref, 2e-2, 2e-2, "bf16 bare %s" % (shape,))
 
 
+# Few tiles and a long K take the split-K cluster kernel: 4 or 8 CTAs per tile, partial tiles
+# exchanged through distributed shared memory, slices of 64 or 32 columns finished per CTA.
+@pytest.mark.parametrize("shape", [(128, 1024, 2048),     # 4 tiles x 8 CTAs, 256-column tiles
+                                   (200, 300, 1544),      # 4 tiles x 4 CTAs, ragged M, N, K (24.1 K blocks)
+                                   (100, 128, 4096),      # 128-column tile x 4 CTAs
+                                   (64, 2000, 2048),      # 8 tiles x 8 CTAs, last tile ragged in N
+                                   (130, 777, 1600)])     # unaligned rows: scalar stores
+def test_bf16_gemm_split_k_cluster_kernel(kf, shape):
+    M, N, K = shape
+    d = ki.gemm_inputs("c2", seed=31, M=M, N=N, K=K)
+    for act, scale, res in [("gelu_tanh", 0.5, True), ("none", 1.0, False), ("chain95", 1.0, True)]:
+        got, ref = run_gemm(kf, d, act, scale, use_res=res)
+        assert_close(got, ref, 2e-2, 2e-2, "bf16 split-K %s %s" % (shape, act))
+    # the same call again gives the same bits (fixed summation order across the cluster)
+    X, W, b = to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"])
+    y1 = kf.gemm_epilogue(X, W, b, "swish")
+    y2 = kf.gemm_epilogue(X, W, b, "swish")
+    assert (y1.view(__import__("torch").int16) == y2.view(__import__("torch").int16)).all()
+
+
+def test_bf16_split_k_layout_pins(kf):
+    """One-hot X rows through the split-K kernel: every K share and column slice lands in place."""
+    M, N, K = 128, 512, 4096
+    r = np.random.default_rng(6)
+    Wv = (r.integers(-64, 65, size=(N, K)) / 64.0)
+    ks = r.integers(0, K, size=M)
+    Xf = np.zeros((M, K)); Xf[np.arange(M), ks] = 1.0
+    Y = kf.gemm_epilogue(to_dev(ki.store(Xf, "bf16")), to_dev(ki.store(Wv, "bf16")))
+    check_status()
+    assert_close(to_f64(Y), Wv[:, ks].T, 0.0, 0.0, "one-hot X rows, split-K")
+    # all-ones: each of the 8 K shares contributes K/8; the exact sum needs all of them once
+    Y = kf.gemm_epilogue(to_dev(ki.store(np.ones((M, K)), "bf16")), to_dev(ki.store(np.ones((N, K)) / 64, "bf16")))
+    assert (to_f64(Y) == K / 64).all()
+
+
 # K >= 2048 with more than 256 rows takes the CTA-pair kernel (256-row tiles over two SMs)
 @pytest.mark.parametrize("shape", [(384, 520, 2048), (257, 256, 2112), (1000, 264, 2048)])
 def test_bf16_gemm_cta_pair_kernel(kf, shape):

@@ -151,8 +151,17 @@ kf_status check_workspace(const void* ws, size_t have, size_t need) {
 }
 
 // one statistic per row and 256-column tile
+// Tile width of the row-reduce first pass.  A softmax that fits in one wave of 64-column tiles
+// takes them instead of 256-column tiles: four times the CTAs and a quarter of the serial epilogue per CTA.
+// The rule uses the B200's SM count as a constant so that the workspace query, which has no
+// device, agrees with the call.
+int rowreduce_bn(int64_t M, int64_t N, int red) {
+  const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + kRowReduceNarrowBN - 1) / kRowReduceNarrowBN);
+  return (red == RED_SOFTMAX && tiles <= 148) ? kRowReduceNarrowBN : kRowReduceBN;
+}
 size_t rowreduce_umma_ws(int64_t M, int64_t N, int red) {
-  const int64_t tiles_n = (N + kRowReduceBN - 1) / kRowReduceBN;
+  const int bn = rowreduce_bn(M, N, red);
+  const int64_t tiles_n = (N + bn - 1) / bn;
   return round256(static_cast<size_t>(M) * tiles_n * (red == RED_SOFTMAX ? 8 : 4));
 }
 // CTA pairs (256-row tiles, each CTA loading half of the W tile) pay off when the K loop is
@@ -353,11 +362,11 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
   if (umma_gemm_ok(in_dtype, K, X, ldx, W, ldw) && (N + kRowReduceBN - 1) / kRowReduceBN <= 8192) {
     vs = check_workspace(workspace, workspace_bytes, rowreduce_umma_ws(M, N, red));
     if (vs != KF_OK) return vs;
-    const bool pair = use_cta_pairs(M, K);
+    const int bn = rowreduce_bn(M, N, red);
+    const bool pair = bn == kRowReduceBN && use_cta_pairs(M, K);
     const int tile_m = pair ? 2 * kBM : kBM;
     const int slots = pair ? d->sm_count / 2 : d->sm_count;
     const int64_t tiles_m64 = (M + tile_m - 1) / tile_m;
-    const int bn = kRowReduceBN;
     const int64_t tiles_n64 = (N + bn - 1) / bn;
     UmmaMaps tm;
     if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, pair ? bn / 2 : bn))
@@ -389,9 +398,9 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
     const int units = p.num_tiles / p.tiles_per_unit;
     const int grid = units < slots ? units : slots;
     if (red == KF_RED_SOFTMAX) {
-      if (launch_umma_softmax(pre_act, out_dtype, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
+      if (launch_umma_softmax(bn, pre_act, out_dtype, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
         return KF_ERR_CUDA;
-      if (launch_softmax_finalize(out_dtype, Mi, Ni, p.tiles_n, p.partial, out, ldo, p.vec_ok, st) !=
+      if (launch_softmax_finalize(out_dtype, Mi, Ni, bn, p.tiles_n, p.partial, out, ldo, p.vec_ok, st) !=
           cudaSuccess)
         return KF_ERR_CUDA;
     } else {

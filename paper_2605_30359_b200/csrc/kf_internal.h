@@ -21,16 +21,19 @@ struct UmmaMaps {
 // tiles); otherwise one CTA per 128-row tile
 cudaError_t launch_umma_elementwise(int bn, int act, int pair, const UmmaMaps& tm,
                                     const UmmaParams& p, int grid, cudaStream_t st);
-cudaError_t launch_umma_softmax(int act, int out_dt, int pair, const UmmaMaps& tm,
+cudaError_t launch_umma_softmax(int bn, int act, int out_dt, int pair, const UmmaMaps& tm,
                                 const UmmaParams& p, int grid, cudaStream_t st);
+cudaError_t launch_umma_softmax_narrow(int act, int out_dt, const UmmaMaps& tm, const UmmaParams& p,
+                                       int grid, cudaStream_t st);
 cudaError_t launch_umma_rowsum(int act, int pair, const UmmaMaps& tm, const UmmaParams& p,
                                int grid, cudaStream_t st);
 cudaError_t launch_umma_conv(int bn, int act, const UmmaMaps& tm, const UmmaParams& p, int grid,
                              cudaStream_t st);
 constexpr int kRowReduceBN = 256;   // tile width of the row-reduce first pass
+constexpr int kRowReduceNarrowBN = 64;   // ... of the softmax first pass of one-wave problems
 
 // second passes of the tensor-core row reductions
-cudaError_t launch_softmax_finalize(int out_dt, int M, int N, int tiles_n, const float* partial,
+cudaError_t launch_softmax_finalize(int out_dt, int M, int N, int bn, int tiles_n, const float* partial,
                                     void* out, long long ldo, int vec_ok, cudaStream_t st);
 cudaError_t launch_rowsum_finalize(int M, int tiles_n, const float* partial, float* out,
                                    cudaStream_t st);

@@ -53,16 +53,28 @@ cudaError_t launch_row_sum(int M, int N, const float* A, long long lda, float* o
   return cudaGetLastError();
 }
 
-cudaError_t launch_softmax_finalize(int out_dt, int M, int N, int tiles_n, const float* partial,
+cudaError_t launch_softmax_finalize(int out_dt, int M, int N, int bn, int tiles_n, const float* partial,
                                     void* out, long long ldo, int vec_ok, cudaStream_t st) {
+  const int bn_shift = bn == 64 ? 6 : 8;
+  if (tiles_n <= 32) {
+    const unsigned grid = static_cast<unsigned>((M + 7) / 8);
+    const float2* pw = reinterpret_cast<const float2*>(partial);
+    if (out_dt == DT_F32)
+      softmax_finalize_warp_kernel<float><<<grid, 256, 0, st>>>(M, N, bn_shift, tiles_n, pw,
+                                                               static_cast<float*>(out), ldo, vec_ok);
+    else
+      softmax_finalize_warp_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
+          M, N, bn_shift, tiles_n, pw, static_cast<__nv_bfloat16*>(out), ldo, vec_ok);
+    return cudaGetLastError();
+  }
   const size_t smem = static_cast<size_t>(tiles_n) * sizeof(float);
   const float2* part = reinterpret_cast<const float2*>(partial);
   if (out_dt == DT_F32)
-    softmax_finalize_kernel<float, kRowReduceBN><<<M, 256, smem, st>>>(
-        N, tiles_n, part, static_cast<float*>(out), ldo, vec_ok);
+    softmax_finalize_kernel<float><<<M, 256, smem, st>>>(
+        N, bn_shift, tiles_n, part, static_cast<float*>(out), ldo, vec_ok);
   else
-    softmax_finalize_kernel<__nv_bfloat16, kRowReduceBN><<<M, 256, smem, st>>>(
-        N, tiles_n, part, static_cast<__nv_bfloat16*>(out), ldo, vec_ok);
+    softmax_finalize_kernel<__nv_bfloat16><<<M, 256, smem, st>>>(
+        N, bn_shift, tiles_n, part, static_cast<__nv_bfloat16*>(out), ldo, vec_ok);
   return cudaGetLastError();
 }
 

@@ -160,12 +160,12 @@ row_sum_kernel(int N, const float* __restrict__ A, long long lda, float* out) {
 
 // ---------------------------------------------------------------- second passes, tensor path
 // Softmax: the first pass left e[m,n] = exp(a[m,n] - mx_t) in `out` and (mx_t, sum_t) per
-// BN-column slice t (half an MMA tile) in `partial`.  Row maximum mx = max_t mx_t, denominator
+// slice t of 2^bn_shift columns (one first-pass tile) in `partial`.  Row maximum mx = max_t mx_t, denominator
 // S = sum_t sum_t*exp(mx_t - mx); the output is e * exp(mx_t - mx) / S, in place.
-template <typename OutT, int BN>
+template <typename OutT>
 __global__ void __launch_bounds__(256)
-softmax_finalize_kernel(int N, int tiles_n, const float2* __restrict__ partial, OutT* out,
-                        long long ldo, int vec_ok) {
+softmax_finalize_kernel(int N, int bn_shift, int tiles_n, const float2* __restrict__ partial,
+                        OutT* out, long long ldo, int vec_ok) {
   extern __shared__ float fac[];   // [tiles_n]
   __shared__ float scratch[32];
   const long long m = blockIdx.x;
@@ -188,7 +188,7 @@ softmax_finalize_kernel(int N, int tiles_n, const float2* __restrict__ partial, 
     const int nvec = N / V;
     uint4* ov = reinterpret_cast<uint4*>(o);
     for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
-      const float f = fac[(i * V) / BN] * inv;
+      const float f = fac[(i * V) >> bn_shift] * inv;
       uint4 w = ov[i];
       if constexpr (sizeof(OutT) == 2) {
         w.x = pack_bf16x2(bf16_lo(w.x) * f, bf16_hi(w.x) * f);
@@ -205,7 +205,61 @@ softmax_finalize_kernel(int N, int tiles_n, const float2* __restrict__ partial, 
     }
   } else {
     for (int n = threadIdx.x; n < N; n += blockDim.x)
-      o[n] = from_f32<OutT>(to_f32(o[n]) * fac[n / BN] * inv);
+      o[n] = from_f32<OutT>(to_f32(o[n]) * fac[n >> bn_shift] * inv);
+  }
+}
+
+// The same second pass for rows of at most 32 slices: one WARP per row (eight rows per block),
+// statistics combined with shuffles, lane t keeping slice t's factor.  Short rows leave most of
+// a 256-thread block idle in the kernel above and pay two block reductions per row.
+template <typename OutT>
+__global__ void __launch_bounds__(256)
+softmax_finalize_warp_kernel(int M, int N, int bn_shift, int tiles_n,
+                             const float2* __restrict__ partial, OutT* out, long long ldo,
+                             int vec_ok) {
+  const int lane = threadIdx.x & 31;
+  const long long m = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  if (m >= M) return;
+  float2 pt = make_float2(-INFINITY, 0.0f);
+  if (lane < tiles_n) pt = partial[m * tiles_n + lane];
+  float mx = pt.x;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  const float fac = lane < tiles_n ? __expf(pt.x - mx) : 0.0f;
+  float s = pt.y * fac;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  const float scale = fac / s;                         // lane t: factor of slice t
+  OutT* o = out + m * ldo;
+  if (vec_ok && (N % 8) == 0) {
+    constexpr int V = 16 / sizeof(OutT);
+    const int nvec = N / V;
+    uint4* ov = reinterpret_cast<uint4*>(o);
+    for (int i0 = 0; i0 < nvec; i0 += 32) {            // uniform trip count: shuffles need all lanes
+      const int i = i0 + lane;
+      const float f = __shfl_sync(0xffffffffu, scale, (min(i, nvec - 1) * V) >> bn_shift);
+      if (i < nvec) {
+        uint4 w = ov[i];
+        if constexpr (sizeof(OutT) == 2) {
+          w.x = pack_bf16x2(bf16_lo(w.x) * f, bf16_hi(w.x) * f);
+          w.y = pack_bf16x2(bf16_lo(w.y) * f, bf16_hi(w.y) * f);
+          w.z = pack_bf16x2(bf16_lo(w.z) * f, bf16_hi(w.z) * f);
+          w.w = pack_bf16x2(bf16_lo(w.w) * f, bf16_hi(w.w) * f);
+        } else {
+          w.x = __float_as_uint(__uint_as_float(w.x) * f);
+          w.y = __float_as_uint(__uint_as_float(w.y) * f);
+          w.z = __float_as_uint(__uint_as_float(w.z) * f);
+          w.w = __float_as_uint(__uint_as_float(w.w) * f);
+        }
+        ov[i] = w;
+      }
+    }
+  } else {
+    for (int n0 = 0; n0 < N; n0 += 32) {
+      const int n = n0 + lane;
+      const float f = __shfl_sync(0xffffffffu, scale, min(n, N - 1) >> bn_shift);
+      if (n < N) o[n] = from_f32<OutT>(to_f32(o[n]) * f);
+    }
   }
 }
 

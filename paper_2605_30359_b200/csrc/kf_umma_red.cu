@@ -4,8 +4,9 @@
 
 namespace kf {
 
-cudaError_t launch_umma_softmax(int act, int out_dt, int pair, const UmmaMaps& tm,
+cudaError_t launch_umma_softmax(int bn, int act, int out_dt, int pair, const UmmaMaps& tm,
                                 const UmmaParams& p, int grid, cudaStream_t st) {
+  if (bn == kRowReduceNarrowBN) return launch_umma_softmax_narrow(act, out_dt, tm, p, grid, st);
   cudaError_t e = cudaErrorInvalidValue;
   dispatch_act(act, [&](auto A) {
     constexpr int ACT = decltype(A)::value;

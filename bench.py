@@ -406,6 +406,7 @@ SWEEP_GEMM = [  # (dtype, M, N, K, act, scale, residual)
     ("bf16", 8192, 4096, 4096, "chain95", 1.0, False), ("bf16", 64, 8192, 8192, "none", 1.0, False),
     ("f32", 128, 256, 512, "relu", 1.0, False), ("f32", 64, 64, 64, "gelu_tanh", 1.0, False),
     ("f32", 512, 512, 256, "sigmoid", 1.0, True),
+    ("f32", 2048, 2048, 2048, "gelu_tanh", 1.0, True), ("f32", 1024, 4096, 1024, "relu", 1.0, False),
 ]
 SWEEP_ROWRED = [  # (M, N, K, pre_act, red)
     (1024, 1024, 1024, "none", "softmax"), (4096, 8192, 2048, "none", "softmax"),

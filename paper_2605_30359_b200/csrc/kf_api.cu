@@ -78,6 +78,19 @@ bool encode_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, in
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
          CUDA_SUCCESS;
 }
+// fp32 row-major [rows, cols] with pitch ld (a multiple of 4 elements) -> boxes of box_rows x 16
+// columns (64 bytes) with the 64-byte swizzle, zero fill outside the tensor.
+bool encode_2d_f32(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld,
+                   int box_rows) {
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 4};
+  const cuuint32_t box[2] = {16u, static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1, 1};
+  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides,
+                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+         CUDA_SUCCESS;
+}
 bool encode_piece(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld) {
   return encode_2d(tm, base, rows, cols, ld, kBM, kPieceCols, CU_TENSOR_MAP_SWIZZLE_64B);
 }
@@ -180,6 +193,19 @@ int pick_tile_n(int64_t M, int64_t N, int sm_count) {
   return cover;
 }
 
+// fp32 chains large enough for the tensor cores take the 3xTF32 kernel (operands split into
+// TF32 hi + lo parts in the workspace); smaller ones stay on the fp32 FMA kernel (measured:
+// 512^3 18.6 us FMA / 35 us tensor, 1024^3 112 / 54 us, 4096^3 6569 / 667 us).
+bool use_tf32x3(int dt, int64_t M, int64_t N, int64_t K) {
+  if (dt != DT_F32 || getenv("KF_NO_TF32X3") != nullptr) return false;
+  return M >= 64 && N >= 64 && K >= 64 && M * N * K >= (int64_t{1} << 29);
+}
+int64_t tf32_kp(int64_t K) { return (K + 3) / 4 * 4; }
+size_t tf32_ws(int64_t M, int64_t N, int64_t K) {
+  return 2 * round256(static_cast<size_t>(M) * tf32_kp(K) * 4) +
+         2 * round256(static_cast<size_t>(N) * tf32_kp(K) * 4);
+}
+
 // Cluster size of the split-K kernel, or 0.  Measured on B200: a narrow-tile CTA spends about
 // 0.28 us per K block whatever the tile width, the cluster exchange costs about 4 us, so
 // splitting pays from about 24 K blocks; clusters of 8 schedule well only while there are few
@@ -234,7 +260,10 @@ kf_status kf_device_status(void) {
   return KF_OK;
 }
 
-size_t kf_gemm_epilogue_workspace_bytes(int64_t, int64_t, int64_t, kf_dtype) { return 0; }
+size_t kf_gemm_epilogue_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype) {
+  if (M < 1 || N < 1 || K < 1) return 0;
+  return use_tf32x3(io_dtype, M, N, K) ? tf32_ws(M, N, K) : 0;
+}
 
 size_t kf_gemm_rowreduce_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype,
                                          kf_rowred red) {
@@ -256,7 +285,6 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
                            int64_t ldx, const void* W, int64_t ldw, const void* bias, kf_act act,
                            float scale, const void* residual, int64_t ldr, void* Y, int64_t ldy,
                            void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  (void)workspace; (void)workspace_bytes;
   kf_status vs = check_gemm_common(M, N, K, io_dtype, X, ldx, W, ldw, bias);
   if (vs != KF_OK) return vs;
   if (!valid_act(act) || Y == nullptr || ldy < N) return KF_ERR_INVALID_ARG;
@@ -269,6 +297,44 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
   if (!device_info(&d)) return KF_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
+  if (use_tf32x3(io_dtype, M, N, K)) {
+    vs = check_workspace(workspace, workspace_bytes, tf32_ws(M, N, K));
+    if (vs != KF_OK) return vs;
+    const int64_t kp = tf32_kp(K);
+    const size_t xb = round256(static_cast<size_t>(M) * kp * 4), wb = round256(static_cast<size_t>(N) * kp * 4);
+    float* xh = static_cast<float*>(workspace);
+    float* xl = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + xb);
+    float* wh = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 2 * xb);
+    float* wl = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 2 * xb + wb);
+    if (launch_tf32_split(M, static_cast<int>(K), static_cast<int>(kp), static_cast<const float*>(X), ldx,
+                          xh, xl, st) != cudaSuccess ||
+        launch_tf32_split(N, static_cast<int>(K), static_cast<int>(kp), static_cast<const float*>(W), ldw,
+                          wh, wl, st) != cudaSuccess)
+      return KF_ERR_CUDA;
+    const int bn = N <= 128 ? 128 : 256;
+    CUtensorMap ah, al, bh, bl;
+    if (!encode_2d_f32(&ah, xh, M, K, kp, kBM) || !encode_2d_f32(&al, xl, M, K, kp, kBM) ||
+        !encode_2d_f32(&bh, wh, N, K, kp, bn) || !encode_2d_f32(&bl, wl, N, K, kp, bn))
+      return KF_ERR_CUDA;
+    Tf32Params p;
+    std::memset(&p, 0, sizeof(p));
+    p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+    p.tiles_m = static_cast<int>((M + kBM - 1) / kBM);
+    p.tiles_n = static_cast<int>((N + bn - 1) / bn);
+    if (static_cast<int64_t>(p.tiles_m) * p.tiles_n > kMaxDim) return KF_ERR_UNSUPPORTED;
+    p.num_tiles = p.tiles_m * p.tiles_n;
+    p.k_blocks = static_cast<int>((K + 15) / 16);
+    p.bias = static_cast<const float*>(bias);
+    p.R = static_cast<const float*>(residual);
+    p.ldr = ldr; p.out = static_cast<float*>(Y); p.ldo = ldy; p.scale = scale; p.act = act;
+    p.vec_ok = (ldy % 4 == 0 && aligned(Y, 16) &&
+                (residual == nullptr || (ldr % 4 == 0 && aligned(residual, 16)))) ? 1 : 0;
+    p.status = d->status;
+    const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
+    if (launch_tf32_chain(bn, ah, al, bh, bl, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
+    g_launches += 3;
+    return KF_OK;
+  }
   int bn_split = 0;
   const int split = umma_gemm_ok(io_dtype, K, X, ldx, W, ldw)
                         ? pick_split_k(M, N, K, d->sm_count, &bn_split) : 0;

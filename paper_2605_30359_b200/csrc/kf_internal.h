@@ -61,6 +61,26 @@ cudaError_t launch_groupnorm_apply(int Nb, int Cout, int groups, long long hw, i
                                    float eps, const float* stats, const void* gamma,
                                    const void* beta, void* y, cudaStream_t st);
 
+// fp32 chain on the tensor cores (3xTF32): split prepass and GEMM kernel
+struct Tf32Params {
+  int M, N, K;
+  int tiles_m, tiles_n, num_tiles, k_blocks;
+  const float* bias;             // [N] or null
+  const float* R;                // [M, ldr] or null
+  long long ldr;
+  float* out;                    // [M, ldo]
+  long long ldo;
+  float scale;
+  int act;
+  int vec_ok;                    // rows of out (and R) start on 16 bytes
+  uint32_t* status;
+};
+cudaError_t launch_tf32_split(long long rows, int K, int kp, const float* in, long long ld, float* hi,
+                              float* lo, cudaStream_t st);
+cudaError_t launch_tf32_chain(int bn, const CUtensorMap& ah, const CUtensorMap& al,
+                              const CUtensorMap& bh, const CUtensorMap& bl, const Tf32Params& p,
+                              int grid, cudaStream_t st);
+
 // split-K cluster kernel of the elementwise chain: bn in {128, 256}, s CTAs per tile
 cudaError_t launch_umma_splitk(int bn, int s, int act, const UmmaMaps& tm, const UmmaParams& p,
                                cudaStream_t st);

@@ -59,6 +59,54 @@ def test_fp32_gelu_variant_is_the_tanh_one(kf):
     assert abs(to_f64(Y)[0, 0] - oracle.act("gelu_erf", -3.0)) > 3e-4
 
 
+# ------------------------------------------------------------------ fp32 on the tensor cores (3xTF32)
+# M*N*K >= 2^29 takes the split-operand tensor-core kernel; the result must stay within the
+# fp32 tolerance whatever K is (accumulation is folded into an fp32 running sum every 512).
+@pytest.mark.parametrize("shape", [(1024, 1024, 512),      # aligned: vector epilogue, one chunk
+                                   (768, 640, 1100),       # three chunks, ragged last K block
+                                   (1000, 999, 600),       # unaligned rows: scalar epilogue
+                                   (256, 512, 4100)])      # nine chunks on two row tiles
+def test_fp32_tensor_core_chain(kf, shape):
+    M, N, K = shape
+    d = ki.gemm_inputs("c2", seed=41, M=M, N=N, K=K, dtype="f32")
+    got, ref = run_gemm(kf, d, "gelu_tanh", 0.5)
+    assert_close(got, ref, 1e-4, 1e-4, "fp32 3xTF32 %s" % (shape,))
+    got, ref = run_gemm(kf, d, "none", 1.0, use_bias=False, use_res=False)
+    assert_close(got, ref, 1e-4, 1e-4, "fp32 3xTF32 bare %s" % (shape,))
+    assert np.abs(got - ref).max() < 3e-5       # an order of magnitude better than one-pass TF32
+
+
+def test_fp32_tensor_core_layout_and_split_pins(kf):
+    """One-hot X rows return W's entries: exact whenever an entry fits hi + lo (22 significant
+    bits), so a wrong K block, swizzle or operand (hi/lo mixed up) shows as a mismatch."""
+    M, N, K = 1024, 1024, 512
+    r = np.random.default_rng(7)
+    Wv = r.integers(-(1 << 21), 1 << 21, size=(N, K)).astype(np.float64) / (1 << 12)
+    ks = r.integers(0, K, size=M)
+    Xf = np.zeros((M, K)); Xf[np.arange(M), ks] = 1.0
+    Y = kf.gemm_epilogue(to_dev(Xf.astype(np.float32)), to_dev(Wv.astype(np.float32)))
+    check_status()
+    assert_close(to_f64(Y), Wv[:, ks].T, 0.0, 0.0, "one-hot X rows, 3xTF32")
+    # x = 1 + 2^-12 needs the lo part: (1 + 2^-12) * 1 summed over K
+    Xs = np.full((M, K), 1.0 + 2.0 ** -12, np.float32)
+    Y = kf.gemm_epilogue(to_dev(Xs), to_dev(np.ones((N, K), np.float32)))
+    assert (to_f64(Y) == K * (1.0 + 2.0 ** -12)).all()
+
+
+def test_fp32_tensor_core_workspace_is_checked(kf):
+    import torch
+    M, N, K = 1024, 1024, 512
+    need = kf.kf_gemm_epilogue_workspace_bytes(M, N, K, kf.KF_F32)
+    assert need == 2 * M * K * 4 + 2 * N * K * 4
+    X = torch.zeros((M, K), device="cuda"); W = torch.zeros((N, K), device="cuda")
+    Y = torch.empty((M, N), device="cuda")
+    ws = torch.empty(need // 2, dtype=torch.uint8, device="cuda")
+    st = kf.kf_gemm_epilogue(M, N, K, kf.KF_F32, X.data_ptr(), K, W.data_ptr(), K, None, 0, 1.0, None, 0,
+                             Y.data_ptr(), N, ws.data_ptr(), need // 2, None)
+    assert st == kf.KF_ERR_WORKSPACE
+    assert kf.kf_gemm_epilogue_workspace_bytes(128, 256, 512, kf.KF_F32) == 0
+
+
 # ------------------------------------------------------------------ bf16 tensor-core GEMM
 def test_bf16_layout_pins_onehot_and_permutation(kf):
     """Products by 0/1 are exact, so any mismatch is a layout / swizzle / descriptor bug."""

@@ -72,7 +72,14 @@ typedef enum { KF_RED_SOFTMAX = 0, KF_RED_SUM = 1 } kf_rowred;
  * torch.nn.Linear, residual and Y are [M,N] (ldr, ldy).  bias and residual may be NULL.
  * Y must not alias X or W; Y may alias residual only if ldr == ldy (same element, same place).
  * Shapes: any M,N,K >= 1.  bf16 problems with K % 8 == 0, ldx % 8 == 0, ldw % 8 == 0 and
- * 16-byte aligned X, W take the tensor-core kernel; everything else takes a scalar kernel. */
+ * 16-byte aligned X, W take the bf16 tensor-core kernels (whole tiles, or a split-K cluster when
+ * there are few tiles and K is long).  fp32 problems with M*N*K >= 2^29 take the tensor cores
+ * too: each operand is split into two TF32 numbers (22 significant bits together), three
+ * products per element pair are accumulated, and partial sums are folded into an fp32 running
+ * sum every 512 elements of K; absolute error about 1e-5 on outputs of magnitude 1, like an
+ * fp32 FMA loop, for any K.  That path needs the workspace kf_gemm_epilogue_workspace_bytes()
+ * returns (the split operands: 8*(M+N)*ceil4(K) bytes) and fails with KF_ERR_WORKSPACE
+ * without it; every other path needs none.  Everything else takes a scalar kernel. */
 kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
                            const void* X, int64_t ldx, const void* W, int64_t ldw,
                            const void* bias, kf_act act, float scale,

@@ -362,8 +362,20 @@ def run_single_workload(args, kf, device, peaks):
         "c5": (2.0 * 128 * 64 * 64 * 128 * 576, 2 * (128 * 64 * 64 * 64 + 128 * 64 * 9 + 128 + 128 * 128 * 64 * 64)),
     }
     specs["pool"] = (specs["c5"][0], 2 * (128 * 64 * 64 * 64 + 128 * 64 * 9 + 128 + 128 * 128 * 16 * 16))
+    specs["f32"] = (2.0 * 2048 ** 3, 4 * (3 * 2048 * 2048 + 2048 + 2048 * 2048))
+    specs["skinny"] = (2.0 * 64 * 8192 * 8192, 2 * (64 * 8192 + 8192 * 8192 + 8192 + 64 * 8192))
     flops, nbytes = specs[name]
-    if name == "pool":      # conv3x3 -> channel softmax -> max-pool 4 on config 5's tensors
+    if name in ("f32", "skinny"):   # fp32 3xTF32 chain 2048^3; bf16 split-K cluster chain 64x8192x8192
+        g = torch.Generator(device=device).manual_seed(0)
+        dt = torch.float32 if name == "f32" else torch.bfloat16
+        M, N, K = (2048, 2048, 2048) if name == "f32" else (64, 8192, 8192)
+        X = torch.randn((M, K), generator=g, device=device).to(dt)
+        W = (torch.randn((N, K), generator=g, device=device) * K ** -0.5).to(dt)
+        b = torch.randn((N,), generator=g, device=device).to(dt)
+        R = torch.randn((M, N), generator=g, device=device).to(dt)
+        o = torch.empty((M, N), dtype=dt, device=device)
+        fn = lambda: kf.gemm_epilogue(X, W, b, "gelu_tanh", 0.5, R, out=o)
+    elif name == "pool":      # conv3x3 -> channel softmax -> max-pool 4 on config 5's tensors
         d = ki.conv_inputs("c5", seed=0)
         t = {k: to_dev(d[k], device) for k in ("x", "w", "bias")}
         o = torch.empty(128, 128, 16, 16, dtype=torch.bfloat16, device=device)
@@ -517,9 +529,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the context table and baselines")
-    ap.add_argument("--workload", default=WORKLOAD, choices=["c1", "c2", "c3", "c4", "c5", "pool"],
+    ap.add_argument("--workload", default=WORKLOAD, choices=["c1", "c2", "c3", "c4", "c5", "pool", "f32", "skinny"],
                     help="c2 is the headline; the others print a reduced line (profiling aid); "
-                         "pool = conv3x3 -> channel softmax -> max-pool on config 5's tensors")
+                         "pool = conv3x3 -> channel softmax -> max-pool on config 5's tensors; "
+                         "f32 = fp32 2048^3 chain (3xTF32 kernel); skinny = bf16 64x8192x8192 (split-K)")
     ap.add_argument("--sweep", action="store_true",
                     help="time every sweep shape against unfused torch; prints fast_1 / avg / geomean")
     args = ap.parse_args()

@@ -175,7 +175,8 @@ int rowreduce_bn(int64_t M, int64_t N, int red) {
 size_t rowreduce_umma_ws(int64_t M, int64_t N, int red) {
   const int bn = rowreduce_bn(M, N, red);
   const int64_t tiles_n = (N + bn - 1) / bn;
-  return round256(static_cast<size_t>(M) * tiles_n * (red == RED_SOFTMAX ? 8 : 4));
+  // softmax: (max, sum) per row and per half tile (one per epilogue group); row sum: one float
+  return round256(static_cast<size_t>(M) * tiles_n * (red == RED_SOFTMAX ? 16 : 4));
 }
 // CTA pairs (256-row tiles, each CTA loading half of the W tile) pay off when the K loop is
 // long: measured +3.6 % at K = 4096, +3.3 % at K = 2048, -4 % at K = 1024 (fewer, larger tiles
@@ -425,7 +426,7 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int Mi = static_cast<int>(M), Ni = static_cast<int>(N), Ki = static_cast<int>(K);
 
-  if (umma_gemm_ok(in_dtype, K, X, ldx, W, ldw) && (N + kRowReduceBN - 1) / kRowReduceBN <= 8192) {
+  if (umma_gemm_ok(in_dtype, K, X, ldx, W, ldw) && (N + kRowReduceBN - 1) / kRowReduceBN <= 4096) {
     vs = check_workspace(workspace, workspace_bytes, rowreduce_umma_ws(M, N, red));
     if (vs != KF_OK) return vs;
     const int bn = rowreduce_bn(M, N, red);
@@ -466,7 +467,7 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
     if (red == KF_RED_SOFTMAX) {
       if (launch_umma_softmax(bn, pre_act, out_dtype, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
         return KF_ERR_CUDA;
-      if (launch_softmax_finalize(out_dtype, Mi, Ni, bn, p.tiles_n, p.partial, out, ldo, p.vec_ok, st) !=
+      if (launch_softmax_finalize(out_dtype, Mi, Ni, bn / 2, 2 * p.tiles_n, p.partial, out, ldo, p.vec_ok, st) !=
           cudaSuccess)
         return KF_ERR_CUDA;
     } else {

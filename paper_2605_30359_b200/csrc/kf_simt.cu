@@ -55,7 +55,8 @@ cudaError_t launch_row_sum(int M, int N, const float* A, long long lda, float* o
 
 cudaError_t launch_softmax_finalize(int out_dt, int M, int N, int bn, int tiles_n, const float* partial,
                                     void* out, long long ldo, int vec_ok, cudaStream_t st) {
-  const int bn_shift = bn == 64 ? 6 : 8;
+  int bn_shift = 0;                      // slices are powers of two (half a first-pass tile)
+  while ((1 << bn_shift) < bn) ++bn_shift;
   if (tiles_n <= 32) {
     const unsigned grid = static_cast<unsigned>((M + 7) / 8);
     const float2* pw = reinterpret_cast<const float2*>(partial);

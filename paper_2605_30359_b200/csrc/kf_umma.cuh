@@ -33,6 +33,12 @@ constexpr int kBK = 64;           // K per stage: 64 bf16 = one 128-byte swizzle
 constexpr int kUmmaK = 16;        // K per tcgen05.mma for 16-bit inputs
 constexpr int kEpiThreads = 128;  // warps 2..5: one per TMEM lane quarter
 constexpr int kNumThreads = 192;  // 6 warps: producer, UMMA issuer, epilogue
+// The softmax epilogue is the longest (two TMEM passes, an exponential per element) and with
+// one warp per scheduler it is latency-bound, so it runs as TWO groups of four warps, each
+// owning half of the tile's columns as a slice of its own: own statistics, own staging, own
+// named barriers, own TMA stores.  The second pass combines slices, so the groups never talk.
+constexpr int epi_groups(int epi) { return epi == 1 /* EPI_SOFTMAX */ ? 2 : 1; }
+constexpr int num_threads(int epi) { return 64 + kEpiThreads * epi_groups(epi); }
 constexpr int kPieceCols = 32;    // epilogue piece: 128 rows x 32 columns
 constexpr int kPieceBytes = kBM * kPieceCols * 2;   // 8 KB of bf16
 constexpr int kMaxDynSmem = 232448;                 // 227 KB opt-in limit per CTA
@@ -75,9 +81,11 @@ struct UmmaCfg {
   static constexpr int kStageA = kBM * kBK * 2;
   static constexpr int kStageB = (CTA2 ? BN / 2 : BN) * kBK * 2;
   static constexpr int kStage = kStageA + kStageB;
-  // staging: elementwise = 2 output + 2 residual pieces; softmax / conv = 2 output pieces
+  // staging: elementwise = 2 output + 2 residual pieces; softmax = 2 output pieces per epilogue
+  // group; conv = 2 output pieces
   static constexpr int kStaging =
-      EPI == EPI_ELEMENTWISE ? 4 * kPieceBytes : (EPI == EPI_ROWSUM ? 0 : 2 * kPieceBytes);
+      EPI == EPI_ELEMENTWISE || EPI == EPI_SOFTMAX ? 4 * kPieceBytes
+                                                    : (EPI == EPI_ROWSUM ? 0 : 2 * kPieceBytes);
   static constexpr int kBarBytes = 256;
   static constexpr int kFit = (kMaxDynSmem - 1024 - kStaging - kBarBytes) / kStage;
   static constexpr int kStages = kFit > 8 ? 8 : kFit;
@@ -116,7 +124,7 @@ __device__ __forceinline__ uint32_t piece_off(int r, int j) {
 }
 
 template <int BN, int EPI, int ACT, typename OutT, bool CTA2>
-__global__ void __launch_bounds__(kNumThreads, 1)
+__global__ void __launch_bounds__(num_threads(EPI), 1)
 umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmY,
                   const UmmaParams p) {
@@ -150,7 +158,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     for (int a = 0; a < 2; ++a) {
       mbar_init(&tmem_full[a], 1);
-      mbar_init(&tmem_empty[a], (kEpiThreads / 32) * (CTA2 ? 2 : 1));
+      mbar_init(&tmem_empty[a], (kEpiThreads / 32) * epi_groups(EPI) * (CTA2 ? 2 : 1));
       mbar_init(&r_full[a], 1);
     }
     *abort_flag = 0;
@@ -256,13 +264,17 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     __syncwarp();
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5)
-    constexpr int PIECES = BN / kPieceCols;
+    constexpr int kGroups = epi_groups(EPI);
+    constexpr int kGroupCols = BN / kGroups;   // columns of the tile one epilogue group owns
+    constexpr int PIECES = kGroupCols / kPieceCols;
+    const int grp = kGroups > 1 ? (warp - 2) >> 2 : 0;
+    const uint32_t bar_a = 1u + 2u * grp, bar_b = 2u + 2u * grp;   // the group's named barriers
     const int quad = warp & 3;                 // TMEM lane quarter this warp may read
     const int row = quad * 32 + lane;          // row of the tile = TMEM lane
-    const int et = threadIdx.x - 64;           // 0..127 among epilogue threads
-    const bool leader = et == 0;               // issues the epilogue's TMA loads and stores
+    const int et = threadIdx.x - 64 - grp * kEpiThreads;   // 0..127 inside the group
+    const bool leader = et == 0;               // issues the group's TMA loads and stores
     const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
-    [[maybe_unused]] uint8_t* ybuf = stg;      // [2][kPieceBytes] output pieces
+    [[maybe_unused]] uint8_t* ybuf = stg + grp * 2 * kPieceBytes;   // [2][kPieceBytes] output pieces
     [[maybe_unused]] uint8_t* rbuf = stg + 2 * kPieceBytes;   // [2][kPieceBytes] residual pieces
     const bool staged = p.staged != 0;
     [[maybe_unused]] const bool has_r = EPI == EPI_ELEMENTWISE && p.R != nullptr;
@@ -302,18 +314,18 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const int m_cta = tm * kTileM + row0;               // first row of this CTA's 128 rows
       const long long m = static_cast<long long>(m_cta) + row;
       [[maybe_unused]] const bool row_ok = m < p.M;
-      [[maybe_unused]] const int n_tile = tn * BN;
-      [[maybe_unused]] const int n_valid = min(BN, p.N - n_tile);   // valid columns in this tile
+      [[maybe_unused]] const int n_tile = tn * BN + grp * kGroupCols;   // the group's first column
+      [[maybe_unused]] const int n_valid = min(kGroupCols, p.N - n_tile);   // its valid columns (may be <= 0)
 
       // One thread polls the accumulator barrier; the rest block in hardware at the named
       // barrier, which hands every epilogue warp the same go/no-go.
       bool ok = true;
       if (leader)
         ok = mbar_wait(&tmem_full[a], aph, abort_flag, p.status, KF_DEV_TIMEOUT_EPILOGUE);
-      ok = named_barrier_and(1, kEpiThreads, ok);
+      ok = named_barrier_and(bar_a, kEpiThreads, ok);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t t_acc = tmem_base + static_cast<uint32_t>(a * BN) + lane_off;
+      const uint32_t t_acc = tmem_base + static_cast<uint32_t>(a * BN + grp * kGroupCols) + lane_off;
       // hand the accumulator back to the UMMA issuer (one arrival per warp)
       auto release_acc = [&]() {
         tc_fence_before_sync();
@@ -372,7 +384,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             // has finished reading the other buffer, so after it (a) this piece may be stored,
             // (b) the other output buffer may be rewritten, (c) rbuf[b] has been consumed by all.
             if (leader) bulk_wait_group_read<0>();
-            rok = named_barrier_and(2, kEpiThreads, rok);
+            rok = named_barrier_and(bar_b, kEpiThreads, rok);
             if (!rok) { alive = false; break; }
             if (leader) {
               tma_store_2d(&tmY, yb, n_tile + c * kPieceCols, m_cta);   // clipped at M, N
@@ -401,7 +413,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 if (col_ok && mr < p.M) rv = p.R[mr * p.ldr + n0 + lane];
                 *reinterpret_cast<__nv_bfloat16*>(rb + piece_off(r, lane >> 3) + (lane & 7) * 2) = rv;
               }
-              named_barrier_sync(2, kEpiThreads);
+              named_barrier_sync(bar_b, kEpiThreads);
             }
             uint32_t v[32];
             tmem_ld_32x32(t_acc + c * 32, v);
@@ -429,7 +441,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                              pack_bf16x2(f[8 * q + 2], f[8 * q + 3]),
                              pack_bf16x2(f[8 * q + 4], f[8 * q + 5]),
                              pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
-            named_barrier_sync(2, kEpiThreads);
+            named_barrier_sync(bar_b, kEpiThreads);
 #pragma unroll 4
             for (int i = 0; i < 32; ++i) {
               const int r = i * 4 + er;
@@ -438,7 +450,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 Y[mr * p.ldo + n0 + lane] =
                     *reinterpret_cast<const __nv_bfloat16*>(yb + piece_off(r, lane >> 3) + (lane & 7) * 2);
             }
-            named_barrier_sync(2, kEpiThreads);        // buffers free for the next piece
+            named_barrier_sync(bar_b, kEpiThreads);        // buffers free for the next piece
           }
           release_acc();
         }
@@ -491,7 +503,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                                pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
               fence_proxy_async_smem();
               if (leader) bulk_wait_group_read<0>();   // the other buffer's store has let go
-              named_barrier_sync(2, kEpiThreads);
+              named_barrier_sync(bar_b, kEpiThreads);
               if (leader) {
                 // the second pass reads these numerators back: ask L2 to keep them
                 tma_store_2d_hint(&tmY, yb, n_tile + c * kPieceCols, m_cta, keep_policy);
@@ -527,7 +539,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (!staged) release_acc();
         if (row_ok) {
           float2* part = reinterpret_cast<float2*>(p.partial);
-          part[m * p.tiles_n + tn] = make_float2(mx, sum);
+          part[(m * p.tiles_n + tn) * kGroups + grp] = make_float2(mx, sum);
         }
       } else if constexpr (EPI == EPI_ROWSUM) {
         float sum = 0.0f;
@@ -591,7 +603,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
             fence_proxy_async_smem();
             if (leader) bulk_wait_group_read<0>();     // the other buffer's store has let go
-            named_barrier_sync(2, kEpiThreads);
+            named_barrier_sync(bar_b, kEpiThreads);
             if (leader) {
               // box = 32 pixels x 128 channels of image img; channels past Cout are clipped
               tma_store_3d(&tmY, yb, pt * BN + c * 32, tm * kBM, img);

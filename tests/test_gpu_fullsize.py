@@ -77,3 +77,48 @@ def test_c5_full_size_sampled_images(kf):
     blk = y.float().reshape(d["Nb"], d["groups"], -1)                # every (image, group) block
     assert float(blk.mean(dim=2).abs().max()) < 3e-3
     assert float((blk.var(dim=2, unbiased=False) - 1).abs().max()) < 1e-2
+
+
+# ------------------------------------------------------------------ the widened paths at bench sizes
+def test_split_k_skinny_full_size(kf):
+    """bench.py --workload skinny: 64 x 8192 x 8192 through the split-K cluster kernel; the oracle
+    recomputes sampled output columns (a column of Y needs one row of W)."""
+    M, N, K = 64, 8192, 8192
+    d = ki.gemm_inputs("c2", seed=5, M=M, N=N, K=K)
+    Y = kf.gemm_epilogue(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "gelu_tanh", 0.5, to_dev(d["R"]))
+    check_status()
+    cols = sample_rows(N, 48, 6)          # both sides of the 64-column slices and 256-column tiles
+    ref = oracle.gemm_epilogue(d["X"], d["W"][cols], d["b"][cols], "gelu_tanh", 0.5,
+                               np.ascontiguousarray(d["R"][:, cols]))
+    assert_close(to_f64(Y[:, cols]), ref, 2e-2, 2e-2, "split-K sampled columns")
+    import torch
+    assert torch.isfinite(Y).all()
+
+
+def test_fp32_tensor_core_full_size_sampled_rows(kf):
+    """bench.py --workload f32: 2048^3 fp32 through the 3xTF32 kernel, sampled rows."""
+    M = N = K = 2048
+    d = ki.gemm_inputs("c2", seed=7, M=M, N=N, K=K, dtype="f32")
+    Y = kf.gemm_epilogue(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "gelu_tanh", 0.5, to_dev(d["R"]))
+    check_status()
+    rows = sample_rows(M, 24, 8)
+    ref = oracle.gemm_epilogue(d["X"][rows], d["W"], d["b"], "gelu_tanh", 0.5, d["R"][rows])
+    assert_close(to_f64(Y[rows]), ref, 1e-4, 1e-4, "fp32 3xTF32 sampled rows")
+    import torch
+    assert torch.isfinite(Y).all()
+    diff = Y - to_dev(d["R"])
+    assert float(diff.min()) > -0.0851           # 0.5 * min GELU = -0.08498...
+
+
+def test_conv_softmax_pool_full_size_sampled_images(kf):
+    """bench.py --workload pool: config 5's tensors, pool 4; the oracle recomputes three images."""
+    d = ki.conv_inputs("c5", seed=0)
+    y = kf.conv3x3_softmax_pool(to_dev(d["x"]), to_dev(d["w"]), to_dev(d["bias"]), 4)
+    check_status()
+    imgs = [0, 63, 127]
+    ref = oracle.conv3x3_softmax_pool(d["x"][imgs], d["w"], d["bias"], 4)
+    got = to_f64(y[imgs])
+    assert_close(got, ref, 2e-2, 2e-2, "conv softmax pool sampled images")
+    assert_close(got, ref, 1e-6, 2e-2, "conv softmax pool sampled images, relative")
+    yy = y.float()
+    assert float(yy.min()) > 0 and float(yy.max()) <= 1.0

@@ -228,6 +228,48 @@ bool use_cta_pairs(int64_t M, int64_t K) {
 }
 size_t rowreduce_simt_ws(int64_t M, int64_t N) { return round256(static_cast<size_t>(M) * N * 4); }
 
+// The fp32 chain on the tensor cores: split prepasses into `ws` (tf32_ws bytes), then the GEMM
+// kernel with its epilogue.  Y may be any fp32 [M, ldy] buffer (the row reductions pass their
+// pre-reduction matrix).
+kf_status run_tf32_chain(int64_t M, int64_t N, int64_t K, const void* X, int64_t ldx, const void* W,
+                         int64_t ldw, const void* bias, int act, float scale, const void* residual,
+                         int64_t ldr, void* Y, int64_t ldy, void* ws, DeviceInfo* d, cudaStream_t st) {
+  const int64_t kp = tf32_kp(K);
+  const size_t xb = round256(static_cast<size_t>(M) * kp * 4), wb = round256(static_cast<size_t>(N) * kp * 4);
+  float* xh = static_cast<float*>(ws);
+  float* xl = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + xb);
+  float* wh = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + 2 * xb);
+  float* wl = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + 2 * xb + wb);
+  if (launch_tf32_split(M, static_cast<int>(K), static_cast<int>(kp), static_cast<const float*>(X), ldx,
+                        xh, xl, st) != cudaSuccess ||
+      launch_tf32_split(N, static_cast<int>(K), static_cast<int>(kp), static_cast<const float*>(W), ldw,
+                        wh, wl, st) != cudaSuccess)
+    return KF_ERR_CUDA;
+  const int bn = N <= 128 ? 128 : 256;
+  CUtensorMap ah, al, bh, bl;
+  if (!encode_2d_f32(&ah, xh, M, K, kp, kBM) || !encode_2d_f32(&al, xl, M, K, kp, kBM) ||
+      !encode_2d_f32(&bh, wh, N, K, kp, bn) || !encode_2d_f32(&bl, wl, N, K, kp, bn))
+    return KF_ERR_CUDA;
+  Tf32Params p;
+  std::memset(&p, 0, sizeof(p));
+  p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+  p.tiles_m = static_cast<int>((M + kBM - 1) / kBM);
+  p.tiles_n = static_cast<int>((N + bn - 1) / bn);
+  if (static_cast<int64_t>(p.tiles_m) * p.tiles_n > kMaxDim) return KF_ERR_UNSUPPORTED;
+  p.num_tiles = p.tiles_m * p.tiles_n;
+  p.k_blocks = static_cast<int>((K + 15) / 16);
+  p.bias = static_cast<const float*>(bias);
+  p.R = static_cast<const float*>(residual);
+  p.ldr = ldr; p.out = static_cast<float*>(Y); p.ldo = ldy; p.scale = scale; p.act = act;
+  p.vec_ok = (ldy % 4 == 0 && aligned(Y, 16) &&
+              (residual == nullptr || (ldr % 4 == 0 && aligned(residual, 16)))) ? 1 : 0;
+  p.status = d->status;
+  const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
+  if (launch_tf32_chain(bn, ah, al, bh, bl, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
+  g_launches += 3;
+  return KF_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -270,7 +312,7 @@ size_t kf_gemm_rowreduce_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dty
                                          kf_rowred red) {
   if (M < 1 || N < 1 || K < 1) return 0;
   if (in_dtype == KF_BF16 && K % 8 == 0) return rowreduce_umma_ws(M, N, red);
-  return rowreduce_simt_ws(M, N);
+  return rowreduce_simt_ws(M, N) + (use_tf32x3(in_dtype, M, N, K) ? tf32_ws(M, N, K) : 0);
 }
 
 size_t kf_conv3x3_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
@@ -301,40 +343,8 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
   if (use_tf32x3(io_dtype, M, N, K)) {
     vs = check_workspace(workspace, workspace_bytes, tf32_ws(M, N, K));
     if (vs != KF_OK) return vs;
-    const int64_t kp = tf32_kp(K);
-    const size_t xb = round256(static_cast<size_t>(M) * kp * 4), wb = round256(static_cast<size_t>(N) * kp * 4);
-    float* xh = static_cast<float*>(workspace);
-    float* xl = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + xb);
-    float* wh = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 2 * xb);
-    float* wl = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 2 * xb + wb);
-    if (launch_tf32_split(M, static_cast<int>(K), static_cast<int>(kp), static_cast<const float*>(X), ldx,
-                          xh, xl, st) != cudaSuccess ||
-        launch_tf32_split(N, static_cast<int>(K), static_cast<int>(kp), static_cast<const float*>(W), ldw,
-                          wh, wl, st) != cudaSuccess)
-      return KF_ERR_CUDA;
-    const int bn = N <= 128 ? 128 : 256;
-    CUtensorMap ah, al, bh, bl;
-    if (!encode_2d_f32(&ah, xh, M, K, kp, kBM) || !encode_2d_f32(&al, xl, M, K, kp, kBM) ||
-        !encode_2d_f32(&bh, wh, N, K, kp, bn) || !encode_2d_f32(&bl, wl, N, K, kp, bn))
-      return KF_ERR_CUDA;
-    Tf32Params p;
-    std::memset(&p, 0, sizeof(p));
-    p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
-    p.tiles_m = static_cast<int>((M + kBM - 1) / kBM);
-    p.tiles_n = static_cast<int>((N + bn - 1) / bn);
-    if (static_cast<int64_t>(p.tiles_m) * p.tiles_n > kMaxDim) return KF_ERR_UNSUPPORTED;
-    p.num_tiles = p.tiles_m * p.tiles_n;
-    p.k_blocks = static_cast<int>((K + 15) / 16);
-    p.bias = static_cast<const float*>(bias);
-    p.R = static_cast<const float*>(residual);
-    p.ldr = ldr; p.out = static_cast<float*>(Y); p.ldo = ldy; p.scale = scale; p.act = act;
-    p.vec_ok = (ldy % 4 == 0 && aligned(Y, 16) &&
-                (residual == nullptr || (ldr % 4 == 0 && aligned(residual, 16)))) ? 1 : 0;
-    p.status = d->status;
-    const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
-    if (launch_tf32_chain(bn, ah, al, bh, bl, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
-    g_launches += 3;
-    return KF_OK;
+    return run_tf32_chain(M, N, K, X, ldx, W, ldw, bias, act, scale, residual, ldr, Y, ldy, workspace,
+                          d, st);
   }
   int bn_split = 0;
   const int split = umma_gemm_ok(io_dtype, K, X, ldx, W, ldw)
@@ -486,11 +496,18 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
     return KF_OK;
   }
   // scalar path: pre-reduction values in fp32, then one CTA per row
-  vs = check_workspace(workspace, workspace_bytes, rowreduce_simt_ws(M, N));
+  const bool tensor32 = use_tf32x3(in_dtype, M, N, K);    // large fp32: GEMM on the tensor cores
+  vs = check_workspace(workspace, workspace_bytes,
+                       rowreduce_simt_ws(M, N) + (tensor32 ? tf32_ws(M, N, K) : 0));
   if (vs != KF_OK) return vs;
   float* A = static_cast<float*>(workspace);
-  if (launch_simt_gemm(in_dtype, 1, pre_act, Mi, Ni, Ki, X, ldx, W, ldw, bias, 1.0f, nullptr, 0, A,
-                       N, st) != cudaSuccess)
+  if (tensor32) {
+    vs = run_tf32_chain(M, N, K, X, ldx, W, ldw, bias, pre_act, 1.0f, nullptr, 0, A, N,
+                        static_cast<uint8_t*>(workspace) + rowreduce_simt_ws(M, N), d, st);
+    if (vs != KF_OK) return vs;
+    g_launches -= 1;      // counted below as the scalar path's GEMM launch
+  } else if (launch_simt_gemm(in_dtype, 1, pre_act, Mi, Ni, Ki, X, ldx, W, ldw, bias, 1.0f, nullptr, 0, A,
+                              N, st) != cudaSuccess)
     return KF_ERR_CUDA;
   cudaError_t e = red == KF_RED_SOFTMAX ? launch_row_softmax(out_dtype, Mi, Ni, A, N, out, ldo, st)
                                         : launch_row_sum(Mi, Ni, A, N, static_cast<float*>(out), st);

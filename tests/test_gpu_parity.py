@@ -353,7 +353,8 @@ def test_rowsum_closed_forms(kf):
 
 
 @pytest.mark.parametrize("red,act", [("softmax", "none"), ("sum", "sigmoid"), ("softmax", "relu")])
-@pytest.mark.parametrize("dtype,shape", [("f32", (33, 70, 31)), ("f32", (128, 256, 512)), ("bf16", (9, 21, 13))])
+@pytest.mark.parametrize("dtype,shape", [("f32", (33, 70, 31)), ("f32", (128, 256, 512)), ("bf16", (9, 21, 13)),
+                                         ("f32", (1024, 1000, 600))])   # GEMM on the tensor cores (3xTF32)
 def test_scalar_path_row_reductions(kf, red, act, dtype, shape):
     M, N, K = shape
     d = ki.gemm_inputs("c3", seed=4, M=M, N=N, K=K, dtype=dtype)

@@ -431,6 +431,7 @@ SWEEP_CONV = [  # (Nb, Cin, H, W, Cout, groups [GroupNorm] or -pool [softmax + m
     (16, 64, 32, 32, 64, 8), (128, 64, 64, 64, 128, 32), (32, 128, 32, 32, 128, 16),
     (8, 64, 128, 128, 64, 4), (64, 64, 16, 16, 256, 32), (10, 3, 30, 30, 16, 4),
     (128, 64, 64, 64, 128, -4), (16, 64, 32, 32, 16, -2),
+    (32, 64, 56, 56, 64, 8), (32, 128, 28, 28, 128, 8), (32, 256, 14, 14, 256, 8), (16, 3, 224, 224, 64, 8),
 ]
 
 

@@ -138,8 +138,10 @@ kf_status kf_gemm_rowreduce_static(int64_t M, int64_t N, int64_t K, kf_dtype in_
  *   groups == 0: y = a.
  * x is NCHW [Nb,Cin,H,Wd], w is OIHW [Cout,Cin,3,3], y is NCHW [Nb,Cout,H,Wd], all dense, of
  * io_dtype.  bias, gamma, beta may be NULL (0, 1, 0).  y must not alias x.
- * bf16 problems with Cin % 64 == 0, Wd in {8,16,32,64,128}, (H*Wd) % 128 == 0 and a 16-byte
- * aligned x take the implicit-GEMM tensor-core kernel; everything else takes a scalar kernel.
+ * bf16 problems take the implicit-GEMM tensor-core kernel whenever some number of image rows
+ * r makes r*Wd a multiple of 32 that is at most 256 (every Wd <= 256 that is a multiple of 8,
+ * also Wd = 7, 14, 28, 56; Wd = 30 is not); Cin is padded to a multiple of 64 in the
+ * workspace copy and H may leave a partial last tile.  Everything else takes a scalar kernel.
  * groups must divide Cout. */
 kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
                               kf_dtype io_dtype, const void* x, const void* w, const void* bias,

@@ -133,15 +133,32 @@ bool umma_gemm_ok(int dt, int64_t K, const void* X, int64_t ldx, const void* W, 
          aligned(W, 16);
 }
 
-bool conv_umma_shape_ok(int dt, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout) {
-  (void)Cout;
-  const bool w_ok = Wd == 8 || Wd == 16 || Wd == 32 || Wd == 64 || Wd == 128;
-  return dt == DT_BF16 && Cin % 64 == 0 && w_ok && (H * Wd) % 128 == 0;
+// Image rows per tile of the tensor-core convolution: the most rows r with r*Wd <= 256 pixels
+// and r*Wd a multiple of 32 (whole epilogue pieces; also a valid UMMA N), preferring r <= H.
+// 0 = no such tiling (Wd > 256, or an odd width whose smallest multiple is too large).
+int conv_rows_per_tile(int64_t H, int64_t Wd) {
+  if (Wd < 1 || Wd > 256) return 0;
+  int64_t g = Wd, b = 32;                        // step = 32 / gcd(Wd, 32)
+  while (b != 0) { const int64_t t = g % b; g = b; b = t; }
+  const int64_t step = 32 / g;
+  if (step * Wd > 256) return 0;
+  int64_t r = (256 / Wd) / step * step;          // largest multiple of step that fits
+  const int64_t cap = (H + step - 1) / step * step;   // no more rows than cover the image
+  if (r > cap) r = cap;
+  return static_cast<int>(r);
 }
-// pixels per tile: 256 when whole tiles of 256 pixels cover the image, else 128
-int conv_tile_pixels(int64_t H, int64_t Wd) { return (H * Wd) % 256 == 0 ? 256 : 128; }
+bool conv_umma_shape_ok(int dt, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout) {
+  (void)Cin; (void)Cout;
+  return dt == DT_BF16 && conv_rows_per_tile(H, Wd) > 0;
+}
+int64_t conv_cpad(int64_t Cin) { return (Cin + 63) / 64 * 64; }   // channels of the NHWC copy
+// pixels per tile (the UMMA N)
+int conv_tile_pixels(int64_t H, int64_t Wd) { return static_cast<int>(conv_rows_per_tile(H, Wd) * Wd); }
 // statistics entries per image: one per pixel tile
-int64_t conv_stat_parts(int64_t H, int64_t Wd) { return (H * Wd) / conv_tile_pixels(H, Wd); }
+int64_t conv_stat_parts(int64_t H, int64_t Wd) {
+  const int r = conv_rows_per_tile(H, Wd);
+  return (H + r - 1) / r;
+}
 size_t conv_stats_bytes(int64_t Nb, int64_t H, int64_t Wd, int64_t Cout) {
   return round256(static_cast<size_t>(Nb) * conv_stat_parts(H, Wd) * Cout * 8);
 }
@@ -320,8 +337,8 @@ size_t kf_conv3x3_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd
   (void)groups;
   if (Nb < 1 || Cin < 1 || H < 1 || Wd < 1 || Cout < 1) return 0;
   if (!conv_umma_shape_ok(io_dtype, Cin, H, Wd, Cout)) return 0;
-  return round256(static_cast<size_t>(Nb) * H * Wd * Cin * 2) +
-         round256(static_cast<size_t>(9) * Cout * Cin * 2) + conv_stats_bytes(Nb, H, Wd, Cout);
+  return round256(static_cast<size_t>(Nb) * H * Wd * conv_cpad(Cin) * 2) +
+         round256(static_cast<size_t>(9) * Cout * conv_cpad(Cin) * 2) + conv_stats_bytes(Nb, H, Wd, Cout);
 }
 
 kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, const void* X,
@@ -538,44 +555,49 @@ kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   int launches = 0;
 
-  if (conv_umma_shape_ok(io_dtype, Cin, H, Wd, Cout) && aligned(x, 16)) {
-    const size_t xt_bytes = round256(static_cast<size_t>(Nb) * hw * Cin * 2);
-    const size_t wr_bytes = round256(static_cast<size_t>(9) * Cout * Cin * 2);
+  if (conv_umma_shape_ok(io_dtype, Cin, H, Wd, Cout)) {
+    const int64_t Cp = conv_cpad(Cin);
+    const size_t xt_bytes = round256(static_cast<size_t>(Nb) * hw * Cp * 2);
+    const size_t wr_bytes = round256(static_cast<size_t>(9) * Cout * Cp * 2);
     const size_t st_bytes = conv_stats_bytes(Nb, H, Wd, Cout);
     kf_status vs = check_workspace(workspace, workspace_bytes, xt_bytes + wr_bytes + st_bytes);
     if (vs != KF_OK) return vs;
     void* xt = workspace;
     void* wr = static_cast<uint8_t*>(workspace) + xt_bytes;
     float* stats = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + xt_bytes + wr_bytes);
-    if (launch_conv_prep(static_cast<int>(Nb), static_cast<int>(Cin), static_cast<int>(H),
-                         static_cast<int>(Wd), static_cast<int>(Cout), x, w, xt, wr, st) != cudaSuccess)
+    if (launch_conv_prep(static_cast<int>(Nb), static_cast<int>(Cin), static_cast<int>(Cp),
+                         static_cast<int>(H), static_cast<int>(Wd), static_cast<int>(Cout), x, w, xt, wr,
+                         st) != cudaSuccess)
       return KF_ERR_CUDA;
     ++launches;
-    const int bn = conv_tile_pixels(H, Wd);            // pixels per tile = UMMA N
-    const int rows = static_cast<int>(bn / Wd);        // image rows per tile
+    const int rows = conv_rows_per_tile(H, Wd);        // image rows per tile
+    const int tile_px = static_cast<int>(rows * Wd);   // pixels per tile = UMMA N
+    const int bn = tile_px > 128 ? 256 : 128;          // kernel instance: room for that many pixels
     UmmaMaps tm;
-    // A: weights [9*Cout, Cin], 128 output channels per tile; B: NHWC activations
-    if (!encode_2d(&tm.a, wr, 9 * Cout, Cin, Cin, kBM) || !encode_nhwc(&tm.b, xt, Nb, H, Wd, Cin, rows))
+    // A: weights [9*Cout, Cp], 128 output channels per tile; B: NHWC activations
+    if (!encode_2d(&tm.a, wr, 9 * Cout, Cp, Cp, kBM) || !encode_nhwc(&tm.b, xt, Nb, H, Wd, Cp, rows))
       return KF_ERR_CUDA;
     tm.r = tm.a; tm.y = tm.a;
     UmmaParams p;
     std::memset(&p, 0, sizeof(p));
-    p.M = static_cast<int>(Nb * hw); p.N = static_cast<int>(Cout); p.K = static_cast<int>(9 * Cin);
-    p.tiles_per_image = static_cast<int>(hw / bn);
+    p.M = static_cast<int>(Nb * hw); p.N = static_cast<int>(Cout); p.K = static_cast<int>(9 * Cp);
+    p.tiles_per_image = static_cast<int>(conv_stat_parts(H, Wd));
+    p.tile_px = tile_px;
     p.tiles_m = static_cast<int>((Cout + kBM - 1) / kBM);              // output-channel tiles
     p.tiles_n = static_cast<int>(Nb) * p.tiles_per_image;              // pixel tiles
     if (static_cast<int64_t>(p.tiles_m) * p.tiles_n > kMaxDim) return KF_ERR_UNSUPPORTED;
     p.num_tiles = p.tiles_m * p.tiles_n;
-    p.kb_per_tap = static_cast<int>(Cin / kBK);
+    p.kb_per_tap = static_cast<int>(Cp / kBK);
     p.k_blocks = 9 * p.kb_per_tap;
     p.tiles_per_unit = 1;
     p.bias = static_cast<const __nv_bfloat16*>(bias);
     p.out = y; p.scale = 1.0f;
     p.partial = groups > 0 ? stats : nullptr;
     p.status = d->status;
-    p.H = static_cast<int>(H); p.Wd = static_cast<int>(Wd); p.Cin = static_cast<int>(Cin);
+    p.H = static_cast<int>(H); p.Wd = static_cast<int>(Wd); p.Cin = static_cast<int>(Cp);
     p.rows_per_tile = rows;
-    p.staged = aligned(y, 16) ? 1 : 0;
+    // the output pieces travel by TMA when every image plane starts on 16 bytes
+    p.staged = (aligned(y, 16) && hw % 8 == 0) ? 1 : 0;
     if (p.staged && !encode_nchw_out(&tm.y, y, Nb, Cout, hw)) return KF_ERR_CUDA;
     const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
     if (launch_umma_conv(bn, act, tm, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;

@@ -49,7 +49,7 @@ cudaError_t launch_row_sum(int M, int N, const float* A, long long lda, float* o
                            cudaStream_t st);
 
 // convolution helpers
-cudaError_t launch_conv_prep(int Nb, int Cin, int H, int Wd, int Cout, const void* x,
+cudaError_t launch_conv_prep(int Nb, int Cin, int Cp, int H, int Wd, int Cout, const void* x,
                              const void* w, void* xt, void* wr, cudaStream_t st);
 cudaError_t launch_conv_direct(int dt, int act, int Nb, int Cin, int H, int Wd, int Cout,
                                const void* x, const void* w, const void* bias, void* y,

@@ -85,15 +85,26 @@ cudaError_t launch_rowsum_finalize(int M, int tiles_n, const float* partial, flo
   return cudaGetLastError();
 }
 
-cudaError_t launch_conv_prep(int Nb, int Cin, int H, int Wd, int Cout, const void* x,
+cudaError_t launch_conv_prep(int Nb, int Cin, int Cp, int H, int Wd, int Cout, const void* x,
                              const void* w, void* xt, void* wr, cudaStream_t st) {
-  const long long x_blocks = static_cast<long long>(Nb) * H * (Cin / 8) * (Wd / 8);
-  const long long total = x_blocks + 9ll * Cout * Cin;
-  const long long grid = (total + 255) / 256;
-  conv_prep_kernel<<<static_cast<unsigned>(grid), 256, 0, st>>>(
-      Nb, Cin, H, Wd, Cout, static_cast<const __nv_bfloat16*>(x),
-      static_cast<const __nv_bfloat16*>(w), static_cast<__nv_bfloat16*>(xt),
-      static_cast<__nv_bfloat16*>(wr), x_blocks);
+  const __nv_bfloat16* xs = static_cast<const __nv_bfloat16*>(x);
+  const __nv_bfloat16* ws = static_cast<const __nv_bfloat16*>(w);
+  __nv_bfloat16* xd = static_cast<__nv_bfloat16*>(xt);
+  __nv_bfloat16* wd = static_cast<__nv_bfloat16*>(wr);
+  if (Cp == Cin && Cin % 8 == 0 && Wd % 8 == 0 && reinterpret_cast<uintptr_t>(x) % 16 == 0) {
+    const long long x_blocks = static_cast<long long>(Nb) * H * (Cin / 8) * (Wd / 8);
+    const long long total = x_blocks + 9ll * Cout * Cin;
+    const long long grid = (total + 255) / 256;
+    conv_prep_kernel<<<static_cast<unsigned>(grid), 256, 0, st>>>(Nb, Cin, H, Wd, Cout, xs, ws, xd, wd,
+                                                                  x_blocks);
+  } else {
+    const long long x_items = static_cast<long long>(Nb) * H * Wd * (Cp / 8);
+    const long long total = x_items + 9ll * Cout * Cp;
+    const long long grid = (total + 255) / 256;
+    if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
+    conv_prep_general_kernel<<<static_cast<unsigned>(grid), 256, 0, st>>>(Nb, Cin, Cp, H, Wd, Cout, xs, ws,
+                                                                          xd, wd, x_items);
+  }
   return cudaGetLastError();
 }
 

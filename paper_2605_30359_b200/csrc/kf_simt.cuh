@@ -319,6 +319,46 @@ conv_prep_kernel(int Nb, int Cin, int H, int Wd, int Cout, const __nv_bfloat16* 
   }
 }
 
+// General form of the prepass: any Cin and Wd, channels padded with zeros to Cp (a multiple of
+// 64, the K block of the implicit GEMM).  One thread per pixel and block of eight channels,
+// pixels fastest across threads: reads run along w, each thread writes one 16-byte vector.
+__global__ void __launch_bounds__(256)
+conv_prep_general_kernel(int Nb, int Cin, int Cp, int H, int Wd, int Cout,
+                         const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
+                         __nv_bfloat16* __restrict__ xt, __nv_bfloat16* __restrict__ wr,
+                         long long x_items) {
+  const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const long long hw = static_cast<long long>(H) * Wd;
+  const int cbk = Cp / 8;
+  if (gid < x_items) {
+    const long long px = gid % hw;                       // pixel inside the image
+    long long t = gid / hw;
+    const int cblk = static_cast<int>(t % cbk);
+    const long long n = t / cbk;
+    unsigned short e[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int c = cblk * 8 + i;
+      e[i] = c < Cin ? __bfloat16_as_ushort(x[(n * Cin + c) * hw + px]) : static_cast<unsigned short>(0);
+    }
+    uint4 o;
+    o.x = e[0] | (static_cast<uint32_t>(e[1]) << 16);
+    o.y = e[2] | (static_cast<uint32_t>(e[3]) << 16);
+    o.z = e[4] | (static_cast<uint32_t>(e[5]) << 16);
+    o.w = e[6] | (static_cast<uint32_t>(e[7]) << 16);
+    *reinterpret_cast<uint4*>(xt + (n * hw + px) * Cp + cblk * 8) = o;
+  } else {
+    const long long i = gid - x_items;                   // index into wr[tap][o][Cp]
+    const long long total = 9ll * Cout * Cp;
+    if (i < total) {
+      const int c = static_cast<int>(i % Cp);
+      const int o = static_cast<int>((i / Cp) % Cout);
+      const int tap = static_cast<int>(i / (static_cast<long long>(Cp) * Cout));
+      wr[i] = c < Cin ? w[(static_cast<long long>(o) * Cin + c) * 9 + tap] : __float2bfloat16_rn(0.0f);
+    }
+  }
+}
+
 // ---------------------------------------------------------------- conv: scalar path
 // One thread per output element, taps with an explicit bounds test; stores act(c) in T.
 template <typename T, int ACT>

@@ -63,6 +63,7 @@ struct UmmaParams {
   int tiles_per_unit;
   // conv only
   int H, Wd, Cin, rows_per_tile, tiles_per_image, kb_per_tap;
+  int tile_px;                 // pixels per tile = rows_per_tile * Wd = UMMA N (a multiple of 32, <= BN)
 };
 
 // The it-th tile of scheduling slot `cta` out of `ncta`, or -1 when the slot has no more work.
@@ -206,7 +207,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if (++s == kStages) { s = 0; ph ^= 1u; }
             continue;
           }
-          mbar_expect_tx(&full[s], C::kStage);
+          // a convolution tile fetches tile_px <= BN pixel rows of 128 bytes
+          mbar_expect_tx(&full[s], EPI == EPI_CONV ? C::kStageA + p.tile_px * kBK * 2 : C::kStage);
           if constexpr (EPI == EPI_CONV) {
             const int tap = kb / p.kb_per_tap, cb = kb % p.kb_per_tap;
             const int r = tap / 3, sx = tap % 3;
@@ -227,7 +229,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   } else if (warp == 1) {
     // ------------------------------------------------------------ UMMA issuer
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16_f32(kTileM, BN);
+      const uint32_t idesc =
+          umma_idesc_bf16_f32(kTileM, EPI == EPI_CONV ? static_cast<uint32_t>(p.tile_px) : BN);
       int s = 0; uint32_t ph = 0; int a = 0; uint32_t aph = 0;
       bool ok = true;
       for (int it = 0; ok; ++it) {
@@ -578,19 +581,27 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int pt = tn % p.tiles_per_image;              // pixel tile inside the image
         const float bias_v = (p.bias != nullptr && ch_ok) ? __bfloat162float(p.bias[ch]) : 0.0f;
         const long long hw = static_cast<long long>(p.H) * p.Wd;
+        const int pieces = p.tile_px / 32;                  // <= PIECES
+        const int px0 = pt * p.tile_px;                     // first pixel of the tile in its image
+        // the last tile of an image may hang over its end: those pixels were read as zeros, are
+        // left out of the statistics and are not stored
+        const int px_valid = static_cast<int>(min(static_cast<long long>(p.tile_px), hw - px0));
         float s1 = 0.0f, s2 = 0.0f;
 #pragma unroll 1
-        for (int c = 0; c < PIECES; ++c, ++g) {
+        for (int c = 0; c < pieces; ++c, ++g) {
           uint32_t v[32];
           tmem_ld_32x32(t_acc + c * 32, v);
           tmem_ld_wait();
-          if (c == PIECES - 1) release_acc();
+          if (c == pieces - 1) release_acc();
           uint32_t w[16];
+          const int left = px_valid - c * 32;               // valid pixels from this piece on
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            const float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + bias_v);
-            const float y1 = act_f<ACT, true>(__uint_as_float(v[2 * j + 1]) + bias_v);
+            float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + bias_v);
+            float y1 = act_f<ACT, true>(__uint_as_float(v[2 * j + 1]) + bias_v);
             w[j] = pack_bf16x2(y0, y1);
+            if (2 * j >= left) y0 = 0.0f;
+            if (2 * j + 1 >= left) y1 = 0.0f;
             s1 += y0 + y1;
             s2 = fmaf(y0, y0, fmaf(y1, y1, s2));
           }
@@ -604,18 +615,19 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             fence_proxy_async_smem();
             if (leader) bulk_wait_group_read<0>();     // the other buffer's store has let go
             named_barrier_sync(bar_b, kEpiThreads);
-            if (leader) {
-              // box = 32 pixels x 128 channels of image img; channels past Cout are clipped
-              tma_store_3d(&tmY, yb, pt * BN + c * 32, tm * kBM, img);
+            if (leader && left > 0) {
+              // box = 32 pixels x 128 channels of image img; channels past Cout and pixels past
+              // the image are clipped
+              tma_store_3d(&tmY, yb, px0 + c * 32, tm * kBM, img);
               bulk_commit_group();
             }
           } else if (ch_ok) {
             __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) +
-                                 (static_cast<long long>(img) * p.N + ch) * hw + pt * BN + c * 32;
+                                 (static_cast<long long>(img) * p.N + ch) * hw + px0 + c * 32;
 #pragma unroll
             for (int j = 0; j < 16; ++j) {       // the output may be only 2-byte aligned here
-              dst[2 * j] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j] & 0xFFFFu));
-              dst[2 * j + 1] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j] >> 16));
+              if (2 * j < left) dst[2 * j] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j] & 0xFFFFu));
+              if (2 * j + 1 < left) dst[2 * j + 1] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j] >> 16));
             }
           }
         }

@@ -392,6 +392,26 @@ def test_bf16_conv_tensor_core_path(kf, cfg):
     assert_close(got, ref, 2e-2, 2e-2, "conv %s" % cfg)
 
 
+# Any width up to 256 whose rows tile into multiples of 32 pixels, any Cin (padded to 64) and any
+# H (the last tile of an image may hang over its end) take the tensor-core convolution too.
+@pytest.mark.parametrize("cfg", [
+    dict(Nb=2, Cin=64, H=56, W=56, Cout=64, groups=8),       # 4 rows x 56 = 224-pixel tiles
+    dict(Nb=2, Cin=128, H=28, W=28, Cout=32, groups=4),      # 8 rows per tile, last tile 4 rows
+    dict(Nb=2, Cin=256, H=14, W=14, Cout=256, groups=8),     # planes of 196 pixels: no TMA store
+    dict(Nb=1, Cin=3, H=32, W=32, Cout=16, groups=4),        # 3 channels padded to 64
+    dict(Nb=2, Cin=32, H=7, W=7, Cout=64, groups=8),         # 32-row box on a 7-row image
+    dict(Nb=1, Cin=64, H=5, W=96, Cout=40, groups=5),        # 2 rows per tile, ragged last tile
+    dict(Nb=1, Cin=20, H=9, W=24, Cout=24, groups=3),        # padded channels, ragged rows
+    dict(Nb=1, Cin=8, H=3, W=224, Cout=8, groups=0),         # one row per tile
+])
+def test_bf16_conv_tensor_core_general_shapes(kf, cfg):
+    d = ki.conv_inputs(seed=6, **cfg)
+    got, ref = run_conv(kf, d)
+    assert_close(got, ref, 2e-2, 2e-2, "conv general %s" % cfg)
+    got, ref = run_conv(kf, d, act="none", groups=0, use_bias=False)
+    assert_close(got, ref, 2e-2, 2e-2, "conv general bare %s" % cfg)
+
+
 def test_bf16_conv_position_pins(kf):
     """Delta kernels and all-ones inputs: exact results that pin tap orientation and padding."""
     Nb, C, H, W = 2, 64, 8, 64

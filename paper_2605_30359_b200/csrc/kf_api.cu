@@ -95,15 +95,15 @@ bool encode_piece(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols,
   return encode_2d(tm, base, rows, cols, ld, kBM, kPieceCols, CU_TENSOR_MAP_SWIZZLE_64B);
 }
 
-// NHWC bf16 activations [Nb,H,W,C] -> boxes of 64 channels x W pixels x rows image rows.
+// NHWC bf16 activations [Nb,H,W,C] -> boxes of 64 channels x box_w pixels x rows image rows.
 bool encode_nhwc(CUtensorMap* tm, const void* base, int64_t Nb, int64_t H, int64_t Wd, int64_t C,
-                 int rows) {
+                 int rows, int box_w) {
   const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(Wd),
                               static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(Nb)};
   const cuuint64_t strides[3] = {static_cast<cuuint64_t>(C) * 2,
                                  static_cast<cuuint64_t>(Wd) * C * 2,
                                  static_cast<cuuint64_t>(H) * Wd * C * 2};
-  const cuuint32_t box[4] = {static_cast<cuuint32_t>(kBK), static_cast<cuuint32_t>(Wd),
+  const cuuint32_t box[4] = {static_cast<cuuint32_t>(kBK), static_cast<cuuint32_t>(box_w),
                              static_cast<cuuint32_t>(rows), 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides,
@@ -136,8 +136,17 @@ bool umma_gemm_ok(int dt, int64_t K, const void* X, int64_t ldx, const void* W, 
 // Image rows per tile of the tensor-core convolution: the most rows r with r*Wd <= 256 pixels
 // and r*Wd a multiple of 32 (whole epilogue pieces; also a valid UMMA N), preferring r <= H.
 // 0 = no such tiling (Wd > 256, or an odd width whose smallest multiple is too large).
+// Segments per image row: 1 up to 256 pixels; wider rows are cut into the fewest equal segments
+// of at most 256 pixels that are multiples of 32 (0 = none exists).
+int conv_w_segs(int64_t Wd) {
+  if (Wd <= 256) return 1;
+  for (int64_t k = (Wd + 255) / 256; k <= Wd / 32; ++k)
+    if (Wd % k == 0 && (Wd / k) % 32 == 0) return static_cast<int>(k);
+  return 0;
+}
 int conv_rows_per_tile(int64_t H, int64_t Wd) {
-  if (Wd < 1 || Wd > 256) return 0;
+  if (Wd > 256) return conv_w_segs(Wd) > 0 ? 1 : 0;
+  if (Wd < 1) return 0;
   int64_t g = Wd, b = 32;                        // step = 32 / gcd(Wd, 32)
   while (b != 0) { const int64_t t = g % b; g = b; b = t; }
   const int64_t step = 32 / g;
@@ -153,11 +162,13 @@ bool conv_umma_shape_ok(int dt, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout
 }
 int64_t conv_cpad(int64_t Cin) { return (Cin + 63) / 64 * 64; }   // channels of the NHWC copy
 // pixels per tile (the UMMA N)
-int conv_tile_pixels(int64_t H, int64_t Wd) { return static_cast<int>(conv_rows_per_tile(H, Wd) * Wd); }
+int conv_tile_pixels(int64_t H, int64_t Wd) {
+  return static_cast<int>(conv_rows_per_tile(H, Wd) * Wd / conv_w_segs(Wd));
+}
 // statistics entries per image: one per pixel tile
 int64_t conv_stat_parts(int64_t H, int64_t Wd) {
   const int r = conv_rows_per_tile(H, Wd);
-  return (H + r - 1) / r;
+  return (H + r - 1) / r * conv_w_segs(Wd);
 }
 size_t conv_stats_bytes(int64_t Nb, int64_t H, int64_t Wd, int64_t Cout) {
   return round256(static_cast<size_t>(Nb) * conv_stat_parts(H, Wd) * Cout * 8);
@@ -571,11 +582,12 @@ kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
       return KF_ERR_CUDA;
     ++launches;
     const int rows = conv_rows_per_tile(H, Wd);        // image rows per tile
-    const int tile_px = static_cast<int>(rows * Wd);   // pixels per tile = UMMA N
+    const int segs = conv_w_segs(Wd);                  // > 1: a tile is one segment of one row
+    const int tile_px = static_cast<int>(rows * Wd / segs);   // pixels per tile = UMMA N
     const int bn = tile_px > 128 ? 256 : 128;          // kernel instance: room for that many pixels
     UmmaMaps tm;
     // A: weights [9*Cout, Cp], 128 output channels per tile; B: NHWC activations
-    if (!encode_2d(&tm.a, wr, 9 * Cout, Cp, Cp, kBM) || !encode_nhwc(&tm.b, xt, Nb, H, Wd, Cp, rows))
+    if (!encode_2d(&tm.a, wr, 9 * Cout, Cp, Cp, kBM) || !encode_nhwc(&tm.b, xt, Nb, H, Wd, Cp, rows, static_cast<int>(Wd / segs)))
       return KF_ERR_CUDA;
     tm.r = tm.a; tm.y = tm.a;
     UmmaParams p;
@@ -583,6 +595,7 @@ kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
     p.M = static_cast<int>(Nb * hw); p.N = static_cast<int>(Cout); p.K = static_cast<int>(9 * Cp);
     p.tiles_per_image = static_cast<int>(conv_stat_parts(H, Wd));
     p.tile_px = tile_px;
+    p.w_segs = segs;
     p.tiles_m = static_cast<int>((Cout + kBM - 1) / kBM);              // output-channel tiles
     p.tiles_n = static_cast<int>(Nb) * p.tiles_per_image;              // pixel tiles
     if (static_cast<int64_t>(p.tiles_m) * p.tiles_n > kMaxDim) return KF_ERR_UNSUPPORTED;

@@ -63,7 +63,9 @@ struct UmmaParams {
   int tiles_per_unit;
   // conv only
   int H, Wd, Cin, rows_per_tile, tiles_per_image, kb_per_tap;
-  int tile_px;                 // pixels per tile = rows_per_tile * Wd = UMMA N (a multiple of 32, <= BN)
+  int tile_px;                 // pixels per tile = UMMA N (a multiple of 32, <= BN): rows_per_tile
+                               // whole rows, or one of w_segs equal segments of a row
+  int w_segs;                  // 1, or segments per row when Wd > 256 (then rows_per_tile = 1)
 };
 
 // The it-th tile of scheduling slot `cta` out of `ncta`, or -1 when the slot has no more work.
@@ -185,11 +187,13 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       for (int it = 0;; ++it) {
         const int tile = sched_tile(p, cta, ncta, it);
         if (tile < 0) break;
-        int tm, tn, img = 0, h0 = 0;
+        int tm, tn, img = 0, h0 = 0, x0 = 0;
         if constexpr (EPI == EPI_CONV) {
           tm = tile % p.tiles_m; tn = tile / p.tiles_m;        // output-channel tile, pixel tile
           img = tn / p.tiles_per_image;
-          h0 = (tn % p.tiles_per_image) * p.rows_per_tile;
+          const int pt = tn % p.tiles_per_image;
+          h0 = (pt / p.w_segs) * p.rows_per_tile;
+          x0 = (pt % p.w_segs) * (p.Wd / p.w_segs);
         } else {
           tm = tile / p.tiles_n; tn = tile % p.tiles_n;
         }
@@ -215,7 +219,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             // A: this tap's weights for 128 output channels.  B: BN pixels x 64 input channels
             // of the window shifted by the tap; out-of-image pixels read zeros (the padding).
             tma_load_2d(sa, &tmA, &full[s], cb * kBK, tap * p.N + tm * kBM);
-            tma_load_4d(sb, &tmB, &full[s], cb * kBK, sx - 1, h0 + r - 1, img);
+            tma_load_4d(sb, &tmB, &full[s], cb * kBK, x0 + sx - 1, h0 + r - 1, img);
           } else {
             tma_load_2d(sa, &tmA, &full[s], kb * kBK, tm * kBM);
             tma_load_2d(sb, &tmB, &full[s], kb * kBK, tn * BN);

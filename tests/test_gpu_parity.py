@@ -403,6 +403,7 @@ def test_bf16_conv_tensor_core_path(kf, cfg):
     dict(Nb=1, Cin=64, H=5, W=96, Cout=40, groups=5),        # 2 rows per tile, ragged last tile
     dict(Nb=1, Cin=20, H=9, W=24, Cout=24, groups=3),        # padded channels, ragged rows
     dict(Nb=1, Cin=8, H=3, W=224, Cout=8, groups=0),         # one row per tile
+    dict(Nb=1, Cin=8, H=4, W=320, Cout=16, groups=2),        # rows cut into two 160-pixel segments
 ])
 def test_bf16_conv_tensor_core_general_shapes(kf, cfg):
     d = ki.conv_inputs(seed=6, **cfg)

@@ -79,7 +79,11 @@ typedef enum { KF_RED_SOFTMAX = 0, KF_RED_SUM = 1 } kf_rowred;
  * sum every 512 elements of K; absolute error about 1e-5 on outputs of magnitude 1, like an
  * fp32 FMA loop, for any K.  That path needs the workspace kf_gemm_epilogue_workspace_bytes()
  * returns (the split operands: 8*(M+N)*ceil4(K) bytes) and fails with KF_ERR_WORKSPACE
- * without it; every other path needs none.  Everything else takes a scalar kernel. */
+ * without it.  bf16 operands that TMA cannot load as they are (K, ldx or ldw not a multiple of
+ * 8, X or W off 16 bytes) are copied into zero-padded dense rows and take the tensor cores too
+ * when M*N*K >= 2^24 and the workspace holds the copies (2*(M+N)*ceil8(K) bytes, rounded up
+ * to 256 per operand; the query returns that size when K % 8 != 0); otherwise they, and
+ * everything else, take a scalar kernel. */
 kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
                            const void* X, int64_t ldx, const void* W, int64_t ldw,
                            const void* bias, kf_act act, float scale,

@@ -222,6 +222,28 @@ int pick_tile_n(int64_t M, int64_t N, int sm_count) {
   return cover;
 }
 
+// bf16 operands the TMA loads cannot take (K not a multiple of 8, a row pitch that is not, a base
+// off 16 bytes) are repacked into the workspace when the problem is large enough for that to
+// pay: dense rows padded with zeros to kp = ceil8(K), then the tensor-core path on the copies.
+int64_t bf16_kp(int64_t K) { return (K + 7) / 8 * 8; }
+size_t bf16_pad_ws(int64_t M, int64_t N, int64_t K) {
+  return round256(static_cast<size_t>(M) * bf16_kp(K) * 2) + round256(static_cast<size_t>(N) * bf16_kp(K) * 2);
+}
+bool bf16_repack_pays(int64_t M, int64_t N, int64_t K) { return M * N * K >= (int64_t{1} << 24); }
+// Repack X and W into `ws`; returns false on a launch error.
+bool repack_bf16(int64_t M, int64_t N, int64_t K, const void* X, int64_t ldx, const void* W, int64_t ldw,
+                 void* ws, const void** Xp, const void** Wp, cudaStream_t st) {
+  const int64_t kp = bf16_kp(K);
+  void* xp = ws;
+  void* wp = static_cast<uint8_t*>(ws) + round256(static_cast<size_t>(M) * kp * 2);
+  if (launch_pad_rows_bf16(M, static_cast<int>(K), static_cast<int>(kp), X, ldx, xp, st) != cudaSuccess ||
+      launch_pad_rows_bf16(N, static_cast<int>(K), static_cast<int>(kp), W, ldw, wp, st) != cudaSuccess)
+    return false;
+  g_launches += 2;
+  *Xp = xp; *Wp = wp;
+  return true;
+}
+
 // fp32 chains large enough for the tensor cores take the 3xTF32 kernel (operands split into
 // TF32 hi + lo parts in the workspace); smaller ones stay on the fp32 FMA kernel (measured:
 // 512^3 18.6 us FMA / 35 us tensor, 1024^3 112 / 54 us, 4096^3 6569 / 667 us).
@@ -333,6 +355,7 @@ kf_status kf_device_status(void) {
 
 size_t kf_gemm_epilogue_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype) {
   if (M < 1 || N < 1 || K < 1) return 0;
+  if (io_dtype == KF_BF16 && K % 8 != 0 && bf16_repack_pays(M, N, K)) return bf16_pad_ws(M, N, K);
   return use_tf32x3(io_dtype, M, N, K) ? tf32_ws(M, N, K) : 0;
 }
 
@@ -340,6 +363,8 @@ size_t kf_gemm_rowreduce_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dty
                                          kf_rowred red) {
   if (M < 1 || N < 1 || K < 1) return 0;
   if (in_dtype == KF_BF16 && K % 8 == 0) return rowreduce_umma_ws(M, N, red);
+  if (in_dtype == KF_BF16 && bf16_repack_pays(M, N, K))
+    return bf16_pad_ws(M, N, K) + rowreduce_umma_ws(M, N, red);
   return rowreduce_simt_ws(M, N) + (use_tf32x3(in_dtype, M, N, K) ? tf32_ws(M, N, K) : 0);
 }
 
@@ -368,6 +393,14 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
   if (!device_info(&d)) return KF_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
+  if (io_dtype == KF_BF16 && !umma_gemm_ok(io_dtype, K, X, ldx, W, ldw) && bf16_repack_pays(M, N, K) &&
+      workspace != nullptr && aligned(workspace, 256) && workspace_bytes >= bf16_pad_ws(M, N, K)) {
+    const void *Xp = nullptr, *Wp = nullptr;
+    if (!repack_bf16(M, N, K, X, ldx, W, ldw, workspace, &Xp, &Wp, st)) return KF_ERR_CUDA;
+    const int64_t kp = bf16_kp(K);
+    return kf_gemm_epilogue(M, N, kp, io_dtype, Xp, kp, Wp, kp, bias, act, scale, residual, ldr, Y, ldy,
+                            nullptr, 0, cuda_stream);
+  }
   if (use_tf32x3(io_dtype, M, N, K)) {
     vs = check_workspace(workspace, workspace_bytes, tf32_ws(M, N, K));
     if (vs != KF_OK) return vs;
@@ -464,6 +497,16 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int Mi = static_cast<int>(M), Ni = static_cast<int>(N), Ki = static_cast<int>(K);
 
+  if (in_dtype == KF_BF16 && !umma_gemm_ok(in_dtype, K, X, ldx, W, ldw) && bf16_repack_pays(M, N, K) &&
+      (N + kRowReduceBN - 1) / kRowReduceBN <= 4096 && workspace != nullptr && aligned(workspace, 256) &&
+      workspace_bytes >= bf16_pad_ws(M, N, K) + rowreduce_umma_ws(M, N, red)) {
+    const void *Xp = nullptr, *Wp = nullptr;
+    if (!repack_bf16(M, N, K, X, ldx, W, ldw, workspace, &Xp, &Wp, st)) return KF_ERR_CUDA;
+    const int64_t kp = bf16_kp(K);
+    const size_t used = bf16_pad_ws(M, N, K);
+    return kf_gemm_rowreduce(M, N, kp, in_dtype, Xp, kp, Wp, kp, bias, pre_act, red, out, ldo, out_dtype,
+                             static_cast<uint8_t*>(workspace) + used, workspace_bytes - used, cuda_stream);
+  }
   if (umma_gemm_ok(in_dtype, K, X, ldx, W, ldw) && (N + kRowReduceBN - 1) / kRowReduceBN <= 4096) {
     vs = check_workspace(workspace, workspace_bytes, rowreduce_umma_ws(M, N, red));
     if (vs != KF_OK) return vs;

@@ -61,6 +61,10 @@ cudaError_t launch_groupnorm_apply(int Nb, int Cout, int groups, long long hw, i
                                    float eps, const float* stats, const void* gamma,
                                    const void* beta, void* y, cudaStream_t st);
 
+// bf16 operand repack (any pitch / alignment -> dense rows padded to 8 columns)
+cudaError_t launch_pad_rows_bf16(long long rows, int K, int kp, const void* in, long long ld, void* out,
+                                 cudaStream_t st);
+
 // fp32 chain on the tensor cores (3xTF32): split prepass and GEMM kernel
 struct Tf32Params {
   int M, N, K;

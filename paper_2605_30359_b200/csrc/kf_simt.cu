@@ -85,6 +85,16 @@ cudaError_t launch_rowsum_finalize(int M, int tiles_n, const float* partial, flo
   return cudaGetLastError();
 }
 
+cudaError_t launch_pad_rows_bf16(long long rows, int K, int kp, const void* in, long long ld, void* out,
+                                 cudaStream_t st) {
+  const long long total = rows * (kp / 8);
+  long long blocks = (total + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  pad_rows_bf16_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(
+      rows, K, kp, static_cast<const __nv_bfloat16*>(in), ld, static_cast<__nv_bfloat16*>(out));
+  return cudaGetLastError();
+}
+
 cudaError_t launch_conv_prep(int Nb, int Cin, int Cp, int H, int Wd, int Cout, const void* x,
                              const void* w, void* xt, void* wr, cudaStream_t st) {
   const __nv_bfloat16* xs = static_cast<const __nv_bfloat16*>(x);

@@ -273,6 +273,32 @@ rowsum_finalize_kernel(int M, int tiles_n, const float* __restrict__ partial, fl
   out[m] = s;
 }
 
+// ---------------------------------------------------------------- operand repack for TMA
+// in [rows, ld] bf16 with any pitch and alignment -> out dense [rows, kp] (kp = K rounded up to
+// 8, padding columns zero): what the tensor-core kernels' TMA loads need.  One thread per group
+// of eight columns.
+__global__ void __launch_bounds__(256)
+pad_rows_bf16_kernel(long long rows, int K, int kp, const __nv_bfloat16* __restrict__ in, long long ld,
+                     __nv_bfloat16* __restrict__ out) {
+  const int gpr = kp / 8;
+  const long long total = rows * gpr;
+  for (long long g = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; g < total;
+       g += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const long long r = g / gpr;
+    const int k = static_cast<int>(g - r * gpr) * 8;
+    const __nv_bfloat16* src = in + r * ld + k;
+    unsigned short e[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) e[j] = (k + j < K) ? __bfloat16_as_ushort(src[j]) : static_cast<unsigned short>(0);
+    uint4 o;
+    o.x = e[0] | (static_cast<uint32_t>(e[1]) << 16);
+    o.y = e[2] | (static_cast<uint32_t>(e[3]) << 16);
+    o.z = e[4] | (static_cast<uint32_t>(e[5]) << 16);
+    o.w = e[6] | (static_cast<uint32_t>(e[7]) << 16);
+    reinterpret_cast<uint4*>(out)[g] = o;
+  }
+}
+
 // ---------------------------------------------------------------- conv: layout prepass
 // x NCHW bf16 -> xt NHWC bf16 (so a pixel's channels are one contiguous, K-major row for the
 // implicit GEMM), and w OIHW -> wr[tap][o][c].  Each thread moves an 8-channel x 8-pixel block:

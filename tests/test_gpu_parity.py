@@ -194,6 +194,23 @@ def test_bf16_split_k_layout_pins(kf):
     assert (to_f64(Y) == K / 64).all()
 
 
+# bf16 operands whose K is not a multiple of 8 cannot be loaded by TMA as they are; problems large
+# enough are repacked (zero-padded rows) into the workspace and take the tensor cores anyway.
+@pytest.mark.parametrize("shape", [(512, 520, 1001), (300, 257, 4099)])
+def test_bf16_gemm_repacked_operands(kf, shape):
+    M, N, K = shape
+    assert kf.kf_gemm_epilogue_workspace_bytes(M, N, K, kf.KF_BF16) > 0
+    d = ki.gemm_inputs("c2", seed=51, M=M, N=N, K=K)
+    got, ref = run_gemm(kf, d, "gelu_tanh", 0.5)
+    assert_close(got, ref, 2e-2, 2e-2, "bf16 repacked %s" % (shape,))
+    d3 = ki.gemm_inputs("c3", seed=52, M=M, N=N, K=K)
+    P = kf.gemm_rowreduce(to_dev(d3["X"]), to_dev(d3["W"]), to_dev(d3["b"]), "none", "softmax")
+    check_status()
+    ref = oracle.gemm_rowreduce(d3["X"], d3["W"], d3["b"], "none", "softmax")
+    assert_close(to_f64(P), ref, 2e-2, 2e-2, "bf16 repacked softmax %s" % (shape,))
+    assert_close(to_f64(P), ref, 1e-7, 2e-2, "bf16 repacked softmax, relative %s" % (shape,))
+
+
 # K >= 2048 with more than 256 rows takes the CTA-pair kernel (256-row tiles over two SMs)
 @pytest.mark.parametrize("shape", [(384, 520, 2048), (257, 256, 2112), (1000, 264, 2048)])
 def test_bf16_gemm_cta_pair_kernel(kf, shape):

@@ -625,14 +625,28 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               tma_store_3d(&tmY, yb, px0 + c * 32, tm * kBM, img);
               bulk_commit_group();
             }
-          } else if (ch_ok) {
-            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) +
-                                 (static_cast<long long>(img) * p.N + ch) * hw + px0 + c * 32;
+          } else {
+            // Image planes that do not start on 16 bytes: no TMA store.  The piece still goes
+            // through shared memory so that the global writes run along pixels: a warp moves
+            // 32 channel rows, its lanes one pixel each (64 contiguous bytes per instruction).
+            uint8_t* yb = ybuf;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {       // the output may be only 2-byte aligned here
-              if (2 * j < left) dst[2 * j] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j] & 0xFFFFu));
-              if (2 * j + 1 < left) dst[2 * j + 1] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j] >> 16));
+            for (int q = 0; q < 4; ++q)
+              *reinterpret_cast<uint4*>(yb + piece_off(row, q)) =
+                  make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+            named_barrier_sync(bar_b, kEpiThreads);
+            const int er = et >> 5;
+            __nv_bfloat16* plane = reinterpret_cast<__nv_bfloat16*>(p.out) +
+                                   static_cast<long long>(img) * p.N * hw + px0 + c * 32 + lane;
+#pragma unroll 4
+            for (int i = 0; i < 32; ++i) {
+              const int r = i * 4 + er;
+              const int cho = tm * kBM + r;
+              if (lane < left && cho < p.N)
+                plane[static_cast<long long>(cho) * hw] =
+                    *reinterpret_cast<const __nv_bfloat16*>(yb + piece_off(r, lane >> 3) + (lane & 7) * 2);
             }
+            named_barrier_sync(bar_b, kEpiThreads);    // the buffer is free for the next piece
           }
         }
         if (p.partial != nullptr && ch_ok) {      // one entry per pixel tile and channel

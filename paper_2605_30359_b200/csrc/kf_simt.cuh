@@ -204,7 +204,33 @@ softmax_finalize_kernel(int N, int bn_shift, int tiles_n, const float2* __restri
       ov[i] = w;
     }
   } else {
-    for (int n = threadIdx.x; n < N; n += blockDim.x)
+    // Rows that do not start on 16 bytes: scalar head up to the first aligned element, 16-byte
+    // vectors for the body (a vector may straddle two slices, so each element looks its factor
+    // up), scalar tail.
+    constexpr int V = 16 / sizeof(OutT);
+    const int mis = static_cast<int>((reinterpret_cast<uintptr_t>(o) & 15u) / sizeof(OutT));
+    const int head = min(N, (V - mis) % V);
+    const int nvec = (N - head) / V;
+    for (int n = threadIdx.x; n < head; n += blockDim.x)
+      o[n] = from_f32<OutT>(to_f32(o[n]) * fac[n >> bn_shift] * inv);
+    uint4* ov = reinterpret_cast<uint4*>(o + head);
+    for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
+      const int n0 = head + i * V;
+      uint4 w = ov[i];
+      if constexpr (sizeof(OutT) == 2) {
+        uint32_t* u = reinterpret_cast<uint32_t*>(&w);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          u[j] = pack_bf16x2(bf16_lo(u[j]) * (fac[(n0 + 2 * j) >> bn_shift] * inv),
+                             bf16_hi(u[j]) * (fac[(n0 + 2 * j + 1) >> bn_shift] * inv));
+      } else {
+        float* u = reinterpret_cast<float*>(&w);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) u[j] *= fac[(n0 + j) >> bn_shift] * inv;
+      }
+      ov[i] = w;
+    }
+    for (int n = head + nvec * V + threadIdx.x; n < N; n += blockDim.x)
       o[n] = from_f32<OutT>(to_f32(o[n]) * fac[n >> bn_shift] * inv);
   }
 }

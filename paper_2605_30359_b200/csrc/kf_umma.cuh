@@ -519,6 +519,32 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               continue;
             }
           }
+          if constexpr (sizeof(OutT) == 2) {
+            // bf16 rows that do not start on 16 bytes: through shared memory, then along rows
+            // (a warp moves 32 rows, its lanes one column each)
+            uint8_t* yb = ybuf;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              *reinterpret_cast<uint4*>(yb + piece_off(row, q)) =
+                  make_uint4(pack_bf16x2(f[8 * q + 0], f[8 * q + 1]),
+                             pack_bf16x2(f[8 * q + 2], f[8 * q + 3]),
+                             pack_bf16x2(f[8 * q + 4], f[8 * q + 5]),
+                             pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
+            named_barrier_sync(bar_b, kEpiThreads);
+            const int er = et >> 5;
+            if (c * 32 + lane < n_valid) {
+#pragma unroll 4
+              for (int i = 0; i < 32; ++i) {
+                const int r = i * 4 + er;
+                const long long mr = static_cast<long long>(m_cta) + r;
+                if (mr < p.M)
+                  P[mr * p.ldo + n_tile + c * 32 + lane] =
+                      *reinterpret_cast<const OutT*>(yb + piece_off(r, lane >> 3) + (lane & 7) * 2);
+              }
+            }
+            named_barrier_sync(bar_b, kEpiThreads);    // the buffer is free for the next piece
+            continue;
+          }
           if (row_ok) {
             const int n0 = n_tile + c * 32;
             if (p.vec_ok && c * 32 + 32 <= n_valid) {

@@ -211,6 +211,23 @@ def test_bf16_gemm_repacked_operands(kf, shape):
     assert_close(to_f64(P), ref, 1e-7, 2e-2, "bf16 repacked softmax, relative %s" % (shape,))
 
 
+# Softmax output rows that do not start on 16 bytes (odd N): numerators leave through shared
+# memory along rows, the second pass works in aligned vectors between a scalar head and tail.
+@pytest.mark.parametrize("shape", [(300, 4101, 136),      # 34 slices: block-per-row second pass
+                                   (260, 1001, 72),       # 64-column tiles, warp-per-row second pass
+                                   (129, 50257, 64)])     # vocabulary-sized odd N
+def test_bf16_softmax_unaligned_rows(kf, shape):
+    M, N, K = shape
+    d = ki.gemm_inputs("c3", seed=61, M=M, N=N, K=K)
+    P = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "none", "softmax")
+    check_status()
+    ref = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "none", "softmax")
+    got = to_f64(P)
+    assert_close(got, ref, 2e-2, 2e-2, "softmax odd N %s" % (shape,))
+    assert_close(got, ref, 1e-7, 2e-2, "softmax odd N, relative %s" % (shape,))
+    assert np.abs(got.sum(axis=1) - 1).max() < 4e-3
+
+
 # K >= 2048 with more than 256 rows takes the CTA-pair kernel (256-row tiles over two SMs)
 @pytest.mark.parametrize("shape", [(384, 520, 2048), (257, 256, 2112), (1000, 264, 2048)])
 def test_bf16_gemm_cta_pair_kernel(kf, shape):

@@ -188,6 +188,15 @@ size_t kf_conv3x3_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd
  * KF_ERR_CUDA.  It is not needed for correct runs; tests call it after each launch. */
 kf_status kf_device_status(void);
 
+/* Self-test of that mechanism (no counterpart in the paper): launches one warp that waits, with
+ * the same bounded wait the kernels use, on an mbarrier nothing will ever complete, with a limit
+ * of limit_ns (1e3 .. 1e9) instead of the kernels' 4 s.  Synchronises the stream.  Returns KF_OK
+ * when the wait gave up after at least limit_ns (*waited_ns, a host pointer or NULL, receives
+ * the time it waited), KF_ERR_UNSUPPORTED when it did not behave so.  As after a real timeout,
+ * the device status word is left set: the next kf_device_status() returns KF_ERR_TIMEOUT and
+ * clears it.  Nothing traps, faults or loops without bound. */
+kf_status kf_selftest_bounded_wait(uint64_t limit_ns, uint64_t* waited_ns, void* cuda_stream);
+
 /* Number of kernels the library has launched from this process since load (all streams). */
 int64_t kf_launch_count(void);
 

@@ -28,7 +28,7 @@ RED = {"softmax": 0, "sum": 1}
 
 EXPORTS = ["kf_gemm_epilogue", "kf_gemm_rowreduce", "kf_gemm_rowreduce_static",
            "kf_conv3x3_epilogue", "kf_conv3x3_softmax_pool",
-           "kf_conv3x3_softmax_pool_workspace_bytes",
+           "kf_conv3x3_softmax_pool_workspace_bytes", "kf_selftest_bounded_wait",
            "kf_gemm_epilogue_workspace_bytes", "kf_gemm_rowreduce_workspace_bytes",
            "kf_conv3x3_workspace_bytes", "kf_device_status", "kf_launch_count",
            "kf_status_string", "kf_version"]
@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
     L.kf_conv3x3_softmax_pool.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp, sz, vp]
     L.kf_conv3x3_softmax_pool_workspace_bytes.restype = sz
     L.kf_conv3x3_softmax_pool_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, ci]
+    L.kf_selftest_bounded_wait.restype = ci
+    L.kf_selftest_bounded_wait.argtypes = [ctypes.c_uint64, ctypes.POINTER(ctypes.c_uint64), vp]
     L.kf_gemm_epilogue_workspace_bytes.restype = sz
     L.kf_gemm_epilogue_workspace_bytes.argtypes = [i64, i64, i64, ci]
     L.kf_gemm_rowreduce_workspace_bytes.restype = sz
@@ -125,6 +127,13 @@ def kf_conv3x3_softmax_pool(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, pool, y,
 
 def kf_conv3x3_softmax_pool_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype) -> int:
     return lib().kf_conv3x3_softmax_pool_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype)
+
+
+def kf_selftest_bounded_wait(limit_ns, stream=None):
+    """Returns (status, nanoseconds waited)."""
+    waited = ctypes.c_uint64(0)
+    st = lib().kf_selftest_bounded_wait(int(limit_ns), ctypes.byref(waited), stream)
+    return st, int(waited.value)
 
 
 def kf_gemm_epilogue_workspace_bytes(M, N, K, io_dtype) -> int:

@@ -320,6 +320,24 @@ kf_status run_tf32_chain(int64_t M, int64_t N, int64_t K, const void* X, int64_t
   return KF_OK;
 }
 
+// Self-test of the bounded wait: one warp arms an mbarrier that nothing will ever complete and
+// waits on it with the given limit.  out[0] = 1 if the wait gave up (the designed outcome),
+// out[1] = nanoseconds it waited.
+__device__ unsigned long long g_selftest_out[2];
+__global__ void bounded_wait_selftest_kernel(uint32_t* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ uint32_t abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    mbar_init_fence();
+    const unsigned long long t0 = globaltimer_ns();
+    const bool completed = mbar_wait(&bar, 0, &abort_flag, status, KF_DEV_TIMEOUT_SELFTEST, limit_ns);
+    g_selftest_out[0] = completed ? 0ull : 1ull;
+    g_selftest_out[1] = globaltimer_ns() - t0;
+  }
+}
+
 }  // namespace
 
 extern "C" {
@@ -351,6 +369,22 @@ kf_status kf_device_status(void) {
     return KF_ERR_TIMEOUT;
   }
   return KF_OK;
+}
+
+kf_status kf_selftest_bounded_wait(uint64_t limit_ns, uint64_t* waited_ns, void* cuda_stream) {
+  if (limit_ns < 1000 || limit_ns > 1000000000ull) return KF_ERR_INVALID_ARG;   // 1 us .. 1 s
+  DeviceInfo* d = nullptr;
+  if (!device_info(&d)) return KF_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(d->status, limit_ns);
+  if (cudaGetLastError() != cudaSuccess) return KF_ERR_CUDA;
+  g_launches += 1;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return KF_ERR_CUDA;
+  unsigned long long out[2] = {0, 0};
+  if (cudaMemcpyFromSymbol(out, g_selftest_out, sizeof(out)) != cudaSuccess) return KF_ERR_CUDA;
+  if (waited_ns != nullptr) *waited_ns = out[1];
+  // the wait must have given up, and not before its limit
+  return (out[0] == 1ull && out[1] >= limit_ns) ? KF_OK : KF_ERR_UNSUPPORTED;
 }
 
 size_t kf_gemm_epilogue_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype) {

@@ -14,6 +14,7 @@ enum : uint32_t {
   KF_DEV_TIMEOUT_PRODUCER = 1u << 0,
   KF_DEV_TIMEOUT_MMA = 1u << 1,
   KF_DEV_TIMEOUT_EPILOGUE = 1u << 2,
+  KF_DEV_TIMEOUT_SELFTEST = 1u << 3,
 };
 
 // A single wait may last this long before the kernel gives up (nanoseconds of %globaltimer).
@@ -75,14 +76,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // ran out of time, in which case it raises the CTA's abort flag and the device status word.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
                                           volatile uint32_t* abort_flag, uint32_t* status,
-                                          uint32_t code) {
+                                          uint32_t code, uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   uint32_t it = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++it & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      if (globaltimer_ns() - t0 > limit_ns) {
         *abort_flag = 1u;
         atomicOr(status, code);
         return false;

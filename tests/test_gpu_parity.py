@@ -568,6 +568,24 @@ def test_conv_softmax_pool_errors(kf):
     assert e.value.status == kf.KF_ERR_INVALID_ARG
 
 
+# ------------------------------------------------------------------ bounded waits
+def test_bounded_wait_gives_up_and_is_reported(kf):
+    """A wait nothing satisfies returns after its limit, raises the device status word, and the
+    context stays usable (no trap, no fault, no unbounded loop)."""
+    assert kf.kf_device_status() == kf.KF_OK
+    st, waited = kf.kf_selftest_bounded_wait(2_000_000)          # 2 ms
+    assert st == kf.KF_OK
+    assert 2_000_000 <= waited < 200_000_000
+    assert kf.kf_device_status() == kf.KF_ERR_TIMEOUT            # reported once ...
+    assert kf.kf_device_status() == kf.KF_OK                     # ... and cleared
+    assert kf.kf_selftest_bounded_wait(10)[0] == kf.KF_ERR_INVALID_ARG
+    assert kf.kf_selftest_bounded_wait(2_000_000_000)[0] == kf.KF_ERR_INVALID_ARG
+    # the library still computes afterwards
+    d = ki.gemm_inputs("c2", seed=71, M=128, N=64, K=64)
+    got, ref = run_gemm(kf, d, "relu")
+    assert_close(got, ref, 2e-2, 2e-2, "after the self-test")
+
+
 # ------------------------------------------------------------------ error handling on the device box
 def test_workspace_errors(kf):
     import torch

@@ -547,7 +547,6 @@ __global__ void __launch_bounds__(512)
 groupnorm_apply_kernel(int Cout, int groups, long long hw, int tiles_per_image, float eps,
                        const float2* __restrict__ stats, const __nv_bfloat16* __restrict__ gamma,
                        const __nv_bfloat16* __restrict__ beta, __nv_bfloat16* y) {
-  __shared__ float scratch[32];
   const int cpg = Cout / groups;
   const long long cnt = static_cast<long long>(cpg) * hw;
   const int g = blockIdx.x % groups;
@@ -567,15 +566,21 @@ groupnorm_apply_kernel(int Cout, int groups, long long hw, int tiles_per_image, 
       if (i < nvec) pre[k] = bv[i];
     }
   }
+  // Every warp adds the group's entries itself (lane-strided, then a shuffle tree): the same
+  // order in every warp, so all warps hold bit-identical statistics, and no block-wide barrier
+  // sits between the prefetch and the stores.
   float s1 = 0.0f, s2 = 0.0f;
-  for (int i = threadIdx.x; i < tiles_per_image * cpg; i += blockDim.x) {
+  for (int i = threadIdx.x & 31; i < tiles_per_image * cpg; i += 32) {
     const int t = i / cpg, c = g * cpg + i % cpg;
     const float2 v = stats[(n * tiles_per_image + t) * Cout + c];
     s1 += v.x;
     s2 += v.y;
   }
-  s1 = block_reduce<false>(s1, scratch);
-  s2 = block_reduce<false>(s2, scratch);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+    s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+  }
   const float mu = s1 / static_cast<float>(cnt);
   const float var = fmaxf(s2 / static_cast<float>(cnt) - mu * mu, 0.0f);
   const float rstd = rsqrtf(var + eps);

@@ -161,10 +161,6 @@ bool conv_umma_shape_ok(int dt, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout
   return dt == DT_BF16 && conv_rows_per_tile(H, Wd) > 0;
 }
 int64_t conv_cpad(int64_t Cin) { return (Cin + 63) / 64 * 64; }   // channels of the NHWC copy
-// pixels per tile (the UMMA N)
-int conv_tile_pixels(int64_t H, int64_t Wd) {
-  return static_cast<int>(conv_rows_per_tile(H, Wd) * Wd / conv_w_segs(Wd));
-}
 // statistics entries per image: one per pixel tile
 int64_t conv_stat_parts(int64_t H, int64_t Wd) {
   const int r = conv_rows_per_tile(H, Wd);

@@ -316,6 +316,7 @@ def _stage(name, host, device):
 
 
 _side_streams = {}
+_last_compute = {}     # device index -> event after the last kernel that read the staging buffers
 
 
 def _side(device):
@@ -334,8 +335,10 @@ def gemm_epilogue_host(X, W, bias=None, act="none", scale=1.0, residual=None, ou
     Copies the inputs to the device, runs the fused kernel and copies Y back into out_host.
     Rows are independent, so the batch is cut into `chunks` row blocks: block i is computed
     while block i+1 is still arriving and block i-1 is already leaving (the copy engines of the
-    two directions run concurrently).  All work is ordered after, and joined back into, `stream`
-    (default: the current stream); synchronise it before reading out_host."""
+    two directions run concurrently).  The kernels run on `stream` (default: the current stream)
+    and the downloads are joined back into it: synchronise it before reading out_host.  Uploads
+    of a call start as soon as the previous call's kernels are done, so back-to-back calls keep
+    both PCIe directions busy."""
     torch = _torch()
     device = device or torch.device("cuda", torch.cuda.current_device())
     s = stream if stream is not None else torch.cuda.current_stream(device)
@@ -348,7 +351,12 @@ def gemm_epilogue_host(X, W, bias=None, act="none", scale=1.0, residual=None, ou
     dR = _stage("R", residual, device) if residual is not None else None
     chunks = max(1, min(int(chunks), M // 256)) if M >= 512 else 1
     bounds = [M * i // chunks for i in range(chunks + 1)]
-    s_in.wait_stream(s)
+    # The inputs are host memory: the uploads need not wait for earlier work on `s`, only for the
+    # kernels of the previous call that still read the (cached) staging buffers.  So the next
+    # call's uploads overlap the previous call's downloads (PCIe runs both directions at once).
+    last = _last_compute.get(device.index)
+    if last is not None:
+        s_in.wait_event(last)
     s_out.wait_stream(s)
     with torch.cuda.stream(s_in):
         dW.copy_(W, non_blocking=True)
@@ -370,5 +378,6 @@ def gemm_epilogue_host(X, W, bias=None, act="none", scale=1.0, residual=None, ou
         s_out.wait_event(computed)
         with torch.cuda.stream(s_out):
             out_host[r0:r1].copy_(dY[r0:r1], non_blocking=True)
+        _last_compute[device.index] = computed
     s.wait_stream(s_out)
     return out_host

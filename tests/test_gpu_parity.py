@@ -630,3 +630,23 @@ def test_host_front_end_matches_device_call(kf):
     ref = kf.gemm_epilogue(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "gelu_tanh", 0.5, to_dev(d["R"]))
     assert torch.equal(out, ref.cpu())
     check_status()
+
+
+def test_host_front_end_back_to_back_calls(kf):
+    """Consecutive host calls share staging buffers and overlap (the next call's uploads run
+    while the previous call's downloads finish): every call must still see its own inputs."""
+    import torch
+    M, N, K = 2048, 512, 256
+    pin = lambda a: torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    sets, outs = [], []
+    for seed in (20, 21, 22, 23):
+        d = ki.gemm_inputs("c2", seed=seed, M=M, N=N, K=K)
+        sets.append((d, pin(d["X"]), pin(d["W"]), pin(d["b"]), pin(d["R"])))
+        outs.append(torch.zeros(M, N, dtype=torch.bfloat16).pin_memory())
+    for (d, hX, hW, hb, hR), out in zip(sets, outs):            # no synchronisation in between
+        kf.gemm_epilogue_host(hX, hW, hb, "gelu_tanh", 0.5, hR, out_host=out)
+    torch.cuda.synchronize()
+    for (d, hX, hW, hb, hR), out in zip(sets, outs):
+        ref = kf.gemm_epilogue(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "gelu_tanh", 0.5, to_dev(d["R"]))
+        assert torch.equal(out, ref.cpu())
+    check_status()

@@ -76,6 +76,16 @@ def test_fp32_tensor_core_chain(kf, shape):
     assert np.abs(got - ref).max() < 3e-5       # an order of magnitude better than one-pass TF32
 
 
+def test_fp32_tensor_core_chain_narrow_n(kf):
+    """N <= 128 takes the 128-column instance of the fp32 tensor-core kernel."""
+    d = ki.gemm_inputs("c2", seed=42, M=4096, N=128, K=1024, dtype="f32")
+    got, ref = run_gemm(kf, d, "sigmoid", 1.0)
+    assert_close(got, ref, 1e-4, 1e-4, "fp32 3xTF32 N=128")
+    d = ki.gemm_inputs("c2", seed=43, M=8192, N=100, K=700, dtype="f32")      # ragged everywhere
+    got, ref = run_gemm(kf, d, "tanh", 2.0)
+    assert_close(got, ref, 1e-4, 1e-4, "fp32 3xTF32 N=100")
+
+
 def test_fp32_tensor_core_layout_and_split_pins(kf):
     """One-hot X rows return W's entries: exact whenever an entry fits hi + lo (22 significant
     bits), so a wrong K block, swizzle or operand (hi/lo mixed up) shows as a mismatch."""

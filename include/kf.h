@@ -146,8 +146,10 @@ kf_status kf_gemm_rowreduce_static(int64_t M, int64_t N, int64_t K, kf_dtype in_
  * r makes r*Wd a multiple of 32 that is at most 256 (every Wd <= 256 that is a multiple of 8,
  * also Wd = 7, 14, 28, 56; Wd = 30 is not); Cin is padded to a multiple of 64 in the
  * workspace copy, H may leave a partial last tile, and rows wider than 256 pixels are cut into
- * equal segments that are multiples of 32 (Wd = 320, 384, 512, ...).  Everything else takes a
- * scalar kernel.
+ * equal segments that are multiples of 32 (Wd = 320, 384, 512, ...).  fp32 problems with the
+ * same tiling and Nb*H*Wd*Cout*Cin >= 2^24 take the tensor cores as well (operands split into
+ * two TF32 numbers each, as in kf_gemm_epilogue; GroupNorm by a two-pass kernel afterwards).
+ * Everything else takes a scalar kernel.
  * groups must divide Cout. */
 kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
                               kf_dtype io_dtype, const void* x, const void* w, const void* bias,

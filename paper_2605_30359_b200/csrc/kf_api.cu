@@ -91,6 +91,21 @@ bool encode_2d_f32(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
          CUDA_SUCCESS;
 }
+// NHWC fp32 activations [Nb,H,W,C] (C a multiple of 16) -> boxes of 16 channels x box_w pixels x
+// rows image rows, 64-byte swizzle, zero fill outside the image.
+bool encode_nhwc_f32(CUtensorMap* tm, const void* base, int64_t Nb, int64_t H, int64_t Wd, int64_t C,
+                     int rows, int box_w) {
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(Wd),
+                              static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(Nb)};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(C) * 4, static_cast<cuuint64_t>(Wd) * C * 4,
+                                 static_cast<cuuint64_t>(H) * Wd * C * 4};
+  const cuuint32_t box[4] = {16u, static_cast<cuuint32_t>(box_w), static_cast<cuuint32_t>(rows), 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(base), dims, strides,
+                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+         CUDA_SUCCESS;
+}
 bool encode_piece(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld) {
   return encode_2d(tm, base, rows, cols, ld, kBM, kPieceCols, CU_TENSOR_MAP_SWIZZLE_64B);
 }
@@ -161,6 +176,16 @@ bool conv_umma_shape_ok(int dt, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout
   return dt == DT_BF16 && conv_rows_per_tile(H, Wd) > 0;
 }
 int64_t conv_cpad(int64_t Cin) { return (Cin + 63) / 64 * 64; }   // channels of the NHWC copy
+// fp32 convolutions large enough for the tensor cores take the 3xTF32 implicit GEMM
+int64_t conv32_cpad(int64_t Cin) { return (Cin + 15) / 16 * 16; }
+bool conv_tf32_ok(int dt, int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout) {
+  if (dt != DT_F32 || getenv("KF_NO_TF32X3") != nullptr) return false;
+  return conv_rows_per_tile(H, Wd) > 0 && Nb * H * Wd * Cout * Cin >= (int64_t{1} << 24);
+}
+size_t conv_tf32_ws(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout) {
+  const int64_t Cp = conv32_cpad(Cin);
+  return 2 * round256(static_cast<size_t>(Nb) * H * Wd * Cp * 4) + 2 * round256(static_cast<size_t>(9) * Cout * Cp * 4);
+}
 // statistics entries per image: one per pixel tile
 int64_t conv_stat_parts(int64_t H, int64_t Wd) {
   const int r = conv_rows_per_tile(H, Wd);
@@ -402,6 +427,7 @@ size_t kf_conv3x3_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd
                                   kf_dtype io_dtype, int groups) {
   (void)groups;
   if (Nb < 1 || Cin < 1 || H < 1 || Wd < 1 || Cout < 1) return 0;
+  if (conv_tf32_ok(io_dtype, Nb, Cin, H, Wd, Cout)) return conv_tf32_ws(Nb, Cin, H, Wd, Cout);
   if (!conv_umma_shape_ok(io_dtype, Cin, H, Wd, Cout)) return 0;
   return round256(static_cast<size_t>(Nb) * H * Wd * conv_cpad(Cin) * 2) +
          round256(static_cast<size_t>(9) * Cout * conv_cpad(Cin) * 2) + conv_stats_bytes(Nb, H, Wd, Cout);
@@ -639,7 +665,56 @@ kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   int launches = 0;
 
-  if (conv_umma_shape_ok(io_dtype, Cin, H, Wd, Cout)) {
+  if (conv_tf32_ok(io_dtype, Nb, Cin, H, Wd, Cout)) {
+    const int64_t Cp = conv32_cpad(Cin);
+    kf_status vs = check_workspace(workspace, workspace_bytes, conv_tf32_ws(Nb, Cin, H, Wd, Cout));
+    if (vs != KF_OK) return vs;
+    const size_t xb = round256(static_cast<size_t>(Nb) * hw * Cp * 4);
+    const size_t wb = round256(static_cast<size_t>(9) * Cout * Cp * 4);
+    float* xh = static_cast<float*>(workspace);
+    float* xl = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + xb);
+    float* wh = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 2 * xb);
+    float* wl = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 2 * xb + wb);
+    if (launch_conv_prep_tf32(static_cast<int>(Nb), static_cast<int>(Cin), static_cast<int>(Cp), hw,
+                              static_cast<int>(Cout), static_cast<const float*>(x),
+                              static_cast<const float*>(w), xh, xl, wh, wl, st) != cudaSuccess)
+      return KF_ERR_CUDA;
+    ++launches;
+    const int rows = conv_rows_per_tile(H, Wd);
+    const int segs = conv_w_segs(Wd);
+    const int tile_px = static_cast<int>(rows * Wd / segs);
+    const int bn = tile_px > 128 ? 256 : 128;
+    CUtensorMap ah, al, bh, bl;
+    if (!encode_2d_f32(&ah, wh, 9 * Cout, Cp, Cp, kBM) || !encode_2d_f32(&al, wl, 9 * Cout, Cp, Cp, kBM) ||
+        !encode_nhwc_f32(&bh, xh, Nb, H, Wd, Cp, rows, static_cast<int>(Wd / segs)) ||
+        !encode_nhwc_f32(&bl, xl, Nb, H, Wd, Cp, rows, static_cast<int>(Wd / segs)))
+      return KF_ERR_CUDA;
+    Tf32ConvParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.Cout = static_cast<int>(Cout); p.H = static_cast<int>(H); p.Wd = static_cast<int>(Wd);
+    p.tiles_per_image = static_cast<int>(conv_stat_parts(H, Wd));
+    p.rows_per_tile = rows; p.w_segs = segs; p.tile_px = tile_px;
+    p.tiles_m = static_cast<int>((Cout + kBM - 1) / kBM);
+    p.tiles_n = static_cast<int>(Nb) * p.tiles_per_image;
+    if (static_cast<int64_t>(p.tiles_m) * p.tiles_n > kMaxDim) return KF_ERR_UNSUPPORTED;
+    p.num_tiles = p.tiles_m * p.tiles_n;
+    p.kb_per_tap = static_cast<int>(Cp / 16);
+    p.k_blocks = 9 * p.kb_per_tap;
+    p.bias = static_cast<const float*>(bias);
+    p.out = static_cast<float*>(y);
+    p.act = act;
+    p.vec_ok = (aligned(y, 16) && hw % 4 == 0) ? 1 : 0;
+    p.status = d->status;
+    const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
+    if (launch_tf32_conv(bn, ah, al, bh, bl, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
+    ++launches;
+    if (groups > 0) {
+      if (launch_groupnorm(io_dtype, static_cast<int>(Nb), static_cast<int>(Cout), groups, hw, eps,
+                           gamma, beta, y, st) != cudaSuccess)
+        return KF_ERR_CUDA;
+      ++launches;
+    }
+  } else if (conv_umma_shape_ok(io_dtype, Cin, H, Wd, Cout)) {
     const int64_t Cp = conv_cpad(Cin);
     const size_t xt_bytes = round256(static_cast<size_t>(Nb) * hw * Cp * 2);
     const size_t wr_bytes = round256(static_cast<size_t>(9) * Cout * Cp * 2);

@@ -79,6 +79,22 @@ struct Tf32Params {
   int vec_ok;                    // rows of out (and R) start on 16 bytes
   uint32_t* status;
 };
+struct Tf32ConvParams {
+  int Cout, H, Wd;
+  int tiles_m, tiles_n, num_tiles;     // output-channel tiles, pixel tiles, both
+  int tiles_per_image, rows_per_tile, w_segs, tile_px;
+  int kb_per_tap, k_blocks;            // K blocks of 16 channels per tap; 9 * kb_per_tap
+  const float* bias;                   // [Cout] or null
+  float* out;                          // NCHW
+  int act;
+  int vec_ok;                          // out is 16-byte aligned and H*W is a multiple of 4
+  uint32_t* status;
+};
+cudaError_t launch_conv_prep_tf32(int Nb, int Cin, int Cp, long long hw, int Cout, const float* x,
+                                  const float* w, float* xh, float* xl, float* wh, float* wl,
+                                  cudaStream_t st);
+cudaError_t launch_tf32_conv(int bn, const CUtensorMap& ah, const CUtensorMap& al, const CUtensorMap& bh,
+                             const CUtensorMap& bl, const Tf32ConvParams& p, int grid, cudaStream_t st);
 cudaError_t launch_tf32_split(long long rows, int K, int kp, const float* in, long long ld, float* hi,
                               float* lo, cudaStream_t st);
 cudaError_t launch_tf32_chain(int bn, const CUtensorMap& ah, const CUtensorMap& al,

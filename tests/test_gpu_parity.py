@@ -498,6 +498,27 @@ def test_conv_scalar_path(kf, dtype, cfg):
     assert_close(got, ref, atol, rtol, "conv scalar %s %s" % (dtype, cfg))
 
 
+# fp32 convolutions of at least 2^24 multiply-adds per tap take the tensor cores (3xTF32 implicit
+# GEMM, chunked accumulation), GroupNorm by the two-pass kernel afterwards.
+@pytest.mark.parametrize("cfg", [
+    dict(Nb=8, Cin=32, H=32, W=32, Cout=64, groups=8),        # 8 rows x 32 pixels per tile
+    dict(Nb=16, Cin=20, H=28, W=28, Cout=72, groups=4),       # channels padded to 32, ragged last tile
+    dict(Nb=32, Cin=64, H=14, W=14, Cout=48, groups=0),       # 16-row box on a 14-row image
+    dict(Nb=8, Cin=256, H=7, W=7, Cout=256, groups=8),        # planes of 49 pixels: scalar stores, 2 chunks... of K
+    dict(Nb=2, Cin=64, H=64, W=64, Cout=130, groups=0),       # two channel tiles, the second nearly empty
+])
+def test_fp32_conv_tensor_core_path(kf, cfg):
+    d = ki.conv_inputs(seed=8, dtype="f32", **cfg)
+    assert kf.kf_conv3x3_workspace_bytes(cfg["Nb"], cfg["Cin"], cfg["H"], cfg["W"], cfg["Cout"], kf.KF_F32,
+                                         cfg["groups"]) > 0
+    got, ref = run_conv(kf, d)
+    tol = 5e-4 if cfg["groups"] > 0 else 1e-4     # rsqrt of the group variance amplifies fp32 rounding
+    assert_close(got, ref, tol, tol, "fp32 conv %s" % cfg)
+    got, ref = run_conv(kf, d, act="none", groups=0, use_bias=False)
+    assert_close(got, ref, 1e-4, 1e-4, "fp32 conv bare %s" % cfg)
+    assert np.abs(got - ref).max() < 3e-5
+
+
 def test_groupnorm_biased_variance_on_gpu(kf):
     # 1x1 image, four channels per group, x = 0 so the activations are the biases {1,2,3,4}/4
     bias = np.array([0.25, 0.5, 0.75, 1.0, 2.0, 2.0, 2.0, 2.0], np.float32)

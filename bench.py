@@ -433,6 +433,8 @@ SWEEP_CONV = [  # (Nb, Cin, H, W, Cout, groups [GroupNorm] or -pool [softmax + m
     (128, 64, 64, 64, 128, -4), (16, 64, 32, 32, 16, -2),
     (32, 64, 56, 56, 64, 8), (32, 128, 28, 28, 128, 8), (32, 256, 14, 14, 256, 8), (16, 3, 224, 224, 64, 8),
 ]
+SWEEP_CONV_F32 = [(32, 64, 56, 56, 64, 8), (16, 64, 32, 32, 64, 8)]   # fp32, ReLU + GroupNorm
+SWEEP_ROWRED_F32 = [(2048, 4096, 1024, "none", "softmax"), (4096, 1024, 1024, "sigmoid", "sum")]
 
 
 def _torch_act(name):
@@ -481,8 +483,8 @@ def run_sweep(kf, device):
                lambda X=X, W=W, b=b, R=R, out=out, act=act, scale=scale:
                kf.gemm_epilogue(X, W, b, act, scale, R, out=out), ref, 2.0 * M * N * K)
         del X, W, b, R, out
-    for M, N, K, pre, red in SWEEP_ROWRED:
-        dt = torch.bfloat16
+    for M, N, K, pre, red, dt in ([r + (torch.bfloat16,) for r in SWEEP_ROWRED] +
+                                  [r + (torch.float32,) for r in SWEEP_ROWRED_F32]):
         X, W, b = rnd((M, K), dt), rnd((N, K), dt, K ** -0.5), rnd((N,), dt, K ** -0.5)
         ta = _torch_act(pre)
         if red == "softmax":
@@ -493,17 +495,18 @@ def run_sweep(kf, device):
             out = torch.empty((M,), dtype=torch.float32, device=device)
             ref = lambda X=X, W=W, b=b, ta=ta: ta(F.linear(X, W, b)).sum(dim=1, dtype=torch.float32)
             cat = "reduction-dominated"
-        record(cat, "bf16 %dx%dx%d %s->%s" % (M, N, K, pre, red),
+        record(cat, "%s %dx%dx%d %s->%s" % ("bf16" if dt == torch.bfloat16 else "f32", M, N, K, pre, red),
                lambda X=X, W=W, b=b, out=out, pre=pre, red=red: kf.gemm_rowreduce(X, W, b, pre, red, out=out),
                ref, 2.0 * M * N * K)
         del X, W, b, out
-    for Nb, Cin, H, Wd, Cout, gp in SWEEP_CONV:
-        dt = torch.bfloat16
+    for Nb, Cin, H, Wd, Cout, gp, dt in ([c + (torch.bfloat16,) for c in SWEEP_CONV] +
+                                         [c + (torch.float32,) for c in SWEEP_CONV_F32]):
+        dn = "bf16" if dt == torch.bfloat16 else "f32"
         x, w, b = rnd((Nb, Cin, H, Wd), dt), rnd((Cout, Cin, 3, 3), dt, (9 * Cin) ** -0.5), rnd((Cout,), dt, 0.1)
         flops = 2.0 * Nb * H * Wd * Cout * Cin * 9
         if gp > 0:
             out = torch.empty((Nb, Cout, H, Wd), dtype=dt, device=device)
-            record("conv-centered", "bf16 conv %dx%dx%dx%d->%d relu GN%d" % (Nb, Cin, H, Wd, Cout, gp),
+            record("conv-centered", "%s conv %dx%dx%dx%d->%d relu GN%d" % (dn, Nb, Cin, H, Wd, Cout, gp),
                    lambda x=x, w=w, b=b, out=out, gp=gp: kf.conv3x3_epilogue(x, w, b, "relu", gp, 1e-5, out=out),
                    lambda x=x, w=w, b=b, gp=gp: F.group_norm(torch.relu(F.conv2d(x, w, b, padding=1)), gp, eps=1e-5),
                    flops)

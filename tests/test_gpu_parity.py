@@ -504,7 +504,7 @@ def test_conv_scalar_path(kf, dtype, cfg):
     dict(Nb=8, Cin=32, H=32, W=32, Cout=64, groups=8),        # 8 rows x 32 pixels per tile
     dict(Nb=16, Cin=20, H=28, W=28, Cout=72, groups=4),       # channels padded to 32, ragged last tile
     dict(Nb=32, Cin=64, H=14, W=14, Cout=48, groups=0),       # 16-row box on a 14-row image
-    dict(Nb=8, Cin=256, H=7, W=7, Cout=256, groups=8),        # planes of 49 pixels: scalar stores, 2 chunks... of K
+    dict(Nb=8, Cin=256, H=7, W=7, Cout=256, groups=8),        # planes of 49 pixels: scalar stores; K = 2304, five chunks
     dict(Nb=2, Cin=64, H=64, W=64, Cout=130, groups=0),       # two channel tiles, the second nearly empty
 ])
 def test_fp32_conv_tensor_core_path(kf, cfg):

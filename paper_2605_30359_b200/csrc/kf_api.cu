@@ -270,7 +270,11 @@ bool repack_bf16(int64_t M, int64_t N, int64_t K, const void* X, int64_t ldx, co
 // 512^3 18.6 us FMA / 35 us tensor, 1024^3 112 / 54 us, 4096^3 6569 / 667 us).
 bool use_tf32x3(int dt, int64_t M, int64_t N, int64_t K) {
   if (dt != DT_F32 || getenv("KF_NO_TF32X3") != nullptr) return false;
-  return M >= 64 && N >= 64 && K >= 64 && M * N * K >= (int64_t{1} << 29);
+  if (M < 64 || N < 64 || K < 64) return false;
+  if (M * N * K >= (int64_t{1} << 29)) return true;
+  // from 2^28 when there are enough tiles to spread over the SMs (768^3: 49.8 us FMA, 28 us here)
+  const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + 255) / 256);
+  return M * N * K >= (int64_t{1} << 28) && tiles >= 12;
 }
 int64_t tf32_kp(int64_t K) { return (K + 3) / 4 * 4; }
 size_t tf32_ws(int64_t M, int64_t N, int64_t K) {

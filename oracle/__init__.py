@@ -20,7 +20,8 @@ _LIB = os.path.join(_HERE, "libkf_oracle.so")
 
 F32, BF16 = 0, 1
 ACT = {"none": 0, "relu": 1, "gelu_tanh": 2, "sigmoid": 3, "gelu_erf": 4, "swish": 5,
-       "tanh": 6, "hardtanh": 7, "chain95": 8}
+       "tanh": 6, "hardtanh": 7, "chain95": 8, "leaky_relu": 9, "elu": 10, "mish": 11,
+       "hardswish": 12, "softplus": 13, "relu6": 14, "hardsigmoid": 15}
 RED = {"softmax": 0, "sum": 1}
 
 

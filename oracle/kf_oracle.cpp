@@ -45,7 +45,11 @@ namespace {
 
 enum { DT_F32 = 0, DT_BF16 = 1 };
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SIGMOID = 3, ACT_GELU_ERF = 4,
-       ACT_SWISH = 5, ACT_TANH = 6, ACT_HARDTANH = 7, ACT_CHAIN95 = 8 };
+       ACT_SWISH = 5, ACT_TANH = 6, ACT_HARDTANH = 7, ACT_CHAIN95 = 8,
+       // further elementwise operators of the paper's benchmark chains (Table 2 lists activation
+       // chains by name only; definitions and default parameters are PyTorch's)
+       ACT_LEAKY_RELU = 9, ACT_ELU = 10, ACT_MISH = 11, ACT_HARDSWISH = 12, ACT_SOFTPLUS = 13,
+       ACT_RELU6 = 14, ACT_HARDSIGMOID = 15 };
 enum { RED_SOFTMAX = 0, RED_SUM = 1 };
 
 int g_threads = 0;  // 0 = OpenMP default
@@ -59,6 +63,8 @@ inline double widen(const void* p, int dt, int64_t i) {
 }
 
 inline double sigmoid(double z) { return 1.0 / (1.0 + std::exp(-z)); }
+// log(1 + e^z) without overflow
+inline double softplus(double z) { return std::fmax(z, 0.0) + std::log1p(std::exp(-std::fabs(z))); }
 
 double act_apply(int act, double z) {
   switch (act) {
@@ -81,6 +87,13 @@ double act_apply(int act, double z) {
       double g = t * 0.5 * (1.0 + std::erf(t * 0.7071067811865475));
       return std::fmin(std::fmax(g, -1.0), 1.0);
     }
+    case ACT_LEAKY_RELU: return z > 0.0 ? z : 0.01 * z;                    // negative slope 0.01
+    case ACT_ELU: return z > 0.0 ? z : std::expm1(z);                      // alpha = 1
+    case ACT_MISH: return z * std::tanh(softplus(z));
+    case ACT_HARDSWISH: return z * std::fmin(std::fmax(z + 3.0, 0.0), 6.0) / 6.0;
+    case ACT_SOFTPLUS: return softplus(z);                                 // beta = 1
+    case ACT_RELU6: return std::fmin(std::fmax(z, 0.0), 6.0);
+    case ACT_HARDSIGMOID: return std::fmin(std::fmax(z / 6.0 + 0.5, 0.0), 1.0);
   }
   return NAN;
 }

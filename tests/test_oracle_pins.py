@@ -81,6 +81,30 @@ def test_gelu_variants_are_distinguishable():
     assert 3.5e-4 < d < 4.7e-4
 
 
+def test_further_activations_against_closed_forms_and_torch():
+    """The seven further activations: closed-form values, then torch's own fp64 routines on a
+    grid (an independent implementation of the same definitions)."""
+    import torch
+    import torch.nn.functional as F
+    e = math.e
+    closed = [("leaky_relu", -2.0, -0.02), ("leaky_relu", 3.0, 3.0), ("elu", -1.0, 1.0 / e - 1.0), ("elu", 2.0, 2.0),
+              ("mish", 0.0, 0.0), ("mish", 1.0, 0.86509838826731), ("mish", -1.0, -0.30340146137411),
+              ("hardswish", 1.0, 2.0 / 3.0), ("hardswish", -3.0, 0.0), ("hardswish", 3.0, 3.0), ("hardswish", -4.0, 0.0),
+              ("softplus", 0.0, math.log(2.0)), ("softplus", 800.0, 800.0), ("softplus", -800.0, 0.0),
+              ("relu6", 7.0, 6.0), ("relu6", -1.0, 0.0), ("relu6", 2.5, 2.5),
+              ("hardsigmoid", 0.0, 0.5), ("hardsigmoid", 3.0, 1.0), ("hardsigmoid", -3.0, 0.0), ("hardsigmoid", 1.5, 0.75)]
+    for name, z, want in closed:
+        assert abs(oracle.act(name, z) - want) < (1e-13 if name == "mish" else 1e-14), (name, z)   # mish: 14 printed digits
+    lib = {"leaky_relu": F.leaky_relu, "elu": F.elu, "mish": F.mish, "hardswish": F.hardswish,
+           "softplus": lambda t: F.softplus(t, threshold=1e9), "relu6": F.relu6, "hardsigmoid": F.hardsigmoid}
+    zs = np.linspace(-12.0, 12.0, 481)
+    t = torch.from_numpy(zs)
+    for name, fn in lib.items():
+        want = fn(t).numpy()
+        got = np.array([oracle.act(name, float(z)) for z in zs])
+        assert np.abs(got - want).max() < 1e-13, name
+
+
 def test_paper_constants_and_chain95():
     g = golden()
     assert abs(g["erf_gelu_inner_scale"] - 1.0 / math.sqrt(2.0)) < 1e-15

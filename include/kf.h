@@ -50,7 +50,12 @@ typedef enum { KF_F32 = 0, KF_BF16 = 1 } kf_dtype;
 /* Activations.  0..3 are the benchmark chains' (the paper's "matmul + relu" class,
  * Appendix A strategy 2); 4..8 are the operators of the paper's worked chain (Appendix C.2):
  * erf-form GELU t*0.5*(1+erf(t/sqrt 2)), swish sigmoid(x)*x, tanh, hardtanh clamp[-1,1], and
- * KF_ACT_CHAIN95 = hardtanh(gelu_erf(tanh(swish(z)))) applied to z = XW^T + bias. */
+ * KF_ACT_CHAIN95 = hardtanh(gelu_erf(tanh(swish(z)))) applied to z = XW^T + bias.  9..15 are
+ * further elementwise operators of operator chains like the paper's (its Table 2 names chain
+ * categories, not formulas): PyTorch's definitions with default parameters - leaky ReLU (slope
+ * 0.01), ELU (alpha 1), Mish z*tanh(softplus z), hardswish z*relu6(z+3)/6, softplus log(1+e^z),
+ * ReLU6, hardsigmoid relu6(z+3)/6.  They share one kernel instantiation and are selected by a
+ * switch inside the epilogue. */
 typedef enum {
   KF_ACT_NONE = 0,
   KF_ACT_RELU = 1,
@@ -60,7 +65,14 @@ typedef enum {
   KF_ACT_SWISH = 5,
   KF_ACT_TANH = 6,
   KF_ACT_HARDTANH = 7,
-  KF_ACT_CHAIN95 = 8
+  KF_ACT_CHAIN95 = 8,
+  KF_ACT_LEAKY_RELU = 9,
+  KF_ACT_ELU = 10,
+  KF_ACT_MISH = 11,
+  KF_ACT_HARDSWISH = 12,
+  KF_ACT_SOFTPLUS = 13,
+  KF_ACT_RELU6 = 14,
+  KF_ACT_HARDSIGMOID = 15
 } kf_act;
 
 typedef enum { KF_RED_SOFTMAX = 0, KF_RED_SUM = 1 } kf_rowred;

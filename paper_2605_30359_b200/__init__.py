@@ -23,7 +23,8 @@ LIB_PATH = os.path.join(_PKG, "libkf.so")
 KF_OK, KF_ERR_INVALID_ARG, KF_ERR_UNSUPPORTED, KF_ERR_WORKSPACE, KF_ERR_CUDA, KF_ERR_TIMEOUT = range(6)
 KF_F32, KF_BF16 = 0, 1
 ACT = {"none": 0, "relu": 1, "gelu_tanh": 2, "sigmoid": 3, "gelu_erf": 4, "swish": 5, "tanh": 6,
-       "hardtanh": 7, "chain95": 8}
+       "hardtanh": 7, "chain95": 8, "leaky_relu": 9, "elu": 10, "mish": 11, "hardswish": 12,
+       "softplus": 13, "relu6": 14, "hardsigmoid": 15}
 RED = {"softmax": 0, "sum": 1}
 
 EXPORTS = ["kf_gemm_epilogue", "kf_gemm_rowreduce", "kf_gemm_rowreduce_static",

@@ -9,7 +9,11 @@
 namespace kf {
 
 enum : int { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SIGMOID = 3, ACT_GELU_ERF = 4,
-             ACT_SWISH = 5, ACT_TANH = 6, ACT_HARDTANH = 7, ACT_CHAIN95 = 8, ACT_COUNT = 9 };
+             ACT_SWISH = 5, ACT_TANH = 6, ACT_HARDTANH = 7, ACT_CHAIN95 = 8,
+             // the codes below share ONE kernel instantiation (ACT_RUNTIME) and are told apart by
+             // a switch on the run-time code inside the epilogue
+             ACT_LEAKY_RELU = 9, ACT_ELU = 10, ACT_MISH = 11, ACT_HARDSWISH = 12, ACT_SOFTPLUS = 13,
+             ACT_RELU6 = 14, ACT_HARDSIGMOID = 15, ACT_COUNT = 16, ACT_RUNTIME = 100 };
 enum : int { RED_SOFTMAX = 0, RED_SUM = 1 };
 enum : int { DT_F32 = 0, DT_BF16 = 1 };
 
@@ -42,9 +46,32 @@ __device__ __forceinline__ float gelu_erf_f(float z) {
   return z * 0.5f * (1.0f + erff(z * 0.7071067811865475f));
 }
 
+// log(1 + e^z) without overflow
+template <bool FAST>
+__device__ __forceinline__ float softplus_f(float z) {
+  if constexpr (FAST) return fmaxf(z, 0.0f) + __logf(1.0f + __expf(-fabsf(z)));
+  else return fmaxf(z, 0.0f) + log1pf(expf(-fabsf(z)));
+}
+// The activations selected at run time (PyTorch's definitions and default parameters).
+template <bool FAST>
+__device__ __forceinline__ float act_rt(int code, float z) {
+  switch (code) {
+    case ACT_LEAKY_RELU: return z > 0.0f ? z : 0.01f * z;
+    case ACT_ELU: return z > 0.0f ? z : (FAST ? __expf(z) - 1.0f : expm1f(z));
+    case ACT_MISH: return z * tanh_f<FAST>(softplus_f<FAST>(z));
+    case ACT_HARDSWISH: return z * fminf(fmaxf(z + 3.0f, 0.0f), 6.0f) * (1.0f / 6.0f);
+    case ACT_SOFTPLUS: return softplus_f<FAST>(z);
+    case ACT_RELU6: return fminf(fmaxf(z, 0.0f), 6.0f);
+    case ACT_HARDSIGMOID: return fminf(fmaxf(fmaf(z, 1.0f / 6.0f, 0.5f), 0.0f), 1.0f);
+    default: return z;
+  }
+}
+
+// `code` is read only by the ACT_RUNTIME instantiation.
 template <int ACT, bool FAST>
-__device__ __forceinline__ float act_f(float z) {
-  if constexpr (ACT == ACT_NONE) return z;
+__device__ __forceinline__ float act_f(float z, int code = 0) {
+  if constexpr (ACT == ACT_RUNTIME) return act_rt<FAST>(code, z);
+  else if constexpr (ACT == ACT_NONE) return z;
   else if constexpr (ACT == ACT_RELU) return fmaxf(z, 0.0f);
   else if constexpr (ACT == ACT_GELU_TANH) return gelu_tanh_f<FAST>(z);
   else if constexpr (ACT == ACT_SIGMOID) return sigmoid_f<FAST>(z);
@@ -73,6 +100,9 @@ __host__ inline bool dispatch_act(int act, F&& f) {
     case ACT_TANH: f(std::integral_constant<int, ACT_TANH>{}); return true;
     case ACT_HARDTANH: f(std::integral_constant<int, ACT_HARDTANH>{}); return true;
     case ACT_CHAIN95: f(std::integral_constant<int, ACT_CHAIN95>{}); return true;
+    case ACT_LEAKY_RELU: case ACT_ELU: case ACT_MISH: case ACT_HARDSWISH: case ACT_SOFTPLUS:
+    case ACT_RELU6: case ACT_HARDSIGMOID:
+      f(std::integral_constant<int, ACT_RUNTIME>{}); return true;
   }
   return false;
 }

@@ -477,6 +477,7 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
     tm.r = tm.a; tm.y = tm.a;
     UmmaParams p;
     std::memset(&p, 0, sizeof(p));
+    p.act_rt = act;
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
     p.tiles_m = static_cast<int>((M + kBM - 1) / kBM);
     p.tiles_n = static_cast<int>((N + bn_split - 1) / bn_split);
@@ -502,6 +503,7 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
       return KF_ERR_CUDA;
     UmmaParams p;
     std::memset(&p, 0, sizeof(p));
+    p.act_rt = act;
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
     const int tile_m = pair ? 2 * kBM : kBM;
     p.tiles_m = static_cast<int>((M + tile_m - 1) / tile_m);
@@ -582,6 +584,7 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
     tm.r = tm.a; tm.y = tm.a;
     UmmaParams p;
     std::memset(&p, 0, sizeof(p));
+    p.act_rt = pre_act;
     p.M = Mi; p.N = Ni; p.K = Ki;
     p.tiles_m = static_cast<int>(tiles_m64);
     p.tiles_n = static_cast<int>(tiles_n64);
@@ -744,6 +747,7 @@ kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
     tm.r = tm.a; tm.y = tm.a;
     UmmaParams p;
     std::memset(&p, 0, sizeof(p));
+    p.act_rt = act;
     p.M = static_cast<int>(Nb * hw); p.N = static_cast<int>(Cout); p.K = static_cast<int>(9 * Cp);
     p.tiles_per_image = static_cast<int>(conv_stat_parts(H, Wd));
     p.tile_px = tile_px;

@@ -20,7 +20,7 @@ static cudaError_t simt_gemm_t(int mode, int act, int M, int N, int K, const voi
       if (err != cudaSuccess) return;
       kern<<<grid, block, kSimtSmemBytes, st>>>(
           M, N, K, static_cast<const T*>(X), ldx, static_cast<const T*>(W), ldw,
-          static_cast<const T*>(bias), scale, static_cast<const T*>(R), ldr, out, ldo);
+          static_cast<const T*>(bias), scale, static_cast<const T*>(R), ldr, out, ldo, act);
       err = cudaGetLastError();
     };
     if (mode == 0) go(simt_gemm_kernel<T, 0, ACT>);
@@ -128,7 +128,7 @@ static cudaError_t conv_direct_t(int act, int Nb, int Cin, int H, int Wd, int Co
     conv_direct_kernel<T, ACT><<<grid, 256, 0, st>>>(Nb, Cin, H, Wd, Cout, static_cast<const T*>(x),
                                                      static_cast<const T*>(w),
                                                      static_cast<const T*>(bias),
-                                                     static_cast<T*>(y));
+                                                     static_cast<T*>(y), act);
   });
   return ok ? cudaGetLastError() : cudaErrorInvalidValue;
 }

@@ -48,7 +48,7 @@ template <typename T, int MODE, int ACT>
 __global__ void __launch_bounds__(256)
 simt_gemm_kernel(int M, int N, int K, const T* __restrict__ X, long long ldx,
                  const T* __restrict__ W, long long ldw, const T* __restrict__ bias, float scale,
-                 const T* R, long long ldr, void* out, long long ldo) {
+                 const T* R, long long ldr, void* out, long long ldo, int act_code) {
   extern __shared__ float sm[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * 32, n0 = blockIdx.y * 32;
@@ -119,11 +119,11 @@ simt_gemm_kernel(int M, int N, int K, const T* __restrict__ X, long long ldx,
         float z = zs[j];
         if (bias != nullptr) z += to_f32(bias[n]);
         if constexpr (MODE == 0) {
-          float y = scale * act_f<ACT, false>(z);
+          float y = scale * act_f<ACT, false>(z, act_code);
           if (R != nullptr) y += to_f32(R[m * ldr + n]);
           reinterpret_cast<T*>(out)[m * ldo + n] = from_f32<T>(y);
         } else {
-          reinterpret_cast<float*>(out)[m * ldo + n] = act_f<ACT, false>(z);
+          reinterpret_cast<float*>(out)[m * ldo + n] = act_f<ACT, false>(z, act_code);
         }
       }
     }
@@ -416,7 +416,7 @@ conv_prep_general_kernel(int Nb, int Cin, int Cp, int H, int Wd, int Cout,
 template <typename T, int ACT>
 __global__ void __launch_bounds__(256)
 conv_direct_kernel(int Nb, int Cin, int H, int Wd, int Cout, const T* __restrict__ x,
-                   const T* __restrict__ w, const T* __restrict__ bias, T* __restrict__ y) {
+                   const T* __restrict__ w, const T* __restrict__ bias, T* __restrict__ y, int act_code) {
   const long long total = static_cast<long long>(Nb) * Cout * H * Wd;
   const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (gid >= total) return;
@@ -440,7 +440,7 @@ conv_direct_kernel(int Nb, int Cin, int H, int Wd, int Cout, const T* __restrict
       }
     }
   }
-  y[gid] = from_f32<T>(act_f<ACT, false>(acc));
+  y[gid] = from_f32<T>(act_f<ACT, false>(acc, act_code));
 }
 
 // ---------------------------------------------------------------- GroupNorm, in place

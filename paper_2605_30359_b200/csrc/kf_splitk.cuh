@@ -63,7 +63,11 @@ __device__ __forceinline__ void apply_act32(int act, float scale, float (&f)[32]
     case ACT_TANH: act32<ACT_TANH>(scale, f); break;
     case ACT_HARDTANH: act32<ACT_HARDTANH>(scale, f); break;
     case ACT_CHAIN95: act32<ACT_CHAIN95>(scale, f); break;
-    default: act32<ACT_NONE>(scale, f); break;
+    case ACT_NONE: act32<ACT_NONE>(scale, f); break;
+    default:                                   // the run-time selected activations
+#pragma unroll
+      for (int j = 0; j < 32; ++j) f[j] = scale * act_rt<true>(act, f[j]);
+      break;
   }
 }
 

@@ -144,7 +144,11 @@ __device__ __forceinline__ void apply_act32_precise(int act, float scale, float 
     case ACT_TANH: act32_precise<ACT_TANH>(scale, f); break;
     case ACT_HARDTANH: act32_precise<ACT_HARDTANH>(scale, f); break;
     case ACT_CHAIN95: act32_precise<ACT_CHAIN95>(scale, f); break;
-    default: act32_precise<ACT_NONE>(scale, f); break;
+    case ACT_NONE: act32_precise<ACT_NONE>(scale, f); break;
+    default:                                   // the run-time selected activations
+#pragma unroll
+      for (int j = 0; j < 32; ++j) f[j] = scale * act_rt<false>(act, f[j]);
+      break;
   }
 }
 

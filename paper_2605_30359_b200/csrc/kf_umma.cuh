@@ -53,6 +53,7 @@ struct UmmaParams {
   long long ldo;
   float* partial;              // row-reduce partial statistics
   float scale;
+  int act_rt;                  // activation code, read by the ACT_RUNTIME instantiations
   int vec_ok;                  // rows of out (and R) are 16-byte aligned (direct path vectors)
   int staged;                  // out (and R) go through shared memory and TMA
   int bias_vec;                // bias is 16-byte aligned
@@ -368,7 +369,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             float f[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j)
-              f[j] = p.scale * act_f<ACT, true>(__uint_as_float(v[j]) + bs[j]);
+              f[j] = p.scale * act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
             if (has_r) {
 #pragma unroll
               for (int q = 0; q < 4; ++q) {
@@ -430,7 +431,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             float f[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j)
-              f[j] = p.scale * act_f<ACT, true>(__uint_as_float(v[j]) + bs[j]);
+              f[j] = p.scale * act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
             if (has_r) {
 #pragma unroll
               for (int q = 0; q < 4; ++q) {
@@ -474,7 +475,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           tmem_ld_wait();
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j]);
+            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
             if (c * 32 + j < n_valid) mx = fmaxf(mx, z);
           }
         }
@@ -493,7 +494,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           float f[32];
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j]);
+            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
             f[j] = __expf(z - mx);
             if (c * 32 + j < n_valid) sum += f[j];
           }
@@ -587,7 +588,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           float part = 0.0f;
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j]);
+            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
             if (c * 32 + j < n_valid) part += z;
           }
           sum += part;
@@ -627,8 +628,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           const int left = px_valid - c * 32;               // valid pixels from this piece on
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + bias_v);
-            float y1 = act_f<ACT, true>(__uint_as_float(v[2 * j + 1]) + bias_v);
+            float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + bias_v, p.act_rt);
+            float y1 = act_f<ACT, true>(__uint_as_float(v[2 * j + 1]) + bias_v, p.act_rt);
             w[j] = pack_bf16x2(y0, y1);
             if (2 * j >= left) y0 = 0.0f;
             if (2 * j + 1 >= left) y1 = 0.0f;

@@ -12,7 +12,9 @@ from gpu_util import assert_close, check_status, to_dev, to_f64, tol_for
 
 pytestmark = pytest.mark.gpu
 
-ACTS = ["none", "relu", "gelu_tanh", "sigmoid", "gelu_erf", "swish", "tanh", "hardtanh", "chain95"]
+ACTS = ["none", "relu", "gelu_tanh", "sigmoid", "gelu_erf", "swish", "tanh", "hardtanh", "chain95",
+        "leaky_relu", "elu", "mish", "hardswish", "softplus", "relu6", "hardsigmoid"]
+RUNTIME_ACTS = ACTS[9:]       # selected by a switch inside one kernel instantiation
 
 
 @pytest.fixture(scope="module")
@@ -115,6 +117,47 @@ def test_fp32_tensor_core_workspace_is_checked(kf):
                              Y.data_ptr(), N, ws.data_ptr(), need // 2, None)
     assert st == kf.KF_ERR_WORKSPACE
     assert kf.kf_gemm_epilogue_workspace_bytes(128, 256, 512, kf.KF_F32) == 0
+
+
+# ------------------------------------------------------------------ run-time selected activations
+@pytest.mark.parametrize("act", RUNTIME_ACTS)
+def test_runtime_activations_every_kernel_family(kf, act):
+    """Each further activation through every kernel family: fp32 FMA kernel, split-K cluster
+    kernel, row reductions (softmax pre-activation and row sum), both convolution kernels."""
+    d = ki.gemm_inputs("c2", seed=81, M=70, N=50, K=40, dtype="f32")                 # fp32 FMA
+    got, ref = run_gemm(kf, d, act, 0.5)
+    assert_close(got, ref, 1e-4, 1e-4, "fp32 %s" % act)
+    d = ki.gemm_inputs("c2", seed=82, M=128, N=512, K=2048)                           # split-K cluster
+    got, ref = run_gemm(kf, d, act, 2.0)
+    assert_close(got, ref, 2e-2, 2e-2, "split-K %s" % act)
+    d = ki.gemm_inputs("c3", seed=83, M=150, N=600, K=136)
+    for red in ("softmax", "sum"):
+        out = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), act, red)
+        ref = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], act, red)
+        assert_close(to_f64(out), ref, 2e-2, 2e-2, "%s of %s" % (red, act))
+        if red == "sum":
+            assert_close(to_f64(out), ref, 1e-3, 3e-3, "row sum of %s, relative" % act)
+    # tensor-core conv; no GroupNorm here: after a squashing activation (hardsigmoid's outputs
+    # have a standard deviation of 0.05) the normalisation multiplies the bf16 rounding of the
+    # stored activations by 20, which says nothing about the activation itself
+    dc = ki.conv_inputs(seed=84, Nb=2, Cin=64, H=8, W=64, Cout=96, groups=0)
+    got, ref = run_conv(kf, dc, act=act)
+    assert_close(got, ref, 2e-2, 2e-2, "conv %s" % act)
+    if act == "mish":
+        dc = ki.conv_inputs(seed=84, Nb=2, Cin=64, H=8, W=64, Cout=96, groups=3)
+        got, ref = run_conv(kf, dc, act=act)
+        assert_close(got, ref, 2e-2, 2e-2, "conv %s + GroupNorm" % act)
+    dc = ki.conv_inputs(seed=85, Nb=1, Cin=3, H=5, W=7, Cout=4, groups=0, dtype="f32")  # direct conv
+    got, ref = run_conv(kf, dc, act=act)
+    assert_close(got, ref, 1e-4, 1e-4, "direct conv %s" % act)
+    check_status()
+
+
+@pytest.mark.parametrize("act", ["mish", "elu", "softplus"])
+def test_runtime_activations_fp32_tensor_core(kf, act):
+    d = ki.gemm_inputs("c2", seed=86, M=1024, N=1024, K=512, dtype="f32")
+    got, ref = run_gemm(kf, d, act, 1.0)
+    assert_close(got, ref, 1e-4, 1e-4, "fp32 3xTF32 %s" % act)
 
 
 # ------------------------------------------------------------------ bf16 tensor-core GEMM

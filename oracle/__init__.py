@@ -22,7 +22,7 @@ F32, BF16 = 0, 1
 ACT = {"none": 0, "relu": 1, "gelu_tanh": 2, "sigmoid": 3, "gelu_erf": 4, "swish": 5,
        "tanh": 6, "hardtanh": 7, "chain95": 8, "leaky_relu": 9, "elu": 10, "mish": 11,
        "hardswish": 12, "softplus": 13, "relu6": 14, "hardsigmoid": 15}
-RED = {"softmax": 0, "sum": 1}
+RED = {"softmax": 0, "sum": 1, "max": 2, "mean": 3, "logsumexp": 4}
 
 
 def build(force: bool = False) -> str:
@@ -108,7 +108,7 @@ def gemm_epilogue(X, W, bias=None, act="none", scale=1.0, residual=None) -> np.n
 
 
 def gemm_rowreduce(X, W, bias=None, pre_act="none", red="softmax") -> np.ndarray:
-    """softmax: fp64 [M,N]; sum: fp64 [M]."""
+    """softmax: fp64 [M,N]; sum, max, mean, logsumexp: fp64 [M]."""
     X = _c(X); dt = _dt(X); W = _c(W, dt); bias = _c(bias, dt)
     M, K = X.shape
     N, K2 = W.shape

@@ -50,7 +50,7 @@ enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SIGMOID = 3, ACT_GELU_
        // chains by name only; definitions and default parameters are PyTorch's)
        ACT_LEAKY_RELU = 9, ACT_ELU = 10, ACT_MISH = 11, ACT_HARDSWISH = 12, ACT_SOFTPLUS = 13,
        ACT_RELU6 = 14, ACT_HARDSIGMOID = 15 };
-enum { RED_SOFTMAX = 0, RED_SUM = 1 };
+enum { RED_SOFTMAX = 0, RED_SUM = 1, RED_MAX = 2, RED_MEAN = 3, RED_LOGSUMEXP = 4 };
 
 int g_threads = 0;  // 0 = OpenMP default
 
@@ -138,6 +138,7 @@ int oracle_gemm_epilogue(int64_t M, int64_t N, int64_t K, int dt, const void* X,
 // A[m,n] = pre_act(sum_k X[m,k] W[n,k] + bias[n])
 // red = SOFTMAX: out[m,n] = exp(A[m,n]-max_n A[m,:]) / sum_n exp(A[m,n]-max)   (out is [M,N])
 // red = SUM:     out[m]   = sum_n A[m,n]                                        (out is [M])
+// red = MAX / MEAN / LOGSUMEXP: out[m] = max_n / mean_n / log sum_n exp of A[m,:]   (out is [M])
 int oracle_gemm_rowreduce(int64_t M, int64_t N, int64_t K, int dt, const void* X, int64_t ldx,
                           const void* W, int64_t ldw, const void* bias, int pre_act, int red,
                           double* out) {
@@ -156,10 +157,21 @@ int oracle_gemm_rowreduce(int64_t M, int64_t N, int64_t K, int dt, const void* X
       double s = 0.0;
       for (int64_t n = 0; n < N; ++n) s += std::exp(a[(size_t)n] - mx);
       for (int64_t n = 0; n < N; ++n) out[m * N + n] = std::exp(a[(size_t)n] - mx) / s;
+    } else if (red == RED_MAX) {
+      double mx = -INFINITY;
+      for (int64_t n = 0; n < N; ++n) mx = std::fmax(mx, a[(size_t)n]);
+      out[m] = mx;
+    } else if (red == RED_LOGSUMEXP) {
+      // log sum_n exp(A[m,n]), with the maximum taken out first as in the softmax above
+      double mx = -INFINITY;
+      for (int64_t n = 0; n < N; ++n) mx = std::fmax(mx, a[(size_t)n]);
+      double s = 0.0;
+      for (int64_t n = 0; n < N; ++n) s += std::exp(a[(size_t)n] - mx);
+      out[m] = mx + std::log(s);
     } else {
       double s = 0.0;
       for (int64_t n = 0; n < N; ++n) s += a[(size_t)n];
-      out[m] = s;
+      out[m] = red == RED_MEAN ? s / (double)N : s;
     }
   }
   return 0;

@@ -105,6 +105,27 @@ def test_further_activations_against_closed_forms_and_torch():
         assert np.abs(got - want).max() < 1e-13, name
 
 
+def test_row_max_mean_logsumexp():
+    """The further row reductions against independent routes: the pre-reduction matrix from the
+    separately pinned elementwise oracle, reduced by numpy / scipy; and softmax = exp(A - lse)."""
+    import scipy.special
+    d = ki.gemm_inputs("c3", seed=9, M=7, N=33, K=20, dtype="f32")
+    A = oracle.gemm_epilogue(d["X"], d["W"], d["b"], "gelu_tanh")
+    mx = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "gelu_tanh", "max")
+    mean = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "gelu_tanh", "mean")
+    lse = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "gelu_tanh", "logsumexp")
+    sm = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "gelu_tanh", "softmax")
+    assert mx.shape == mean.shape == lse.shape == (7,)
+    assert np.array_equal(mx, A.max(axis=1))
+    assert np.abs(mean - A.mean(axis=1)).max() < 1e-15
+    assert np.abs(lse - scipy.special.logsumexp(A, axis=1)).max() < 1e-14
+    assert np.abs(sm - np.exp(A - lse[:, None])).max() < 1e-15
+    # one column: max = mean = logsumexp = the value itself; large values do not overflow
+    X = np.zeros((3, 4), np.float32); W = np.zeros((1, 4), np.float32); b = np.array([900.0], np.float32)
+    for red in ("max", "mean", "logsumexp"):
+        assert np.array_equal(oracle.gemm_rowreduce(X, W, b, "none", red), np.full(3, 900.0))
+
+
 def test_paper_constants_and_chain95():
     g = golden()
     assert abs(g["erf_gelu_inner_scale"] - 1.0 / math.sqrt(2.0)) < 1e-15

@@ -75,7 +75,13 @@ typedef enum {
   KF_ACT_HARDSIGMOID = 15
 } kf_act;
 
-typedef enum { KF_RED_SOFTMAX = 0, KF_RED_SUM = 1 } kf_rowred;
+typedef enum {
+  KF_RED_SOFTMAX = 0,
+  KF_RED_SUM = 1,
+  KF_RED_MAX = 2,
+  KF_RED_MEAN = 3,
+  KF_RED_LOGSUMEXP = 4
+} kf_rowred;
 
 /* GEMM + elementwise epilogue (Appendix A, "Operator Fusion": matmul + activation class;
  * Table 2 "Matmul-centered").
@@ -109,6 +115,10 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
  *                   out is [M,N] with leading dimension ldo, dtype out_dtype.
  *   KF_RED_SUM:     out[m] = sum_n A[m,n], out is [M] fp32 (out_dtype must be KF_F32, ldo
  *                   ignored).
+ *   KF_RED_MAX, KF_RED_MEAN, KF_RED_LOGSUMEXP: out[m] = max_n A[m,n], (sum_n A[m,n]) / N,
+ *                   log sum_n exp A[m,n] (computed as max + log sum exp(A - max)); out as for
+ *                   KF_RED_SUM.  Further reductions of chains like the paper's (Table 2,
+ *                   "Mixed reduction" / "Reduction-dominated"); PyTorch's definitions.
  * The reduction is deterministic (no floating-point atomics): repeated calls give identical
  * bits.  The workspace holds per-tile partial statistics. */
 kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype,

@@ -25,7 +25,7 @@ KF_F32, KF_BF16 = 0, 1
 ACT = {"none": 0, "relu": 1, "gelu_tanh": 2, "sigmoid": 3, "gelu_erf": 4, "swish": 5, "tanh": 6,
        "hardtanh": 7, "chain95": 8, "leaky_relu": 9, "elu": 10, "mish": 11, "hardswish": 12,
        "softplus": 13, "relu6": 14, "hardsigmoid": 15}
-RED = {"softmax": 0, "sum": 1}
+RED = {"softmax": 0, "sum": 1, "max": 2, "mean": 3, "logsumexp": 4}
 
 EXPORTS = ["kf_gemm_epilogue", "kf_gemm_rowreduce", "kf_gemm_rowreduce_static",
            "kf_conv3x3_epilogue", "kf_conv3x3_softmax_pool",
@@ -234,13 +234,14 @@ def gemm_epilogue(X, W, bias=None, act="none", scale=1.0, residual=None, out=Non
 
 def gemm_rowreduce(X, W, bias=None, pre_act="none", red="softmax", out_dtype=None, out=None,
                    stream=None):
-    """softmax: out[M,N] = softmax_n(pre_act(X @ W.T + bias)); sum: out[M] fp32 = row sums."""
+    """softmax: out[M,N] = softmax_n(pre_act(X @ W.T + bias)); sum / max / mean / logsumexp:
+    out[M] fp32 = that reduction of every row."""
     torch = _torch()
     _check_cuda(X, W, bias, out)
     M, K = X.shape
     N = W.shape[0]
     dt = _kf_dtype(X)
-    if red == "sum":
+    if red != "softmax":
         if out is None:
             out = torch.empty((M,), dtype=torch.float32, device=X.device)
         odt, ldo = KF_F32, 1

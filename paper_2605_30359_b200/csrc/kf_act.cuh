@@ -14,7 +14,7 @@ enum : int { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SIGMOID = 3, ACT
              // a switch on the run-time code inside the epilogue
              ACT_LEAKY_RELU = 9, ACT_ELU = 10, ACT_MISH = 11, ACT_HARDSWISH = 12, ACT_SOFTPLUS = 13,
              ACT_RELU6 = 14, ACT_HARDSIGMOID = 15, ACT_COUNT = 16, ACT_RUNTIME = 100 };
-enum : int { RED_SOFTMAX = 0, RED_SUM = 1 };
+enum : int { RED_SOFTMAX = 0, RED_SUM = 1, RED_MAX = 2, RED_MEAN = 3, RED_LOGSUMEXP = 4, RED_COUNT = 5 };
 enum : int { DT_F32 = 0, DT_BF16 = 1 };
 
 __device__ __forceinline__ float tanh_approx(float x) {

@@ -217,15 +217,17 @@ kf_status check_workspace(const void* ws, size_t have, size_t need) {
 // takes them instead of 256-column tiles: four times the CTAs and a quarter of the serial epilogue per CTA.
 // The rule uses the B200's SM count as a constant so that the workspace query, which has no
 // device, agrees with the call.
+// reductions that run the softmax first pass (per-slice maximum and sum of exponentials)
+bool softmax_like(int red) { return red == RED_SOFTMAX || red == RED_MAX || red == RED_LOGSUMEXP; }
 int rowreduce_bn(int64_t M, int64_t N, int red) {
   const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + kRowReduceNarrowBN - 1) / kRowReduceNarrowBN);
-  return (red == RED_SOFTMAX && tiles <= 148) ? kRowReduceNarrowBN : kRowReduceBN;
+  return (softmax_like(red) && tiles <= 148) ? kRowReduceNarrowBN : kRowReduceBN;
 }
 size_t rowreduce_umma_ws(int64_t M, int64_t N, int red) {
   const int bn = rowreduce_bn(M, N, red);
   const int64_t tiles_n = (N + bn - 1) / bn;
   // softmax: (max, sum) per row and per half tile (one per epilogue group); row sum: one float
-  return round256(static_cast<size_t>(M) * tiles_n * (red == RED_SOFTMAX ? 16 : 4));
+  return round256(static_cast<size_t>(M) * tiles_n * (softmax_like(red) ? 16 : 4));
 }
 // CTA pairs (256-row tiles, each CTA loading half of the W tile) pay off when the K loop is
 // long: measured +3.6 % at K = 4096, +3.3 % at K = 2048, -4 % at K = 1024 (fewer, larger tiles
@@ -549,8 +551,8 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
   kf_status vs = check_gemm_common(M, N, K, in_dtype, X, ldx, W, ldw, bias);
   if (vs != KF_OK) return vs;
   if (!valid_act(pre_act) || out == nullptr || !valid_dtype(out_dtype)) return KF_ERR_INVALID_ARG;
-  if (red != KF_RED_SOFTMAX && red != KF_RED_SUM) return KF_ERR_INVALID_ARG;
-  if (red == KF_RED_SUM && out_dtype != KF_F32) return KF_ERR_INVALID_ARG;
+  if (red < 0 || red >= RED_COUNT) return KF_ERR_INVALID_ARG;
+  if (red != KF_RED_SOFTMAX && out_dtype != KF_F32) return KF_ERR_INVALID_ARG;
   if (red == KF_RED_SOFTMAX && ldo < N) return KF_ERR_INVALID_ARG;
   if (!aligned(out, esize(out_dtype))) return KF_ERR_INVALID_ARG;
   if (out == X || out == W) return KF_ERR_INVALID_ARG;
@@ -593,13 +595,15 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
     p.k_blocks = static_cast<int>((K + kBK - 1) / kBK);
     p.tiles_per_unit = 1;
     p.bias = static_cast<const __nv_bfloat16*>(bias);
-    p.out = out; p.ldo = ldo; p.scale = 1.0f;
+    p.out = out; p.ldo = ldo;
+    p.scale = red == KF_RED_MEAN ? 1.0f / static_cast<float>(N) : 1.0f;
+    p.stats_only = red == KF_RED_LOGSUMEXP ? 1 : (red == KF_RED_MAX ? 2 : 0);
     p.partial = static_cast<float*>(workspace);
     // Row sum: when giving each CTA whole row blocks costs no extra wave, the epilogue carries
     // the sum across the block's tiles and writes out[m] itself: no partials, no second pass.
     const int64_t waves_rr = (tiles_m64 * tiles_n64 + slots - 1) / slots;
     const int64_t waves_own = ((tiles_m64 + slots - 1) / slots) * tiles_n64;
-    const bool row_owner = red == KF_RED_SUM && waves_own <= waves_rr;
+    const bool row_owner = (red == KF_RED_SUM || red == KF_RED_MEAN) && waves_own <= waves_rr;
     if (row_owner) { p.tiles_per_unit = p.tiles_n; p.partial = nullptr; }
     p.vec_ok = (red == KF_RED_SOFTMAX && (ldo * esize(out_dtype)) % 16 == 0 && aligned(out, 16)) ? 1 : 0;
     p.bias_vec = aligned(bias, 16) ? 1 : 0;
@@ -608,7 +612,15 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
     p.status = d->status;
     const int units = p.num_tiles / p.tiles_per_unit;
     const int grid = units < slots ? units : slots;
-    if (red == KF_RED_SOFTMAX) {
+    if (red == KF_RED_MAX || red == KF_RED_LOGSUMEXP) {
+      // the softmax first pass without numerators (bf16 instance; nothing is stored), then the
+      // per-slice statistics combined per row
+      if (launch_umma_softmax(bn, pre_act, KF_BF16, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
+        return KF_ERR_CUDA;
+      if (launch_rowstat_finalize(red, Mi, 2 * p.tiles_n, p.partial, static_cast<float*>(out), st) !=
+          cudaSuccess)
+        return KF_ERR_CUDA;
+    } else if (red == KF_RED_SOFTMAX) {
       if (launch_umma_softmax(bn, pre_act, out_dtype, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
         return KF_ERR_CUDA;
       if (launch_softmax_finalize(out_dtype, Mi, Ni, bn / 2, 2 * p.tiles_n, p.partial, out, ldo, p.vec_ok, st) !=
@@ -618,7 +630,7 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
       if (launch_umma_rowsum(pre_act, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
         return KF_ERR_CUDA;
       if (!row_owner) {
-        if (launch_rowsum_finalize(Mi, p.tiles_n, p.partial, static_cast<float*>(out), st) !=
+        if (launch_rowsum_finalize(Mi, p.tiles_n, p.partial, static_cast<float*>(out), p.scale, st) !=
             cudaSuccess)
           return KF_ERR_CUDA;
         g_launches += 1;
@@ -644,7 +656,7 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
                               N, st) != cudaSuccess)
     return KF_ERR_CUDA;
   cudaError_t e = red == KF_RED_SOFTMAX ? launch_row_softmax(out_dtype, Mi, Ni, A, N, out, ldo, st)
-                                        : launch_row_sum(Mi, Ni, A, N, static_cast<float*>(out), st);
+                                        : launch_row_reduce(red, Mi, Ni, A, N, static_cast<float*>(out), st);
   if (e != cudaSuccess) return KF_ERR_CUDA;
   g_launches += 2;
   return KF_OK;
@@ -844,7 +856,7 @@ extern "C" kf_status kf_gemm_rowreduce_static(int64_t M, int64_t N, int64_t K, k
                                               kf_rowred red, void* out, int64_t ldo,
                                               kf_dtype out_dtype, void* cuda_stream) {
   // Refuse, before touching the device, any problem whose partial statistics do not fit.
-  if (M >= 1 && N >= 1 && K >= 1 && (red == KF_RED_SOFTMAX || red == KF_RED_SUM) &&
+  if (M >= 1 && N >= 1 && K >= 1 && red >= 0 && red < RED_COUNT &&
       (in_dtype == KF_F32 || in_dtype == KF_BF16) &&
       kf_gemm_rowreduce_workspace_bytes(M, N, K, in_dtype, red) > KF_STATIC_SCRATCH_BYTES)
     return KF_ERR_WORKSPACE;

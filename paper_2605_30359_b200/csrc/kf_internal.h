@@ -35,8 +35,10 @@ constexpr int kRowReduceNarrowBN = 64;   // ... of the softmax first pass of one
 // second passes of the tensor-core row reductions
 cudaError_t launch_softmax_finalize(int out_dt, int M, int N, int bn, int tiles_n, const float* partial,
                                     void* out, long long ldo, int vec_ok, cudaStream_t st);
-cudaError_t launch_rowsum_finalize(int M, int tiles_n, const float* partial, float* out,
+cudaError_t launch_rowsum_finalize(int M, int tiles_n, const float* partial, float* out, float scale,
                                    cudaStream_t st);
+cudaError_t launch_rowstat_finalize(int red, int M, int slices, const float* partial, float* out,
+                                    cudaStream_t st);
 
 // scalar chains (fp32, and bf16 shapes the tensor-core kernels do not take)
 cudaError_t launch_simt_gemm(int dt, int mode, int act, int M, int N, int K, const void* X,
@@ -45,8 +47,8 @@ cudaError_t launch_simt_gemm(int dt, int mode, int act, int M, int N, int K, con
                              cudaStream_t st);
 cudaError_t launch_row_softmax(int out_dt, int M, int N, const float* A, long long lda, void* out,
                                long long ldo, cudaStream_t st);
-cudaError_t launch_row_sum(int M, int N, const float* A, long long lda, float* out,
-                           cudaStream_t st);
+cudaError_t launch_row_reduce(int red, int M, int N, const float* A, long long lda, float* out,
+                              cudaStream_t st);
 
 // convolution helpers
 cudaError_t launch_conv_prep(int Nb, int Cin, int Cp, int H, int Wd, int Cout, const void* x,

@@ -47,9 +47,9 @@ cudaError_t launch_row_softmax(int out_dt, int M, int N, const float* A, long lo
   return cudaGetLastError();
 }
 
-cudaError_t launch_row_sum(int M, int N, const float* A, long long lda, float* out,
-                           cudaStream_t st) {
-  row_sum_kernel<<<M, 256, 0, st>>>(N, A, lda, out);
+cudaError_t launch_row_reduce(int red, int M, int N, const float* A, long long lda, float* out,
+                              cudaStream_t st) {
+  row_reduce_kernel<<<M, 256, 0, st>>>(N, A, lda, out, red);
   return cudaGetLastError();
 }
 
@@ -79,9 +79,16 @@ cudaError_t launch_softmax_finalize(int out_dt, int M, int N, int bn, int tiles_
   return cudaGetLastError();
 }
 
-cudaError_t launch_rowsum_finalize(int M, int tiles_n, const float* partial, float* out,
+cudaError_t launch_rowsum_finalize(int M, int tiles_n, const float* partial, float* out, float scale,
                                    cudaStream_t st) {
-  rowsum_finalize_kernel<<<(M + 255) / 256, 256, 0, st>>>(M, tiles_n, partial, out);
+  rowsum_finalize_kernel<<<(M + 255) / 256, 256, 0, st>>>(M, tiles_n, partial, out, scale);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rowstat_finalize(int red, int M, int slices, const float* partial, float* out,
+                                    cudaStream_t st) {
+  rowstat_finalize_kernel<<<(M + 255) / 256, 256, 0, st>>>(
+      M, slices, reinterpret_cast<const float2*>(partial), out, red);
   return cudaGetLastError();
 }
 

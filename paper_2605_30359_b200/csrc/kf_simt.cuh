@@ -148,14 +148,29 @@ row_softmax_kernel(int N, const float* __restrict__ A, long long lda, OutT* out,
   for (int n = threadIdx.x; n < N; n += blockDim.x) o[n] = from_f32<OutT>(expf(a[n] - mx) / s);
 }
 
+// Scalar-valued row reductions of a materialised fp32 matrix: sum, mean, max, log-sum-exp.
 __global__ void __launch_bounds__(256)
-row_sum_kernel(int N, const float* __restrict__ A, long long lda, float* out) {
+row_reduce_kernel(int N, const float* __restrict__ A, long long lda, float* out, int red) {
   __shared__ float scratch[32];
   const float* a = A + static_cast<long long>(blockIdx.x) * lda;
+  if (red == RED_SUM || red == RED_MEAN) {
+    float s = 0.0f;
+    for (int n = threadIdx.x; n < N; n += blockDim.x) s += a[n];
+    s = block_reduce<false>(s, scratch);
+    if (threadIdx.x == 0) out[blockIdx.x] = red == RED_MEAN ? s / static_cast<float>(N) : s;
+    return;
+  }
+  float mx = -INFINITY;
+  for (int n = threadIdx.x; n < N; n += blockDim.x) mx = fmaxf(mx, a[n]);
+  mx = block_reduce<true>(mx, scratch);
+  if (red == RED_MAX) {
+    if (threadIdx.x == 0) out[blockIdx.x] = mx;
+    return;
+  }
   float s = 0.0f;
-  for (int n = threadIdx.x; n < N; n += blockDim.x) s += a[n];
+  for (int n = threadIdx.x; n < N; n += blockDim.x) s += expf(a[n] - mx);
   s = block_reduce<false>(s, scratch);
-  if (threadIdx.x == 0) out[blockIdx.x] = s;
+  if (threadIdx.x == 0) out[blockIdx.x] = mx + logf(s);
 }
 
 // ---------------------------------------------------------------- second passes, tensor path
@@ -289,14 +304,32 @@ softmax_finalize_warp_kernel(int M, int N, int bn_shift, int tiles_n,
   }
 }
 
-// Row sum: out[m] = sum_t partial[m,t] in increasing t.
+// Row sum: out[m] = scale * sum_t partial[m,t] in increasing t (scale = 1/N for the mean).
 __global__ void __launch_bounds__(256)
-rowsum_finalize_kernel(int M, int tiles_n, const float* __restrict__ partial, float* out) {
+rowsum_finalize_kernel(int M, int tiles_n, const float* __restrict__ partial, float* out, float scale) {
   const long long m = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (m >= M) return;
   float s = 0.0f;
   for (int t = 0; t < tiles_n; ++t) s += partial[m * tiles_n + t];
-  out[m] = s;
+  out[m] = s * scale;
+}
+
+// Row maximum / log-sum-exp from the softmax first pass's per-slice (max, sum of exp) run in
+// statistics-only mode: mx = max_t mx_t; lse = mx + log sum_t sum_t * exp(mx_t - mx).
+__global__ void __launch_bounds__(256)
+rowstat_finalize_kernel(int M, int slices, const float2* __restrict__ partial, float* out, int red) {
+  const long long m = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (m >= M) return;
+  const float2* part = partial + m * slices;
+  float mx = -INFINITY;
+  for (int t = 0; t < slices; ++t) mx = fmaxf(mx, part[t].x);
+  if (red == RED_MAX) { out[m] = mx; return; }
+  float s = 0.0f;
+  for (int t = 0; t < slices; ++t) {
+    const float2 q = part[t];
+    s += q.y * expf(q.x - mx);          // an empty slice holds (-inf, 0) and adds 0
+  }
+  out[m] = mx + logf(s);
 }
 
 // ---------------------------------------------------------------- operand repack for TMA

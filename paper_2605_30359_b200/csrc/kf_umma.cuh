@@ -54,6 +54,8 @@ struct UmmaParams {
   float* partial;              // row-reduce partial statistics
   float scale;
   int act_rt;                  // activation code, read by the ACT_RUNTIME instantiations
+  int stats_only;              // softmax first pass without numerators: 1 = (max, sum of exp)
+                               // for the log-sum-exp, 2 = maximum only
   int vec_ok;                  // rows of out (and R) are 16-byte aligned (direct path vectors)
   int staged;                  // out (and R) go through shared memory and TMA
   int bias_vec;                // bias is 16-byte aligned
@@ -480,10 +482,11 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
         }
         // pass 2: numerators e = exp(a - mx), their fp32 sum, e stored in the output dtype
+        // (statistics-only runs skip the stores; a maximum-only run skips the pass)
         OutT* P = reinterpret_cast<OutT*>(p.out);
         float sum = 0.0f;
 #pragma unroll 1
-        for (int c = 0; c < PIECES; ++c, ++g) {
+        for (int c = 0; c < PIECES && p.stats_only != 2; ++c, ++g) {
           if (!staged && c * 32 >= n_valid) break;
           uint32_t v[32];
           tmem_ld_32x32(t_acc + c * 32, v);
@@ -498,6 +501,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             f[j] = __expf(z - mx);
             if (c * 32 + j < n_valid) sum += f[j];
           }
+          if (p.stats_only != 0) continue;
           if constexpr (sizeof(OutT) == 2) {
             if (staged) {
               const int b = static_cast<int>(g & 1);
@@ -599,7 +603,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         } else {
           // this CTA owns the whole row block: add the tiles in order, write the row sum once
           unit_sum = (tn == 0) ? sum : unit_sum + sum;
-          if (tn == p.tiles_n - 1 && row_ok) reinterpret_cast<float*>(p.out)[m] = unit_sum;
+          if (tn == p.tiles_n - 1 && row_ok) reinterpret_cast<float*>(p.out)[m] = unit_sum * p.scale;
         }
       } else {
         // EPI_CONV: rows = output channels, columns = BN consecutive pixels of one image, so a

@@ -454,6 +454,40 @@ def test_scalar_path_row_reductions(kf, red, act, dtype, shape):
         assert_close(to_f64(out), ref, 1e-7, 2e-4 if dtype == "f32" else 2e-2, "relative")
 
 
+# ------------------------------------------------------------------ row max / mean / log-sum-exp
+@pytest.mark.parametrize("red", ["max", "mean", "logsumexp"])
+@pytest.mark.parametrize("dtype,shape", [("bf16", (300, 1000, 136)),      # 64-column tiles, ragged
+                                         ("bf16", (2500, 2056, 264)),     # 256-column tiles, several waves
+                                         ("bf16", (9, 21, 13)),           # scalar path
+                                         ("f32", (130, 70, 33)),          # fp32 scalar path
+                                         ("f32", (1024, 1000, 600))])     # fp32 GEMM on the tensor cores
+def test_row_max_mean_logsumexp(kf, red, dtype, shape):
+    M, N, K = shape
+    d = ki.gemm_inputs("c3", seed=91, M=M, N=N, K=K, dtype=dtype)
+    out = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "gelu_tanh", red)
+    check_status()
+    assert tuple(out.shape) == (M,)
+    ref = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "gelu_tanh", red)
+    atol, rtol = tol_for(dtype)
+    assert_close(to_f64(out), ref, atol, rtol, "%s %s %s" % (red, dtype, shape))
+    # tighter: a mean averages the rounding of N terms, max and log-sum-exp are dominated by few
+    tight = {"max": 5e-3, "mean": 2e-3, "logsumexp": 5e-3}[red] if dtype == "bf16" else 1e-4
+    assert np.abs(to_f64(out) - ref).max() < tight
+
+
+def test_row_reductions_reject_bad_arguments(kf):
+    import torch
+    X = torch.zeros((8, 8), device="cuda", dtype=torch.bfloat16)
+    out = torch.zeros((8,), device="cuda", dtype=torch.bfloat16)
+    for red in (2, 3, 4):        # a scalar-valued reduction needs an fp32 output
+        st = kf.kf_gemm_rowreduce(8, 8, 8, kf.KF_BF16, X.data_ptr(), 8, X.data_ptr(), 8, None, 0, red,
+                                  out.data_ptr(), 1, kf.KF_BF16, None, 0, None)
+        assert st == kf.KF_ERR_INVALID_ARG
+    st = kf.kf_gemm_rowreduce(8, 8, 8, kf.KF_BF16, X.data_ptr(), 8, X.data_ptr(), 8, None, 0, 5,
+                              out.data_ptr(), 1, kf.KF_F32, None, 0, None)
+    assert st == kf.KF_ERR_INVALID_ARG
+
+
 # ------------------------------------------------------------------ convolution + GroupNorm
 def run_conv(kf, d, act="relu", groups=None, gamma=None, beta=None, use_bias=True):
     groups = d["groups"] if groups is None else groups

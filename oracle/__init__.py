@@ -57,6 +57,8 @@ def _load():
                                           vp, vp, vp]
         lib.oracle_conv3x3_softmax_pool.restype = ci
         lib.oracle_conv3x3_softmax_pool.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, i64, vp]
+        lib.oracle_conv3x3_act_gap.restype = ci
+        lib.oracle_conv3x3_act_gap.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, vp]
         _lib = lib
     return _lib
 
@@ -143,5 +145,17 @@ def conv3x3_softmax_pool(x, w, bias=None, pool=1):
     y = np.empty((Nb, Cout, H // pool, Wd // pool), np.float64)
     rc = _load().oracle_conv3x3_softmax_pool(Nb, Cin, H, Wd, Cout, dt, _ptr(x), _ptr(w), _ptr(bias),
                                              int(pool), _ptr(y))
+    assert rc == 0
+    return y
+
+
+def conv3x3_act_gap(x, w, bias=None, act="none"):
+    """mean over H, W of act(conv3x3_pad1(x, w) + bias), fp64 [Nb, Cout]."""
+    x = _c(x); dt = _dt(x); w = _c(w, dt); bias = _c(bias, dt)
+    Nb, Cin, H, Wd = x.shape
+    Cout = w.shape[0]
+    y = np.empty((Nb, Cout), np.float64)
+    rc = _load().oracle_conv3x3_act_gap(Nb, Cin, H, Wd, Cout, dt, _ptr(x), _ptr(w), _ptr(bias),
+                                        ACT[act], _ptr(y))
     assert rc == 0
     return y

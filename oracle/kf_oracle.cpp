@@ -289,4 +289,31 @@ int oracle_conv3x3_softmax_pool(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, 
   return 0;
 }
 
+// c[n,o,h,w] = bias[o] + sum_{c,r,s} x[n,c,h+r-1,w+s-1] * wt[o,c,r,s]   (as above)
+// y[n,o]     = (1 / (H*Wd)) * sum_{h,w} act(c[n,o,h,w])      -- global average pooling
+// y is fp64 [Nb, Cout].
+int oracle_conv3x3_act_gap(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout, int dt,
+                           const void* x, const void* wt, const void* bias, int act, double* y) {
+#pragma omp parallel for schedule(dynamic) num_threads(nthreads())
+  for (int64_t n = 0; n < Nb; ++n)
+    for (int64_t o = 0; o < Cout; ++o) {
+      double total = 0.0;
+      for (int64_t h = 0; h < H; ++h)
+        for (int64_t w = 0; w < Wd; ++w) {
+          double acc = bias ? widen(bias, dt, o) : 0.0;
+          for (int64_t c = 0; c < Cin; ++c)
+            for (int64_t r = 0; r < 3; ++r)
+              for (int64_t q = 0; q < 3; ++q) {
+                const int64_t hh = h + r - 1, ww = w + q - 1;
+                if (hh < 0 || hh >= H || ww < 0 || ww >= Wd) continue;
+                acc += widen(x, dt, ((n * Cin + c) * H + hh) * Wd + ww) *
+                       widen(wt, dt, ((o * Cin + c) * 3 + r) * 3 + q);
+              }
+          total += act_apply(act, acc);
+        }
+      y[n * Cout + o] = total / (double)(H * Wd);
+    }
+  return 0;
+}
+
 }  // extern "C"

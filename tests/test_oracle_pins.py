@@ -126,6 +126,22 @@ def test_row_max_mean_logsumexp():
         assert np.array_equal(oracle.gemm_rowreduce(X, W, b, "none", red), np.full(3, 900.0))
 
 
+def test_conv_act_global_average_pool():
+    """Global average pooling after the convolution: against the separately pinned convolution
+    averaged by numpy, and a closed form (all-ones image and kernel: each output pixel counts
+    its in-image taps, 9 inside, 6 on an edge, 4 in a corner)."""
+    d = ki.conv_inputs(seed=5, Nb=2, Cin=3, H=5, W=6, Cout=4, groups=0, dtype="f32")
+    for act in ("none", "relu", "mish"):
+        full = oracle.conv3x3_gn(d["x"], d["w"], d["bias"], act, 0)
+        got = oracle.conv3x3_act_gap(d["x"], d["w"], d["bias"], act)
+        assert got.shape == (2, 4)
+        assert np.abs(got - full.mean(axis=(2, 3))).max() < 1e-15
+    H, W, C = 4, 7, 2
+    ones = oracle.conv3x3_act_gap(np.ones((1, C, H, W), np.float32), np.ones((3, C, 3, 3), np.float32), None, "none")
+    taps = 9 * (H - 2) * (W - 2) + 6 * (2 * (H - 2) + 2 * (W - 2)) + 4 * 4
+    assert np.abs(ones - C * taps / (H * W)).max() < 1e-13
+
+
 def test_paper_constants_and_chain95():
     g = golden()
     assert abs(g["erf_gelu_inner_scale"] - 1.0 / math.sqrt(2.0)) < 1e-15

@@ -434,6 +434,7 @@ SWEEP_CONV = [  # (Nb, Cin, H, W, Cout, groups [GroupNorm] or -pool [softmax + m
     (32, 64, 56, 56, 64, 8), (32, 128, 28, 28, 128, 8), (32, 256, 14, 14, 256, 8), (16, 3, 224, 224, 64, 8),
 ]
 SWEEP_CONV_F32 = [(32, 64, 56, 56, 64, 8), (16, 64, 32, 32, 64, 8)]   # fp32, ReLU + GroupNorm
+SWEEP_CONV_GAP = [(128, 64, 64, 64, 128), (32, 64, 56, 56, 64)]        # bf16, ReLU + global average pool
 SWEEP_ROWRED_F32 = [(2048, 4096, 1024, "none", "softmax"), (4096, 1024, 1024, "sigmoid", "sum")]
 
 
@@ -517,6 +518,15 @@ def run_sweep(kf, device):
                    lambda x=x, w=w, b=b, out=out, pool=pool: kf.conv3x3_softmax_pool(x, w, b, pool, out=out),
                    lambda x=x, w=w, b=b, pool=pool: F.max_pool2d(torch.softmax(F.conv2d(x, w, b, padding=1), dim=1), pool),
                    flops)
+        del x, w, b, out
+    for Nb, Cin, H, Wd, Cout in SWEEP_CONV_GAP:
+        dt = torch.bfloat16
+        x, w, b = rnd((Nb, Cin, H, Wd), dt), rnd((Cout, Cin, 3, 3), dt, (9 * Cin) ** -0.5), rnd((Cout,), dt, 0.1)
+        out = torch.empty((Nb, Cout), dtype=torch.float32, device=device)
+        record("conv-centered", "bf16 conv %dx%dx%dx%d->%d relu global-avg-pool" % (Nb, Cin, H, Wd, Cout),
+               lambda x=x, w=w, b=b, out=out: kf.conv3x3_act_gap(x, w, b, "relu", out=out),
+               lambda x=x, w=w, b=b: torch.relu(F.conv2d(x, w, b, padding=1)).mean(dim=(2, 3)),
+               2.0 * Nb * H * Wd * Cout * Cin * 9)
         del x, w, b, out
     sp = np.array([r["speedup"] for r in rows])
     summary = {"shapes": len(rows), "fast_1": round(float((sp > 1.0).mean()), 3),

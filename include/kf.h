@@ -198,6 +198,21 @@ kf_status kf_conv3x3_softmax_pool(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd
 size_t kf_conv3x3_softmax_pool_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd,
                                                int64_t Cout, kf_dtype io_dtype);
 
+/* 3x3 convolution (pad 1) + bias + activation + global average pooling: one number per image and
+ * output channel.  A reduction-dominated conv chain in the sense of the paper's Table 2; the
+ * pooling is PyTorch's AdaptiveAvgPool2d(1).
+ *   out[n,o] = (1 / (H*Wd)) * sum_{h,w} act( bias[o] + sum_{c,r,s} x[n,c,h+r-1,w+s-1]*w[o,c,r,s] )
+ * x NCHW, w OIHW of io_dtype; out is [Nb,Cout] fp32, dense.  On the bf16 tensor-core path (same
+ * shapes as kf_conv3x3_epilogue) the per-channel sums are taken in the convolution's epilogue
+ * from the fp32 values and the activation tensor is never written; on the other paths it is
+ * written to the workspace in io_dtype and averaged by a second kernel. */
+kf_status kf_conv3x3_act_gap(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                             kf_dtype io_dtype, const void* x, const void* w, const void* bias,
+                             kf_act act, float* out,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream);
+size_t kf_conv3x3_act_gap_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                                          kf_dtype io_dtype);
+
 /* Workspace sizes in bytes for the calls above with the same arguments (0 = none needed).
  * Pure host arithmetic; no CUDA call is made. */
 size_t kf_gemm_epilogue_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype);

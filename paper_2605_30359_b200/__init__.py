@@ -30,6 +30,7 @@ RED = {"softmax": 0, "sum": 1, "max": 2, "mean": 3, "logsumexp": 4}
 EXPORTS = ["kf_gemm_epilogue", "kf_gemm_rowreduce", "kf_gemm_rowreduce_static",
            "kf_conv3x3_epilogue", "kf_conv3x3_softmax_pool",
            "kf_conv3x3_softmax_pool_workspace_bytes", "kf_selftest_bounded_wait",
+           "kf_conv3x3_act_gap", "kf_conv3x3_act_gap_workspace_bytes",
            "kf_gemm_epilogue_workspace_bytes", "kf_gemm_rowreduce_workspace_bytes",
            "kf_conv3x3_workspace_bytes", "kf_device_status", "kf_launch_count",
            "kf_status_string", "kf_version"]
@@ -70,6 +71,10 @@ def lib() -> ctypes.CDLL:
     L.kf_conv3x3_softmax_pool.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp, sz, vp]
     L.kf_conv3x3_softmax_pool_workspace_bytes.restype = sz
     L.kf_conv3x3_softmax_pool_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, ci]
+    L.kf_conv3x3_act_gap.restype = ci
+    L.kf_conv3x3_act_gap.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp, sz, vp]
+    L.kf_conv3x3_act_gap_workspace_bytes.restype = sz
+    L.kf_conv3x3_act_gap_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, ci]
     L.kf_selftest_bounded_wait.restype = ci
     L.kf_selftest_bounded_wait.argtypes = [ctypes.c_uint64, ctypes.POINTER(ctypes.c_uint64), vp]
     L.kf_gemm_epilogue_workspace_bytes.restype = sz
@@ -128,6 +133,16 @@ def kf_conv3x3_softmax_pool(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, pool, y,
 
 def kf_conv3x3_softmax_pool_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype) -> int:
     return lib().kf_conv3x3_softmax_pool_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype)
+
+
+def kf_conv3x3_act_gap(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, out, workspace,
+                       workspace_bytes, stream) -> int:
+    return lib().kf_conv3x3_act_gap(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, out, workspace,
+                                    workspace_bytes, stream)
+
+
+def kf_conv3x3_act_gap_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype) -> int:
+    return lib().kf_conv3x3_act_gap_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype)
 
 
 def kf_selftest_bounded_wait(limit_ns, stream=None):
@@ -299,6 +314,26 @@ def conv3x3_softmax_pool(x, w, bias=None, pool=1, out=None, stream=None):
                                  _ptr(out), _ptr(ws), nb, _stream_ptr(stream))
     if st != KF_OK:
         raise KfError(st, "kf_conv3x3_softmax_pool")
+    return out
+
+
+def conv3x3_act_gap(x, w, bias=None, act="none", out=None, stream=None):
+    """out[Nb, Cout] fp32 = mean over H, W of act(conv3x3_pad1(x, w) + bias); NCHW / OIHW."""
+    torch = _torch()
+    _check_cuda(x, w, bias, out)
+    if not (x.is_contiguous() and w.is_contiguous()):
+        raise ValueError("conv3x3_act_gap takes contiguous NCHW / OIHW tensors")
+    Nb, Cin, H, Wd = x.shape
+    Cout = w.shape[0]
+    dt = _kf_dtype(x)
+    if out is None:
+        out = torch.empty((Nb, Cout), dtype=torch.float32, device=x.device)
+    nb = kf_conv3x3_act_gap_workspace_bytes(Nb, Cin, H, Wd, Cout, dt)
+    ws = workspace(nb, x.device)
+    st = kf_conv3x3_act_gap(Nb, Cin, H, Wd, Cout, dt, _ptr(x), _ptr(w), _ptr(bias), ACT[act],
+                            _ptr(out), _ptr(ws), nb, _stream_ptr(stream))
+    if st != KF_OK:
+        raise KfError(st, "kf_conv3x3_act_gap")
     return out
 
 

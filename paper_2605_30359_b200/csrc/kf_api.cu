@@ -662,15 +662,21 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
   return KF_OK;
 }
 
-kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+// The convolution chain.  gap_out == nullptr: y = GroupNorm(act(conv + bias)) as documented for
+// kf_conv3x3_epilogue.  gap_out != nullptr (groups must be 0): additionally gap_out[n,o] = mean
+// over the image of act(conv + bias); on the bf16 tensor-core path the activations are then not
+// stored at all (y may be null there), on the other paths y is a scratch buffer.
+static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
                               kf_dtype io_dtype, const void* x, const void* w, const void* bias,
                               kf_act act, int groups, float eps, const void* gamma,
                               const void* beta, void* y, void* workspace, size_t workspace_bytes,
-                              void* cuda_stream) {
+                              void* cuda_stream, float* gap_out) {
   if (Nb < 1 || Cin < 1 || H < 1 || Wd < 1 || Cout < 1) return KF_ERR_INVALID_ARG;
   if (Nb > kMaxDim || Cin > kMaxDim || H > kMaxDim || Wd > kMaxDim || Cout > kMaxDim) return KF_ERR_INVALID_ARG;
   if (!valid_dtype(io_dtype) || !valid_act(act)) return KF_ERR_INVALID_ARG;
-  if (x == nullptr || w == nullptr || y == nullptr || y == x) return KF_ERR_INVALID_ARG;
+  const bool gap_in_epilogue = gap_out != nullptr && !conv_tf32_ok(io_dtype, Nb, Cin, H, Wd, Cout) &&
+                               conv_umma_shape_ok(io_dtype, Cin, H, Wd, Cout);
+  if (x == nullptr || w == nullptr || (y == nullptr && !gap_in_epilogue) || y == x) return KF_ERR_INVALID_ARG;
   if (groups < 0 || (groups > 0 && Cout % groups != 0)) return KF_ERR_INVALID_ARG;
   if (groups > 0 && !(eps >= 0.0f)) return KF_ERR_INVALID_ARG;
   const size_t es = esize(io_dtype);
@@ -773,16 +779,23 @@ kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
     p.tiles_per_unit = 1;
     p.bias = static_cast<const __nv_bfloat16*>(bias);
     p.out = y; p.scale = 1.0f;
-    p.partial = groups > 0 ? stats : nullptr;
+    p.partial = (groups > 0 || gap_in_epilogue) ? stats : nullptr;
+    p.stats_only = gap_in_epilogue ? 1 : 0;      // means only: the activations are not stored
     p.status = d->status;
     p.H = static_cast<int>(H); p.Wd = static_cast<int>(Wd); p.Cin = static_cast<int>(Cp);
     p.rows_per_tile = rows;
     // the output pieces travel by TMA when every image plane starts on 16 bytes
-    p.staged = (aligned(y, 16) && hw % 8 == 0) ? 1 : 0;
+    p.staged = (!gap_in_epilogue && aligned(y, 16) && hw % 8 == 0) ? 1 : 0;
     if (p.staged && !encode_nchw_out(&tm.y, y, Nb, Cout, hw)) return KF_ERR_CUDA;
     const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
     if (launch_umma_conv(bn, act, tm, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
     ++launches;
+    if (gap_in_epilogue) {
+      if (launch_gap_finalize(static_cast<int>(Nb), static_cast<int>(Cout),
+                              static_cast<int>(conv_stat_parts(H, Wd)), hw, stats, gap_out, st) != cudaSuccess)
+        return KF_ERR_CUDA;
+      ++launches;
+    }
     if (groups > 0) {
       if (launch_groupnorm_apply(static_cast<int>(Nb), static_cast<int>(Cout), groups, hw,
                                  static_cast<int>(conv_stat_parts(H, Wd)), eps, stats, gamma, beta,
@@ -803,8 +816,49 @@ kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
       ++launches;
     }
   }
+  if (gap_out != nullptr && !gap_in_epilogue) {
+    if (launch_plane_mean(io_dtype, Nb * Cout, hw, y, gap_out, st) != cudaSuccess) return KF_ERR_CUDA;
+    ++launches;
+  }
   g_launches += launches;
   return KF_OK;
+}
+
+kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                              kf_dtype io_dtype, const void* x, const void* w, const void* bias,
+                              kf_act act, int groups, float eps, const void* gamma,
+                              const void* beta, void* y, void* workspace, size_t workspace_bytes,
+                              void* cuda_stream) {
+  return conv3x3_impl(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, groups, eps, gamma, beta, y,
+                      workspace, workspace_bytes, cuda_stream, nullptr);
+}
+
+size_t kf_conv3x3_act_gap_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                                          kf_dtype io_dtype) {
+  if (Nb < 1 || Cin < 1 || H < 1 || Wd < 1 || Cout < 1) return 0;
+  const size_t conv_ws = kf_conv3x3_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype, 0);
+  if (!conv_tf32_ok(io_dtype, Nb, Cin, H, Wd, Cout) && conv_umma_shape_ok(io_dtype, Cin, H, Wd, Cout))
+    return conv_ws;                     // the means come out of the convolution's epilogue
+  return round256(static_cast<size_t>(Nb) * Cout * H * Wd * esize(io_dtype)) + conv_ws;
+}
+
+kf_status kf_conv3x3_act_gap(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                             kf_dtype io_dtype, const void* x, const void* w, const void* bias,
+                             kf_act act, float* out, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream) {
+  if (Nb < 1 || Cin < 1 || H < 1 || Wd < 1 || Cout < 1) return KF_ERR_INVALID_ARG;
+  if (!valid_dtype(io_dtype) || out == nullptr || !aligned(out, 4)) return KF_ERR_INVALID_ARG;
+  if (Nb > kMaxDim || Cout > kMaxDim || H > kMaxDim || Wd > kMaxDim) return KF_ERR_INVALID_ARG;
+  kf_status vs = check_workspace(workspace, workspace_bytes,
+                                 kf_conv3x3_act_gap_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype));
+  if (vs != KF_OK) return vs;
+  if (!conv_tf32_ok(io_dtype, Nb, Cin, H, Wd, Cout) && conv_umma_shape_ok(io_dtype, Cin, H, Wd, Cout))
+    return conv3x3_impl(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, 0, 0.0f, nullptr, nullptr, nullptr,
+                        workspace, workspace_bytes, cuda_stream, out);
+  const size_t y_bytes = round256(static_cast<size_t>(Nb) * Cout * H * Wd * esize(io_dtype));
+  const size_t rest = workspace_bytes - y_bytes;
+  return conv3x3_impl(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, 0, 0.0f, nullptr, nullptr, workspace,
+                      rest ? static_cast<uint8_t*>(workspace) + y_bytes : nullptr, rest, cuda_stream, out);
 }
 
 }  // extern "C"

@@ -63,6 +63,12 @@ cudaError_t launch_groupnorm_apply(int Nb, int Cout, int groups, long long hw, i
                                    float eps, const float* stats, const void* gamma,
                                    const void* beta, void* y, cudaStream_t st);
 
+// global average pooling: from the convolution's statistics, or from a stored NCHW tensor
+cudaError_t launch_gap_finalize(int Nb, int Cout, int parts, long long hw, const float* stats, float* out,
+                                cudaStream_t st);
+cudaError_t launch_plane_mean(int dt, long long rows, long long len, const void* in, float* out,
+                              cudaStream_t st);
+
 // bf16 operand repack (any pitch / alignment -> dense rows padded to 8 columns)
 cudaError_t launch_pad_rows_bf16(long long rows, int K, int kp, const void* in, long long ld, void* out,
                                  cudaStream_t st);

@@ -92,6 +92,25 @@ cudaError_t launch_rowstat_finalize(int red, int M, int slices, const float* par
   return cudaGetLastError();
 }
 
+cudaError_t launch_gap_finalize(int Nb, int Cout, int parts, long long hw, const float* stats, float* out,
+                                cudaStream_t st) {
+  const long long total = static_cast<long long>(Nb) * Cout;
+  gap_finalize_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, st>>>(
+      Nb, Cout, parts, hw, reinterpret_cast<const float2*>(stats), out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_plane_mean(int dt, long long rows, long long len, const void* in, float* out,
+                              cudaStream_t st) {
+  if (rows > 0x7fffffffLL) return cudaErrorInvalidValue;
+  if (dt == DT_F32)
+    plane_mean_kernel<float><<<static_cast<unsigned>(rows), 256, 0, st>>>(len, static_cast<const float*>(in), out);
+  else
+    plane_mean_kernel<__nv_bfloat16><<<static_cast<unsigned>(rows), 256, 0, st>>>(
+        len, static_cast<const __nv_bfloat16*>(in), out);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_pad_rows_bf16(long long rows, int K, int kp, const void* in, long long ld, void* out,
                                  cudaStream_t st) {
   const long long total = rows * (kp / 8);

@@ -646,6 +646,34 @@ groupnorm_apply_kernel(int Cout, int groups, long long hw, int tiles_per_image, 
   }
 }
 
+// ---------------------------------------------------------------- global average pooling
+// From the convolution epilogue's statistics: out[n,c] = (sum over the image's pixel tiles of the
+// per-tile channel sums) / (H*W), tiles added in increasing order.
+__global__ void __launch_bounds__(256)
+gap_finalize_kernel(int Nb, int Cout, int parts, long long hw, const float2* __restrict__ stats,
+                    float* __restrict__ out) {
+  const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (gid >= static_cast<long long>(Nb) * Cout) return;
+  const long long n = gid / Cout;
+  const int c = static_cast<int>(gid - n * Cout);
+  float s = 0.0f;
+  for (int t = 0; t < parts; ++t) s += stats[(n * parts + t) * Cout + c].x;
+  out[gid] = s / static_cast<float>(hw);
+}
+
+// From a stored NCHW tensor: out[row] = mean of the row's `len` contiguous elements (a row is
+// one image plane).  One CTA per row.
+template <typename T>
+__global__ void __launch_bounds__(256)
+plane_mean_kernel(long long len, const T* __restrict__ in, float* __restrict__ out) {
+  __shared__ float scratch[32];
+  const T* a = in + static_cast<long long>(blockIdx.x) * len;
+  float s = 0.0f;
+  for (long long i = threadIdx.x; i < len; i += blockDim.x) s += to_f32(a[i]);
+  s = block_reduce<false>(s, scratch);
+  if (threadIdx.x == 0) out[blockIdx.x] = s / static_cast<float>(len);
+}
+
 // ---------------------------------------------------------------- channel softmax + max-pool
 // Second pass of conv -> softmax over channels -> max-pool.  `a` holds the convolution output
 // NCHW.  One thread per pooled output pixel: for each of the pool x pool input pixels the

@@ -640,6 +640,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             s1 += y0 + y1;
             s2 = fmaf(y0, y0, fmaf(y1, y1, s2));
           }
+          if (p.stats_only != 0) continue;     // only the per-channel statistics are wanted
           if (staged) {
             const int b = static_cast<int>(g & 1);
             uint8_t* yb = ybuf + b * kPieceBytes;

@@ -609,6 +609,29 @@ def test_groupnorm_biased_variance_on_gpu(kf):
     assert (got[0, 4:, 0, 0] == 0).all()
 
 
+# ------------------------------------------------------------------ conv -> activation -> global average pool
+@pytest.mark.parametrize("dtype,cfg", [
+    ("bf16", dict(Nb=2, Cin=64, H=8, W=64, Cout=128)),      # means from the tensor-core epilogue
+    ("bf16", dict(Nb=3, Cin=64, H=13, W=64, Cout=96)),      # ragged last tile: its empty rows must not count
+    ("bf16", dict(Nb=2, Cin=128, H=28, W=28, Cout=32)),     # 8-row tiles, padded box
+    ("bf16", dict(Nb=2, Cin=8, H=6, W=30, Cout=16)),        # width without a tiling: direct conv + plane means
+    ("f32", dict(Nb=8, Cin=32, H=32, W=32, Cout=64)),       # fp32 tensor-core conv + plane means
+    ("f32", dict(Nb=2, Cin=3, H=5, W=7, Cout=6)),           # fp32 direct conv
+])
+@pytest.mark.parametrize("act", ["relu", "mish"])
+def test_conv_act_global_average_pool(kf, dtype, cfg, act):
+    d = ki.conv_inputs(seed=14, dtype=dtype, groups=0, **cfg)
+    out = kf.conv3x3_act_gap(to_dev(d["x"]), to_dev(d["w"]), to_dev(d["bias"]), act)
+    check_status()
+    assert tuple(out.shape) == (cfg["Nb"], cfg["Cout"]) and str(out.dtype) == "torch.float32"
+    ref = oracle.conv3x3_act_gap(d["x"], d["w"], d["bias"], act)
+    atol, rtol = tol_for(dtype)
+    assert_close(to_f64(out), ref, atol, rtol, "conv gap %s %s %s" % (dtype, cfg, act))
+    # a mean of hundreds of terms: far tighter than the elementwise tolerance (bf16 planes that
+    # are stored first carry their rounding, 2^-9 relative per term, averaged)
+    assert np.abs(to_f64(out) - ref).max() < (2e-3 if dtype == "bf16" else 2e-5)
+
+
 # ------------------------------------------------------------------ conv -> channel softmax -> max-pool
 def run_conv_softmax_pool(kf, d, pool, use_bias=True):
     bias = d["bias"] if use_bias else None

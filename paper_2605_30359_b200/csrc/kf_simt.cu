@@ -10,7 +10,10 @@ static cudaError_t simt_gemm_t(int mode, int act, int M, int N, int K, const voi
                                long long ldx, const void* W, long long ldw, const void* bias,
                                float scale, const void* R, long long ldr, void* out, long long ldo,
                                cudaStream_t st) {
-  const dim3 grid((M + 31) / 32, (N + 31) / 32), block(256);   // rows on x: up to 2^31-1 tiles
+  // 16 x 16 tiles when 32 x 32 tiles would occupy less than half of a B200's SMs
+  const bool small = static_cast<long long>((M + 31) / 32) * ((N + 31) / 32) < 74;
+  const int t = small ? 16 : 32;
+  const dim3 grid((M + t - 1) / t, (N + t - 1) / t), block(256);   // rows on x: up to 2^31-1 tiles
   if (grid.y > 65535u) return cudaErrorInvalidValue;
   cudaError_t err = cudaSuccess;
   bool ok = dispatch_act(act, [&](auto A) {
@@ -23,8 +26,13 @@ static cudaError_t simt_gemm_t(int mode, int act, int M, int N, int K, const voi
           static_cast<const T*>(bias), scale, static_cast<const T*>(R), ldr, out, ldo, act);
       err = cudaGetLastError();
     };
-    if (mode == 0) go(simt_gemm_kernel<T, 0, ACT>);
-    else go(simt_gemm_kernel<T, 1, ACT>);
+    if (small) {
+      if (mode == 0) go(simt_gemm_kernel<T, 0, ACT, 16, 16>);
+      else go(simt_gemm_kernel<T, 1, ACT, 16, 16>);
+    } else {
+      if (mode == 0) go(simt_gemm_kernel<T, 0, ACT, 32, 32>);
+      else go(simt_gemm_kernel<T, 1, ACT, 32, 32>);
+    }
   });
   return ok ? err : cudaErrorInvalidValue;
 }

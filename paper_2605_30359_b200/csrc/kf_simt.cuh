@@ -33,7 +33,7 @@ __device__ __forceinline__ float block_reduce(float v, float* scratch /*[32]*/) 
 }
 
 // ---------------------------------------------------------------- scalar GEMM + epilogue
-// 32x32 output tile per CTA of eight warps.  The warps split K: in each pass over 256 values of
+// TM x TN output tile per CTA of eight warps (32 x 32 below unless said otherwise).  The warps split K: in each pass over 256 values of
 // k, warp w owns k in [32w, 32w+32), loads its 32x32 slabs of X and W with coalesced reads
 // (lane = k), stages them k-major in its private shared memory and accumulates the whole 32x32
 // tile with an 8x4 register block per lane (32 FMAs per three 16-byte shared loads).  The next
@@ -44,30 +44,37 @@ __device__ __forceinline__ float block_reduce(float v, float* scratch /*[32]*/) 
 constexpr int kSimtLd = 36;                                   // staged row pitch in floats
 constexpr int kSimtSmemBytes = 8 * 2 * 32 * kSimtLd * 4;      // 73,728 bytes of dynamic smem
 
-template <typename T, int MODE, int ACT>
+// TM x TN = 32 x 32, or 16 x 16 for problems whose 32 x 32 tiles would leave most SMs idle (the
+// register block is (TM/4) x (TN/8) per lane; staging pitch and shared memory are the same).
+template <typename T, int MODE, int ACT, int TM, int TN>
 __global__ void __launch_bounds__(256)
 simt_gemm_kernel(int M, int N, int K, const T* __restrict__ X, long long ldx,
                  const T* __restrict__ W, long long ldw, const T* __restrict__ bias, float scale,
                  const T* R, long long ldr, void* out, long long ldo, int act_code) {
+  constexpr int RM = TM / 4, RN = TN / 8;             // register block of a lane
   extern __shared__ float sm[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * 32, n0 = blockIdx.y * 32;
+  const int m0 = blockIdx.x * TM, n0 = blockIdx.y * TN;
   float* As = sm + warp * (2 * 32 * kSimtLd);
   float* Bs = As + 32 * kSimtLd;
   const int ly = lane >> 3, lx = lane & 7;
-  float acc[8][4];
+  float acc[RM][RN];
 #pragma unroll
-  for (int i = 0; i < 8; ++i)
+  for (int i = 0; i < RM; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
-  float ra[32], rb[32];
+    for (int j = 0; j < RN; ++j) acc[i][j] = 0.0f;
+  float ra[TM], rb[TN];
   auto load_slab = [&](int kw) {
     const int k = kw + lane;
     const bool k_ok = k < K;
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      const long long m = m0 + i, n = n0 + i;
+    for (int i = 0; i < TM; ++i) {
+      const long long m = m0 + i;
       ra[i] = (k_ok && m < M) ? to_f32(X[m * ldx + k]) : 0.0f;
+    }
+#pragma unroll
+    for (int i = 0; i < TN; ++i) {
+      const long long n = n0 + i;
       rb[i] = (k_ok && n < N) ? to_f32(W[n * ldw + k]) : 0.0f;
     }
   };
@@ -75,46 +82,50 @@ simt_gemm_kernel(int M, int N, int K, const T* __restrict__ X, long long ldx,
   if (kw < K) load_slab(kw);
   for (; kw < K; kw += 256) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      As[lane * kSimtLd + i] = ra[i];
-      Bs[lane * kSimtLd + i] = rb[i];
-    }
+    for (int i = 0; i < TM; ++i) As[lane * kSimtLd + i] = ra[i];
+#pragma unroll
+    for (int i = 0; i < TN; ++i) Bs[lane * kSimtLd + i] = rb[i];
     __syncwarp();
     if (kw + 256 < K) load_slab(kw + 256);
 #pragma unroll 8
     for (int kk = 0; kk < 32; ++kk) {
-      const float4 a0 = *reinterpret_cast<const float4*>(&As[kk * kSimtLd + ly * 8]);
-      const float4 a1 = *reinterpret_cast<const float4*>(&As[kk * kSimtLd + ly * 8 + 4]);
-      const float4 b = *reinterpret_cast<const float4*>(&Bs[kk * kSimtLd + lx * 4]);
-      const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-      const float bb[4] = {b.x, b.y, b.z, b.w};
+      float a[RM], bb[RN];
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
+      for (int i = 0; i < RM; i += 4)
+        *reinterpret_cast<float4*>(&a[i]) = *reinterpret_cast<const float4*>(&As[kk * kSimtLd + ly * RM + i]);
+      if constexpr (RN == 4) {
+        *reinterpret_cast<float4*>(&bb[0]) = *reinterpret_cast<const float4*>(&Bs[kk * kSimtLd + lx * 4]);
+      } else {
+        *reinterpret_cast<float2*>(&bb[0]) = *reinterpret_cast<const float2*>(&Bs[kk * kSimtLd + lx * 2]);
+      }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], bb[j], acc[i][j]);
+      for (int i = 0; i < RM; ++i)
+#pragma unroll
+        for (int j = 0; j < RN; ++j) acc[i][j] = fmaf(a[i], bb[j], acc[i][j]);
     }
     __syncwarp();
   }
   __syncthreads();                       // staging is dead: reuse it for the partial tiles
-  float* red = sm;                       // [8 warps][32 rows][32 cols]
+  float* red = sm;                       // [8 warps][TM rows][TN cols]
 #pragma unroll
-  for (int i = 0; i < 8; ++i)
-    *reinterpret_cast<float4*>(&red[(warp * 32 + ly * 8 + i) * 32 + lx * 4]) =
-        make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+  for (int i = 0; i < RM; ++i)
+#pragma unroll
+    for (int j = 0; j < RN; ++j) red[(warp * TM + ly * RM + i) * TN + lx * RN + j] = acc[i][j];
   __syncthreads();
-  const int r = threadIdx.x >> 3, c4 = (threadIdx.x & 7) * 4;
-  float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  constexpr int VEC = TM * TN / 256;     // outputs per thread, consecutive columns
+  const int r = threadIdx.x / (TN / VEC), c0 = (threadIdx.x % (TN / VEC)) * VEC;
+  float zs[VEC];
 #pragma unroll
-  for (int w = 0; w < 8; ++w) {
-    const float4 v = *reinterpret_cast<const float4*>(&red[(w * 32 + r) * 32 + c4]);
-    z4.x += v.x; z4.y += v.y; z4.z += v.z; z4.w += v.w;
-  }
-  const float zs[4] = {z4.x, z4.y, z4.z, z4.w};
+  for (int j = 0; j < VEC; ++j) zs[j] = 0.0f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w)
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) zs[j] += red[(w * TM + r) * TN + c0 + j];
   const long long m = m0 + r;
   if (m < M) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int n = n0 + c4 + j;
+    for (int j = 0; j < VEC; ++j) {
+      const int n = n0 + c0 + j;
       if (n < N) {
         float z = zs[j];
         if (bias != nullptr) z += to_f32(bias[n]);

@@ -59,6 +59,8 @@ def _load():
         lib.oracle_conv3x3_softmax_pool.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, i64, vp]
         lib.oracle_conv3x3_act_gap.restype = ci
         lib.oracle_conv3x3_act_gap.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, vp]
+        lib.oracle_gemm_groupnorm.restype = ci
+        lib.oracle_gemm_groupnorm.argtypes = [i64, i64, i64, ci, vp, i64, vp, i64, vp, i64, dbl, vp, vp, ci, vp]
         _lib = lib
     return _lib
 
@@ -159,3 +161,16 @@ def conv3x3_act_gap(x, w, bias=None, act="none"):
                                         ACT[act], _ptr(y))
     assert rc == 0
     return y
+
+
+def gemm_groupnorm(X, W, bias=None, groups=1, eps=1e-5, gamma=None, beta=None, post_act="none"):
+    """post_act(GroupNorm over column groups of (X W^T + bias)), fp64 [M,N]."""
+    X = _c(X); dt = _dt(X); W = _c(W, dt); bias = _c(bias, dt)
+    gamma = _c(gamma, dt); beta = _c(beta, dt)
+    M, K = X.shape
+    N = W.shape[0]
+    Y = np.empty((M, N), np.float64)
+    rc = _load().oracle_gemm_groupnorm(M, N, K, dt, _ptr(X), K, _ptr(W), K, _ptr(bias), int(groups),
+                                       float(eps), _ptr(gamma), _ptr(beta), ACT[post_act], _ptr(Y))
+    assert rc == 0
+    return Y

@@ -316,4 +316,41 @@ int oracle_conv3x3_act_gap(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64
   return 0;
 }
 
+// Z[m,n] = sum_k X[m,k] * W[n,k] + bias[n]
+// per row m and group g of gs = N/groups consecutive columns:
+//   mu = mean_n Z, var = mean_n (Z-mu)^2 (biased), U = (Z-mu)/sqrt(var+eps)*gamma[n]+beta[n]
+// Y[m,n] = post_act(U[m,n]).   GroupNorm of a [M,N] matrix with N as the channel axis, as
+// torch.nn.GroupNorm treats a 2-D input.  gamma/beta null => 1/0.  Y is fp64 [M,N], dense.
+int oracle_gemm_groupnorm(int64_t M, int64_t N, int64_t K, int dt, const void* X, int64_t ldx,
+                          const void* W, int64_t ldw, const void* bias, int64_t groups, double eps,
+                          const void* gamma, const void* beta, int post_act, double* Y) {
+  if (groups < 1 || N % groups != 0) return 1;
+  const int64_t gs = N / groups;
+#pragma omp parallel for schedule(static) num_threads(nthreads())
+  for (int64_t m = 0; m < M; ++m) {
+    std::vector<double> z((size_t)N);
+    for (int64_t n = 0; n < N; ++n) {
+      double a = 0.0;
+      for (int64_t k = 0; k < K; ++k) a += widen(X, dt, m * ldx + k) * widen(W, dt, n * ldw + k);
+      if (bias) a += widen(bias, dt, n);
+      z[(size_t)n] = a;
+    }
+    for (int64_t g = 0; g < groups; ++g) {
+      double mu = 0.0;
+      for (int64_t n = g * gs; n < (g + 1) * gs; ++n) mu += z[(size_t)n];
+      mu /= (double)gs;
+      double var = 0.0;
+      for (int64_t n = g * gs; n < (g + 1) * gs; ++n) var += (z[(size_t)n] - mu) * (z[(size_t)n] - mu);
+      var /= (double)gs;
+      const double rstd = 1.0 / std::sqrt(var + eps);
+      for (int64_t n = g * gs; n < (g + 1) * gs; ++n) {
+        const double ga = gamma ? widen(gamma, dt, n) : 1.0;
+        const double be = beta ? widen(beta, dt, n) : 0.0;
+        Y[m * N + n] = act_apply(post_act, (z[(size_t)n] - mu) * rstd * ga + be);
+      }
+    }
+  }
+  return 0;
+}
+
 }  // extern "C"

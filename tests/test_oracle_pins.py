@@ -142,6 +142,30 @@ def test_conv_act_global_average_pool():
     assert np.abs(ones - C * taps / (H * W)).max() < 1e-13
 
 
+def test_gemm_groupnorm_against_torch_and_moments():
+    """GroupNorm over column groups of a GEMM output: torch's own fp64 group_norm applied to the
+    separately pinned pre-normalisation matrix; unit moments per (row, group); a 2-element group
+    closed form ((-1, +1) whatever the two values, as long as they differ)."""
+    import torch
+    import torch.nn.functional as F
+    d = ki.gemm_inputs("c3", seed=11, M=6, N=48, K=20, dtype="f32")
+    Z = oracle.gemm_epilogue(d["X"], d["W"], d["b"], "none")
+    gamma = ki.store(ki.uniform(11, 7, (48,), 0.5, 1.5), "f32")
+    beta = ki.store(ki.uniform(11, 8, (48,), -1.0, 1.0), "f32")
+    for groups in (1, 3, 12, 48 // 2):
+        want = F.group_norm(torch.from_numpy(Z), groups, torch.from_numpy(gamma.astype(np.float64)),
+                            torch.from_numpy(beta.astype(np.float64)), 1e-5).numpy()
+        got = oracle.gemm_groupnorm(d["X"], d["W"], d["b"], groups, 1e-5, gamma, beta)
+        assert np.abs(got - want).max() < 1e-12, groups
+        swish = oracle.gemm_groupnorm(d["X"], d["W"], d["b"], groups, 1e-5, gamma, beta, "swish")
+        assert np.abs(swish - want / (1.0 + np.exp(-want))).max() < 1e-12
+    plain = oracle.gemm_groupnorm(d["X"], d["W"], d["b"], 4, 0.0).reshape(6, 4, 12)
+    assert np.abs(plain.mean(axis=2)).max() < 1e-14
+    assert np.abs(plain.var(axis=2) - 1.0).max() < 1e-13
+    two = oracle.gemm_groupnorm(d["X"], d["W"], d["b"], 24, 0.0).reshape(6, 24, 2)
+    assert np.abs(np.sort(two, axis=2) - np.array([-1.0, 1.0])).max() < 1e-9
+
+
 def test_paper_constants_and_chain95():
     g = golden()
     assert abs(g["erf_gelu_inner_scale"] - 1.0 / math.sqrt(2.0)) < 1e-15

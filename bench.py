@@ -434,6 +434,7 @@ SWEEP_CONV = [  # (Nb, Cin, H, W, Cout, groups [GroupNorm] or -pool [softmax + m
     (32, 64, 56, 56, 64, 8), (32, 128, 28, 28, 128, 8), (32, 256, 14, 14, 256, 8), (16, 3, 224, 224, 64, 8),
 ]
 SWEEP_CONV_F32 = [(32, 64, 56, 56, 64, 8), (16, 64, 32, 32, 64, 8)]   # fp32, ReLU + GroupNorm
+SWEEP_GEMM_GN = [(8192, 4096, 4096, 128), (1024, 1024, 1024, 32), (128, 1024, 512, 32)]   # bf16, GroupNorm + swish
 SWEEP_CONV_GAP = [(128, 64, 64, 64, 128), (32, 64, 56, 56, 64)]        # bf16, ReLU + global average pool
 SWEEP_ROWRED_F32 = [(2048, 4096, 1024, "none", "softmax"), (4096, 1024, 1024, "sigmoid", "sum")]
 
@@ -519,6 +520,20 @@ def run_sweep(kf, device):
                    lambda x=x, w=w, b=b, pool=pool: F.max_pool2d(torch.softmax(F.conv2d(x, w, b, padding=1), dim=1), pool),
                    flops)
         del x, w, b, out
+    for M, N, K, groups in SWEEP_GEMM_GN:
+        dt = torch.bfloat16
+        X, W, b = rnd((M, K), dt), rnd((N, K), dt, K ** -0.5), rnd((N,), dt, K ** -0.5)
+        ga, be = rnd((N,), dt, 0.1) + 1.0, rnd((N,), dt, 0.1)
+        out = torch.empty((M, N), dtype=dt, device=device)
+
+        def ref(X=X, W=W, b=b, ga=ga, be=be, groups=groups):
+            z = F.group_norm(F.linear(X, W, b), groups, ga, be, 1e-5)
+            return torch.sigmoid(z) * z
+
+        record("mixed-reduction", "bf16 %dx%dx%d GroupNorm%d swish" % (M, N, K, groups),
+               lambda X=X, W=W, b=b, ga=ga, be=be, out=out, groups=groups:
+               kf.gemm_groupnorm(X, W, b, groups, 1e-5, ga, be, "swish", out=out), ref, 2.0 * M * N * K)
+        del X, W, b, ga, be, out
     for Nb, Cin, H, Wd, Cout in SWEEP_CONV_GAP:
         dt = torch.bfloat16
         x, w, b = rnd((Nb, Cin, H, Wd), dt), rnd((Cout, Cin, 3, 3), dt, (9 * Cin) ** -0.5), rnd((Cout,), dt, 0.1)

@@ -108,6 +108,26 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
                            const void* residual, int64_t ldr, void* Y, int64_t ldy,
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* GEMM + bias + GroupNorm over groups of consecutive columns + activation (a "mixed reduction"
+ * chain in the sense of the paper's Table 2; the normalisation is torch.nn.GroupNorm applied to
+ * a [M,N] matrix, N being the channel axis).  With Z[m,n] = sum_k X[m,k]*W[n,k] + bias[n] and
+ * gs = N / groups, per row m and group g (columns [g*gs, (g+1)*gs)):
+ *   mu = mean Z, var = mean (Z-mu)^2 (biased), Y = post_act((Z-mu)/sqrt(var+eps)*gamma[n]+beta[n]).
+ * gamma, beta [N] of io_dtype, may be NULL (1, 0); groups must divide N (groups = 1 normalises
+ * the whole row, as a LayerNorm does).  bf16 problems whose group size is 32, 64,
+ * 128 or 256, with TMA-loadable operands (see kf_gemm_epilogue) and a 16-byte aligned Y with
+ * ldy % 8 == 0, run in ONE tensor-core kernel: a tile of 256 columns holds whole groups, so the
+ * epilogue takes the statistics from the accumulator and normalises before storing.  Everything
+ * else computes Z in fp32 into the workspace (M*N*4 bytes, plus the split operands for large fp32
+ * problems) and normalises with a second kernel. */
+kf_status kf_gemm_groupnorm(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
+                            const void* X, int64_t ldx, const void* W, int64_t ldw,
+                            const void* bias, int groups, float eps, const void* gamma,
+                            const void* beta, kf_act post_act, void* Y, int64_t ldy,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+size_t kf_gemm_groupnorm_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
+                                         int groups);
+
 /* GEMM + row reduction over N (Appendix A, "Algorithmic Optimization": online softmax;
  * Appendix C.1 prints the three-pass softmax definition; Table 2 "Mixed reduction" and
  * "Reduction-dominated").  With A[m,n] = pre_act( sum_k X[m,k]*W[n,k] + bias[n] ):

@@ -31,6 +31,7 @@ EXPORTS = ["kf_gemm_epilogue", "kf_gemm_rowreduce", "kf_gemm_rowreduce_static",
            "kf_conv3x3_epilogue", "kf_conv3x3_softmax_pool",
            "kf_conv3x3_softmax_pool_workspace_bytes", "kf_selftest_bounded_wait",
            "kf_conv3x3_act_gap", "kf_conv3x3_act_gap_workspace_bytes",
+           "kf_gemm_groupnorm", "kf_gemm_groupnorm_workspace_bytes",
            "kf_gemm_epilogue_workspace_bytes", "kf_gemm_rowreduce_workspace_bytes",
            "kf_conv3x3_workspace_bytes", "kf_device_status", "kf_launch_count",
            "kf_status_string", "kf_version"]
@@ -71,6 +72,11 @@ def lib() -> ctypes.CDLL:
     L.kf_conv3x3_softmax_pool.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp, sz, vp]
     L.kf_conv3x3_softmax_pool_workspace_bytes.restype = sz
     L.kf_conv3x3_softmax_pool_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, ci]
+    L.kf_gemm_groupnorm.restype = ci
+    L.kf_gemm_groupnorm.argtypes = [i64, i64, i64, ci, vp, i64, vp, i64, vp, ci, ctypes.c_float, vp, vp, ci,
+                                    vp, i64, vp, sz, vp]
+    L.kf_gemm_groupnorm_workspace_bytes.restype = sz
+    L.kf_gemm_groupnorm_workspace_bytes.argtypes = [i64, i64, i64, ci, ci]
     L.kf_conv3x3_act_gap.restype = ci
     L.kf_conv3x3_act_gap.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp, sz, vp]
     L.kf_conv3x3_act_gap_workspace_bytes.restype = sz
@@ -133,6 +139,16 @@ def kf_conv3x3_softmax_pool(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, pool, y,
 
 def kf_conv3x3_softmax_pool_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype) -> int:
     return lib().kf_conv3x3_softmax_pool_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype)
+
+
+def kf_gemm_groupnorm(M, N, K, io_dtype, X, ldx, W, ldw, bias, groups, eps, gamma, beta, post_act, Y, ldy,
+                      workspace, workspace_bytes, stream) -> int:
+    return lib().kf_gemm_groupnorm(M, N, K, io_dtype, X, ldx, W, ldw, bias, groups, eps, gamma, beta,
+                                   post_act, Y, ldy, workspace, workspace_bytes, stream)
+
+
+def kf_gemm_groupnorm_workspace_bytes(M, N, K, io_dtype, groups) -> int:
+    return lib().kf_gemm_groupnorm_workspace_bytes(M, N, K, io_dtype, groups)
 
 
 def kf_conv3x3_act_gap(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, out, workspace,
@@ -314,6 +330,31 @@ def conv3x3_softmax_pool(x, w, bias=None, pool=1, out=None, stream=None):
                                  _ptr(out), _ptr(ws), nb, _stream_ptr(stream))
     if st != KF_OK:
         raise KfError(st, "kf_conv3x3_softmax_pool")
+    return out
+
+
+def gemm_groupnorm(X, W, bias=None, groups=1, eps=1e-5, gamma=None, beta=None, post_act="none", out=None,
+                   stream=None):
+    """Y = post_act(GroupNorm over groups of N/groups consecutive columns of (X @ W.T + bias))."""
+    torch = _torch()
+    _check_cuda(X, W, bias, gamma, beta, out)
+    M, K = X.shape
+    N = W.shape[0]
+    dt = _kf_dtype(X)
+    if out is None:
+        out = torch.empty((M, N), dtype=X.dtype, device=X.device)
+    nb = kf_gemm_groupnorm_workspace_bytes(M, N, K, dt, int(groups))
+    if nb == 0 and dt == KF_BF16:
+        # the query cannot see pitches and alignment: give the fallback its scratch when needed
+        if not (X.stride(0) % 8 == 0 and W.stride(0) % 8 == 0 and out.stride(0) % 8 == 0 and
+                X.data_ptr() % 16 == 0 and W.data_ptr() % 16 == 0 and out.data_ptr() % 16 == 0):
+            nb = M * N * 4
+    ws = workspace(nb, X.device)
+    st = kf_gemm_groupnorm(M, N, K, dt, _ptr(X), X.stride(0), _ptr(W), W.stride(0), _ptr(bias), int(groups),
+                           float(eps), _ptr(gamma), _ptr(beta), ACT[post_act], _ptr(out), out.stride(0),
+                           _ptr(ws), nb, _stream_ptr(stream))
+    if st != KF_OK:
+        raise KfError(st, "kf_gemm_groupnorm")
     return out
 
 

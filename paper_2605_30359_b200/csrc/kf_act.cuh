@@ -87,6 +87,23 @@ __device__ __forceinline__ float act_f(float z, int code = 0) {
   }
 }
 
+// Any activation by its run-time code (scalar kernels where the epilogue is not the hot part).
+template <bool FAST>
+__device__ __forceinline__ float act_any(int code, float z) {
+  switch (code) {
+    case ACT_NONE: return z;
+    case ACT_RELU: return act_f<ACT_RELU, FAST>(z);
+    case ACT_GELU_TANH: return act_f<ACT_GELU_TANH, FAST>(z);
+    case ACT_SIGMOID: return act_f<ACT_SIGMOID, FAST>(z);
+    case ACT_GELU_ERF: return act_f<ACT_GELU_ERF, FAST>(z);
+    case ACT_SWISH: return act_f<ACT_SWISH, FAST>(z);
+    case ACT_TANH: return act_f<ACT_TANH, FAST>(z);
+    case ACT_HARDTANH: return act_f<ACT_HARDTANH, FAST>(z);
+    case ACT_CHAIN95: return act_f<ACT_CHAIN95, FAST>(z);
+    default: return act_rt<FAST>(code, z);
+  }
+}
+
 // Runtime-to-compile-time dispatch over the activation code.
 template <typename F>
 __host__ inline bool dispatch_act(int act, F&& f) {

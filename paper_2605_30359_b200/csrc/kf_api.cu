@@ -543,6 +543,90 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
   return KF_OK;
 }
 
+size_t kf_gemm_groupnorm_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, int groups) {
+  if (M < 1 || N < 1 || K < 1 || groups < 1 || N % groups != 0) return 0;
+  const int64_t gs = N / groups;
+  if (io_dtype == KF_BF16 && K % 8 == 0 && (gs == 32 || gs == 64 || gs == 128 || gs == 256)) return 0;
+  return rowreduce_simt_ws(M, N) + (use_tf32x3(io_dtype, M, N, K) ? tf32_ws(M, N, K) : 0);
+}
+
+kf_status kf_gemm_groupnorm(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, const void* X,
+                            int64_t ldx, const void* W, int64_t ldw, const void* bias, int groups,
+                            float eps, const void* gamma, const void* beta, kf_act post_act, void* Y,
+                            int64_t ldy, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  kf_status vs = check_gemm_common(M, N, K, io_dtype, X, ldx, W, ldw, bias);
+  if (vs != KF_OK) return vs;
+  if (!valid_act(post_act) || Y == nullptr || ldy < N || groups < 1 || N % groups != 0) return KF_ERR_INVALID_ARG;
+  if (!(eps >= 0.0f) || Y == X || Y == W) return KF_ERR_INVALID_ARG;
+  const size_t es = esize(io_dtype);
+  if (!aligned(Y, es) || !aligned(gamma, es) || !aligned(beta, es)) return KF_ERR_INVALID_ARG;
+  DeviceInfo* d = nullptr;
+  if (!device_info(&d)) return KF_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t gs = N / groups;
+  const bool staged_ok = ldy % 8 == 0 && aligned(Y, 16);
+  if (umma_gemm_ok(io_dtype, K, X, ldx, W, ldw) && staged_ok &&
+      (gs == 32 || gs == 64 || gs == 128 || gs == 256)) {
+    // whole groups lie inside every tile: statistics and normalisation in the epilogue
+    // tile width as for the plain chain, but never narrower than a group
+    int bn = pick_tile_n(M, N, d->sm_count);
+    if (bn < gs) bn = static_cast<int>(gs);
+    const bool pair = bn == 256 && use_cta_pairs(M, K);
+    UmmaMaps tm;
+    if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, pair ? bn / 2 : bn))
+      return KF_ERR_CUDA;
+    UmmaParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.act_rt = post_act;
+    p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+    const int tile_m = pair ? 2 * kBM : kBM;
+    p.tiles_m = static_cast<int>((M + tile_m - 1) / tile_m);
+    p.tiles_n = static_cast<int>((N + bn - 1) / bn);
+    if (static_cast<int64_t>(p.tiles_m) * p.tiles_n > kMaxDim) return KF_ERR_UNSUPPORTED;
+    p.num_tiles = p.tiles_m * p.tiles_n;
+    p.k_blocks = static_cast<int>((K + kBK - 1) / kBK);
+    p.tiles_per_unit = 1;
+    p.bias = static_cast<const __nv_bfloat16*>(bias);
+    p.out = Y; p.ldo = ldy; p.scale = 1.0f;
+    p.vec_ok = 1; p.staged = 1;
+    p.bias_vec = aligned(bias, 16) ? 1 : 0;
+    p.gn_pieces = static_cast<int>(gs / 32);
+    p.gn_eps = eps;
+    p.gn_gamma = static_cast<const __nv_bfloat16*>(gamma);
+    p.gn_beta = static_cast<const __nv_bfloat16*>(beta);
+    tm.r = tm.a;
+    if (!encode_piece(&tm.y, Y, M, N, ldy)) return KF_ERR_CUDA;
+    p.status = d->status;
+    const int slots = pair ? d->sm_count / 2 : d->sm_count;
+    const int grid = p.num_tiles < slots ? p.num_tiles : slots;
+    if (launch_umma_elementwise(bn, post_act, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
+      return KF_ERR_CUDA;
+    g_launches += 1;
+    return KF_OK;
+  }
+  // scalar path: pre-normalisation values in fp32 (the FMA kernel, or the fp32 tensor-core
+  // chain for large fp32 problems), then one CTA per row
+  const bool tensor32 = use_tf32x3(io_dtype, M, N, K);
+  vs = check_workspace(workspace, workspace_bytes, rowreduce_simt_ws(M, N) + (tensor32 ? tf32_ws(M, N, K) : 0));
+  if (vs != KF_OK) return vs;
+  float* A = static_cast<float*>(workspace);
+  if (tensor32) {
+    vs = run_tf32_chain(M, N, K, X, ldx, W, ldw, bias, ACT_NONE, 1.0f, nullptr, 0, A, N,
+                        static_cast<uint8_t*>(workspace) + rowreduce_simt_ws(M, N), d, st);
+    if (vs != KF_OK) return vs;
+  } else {
+    if (launch_simt_gemm(io_dtype, 1, ACT_NONE, static_cast<int>(M), static_cast<int>(N),
+                         static_cast<int>(K), X, ldx, W, ldw, bias, 1.0f, nullptr, 0, A, N, st) != cudaSuccess)
+      return KF_ERR_CUDA;
+    g_launches += 1;
+  }
+  if (launch_row_groupnorm(io_dtype, static_cast<int>(M), static_cast<int>(N), static_cast<int>(gs), eps, A,
+                           N, gamma, beta, post_act, Y, ldy, st) != cudaSuccess)
+    return KF_ERR_CUDA;
+  g_launches += 1;
+  return KF_OK;
+}
+
 kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, const void* X,
                             int64_t ldx, const void* W, int64_t ldw, const void* bias,
                             kf_act pre_act, kf_rowred red, void* out, int64_t ldo,
@@ -551,7 +635,7 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
   kf_status vs = check_gemm_common(M, N, K, in_dtype, X, ldx, W, ldw, bias);
   if (vs != KF_OK) return vs;
   if (!valid_act(pre_act) || out == nullptr || !valid_dtype(out_dtype)) return KF_ERR_INVALID_ARG;
-  if (red < 0 || red >= RED_COUNT) return KF_ERR_INVALID_ARG;
+  if (static_cast<int>(red) < 0 || static_cast<int>(red) >= RED_COUNT) return KF_ERR_INVALID_ARG;
   if (red != KF_RED_SOFTMAX && out_dtype != KF_F32) return KF_ERR_INVALID_ARG;
   if (red == KF_RED_SOFTMAX && ldo < N) return KF_ERR_INVALID_ARG;
   if (!aligned(out, esize(out_dtype))) return KF_ERR_INVALID_ARG;
@@ -910,7 +994,7 @@ extern "C" kf_status kf_gemm_rowreduce_static(int64_t M, int64_t N, int64_t K, k
                                               kf_rowred red, void* out, int64_t ldo,
                                               kf_dtype out_dtype, void* cuda_stream) {
   // Refuse, before touching the device, any problem whose partial statistics do not fit.
-  if (M >= 1 && N >= 1 && K >= 1 && red >= 0 && red < RED_COUNT &&
+  if (M >= 1 && N >= 1 && K >= 1 && static_cast<int>(red) >= 0 && static_cast<int>(red) < RED_COUNT &&
       (in_dtype == KF_F32 || in_dtype == KF_BF16) &&
       kf_gemm_rowreduce_workspace_bytes(M, N, K, in_dtype, red) > KF_STATIC_SCRATCH_BYTES)
     return KF_ERR_WORKSPACE;

@@ -63,6 +63,11 @@ cudaError_t launch_groupnorm_apply(int Nb, int Cout, int groups, long long hw, i
                                    float eps, const float* stats, const void* gamma,
                                    const void* beta, void* y, cudaStream_t st);
 
+// GroupNorm over column groups of an fp32 matrix + activation (scalar path of kf_gemm_groupnorm)
+cudaError_t launch_row_groupnorm(int dt, int M, int N, int gs, float eps, const float* A, long long lda,
+                                 const void* gamma, const void* beta, int act, void* Y, long long ldy,
+                                 cudaStream_t st);
+
 // global average pooling: from the convolution's statistics, or from a stored NCHW tensor
 cudaError_t launch_gap_finalize(int Nb, int Cout, int parts, long long hw, const float* stats, float* out,
                                 cudaStream_t st);

@@ -100,6 +100,20 @@ cudaError_t launch_rowstat_finalize(int red, int M, int slices, const float* par
   return cudaGetLastError();
 }
 
+cudaError_t launch_row_groupnorm(int dt, int M, int N, int gs, float eps, const float* A, long long lda,
+                                 const void* gamma, const void* beta, int act, void* Y, long long ldy,
+                                 cudaStream_t st) {
+  if (dt == DT_F32)
+    row_groupnorm_kernel<float><<<M, 256, 0, st>>>(N, gs, eps, A, lda, static_cast<const float*>(gamma),
+                                                   static_cast<const float*>(beta), act,
+                                                   static_cast<float*>(Y), ldy);
+  else
+    row_groupnorm_kernel<__nv_bfloat16><<<M, 256, 0, st>>>(
+        N, gs, eps, A, lda, static_cast<const __nv_bfloat16*>(gamma),
+        static_cast<const __nv_bfloat16*>(beta), act, static_cast<__nv_bfloat16*>(Y), ldy);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_gap_finalize(int Nb, int Cout, int parts, long long hw, const float* stats, float* out,
                                 cudaStream_t st) {
   const long long total = static_cast<long long>(Nb) * Cout;

@@ -54,6 +54,12 @@ struct UmmaParams {
   float* partial;              // row-reduce partial statistics
   float scale;
   int act_rt;                  // activation code, read by the ACT_RUNTIME instantiations
+  // GroupNorm over groups of gn_pieces * 32 consecutive columns in the elementwise epilogue
+  // (0 = off): y = scale * act((z - mu) * rstd * gamma + beta) with mu, rstd per row and group
+  int gn_pieces;
+  float gn_eps;
+  const __nv_bfloat16* gn_gamma;   // [N] or null (1)
+  const __nv_bfloat16* gn_beta;    // [N] or null (0)
   int stats_only;              // softmax first pass without numerators: 1 = (max, sum of exp)
                                // for the log-sum-exp, 2 = maximum only
   int vec_ok;                  // rows of out (and R) are 16-byte aligned (direct path vectors)
@@ -119,6 +125,29 @@ __device__ __forceinline__ void load_bias32(const UmmaParams& p, int n0, float (
 #pragma unroll
     for (int j = 0; j < 32; ++j)
       b[j] = (n0 + j < p.N) ? __bfloat162float(p.bias[n0 + j]) : 0.0f;
+  }
+}
+
+// 32 consecutive values of a bf16 vector of length N as fp32 (`dflt` past N or for a null
+// pointer); 16-byte loads when the vector is 16-byte aligned.
+__device__ __forceinline__ void load_vec32(const __nv_bfloat16* ptr, int N, int n0, float dflt,
+                                           float (&o)[32]) {
+  if (ptr == nullptr) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) o[j] = dflt;
+  } else if ((reinterpret_cast<uintptr_t>(ptr) & 15u) == 0 && n0 + 32 <= N) {
+    const uint4* bp = reinterpret_cast<const uint4*>(ptr + n0);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint4 w = __ldg(bp + q);
+      o[8 * q + 0] = bf16_lo(w.x); o[8 * q + 1] = bf16_hi(w.x);
+      o[8 * q + 2] = bf16_lo(w.y); o[8 * q + 3] = bf16_hi(w.y);
+      o[8 * q + 4] = bf16_lo(w.z); o[8 * q + 5] = bf16_hi(w.z);
+      o[8 * q + 6] = bf16_lo(w.w); o[8 * q + 7] = bf16_hi(w.w);
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) o[j] = (n0 + j < N) ? __bfloat162float(ptr[n0 + j]) : dflt;
   }
 }
 
@@ -349,6 +378,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       if constexpr (EPI == EPI_ELEMENTWISE) {
         __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(p.out);
         if (staged) {
+          [[maybe_unused]] float gn_mu = 0.0f, gn_rstd = 1.0f;
 #pragma unroll 1
           for (int c = 0; c < PIECES; ++c, ++g) {
             const int b = static_cast<int>(g & 1);
@@ -362,6 +392,27 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               for (int q = 0; q < 4; ++q)
                 rv[q] = *reinterpret_cast<const uint4*>(rb + piece_off(row, q));
             }
+            if (p.gn_pieces > 0 && c % p.gn_pieces == 0) {
+              // statistics of the group that starts here: its columns are all in this tile
+              float s1 = 0.0f, s2 = 0.0f;
+#pragma unroll 1
+              for (int q = 0; q < p.gn_pieces; ++q) {
+                uint32_t u[32];
+                tmem_ld_32x32(t_acc + (c + q) * kPieceCols, u);
+                float bq[32];
+                load_bias32(p, n_tile + (c + q) * kPieceCols, bq);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                  const float z = __uint_as_float(u[j]) + bq[j];
+                  s1 += z;
+                  s2 = fmaf(z, z, s2);
+                }
+              }
+              const float inv_n = 1.0f / static_cast<float>(p.gn_pieces * kPieceCols);
+              gn_mu = s1 * inv_n;
+              gn_rstd = rsqrtf(fmaxf(s2 * inv_n - gn_mu * gn_mu, 0.0f) + p.gn_eps);
+            }
             uint32_t v[32];
             tmem_ld_32x32(t_acc + c * kPieceCols, v);
             float bs[32];
@@ -369,9 +420,20 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             tmem_ld_wait();
             if (c == PIECES - 1) release_acc();
             float f[32];
+            if (p.gn_pieces > 0) {
+              float ga[32], be[32];
+              load_vec32(p.gn_gamma, p.N, n_tile + c * kPieceCols, 1.0f, ga);
+              load_vec32(p.gn_beta, p.N, n_tile + c * kPieceCols, 0.0f, be);
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              f[j] = p.scale * act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
+              for (int j = 0; j < 32; ++j) {
+                const float u = (__uint_as_float(v[j]) + bs[j] - gn_mu) * gn_rstd;
+                f[j] = p.scale * act_f<ACT, true>(fmaf(u, ga[j], be[j]), p.act_rt);
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                f[j] = p.scale * act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
+            }
             if (has_r) {
 #pragma unroll
               for (int q = 0; q < 4; ++q) {

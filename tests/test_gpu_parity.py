@@ -488,6 +488,38 @@ def test_row_reductions_reject_bad_arguments(kf):
     assert st == kf.KF_ERR_INVALID_ARG
 
 
+# ------------------------------------------------------------------ GEMM + GroupNorm over column groups
+@pytest.mark.parametrize("dtype,shape,groups", [
+    ("bf16", (300, 1024, 136), 32),      # groups of 32 columns: one piece each, in the epilogue
+    ("bf16", (257, 512, 72), 2),         # groups of 256: a whole tile
+    ("bf16", (1000, 640, 2048), 5),      # groups of 128, CTA pairs, ragged last tile (640 = 2.5 tiles)
+    ("bf16", (130, 192, 64), 3),         # groups of 64
+    ("bf16", (64, 96, 40), 4),           # groups of 24: second-kernel path
+    ("bf16", (64, 1024, 64), 1),         # one group of 1024 (LayerNorm): second-kernel path
+    ("f32", (70, 60, 33), 5),            # fp32 scalar path
+    ("f32", (1024, 1024, 512), 16),      # fp32 GEMM on the tensor cores, then the row kernel
+])
+def test_gemm_groupnorm(kf, dtype, shape, groups):
+    M, N, K = shape
+    d = ki.gemm_inputs("c3", seed=95, M=M, N=N, K=K, dtype=dtype)
+    gamma = ki.store(ki.uniform(95, 7, (N,), 0.5, 1.5), dtype)
+    beta = ki.store(ki.uniform(95, 8, (N,), -1.0, 1.0), dtype)
+    atol, rtol = tol_for(dtype)
+    if dtype == "f32":
+        atol = rtol = 5e-4                 # rsqrt of the group variance amplifies fp32 rounding
+    for post, g_, b_ in (("none", None, None), ("swish", gamma, beta)):
+        Y = kf.gemm_groupnorm(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), groups, 1e-5,
+                              to_dev(g_), to_dev(b_), post)
+        check_status()
+        ref = oracle.gemm_groupnorm(d["X"], d["W"], d["b"], groups, 1e-5, g_, b_, post)
+        assert_close(to_f64(Y), ref, atol, rtol, "gemm groupnorm %s %s g=%d %s" % (dtype, shape, groups, post))
+    # unit moments of every (row, group) of the plain normalisation
+    Y = to_f64(kf.gemm_groupnorm(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), groups, 1e-5))
+    blk = Y.reshape(M, groups, N // groups)
+    assert np.abs(blk.mean(axis=2)).max() < (2e-2 if dtype == "bf16" else 1e-4)
+    assert np.abs(blk.var(axis=2) - 1.0).max() < (5e-2 if dtype == "bf16" else 1e-3)
+
+
 # ------------------------------------------------------------------ convolution + GroupNorm
 def run_conv(kf, d, act="relu", groups=None, gamma=None, beta=None, use_bias=True):
     groups = d["groups"] if groups is None else groups

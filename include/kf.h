@@ -117,8 +117,10 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
  * the whole row, as a LayerNorm does).  bf16 problems whose group size is 32, 64,
  * 128 or 256, with TMA-loadable operands (see kf_gemm_epilogue) and a 16-byte aligned Y with
  * ldy % 8 == 0, run in ONE tensor-core kernel: a tile of 256 columns holds whole groups, so the
- * epilogue takes the statistics from the accumulator and normalises before storing.  Everything
- * else computes Z in fp32 into the workspace (M*N*4 bytes, plus the split operands for large fp32
+ * epilogue takes the statistics from the accumulator and normalises before storing.  Group
+ * sizes that are multiples of 256 take the same GEMM kernel storing Z plus per-tile statistics
+ * (workspace: 8 bytes per row and 256 columns) and a row kernel that normalises in place.
+ * Everything else computes Z in fp32 into the workspace (M*N*4 bytes, plus the split operands for large fp32
  * problems) and normalises with a second kernel. */
 kf_status kf_gemm_groupnorm(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
                             const void* X, int64_t ldx, const void* W, int64_t ldw,

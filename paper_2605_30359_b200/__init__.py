@@ -344,11 +344,11 @@ def gemm_groupnorm(X, W, bias=None, groups=1, eps=1e-5, gamma=None, beta=None, p
     if out is None:
         out = torch.empty((M, N), dtype=X.dtype, device=X.device)
     nb = kf_gemm_groupnorm_workspace_bytes(M, N, K, dt, int(groups))
-    if nb == 0 and dt == KF_BF16:
+    if dt == KF_BF16:
         # the query cannot see pitches and alignment: give the fallback its scratch when needed
         if not (X.stride(0) % 8 == 0 and W.stride(0) % 8 == 0 and out.stride(0) % 8 == 0 and
                 X.data_ptr() % 16 == 0 and W.data_ptr() % 16 == 0 and out.data_ptr() % 16 == 0):
-            nb = M * N * 4
+            nb = max(nb, M * N * 4)
     ws = workspace(nb, X.device)
     st = kf_gemm_groupnorm(M, N, K, dt, _ptr(X), X.stride(0), _ptr(W), W.stride(0), _ptr(bias), int(groups),
                            float(eps), _ptr(gamma), _ptr(beta), ACT[post_act], _ptr(out), out.stride(0),

@@ -547,6 +547,8 @@ size_t kf_gemm_groupnorm_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dty
   if (M < 1 || N < 1 || K < 1 || groups < 1 || N % groups != 0) return 0;
   const int64_t gs = N / groups;
   if (io_dtype == KF_BF16 && K % 8 == 0 && (gs == 32 || gs == 64 || gs == 128 || gs == 256)) return 0;
+  if (io_dtype == KF_BF16 && K % 8 == 0 && gs % 256 == 0)          // per (row, tile) statistics
+    return round256(static_cast<size_t>(M) * ((N + 255) / 256) * 8);
   return rowreduce_simt_ws(M, N) + (use_tf32x3(io_dtype, M, N, K) ? tf32_ws(M, N, K) : 0);
 }
 
@@ -602,6 +604,48 @@ kf_status kf_gemm_groupnorm(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, 
     if (launch_umma_elementwise(bn, post_act, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
       return KF_ERR_CUDA;
     g_launches += 1;
+    return KF_OK;
+  }
+  if (umma_gemm_ok(io_dtype, K, X, ldx, W, ldw) && staged_ok && gs % 256 == 0 && N / 256 <= 4096) {
+    // groups of whole 256-column tiles (a LayerNorm of a wide row, for one): the GEMM kernel
+    // stores z in bf16 and each tile's exact (sum, sum of squares) per row; a second kernel
+    // normalises the rows in place
+    const int bn = 256;
+    const size_t need = round256(static_cast<size_t>(M) * ((N + 255) / 256) * 8);
+    vs = check_workspace(workspace, workspace_bytes, need);
+    if (vs != KF_OK) return vs;
+    const bool pair = use_cta_pairs(M, K);
+    UmmaMaps tm;
+    if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, pair ? bn / 2 : bn))
+      return KF_ERR_CUDA;
+    UmmaParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.act_rt = ACT_NONE;
+    p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+    const int tile_m = pair ? 2 * kBM : kBM;
+    p.tiles_m = static_cast<int>((M + tile_m - 1) / tile_m);
+    p.tiles_n = static_cast<int>((N + bn - 1) / bn);
+    if (static_cast<int64_t>(p.tiles_m) * p.tiles_n > kMaxDim) return KF_ERR_UNSUPPORTED;
+    p.num_tiles = p.tiles_m * p.tiles_n;
+    p.k_blocks = static_cast<int>((K + kBK - 1) / kBK);
+    p.tiles_per_unit = 1;
+    p.bias = static_cast<const __nv_bfloat16*>(bias);
+    p.out = Y; p.ldo = ldy; p.scale = 1.0f;
+    p.vec_ok = 1; p.staged = 1;
+    p.bias_vec = aligned(bias, 16) ? 1 : 0;
+    p.gn_tile_stats = 1;
+    p.partial = static_cast<float*>(workspace);
+    tm.r = tm.a;
+    if (!encode_piece(&tm.y, Y, M, N, ldy)) return KF_ERR_CUDA;
+    p.status = d->status;
+    const int slots = pair ? d->sm_count / 2 : d->sm_count;
+    const int grid = p.num_tiles < slots ? p.num_tiles : slots;
+    if (launch_umma_elementwise(bn, ACT_NONE, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
+      return KF_ERR_CUDA;
+    if (launch_row_groupnorm_apply(static_cast<int>(M), static_cast<int>(N), static_cast<int>(gs), p.tiles_n,
+                                   eps, p.partial, gamma, beta, post_act, Y, ldy, st) != cudaSuccess)
+      return KF_ERR_CUDA;
+    g_launches += 2;
     return KF_OK;
   }
   // scalar path: pre-normalisation values in fp32 (the FMA kernel, or the fp32 tensor-core

@@ -68,6 +68,10 @@ cudaError_t launch_row_groupnorm(int dt, int M, int N, int gs, float eps, const 
                                  const void* gamma, const void* beta, int act, void* Y, long long ldy,
                                  cudaStream_t st);
 
+cudaError_t launch_row_groupnorm_apply(int M, int N, int gs, int tiles_n, float eps, const float* stats,
+                                       const void* gamma, const void* beta, int act, void* Y,
+                                       long long ldy, cudaStream_t st);
+
 // global average pooling: from the convolution's statistics, or from a stored NCHW tensor
 cudaError_t launch_gap_finalize(int Nb, int Cout, int parts, long long hw, const float* stats, float* out,
                                 cudaStream_t st);

@@ -114,6 +114,16 @@ cudaError_t launch_row_groupnorm(int dt, int M, int N, int gs, float eps, const 
   return cudaGetLastError();
 }
 
+cudaError_t launch_row_groupnorm_apply(int M, int N, int gs, int tiles_n, float eps, const float* stats,
+                                       const void* gamma, const void* beta, int act, void* Y,
+                                       long long ldy, cudaStream_t st) {
+  const size_t smem = static_cast<size_t>(N / gs) * sizeof(float2);
+  row_groupnorm_apply_kernel<<<M, 256, smem, st>>>(
+      N, gs, tiles_n, eps, reinterpret_cast<const float2*>(stats), static_cast<const __nv_bfloat16*>(gamma),
+      static_cast<const __nv_bfloat16*>(beta), act, static_cast<__nv_bfloat16*>(Y), ldy);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_gap_finalize(int Nb, int Cout, int parts, long long hw, const float* stats, float* out,
                                 cudaStream_t st) {
   const long long total = static_cast<long long>(Nb) * Cout;

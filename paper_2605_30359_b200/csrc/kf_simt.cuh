@@ -216,6 +216,46 @@ row_groupnorm_kernel(int N, int gs, float eps, const float* __restrict__ A, long
   }
 }
 
+// Second pass of a GroupNorm whose groups span whole 256-column tiles: the first pass left
+// z (rounded to bf16) in Y and per (row, tile) the exact fp32 (sum, sum of squares) of z.  One
+// CTA per row: the group statistics from the tiles' entries (added in increasing order), then
+// the row normalised in place, 16 bytes per thread and step.
+__global__ void __launch_bounds__(256)
+row_groupnorm_apply_kernel(int N, int gs, int tiles_n, float eps, const float2* __restrict__ stats,
+                           const __nv_bfloat16* __restrict__ gamma,
+                           const __nv_bfloat16* __restrict__ beta, int act_code, __nv_bfloat16* Y,
+                           long long ldy) {
+  extern __shared__ float2 mr[];            // [groups] (mu, rstd)
+  const int groups = N / gs, tpg = gs / 256;
+  const float2* part = stats + static_cast<long long>(blockIdx.x) * tiles_n;
+  for (int g = threadIdx.x; g < groups; g += blockDim.x) {
+    float s1 = 0.0f, s2 = 0.0f;
+    for (int t = 0; t < tpg; ++t) { const float2 q = part[g * tpg + t]; s1 += q.x; s2 += q.y; }
+    const float mu = s1 / static_cast<float>(gs);
+    mr[g] = make_float2(mu, rsqrtf(fmaxf(s2 / static_cast<float>(gs) - mu * mu, 0.0f) + eps));
+  }
+  __syncthreads();
+  uint4* row = reinterpret_cast<uint4*>(Y + static_cast<long long>(blockIdx.x) * ldy);
+  for (int i = threadIdx.x; i < N / 8; i += blockDim.x) {
+    const int n0 = i * 8;
+    const float2 st = mr[n0 / gs];
+    uint4 w = row[i];
+    uint32_t* u = reinterpret_cast<uint32_t*>(&w);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + 2 * j;
+      const float g0 = gamma != nullptr ? __bfloat162float(gamma[n]) : 1.0f;
+      const float g1 = gamma != nullptr ? __bfloat162float(gamma[n + 1]) : 1.0f;
+      const float b0 = beta != nullptr ? __bfloat162float(beta[n]) : 0.0f;
+      const float b1 = beta != nullptr ? __bfloat162float(beta[n + 1]) : 0.0f;
+      const float y0 = act_any<true>(act_code, fmaf((bf16_lo(u[j]) - st.x) * st.y, g0, b0));
+      const float y1 = act_any<true>(act_code, fmaf((bf16_hi(u[j]) - st.x) * st.y, g1, b1));
+      u[j] = pack_bf16x2(y0, y1);
+    }
+    row[i] = w;
+  }
+}
+
 // ---------------------------------------------------------------- second passes, tensor path
 // Softmax: the first pass left e[m,n] = exp(a[m,n] - mx_t) in `out` and (mx_t, sum_t) per
 // slice t of 2^bn_shift columns (one first-pass tile) in `partial`.  Row maximum mx = max_t mx_t, denominator

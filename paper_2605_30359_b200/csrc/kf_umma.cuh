@@ -57,6 +57,9 @@ struct UmmaParams {
   // GroupNorm over groups of gn_pieces * 32 consecutive columns in the elementwise epilogue
   // (0 = off): y = scale * act((z - mu) * rstd * gamma + beta) with mu, rstd per row and group
   int gn_pieces;
+  // 1: also write this row's (sum, sum of squares) of z = XW^T + b over the tile's columns to
+  // partial[m * tiles_n + tn] (float2) - the first pass of a GroupNorm whose groups span tiles
+  int gn_tile_stats;
   float gn_eps;
   const __nv_bfloat16* gn_gamma;   // [N] or null (1)
   const __nv_bfloat16* gn_beta;    // [N] or null (0)
@@ -379,6 +382,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(p.out);
         if (staged) {
           [[maybe_unused]] float gn_mu = 0.0f, gn_rstd = 1.0f;
+          float ts1 = 0.0f, ts2 = 0.0f;
 #pragma unroll 1
           for (int c = 0; c < PIECES; ++c, ++g) {
             const int b = static_cast<int>(g & 1);
@@ -431,8 +435,11 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               }
             } else {
 #pragma unroll
-              for (int j = 0; j < 32; ++j)
-                f[j] = p.scale * act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
+              for (int j = 0; j < 32; ++j) {
+                const float z = __uint_as_float(v[j]) + bs[j];
+                if (p.gn_tile_stats) { ts1 += z; ts2 = fmaf(z, z, ts2); }   // columns past N hold 0
+                f[j] = p.scale * act_f<ACT, true>(z, p.act_rt);
+              }
             }
             if (has_r) {
 #pragma unroll
@@ -464,6 +471,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               if (has_r && g + 2 < total_pieces) issue_r(g + 2);
             }
           }
+          if (p.gn_tile_stats && alive && row_ok)
+            reinterpret_cast<float2*>(p.partial)[m * p.tiles_n + tn] = make_float2(ts1, ts2);
         } else {
           // Output (or residual) rows that do not start on 16 bytes: no TMA.  Pieces still go
           // through shared memory so that global accesses run along rows: a warp moves 32 rows,

@@ -494,8 +494,10 @@ def test_row_reductions_reject_bad_arguments(kf):
     ("bf16", (257, 512, 72), 2),         # groups of 256: a whole tile
     ("bf16", (1000, 640, 2048), 5),      # groups of 128, CTA pairs, ragged last tile (640 = 2.5 tiles)
     ("bf16", (130, 192, 64), 3),         # groups of 64
-    ("bf16", (64, 96, 40), 4),           # groups of 24: second-kernel path
-    ("bf16", (64, 1024, 64), 1),         # one group of 1024 (LayerNorm): second-kernel path
+    ("bf16", (64, 96, 40), 4),           # groups of 24: FMA kernel + row kernel
+    ("bf16", (64, 1024, 64), 1),         # one group of 1024 (LayerNorm): tile statistics + row pass
+    ("bf16", (300, 2048, 136), 4),       # groups of 512 = two tiles each, ragged M
+    ("bf16", (512, 1024, 2048), 1),      # the same through the CTA-pair kernel
     ("f32", (70, 60, 33), 5),            # fp32 scalar path
     ("f32", (1024, 1024, 512), 16),      # fp32 GEMM on the tensor cores, then the row kernel
 ])

@@ -648,6 +648,18 @@ kf_status kf_gemm_groupnorm(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, 
     g_launches += 2;
     return KF_OK;
   }
+  if (umma_gemm_ok(io_dtype, K, X, ldx, W, ldw) && bf16_repack_pays(M, N, K)) {
+    // any other group size on a problem worth the tensor cores: z through the fused GEMM chain
+    // into Y (bf16), then the row kernel in place (statistics from the stored z)
+    vs = kf_gemm_epilogue(M, N, K, io_dtype, X, ldx, W, ldw, bias, KF_ACT_NONE, 1.0f, nullptr, 0, Y, ldy,
+                          nullptr, 0, cuda_stream);
+    if (vs != KF_OK) return vs;
+    if (launch_row_groupnorm_inplace(static_cast<int>(M), static_cast<int>(N), static_cast<int>(gs), eps,
+                                     gamma, beta, post_act, Y, ldy, st) != cudaSuccess)
+      return KF_ERR_CUDA;
+    g_launches += 1;
+    return KF_OK;
+  }
   // scalar path: pre-normalisation values in fp32 (the FMA kernel, or the fp32 tensor-core
   // chain for large fp32 problems), then one CTA per row
   const bool tensor32 = use_tf32x3(io_dtype, M, N, K);

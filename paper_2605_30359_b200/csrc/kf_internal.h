@@ -68,6 +68,9 @@ cudaError_t launch_row_groupnorm(int dt, int M, int N, int gs, float eps, const 
                                  const void* gamma, const void* beta, int act, void* Y, long long ldy,
                                  cudaStream_t st);
 
+cudaError_t launch_row_groupnorm_inplace(int M, int N, int gs, float eps, const void* gamma,
+                                         const void* beta, int act, void* Y, long long ldy,
+                                         cudaStream_t st);
 cudaError_t launch_row_groupnorm_apply(int M, int N, int gs, int tiles_n, float eps, const float* stats,
                                        const void* gamma, const void* beta, int act, void* Y,
                                        long long ldy, cudaStream_t st);

@@ -104,13 +104,24 @@ cudaError_t launch_row_groupnorm(int dt, int M, int N, int gs, float eps, const 
                                  const void* gamma, const void* beta, int act, void* Y, long long ldy,
                                  cudaStream_t st) {
   if (dt == DT_F32)
-    row_groupnorm_kernel<float><<<M, 256, 0, st>>>(N, gs, eps, A, lda, static_cast<const float*>(gamma),
-                                                   static_cast<const float*>(beta), act,
-                                                   static_cast<float*>(Y), ldy);
+    row_groupnorm_kernel<float, float><<<M, 256, 0, st>>>(N, gs, eps, A, lda, static_cast<const float*>(gamma),
+                                                          static_cast<const float*>(beta), act,
+                                                          static_cast<float*>(Y), ldy);
   else
-    row_groupnorm_kernel<__nv_bfloat16><<<M, 256, 0, st>>>(
+    row_groupnorm_kernel<__nv_bfloat16, float><<<M, 256, 0, st>>>(
         N, gs, eps, A, lda, static_cast<const __nv_bfloat16*>(gamma),
         static_cast<const __nv_bfloat16*>(beta), act, static_cast<__nv_bfloat16*>(Y), ldy);
+  return cudaGetLastError();
+}
+
+// in place on a bf16 matrix that holds z
+cudaError_t launch_row_groupnorm_inplace(int M, int N, int gs, float eps, const void* gamma,
+                                         const void* beta, int act, void* Y, long long ldy,
+                                         cudaStream_t st) {
+  __nv_bfloat16* y = static_cast<__nv_bfloat16*>(Y);
+  row_groupnorm_kernel<__nv_bfloat16, __nv_bfloat16><<<M, 256, 0, st>>>(
+      N, gs, eps, y, ldy, static_cast<const __nv_bfloat16*>(gamma), static_cast<const __nv_bfloat16*>(beta),
+      act, y, ldy);
   return cudaGetLastError();
 }
 

@@ -187,23 +187,24 @@ row_reduce_kernel(int N, const float* __restrict__ A, long long lda, float* out,
 // GroupNorm over groups of gs consecutive columns of a materialised fp32 matrix A[M,N] (the
 // pre-normalisation values), then the activation: one CTA per row, one warp per group at a
 // time; mean and biased variance in two passes over the group.
-template <typename T>
+// (TA = float: the fp32 matrix from the workspace; TA = T with A == Y: in place on a stored bf16 z.)
+template <typename T, typename TA>
 __global__ void __launch_bounds__(256)
-row_groupnorm_kernel(int N, int gs, float eps, const float* __restrict__ A, long long lda,
+row_groupnorm_kernel(int N, int gs, float eps, const TA* A, long long lda,
                      const T* __restrict__ gamma, const T* __restrict__ beta, int act_code,
-                     T* __restrict__ Y, long long ldy) {
+                     T* Y, long long ldy) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const float* a = A + static_cast<long long>(blockIdx.x) * lda;
+  const TA* a = A + static_cast<long long>(blockIdx.x) * lda;
   T* y = Y + static_cast<long long>(blockIdx.x) * ldy;
   for (int g = warp; g < N / gs; g += 8) {
     const int n0 = g * gs;
     float s = 0.0f;
-    for (int i = lane; i < gs; i += 32) s += a[n0 + i];
+    for (int i = lane; i < gs; i += 32) s += to_f32(a[n0 + i]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     const float mu = s / static_cast<float>(gs);
     float v = 0.0f;
-    for (int i = lane; i < gs; i += 32) { const float d = a[n0 + i] - mu; v = fmaf(d, d, v); }
+    for (int i = lane; i < gs; i += 32) { const float d = to_f32(a[n0 + i]) - mu; v = fmaf(d, d, v); }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     const float rstd = rsqrtf(v / static_cast<float>(gs) + eps);
@@ -211,7 +212,7 @@ row_groupnorm_kernel(int N, int gs, float eps, const float* __restrict__ A, long
       const int n = n0 + i;
       const float ga = gamma != nullptr ? to_f32(gamma[n]) : 1.0f;
       const float be = beta != nullptr ? to_f32(beta[n]) : 0.0f;
-      y[n] = from_f32<T>(act_any<false>(act_code, (a[n] - mu) * rstd * ga + be));
+      y[n] = from_f32<T>(act_any<false>(act_code, (to_f32(a[n]) - mu) * rstd * ga + be));
     }
   }
 }

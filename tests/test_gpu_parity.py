@@ -495,6 +495,7 @@ def test_row_reductions_reject_bad_arguments(kf):
     ("bf16", (1000, 640, 2048), 5),      # groups of 128, CTA pairs, ragged last tile (640 = 2.5 tiles)
     ("bf16", (130, 192, 64), 3),         # groups of 64
     ("bf16", (64, 96, 40), 4),           # groups of 24: FMA kernel + row kernel
+    ("bf16", (512, 960, 264), 8),        # groups of 120 on a larger problem: fused GEMM + in-place row kernel
     ("bf16", (64, 1024, 64), 1),         # one group of 1024 (LayerNorm): tile statistics + row pass
     ("bf16", (300, 2048, 136), 4),       # groups of 512 = two tiles each, ragged M
     ("bf16", (512, 1024, 2048), 1),      # the same through the CTA-pair kernel

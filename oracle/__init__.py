@@ -61,6 +61,8 @@ def _load():
         lib.oracle_conv3x3_act_gap.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, vp]
         lib.oracle_gemm_groupnorm.restype = ci
         lib.oracle_gemm_groupnorm.argtypes = [i64, i64, i64, ci, vp, i64, vp, i64, vp, i64, dbl, vp, vp, ci, vp]
+        lib.oracle_conv3x3_act_pool.restype = ci
+        lib.oracle_conv3x3_act_pool.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, ci, i64, vp]
         _lib = lib
     return _lib
 
@@ -174,3 +176,18 @@ def gemm_groupnorm(X, W, bias=None, groups=1, eps=1e-5, gamma=None, beta=None, p
                                        float(eps), _ptr(gamma), _ptr(beta), ACT[post_act], _ptr(Y))
     assert rc == 0
     return Y
+
+
+POOL = {"max": 0, "avg": 1}
+
+
+def conv3x3_act_pool(x, w, bias=None, act="none", kind="max", pool=2):
+    """max / average pooling (kernel = stride = pool) of act(conv3x3_pad1(x, w) + bias), fp64 NCHW."""
+    x = _c(x); dt = _dt(x); w = _c(w, dt); bias = _c(bias, dt)
+    Nb, Cin, H, Wd = x.shape
+    Cout = w.shape[0]
+    y = np.empty((Nb, Cout, H // pool, Wd // pool), np.float64)
+    rc = _load().oracle_conv3x3_act_pool(Nb, Cin, H, Wd, Cout, dt, _ptr(x), _ptr(w), _ptr(bias), ACT[act],
+                                         POOL[kind], int(pool), _ptr(y))
+    assert rc == 0
+    return y

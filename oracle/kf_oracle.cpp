@@ -353,4 +353,46 @@ int oracle_gemm_groupnorm(int64_t M, int64_t N, int64_t K, int dt, const void* X
   return 0;
 }
 
+// c[n,o,h,w] = bias[o] + sum_{c,r,s} x[n,c,h+r-1,w+s-1] * wt[o,c,r,s]   (as above),  a = act(c)
+// y[n,o,i,j] = max (kind 0) or mean (kind 1) of a over the pool x pool window starting at
+//              (i*pool, j*pool); windows do not overlap, a ragged rim is dropped (torch's
+//              max_pool2d / avg_pool2d with kernel = stride = pool).   y is fp64 [Nb,Cout,H/pool,Wd/pool].
+int oracle_conv3x3_act_pool(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout, int dt,
+                            const void* x, const void* wt, const void* bias, int act, int kind,
+                            int64_t pool, double* y) {
+  if (pool < 1 || (kind != 0 && kind != 1)) return 1;
+  const int64_t Ho = H / pool, Wo = Wd / pool;
+#pragma omp parallel for schedule(dynamic) num_threads(nthreads())
+  for (int64_t n = 0; n < Nb; ++n) {
+    std::vector<double> a((size_t)(H * Wd));
+    for (int64_t o = 0; o < Cout; ++o) {
+      for (int64_t h = 0; h < H; ++h)
+        for (int64_t w = 0; w < Wd; ++w) {
+          double acc = bias ? widen(bias, dt, o) : 0.0;
+          for (int64_t c = 0; c < Cin; ++c)
+            for (int64_t r = 0; r < 3; ++r)
+              for (int64_t q = 0; q < 3; ++q) {
+                const int64_t hh = h + r - 1, ww = w + q - 1;
+                if (hh < 0 || hh >= H || ww < 0 || ww >= Wd) continue;
+                acc += widen(x, dt, ((n * Cin + c) * H + hh) * Wd + ww) *
+                       widen(wt, dt, ((o * Cin + c) * 3 + r) * 3 + q);
+              }
+          a[(size_t)(h * Wd + w)] = act_apply(act, acc);
+        }
+      for (int64_t i = 0; i < Ho; ++i)
+        for (int64_t j = 0; j < Wo; ++j) {
+          double best = -INFINITY, sum = 0.0;
+          for (int64_t r = 0; r < pool; ++r)
+            for (int64_t q = 0; q < pool; ++q) {
+              const double v = a[(size_t)((i * pool + r) * Wd + j * pool + q)];
+              best = std::fmax(best, v);
+              sum += v;
+            }
+          y[((n * Cout + o) * Ho + i) * Wo + j] = kind == 0 ? best : sum / (double)(pool * pool);
+        }
+    }
+  }
+  return 0;
+}
+
 }  // extern "C"

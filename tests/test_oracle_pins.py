@@ -166,6 +166,24 @@ def test_gemm_groupnorm_against_torch_and_moments():
     assert np.abs(np.sort(two, axis=2) - np.array([-1.0, 1.0])).max() < 1e-9
 
 
+def test_conv_act_pool_against_torch_pooling():
+    """Spatial pooling after conv + activation: torch's own max_pool2d / avg_pool2d (fp64) applied
+    to the separately pinned convolution, ragged rims included; pool 1 is the identity."""
+    import torch
+    import torch.nn.functional as F
+    d = ki.conv_inputs(seed=6, Nb=2, Cin=3, H=7, W=9, Cout=4, groups=0, dtype="f32")
+    for act in ("relu", "swish"):
+        full = oracle.conv3x3_gn(d["x"], d["w"], d["bias"], act, 0)
+        t = torch.from_numpy(full)
+        for pool in (1, 2, 3, 4):
+            mx = oracle.conv3x3_act_pool(d["x"], d["w"], d["bias"], act, "max", pool)
+            av = oracle.conv3x3_act_pool(d["x"], d["w"], d["bias"], act, "avg", pool)
+            assert mx.shape == (2, 4, 7 // pool, 9 // pool)
+            assert np.array_equal(mx, F.max_pool2d(t, pool).numpy())
+            assert np.abs(av - F.avg_pool2d(t, pool).numpy()).max() < 1e-15
+        assert np.array_equal(oracle.conv3x3_act_pool(d["x"], d["w"], d["bias"], act, "max", 1), full)
+
+
 def test_paper_constants_and_chain95():
     g = golden()
     assert abs(g["erf_gelu_inner_scale"] - 1.0 / math.sqrt(2.0)) < 1e-15

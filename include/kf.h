@@ -235,6 +235,25 @@ kf_status kf_conv3x3_act_gap(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int
 size_t kf_conv3x3_act_gap_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
                                           kf_dtype io_dtype);
 
+/* 3x3 convolution (pad 1) + bias + activation + max or average pooling (kernel = stride = pool,
+ * no padding; PyTorch's MaxPool2d(pool) / AvgPool2d(pool)): the conv + activation + pooling
+ * chains among the reduction-dominated operator sequences of the paper's Table 2.
+ *   a[n,o,h,w] = act( bias[o] + sum_{c,r,s} x[n,c,h+r-1,w+s-1] * w[o,c,r,s] )
+ *   y[n,o,i,j] = max (pool_kind 0) or mean (pool_kind 1) of a over the pool x pool window at
+ *                (i*pool, j*pool)
+ * x NCHW [Nb,Cin,H,Wd], w OIHW, y NCHW [Nb,Cout,H/pool,Wd/pool] (floor; a ragged rim is dropped),
+ * all dense, of io_dtype; bias may be NULL; pool >= 1.  pool above H or Wd gives an empty y and
+ * the call returns KF_OK without work.  bf16 with pool 2, Wd a multiple of 32 (at most 128) and
+ * even H pools inside the tensor-core convolution's epilogue from the fp32 activations, which are
+ * then never written; every other case writes a (io_dtype) to the workspace with the kernels of
+ * kf_conv3x3_epilogue and pools it with a second kernel.  Other pool_kind: KF_ERR_INVALID_ARG. */
+kf_status kf_conv3x3_act_pool(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                              kf_dtype io_dtype, const void* x, const void* w, const void* bias,
+                              kf_act act, int pool_kind, int pool, void* y,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+size_t kf_conv3x3_act_pool_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                                           kf_dtype io_dtype, int pool);
+
 /* Workspace sizes in bytes for the calls above with the same arguments (0 = none needed).
  * Pure host arithmetic; no CUDA call is made. */
 size_t kf_gemm_epilogue_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype);

@@ -31,6 +31,7 @@ EXPORTS = ["kf_gemm_epilogue", "kf_gemm_rowreduce", "kf_gemm_rowreduce_static",
            "kf_conv3x3_epilogue", "kf_conv3x3_softmax_pool",
            "kf_conv3x3_softmax_pool_workspace_bytes", "kf_selftest_bounded_wait",
            "kf_conv3x3_act_gap", "kf_conv3x3_act_gap_workspace_bytes",
+           "kf_conv3x3_act_pool", "kf_conv3x3_act_pool_workspace_bytes",
            "kf_gemm_groupnorm", "kf_gemm_groupnorm_workspace_bytes",
            "kf_gemm_epilogue_workspace_bytes", "kf_gemm_rowreduce_workspace_bytes",
            "kf_conv3x3_workspace_bytes", "kf_device_status", "kf_launch_count",
@@ -81,6 +82,10 @@ def lib() -> ctypes.CDLL:
     L.kf_conv3x3_act_gap.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp, sz, vp]
     L.kf_conv3x3_act_gap_workspace_bytes.restype = sz
     L.kf_conv3x3_act_gap_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, ci]
+    L.kf_conv3x3_act_pool.restype = ci
+    L.kf_conv3x3_act_pool.argtypes = [i64, i64, i64, i64, i64, ci, vp, vp, vp, ci, ci, ci, vp, vp, sz, vp]
+    L.kf_conv3x3_act_pool_workspace_bytes.restype = sz
+    L.kf_conv3x3_act_pool_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, ci, ci]
     L.kf_selftest_bounded_wait.restype = ci
     L.kf_selftest_bounded_wait.argtypes = [ctypes.c_uint64, ctypes.POINTER(ctypes.c_uint64), vp]
     L.kf_gemm_epilogue_workspace_bytes.restype = sz
@@ -159,6 +164,16 @@ def kf_conv3x3_act_gap(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, out, wor
 
 def kf_conv3x3_act_gap_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype) -> int:
     return lib().kf_conv3x3_act_gap_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype)
+
+
+def kf_conv3x3_act_pool(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, pool_kind, pool, y,
+                        workspace, workspace_bytes, stream) -> int:
+    return lib().kf_conv3x3_act_pool(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, pool_kind,
+                                     pool, y, workspace, workspace_bytes, stream)
+
+
+def kf_conv3x3_act_pool_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype, pool) -> int:
+    return lib().kf_conv3x3_act_pool_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype, pool)
 
 
 def kf_selftest_bounded_wait(limit_ns, stream=None):
@@ -375,6 +390,29 @@ def conv3x3_act_gap(x, w, bias=None, act="none", out=None, stream=None):
                             _ptr(out), _ptr(ws), nb, _stream_ptr(stream))
     if st != KF_OK:
         raise KfError(st, "kf_conv3x3_act_gap")
+    return out
+
+
+POOL = {"max": 0, "avg": 1}
+
+
+def conv3x3_act_pool(x, w, bias=None, act="none", kind="max", pool=2, out=None, stream=None):
+    """out[Nb, Cout, H//pool, W//pool] = max / average pooling of act(conv3x3_pad1(x, w) + bias)."""
+    torch = _torch()
+    _check_cuda(x, w, bias, out)
+    if not (x.is_contiguous() and w.is_contiguous()):
+        raise ValueError("conv3x3_act_pool takes contiguous NCHW / OIHW tensors")
+    Nb, Cin, H, Wd = x.shape
+    Cout = w.shape[0]
+    dt = _kf_dtype(x)
+    if out is None:
+        out = torch.empty((Nb, Cout, H // max(pool, 1), Wd // max(pool, 1)), dtype=x.dtype, device=x.device)
+    nb = kf_conv3x3_act_pool_workspace_bytes(Nb, Cin, H, Wd, Cout, dt, pool)
+    ws = workspace(nb, x.device)
+    st = kf_conv3x3_act_pool(Nb, Cin, H, Wd, Cout, dt, _ptr(x), _ptr(w), _ptr(bias), ACT[act],
+                             POOL[kind], pool, _ptr(out), _ptr(ws), nb, _stream_ptr(stream))
+    if st != KF_OK:
+        raise KfError(st, "kf_conv3x3_act_pool")
     return out
 
 

@@ -176,6 +176,14 @@ bool conv_umma_shape_ok(int dt, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout
   return dt == DT_BF16 && conv_rows_per_tile(H, Wd) > 0;
 }
 int64_t conv_cpad(int64_t Cin) { return (Cin + 63) / 64 * 64; }   // channels of the NHWC copy
+// 2x2 pooling inside the bf16 tensor-core convolution's epilogue: a tile must hold whole pairs of
+// image rows and its 32-pixel pieces whole half-rows (Wd a multiple of 32), H must be even.
+bool conv_pool_fused_ok(int dt, int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout, int pool) {
+  (void)Nb; (void)Cin; (void)Cout;
+  if (dt != DT_BF16 || pool != 2 || !conv_umma_shape_ok(dt, Cin, H, Wd, Cout)) return false;
+  const int rows = conv_rows_per_tile(H, Wd);
+  return Wd % 32 == 0 && Wd <= 256 && rows % 2 == 0 && H % 2 == 0 && getenv("KF_NO_FUSED_POOL") == nullptr;
+}
 // fp32 convolutions large enough for the tensor cores take the 3xTF32 implicit GEMM
 int64_t conv32_cpad(int64_t Cin) { return (Cin + 15) / 16 * 16; }
 bool conv_tf32_ok(int dt, int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout) {
@@ -810,7 +818,7 @@ static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
                               kf_dtype io_dtype, const void* x, const void* w, const void* bias,
                               kf_act act, int groups, float eps, const void* gamma,
                               const void* beta, void* y, void* workspace, size_t workspace_bytes,
-                              void* cuda_stream, float* gap_out) {
+                              void* cuda_stream, float* gap_out, int pool2) {
   if (Nb < 1 || Cin < 1 || H < 1 || Wd < 1 || Cout < 1) return KF_ERR_INVALID_ARG;
   if (Nb > kMaxDim || Cin > kMaxDim || H > kMaxDim || Wd > kMaxDim || Cout > kMaxDim) return KF_ERR_INVALID_ARG;
   if (!valid_dtype(io_dtype) || !valid_act(act)) return KF_ERR_INVALID_ARG;
@@ -926,6 +934,7 @@ static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
     p.rows_per_tile = rows;
     // the output pieces travel by TMA when every image plane starts on 16 bytes
     p.staged = (!gap_in_epilogue && aligned(y, 16) && hw % 8 == 0) ? 1 : 0;
+    if (pool2 != 0) { p.pool2 = pool2; p.staged = 0; p.vec_ok = aligned(y, 16) ? 1 : 0; }
     if (p.staged && !encode_nchw_out(&tm.y, y, Nb, Cout, hw)) return KF_ERR_CUDA;
     const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
     if (launch_umma_conv(bn, act, tm, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
@@ -970,7 +979,42 @@ kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
                               const void* beta, void* y, void* workspace, size_t workspace_bytes,
                               void* cuda_stream) {
   return conv3x3_impl(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, groups, eps, gamma, beta, y,
-                      workspace, workspace_bytes, cuda_stream, nullptr);
+                      workspace, workspace_bytes, cuda_stream, nullptr, 0);
+}
+
+size_t kf_conv3x3_act_pool_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                                           kf_dtype io_dtype, int pool) {
+  if (Nb < 1 || Cin < 1 || H < 1 || Wd < 1 || Cout < 1) return 0;
+  const size_t conv_ws = kf_conv3x3_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype, 0);
+  if (conv_pool_fused_ok(io_dtype, Nb, Cin, H, Wd, Cout, pool)) return conv_ws;
+  return round256(static_cast<size_t>(Nb) * Cout * H * Wd * esize(io_dtype)) + conv_ws;
+}
+
+kf_status kf_conv3x3_act_pool(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
+                              kf_dtype io_dtype, const void* x, const void* w, const void* bias,
+                              kf_act act, int pool_kind, int pool, void* y, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream) {
+  if (Nb < 1 || Cin < 1 || H < 1 || Wd < 1 || Cout < 1) return KF_ERR_INVALID_ARG;
+  if (!valid_dtype(io_dtype) || pool < 1 || (pool_kind != 0 && pool_kind != 1)) return KF_ERR_INVALID_ARG;
+  if (Nb > kMaxDim || Cout > kMaxDim || H > kMaxDim || Wd > kMaxDim) return KF_ERR_INVALID_ARG;
+  if (H / pool == 0 || Wd / pool == 0) return KF_OK;   // empty result: nothing to compute
+  if (y == nullptr || !aligned(y, esize(io_dtype)) || y == x) return KF_ERR_INVALID_ARG;
+  kf_status vs = check_workspace(workspace, workspace_bytes,
+                                 kf_conv3x3_act_pool_workspace_bytes(Nb, Cin, H, Wd, Cout, io_dtype, pool));
+  if (vs != KF_OK) return vs;
+  if (conv_pool_fused_ok(io_dtype, Nb, Cin, H, Wd, Cout, pool))
+    return conv3x3_impl(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, 0, 0.0f, nullptr, nullptr, y,
+                        workspace, workspace_bytes, cuda_stream, nullptr, pool_kind + 1);
+  const size_t a_bytes = round256(static_cast<size_t>(Nb) * Cout * H * Wd * esize(io_dtype));
+  const size_t rest = workspace_bytes - a_bytes;
+  vs = conv3x3_impl(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, 0, 0.0f, nullptr, nullptr, workspace,
+                    rest ? static_cast<uint8_t*>(workspace) + a_bytes : nullptr, rest, cuda_stream, nullptr, 0);
+  if (vs != KF_OK) return vs;
+  if (launch_pool2d(io_dtype, Nb * Cout, static_cast<int>(H), static_cast<int>(Wd), pool, pool_kind, workspace,
+                    y, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return KF_ERR_CUDA;
+  g_launches += 1;
+  return KF_OK;
 }
 
 size_t kf_conv3x3_act_gap_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
@@ -994,11 +1038,11 @@ kf_status kf_conv3x3_act_gap(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int
   if (vs != KF_OK) return vs;
   if (!conv_tf32_ok(io_dtype, Nb, Cin, H, Wd, Cout) && conv_umma_shape_ok(io_dtype, Cin, H, Wd, Cout))
     return conv3x3_impl(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, 0, 0.0f, nullptr, nullptr, nullptr,
-                        workspace, workspace_bytes, cuda_stream, out);
+                        workspace, workspace_bytes, cuda_stream, out, 0);
   const size_t y_bytes = round256(static_cast<size_t>(Nb) * Cout * H * Wd * esize(io_dtype));
   const size_t rest = workspace_bytes - y_bytes;
   return conv3x3_impl(Nb, Cin, H, Wd, Cout, io_dtype, x, w, bias, act, 0, 0.0f, nullptr, nullptr, workspace,
-                      rest ? static_cast<uint8_t*>(workspace) + y_bytes : nullptr, rest, cuda_stream, out);
+                      rest ? static_cast<uint8_t*>(workspace) + y_bytes : nullptr, rest, cuda_stream, out, 0);
 }
 
 }  // extern "C"

@@ -75,6 +75,10 @@ cudaError_t launch_row_groupnorm_apply(int M, int N, int gs, int tiles_n, float 
                                        const void* gamma, const void* beta, int act, void* Y,
                                        long long ldy, cudaStream_t st);
 
+// max / average pooling (kernel = stride = pool) of an NCHW tensor
+cudaError_t launch_pool2d(int dt, long long planes, int H, int Wd, int pool, int kind, const void* in,
+                          void* out, cudaStream_t st);
+
 // global average pooling: from the convolution's statistics, or from a stored NCHW tensor
 cudaError_t launch_gap_finalize(int Nb, int Cout, int parts, long long hw, const float* stats, float* out,
                                 cudaStream_t st);

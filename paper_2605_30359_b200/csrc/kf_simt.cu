@@ -135,6 +135,21 @@ cudaError_t launch_row_groupnorm_apply(int M, int N, int gs, int tiles_n, float 
   return cudaGetLastError();
 }
 
+cudaError_t launch_pool2d(int dt, long long planes, int H, int Wd, int pool, int kind, const void* in,
+                          void* out, cudaStream_t st) {
+  const long long total = planes * (H / pool) * (Wd / pool);
+  if (total == 0) return cudaSuccess;
+  const long long grid = (total + 255) / 256;
+  if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
+  if (dt == DT_F32)
+    pool2d_kernel<float><<<static_cast<unsigned>(grid), 256, 0, st>>>(
+        planes, H, Wd, pool, kind, static_cast<const float*>(in), static_cast<float*>(out));
+  else
+    pool2d_kernel<__nv_bfloat16><<<static_cast<unsigned>(grid), 256, 0, st>>>(
+        planes, H, Wd, pool, kind, static_cast<const __nv_bfloat16*>(in), static_cast<__nv_bfloat16*>(out));
+  return cudaGetLastError();
+}
+
 cudaError_t launch_gap_finalize(int Nb, int Cout, int parts, long long hw, const float* stats, float* out,
                                 cudaStream_t st) {
   const long long total = static_cast<long long>(Nb) * Cout;

@@ -730,6 +730,31 @@ groupnorm_apply_kernel(int Cout, int groups, long long hw, int tiles_per_image, 
   }
 }
 
+// ---------------------------------------------------------------- spatial pooling of an NCHW tensor
+// out[plane, i, j] = max (kind 0) or mean (kind 1) over the pool x pool window at (i*pool, j*pool)
+// of in[plane, :, :]; one thread per output element, consecutive threads along j.
+template <typename T>
+__global__ void __launch_bounds__(256)
+pool2d_kernel(long long planes, int H, int Wd, int pool, int kind, const T* __restrict__ in,
+              T* __restrict__ out) {
+  const int Ho = H / pool, Wo = Wd / pool;
+  const long long total = planes * Ho * Wo;
+  const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (gid >= total) return;
+  const int j = static_cast<int>(gid % Wo);
+  const int i = static_cast<int>((gid / Wo) % Ho);
+  const long long pl = gid / (static_cast<long long>(Wo) * Ho);
+  const T* src = in + (pl * H + static_cast<long long>(i) * pool) * Wd + static_cast<long long>(j) * pool;
+  float best = -INFINITY, sum = 0.0f;
+  for (int r = 0; r < pool; ++r)
+    for (int q = 0; q < pool; ++q) {
+      const float v = to_f32(src[static_cast<long long>(r) * Wd + q]);
+      best = fmaxf(best, v);
+      sum += v;
+    }
+  out[gid] = from_f32<T>(kind == 0 ? best : sum / static_cast<float>(pool * pool));
+}
+
 // ---------------------------------------------------------------- global average pooling
 // From the convolution epilogue's statistics: out[n,c] = (sum over the image's pixel tiles of the
 // per-tile channel sums) / (H*W), tiles added in increasing order.

@@ -78,6 +78,8 @@ struct UmmaParams {
   int tile_px;                 // pixels per tile = UMMA N (a multiple of 32, <= BN): rows_per_tile
                                // whole rows, or one of w_segs equal segments of a row
   int w_segs;                  // 1, or segments per row when Wd > 256 (then rows_per_tile = 1)
+  int pool2;                   // convolution: 0, or 2x2 pooling in the epilogue (1 = max, 2 = mean);
+                               // needs w_segs == 1, Wd % 32 == 0, rows_per_tile and H even
 };
 
 // The it-th tile of scheduling slot `cta` out of `ncta`, or -1 when the slot has no more work.
@@ -693,6 +695,59 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // left out of the statistics and are not stored
         const int px_valid = static_cast<int>(min(static_cast<long long>(p.tile_px), hw - px0));
         float s1 = 0.0f, s2 = 0.0f;
+        if (p.pool2 != 0) {
+          // 2x2 pooling of a = act(z + b): the tile holds whole pairs of image rows, a 32-pixel
+          // piece is a stretch of one row, so the thread combines the pieces at the same place
+          // of an even and the following odd row into 16 pooled pixels (32 contiguous bytes of
+          // the pooled NCHW plane).  The activations themselves are never stored.
+          const int wp = p.Wd / 32;                          // pieces per image row
+          const int Wo = p.Wd / 2;
+          const int h0 = pt * p.rows_per_tile;               // first image row of the tile
+          const int pairs = min(p.rows_per_tile, p.H - h0) / 2;
+          __nv_bfloat16* plane = reinterpret_cast<__nv_bfloat16*>(p.out) +
+                                 (static_cast<long long>(img) * p.N + ch) * (hw / 4) +
+                                 static_cast<long long>(h0 / 2) * Wo;
+#pragma unroll 1
+          for (int c = 0; c < pairs * wp; ++c) {
+            const int pr = c / wp, hh = c - pr * wp;
+            uint32_t v0[32], v1[32];
+            tmem_ld_32x32(t_acc + (2 * pr * wp + hh) * 32, v0);
+            tmem_ld_32x32(t_acc + ((2 * pr + 1) * wp + hh) * 32, v1);
+            tmem_ld_wait();
+            if (c == pairs * wp - 1) release_acc();
+            uint32_t w[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              float o[2];
+#pragma unroll
+              for (int t = 0; t < 2; ++t) {
+                const int i = 4 * j + 2 * t;
+                const float a00 = act_f<ACT, true>(__uint_as_float(v0[i]) + bias_v, p.act_rt);
+                const float a01 = act_f<ACT, true>(__uint_as_float(v0[i + 1]) + bias_v, p.act_rt);
+                const float a10 = act_f<ACT, true>(__uint_as_float(v1[i]) + bias_v, p.act_rt);
+                const float a11 = act_f<ACT, true>(__uint_as_float(v1[i + 1]) + bias_v, p.act_rt);
+                o[t] = p.pool2 == 1 ? fmaxf(fmaxf(a00, a01), fmaxf(a10, a11))
+                                    : 0.25f * ((a00 + a01) + (a10 + a11));
+              }
+              w[j] = pack_bf16x2(o[0], o[1]);
+            }
+            if (ch_ok) {
+              __nv_bfloat16* dst = plane + static_cast<long long>(pr) * Wo + hh * 16;
+              if (p.vec_ok) {
+                *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4*>(dst + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {      // the plane may start on any 2-byte boundary
+                  dst[2 * j] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j] & 0xffffu));
+                  dst[2 * j + 1] = __ushort_as_bfloat16(static_cast<unsigned short>(w[j] >> 16));
+                }
+              }
+            }
+          }
+          if (++a == 2) { a = 0; aph ^= 1u; }
+          continue;
+        }
 #pragma unroll 1
         for (int c = 0; c < pieces; ++c, ++g) {
           uint32_t v[32];

@@ -784,6 +784,68 @@ def test_calls_on_a_side_stream(kf):
     assert_close(to_f64(Y), ref, 2e-2, 2e-2, "side stream")
 
 
+# ------------------------------------------------------------------ conv -> activation -> max / average pool
+@pytest.mark.parametrize("dtype,cfg,pool", [
+    ("bf16", dict(Nb=2, Cin=64, H=8, W=64, Cout=128), 2),     # pooled in the epilogue: 4-row tiles
+    ("bf16", dict(Nb=3, Cin=32, H=14, W=32, Cout=72), 2),     # 8-row tiles, last tile holds 6 rows; ragged channels
+    ("bf16", dict(Nb=2, Cin=16, H=6, W=96, Cout=130), 2),     # 2-row tiles of 192 pixels; second channel tile nearly empty
+    ("bf16", dict(Nb=2, Cin=64, H=4, W=128, Cout=64), 2),     # 2-row tiles of 256 pixels
+    ("bf16", dict(Nb=2, Cin=64, H=4, W=256, Cout=64), 2),     # one row per tile: conv, then the pooling kernel
+    ("bf16", dict(Nb=2, Cin=64, H=9, W=64, Cout=32), 2),      # odd H: last row dropped; two passes
+    ("bf16", dict(Nb=2, Cin=64, H=8, W=64, Cout=32), 3),      # pool 3 with a ragged rim
+    ("bf16", dict(Nb=2, Cin=8, H=7, W=30, Cout=16), 2),       # direct convolution + pooling kernel
+    ("bf16", dict(Nb=1, Cin=8, H=8, W=32, Cout=16), 4),
+    ("f32", dict(Nb=8, Cin=32, H=32, W=32, Cout=64), 2),      # fp32 tensor-core conv + pooling kernel
+    ("f32", dict(Nb=2, Cin=3, H=5, W=7, Cout=6), 2),          # fp32 direct conv
+    ("f32", dict(Nb=2, Cin=3, H=5, W=7, Cout=6), 1),          # pool 1: the activations themselves
+])
+@pytest.mark.parametrize("kind", ["max", "avg"])
+def test_conv_act_pool(kf, dtype, cfg, pool, kind):
+    d = ki.conv_inputs(seed=16, dtype=dtype, groups=0, **cfg)
+    for act in ("relu", "tanh"):          # tanh is not monotone-free of sign: pooling after, not before
+        out = kf.conv3x3_act_pool(to_dev(d["x"]), to_dev(d["w"]), to_dev(d["bias"]), act, kind, pool)
+        check_status()
+        assert tuple(out.shape) == (cfg["Nb"], cfg["Cout"], cfg["H"] // pool, cfg["W"] // pool)
+        ref = oracle.conv3x3_act_pool(d["x"], d["w"], d["bias"], act, kind, pool)
+        atol, rtol = tol_for(dtype)
+        assert_close(to_f64(out), ref, atol, rtol, "conv pool %s %s %s %d %s" % (dtype, cfg, kind, pool, act))
+
+
+def test_conv_act_pool_fused_and_two_pass_agree(kf, monkeypatch):
+    """The pooling in the convolution's epilogue and the two-kernel route see the same fp32
+    activations; the two-kernel route rounds them to bf16 before pooling, so max pooling (which
+    commutes with the monotone rounding) must agree bit for bit."""
+    import torch
+    cfg = dict(Nb=2, Cin=64, H=16, W=64, Cout=96)
+    d = ki.conv_inputs(seed=17, dtype="bf16", groups=0, **cfg)
+    args = (to_dev(d["x"]), to_dev(d["w"]), to_dev(d["bias"]), "swish", "max", 2)
+    assert kf.kf_conv3x3_act_pool_workspace_bytes(2, 64, 16, 64, 96, kf.KF_BF16, 2) == \
+        kf.kf_conv3x3_workspace_bytes(2, 64, 16, 64, 96, kf.KF_BF16, 0)
+    fused = kf.conv3x3_act_pool(*args).clone()
+    monkeypatch.setenv("KF_NO_FUSED_POOL", "1")
+    two = kf.conv3x3_act_pool(*args)
+    torch.cuda.synchronize()
+    assert torch.equal(fused, two)
+    check_status()
+
+
+def test_conv_act_pool_unaligned_output_and_empty(kf):
+    import torch
+    cfg = dict(Nb=1, Cin=16, H=4, W=32, Cout=8)
+    d = ki.conv_inputs(seed=18, dtype="bf16", groups=0, **cfg)
+    buf = torch.zeros(1 + 8 * 2 * 16 + 1, dtype=torch.bfloat16, device="cuda")
+    out = buf[1:-1].view(1, 8, 2, 16)                     # 2-byte aligned only
+    kf.conv3x3_act_pool(to_dev(d["x"]), to_dev(d["w"]), to_dev(d["bias"]), "relu", "avg", 2, out=out)
+    check_status()
+    ref = oracle.conv3x3_act_pool(d["x"], d["w"], d["bias"], "relu", "avg", 2)
+    assert_close(to_f64(out), ref, 2e-2, 2e-2, "unaligned pooled output")
+    assert float(buf[0]) == 0.0 and float(buf[-1]) == 0.0
+    empty = kf.conv3x3_act_pool(to_dev(d["x"]), to_dev(d["w"]), None, "relu", "max", 5)
+    assert tuple(empty.shape) == (1, 8, 0, 6)
+    with pytest.raises(kf.KfError):
+        kf.conv3x3_act_pool(to_dev(d["x"]), to_dev(d["w"]), None, "relu", "max", 0)
+
+
 def test_host_front_end_matches_device_call(kf):
     """gemm_epilogue_host (chunked copies on side streams) gives the same bits as one device call."""
     import torch

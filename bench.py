@@ -436,6 +436,11 @@ SWEEP_CONV = [  # (Nb, Cin, H, W, Cout, groups [GroupNorm] or -pool [softmax + m
 SWEEP_CONV_F32 = [(32, 64, 56, 56, 64, 8), (16, 64, 32, 32, 64, 8)]   # fp32, ReLU + GroupNorm
 SWEEP_GEMM_GN = [(8192, 4096, 4096, 128), (1024, 1024, 1024, 32), (128, 1024, 512, 32)]   # bf16, GroupNorm + swish
 SWEEP_CONV_GAP = [(128, 64, 64, 64, 128), (32, 64, 56, 56, 64)]        # bf16, ReLU + global average pool
+SWEEP_CONV_POOL = [  # bf16 (Nb, Cin, H, W, Cout, act, kind, pool)
+    (128, 64, 64, 64, 128, "relu", "max", 2), (128, 64, 64, 64, 128, "swish", "avg", 2),
+    (32, 128, 32, 32, 128, "relu", "max", 2), (32, 64, 56, 56, 64, "relu", "max", 2),
+    (16, 64, 128, 128, 64, "relu", "avg", 4),
+]
 SWEEP_ROWRED_F32 = [(2048, 4096, 1024, "none", "softmax"), (4096, 1024, 1024, "sigmoid", "sum")]
 
 
@@ -541,6 +546,17 @@ def run_sweep(kf, device):
         record("conv-centered", "bf16 conv %dx%dx%dx%d->%d relu global-avg-pool" % (Nb, Cin, H, Wd, Cout),
                lambda x=x, w=w, b=b, out=out: kf.conv3x3_act_gap(x, w, b, "relu", out=out),
                lambda x=x, w=w, b=b: torch.relu(F.conv2d(x, w, b, padding=1)).mean(dim=(2, 3)),
+               2.0 * Nb * H * Wd * Cout * Cin * 9)
+        del x, w, b, out
+    for Nb, Cin, H, Wd, Cout, act, kind, pool in SWEEP_CONV_POOL:
+        dt = torch.bfloat16
+        x, w, b = rnd((Nb, Cin, H, Wd), dt), rnd((Cout, Cin, 3, 3), dt, (9 * Cin) ** -0.5), rnd((Cout,), dt, 0.1)
+        out = torch.empty((Nb, Cout, H // pool, Wd // pool), dtype=dt, device=device)
+        ta, tp = _torch_act(act), (F.max_pool2d if kind == "max" else F.avg_pool2d)
+        record("conv-centered", "bf16 conv %dx%dx%dx%d->%d %s %s-pool%d" % (Nb, Cin, H, Wd, Cout, act, kind, pool),
+               lambda x=x, w=w, b=b, out=out, act=act, kind=kind, pool=pool:
+               kf.conv3x3_act_pool(x, w, b, act, kind, pool, out=out),
+               lambda x=x, w=w, b=b, ta=ta, tp=tp, pool=pool: tp(ta(F.conv2d(x, w, b, padding=1)), pool),
                2.0 * Nb * H * Wd * Cout * Cin * 9)
         del x, w, b, out
     sp = np.array([r["speedup"] for r in rows])

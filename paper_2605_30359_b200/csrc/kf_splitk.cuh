@@ -94,7 +94,9 @@ umma_splitk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(recv_bar + 1);
   volatile uint32_t* abort_flag = tmem_holder + 1;
 
-  const int warp = threadIdx.x >> 5;
+  // warp index from a shuffle: provably warp-uniform, so the loops below keep their TMA / MMA
+  // operands in uniform registers
+  const int warp = __shfl_sync(0xffffffffu, static_cast<int>(threadIdx.x >> 5), 0);
   const int lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -114,38 +116,41 @@ umma_splitk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
 
   bool have_acc = false;       // epilogue threads: this CTA's accumulator is complete
   if (warp == 0) {
-    if (lane == 0) {
-      int s = 0; uint32_t ph = 0;
-      for (int kb = kb0; kb < kb1; ++kb) {
-        if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_PRODUCER)) break;
-        uint8_t* sa = ring + s * C::kStage;
+    // every lane waits (warp-uniform loop), one elected lane issues
+    int s = 0; uint32_t ph = 0;
+    for (int kb = kb0; kb < kb1; ++kb) {
+      bool ok = mbar_wait(&empty[s], ph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_PRODUCER);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      uint8_t* sa = ring + s * C::kStage;
+      if (elect_one()) {
         mbar_expect_tx(&full[s], C::kStage);
         tma_load_2d(sa, &tmA, &full[s], kb * kBK, tm * kBM);
         tma_load_2d(sa + kBM * kBK * 2, &tmB, &full[s], kb * kBK, tn * BN);
-        if (++s == kStages) { s = 0; ph ^= 1u; }
       }
+      if (++s == kStages) { s = 0; ph ^= 1u; }
     }
     __syncwarp();
   } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16_f32(kBM, BN);
-      int s = 0; uint32_t ph = 0;
-      bool ok = true;
-      for (int kb = kb0; kb < kb1; ++kb) {
-        ok = mbar_wait(&full[s], ph, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
-        if (!ok) break;
-        tc_fence_after_sync();
-        const uint32_t sa = smem_u32(ring + s * C::kStage);
-        const uint64_t adesc = smem_desc_kmajor_sw128(sa);
-        const uint64_t bdesc = smem_desc_kmajor_sw128(sa + kBM * kBK * 2);
+    constexpr uint32_t idesc = umma_idesc_bf16_f32(kBM, BN);
+    int s = 0; uint32_t ph = 0;
+    bool ok = true;
+    for (int kb = kb0; kb < kb1; ++kb) {
+      ok = mbar_wait(&full[s], ph, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t sa = smem_u32(ring + s * C::kStage);
+      const uint64_t adesc = smem_desc_kmajor_sw128(sa);
+      const uint64_t bdesc = smem_desc_kmajor_sw128(sa + kBM * kBK * 2);
+      if (elect_one()) {
 #pragma unroll
         for (int k = 0; k < kBK / kUmmaK; ++k)
           umma_f16_ss(tmem_base, adesc + 2u * k, bdesc + 2u * k, idesc, (kb > kb0 || k != 0) ? 1u : 0u);
         umma_commit(&empty[s]);
-        if (++s == kStages) { s = 0; ph ^= 1u; }
       }
-      if (ok) umma_commit(tmem_full);
+      if (++s == kStages) { s = 0; ph ^= 1u; }
     }
+    if (ok && elect_one()) umma_commit(tmem_full);
     __syncwarp();
   } else {
     bool ok = true;

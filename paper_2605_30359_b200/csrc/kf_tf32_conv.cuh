@@ -69,7 +69,9 @@ tf32x3_conv_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_consta
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tmem_empty + 2);
   volatile uint32_t* abort_flag = tmem_holder + 1;
 
-  const int warp = threadIdx.x >> 5;
+  // warp index from a shuffle: provably warp-uniform, so the loops below keep their TMA / MMA
+  // operands in uniform registers
+  const int warp = __shfl_sync(0xffffffffu, static_cast<int>(threadIdx.x >> 5), 0);
   const int lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -90,7 +92,8 @@ tf32x3_conv_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_consta
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    // every lane waits (warp-uniform loop), one elected lane issues
+    {
       int s = 0; uint32_t ph = 0;
       bool ok = true;
       for (int tile = cta; tile < p.num_tiles && ok; tile += ncta) {
@@ -101,16 +104,19 @@ tf32x3_conv_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_consta
         const int x0 = (pt % p.w_segs) * (p.Wd / p.w_segs);
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           ok = mbar_wait(&empty[s], ph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_PRODUCER);
+          ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           const int tap = kb / p.kb_per_tap, cb = kb % p.kb_per_tap;
           const int r = tap / 3, sx = tap % 3;
           uint8_t* st = ring + s * C::kStage;
-          mbar_expect_tx(&full[s], 2 * C::kTileA + 2 * b_bytes);
-          tma_load_2d(st, &tmAh, &full[s], cb * kTfBK, tap * p.Cout + tm * kBM);
-          tma_load_2d(st + C::kTileA, &tmAl, &full[s], cb * kTfBK, tap * p.Cout + tm * kBM);
-          tma_load_4d(st + 2 * C::kTileA, &tmBh, &full[s], cb * kTfBK, x0 + sx - 1, h0 + r - 1, img);
-          tma_load_4d(st + 2 * C::kTileA + C::kTileB, &tmBl, &full[s], cb * kTfBK, x0 + sx - 1,
-                      h0 + r - 1, img);
+          if (elect_one()) {
+            mbar_expect_tx(&full[s], 2 * C::kTileA + 2 * b_bytes);
+            tma_load_2d(st, &tmAh, &full[s], cb * kTfBK, tap * p.Cout + tm * kBM);
+            tma_load_2d(st + C::kTileA, &tmAl, &full[s], cb * kTfBK, tap * p.Cout + tm * kBM);
+            tma_load_4d(st + 2 * C::kTileA, &tmBh, &full[s], cb * kTfBK, x0 + sx - 1, h0 + r - 1, img);
+            tma_load_4d(st + 2 * C::kTileA + C::kTileB, &tmBl, &full[s], cb * kTfBK, x0 + sx - 1,
+                        h0 + r - 1, img);
+          }
           if (++s == kStages) { s = 0; ph ^= 1u; }
         }
       }
@@ -118,7 +124,7 @@ tf32x3_conv_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_consta
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    {
       const uint32_t idesc = umma_idesc_tf32_f32(kBM, static_cast<uint32_t>(p.tile_px));
       int s = 0; uint32_t ph = 0; uint32_t cph = 0;
       bool ok = true;
@@ -127,10 +133,12 @@ tf32x3_conv_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_consta
           const bool chunk_start = kb % kTfChunk == 0;
           if (chunk_start) {
             ok = mbar_wait(&tmem_empty[0], cph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
+            ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after_sync();
           }
           ok = mbar_wait(&full[s], ph, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
+          ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after_sync();
           const uint32_t st = smem_u32(ring + s * C::kStage);
@@ -138,18 +146,19 @@ tf32x3_conv_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_consta
           const uint64_t al = smem_desc_kmajor_sw64(st + C::kTileA);
           const uint64_t bh = smem_desc_kmajor_sw64(st + 2 * C::kTileA);
           const uint64_t bl = smem_desc_kmajor_sw64(st + 2 * C::kTileA + C::kTileB);
+          const bool chunk_end = kb % kTfChunk == kTfChunk - 1 || kb == p.k_blocks - 1;
+          if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < kTfBK / kTfUmmaK; ++k) {
-            umma_tf32_ss(tmem_base, ah + 2u * k, bl + 2u * k, idesc, (chunk_start && k == 0) ? 0u : 1u);
-            umma_tf32_ss(tmem_base, al + 2u * k, bh + 2u * k, idesc, 1u);
-            umma_tf32_ss(tmem_base, ah + 2u * k, bh + 2u * k, idesc, 1u);
+            for (int k = 0; k < kTfBK / kTfUmmaK; ++k) {
+              umma_tf32_ss(tmem_base, ah + 2u * k, bl + 2u * k, idesc, (chunk_start && k == 0) ? 0u : 1u);
+              umma_tf32_ss(tmem_base, al + 2u * k, bh + 2u * k, idesc, 1u);
+              umma_tf32_ss(tmem_base, ah + 2u * k, bh + 2u * k, idesc, 1u);
+            }
+            umma_commit(&empty[s]);
+            if (chunk_end) umma_commit(&tmem_full[0]);
           }
-          umma_commit(&empty[s]);
           if (++s == kStages) { s = 0; ph ^= 1u; }
-          if (kb % kTfChunk == kTfChunk - 1 || kb == p.k_blocks - 1) {
-            umma_commit(&tmem_full[0]);
-            cph ^= 1u;
-          }
+          if (chunk_end) cph ^= 1u;
         }
       }
     }

@@ -109,6 +109,10 @@ bool encode_nhwc_f32(CUtensorMap* tm, const void* base, int64_t Nb, int64_t H, i
 bool encode_piece(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld) {
   return encode_2d(tm, base, rows, cols, ld, kBM, kPieceCols, CU_TENSOR_MAP_SWIZZLE_64B);
 }
+// the elementwise epilogue moves a piece as four slabs of 32 rows, one per warp
+bool encode_warp_piece(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld) {
+  return encode_2d(tm, base, rows, cols, ld, 32, kPieceCols, CU_TENSOR_MAP_SWIZZLE_64B);
+}
 
 // NHWC bf16 activations [Nb,H,W,C] -> boxes of 64 channels x box_w pixels x rows image rows.
 bool encode_nhwc(CUtensorMap* tm, const void* base, int64_t Nb, int64_t H, int64_t Wd, int64_t C,
@@ -292,6 +296,12 @@ size_t tf32_ws(int64_t M, int64_t N, int64_t K) {
          2 * round256(static_cast<size_t>(N) * tf32_kp(K) * 4);
 }
 
+// Tuning thresholds can be overridden from the environment (measurement aid).
+int env_int(const char* name, int dflt) {
+  const char* v = getenv(name);
+  return (v != nullptr && *v != '\0') ? atoi(v) : dflt;
+}
+
 // Cluster size of the split-K kernel, or 0.  Measured on B200: a narrow-tile CTA spends about
 // 0.28 us per K block whatever the tile width, the cluster exchange costs about 4 us, so
 // splitting pays from about 24 K blocks; clusters of 8 schedule well only while there are few
@@ -302,14 +312,14 @@ int pick_split_k(int64_t M, int64_t N, int64_t K, int sm_count, int* bn_out) {
   const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + bn - 1) / bn);
   const int64_t kb = (K + kBK - 1) / kBK;
   *bn_out = bn;
-  if (kb < 24) return 0;
+  if (kb < env_int("KF_SPLITK_MIN_KB", 24)) return 0;
   if (bn == 256 && kb >= 32 && tiles * 8 <= 64) return 8;
   if (tiles * 4 <= sm_count - sm_count % 4) return 4;
   return 0;
 }
 
 bool use_cta_pairs(int64_t M, int64_t K) {
-  return M > 256 && K >= 2048 && getenv("KF_NO_PAIR") == nullptr;
+  return M > 256 && K >= env_int("KF_PAIR_MIN_K", 2048) && getenv("KF_NO_PAIR") == nullptr;
 }
 size_t rowreduce_simt_ws(int64_t M, int64_t N) { return round256(static_cast<size_t>(M) * N * 4); }
 
@@ -532,8 +542,8 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
     p.staged = p.vec_ok;
     tm.r = tm.a; tm.y = tm.a;
     if (p.staged) {
-      if (!encode_piece(&tm.y, Y, M, N, ldy)) return KF_ERR_CUDA;
-      if (residual != nullptr && !encode_piece(&tm.r, residual, M, N, ldr)) return KF_ERR_CUDA;
+      if (!encode_warp_piece(&tm.y, Y, M, N, ldy)) return KF_ERR_CUDA;
+      if (residual != nullptr && !encode_warp_piece(&tm.r, residual, M, N, ldr)) return KF_ERR_CUDA;
     }
     p.status = d->status;
     const int slots = pair ? d->sm_count / 2 : d->sm_count;       // CTAs, or CTA pairs
@@ -554,9 +564,9 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
 size_t kf_gemm_groupnorm_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, int groups) {
   if (M < 1 || N < 1 || K < 1 || groups < 1 || N % groups != 0) return 0;
   const int64_t gs = N / groups;
-  if (io_dtype == KF_BF16 && K % 8 == 0 && (gs == 32 || gs == 64 || gs == 128 || gs == 256)) return 0;
-  if (io_dtype == KF_BF16 && K % 8 == 0 && gs % 256 == 0)          // per (row, tile) statistics
-    return round256(static_cast<size_t>(M) * ((N + 255) / 256) * 8);
+  if (io_dtype == KF_BF16 && K % 8 == 0 && (gs == 32 || gs == 64 || gs == 128)) return 0;
+  if (io_dtype == KF_BF16 && K % 8 == 0 && gs % 256 == 0)          // per (row, half tile) statistics
+    return round256(static_cast<size_t>(M) * ((N + 255) / 256) * 16);
   return rowreduce_simt_ws(M, N) + (use_tf32x3(io_dtype, M, N, K) ? tf32_ws(M, N, K) : 0);
 }
 
@@ -576,11 +586,11 @@ kf_status kf_gemm_groupnorm(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, 
   const int64_t gs = N / groups;
   const bool staged_ok = ldy % 8 == 0 && aligned(Y, 16);
   if (umma_gemm_ok(io_dtype, K, X, ldx, W, ldw) && staged_ok &&
-      (gs == 32 || gs == 64 || gs == 128 || gs == 256)) {
-    // whole groups lie inside every tile: statistics and normalisation in the epilogue
-    // tile width as for the plain chain, but never narrower than a group
+      (gs == 32 || gs == 64 || gs == 128)) {
+    // whole groups lie inside the half tile of one epilogue group: statistics and normalisation
+    // in the epilogue; tile width as for the plain chain, but never narrower than two groups
     int bn = pick_tile_n(M, N, d->sm_count);
-    if (bn < gs) bn = static_cast<int>(gs);
+    if (bn < 2 * gs) bn = static_cast<int>(2 * gs);
     const bool pair = bn == 256 && use_cta_pairs(M, K);
     UmmaMaps tm;
     if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, pair ? bn / 2 : bn))
@@ -605,7 +615,7 @@ kf_status kf_gemm_groupnorm(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, 
     p.gn_gamma = static_cast<const __nv_bfloat16*>(gamma);
     p.gn_beta = static_cast<const __nv_bfloat16*>(beta);
     tm.r = tm.a;
-    if (!encode_piece(&tm.y, Y, M, N, ldy)) return KF_ERR_CUDA;
+    if (!encode_warp_piece(&tm.y, Y, M, N, ldy)) return KF_ERR_CUDA;
     p.status = d->status;
     const int slots = pair ? d->sm_count / 2 : d->sm_count;
     const int grid = p.num_tiles < slots ? p.num_tiles : slots;
@@ -619,7 +629,7 @@ kf_status kf_gemm_groupnorm(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, 
     // stores z in bf16 and each tile's exact (sum, sum of squares) per row; a second kernel
     // normalises the rows in place
     const int bn = 256;
-    const size_t need = round256(static_cast<size_t>(M) * ((N + 255) / 256) * 8);
+    const size_t need = round256(static_cast<size_t>(M) * ((N + 255) / 256) * 16);
     vs = check_workspace(workspace, workspace_bytes, need);
     if (vs != KF_OK) return vs;
     const bool pair = use_cta_pairs(M, K);
@@ -644,13 +654,14 @@ kf_status kf_gemm_groupnorm(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, 
     p.gn_tile_stats = 1;
     p.partial = static_cast<float*>(workspace);
     tm.r = tm.a;
-    if (!encode_piece(&tm.y, Y, M, N, ldy)) return KF_ERR_CUDA;
+    if (!encode_warp_piece(&tm.y, Y, M, N, ldy)) return KF_ERR_CUDA;
     p.status = d->status;
     const int slots = pair ? d->sm_count / 2 : d->sm_count;
     const int grid = p.num_tiles < slots ? p.num_tiles : slots;
     if (launch_umma_elementwise(bn, ACT_NONE, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
       return KF_ERR_CUDA;
-    if (launch_row_groupnorm_apply(static_cast<int>(M), static_cast<int>(N), static_cast<int>(gs), p.tiles_n,
+    // the single-CTA kernel's two epilogue groups leave one entry per half tile
+    if (launch_row_groupnorm_apply(static_cast<int>(M), static_cast<int>(N), static_cast<int>(gs), (pair ? 1 : 2) * p.tiles_n,
                                    eps, p.partial, gamma, beta, post_act, Y, ldy, st) != cudaSuccess)
       return KF_ERR_CUDA;
     g_launches += 2;

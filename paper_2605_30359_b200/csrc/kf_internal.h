@@ -148,7 +148,7 @@ inline cudaError_t launch_umma_instance(const UmmaMaps& tm, const UmmaParams& p,
   if constexpr (CTA2) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * grid, 1, 1);
-    cfg.blockDim = dim3(num_threads(EPI), 1, 1);
+    cfg.blockDim = dim3(num_threads(EPI, BN, CTA2), 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -160,7 +160,7 @@ inline cudaError_t launch_umma_instance(const UmmaMaps& tm, const UmmaParams& p,
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kern, tm.a, tm.b, tm.r, tm.y, p);
   } else {
-    kern<<<grid, num_threads(EPI), smem, st>>>(tm.a, tm.b, tm.r, tm.y, p);
+    kern<<<grid, num_threads(EPI, BN, CTA2), smem, st>>>(tm.a, tm.b, tm.r, tm.y, p);
     return cudaGetLastError();
   }
 }

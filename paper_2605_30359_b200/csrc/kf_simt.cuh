@@ -218,16 +218,17 @@ row_groupnorm_kernel(int N, int gs, float eps, const TA* A, long long lda,
 }
 
 // Second pass of a GroupNorm whose groups span whole 256-column tiles: the first pass left
-// z (rounded to bf16) in Y and per (row, tile) the exact fp32 (sum, sum of squares) of z.  One
-// CTA per row: the group statistics from the tiles' entries (added in increasing order), then
-// the row normalised in place, 16 bytes per thread and step.
+// z (rounded to bf16) in Y and per (row, slice) the exact fp32 (sum, sum of squares) of z, a
+// slice being a 256-column tile or half of one; `tiles_n` counts the slices of a row.  One CTA per row: the group
+// statistics from the entries (added in increasing order), then the row normalised in place,
+// 16 bytes per thread and step.
 __global__ void __launch_bounds__(256)
 row_groupnorm_apply_kernel(int N, int gs, int tiles_n, float eps, const float2* __restrict__ stats,
                            const __nv_bfloat16* __restrict__ gamma,
                            const __nv_bfloat16* __restrict__ beta, int act_code, __nv_bfloat16* Y,
                            long long ldy) {
   extern __shared__ float2 mr[];            // [groups] (mu, rstd)
-  const int groups = N / gs, tpg = gs / 256;
+  const int groups = N / gs, tpg = static_cast<int>(static_cast<long long>(gs) * tiles_n / N);   // entries per group
   const float2* part = stats + static_cast<long long>(blockIdx.x) * tiles_n;
   for (int g = threadIdx.x; g < groups; g += blockDim.x) {
     float s1 = 0.0f, s2 = 0.0f;

@@ -37,8 +37,16 @@ constexpr int kNumThreads = 192;  // 6 warps: producer, UMMA issuer, epilogue
 // one warp per scheduler it is latency-bound, so it runs as TWO groups of four warps, each
 // owning half of the tile's columns as a slice of its own: own statistics, own staging, own
 // named barriers, own TMA stores.  The second pass combines slices, so the groups never talk.
-constexpr int epi_groups(int epi) { return epi == 1 /* EPI_SOFTMAX */ ? 2 : 1; }
-constexpr int num_threads(int epi) { return 64 + kEpiThreads * epi_groups(epi); }
+// Epilogue groups of four warps, each owning BN / groups columns of every tile: two for the softmax
+// first pass and for the elementwise chain (one warp per scheduler left the epilogue latency-bound:
+// a 128x256 tile took 7 us to drain, more than its MMAs take up to K = 1536), one where a group
+// would be narrower than a 32-column piece and for the other epilogues.
+// The CTA-pair form (large K only: its epilogue hides behind the MMAs anyway, and the extra warps
+// cost it 2 %) keeps one group.
+constexpr int epi_groups(int epi, int bn, bool cta2) {
+  return epi == 1 /* EPI_SOFTMAX */ || (epi == 0 /* EPI_ELEMENTWISE */ && bn >= 64 && !cta2) ? 2 : 1;
+}
+constexpr int num_threads(int epi, int bn, bool cta2) { return 64 + kEpiThreads * epi_groups(epi, bn, cta2); }
 constexpr int kPieceCols = 32;    // epilogue piece: 128 rows x 32 columns
 constexpr int kPieceBytes = kBM * kPieceCols * 2;   // 8 KB of bf16
 constexpr int kMaxDynSmem = 232448;                 // 227 KB opt-in limit per CTA
@@ -104,10 +112,12 @@ struct UmmaCfg {
       EPI == EPI_ELEMENTWISE || EPI == EPI_SOFTMAX ? 4 * kPieceBytes
                                                     : (EPI == EPI_ROWSUM ? 0 : 2 * kPieceBytes);
   static constexpr int kBarBytes = 256;
-  static constexpr int kFit = (kMaxDynSmem - 1024 - kStaging - kBarBytes) / kStage;
+  // elementwise: the tile's BN bias values as fp32, staged once per tile
+  static constexpr int kBiasBytes = EPI == EPI_ELEMENTWISE ? BN * 4 : 0;
+  static constexpr int kFit = (kMaxDynSmem - 1024 - kStaging - kBarBytes - kBiasBytes) / kStage;
   static constexpr int kStages = kFit > 8 ? 8 : kFit;
   static constexpr int kRing = kStage * kStages;
-  static constexpr int kTotal = 1024 /*alignment slack*/ + kRing + kStaging + kBarBytes;
+  static constexpr int kTotal = 1024 /*alignment slack*/ + kRing + kStaging + kBarBytes + kBiasBytes;
 };
 
 // 32 consecutive bias values as fp32 (zeros past N or without a bias).  All lanes read the same
@@ -163,8 +173,17 @@ __device__ __forceinline__ uint32_t piece_off(int r, int j) {
   return static_cast<uint32_t>(r * 64 + ((j ^ ((r >> 1) & 3)) << 4));
 }
 
+// 32 consecutive staged bias values (shared memory, same address in every lane: broadcast).
+__device__ __forceinline__ void load_sbias32(const float* sb, float (&b)[32]) {
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    const float4 t = *reinterpret_cast<const float4*>(sb + 4 * q);
+    b[4 * q + 0] = t.x; b[4 * q + 1] = t.y; b[4 * q + 2] = t.z; b[4 * q + 3] = t.w;
+  }
+}
+
 template <int BN, int EPI, int ACT, typename OutT, bool CTA2>
-__global__ void __launch_bounds__(num_threads(EPI), 1)
+__global__ void __launch_bounds__(num_threads(EPI, BN, CTA2), 1)
 umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmY,
                   const UmmaParams p) {
@@ -188,7 +207,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   uint64_t* tmem_full = empty + kStages;
   uint64_t* tmem_empty = tmem_full + 2;
   uint64_t* r_full = tmem_empty + 2;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(r_full + 2);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(r_full + 8);   // r_full: [epilogue warp][2]
   volatile uint32_t* abort_flag = tmem_holder + 1;
 
   // The warp index comes out of a shuffle so that the compiler knows it is the same in every
@@ -204,8 +223,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     for (int a = 0; a < 2; ++a) {
       mbar_init(&tmem_full[a], 1);
-      mbar_init(&tmem_empty[a], (kEpiThreads / 32) * epi_groups(EPI) * (CTA2 ? 2 : 1));
-      mbar_init(&r_full[a], 1);
+      mbar_init(&tmem_empty[a], (kEpiThreads / 32) * epi_groups(EPI, BN, CTA2) * (CTA2 ? 2 : 1));
+      for (int w = 0; w < 4; ++w) mbar_init(&r_full[2 * w + a], 1);   // one per epilogue warp
     }
     *abort_flag = 0;
     mbar_init_fence();
@@ -327,7 +346,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     __syncwarp();
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5)
-    constexpr int kGroups = epi_groups(EPI);
+    constexpr int kGroups = epi_groups(EPI, BN, CTA2);
+    constexpr int NB = 2 / kGroups;            // elementwise: staging buffers per group (4 pieces in all)
     constexpr int kGroupCols = BN / kGroups;   // columns of the tile one epilogue group owns
     constexpr int PIECES = kGroupCols / kPieceCols;
     const int grp = kGroups > 1 ? (warp - 2) >> 2 : 0;
@@ -336,10 +356,14 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const int row = quad * 32 + lane;          // row of the tile = TMEM lane
     const int et = threadIdx.x - 64 - grp * kEpiThreads;   // 0..127 inside the group
     const bool leader = et == 0;               // issues the group's TMA loads and stores
+    [[maybe_unused]] const bool lead_warp = warp == 2 + 4 * grp;   // its warp (a warp-uniform predicate)
     const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
     [[maybe_unused]] uint8_t* ybuf = stg + grp * 2 * kPieceBytes;   // [2][kPieceBytes] output pieces
-    [[maybe_unused]] uint8_t* rbuf = stg + 2 * kPieceBytes;   // [2][kPieceBytes] residual pieces
+    // elementwise: per group NB output pieces, then NB residual pieces (each warp owns a 2 KB slab of each)
+    [[maybe_unused]] uint8_t* rbuf = ybuf + NB * kPieceBytes;
+    [[maybe_unused]] uint64_t* my_r_full = &r_full[(warp - 2) * NB];   // [NB]
     const bool staged = p.staged != 0;
+    [[maybe_unused]] float* sbias = reinterpret_cast<float*>(stg + C::kStaging + C::kBarBytes) + grp * kGroupCols;   // the group's [kGroupCols] of [BN]
     [[maybe_unused]] const bool has_r = EPI == EPI_ELEMENTWISE && p.R != nullptr;
     const int num_units = p.num_tiles / p.tiles_per_unit;
     const int my_tiles = cta < num_units ? (num_units - cta + ncta - 1) / ncta * p.tiles_per_unit : 0;
@@ -351,15 +375,19 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     [[maybe_unused]] auto issue_r = [&](long long gi) {
       const int ti = static_cast<int>(gi / PIECES), c = static_cast<int>(gi % PIECES);
       const int tile = sched_tile(p, cta, ncta, ti);
-      const int b = static_cast<int>(gi & 1);
-      mbar_expect_tx(&r_full[b], kPieceBytes);
-      tma_load_2d(rbuf + b * kPieceBytes, &tmR, &r_full[b],
-                  (tile % p.tiles_n) * BN + c * kPieceCols, (tile / p.tiles_n) * kTileM + row0);
+      const int b = static_cast<int>(gi % NB);
+      // this warp's 32 rows of the group's piece (2 KB of the 8 KB buffer)
+      mbar_expect_tx(&my_r_full[b], kPieceBytes / 4);
+      tma_load_2d(rbuf + b * kPieceBytes + quad * (kPieceBytes / 4), &tmR, &my_r_full[b],
+                  (tile % p.tiles_n) * BN + grp * kGroupCols + c * kPieceCols,
+                  (tile / p.tiles_n) * kTileM + row0 + quad * 32);
     };
     if constexpr (EPI == EPI_ELEMENTWISE) {
-      if (staged && has_r && leader) {
-        if (total_pieces > 0) issue_r(0);
-        if (total_pieces > 1) issue_r(1);
+      if (staged && has_r) {
+        if (elect_one()) {
+          for (int i = 0; i < NB; ++i)
+            if (total_pieces > i) issue_r(i);
+        }
       }
     }
 
@@ -380,6 +408,17 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       [[maybe_unused]] const int n_tile = tn * BN + grp * kGroupCols;   // the group's first column
       [[maybe_unused]] const int n_valid = min(kGroupCols, p.N - n_tile);   // its valid columns (may be <= 0)
 
+      // Elementwise: this thread's two of the tile's BN bias values, fetched before the wait for
+      // the accumulator so that the L2 latency is hidden, and staged in shared memory after it
+      // (per piece every lane then reads the same 32 values: broadcast loads).
+      [[maybe_unused]] float2 bpre = make_float2(0.0f, 0.0f);
+      if constexpr (EPI == EPI_ELEMENTWISE) {
+        const int n = n_tile + 2 * et;
+        if (p.bias != nullptr && 2 * et < kGroupCols) {
+          if (n < p.N) bpre.x = __bfloat162float(p.bias[n]);
+          if (n + 1 < p.N) bpre.y = __bfloat162float(p.bias[n + 1]);
+        }
+      }
       // One thread polls the accumulator barrier; the rest block in hardware at the named
       // barrier, which hands every epilogue warp the same go/no-go.
       bool ok = true;
@@ -388,6 +427,11 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       ok = named_barrier_and(bar_a, kEpiThreads, ok);
       if (!ok) break;
       tc_fence_after_sync();
+      if constexpr (EPI == EPI_ELEMENTWISE) {
+        // every thread is past its last read of the previous tile's values (barrier above)
+        if (2 * et < kGroupCols) *reinterpret_cast<float2*>(sbias + 2 * et) = bpre;
+        named_barrier_sync(bar_b, kEpiThreads);
+      }
       const uint32_t t_acc = tmem_base + static_cast<uint32_t>(a * BN + grp * kGroupCols) + lane_off;
       // hand the accumulator back to the UMMA issuer (one arrival per warp)
       auto release_acc = [&]() {
@@ -406,16 +450,21 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           float ts1 = 0.0f, ts2 = 0.0f;
 #pragma unroll 1
           for (int c = 0; c < PIECES; ++c, ++g) {
-            const int b = static_cast<int>(g & 1);
+            const int b = static_cast<int>(g % NB);
             uint4 rv[4];
-            bool rok = true;
             if (has_r) {
-              rok = mbar_wait(&r_full[b], static_cast<uint32_t>((g >> 1) & 1), abort_flag, p.status,
-                              KF_DEV_TIMEOUT_EPILOGUE);
-              const uint8_t* rb = rbuf + b * kPieceBytes;
+              // this warp's slab of the residual piece, then at once the request for the piece
+              // that will use the same buffer
+              bool rok = mbar_wait(&my_r_full[b], static_cast<uint32_t>((g / NB) & 1), abort_flag, p.status,
+                                   KF_DEV_TIMEOUT_EPILOGUE);
+              if (!__all_sync(0xffffffffu, rok)) { alive = false; break; }
 #pragma unroll
               for (int q = 0; q < 4; ++q)
-                rv[q] = *reinterpret_cast<const uint4*>(rb + piece_off(row, q));
+                rv[q] = *reinterpret_cast<const uint4*>(rbuf + b * kPieceBytes + piece_off(row, q));
+              __syncwarp();
+              if (elect_one()) {
+                if (g + NB < total_pieces) issue_r(g + NB);
+              }
             }
             if (p.gn_pieces > 0 && c % p.gn_pieces == 0) {
               // statistics of the group that starts here: its columns are all in this tile
@@ -425,7 +474,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 uint32_t u[32];
                 tmem_ld_32x32(t_acc + (c + q) * kPieceCols, u);
                 float bq[32];
-                load_bias32(p, n_tile + (c + q) * kPieceCols, bq);
+                load_sbias32(sbias + (c + q) * kPieceCols, bq);
                 tmem_ld_wait();
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
@@ -441,7 +490,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             uint32_t v[32];
             tmem_ld_32x32(t_acc + c * kPieceCols, v);
             float bs[32];
-            load_bias32(p, n_tile + c * kPieceCols, bs);
+            load_sbias32(sbias + c * kPieceCols, bs);
             tmem_ld_wait();
             if (c == PIECES - 1) release_acc();
             float f[32];
@@ -471,6 +520,11 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 f[8 * q + 6] += bf16_lo(rv[q].w); f[8 * q + 7] += bf16_hi(rv[q].w);
               }
             }
+            // Every warp stages and stores its own 32 rows of the piece (a 2 KB slab of the 8 KB
+            // buffer, TMA box of 32 rows): no barrier between the warps anywhere in this loop.
+            // First the store issued from this slab NB pieces ago must have finished reading it.
+            bulk_wait_group_read<NB - 1>();     // a no-op in the lanes that issue no stores
+            __syncwarp();
             uint8_t* yb = ybuf + b * kPieceBytes;
 #pragma unroll
             for (int q = 0; q < 4; ++q)
@@ -480,20 +534,16 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                              pack_bf16x2(f[8 * q + 4], f[8 * q + 5]),
                              pack_bf16x2(f[8 * q + 6], f[8 * q + 7]));
             fence_proxy_async_smem();
-            // One barrier per piece.  Before it the leader makes sure the previous piece's store
-            // has finished reading the other buffer, so after it (a) this piece may be stored,
-            // (b) the other output buffer may be rewritten, (c) rbuf[b] has been consumed by all.
-            if (leader) bulk_wait_group_read<0>();
-            rok = named_barrier_and(bar_b, kEpiThreads, rok);
-            if (!rok) { alive = false; break; }
-            if (leader) {
-              tma_store_2d(&tmY, yb, n_tile + c * kPieceCols, m_cta);   // clipped at M, N
+            __syncwarp();
+            if (elect_one()) {
+              if (m_cta + quad * 32 < p.M && n_tile + c * kPieceCols < p.N)
+                tma_store_2d(&tmY, yb + quad * (kPieceBytes / 4), n_tile + c * kPieceCols,
+                             m_cta + quad * 32);                     // clipped at M, N
               bulk_commit_group();
-              if (has_r && g + 2 < total_pieces) issue_r(g + 2);
             }
           }
           if (p.gn_tile_stats && alive && row_ok)
-            reinterpret_cast<float2*>(p.partial)[m * p.tiles_n + tn] = make_float2(ts1, ts2);
+            reinterpret_cast<float2*>(p.partial)[(m * p.tiles_n + tn) * kGroups + grp] = make_float2(ts1, ts2);
         } else {
           // Output (or residual) rows that do not start on 16 bytes: no TMA.  Pieces still go
           // through shared memory so that global accesses run along rows: a warp moves 32 rows,
@@ -520,7 +570,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             uint32_t v[32];
             tmem_ld_32x32(t_acc + c * 32, v);
             float bs[32];
-            load_bias32(p, n0, bs);
+            load_sbias32(sbias + c * 32, bs);
             tmem_ld_wait();
             float f[32];
 #pragma unroll
@@ -833,7 +883,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       }
       if (++a == 2) { a = 0; aph ^= 1u; }
     }
-    if (leader) bulk_wait_group<0>();          // every output store has completed
+    bulk_wait_group<0>();          // every output store has completed (a no-op in lanes that issued none)
   }
 
   // ---------------------------------------------------------------- teardown

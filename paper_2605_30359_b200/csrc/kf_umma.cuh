@@ -112,8 +112,8 @@ struct UmmaCfg {
       EPI == EPI_ELEMENTWISE || EPI == EPI_SOFTMAX ? 4 * kPieceBytes
                                                     : (EPI == EPI_ROWSUM ? 0 : 2 * kPieceBytes);
   static constexpr int kBarBytes = 256;
-  // elementwise: the tile's BN bias values as fp32, staged once per tile
-  static constexpr int kBiasBytes = EPI == EPI_ELEMENTWISE ? BN * 4 : 0;
+  // GEMM epilogues: the tile's BN bias values as fp32, staged once per tile
+  static constexpr int kBiasBytes = EPI == EPI_CONV ? 0 : BN * 4;
   static constexpr int kFit = (kMaxDynSmem - 1024 - kStaging - kBarBytes - kBiasBytes) / kStage;
   static constexpr int kStages = kFit > 8 ? 8 : kFit;
   static constexpr int kRing = kStage * kStages;
@@ -408,11 +408,11 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       [[maybe_unused]] const int n_tile = tn * BN + grp * kGroupCols;   // the group's first column
       [[maybe_unused]] const int n_valid = min(kGroupCols, p.N - n_tile);   // its valid columns (may be <= 0)
 
-      // Elementwise: this thread's two of the tile's BN bias values, fetched before the wait for
+      // GEMM epilogues: this thread's two of the group's bias values, fetched before the wait for
       // the accumulator so that the L2 latency is hidden, and staged in shared memory after it
       // (per piece every lane then reads the same 32 values: broadcast loads).
       [[maybe_unused]] float2 bpre = make_float2(0.0f, 0.0f);
-      if constexpr (EPI == EPI_ELEMENTWISE) {
+      if constexpr (EPI != EPI_CONV) {
         const int n = n_tile + 2 * et;
         if (p.bias != nullptr && 2 * et < kGroupCols) {
           if (n < p.N) bpre.x = __bfloat162float(p.bias[n]);
@@ -427,7 +427,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       ok = named_barrier_and(bar_a, kEpiThreads, ok);
       if (!ok) break;
       tc_fence_after_sync();
-      if constexpr (EPI == EPI_ELEMENTWISE) {
+      if constexpr (EPI != EPI_CONV) {
         // every thread is past its last read of the previous tile's values (barrier above)
         if (2 * et < kGroupCols) *reinterpret_cast<float2*>(sbias + 2 * et) = bpre;
         named_barrier_sync(bar_b, kEpiThreads);
@@ -615,7 +615,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           uint32_t v[32];
           tmem_ld_32x32(t_acc + c * 32, v);
           float bs[32];
-          load_bias32(p, n_tile + c * 32, bs);
+          load_sbias32(sbias + c * 32, bs);
           tmem_ld_wait();
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -633,7 +633,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           uint32_t v[32];
           tmem_ld_32x32(t_acc + c * 32, v);
           float bs[32];
-          load_bias32(p, n_tile + c * 32, bs);
+          load_sbias32(sbias + c * 32, bs);
           tmem_ld_wait();
           if (staged && c == PIECES - 1) release_acc();
           float f[32];
@@ -729,7 +729,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           uint32_t v[32];
           tmem_ld_32x32(t_acc + c * 32, v);
           float bs[32];
-          load_bias32(p, n_tile + c * 32, bs);
+          load_sbias32(sbias + c * 32, bs);
           tmem_ld_wait();
           float part = 0.0f;
 #pragma unroll

@@ -670,8 +670,7 @@ groupnorm_apply_kernel(int Cout, int groups, long long hw, int tiles_per_image, 
                        const __nv_bfloat16* __restrict__ beta, __nv_bfloat16* y) {
   const int cpg = Cout / groups;
   const long long cnt = static_cast<long long>(cpg) * hw;
-  // (Taking the images last written, which are still in L2, first made this in-place pass slower:
-  // 154 -> 159 us on the 128-image benchmark shape; the read-only second passes do gain from it.)
+  // increasing image order: the convolution wrote the first images last, they are still in L2
   const int g = blockIdx.x % groups;
   const long long n = blockIdx.x / groups;
   __nv_bfloat16* blk = y + (n * Cout + static_cast<long long>(g) * cpg) * hw;
@@ -890,7 +889,7 @@ channel_softmax_pool_tiled_kernel(int Nb, int C, int H, int Wd, int tw, const T*
   T* s = reinterpret_cast<T*>(smem_raw);
   const int Ho = H / POOL, Wo = Wd / POOL;
   const int col_tiles = (Wo + tw - 1) / tw;
-  long long b = static_cast<long long>(gridDim.x) - 1 - blockIdx.x;    // last-written images first (still in L2)
+  long long b = blockIdx.x;    // first images first: the convolution wrote those last (still in L2)
   const int jt = static_cast<int>(b % col_tiles); b /= col_tiles;
   const int i = static_cast<int>(b % Ho);
   const long long n = b / Ho;

@@ -91,6 +91,14 @@ struct UmmaParams {
 };
 
 // The it-th tile of scheduling slot `cta` out of `ncta`, or -1 when the slot has no more work.
+// Convolution: the i-th scheduled pixel tile.  Images are taken last to first, so that the images
+// written last, which are the ones still in L2 when the kernel ends, are the first ones the pass
+// that follows (normalisation, pooling: increasing image order) reads.
+__device__ __forceinline__ int conv_pixel_tile(const UmmaParams& p, int i) {
+  const int img = p.tiles_n / p.tiles_per_image - 1 - i / p.tiles_per_image;
+  return img * p.tiles_per_image + i % p.tiles_per_image;
+}
+
 __device__ __forceinline__ int sched_tile(const UmmaParams& p, int cta, int ncta, int it) {
   const int tpu = p.tiles_per_unit;
   const int unit = cta + (it / tpu) * ncta;
@@ -252,7 +260,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (tile < 0) break;
         int tm, tn, img = 0, h0 = 0, x0 = 0;
         if constexpr (EPI == EPI_CONV) {
-          tm = tile % p.tiles_m; tn = tile / p.tiles_m;        // output-channel tile, pixel tile
+          tm = tile % p.tiles_m; tn = conv_pixel_tile(p, tile / p.tiles_m);   // output-channel tile, pixel tile
           img = tn / p.tiles_per_image;
           const int pt = tn % p.tiles_per_image;
           h0 = (pt / p.w_segs) * p.rows_per_tile;
@@ -400,7 +408,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const int tile = sched_tile(p, cta, ncta, it);
       if (tile < 0) break;
       int tm, tn;
-      if constexpr (EPI == EPI_CONV) { tm = tile % p.tiles_m; tn = tile / p.tiles_m; }
+      if constexpr (EPI == EPI_CONV) { tm = tile % p.tiles_m; tn = conv_pixel_tile(p, tile / p.tiles_m); }
       else { tm = tile / p.tiles_n; tn = tile % p.tiles_n; }
       const int m_cta = tm * kTileM + row0;               // first row of this CTA's 128 rows
       const long long m = static_cast<long long>(m_cta) + row;

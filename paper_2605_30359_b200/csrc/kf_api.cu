@@ -303,8 +303,8 @@ int env_int(const char* name, int dflt) {
 }
 
 // Cluster size of the split-K kernel, or 0.  Measured on B200: a narrow-tile CTA spends about
-// 0.28 us per K block whatever the tile width, the cluster exchange costs about 4 us, so
-// splitting pays from about 24 K blocks; clusters of 8 schedule well only while there are few
+// 0.16 us per K block, the cluster exchange costs about 4 us, so splitting pays from about 28 K
+// blocks (K = 1536: 9.9 us split, 8.9 us plain; K = 2048: 9.4 against 10.7 us); clusters of 8 schedule well only while there are few
 // of them (16 clusters of 8 already ran in two waves).
 int pick_split_k(int64_t M, int64_t N, int64_t K, int sm_count, int* bn_out) {
   if (getenv("KF_NO_SPLITK") != nullptr) return 0;
@@ -312,7 +312,7 @@ int pick_split_k(int64_t M, int64_t N, int64_t K, int sm_count, int* bn_out) {
   const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + bn - 1) / bn);
   const int64_t kb = (K + kBK - 1) / kBK;
   *bn_out = bn;
-  if (kb < env_int("KF_SPLITK_MIN_KB", 24)) return 0;
+  if (kb < env_int("KF_SPLITK_MIN_KB", 28)) return 0;
   if (bn == 256 && kb >= 32 && tiles * 8 <= 64) return 8;
   if (tiles * 4 <= sm_count - sm_count % 4) return 4;
   return 0;

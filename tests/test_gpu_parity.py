@@ -215,10 +215,10 @@ def test_bf16_gemm_tile_widths_and_unaligned_rows(kf, shape):
 # Few tiles and a long K take the split-K cluster kernel: 4 or 8 CTAs per tile, partial tiles
 # exchanged through distributed shared memory, slices of 64 or 32 columns finished per CTA.
 @pytest.mark.parametrize("shape", [(128, 1024, 2048),     # 4 tiles x 8 CTAs, 256-column tiles
-                                   (200, 300, 1544),      # 4 tiles x 4 CTAs, ragged M, N, K (24.1 K blocks)
+                                   (200, 300, 1800),      # 4 tiles x 4 CTAs, ragged M, N, K (28.1 K blocks)
                                    (100, 128, 4096),      # 128-column tile x 4 CTAs
                                    (64, 2000, 2048),      # 8 tiles x 8 CTAs, last tile ragged in N
-                                   (130, 777, 1600)])     # unaligned rows: scalar stores
+                                   (130, 777, 1848)])     # unaligned rows: scalar stores
 def test_bf16_gemm_split_k_cluster_kernel(kf, shape):
     M, N, K = shape
     d = ki.gemm_inputs("c2", seed=31, M=M, N=N, K=K)

@@ -523,6 +523,66 @@ def test_gemm_groupnorm(kf, dtype, shape, groups):
     assert np.abs(blk.var(axis=2) - 1.0).max() < (5e-2 if dtype == "bf16" else 1e-3)
 
 
+# ------------------------------------------------------------------ seeded shape fuzz across the dispatch rules
+def _fuzz_shapes(seed, count):
+    """bf16 GEMM shapes around the dispatch boundaries: tile widths 32..256, one or two epilogue
+    groups, CTA pairs (M > 256, K >= 2048), split-K (few tiles, K >= 1792), rows that TMA cannot
+    store (odd N), operands that TMA cannot load (K not a multiple of 8: repacked or scalar)."""
+    r = np.random.default_rng(seed)
+    out = []
+    for _ in range(count):
+        M = int(r.choice([1, 31, 64, 100, 128, 129, 257, 300, 512, 640]))
+        N = int(r.choice([8, 40, 64, 96, 136, 256, 264, 333, 512, 776, 1024]))
+        K = int(r.choice([8, 64, 72, 200, 512, 1000, 1027, 1536, 1800, 2048, 2304]))
+        out.append((M, N, K))
+    return out
+
+
+@pytest.mark.parametrize("shape", _fuzz_shapes(2024, 28))
+def test_fuzz_bf16_gemm_chain(kf, shape):
+    M, N, K = shape
+    d = ki.gemm_inputs("c2", seed=M + 3 * N + 7 * K, M=M, N=N, K=K)
+    opts = [("gelu_tanh", 0.5, True, True), ("relu", 1.0, True, False), ("none", 1.0, False, False),
+            ("mish", 2.0, False, True)]
+    act, scale, use_bias, use_res = opts[(M + N + K) % 4]
+    got, ref = run_gemm(kf, d, act, scale, use_bias=use_bias, use_res=use_res)
+    assert_close(got, ref, 2e-2, 2e-2, "fuzz chain %s %s" % (shape, act))
+
+
+@pytest.mark.parametrize("shape", _fuzz_shapes(77, 16))
+def test_fuzz_bf16_gemm_rowreduce(kf, shape):
+    M, N, K = shape
+    d = ki.gemm_inputs("c3", seed=M + 5 * N + K, M=M, N=N, K=K)
+    for act, red in (("none", "softmax"), ("sigmoid", "sum"), ("relu", "logsumexp")):
+        out = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), act, red)
+        check_status()
+        ref = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], act, red)
+        if red == "softmax":
+            assert_close(to_f64(out), ref, 2e-2, 2e-2, "fuzz softmax %s" % (shape,))
+            assert np.abs(to_f64(out).sum(axis=1) - 1.0).max() < 2e-2
+        else:
+            # a sum of N terms, each within the bf16-input tolerance: compare relative to N
+            err = np.abs(to_f64(out) - ref).max()
+            assert err <= 2e-2 * max(1.0, np.abs(ref).max()), "fuzz %s %s: %g" % (red, shape, err)
+
+
+@pytest.mark.parametrize("shape,groups", [((300, 256, 512), 8), ((129, 512, 1000), 4), ((64, 1024, 2048), 8),
+                                          ((640, 768, 256), 3), ((257, 384, 72), 12), ((100, 512, 2304), 2),
+                                          ((512, 256, 64), 1)])
+def test_fuzz_bf16_gemm_groupnorm(kf, shape, groups):
+    """Group widths 32, 64, 128 (inside one epilogue group's half tile), 256 (per-slice statistics
+    + second pass, single-CTA and pair kernels), 1024 and an odd width (row kernel)."""
+    M, N, K = shape
+    d = ki.gemm_inputs("c3", seed=N + K, M=M, N=N, K=K)
+    gamma = ki.store(ki.uniform(5, 7, (N,), 0.5, 1.5), "bf16")
+    beta = ki.store(ki.uniform(5, 8, (N,), -1.0, 1.0), "bf16")
+    Y = kf.gemm_groupnorm(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), groups, 1e-5, to_dev(gamma),
+                          to_dev(beta), "swish")
+    check_status()
+    ref = oracle.gemm_groupnorm(d["X"], d["W"], d["b"], groups, 1e-5, gamma, beta, "swish")
+    assert_close(to_f64(Y), ref, 2e-2, 2e-2, "fuzz gemm groupnorm %s g=%d" % (shape, groups))
+
+
 # ------------------------------------------------------------------ convolution + GroupNorm
 def run_conv(kf, d, act="relu", groups=None, gamma=None, beta=None, use_bias=True):
     groups = d["groups"] if groups is None else groups

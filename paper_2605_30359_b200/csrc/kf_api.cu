@@ -131,14 +131,14 @@ bool encode_nhwc(CUtensorMap* tm, const void* base, int64_t Nb, int64_t H, int64
          CUDA_SUCCESS;
 }
 
-// NCHW bf16 output seen as [Nb][C][H*W] -> store boxes of 32 pixels x 128 channels of one image
+// NCHW bf16 output seen as [Nb][C][H*W] -> store boxes of 32 pixels x 32 channels of one image
 // (64-byte swizzle like every epilogue piece); channels past C are clipped.
 bool encode_nchw_out(CUtensorMap* tm, const void* base, int64_t Nb, int64_t C, int64_t hw) {
   const cuuint64_t dims[3] = {static_cast<cuuint64_t>(hw), static_cast<cuuint64_t>(C),
                               static_cast<cuuint64_t>(Nb)};
   const cuuint64_t strides[2] = {static_cast<cuuint64_t>(hw) * 2,
                                  static_cast<cuuint64_t>(C) * hw * 2};
-  const cuuint32_t box[3] = {static_cast<cuuint32_t>(kPieceCols), static_cast<cuuint32_t>(kBM), 1};
+  const cuuint32_t box[3] = {static_cast<cuuint32_t>(kPieceCols), 32, 1};   // one warp's slab of a piece
   const cuuint32_t estr[3] = {1, 1, 1};
   return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides,
                   box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,

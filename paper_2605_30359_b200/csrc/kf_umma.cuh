@@ -845,19 +845,22 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
           if (p.stats_only != 0) continue;     // only the per-channel statistics are wanted
           if (staged) {
+            // every warp stages and stores its own 32 channels of the piece (2 KB slab, TMA box
+            // of 32 pixels x 32 channels): no barrier between the warps
             const int b = static_cast<int>(g & 1);
             uint8_t* yb = ybuf + b * kPieceBytes;
+            bulk_wait_group_read<1>();       // the store from this buffer two pieces ago has let go
+            __syncwarp();
 #pragma unroll
             for (int q = 0; q < 4; ++q)
               *reinterpret_cast<uint4*>(yb + piece_off(row, q)) =
                   make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
             fence_proxy_async_smem();
-            if (leader) bulk_wait_group_read<0>();     // the other buffer's store has let go
-            named_barrier_sync(bar_b, kEpiThreads);
-            if (leader && left > 0) {
-              // box = 32 pixels x 128 channels of image img; channels past Cout and pixels past
-              // the image are clipped
-              tma_store_3d(&tmY, yb, px0 + c * 32, tm * kBM, img);
+            __syncwarp();
+            if (elect_one()) {
+              // channels past Cout and pixels past the image are clipped
+              if (left > 0 && tm * kBM + quad * 32 < p.N)
+                tma_store_3d(&tmY, yb + quad * (kPieceBytes / 4), px0 + c * 32, tm * kBM + quad * 32, img);
               bulk_commit_group();
             }
           } else {

@@ -114,12 +114,13 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
  * gs = N / groups, per row m and group g (columns [g*gs, (g+1)*gs)):
  *   mu = mean Z, var = mean (Z-mu)^2 (biased), Y = post_act((Z-mu)/sqrt(var+eps)*gamma[n]+beta[n]).
  * gamma, beta [N] of io_dtype, may be NULL (1, 0); groups must divide N (groups = 1 normalises
- * the whole row, as a LayerNorm does).  bf16 problems whose group size is 32, 64,
- * 128 or 256, with TMA-loadable operands (see kf_gemm_epilogue) and a 16-byte aligned Y with
- * ldy % 8 == 0, run in ONE tensor-core kernel: a tile of 256 columns holds whole groups, so the
- * epilogue takes the statistics from the accumulator and normalises before storing.  Group
- * sizes that are multiples of 256 take the same GEMM kernel storing Z plus per-tile statistics
- * (workspace: 8 bytes per row and 256 columns) and a row kernel that normalises in place.
+ * the whole row, as a LayerNorm does).  bf16 problems whose group size is 32, 64 or
+ * 128, with TMA-loadable operands (see kf_gemm_epilogue) and a 16-byte aligned Y with
+ * ldy % 8 == 0, run in ONE tensor-core kernel: the half tile an epilogue group owns holds whole
+ * groups, so the epilogue takes the statistics from the accumulator and normalises before
+ * storing.  Group sizes that are multiples of 256 take the same GEMM kernel storing Z plus
+ * per-slice statistics (workspace: 16 bytes per row and 256 columns) and a row kernel that
+ * normalises in place.
  * Everything else computes Z in fp32 into the workspace (M*N*4 bytes, plus the split operands for large fp32
  * problems) and normalises with a second kernel. */
 kf_status kf_gemm_groupnorm(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
@@ -163,7 +164,7 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype,
  * The call allocates nothing: no cudaMalloc/cudaFree, no allocating library routine.
  *   - Limit: a problem whose kf_gemm_rowreduce_workspace_bytes() exceeds
  *     KF_STATIC_SCRATCH_BYTES is refused with KF_ERR_WORKSPACE and nothing is launched
- *     (bf16, K % 8 == 0: M * ceil(N/256) * 8 bytes for softmax, * 4 for sum; otherwise M*N*4).
+ *     (bf16, K % 8 == 0: M * ceil(N/256) * 16 bytes for softmax, * 4 for sum; otherwise M*N*4).
  *   - The first call on each device looks up the array's device address (a one-time host-side
  *     query, made with that device current).  Make that first call outside any stream capture.
  *   - All calls on a device share the one array, and it keeps whatever the last call wrote.

@@ -401,6 +401,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
     int a = 0; uint32_t aph = 0;
     bool alive = true;
+    bool warp_failed = false;    // this warp gave up on one of its own waits inside a tile
     [[maybe_unused]] uint64_t keep_policy = 0;
     if constexpr (EPI == EPI_SOFTMAX) keep_policy = l2_policy_evict_last();
     [[maybe_unused]] float unit_sum = 0.0f;    // row sum carried across the tiles of a unit
@@ -432,7 +433,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       bool ok = true;
       if (leader)
         ok = mbar_wait(&tmem_full[a], aph, abort_flag, p.status, KF_DEV_TIMEOUT_EPILOGUE);
-      ok = named_barrier_and(bar_a, kEpiThreads, ok);
+      ok = named_barrier_and(bar_a, kEpiThreads, ok && !warp_failed);
       if (!ok) break;
       tc_fence_after_sync();
       if constexpr (EPI != EPI_CONV) {
@@ -465,7 +466,9 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               // that will use the same buffer
               bool rok = mbar_wait(&my_r_full[b], static_cast<uint32_t>((g / NB) & 1), abort_flag, p.status,
                                    KF_DEV_TIMEOUT_EPILOGUE);
-              if (!__all_sync(0xffffffffu, rok)) { alive = false; break; }
+              // a slab that never arrived: the status word has the time-out; keep going (every
+              // warp of the group must reach the group's barriers) and leave with the others
+              if (!rok) warp_failed = true;
 #pragma unroll
               for (int q = 0; q < 4; ++q)
                 rv[q] = *reinterpret_cast<const uint4*>(rbuf + b * kPieceBytes + piece_off(row, q));

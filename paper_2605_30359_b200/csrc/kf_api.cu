@@ -321,6 +321,17 @@ int pick_split_k(int64_t M, int64_t N, int64_t K, int sm_count, int* bn_out) {
 bool use_cta_pairs(int64_t M, int64_t K) {
   return M > 256 && K >= env_int("KF_PAIR_MIN_K", 2048) && getenv("KF_NO_PAIR") == nullptr;
 }
+// The elementwise chain: the pair kernel runs one epilogue group, the single-CTA kernel two, so
+// pairs pay only where a CTA has enough MMA work to hide its epilogues behind: from about 128
+// K blocks of 64 per CTA (measured with GELU(erf)*s+R: 2048^3 29.1 us in pairs, 25.0 us
+// single; 2048x4096x2048 43.3 / 38.2; 1024x4096x4096 37.4 / 35.2; 4096^3 105.4 / 115.3;
+// 8192x1024x8192 107.5 / 112.4).
+bool use_cta_pairs_chain(int64_t M, int64_t N, int64_t K, int sm_count) {
+  if (!use_cta_pairs(M, K)) return false;
+  const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + 255) / 256);
+  const int64_t kb = (K + kBK - 1) / kBK;
+  return tiles * kb >= static_cast<int64_t>(env_int("KF_PAIR_MIN_KB_PER_CTA", 128)) * sm_count;
+}
 size_t rowreduce_simt_ws(int64_t M, int64_t N) { return round256(static_cast<size_t>(M) * N * 4); }
 
 // The fp32 chain on the tensor cores: split prepasses into `ws` (tf32_ws bytes), then the GEMM
@@ -517,7 +528,7 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
   }
   if (umma_gemm_ok(io_dtype, K, X, ldx, W, ldw)) {
     const int bn = pick_tile_n(M, N, d->sm_count);
-    const bool pair = bn == 256 && use_cta_pairs(M, K);
+    const bool pair = bn == 256 && use_cta_pairs_chain(M, N, K, d->sm_count);
     UmmaMaps tm;
     if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, pair ? bn / 2 : bn))
       return KF_ERR_CUDA;
@@ -591,7 +602,7 @@ kf_status kf_gemm_groupnorm(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, 
     // in the epilogue; tile width as for the plain chain, but never narrower than two groups
     int bn = pick_tile_n(M, N, d->sm_count);
     if (bn < 2 * gs) bn = static_cast<int>(2 * gs);
-    const bool pair = bn == 256 && use_cta_pairs(M, K);
+    const bool pair = bn == 256 && use_cta_pairs_chain(M, N, K, d->sm_count);
     UmmaMaps tm;
     if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, pair ? bn / 2 : bn))
       return KF_ERR_CUDA;
@@ -632,7 +643,7 @@ kf_status kf_gemm_groupnorm(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, 
     const size_t need = round256(static_cast<size_t>(M) * ((N + 255) / 256) * 16);
     vs = check_workspace(workspace, workspace_bytes, need);
     if (vs != KF_OK) return vs;
-    const bool pair = use_cta_pairs(M, K);
+    const bool pair = use_cta_pairs_chain(M, N, K, d->sm_count);
     UmmaMaps tm;
     if (!encode_2d(&tm.a, X, M, K, ldx, kBM) || !encode_2d(&tm.b, W, N, K, ldw, pair ? bn / 2 : bn))
       return KF_ERR_CUDA;

@@ -281,18 +281,21 @@ def test_bf16_softmax_unaligned_rows(kf, shape):
     assert np.abs(got.sum(axis=1) - 1).max() < 4e-3
 
 
-# K >= 2048 with more than 256 rows takes the CTA-pair kernel (256-row tiles over two SMs)
+# K >= 2048 with more than 256 rows and enough K blocks per CTA takes the CTA-pair kernel (256-row
+# tiles over two SMs); these small shapes reach it with the work threshold switched off
 @pytest.mark.parametrize("shape", [(384, 520, 2048), (257, 256, 2112), (1000, 264, 2048)])
-def test_bf16_gemm_cta_pair_kernel(kf, shape):
+def test_bf16_gemm_cta_pair_kernel(kf, shape, monkeypatch):
+    monkeypatch.setenv("KF_PAIR_MIN_KB_PER_CTA", "0")
     M, N, K = shape
     d = ki.gemm_inputs("c2", seed=12, M=M, N=N, K=K)
     got, ref = run_gemm(kf, d, "gelu_tanh", 0.5)
     assert_close(got, ref, 2e-2, 2e-2, "bf16 pair %s" % (shape,))
 
 
-def test_bf16_cta_pair_layout_pins(kf):
+def test_bf16_cta_pair_layout_pins(kf, monkeypatch):
     """One-hot rows through the pair kernel: each CTA's A half and B half must land where the
     256-row MMA expects them."""
+    monkeypatch.setenv("KF_PAIR_MIN_KB_PER_CTA", "0")
     M, N, K = 640, 512, 2048
     r = np.random.default_rng(6)
     Wv = (r.integers(-64, 65, size=(N, K)) / 64.0)
@@ -502,8 +505,10 @@ def test_row_reductions_reject_bad_arguments(kf):
     ("f32", (70, 60, 33), 5),            # fp32 scalar path
     ("f32", (1024, 1024, 512), 16),      # fp32 GEMM on the tensor cores, then the row kernel
 ])
-def test_gemm_groupnorm(kf, dtype, shape, groups):
+def test_gemm_groupnorm(kf, dtype, shape, groups, monkeypatch):
     M, N, K = shape
+    if K >= 2048:
+        monkeypatch.setenv("KF_PAIR_MIN_KB_PER_CTA", "0")    # small shapes through the CTA-pair kernel
     d = ki.gemm_inputs("c3", seed=95, M=M, N=N, K=K, dtype=dtype)
     gamma = ki.store(ki.uniform(95, 7, (N,), 0.5, 1.5), dtype)
     beta = ki.store(ki.uniform(95, 8, (N,), -1.0, 1.0), dtype)
@@ -539,7 +544,7 @@ def _fuzz_shapes(seed, count):
 
 
 @pytest.mark.parametrize("shape", _fuzz_shapes(2024, 28))
-def test_fuzz_bf16_gemm_chain(kf, shape):
+def test_fuzz_bf16_gemm_chain(kf, shape, monkeypatch):
     M, N, K = shape
     d = ki.gemm_inputs("c2", seed=M + 3 * N + 7 * K, M=M, N=N, K=K)
     opts = [("gelu_tanh", 0.5, True, True), ("relu", 1.0, True, False), ("none", 1.0, False, False),
@@ -547,6 +552,10 @@ def test_fuzz_bf16_gemm_chain(kf, shape):
     act, scale, use_bias, use_res = opts[(M + N + K) % 4]
     got, ref = run_gemm(kf, d, act, scale, use_bias=use_bias, use_res=use_res)
     assert_close(got, ref, 2e-2, 2e-2, "fuzz chain %s %s" % (shape, act))
+    if M > 256 and K >= 2048:         # the same through the CTA-pair kernel (work threshold off)
+        monkeypatch.setenv("KF_PAIR_MIN_KB_PER_CTA", "0")
+        got, ref = run_gemm(kf, d, act, scale, use_bias=use_bias, use_res=use_res)
+        assert_close(got, ref, 2e-2, 2e-2, "fuzz chain, pairs %s %s" % (shape, act))
 
 
 @pytest.mark.parametrize("shape", _fuzz_shapes(77, 16))

@@ -55,8 +55,8 @@ def load_peaks():
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the config-2 kernel, from the ncu
-# capture summarised in profiles/umma_chain_kernel_c2_gelu_residual.md (213.7 MB + 52.9 MB)
-TRAFFIC_C2_BYTES = 266.6e6
+# capture summarised in profiles/umma_chain_kernel_c2_gelu_residual.md (214.7 MB + 52.8 MB)
+TRAFFIC_C2_BYTES = 267.4e6
 
 
 # ------------------------------------------------------------------ clocks during the timed region

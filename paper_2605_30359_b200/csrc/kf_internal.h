@@ -29,6 +29,9 @@ cudaError_t launch_umma_rowsum(int act, int pair, const UmmaMaps& tm, const Umma
                                int grid, cudaStream_t st);
 cudaError_t launch_umma_conv(int bn, int act, const UmmaMaps& tm, const UmmaParams& p, int grid,
                              cudaStream_t st);
+// the cluster form with GroupNorm in the epilogue: `images` units, p.gn_cluster CTAs per cluster
+cudaError_t launch_umma_conv_gn(int bn, int act, const UmmaMaps& tm, const UmmaParams& p, int images,
+                                cudaStream_t st);
 constexpr int kRowReduceBN = 256;   // tile width of the row-reduce first pass
 constexpr int kRowReduceNarrowBN = 64;   // ... of the softmax first pass of one-wave problems
 
@@ -137,14 +140,45 @@ cudaError_t launch_channel_softmax_pool(int dt, int Nb, int C, int H, int Wd, in
 // `grid` counts scheduled CTAs for the single-CTA kernel and CTA PAIRS for the pair kernel
 // (which launches 2*grid CTAs in clusters of two).
 template <int BN, int EPI, int ACT, typename OutT, bool CTA2 = false>
+// `cluster` > 0 (EPI_CONV_GN): `grid` counts the images; the launch uses as many clusters of that
+// many CTAs as can be resident at once (at most one per image).
 inline cudaError_t launch_umma_instance(const UmmaMaps& tm, const UmmaParams& p, int grid,
-                                        cudaStream_t st) {
+                                        cudaStream_t st, int cluster = 0) {
   using C = UmmaCfg<BN, EPI, CTA2>;
   constexpr int smem = C::kTotal;
   static_assert(smem <= kMaxDynSmem, "shared-memory plan exceeds the per-CTA limit");
   auto kern = umma_chain_kernel<BN, EPI, ACT, OutT, CTA2>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
+  if (cluster > 0) {
+    if (cluster > 8) {
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+      if (e != cudaSuccess) return e;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cluster, 1, 1);
+    cfg.blockDim = dim3(num_threads(EPI, BN, CTA2), 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    static int resident[17] = {0};             // clusters of this size that fit on the device
+    if (resident[cluster] == 0) {
+      int n = 0;
+      e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+      if (e != cudaSuccess) return e;
+      if (n < 1) return cudaErrorInvalidConfiguration;
+      resident[cluster] = n;
+    }
+    const int clusters = grid < resident[cluster] ? grid : resident[cluster];
+    cfg.gridDim = dim3(clusters * cluster, 1, 1);
+    return cudaLaunchKernelEx(&cfg, kern, tm.a, tm.b, tm.r, tm.y, p);
+  }
   if constexpr (CTA2) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * grid, 1, 1);

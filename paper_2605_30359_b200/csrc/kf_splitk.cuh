@@ -35,16 +35,8 @@ struct SplitKCfg {
   static_assert(kTotal <= kMaxDynSmem, "shared-memory plan exceeds the per-CTA limit");
 };
 
-// Bulk copy from this CTA's shared memory into a peer's; the bytes complete on the PEER's
-// mbarrier.  Addresses and size are multiples of 16 bytes.  (Remote st.shared::cluster stores
-// moved the same 96 KB in 5 us; the copy engine does it in a fraction of that.)
-__device__ __forceinline__ void bulk_copy_to_peer(uint32_t dst_cluster_addr, uint32_t src_cta_addr,
-                                                  uint32_t bytes, uint32_t mbar_cluster_addr) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-      ::"r"(dst_cluster_addr), "r"(src_cta_addr), "r"(bytes), "r"(mbar_cluster_addr)
-      : "memory");
-}
+// (Remote st.shared::cluster stores moved the 96 KB of one exchange in 5 us; bulk_copy_to_peer,
+// i.e. the copy engine, does it in a fraction of that.)
 
 // f[j] = scale * act(f[j]) for a run-time activation code (this kernel is latency-bound; one
 // instantiation per tile shape keeps the library small).

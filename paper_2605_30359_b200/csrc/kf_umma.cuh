@@ -26,7 +26,11 @@
 
 namespace kf {
 
-enum : int { EPI_ELEMENTWISE = 0, EPI_SOFTMAX = 1, EPI_ROWSUM = 2, EPI_CONV = 3 };
+// EPI_CONV_GN: the convolution with GroupNorm finished inside the epilogue; the CTAs that hold
+// the tiles of one image form a cluster and exchange the group statistics through distributed
+// shared memory (two epilogue groups).
+enum : int { EPI_ELEMENTWISE = 0, EPI_SOFTMAX = 1, EPI_ROWSUM = 2, EPI_CONV = 3, EPI_CONV_GN = 4 };
+constexpr bool is_conv(int epi) { return epi == 3 || epi == 4; }
 
 constexpr int kBM = 128;          // tile rows = UMMA M = TMEM lanes
 constexpr int kBK = 64;           // K per stage: 64 bf16 = one 128-byte swizzled row
@@ -44,7 +48,9 @@ constexpr int kNumThreads = 192;  // 6 warps: producer, UMMA issuer, epilogue
 // The CTA-pair form (large K only: its epilogue hides behind the MMAs anyway, and the extra warps
 // cost it 2 %) keeps one group.
 constexpr int epi_groups(int epi, int bn, bool cta2) {
-  return epi == 1 /* EPI_SOFTMAX */ || (epi == 0 /* EPI_ELEMENTWISE */ && bn >= 64 && !cta2) ? 2 : 1;
+  return epi == 1 /* EPI_SOFTMAX */ || epi == 4 /* EPI_CONV_GN */ ||
+                 (epi == 0 /* EPI_ELEMENTWISE */ && bn >= 64 && !cta2)
+             ? 2 : 1;
 }
 constexpr int num_threads(int epi, int bn, bool cta2) { return 64 + kEpiThreads * epi_groups(epi, bn, cta2); }
 constexpr int kPieceCols = 32;    // epilogue piece: 128 rows x 32 columns
@@ -86,6 +92,8 @@ struct UmmaParams {
   int tile_px;                 // pixels per tile = UMMA N (a multiple of 32, <= BN): rows_per_tile
                                // whole rows, or one of w_segs equal segments of a row
   int w_segs;                  // 1, or segments per row when Wd > 256 (then rows_per_tile = 1)
+  int gn_cluster;              // EPI_CONV_GN: CTAs per cluster = pixel tiles per image (2, 4, 8 or 16)
+  int gn_groups;               // EPI_CONV_GN: GroupNorm groups (channels per group a power of two, 4..32)
   int pool2;                   // convolution: 0, or 2x2 pooling in the epilogue (1 = max, 2 = mean);
                                // needs w_segs == 1, Wd % 32 == 0, rows_per_tile and H even
 };
@@ -118,14 +126,16 @@ struct UmmaCfg {
   // group; conv = 2 output pieces
   static constexpr int kStaging =
       EPI == EPI_ELEMENTWISE || EPI == EPI_SOFTMAX ? 4 * kPieceBytes
-                                                    : (EPI == EPI_ROWSUM ? 0 : 2 * kPieceBytes);
+                                                    : (EPI == EPI_ROWSUM ? 0 : 2 * kPieceBytes);     // EPI_CONV_GN: one piece per epilogue group
   static constexpr int kBarBytes = 256;
   // GEMM epilogues: the tile's BN bias values as fp32, staged once per tile
-  static constexpr int kBiasBytes = EPI == EPI_CONV ? 0 : BN * 4;
-  static constexpr int kFit = (kMaxDynSmem - 1024 - kStaging - kBarBytes - kBiasBytes) / kStage;
+  static constexpr int kBiasBytes = EPI == EPI_CONV ? 0 : BN * 4;   // EPI_CONV_GN: the statistics it sends
+  // EPI_CONV_GN: statistics arriving from the cluster, [2 buffers][16 CTAs x 2 groups][32 x float2]
+  static constexpr int kInboxBytes = EPI == EPI_CONV_GN ? 2 * 32 * 256 : 0;
+  static constexpr int kFit = (kMaxDynSmem - 1024 - kStaging - kBarBytes - kBiasBytes - kInboxBytes) / kStage;
   static constexpr int kStages = kFit > 8 ? 8 : kFit;
   static constexpr int kRing = kStage * kStages;
-  static constexpr int kTotal = 1024 /*alignment slack*/ + kRing + kStaging + kBarBytes + kBiasBytes;
+  static constexpr int kTotal = 1024 /*alignment slack*/ + kRing + kStaging + kBarBytes + kBiasBytes + kInboxBytes;
 };
 
 // 32 consecutive bias values as fp32 (zeros past N or without a bias).  All lanes read the same
@@ -196,14 +206,27 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmY,
                   const UmmaParams p) {
   using C = UmmaCfg<BN, EPI, CTA2>;
-  static_assert(!CTA2 || EPI != EPI_CONV, "the convolution runs one CTA per tile");
+  static_assert(!CTA2 || !is_conv(EPI), "the convolution runs one CTA per tile");
   constexpr int kTileM = CTA2 ? 2 * kBM : kBM;            // rows of one scheduled tile
   // In a pair, rank 0 issues the MMAs; both ranks load, and both run the epilogue on their own
   // 128 accumulator rows.  `cta` / `ncta` index the tile schedule (pairs count once).
   uint32_t rank = 0;
   if constexpr (CTA2) rank = cluster_ctarank();
-  const int cta = CTA2 ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
-  const int ncta = CTA2 ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
+  int cta = CTA2 ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+  int ncta = CTA2 ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
+  // EPI_CONV_GN: a cluster takes whole images (the schedule counts clusters and images), its CTA
+  // of rank r the r-th pixel tile of each
+  [[maybe_unused]] uint32_t crank = 0;
+  if constexpr (EPI == EPI_CONV_GN) {
+    crank = cluster_ctarank();
+    cta = static_cast<int>(blockIdx.x) / p.gn_cluster;
+    ncta = static_cast<int>(gridDim.x) / p.gn_cluster;
+  }
+  auto tile_at = [&](int it) -> int {
+    const int t = sched_tile(p, cta, ncta, it);
+    if constexpr (EPI == EPI_CONV_GN) return t < 0 ? t : t * p.gn_cluster + static_cast<int>(crank);
+    else return t;
+  };
   constexpr int kStages = C::kStages;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -215,7 +238,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   uint64_t* tmem_full = empty + kStages;
   uint64_t* tmem_empty = tmem_full + 2;
   uint64_t* r_full = tmem_empty + 2;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(r_full + 8);   // r_full: [epilogue warp][2]
+  uint64_t* rbar = r_full + 8;             // EPI_CONV_GN: [2] statistics from the cluster have arrived
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(rbar + 2);   // r_full: [epilogue warp][2]
   volatile uint32_t* abort_flag = tmem_holder + 1;
 
   // The warp index comes out of a shuffle so that the compiler knows it is the same in every
@@ -233,6 +257,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       mbar_init(&tmem_full[a], 1);
       mbar_init(&tmem_empty[a], (kEpiThreads / 32) * epi_groups(EPI, BN, CTA2) * (CTA2 ? 2 : 1));
       for (int w = 0; w < 4; ++w) mbar_init(&r_full[2 * w + a], 1);   // one per epilogue warp
+      mbar_init(&rbar[a], 1);
     }
     *abort_flag = 0;
     mbar_init_fence();
@@ -245,7 +270,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     else { tmem_alloc(tmem_holder, 2 * BN); tmem_relinquish(); }
   }
   tc_fence_before_sync();
-  if constexpr (CTA2) cluster_sync_all();   // the peer's barriers exist before anyone signals them
+  if constexpr (CTA2 || EPI == EPI_CONV_GN) cluster_sync_all();   // the peers' barriers exist before anyone signals them
   else __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_holder;
@@ -256,10 +281,10 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     {
       int s = 0; uint32_t ph = 0;
       for (int it = 0;; ++it) {
-        const int tile = sched_tile(p, cta, ncta, it);
+        const int tile = tile_at(it);
         if (tile < 0) break;
         int tm, tn, img = 0, h0 = 0, x0 = 0;
-        if constexpr (EPI == EPI_CONV) {
+        if constexpr (is_conv(EPI)) {
           tm = tile % p.tiles_m; tn = conv_pixel_tile(p, tile / p.tiles_m);   // output-channel tile, pixel tile
           img = tn / p.tiles_per_image;
           const int pt = tn % p.tiles_per_image;
@@ -282,7 +307,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               tma_load_2d_pair(sa, &tmA, &full[s], kb * kBK, tm * kTileM + static_cast<int>(rank) * kBM);
               tma_load_2d_pair(sb, &tmB, &full[s], kb * kBK, tn * BN + static_cast<int>(rank) * (BN / 2));
             }
-          } else if constexpr (EPI == EPI_CONV) {
+          } else if constexpr (is_conv(EPI)) {
             const int tap = kb / p.kb_per_tap, cb = kb % p.kb_per_tap;
             const int r = tap / 3, sx = tap % 3;
             if (elect_one()) {
@@ -311,11 +336,11 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // every lane waits (warp-uniform loop), one elected lane issues the MMAs and the commits
     if (rank == 0) {
       const uint32_t idesc =
-          umma_idesc_bf16_f32(kTileM, EPI == EPI_CONV ? static_cast<uint32_t>(p.tile_px) : BN);
+          umma_idesc_bf16_f32(kTileM, is_conv(EPI) ? static_cast<uint32_t>(p.tile_px) : BN);
       int s = 0; uint32_t ph = 0; int a = 0; uint32_t aph = 0;
       bool ok = true;
       for (int it = 0; ok; ++it) {
-        if (sched_tile(p, cta, ncta, it) < 0) break;
+        if (tile_at(it) < 0) break;
         ok = mbar_wait(&tmem_empty[a], aph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -406,10 +431,10 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     if constexpr (EPI == EPI_SOFTMAX) keep_policy = l2_policy_evict_last();
     [[maybe_unused]] float unit_sum = 0.0f;    // row sum carried across the tiles of a unit
     for (int it = 0; alive; ++it) {
-      const int tile = sched_tile(p, cta, ncta, it);
+      const int tile = tile_at(it);
       if (tile < 0) break;
       int tm, tn;
-      if constexpr (EPI == EPI_CONV) { tm = tile % p.tiles_m; tn = conv_pixel_tile(p, tile / p.tiles_m); }
+      if constexpr (is_conv(EPI)) { tm = tile % p.tiles_m; tn = conv_pixel_tile(p, tile / p.tiles_m); }
       else { tm = tile / p.tiles_n; tn = tile % p.tiles_n; }
       const int m_cta = tm * kTileM + row0;               // first row of this CTA's 128 rows
       const long long m = static_cast<long long>(m_cta) + row;
@@ -421,7 +446,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       // the accumulator so that the L2 latency is hidden, and staged in shared memory after it
       // (per piece every lane then reads the same 32 values: broadcast loads).
       [[maybe_unused]] float2 bpre = make_float2(0.0f, 0.0f);
-      if constexpr (EPI != EPI_CONV) {
+      if constexpr (!is_conv(EPI)) {
         const int n = n_tile + 2 * et;
         if (p.bias != nullptr && 2 * et < kGroupCols) {
           if (n < p.N) bpre.x = __bfloat162float(p.bias[n]);
@@ -436,7 +461,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       ok = named_barrier_and(bar_a, kEpiThreads, ok && !warp_failed);
       if (!ok) break;
       tc_fence_after_sync();
-      if constexpr (EPI != EPI_CONV) {
+      if constexpr (!is_conv(EPI)) {
         // every thread is past its last read of the previous tile's values (barrier above)
         if (2 * et < kGroupCols) *reinterpret_cast<float2*>(sbias + 2 * et) = bpre;
         named_barrier_sync(bar_b, kEpiThreads);
@@ -775,6 +800,107 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // left out of the statistics and are not stored
         const int px_valid = static_cast<int>(min(static_cast<long long>(p.tile_px), hw - px0));
         float s1 = 0.0f, s2 = 0.0f;
+        if constexpr (EPI == EPI_CONV_GN) {
+          // GroupNorm without a second kernel.  The CTAs of this cluster hold the tiles of one
+          // image, one each.  The accumulator stays in TMEM while (1) each epilogue group adds
+          // up its half of the tile per channel and, by shuffles, per GroupNorm group (sum, sum
+          // of squares), (2) sends those 32 pairs to every CTA of the cluster with bulk copies
+          // through distributed shared memory, which complete on the receiver's mbarrier, (3)
+          // waits (bounded) for the 2 x cluster-size contributions to its own inbox, adds them
+          // in a fixed order, and (4) reads the accumulator again, normalises and stores.
+          // Meanwhile the MMA warp fills the other accumulator.  Buffers alternate per tile; a
+          // CTA sends tile k+2 only after every peer has sent tile k+1, i.e. after every peer
+          // has finished reading tile k's buffers.
+          constexpr int kGP = kGroupCols / 32;                    // pieces per epilogue group
+          const int my_pieces = max(0, min(kGP, pieces - grp * kGP));
+          const int piece0 = grp * kGP;
+          const int buf = it & 1;
+          const int csize = p.gn_cluster;
+          const int cpg = p.N / p.gn_groups;                      // channels per group: 4, 8, 16 or 32
+          float2* sbuf = reinterpret_cast<float2*>(stg + C::kStaging + C::kBarBytes) + (buf * 2 + grp) * 32;
+          float2* inbox = reinterpret_cast<float2*>(stg + C::kStaging + C::kBarBytes + C::kBiasBytes);
+          uint8_t* yslab = stg + grp * kPieceBytes;               // the group's staging piece
+#pragma unroll 1
+          for (int c = 0; c < my_pieces; ++c) {
+            uint32_t v[32];
+            tmem_ld_32x32(t_acc + c * 32, v);
+            tmem_ld_wait();
+            const int left = px_valid - (piece0 + c) * 32;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + bias_v, p.act_rt);
+              float y1 = act_f<ACT, true>(__uint_as_float(v[2 * j + 1]) + bias_v, p.act_rt);
+              if (2 * j >= left) y0 = 0.0f;
+              if (2 * j + 1 >= left) y1 = 0.0f;
+              s1 += y0 + y1;
+              s2 = fmaf(y0, y0, fmaf(y1, y1, s2));
+            }
+          }
+          for (int o = cpg >> 1; o > 0; o >>= 1) {                // the group's channels: adjacent lanes
+            s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+            s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+          }
+          if ((row & (cpg - 1)) == 0) sbuf[row / cpg] = make_float2(s1, s2);
+          fence_proxy_async_smem();
+          named_barrier_sync(bar_b, kEpiThreads);
+          if (lead_warp) {
+            if (elect_one()) {
+              if (grp == 0) mbar_expect_tx(&rbar[buf], static_cast<uint32_t>(csize) * 2u * 256u);
+              const uint32_t dst = smem_u32(inbox + ((buf * 16 + static_cast<int>(crank)) * 2 + grp) * 32);
+              for (int r = 0; r < csize; ++r)
+                bulk_copy_to_peer(mapa_shared(dst, r), smem_u32(sbuf), 256u, mapa_shared(smem_u32(&rbar[buf]), r));
+            }
+          }
+          // every thread waits itself (it reads what the copies wrote), then one verdict for all
+          bool all_in = mbar_wait(&rbar[buf], static_cast<uint32_t>((it >> 1) & 1), abort_flag, p.status,
+                                  KF_DEV_TIMEOUT_EPILOGUE);
+          all_in = named_barrier_and(bar_a, kEpiThreads, all_in);
+          if (!all_in) break;
+          float sc = 0.0f, sh = 0.0f;
+          {
+            const float2* ib = inbox + buf * 16 * 2 * 32 + row / cpg;
+            float g1 = 0.0f, g2 = 0.0f;
+            for (int r = 0; r < 2 * csize; ++r) { const float2 q = ib[r * 32]; g1 += q.x; g2 += q.y; }
+            const float cnt = static_cast<float>(static_cast<long long>(cpg) * hw);
+            const float mu = g1 / cnt;
+            const float rstd = rsqrtf(fmaxf(g2 / cnt - mu * mu, 0.0f) + p.gn_eps);
+            const float ga = (p.gn_gamma != nullptr && ch_ok) ? __bfloat162float(p.gn_gamma[ch]) : 1.0f;
+            const float be = (p.gn_beta != nullptr && ch_ok) ? __bfloat162float(p.gn_beta[ch]) : 0.0f;
+            sc = rstd * ga;
+            sh = fmaf(-mu, sc, be);
+          }
+          if (my_pieces == 0) release_acc();
+#pragma unroll 1
+          for (int c = 0; c < my_pieces; ++c) {
+            uint32_t v[32];
+            tmem_ld_32x32(t_acc + c * 32, v);
+            tmem_ld_wait();
+            if (c == my_pieces - 1) release_acc();
+            uint32_t w[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + bias_v, p.act_rt);
+              const float y1 = act_f<ACT, true>(__uint_as_float(v[2 * j + 1]) + bias_v, p.act_rt);
+              w[j] = pack_bf16x2(fmaf(y0, sc, sh), fmaf(y1, sc, sh));
+            }
+            bulk_wait_group_read<0>();       // this warp's previous store has let go of the slab
+            __syncwarp();
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              *reinterpret_cast<uint4*>(yslab + piece_off(row, q)) =
+                  make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (elect_one()) {
+              if (px_valid - (piece0 + c) * 32 > 0 && tm * kBM + quad * 32 < p.N)
+                tma_store_3d(&tmY, yslab + quad * (kPieceBytes / 4), px0 + (piece0 + c) * 32,
+                             tm * kBM + quad * 32, img);
+              bulk_commit_group();
+            }
+          }
+          if (++a == 2) { a = 0; aph ^= 1u; }
+          continue;
+        }
         if (p.pool2 != 0) {
           // 2x2 pooling of a = act(z + b): the tile holds whole pairs of image rows, a 32-pixel
           // piece is a stretch of one row, so the thread combines the pieces at the same place
@@ -910,7 +1036,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     __syncthreads();
   }
   // a pair leaves together: the peer's MMAs read this CTA's shared memory and signal its barriers
-  if constexpr (CTA2) cluster_sync_all();
+  if constexpr (CTA2 || EPI == EPI_CONV_GN) cluster_sync_all();
   if (warp == 1) {
     __syncwarp();
     tc_fence_after_sync();

@@ -713,6 +713,31 @@ def test_groupnorm_biased_variance_on_gpu(kf):
     assert (got[0, 4:, 0, 0] == 0).all()
 
 
+# GroupNorm finished inside the convolution kernel: the CTAs holding one image's 2, 4, 8 or 16 pixel
+# tiles form a cluster and exchange the group statistics through distributed shared memory
+# (bf16, Cout <= 128, groups of 4..32 channels).
+@pytest.mark.parametrize("cfg", [
+    dict(Nb=3, Cin=64, H=8, W=64, Cout=128, groups=32),      # clusters of 2, groups of 4 channels
+    dict(Nb=2, Cin=32, H=28, W=28, Cout=96, groups=12),      # clusters of 4, ragged last tile, 96 of 128 channel rows
+    dict(Nb=2, Cin=16, H=32, W=64, Cout=64, groups=2),       # clusters of 8, groups of 32 channels
+    dict(Nb=9, Cin=64, H=64, W=64, Cout=128, groups=8),      # clusters of 16, more images than resident clusters
+])
+def test_conv_groupnorm_cluster_kernel(kf, cfg, monkeypatch):
+    d = ki.conv_inputs(seed=21, dtype="bf16", **cfg)
+    gamma = ki.store(ki.uniform(21, 7, (cfg["Cout"],), 0.5, 1.5), "bf16")
+    beta = ki.store(ki.uniform(21, 8, (cfg["Cout"],), -1.0, 1.0), "bf16")
+    for act, g_, b_ in (("relu", None, None), ("mish", gamma, beta)):
+        got, ref = run_conv(kf, d, act=act, gamma=g_, beta=b_)
+        assert_close(got, ref, 2e-2, 2e-2, "conv GN cluster %s %s" % (cfg, act))
+    # the two-kernel route on the same inputs: same statistics, activations rounded to bf16
+    # before instead of after the normalisation
+    fused, _ = run_conv(kf, d)
+    monkeypatch.setenv("KF_NO_FUSED_GN", "1")
+    two, ref = run_conv(kf, d)
+    assert_close(two, ref, 2e-2, 2e-2, "conv GN two kernels %s" % (cfg,))
+    assert (np.abs(fused - two) <= 2.0 ** -7 * np.maximum(1.0, np.abs(two))).all()      # two bf16 ulps
+
+
 # ------------------------------------------------------------------ conv -> activation -> global average pool
 @pytest.mark.parametrize("dtype,cfg", [
     ("bf16", dict(Nb=2, Cin=64, H=8, W=64, Cout=128)),      # means from the tensor-core epilogue

@@ -972,9 +972,16 @@ static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
       p.gn_beta = static_cast<const __nv_bfloat16*>(beta);
       p.partial = nullptr;
       p.num_tiles = static_cast<int>(Nb);          // the schedule counts images
-      if (launch_umma_conv_gn(bn, act, tm, p, static_cast<int>(Nb), st) != cudaSuccess) return KF_ERR_CUDA;
-      g_launches += launches + 1;
-      return KF_OK;
+      if (launch_umma_conv_gn(bn, act, tm, p, static_cast<int>(Nb), st) == cudaSuccess) {
+        g_launches += launches + 1;
+        return KF_OK;
+      }
+      // no cluster of that size can be resident here (or the launch was refused): clear the
+      // error and take the two-kernel route
+      (void)cudaGetLastError();
+      p.gn_cluster = 0; p.gn_groups = 0; p.gn_gamma = nullptr; p.gn_beta = nullptr;
+      p.partial = stats;
+      p.num_tiles = p.tiles_m * p.tiles_n;
     }
     const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
     if (launch_umma_conv(bn, act, tm, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;

@@ -92,7 +92,7 @@ struct UmmaParams {
   int tile_px;                 // pixels per tile = UMMA N (a multiple of 32, <= BN): rows_per_tile
                                // whole rows, or one of w_segs equal segments of a row
   int w_segs;                  // 1, or segments per row when Wd > 256 (then rows_per_tile = 1)
-  int gn_cluster;              // EPI_CONV_GN: CTAs per cluster = pixel tiles per image (2, 4, 8 or 16)
+  int gn_cluster;              // EPI_CONV_GN: CTAs per cluster = pixel tiles per image (1, 2, 4, 8 or 16)
   int gn_groups;               // EPI_CONV_GN: GroupNorm groups (channels per group a power of two, 4..32)
   int pool2;                   // convolution: 0, or 2x2 pooling in the epilogue (1 = max, 2 = mean);
                                // needs w_segs == 1, Wd % 32 == 0, rows_per_tile and H even
@@ -214,8 +214,8 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   if constexpr (CTA2) rank = cluster_ctarank();
   int cta = CTA2 ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
   int ncta = CTA2 ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
-  // EPI_CONV_GN: a cluster takes whole images (the schedule counts clusters and images), its CTA
-  // of rank r the r-th pixel tile of each
+  // EPI_CONV_GN: a cluster takes whole (image, channel tile) units (the schedule counts clusters
+  // and units), its CTA of rank r the r-th pixel tile of each
   [[maybe_unused]] uint32_t crank = 0;
   if constexpr (EPI == EPI_CONV_GN) {
     crank = cluster_ctarank();
@@ -224,8 +224,13 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   }
   auto tile_at = [&](int it) -> int {
     const int t = sched_tile(p, cta, ncta, it);
-    if constexpr (EPI == EPI_CONV_GN) return t < 0 ? t : t * p.gn_cluster + static_cast<int>(crank);
-    else return t;
+    if constexpr (EPI == EPI_CONV_GN) {
+      // unit t = (image, channel tile); this CTA takes the pixel tile of its rank
+      if (t < 0) return t;
+      return ((t / p.tiles_m) * p.gn_cluster + static_cast<int>(crank)) * p.tiles_m + t % p.tiles_m;
+    } else {
+      return t;
+    }
   };
   constexpr int kStages = C::kStages;
   extern __shared__ uint8_t smem_raw[];

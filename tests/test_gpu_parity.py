@@ -721,6 +721,8 @@ def test_groupnorm_biased_variance_on_gpu(kf):
     dict(Nb=2, Cin=32, H=28, W=28, Cout=96, groups=12),      # clusters of 4, ragged last tile, 96 of 128 channel rows
     dict(Nb=2, Cin=16, H=32, W=64, Cout=64, groups=2),       # clusters of 8, groups of 32 channels
     dict(Nb=9, Cin=64, H=64, W=64, Cout=128, groups=8),      # clusters of 16, more images than resident clusters
+    dict(Nb=4, Cin=64, H=16, W=16, Cout=256, groups=32),     # one tile per image and channel tile: no peers, two channel tiles
+    dict(Nb=3, Cin=32, H=14, W=14, Cout=160, groups=5),      # the same with a ragged second channel tile, groups of 32
 ])
 def test_conv_groupnorm_cluster_kernel(kf, cfg, monkeypatch):
     d = ki.conv_inputs(seed=21, dtype="bf16", **cfg)

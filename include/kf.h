@@ -196,8 +196,8 @@ kf_status kf_gemm_rowreduce_static(int64_t M, int64_t N, int64_t K, kf_dtype in_
  * two TF32 numbers each, as in kf_gemm_epilogue; GroupNorm by a two-pass kernel afterwards).
  * Everything else takes a scalar kernel.
  * GroupNorm: the tensor-core convolution leaves per-tile channel statistics and a second kernel
- * normalises in place; with Cout <= 128, 2, 4, 8 or 16 tiles per image and 4, 8, 16 or 32
- * channels per group (bf16, 16-byte aligned y, H*Wd % 8 == 0) the CTAs of an image form a
+ * normalises in place; with 1..8 or 16 tiles per image and 4, 8, 16 or 32 channels per group
+ * (bf16, 16-byte aligned y, H*Wd % 8 == 0) the CTAs of an image (and channel tile) form a
  * cluster, exchange the statistics through distributed shared memory and normalise inside the
  * convolution kernel: one kernel after the NHWC copy, the activations are written once.
  * groups must divide Cout. */

@@ -958,13 +958,13 @@ static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
     p.staged = (!gap_in_epilogue && aligned(y, 16) && hw % 8 == 0) ? 1 : 0;
     if (pool2 != 0) { p.pool2 = pool2; p.staged = 0; p.vec_ok = aligned(y, 16) ? 1 : 0; }
     if (p.staged && !encode_nchw_out(&tm.y, y, Nb, Cout, hw)) return KF_ERR_CUDA;
-    // GroupNorm inside the epilogue: an image's pixel tiles = one cluster of 1, 2, 4, 8 or 16
-    // CTAs (per channel tile), groups of 4..32 channels (a power of two: they never straddle a
+    // GroupNorm inside the epilogue: an image's pixel tiles = one cluster of 1..8 or 16 CTAs
+    // (per channel tile), groups of 4..32 channels (a power of two: they never straddle a
     // 128-channel tile), stores by TMA
     const int64_t cpg = groups > 0 ? Cout / groups : 0;
     const int tpi = p.tiles_per_image;
     const bool gn_fused = groups > 0 && p.staged &&
-                          (tpi == 1 || tpi == 2 || tpi == 4 || tpi == 8 || tpi == 16) &&
+                          tpi >= 1 && (tpi <= 8 || tpi == 16) &&      // 9..15 pack badly into GPCs (56x56: 43.6 us against 41.5)
                           (cpg == 4 || cpg == 8 || cpg == 16 || cpg == 32) &&
                           getenv("KF_NO_FUSED_GN") == nullptr;
     if (gn_fused) {

@@ -723,6 +723,8 @@ def test_groupnorm_biased_variance_on_gpu(kf):
     dict(Nb=9, Cin=64, H=64, W=64, Cout=128, groups=8),      # clusters of 16, more images than resident clusters
     dict(Nb=4, Cin=64, H=16, W=16, Cout=256, groups=32),     # one tile per image and channel tile: no peers, two channel tiles
     dict(Nb=3, Cin=32, H=14, W=14, Cout=160, groups=5),      # the same with a ragged second channel tile, groups of 32
+    dict(Nb=3, Cin=16, H=28, W=40, Cout=64, groups=8),       # clusters of 7 (four rows of 40 pixels per tile)
+    dict(Nb=4, Cin=16, H=6, W=96, Cout=32, groups=8),        # clusters of 3
 ])
 def test_conv_groupnorm_cluster_kernel(kf, cfg, monkeypatch):
     d = ki.conv_inputs(seed=21, dtype="bf16", **cfg)

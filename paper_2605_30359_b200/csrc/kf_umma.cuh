@@ -1,22 +1,25 @@
 // kf_umma.cuh -- the tensor-core mainloop shared by every bf16 chain, with its epilogues.
 //
 // One persistent CTA per SM walks output tiles of 128 rows x BN columns.  Warp roles:
-//   warp 0 (one lane)  TMA producer: fills a ring of shared-memory stages (A 128x64, B BNx64
+//   warp 0             TMA producer: fills a ring of shared-memory stages (A 128x64, B BNx64
 //                      bf16, 128-byte swizzle) and signals `full[s]` by transaction bytes.  For
 //                      the convolution A is the weight tile of one tap (rows = output channels)
 //                      and B the shifted window of BN pixels, so that the accumulator comes out
 //                      channel-major like the NCHW output.
-//   warp 1 (one lane)  UMMA issuer: four tcgen05.mma (K=16 each) per stage into one of two
+//   warp 1             UMMA issuer: four tcgen05.mma (K=16 each) per stage into one of two
 //                      TMEM accumulators, tcgen05.commit to `empty[s]` (stage free) and, after
 //                      the last K block, to `tmem_full[a]`.
-//   warps 2..5         epilogue: tcgen05.ld the accumulator (thread = one row of the tile),
-//                      apply the chain's epilogue in fp32 registers and release the accumulator
-//                      through `tmem_empty[a]` so the next tile's MMAs overlap.  Results leave
-//                      through shared-memory staging and TMA stores (the residual arrives the
-//                      same way, by TMA loads issued two pieces ahead): a row-per-lane global
-//                      access touches 32 cache lines per instruction and was measured to cost
-//                      the mainloop 10-15 % of its speed; a direct path remains for operands
-//                      whose alignment TMA cannot take.
+//                      In both warps every lane runs the loop and waits, a vote makes the outcome
+//                      warp-uniform and one elected lane issues (operands in uniform registers).
+//   warps 2..5 (and 6..9 where a second epilogue group runs: see epi_groups)
+//                      epilogue: tcgen05.ld the accumulator (thread = one row of the tile; a
+//                      group owns BN / groups columns), apply the chain's epilogue in fp32
+//                      registers and release the accumulator through `tmem_empty[a]` so the next
+//                      tile's MMAs overlap.  Results leave through shared-memory staging and TMA
+//                      stores (the residual arrives the same way): a row-per-lane global access
+//                      touches 32 cache lines per instruction and was measured to cost the
+//                      mainloop 10-15 % of its speed; a direct path remains for operands whose
+//                      alignment TMA cannot take.
 // Every wait is bounded (mbar_wait); a wait that runs out raises the CTA's abort flag, all
 // roles leave their loops, in-flight copies are given time to land, TMEM is freed.
 #pragma once
@@ -35,7 +38,7 @@ constexpr bool is_conv(int epi) { return epi == 3 || epi == 4; }
 constexpr int kBM = 128;          // tile rows = UMMA M = TMEM lanes
 constexpr int kBK = 64;           // K per stage: 64 bf16 = one 128-byte swizzled row
 constexpr int kUmmaK = 16;        // K per tcgen05.mma for 16-bit inputs
-constexpr int kEpiThreads = 128;  // warps 2..5: one per TMEM lane quarter
+constexpr int kEpiThreads = 128;  // threads of one epilogue group: four warps, one per TMEM lane quarter
 constexpr int kNumThreads = 192;  // 6 warps: producer, UMMA issuer, epilogue
 // The softmax epilogue is the longest (two TMEM passes, an exponential per element) and with
 // one warp per scheduler it is latency-bound, so it runs as TWO groups of four warps, each
@@ -383,7 +386,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------ epilogue (warps 2..5, and 6..9 with two groups)
     constexpr int kGroups = epi_groups(EPI, BN, CTA2);
     constexpr int NB = 2 / kGroups;            // elementwise: staging buffers per group (4 pieces in all)
     constexpr int kGroupCols = BN / kGroups;   // columns of the tile one epilogue group owns
@@ -393,7 +396,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const int quad = warp & 3;                 // TMEM lane quarter this warp may read
     const int row = quad * 32 + lane;          // row of the tile = TMEM lane
     const int et = threadIdx.x - 64 - grp * kEpiThreads;   // 0..127 inside the group
-    const bool leader = et == 0;               // issues the group's TMA loads and stores
+    const bool leader = et == 0;               // polls for the group; issues the whole-piece TMA stores where those are used
     [[maybe_unused]] const bool lead_warp = warp == 2 + 4 * grp;   // its warp (a warp-uniform predicate)
     const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
     [[maybe_unused]] uint8_t* ybuf = stg + grp * 2 * kPieceBytes;   // [2][kPieceBytes] output pieces

@@ -1031,7 +1031,9 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       }
       if (++a == 2) { a = 0; aph ^= 1u; }
     }
-    bulk_wait_group<0>();          // every output store has completed (a no-op in lanes that issued none)
+    // every output store has finished reading shared memory (a no-op in lanes that issued none);
+    // the writes themselves complete with the kernel, like any store in flight at exit
+    bulk_wait_group_read<0>();
   }
 
   // ---------------------------------------------------------------- teardown

@@ -122,3 +122,41 @@ def test_conv_softmax_pool_full_size_sampled_images(kf):
     assert_close(got, ref, 1e-6, 2e-2, "conv softmax pool sampled images, relative")
     yy = y.float()
     assert float(yy.min()) > 0 and float(yy.max()) <= 1.0
+
+
+def test_short_k_chain_full_size_sampled_rows(kf):
+    """4096x4096x512 + bias + GELU*0.5 + residual: the single-CTA kernel with two epilogue groups
+    and per-warp slabs, several waves, epilogue-bound."""
+    d = ki.gemm_inputs("c2", seed=5, M=4096, N=4096, K=512)
+    Y = kf.gemm_epilogue(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "gelu_tanh", 0.5, to_dev(d["R"]))
+    check_status()
+    rows = sample_rows(4096, 48, 6)
+    ref = oracle.gemm_epilogue(d["X"][rows], d["W"], d["b"], "gelu_tanh", 0.5, d["R"][rows])
+    assert_close(to_f64(Y[rows]), ref, 2e-2, 2e-2, "short-K chain sampled rows")
+    import torch
+    assert torch.isfinite(Y).all()
+    assert float((Y.float() - to_dev(d["R"]).float()).min()) > -0.12
+
+
+def test_conv_act_pool_full_size_sampled_images(kf):
+    """conv + ReLU + max-pool 2 on config 5's tensors: pooled inside the convolution epilogue."""
+    d = ki.conv_inputs("c5", seed=0)
+    y = kf.conv3x3_act_pool(to_dev(d["x"]), to_dev(d["w"]), to_dev(d["bias"]), "relu", "max", 2)
+    check_status()
+    assert tuple(y.shape) == (128, 128, 32, 32)
+    imgs = [0, 63, 127]
+    ref = oracle.conv3x3_act_pool(d["x"][imgs], d["w"], d["bias"], "relu", "max", 2)
+    assert_close(to_f64(y[imgs]), ref, 2e-2, 2e-2, "conv relu max-pool sampled images")
+    assert float(y.float().min()) >= 0.0
+
+
+def test_c5_two_kernel_route_full_size_sampled_images(kf, monkeypatch):
+    """Config 5 through the convolution + separate normalisation kernels (the route shapes take
+    that do not qualify for the cluster form)."""
+    monkeypatch.setenv("KF_NO_FUSED_GN", "1")
+    d = ki.conv_inputs("c5", seed=0)
+    y = kf.conv3x3_epilogue(to_dev(d["x"]), to_dev(d["w"]), to_dev(d["bias"]), "relu", d["groups"], d["eps"])
+    check_status()
+    imgs = [0, 77, 127]
+    ref = oracle.conv3x3_gn(d["x"][imgs], d["w"], d["bias"], "relu", d["groups"], d["eps"], None, None)
+    assert_close(to_f64(y[imgs]), ref, 2e-2, 2e-2, "c5 two-kernel route sampled images")

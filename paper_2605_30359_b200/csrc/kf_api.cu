@@ -307,14 +307,29 @@ int env_int(const char* name, int dflt) {
 // blocks (K = 1536: 9.9 us split, 8.9 us plain; K = 2048: 9.4 against 10.7 us); clusters of 8 schedule well only while there are few
 // of them (16 clusters of 8 already ran in two waves).
 int pick_split_k(int64_t M, int64_t N, int64_t K, int sm_count, int* bn_out) {
+  *bn_out = N <= 128 ? 128 : 256;
   if (getenv("KF_NO_SPLITK") != nullptr) return 0;
-  const int bn = N <= 128 ? 128 : 256;
-  const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + bn - 1) / bn);
   const int64_t kb = (K + kBK - 1) / kBK;
-  *bn_out = bn;
   if (kb < env_int("KF_SPLITK_MIN_KB", 28)) return 0;
-  if (bn == 256 && kb >= 32 && tiles * 8 <= 64) return 8;
-  if (tiles * 4 <= sm_count - sm_count % 4) return 4;
+  // cluster size for tiles of `bn` columns, and the CTAs that gives
+  auto split_for = [&](int bn, int64_t* ctas) {
+    const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + bn - 1) / bn);
+    int sk = 0;
+    if (bn == 256 && kb >= 32 && tiles * 8 <= 64) sk = 8;
+    else if (tiles * 4 <= sm_count - sm_count % 4) sk = 4;
+    else if (bn == 128 && tiles * 2 <= sm_count - sm_count % 2) sk = 2;
+    *ctas = tiles * sk;
+    return sk;
+  };
+  int64_t c256 = 0, c128 = 0;
+  const int s256 = N > 128 ? split_for(256, &c256) : 0;
+  const int s128 = split_for(128, &c128);
+  // the width that occupies more SMs; 256 columns on a tie (128x4096x8192: 64 CTAs of 256
+  // columns 21.0 us, 128 CTAs of 128 columns 16.4 us; 64x8192x8192: 128 CTAs either way,
+  // 32.9 us at 256 columns, 35.5 us at 128)
+  if (s128 != 0 && c128 > c256) { *bn_out = 128; return s128; }
+  if (s256 != 0) { *bn_out = 256; return s256; }
+  if (s128 != 0) { *bn_out = 128; return s128; }
   return 0;
 }
 

@@ -806,8 +806,11 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
           cudaSuccess)
         return KF_ERR_CUDA;
     } else if (red == KF_RED_SOFTMAX) {
+      // a row that lies in one tile is finished in the GEMM epilogue: no second kernel
+      p.softmax_fused = (p.tiles_n == 1 && getenv("KF_NO_FUSED_SOFTMAX") == nullptr) ? 1 : 0;
       if (launch_umma_softmax(bn, pre_act, out_dtype, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
         return KF_ERR_CUDA;
+      if (p.softmax_fused) { g_launches += 1; return KF_OK; }
       if (launch_softmax_finalize(out_dtype, Mi, Ni, bn / 2, 2 * p.tiles_n, p.partial, out, ldo, p.vec_ok, st) !=
           cudaSuccess)
         return KF_ERR_CUDA;

@@ -95,6 +95,7 @@ struct UmmaParams {
   int tile_px;                 // pixels per tile = UMMA N (a multiple of 32, <= BN): rows_per_tile
                                // whole rows, or one of w_segs equal segments of a row
   int w_segs;                  // 1, or segments per row when Wd > 256 (then rows_per_tile = 1)
+  int softmax_fused;           // EPI_SOFTMAX: the row lies in one tile (tiles_n == 1): finish it in the epilogue
   int gn_cluster;              // EPI_CONV_GN: CTAs per cluster = pixel tiles per image (1, 2, 4, 8 or 16)
   int gn_groups;               // EPI_CONV_GN: GroupNorm groups (channels per group a power of two, 4..32)
   int pool2;                   // convolution: 0, or 2x2 pooling in the epilogue (1 = max, 2 = mean);
@@ -667,10 +668,32 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if (c * 32 + j < n_valid) mx = fmaxf(mx, z);
           }
         }
+        // A row that lies in this one tile (tiles_n == 1) is finished here: the two groups
+        // exchange their maxima and their sums through shared memory (five barriers over both
+        // groups per tile), a third pass over the accumulator stores the probabilities, and no
+        // second kernel runs.  phase 0: the two-kernel form; 1: sum only; 2: scaled stores.
+        const bool whole_row = p.softmax_fused != 0;
+        float* xch = reinterpret_cast<float*>(stg);                   // [2 groups][128 rows], in staging
+        if (whole_row) {
+          bulk_wait_group_read<0>();               // the previous tile's stores have let go of staging ...
+          named_barrier_sync(5u, kGroups * kEpiThreads);         // ... in both groups
+          xch[grp * kEpiThreads + et] = mx;
+          named_barrier_sync(5u, kGroups * kEpiThreads);
+          mx = fmaxf(mx, xch[(grp ^ 1) * kEpiThreads + et]);
+          named_barrier_sync(5u, kGroups * kEpiThreads);         // both maxima read: the slots are reused
+        }
         // pass 2: numerators e = exp(a - mx), their fp32 sum, e stored in the output dtype
         // (statistics-only runs skip the stores; a maximum-only run skips the pass)
         OutT* P = reinterpret_cast<OutT*>(p.out);
         float sum = 0.0f;
+        float inv = 1.0f;
+        for (int phase = whole_row ? 1 : 0; phase <= (whole_row ? 2 : 0); ++phase) {
+        if (phase == 2) {
+          xch[grp * kEpiThreads + et] = sum;
+          named_barrier_sync(5u, kGroups * kEpiThreads);
+          inv = 1.0f / (xch[et] + xch[kEpiThreads + et]);           // group 0 + group 1: fixed order
+          named_barrier_sync(5u, kGroups * kEpiThreads);         // read before staging is written again
+        }
 #pragma unroll 1
         for (int c = 0; c < PIECES && p.stats_only != 2; ++c, ++g) {
           if (!staged && c * 32 >= n_valid) break;
@@ -679,15 +702,15 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           float bs[32];
           load_sbias32(sbias + c * 32, bs);
           tmem_ld_wait();
-          if (staged && c == PIECES - 1) release_acc();
+          if (staged && c == PIECES - 1 && phase != 1) release_acc();
           float f[32];
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
-            f[j] = __expf(z - mx);
-            if (c * 32 + j < n_valid) sum += f[j];
+            f[j] = __expf(z - mx) * inv;
+            if (phase != 2 && c * 32 + j < n_valid) sum += f[j];
           }
-          if (p.stats_only != 0) continue;
+          if (p.stats_only != 0 || phase == 1) continue;
           if constexpr (sizeof(OutT) == 2) {
             if (staged) {
               const int b = static_cast<int>(g & 1);
@@ -760,8 +783,9 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
           }
         }
+        }   // phase
         if (!staged) release_acc();
-        if (row_ok) {
+        if (row_ok && !whole_row) {
           float2* part = reinterpret_cast<float2*>(p.partial);
           part[(m * p.tiles_n + tn) * kGroups + grp] = make_float2(mx, sum);
         }

@@ -528,6 +528,39 @@ def test_gemm_groupnorm(kf, dtype, shape, groups, monkeypatch):
     assert np.abs(blk.var(axis=2) - 1.0).max() < (5e-2 if dtype == "bf16" else 1e-3)
 
 
+# Rows that lie in one tile (N <= 256, or <= 64 on the narrow-tile kernel): the softmax is finished
+# inside the GEMM epilogue (maxima and sums exchanged between the two epilogue groups), no second
+# kernel runs.
+@pytest.mark.parametrize("shape", [(20000, 256, 64), (19000, 200, 264), (4096, 136, 64), (129, 64, 128),
+                                   (77, 40, 72), (5120, 256, 2048), (19500, 250, 72), (128, 8, 64),
+                                   (300, 256, 512)])
+def test_bf16_softmax_whole_row_in_one_tile(kf, shape, monkeypatch):
+    M, N, K = shape
+    d = ki.gemm_inputs("c3", seed=41, M=M, N=N, K=K)
+    args = (to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]))
+    before = kf.kf_launch_count()
+    P = kf.gemm_rowreduce(*args, "relu", "softmax")
+    launches = kf.kf_launch_count() - before
+    check_status()
+    ref = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "relu", "softmax")
+    got = to_f64(P)
+    assert_close(got, ref, 2e-2, 2e-2, "softmax in one tile %s" % (shape,))
+    assert np.abs(got.sum(axis=1) - 1.0).max() < 1e-2
+    # 64-column tiles when they fit in one wave, else 256-column tiles; one tile per row = one kernel
+    bn = 64 if ((M + 127) // 128) * ((N + 63) // 64) <= 148 else 256
+    assert launches == (1 if N <= bn else 2)
+    # the two-kernel route gives the same probabilities up to the rounding of the numerators
+    monkeypatch.setenv("KF_NO_FUSED_SOFTMAX", "1")
+    P2 = to_f64(kf.gemm_rowreduce(*args, "relu", "softmax"))
+    assert np.abs(P2 - got).max() <= 2.0 ** -7 * max(1e-30, got.max())
+    # fp32 probabilities from the same kernel family
+    monkeypatch.delenv("KF_NO_FUSED_SOFTMAX")
+    import torch
+    P32 = kf.gemm_rowreduce(*args, "relu", "softmax", out_dtype=torch.float32)
+    check_status()
+    assert_close(to_f64(P32), ref, 2e-2, 2e-2, "softmax in one tile, fp32 out %s" % (shape,))
+
+
 # ------------------------------------------------------------------ seeded shape fuzz across the dispatch rules
 def _fuzz_shapes(seed, count):
     """bf16 GEMM shapes around the dispatch boundaries: tile widths 32..256, one or two epilogue

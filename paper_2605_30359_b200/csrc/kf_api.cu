@@ -806,6 +806,21 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
           cudaSuccess)
         return KF_ERR_CUDA;
     } else if (red == KF_RED_SOFTMAX) {
+      // 2..16 narrow column tiles per row: the CTAs that hold a row block's tiles form a cluster,
+      // exchange (maximum, sum) per row through distributed shared memory and store final
+      // probabilities: one kernel
+      if (bn == kRowReduceNarrowBN && p.tiles_n >= 2 && p.tiles_n <= 16 &&
+          getenv("KF_NO_CLUSTER_SOFTMAX") == nullptr) {
+        UmmaParams pc = p;
+        pc.gn_cluster = p.tiles_n;
+        pc.num_tiles = p.tiles_m;            // the schedule counts row blocks
+        pc.tiles_per_unit = 1;
+        if (launch_umma_softmax_cluster(pre_act, out_dtype, tm, pc, p.tiles_m, st) == cudaSuccess) {
+          g_launches += 1;
+          return KF_OK;
+        }
+        (void)cudaGetLastError();            // no such cluster can be resident: the two-kernel route
+      }
       // a row that lies in one tile is finished in the GEMM epilogue: no second kernel
       p.softmax_fused = (p.tiles_n == 1 && getenv("KF_NO_FUSED_SOFTMAX") == nullptr) ? 1 : 0;
       if (launch_umma_softmax(bn, pre_act, out_dtype, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)

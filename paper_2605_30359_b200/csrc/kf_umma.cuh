@@ -32,8 +32,14 @@ namespace kf {
 // EPI_CONV_GN: the convolution with GroupNorm finished inside the epilogue; the CTAs that hold
 // the tiles of one image form a cluster and exchange the group statistics through distributed
 // shared memory (two epilogue groups).
-enum : int { EPI_ELEMENTWISE = 0, EPI_SOFTMAX = 1, EPI_ROWSUM = 2, EPI_CONV = 3, EPI_CONV_GN = 4 };
+// EPI_SOFTMAX_CL: the softmax of a row whose column tiles are held by the CTAs of one cluster: the
+// per-row (maximum, sum) pairs travel through distributed shared memory and every CTA stores
+// final probabilities (one kernel, no second pass).
+enum : int { EPI_ELEMENTWISE = 0, EPI_SOFTMAX = 1, EPI_ROWSUM = 2, EPI_CONV = 3, EPI_CONV_GN = 4,
+             EPI_SOFTMAX_CL = 5 };
 constexpr bool is_conv(int epi) { return epi == 3 || epi == 4; }
+constexpr bool is_softmax(int epi) { return epi == 1 || epi == 5; }
+constexpr bool is_cluster_epi(int epi) { return epi == 4 || epi == 5; }
 
 constexpr int kBM = 128;          // tile rows = UMMA M = TMEM lanes
 constexpr int kBK = 64;           // K per stage: 64 bf16 = one 128-byte swizzled row
@@ -51,7 +57,7 @@ constexpr int kNumThreads = 192;  // 6 warps: producer, UMMA issuer, epilogue
 // The CTA-pair form (large K only: its epilogue hides behind the MMAs anyway, and the extra warps
 // cost it 2 %) keeps one group.
 constexpr int epi_groups(int epi, int bn, bool cta2) {
-  return epi == 1 /* EPI_SOFTMAX */ || epi == 4 /* EPI_CONV_GN */ ||
+  return epi == 1 /* EPI_SOFTMAX */ || epi == 4 /* EPI_CONV_GN */ || epi == 5 /* EPI_SOFTMAX_CL */ ||
                  (epi == 0 /* EPI_ELEMENTWISE */ && bn >= 64 && !cta2)
              ? 2 : 1;
 }
@@ -96,7 +102,8 @@ struct UmmaParams {
                                // whole rows, or one of w_segs equal segments of a row
   int w_segs;                  // 1, or segments per row when Wd > 256 (then rows_per_tile = 1)
   int softmax_fused;           // EPI_SOFTMAX: the row lies in one tile (tiles_n == 1): finish it in the epilogue
-  int gn_cluster;              // EPI_CONV_GN: CTAs per cluster = pixel tiles per image (1, 2, 4, 8 or 16)
+  int gn_cluster;              // EPI_CONV_GN: CTAs per cluster = pixel tiles per image (1..8 or 16);
+                               // EPI_SOFTMAX_CL: CTAs per cluster = column tiles per row (2..16)
   int gn_groups;               // EPI_CONV_GN: GroupNorm groups (channels per group a power of two, 4..32)
   int pool2;                   // convolution: 0, or 2x2 pooling in the epilogue (1 = max, 2 = mean);
                                // needs w_segs == 1, Wd % 32 == 0, rows_per_tile and H even
@@ -129,13 +136,15 @@ struct UmmaCfg {
   // staging: elementwise = 2 output + 2 residual pieces; softmax = 2 output pieces per epilogue
   // group; conv = 2 output pieces
   static constexpr int kStaging =
-      EPI == EPI_ELEMENTWISE || EPI == EPI_SOFTMAX ? 4 * kPieceBytes
+      EPI == EPI_ELEMENTWISE || is_softmax(EPI) ? 4 * kPieceBytes
                                                     : (EPI == EPI_ROWSUM ? 0 : 2 * kPieceBytes);     // EPI_CONV_GN: one piece per epilogue group
   static constexpr int kBarBytes = 256;
   // GEMM epilogues: the tile's BN bias values as fp32, staged once per tile
   static constexpr int kBiasBytes = EPI == EPI_CONV ? 0 : BN * 4;   // EPI_CONV_GN: the statistics it sends
   // EPI_CONV_GN: statistics arriving from the cluster, [2 buffers][16 CTAs x 2 groups][32 x float2]
-  static constexpr int kInboxBytes = EPI == EPI_CONV_GN ? 2 * 32 * 256 : 0;
+  // EPI_SOFTMAX_CL: [2 buffers][16 CTAs x 2 groups][128 rows x float2] arriving, then the
+  // [2 buffers][2 groups][128 x float2] it sends
+  static constexpr int kInboxBytes = EPI == EPI_CONV_GN ? 2 * 32 * 256 : (EPI == EPI_SOFTMAX_CL ? 2 * 32 * 1024 + 4 * 1024 : 0);
   static constexpr int kFit = (kMaxDynSmem - 1024 - kStaging - kBarBytes - kBiasBytes - kInboxBytes) / kStage;
   static constexpr int kStages = kFit > 8 ? 8 : kFit;
   static constexpr int kRing = kStage * kStages;
@@ -221,7 +230,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   // EPI_CONV_GN: a cluster takes whole (image, channel tile) units (the schedule counts clusters
   // and units), its CTA of rank r the r-th pixel tile of each
   [[maybe_unused]] uint32_t crank = 0;
-  if constexpr (EPI == EPI_CONV_GN) {
+  if constexpr (is_cluster_epi(EPI)) {
     crank = cluster_ctarank();
     cta = static_cast<int>(blockIdx.x) / p.gn_cluster;
     ncta = static_cast<int>(gridDim.x) / p.gn_cluster;
@@ -232,6 +241,9 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       // unit t = (image, channel tile); this CTA takes the pixel tile of its rank
       if (t < 0) return t;
       return ((t / p.tiles_m) * p.gn_cluster + static_cast<int>(crank)) * p.tiles_m + t % p.tiles_m;
+    } else if constexpr (EPI == EPI_SOFTMAX_CL) {
+      // unit t = row block; this CTA takes the column tile of its rank (tiles_n == cluster size)
+      return t < 0 ? t : t * p.gn_cluster + static_cast<int>(crank);
     } else {
       return t;
     }
@@ -279,7 +291,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     else { tmem_alloc(tmem_holder, 2 * BN); tmem_relinquish(); }
   }
   tc_fence_before_sync();
-  if constexpr (CTA2 || EPI == EPI_CONV_GN) cluster_sync_all();   // the peers' barriers exist before anyone signals them
+  if constexpr (CTA2 || is_cluster_epi(EPI)) cluster_sync_all();   // the peers' barriers exist before anyone signals them
   else __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_holder;
@@ -437,7 +449,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     bool alive = true;
     bool warp_failed = false;    // this warp gave up on one of its own waits inside a tile
     [[maybe_unused]] uint64_t keep_policy = 0;
-    if constexpr (EPI == EPI_SOFTMAX) keep_policy = l2_policy_evict_last();
+    if constexpr (is_softmax(EPI)) keep_policy = l2_policy_evict_last();
     [[maybe_unused]] float unit_sum = 0.0f;    // row sum carried across the tiles of a unit
     for (int it = 0; alive; ++it) {
       const int tile = tile_at(it);
@@ -651,7 +663,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
           release_acc();
         }
-      } else if constexpr (EPI == EPI_SOFTMAX) {
+      } else if constexpr (is_softmax(EPI)) {
         // pass 1: tile maximum of a = pre_act(z + b) over the valid columns of this row
         float mx = -INFINITY;
 #pragma unroll 1
@@ -672,9 +684,10 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // exchange their maxima and their sums through shared memory (five barriers over both
         // groups per tile), a third pass over the accumulator stores the probabilities, and no
         // second kernel runs.  phase 0: the two-kernel form; 1: sum only; 2: scaled stores.
-        const bool whole_row = p.softmax_fused != 0;
+        constexpr bool kCl = EPI == EPI_SOFTMAX_CL;
+        const bool whole_row = kCl || p.softmax_fused != 0;
         float* xch = reinterpret_cast<float*>(stg);                   // [2 groups][128 rows], in staging
-        if (whole_row) {
+        if (whole_row && !kCl) {
           bulk_wait_group_read<0>();               // the previous tile's stores have let go of staging ...
           named_barrier_sync(5u, kGroups * kEpiThreads);         // ... in both groups
           xch[grp * kEpiThreads + et] = mx;
@@ -688,11 +701,46 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         float sum = 0.0f;
         float inv = 1.0f;
         for (int phase = whole_row ? 1 : 0; phase <= (whole_row ? 2 : 0); ++phase) {
-        if (phase == 2) {
+        if (phase == 2 && !kCl) {
           xch[grp * kEpiThreads + et] = sum;
           named_barrier_sync(5u, kGroups * kEpiThreads);
           inv = 1.0f / (xch[et] + xch[kEpiThreads + et]);           // group 0 + group 1: fixed order
           named_barrier_sync(5u, kGroups * kEpiThreads);         // read before staging is written again
+        }
+        if constexpr (kCl) {
+          if (phase == 2) {
+            // This group's (maximum, sum of exp(a - maximum)) per row goes to every CTA of the
+            // cluster (bulk copies through distributed shared memory, completing on the
+            // receiver's mbarrier); from the 2 x cluster-size pairs that arrive here every
+            // thread forms its row's maximum M and denominator S = sum s_i * exp(m_i - M) in a
+            // fixed order.  Buffers alternate per tile (see EPI_CONV_GN for why two suffice).
+            const int buf = it & 1;
+            const int csize = p.gn_cluster;
+            float2* inbox = reinterpret_cast<float2*>(stg + C::kStaging + C::kBarBytes + C::kBiasBytes);
+            float2* sbuf = inbox + 2 * 32 * 128 + (buf * 2 + grp) * 128;
+            sbuf[et] = make_float2(mx, sum);
+            fence_proxy_async_smem();
+            named_barrier_sync(bar_b, kEpiThreads);
+            if (lead_warp) {
+              if (elect_one()) {
+                if (grp == 0) mbar_expect_tx(&rbar[buf], static_cast<uint32_t>(csize) * 2u * 1024u);
+                const uint32_t dst = smem_u32(inbox + ((buf * 16 + static_cast<int>(crank)) * 2 + grp) * 128);
+                for (int r = 0; r < csize; ++r)
+                  bulk_copy_to_peer(mapa_shared(dst, r), smem_u32(sbuf), 1024u, mapa_shared(smem_u32(&rbar[buf]), r));
+              }
+            }
+            bool all_in = mbar_wait(&rbar[buf], static_cast<uint32_t>((it >> 1) & 1), abort_flag, p.status,
+                                    KF_DEV_TIMEOUT_EPILOGUE);
+            all_in = named_barrier_and(bar_a, kEpiThreads, all_in);
+            if (!all_in) { alive = false; break; }
+            const float2* ib = inbox + buf * 32 * 128 + et;
+            float big = -INFINITY;
+            for (int r = 0; r < 2 * csize; ++r) big = fmaxf(big, ib[r * 128].x);
+            float den = 0.0f;
+            for (int r = 0; r < 2 * csize; ++r) { const float2 q = ib[r * 128]; den += q.y * __expf(q.x - big); }
+            mx = big;
+            inv = 1.0f / den;
+          }
         }
 #pragma unroll 1
         for (int c = 0; c < PIECES && p.stats_only != 2; ++c, ++g) {
@@ -784,6 +832,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
         }
         }   // phase
+        if (!alive) break;
         if (!staged) release_acc();
         if (row_ok && !whole_row) {
           float2* part = reinterpret_cast<float2*>(p.partial);
@@ -1070,7 +1119,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     __syncthreads();
   }
   // a pair leaves together: the peer's MMAs read this CTA's shared memory and signal its barriers
-  if constexpr (CTA2 || EPI == EPI_CONV_GN) cluster_sync_all();
+  if constexpr (CTA2 || is_cluster_epi(EPI)) cluster_sync_all();
   if (warp == 1) {
     __syncwarp();
     tc_fence_after_sync();

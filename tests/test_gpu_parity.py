@@ -533,8 +533,11 @@ def test_gemm_groupnorm(kf, dtype, shape, groups, monkeypatch):
 # kernel runs.
 @pytest.mark.parametrize("shape", [(20000, 256, 64), (19000, 200, 264), (4096, 136, 64), (129, 64, 128),
                                    (77, 40, 72), (5120, 256, 2048), (19500, 250, 72), (128, 8, 64),
-                                   (300, 256, 512)])
-def test_bf16_softmax_whole_row_in_one_tile(kf, shape, monkeypatch):
+                                   (300, 256, 512),          # clusters of 4 column tiles
+                                   (1000, 1000, 304),        # clusters of 16, ragged last tile (1000 = 15.6 x 64)
+                                   (2500, 136, 1024),        # clusters of 3, more row blocks than resident clusters
+                                   (128, 1024, 2048)])       # clusters of 16 x 32 K blocks
+def test_bf16_softmax_one_kernel(kf, shape, monkeypatch):
     M, N, K = shape
     d = ki.gemm_inputs("c3", seed=41, M=M, N=N, K=K)
     args = (to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]))
@@ -546,15 +549,18 @@ def test_bf16_softmax_whole_row_in_one_tile(kf, shape, monkeypatch):
     got = to_f64(P)
     assert_close(got, ref, 2e-2, 2e-2, "softmax in one tile %s" % (shape,))
     assert np.abs(got.sum(axis=1) - 1.0).max() < 1e-2
-    # 64-column tiles when they fit in one wave, else 256-column tiles; one tile per row = one kernel
+    # 64-column tiles when they fit in one wave, else 256-column tiles.  One kernel when a row
+    # lies in one tile, or in 2..16 narrow tiles (their CTAs form a cluster); else two.
     bn = 64 if ((M + 127) // 128) * ((N + 63) // 64) <= 148 else 256
-    assert launches == (1 if N <= bn else 2)
+    assert launches == (1 if (N <= bn or (bn == 64 and (N + 63) // 64 <= 16)) else 2)
     # the two-kernel route gives the same probabilities up to the rounding of the numerators
     monkeypatch.setenv("KF_NO_FUSED_SOFTMAX", "1")
+    monkeypatch.setenv("KF_NO_CLUSTER_SOFTMAX", "1")
     P2 = to_f64(kf.gemm_rowreduce(*args, "relu", "softmax"))
     assert np.abs(P2 - got).max() <= 2.0 ** -7 * max(1e-30, got.max())
     # fp32 probabilities from the same kernel family
     monkeypatch.delenv("KF_NO_FUSED_SOFTMAX")
+    monkeypatch.delenv("KF_NO_CLUSTER_SOFTMAX")
     import torch
     P32 = kf.gemm_rowreduce(*args, "relu", "softmax", out_dtype=torch.float32)
     check_status()

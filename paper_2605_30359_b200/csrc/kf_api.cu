@@ -809,8 +809,11 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
       // 2..16 narrow column tiles per row: the CTAs that hold a row block's tiles form a cluster,
       // exchange (maximum, sum) per row through distributed shared memory and store final
       // probabilities: one kernel
+      // (only while every row block's cluster is resident at once: 7 clusters of 16, 15 of 8, 33
+      // of 4 fit on the GPU; 1024^3, eight row blocks of 16 tiles, took 19.1 us in two rounds
+      // against 17.0 us for the two-kernel route)
       if (bn == kRowReduceNarrowBN && p.tiles_n >= 2 && p.tiles_n <= 16 &&
-          getenv("KF_NO_CLUSTER_SOFTMAX") == nullptr) {
+          static_cast<int64_t>(p.tiles_m) * p.tiles_n <= 112 && getenv("KF_NO_CLUSTER_SOFTMAX") == nullptr) {
         UmmaParams pc = p;
         pc.gn_cluster = p.tiles_n;
         pc.num_tiles = p.tiles_m;            // the schedule counts row blocks

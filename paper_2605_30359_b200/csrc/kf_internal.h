@@ -2,6 +2,7 @@
 // that instantiate the kernels.  Every launcher enqueues on `st` and returns the launch's
 // cudaError_t; none synchronises.
 #pragma once
+#include <cstdlib>
 
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -197,8 +198,20 @@ inline cudaError_t launch_umma_instance(const UmmaMaps& tm, const UmmaParams& p,
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kern, tm.a, tm.b, tm.r, tm.y, p);
   } else {
-    kern<<<grid, num_threads(EPI, BN, CTA2), smem, st>>>(tm.a, tm.b, tm.r, tm.y, p);
-    return cudaGetLastError();
+    // programmatic dependent launch: with few CTAs the next launch of the stream starts on the
+    // idle SMs and has its prologue behind it when this kernel ends (see griddep_wait)
+    static const bool pdl = getenv("KF_NO_PDL") == nullptr;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(num_threads(EPI, BN, CTA2), 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, tm.a, tm.b, tm.r, tm.y, p);
   }
 }
 

@@ -300,6 +300,11 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   else __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_holder;
+  // Everything above touched only this CTA's shared memory, TMEM and parameters.  A launch that
+  // was allowed to start early waits here for the kernel before it; the kernel after this one
+  // may start its own prologue now.
+  griddep_wait();
+  griddep_launch_dependents();
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer

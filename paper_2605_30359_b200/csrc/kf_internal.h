@@ -164,11 +164,13 @@ inline cudaError_t launch_umma_instance(const UmmaMaps& tm, const UmmaParams& p,
     cfg.blockDim = dim3(num_threads(EPI, BN, CTA2), 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = cluster;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     static int resident[17] = {0};             // clusters of this size that fit on the device
@@ -181,6 +183,8 @@ inline cudaError_t launch_umma_instance(const UmmaMaps& tm, const UmmaParams& p,
     }
     const int clusters = grid < resident[cluster] ? grid : resident[cluster];
     cfg.gridDim = dim3(clusters * cluster, 1, 1);
+    static const bool pdl_cl = getenv("KF_NO_PDL") == nullptr;
+    cfg.numAttrs = pdl_cl ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, kern, tm.a, tm.b, tm.r, tm.y, p);
   }
   if constexpr (CTA2) {

@@ -1,5 +1,6 @@
 // Launchers for the CUDA-core kernels.
 #include <type_traits>
+#include <cstdlib>
 #include "kf_internal.h"
 #include "kf_simt.cuh"
 
@@ -21,10 +22,19 @@ static cudaError_t simt_gemm_t(int mode, int act, int M, int N, int K, const voi
     auto go = [&](auto kern) {
       err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSimtSmemBytes);
       if (err != cudaSuccess) return;
-      kern<<<grid, block, kSimtSmemBytes, st>>>(
-          M, N, K, static_cast<const T*>(X), ldx, static_cast<const T*>(W), ldw,
-          static_cast<const T*>(bias), scale, static_cast<const T*>(R), ldr, out, ldo, act);
-      err = cudaGetLastError();
+      static const bool pdl = getenv("KF_NO_PDL") == nullptr;
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = grid;
+      cfg.blockDim = block;
+      cfg.dynamicSmemBytes = kSimtSmemBytes;
+      cfg.stream = st;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = pdl ? 1 : 0;
+      err = cudaLaunchKernelEx(&cfg, kern, M, N, K, static_cast<const T*>(X), ldx, static_cast<const T*>(W), ldw,
+                               static_cast<const T*>(bias), scale, static_cast<const T*>(R), ldr, out, ldo, act);
     };
     if (small) {
       if (mode == 0) go(simt_gemm_kernel<T, 0, ACT, 16, 16>);

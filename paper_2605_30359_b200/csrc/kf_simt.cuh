@@ -53,6 +53,10 @@ simt_gemm_kernel(int M, int N, int K, const T* __restrict__ X, long long ldx,
                  const T* R, long long ldr, void* out, long long ldo, int act_code) {
   constexpr int RM = TM / 4, RN = TN / 8;             // register block of a lane
   extern __shared__ float sm[];
+  // launched with programmatic stream serialization: wait for the kernel before this one, let
+  // the one after it be scheduled
+  griddep_wait();
+  griddep_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * TM, n0 = blockIdx.y * TN;
   float* As = sm + warp * (2 * 32 * kSimtLd);

@@ -12,6 +12,7 @@
 // Synchronisation: every thread of every CTA executes the same two cluster barriers, whatever
 // happened before (a wait that ran out only skips work), so no CTA can be left waiting.
 #pragma once
+#include <cstdlib>
 
 #include "kf_umma.cuh"
 
@@ -105,6 +106,10 @@ umma_splitk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_holder;
+  // a launch that was allowed to start early waits here for the kernel before it; the next
+  // launch of the stream may start its prologue
+  griddep_wait();
+  griddep_launch_dependents();
 
   bool have_acc = false;       // epilogue threads: this CTA's accumulator is complete
   if (warp == 0) {
@@ -309,13 +314,16 @@ inline cudaError_t launch_splitk_instance(const CUtensorMap& tmA, const CUtensor
   cfg.blockDim = dim3(kNumThreads, 1, 1);
   cfg.dynamicSmemBytes = C::kTotal;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = S;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  static const bool pdl = getenv("KF_NO_PDL") == nullptr;
+  cfg.numAttrs = pdl ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, p, act);
 }
 

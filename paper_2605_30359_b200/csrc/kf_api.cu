@@ -688,7 +688,8 @@ kf_status kf_gemm_groupnorm(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, 
       return KF_ERR_CUDA;
     // the single-CTA kernel's two epilogue groups leave one entry per half tile
     if (launch_row_groupnorm_apply(static_cast<int>(M), static_cast<int>(N), static_cast<int>(gs), (pair ? 1 : 2) * p.tiles_n,
-                                   eps, p.partial, gamma, beta, post_act, Y, ldy, st) != cudaSuccess)
+                                   eps, p.partial, gamma, beta, post_act, Y, ldy, st,
+                                   (pair ? 2 : 1) * grid < d->sm_count) != cudaSuccess)
       return KF_ERR_CUDA;
     g_launches += 2;
     return KF_OK;
@@ -797,13 +798,15 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
     p.status = d->status;
     const int units = p.num_tiles / p.tiles_per_unit;
     const int grid = units < slots ? units : slots;
+    // a first pass that leaves SMs idle lets the second kernel start early (see launch_after)
+    const bool partial_wave = (pair ? 2 : 1) * grid < d->sm_count;
     if (red == KF_RED_MAX || red == KF_RED_LOGSUMEXP) {
       // the softmax first pass without numerators (bf16 instance; nothing is stored), then the
       // per-slice statistics combined per row
       if (launch_umma_softmax(bn, pre_act, KF_BF16, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
         return KF_ERR_CUDA;
-      if (launch_rowstat_finalize(red, Mi, 2 * p.tiles_n, p.partial, static_cast<float*>(out), st) !=
-          cudaSuccess)
+      if (launch_rowstat_finalize(red, Mi, 2 * p.tiles_n, p.partial, static_cast<float*>(out), st,
+                                  partial_wave) != cudaSuccess)
         return KF_ERR_CUDA;
     } else if (red == KF_RED_SOFTMAX) {
       // 2..16 narrow column tiles per row: the CTAs that hold a row block's tiles form a cluster,
@@ -829,15 +832,15 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
       if (launch_umma_softmax(bn, pre_act, out_dtype, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
         return KF_ERR_CUDA;
       if (p.softmax_fused) { g_launches += 1; return KF_OK; }
-      if (launch_softmax_finalize(out_dtype, Mi, Ni, bn / 2, 2 * p.tiles_n, p.partial, out, ldo, p.vec_ok, st) !=
-          cudaSuccess)
+      if (launch_softmax_finalize(out_dtype, Mi, Ni, bn / 2, 2 * p.tiles_n, p.partial, out, ldo, p.vec_ok, st,
+                                  partial_wave) != cudaSuccess)
         return KF_ERR_CUDA;
     } else {
       if (launch_umma_rowsum(pre_act, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
         return KF_ERR_CUDA;
       if (!row_owner) {
-        if (launch_rowsum_finalize(Mi, p.tiles_n, p.partial, static_cast<float*>(out), p.scale, st) !=
-            cudaSuccess)
+        if (launch_rowsum_finalize(Mi, p.tiles_n, p.partial, static_cast<float*>(out), p.scale, st,
+                                   partial_wave) != cudaSuccess)
           return KF_ERR_CUDA;
         g_launches += 1;
       }
@@ -1025,14 +1028,15 @@ static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
     ++launches;
     if (gap_in_epilogue) {
       if (launch_gap_finalize(static_cast<int>(Nb), static_cast<int>(Cout),
-                              static_cast<int>(conv_stat_parts(H, Wd)), hw, stats, gap_out, st) != cudaSuccess)
+                              static_cast<int>(conv_stat_parts(H, Wd)), hw, stats, gap_out, st,
+                              grid < d->sm_count) != cudaSuccess)
         return KF_ERR_CUDA;
       ++launches;
     }
     if (groups > 0) {
       if (launch_groupnorm_apply(static_cast<int>(Nb), static_cast<int>(Cout), groups, hw,
                                  static_cast<int>(conv_stat_parts(H, Wd)), eps, stats, gamma, beta,
-                                 y, st) != cudaSuccess)
+                                 y, st, grid < d->sm_count) != cudaSuccess)
         return KF_ERR_CUDA;
       ++launches;
     }

@@ -41,11 +41,11 @@ constexpr int kRowReduceNarrowBN = 64;   // ... of the softmax first pass of one
 
 // second passes of the tensor-core row reductions
 cudaError_t launch_softmax_finalize(int out_dt, int M, int N, int bn, int tiles_n, const float* partial,
-                                    void* out, long long ldo, int vec_ok, cudaStream_t st);
+                                    void* out, long long ldo, int vec_ok, cudaStream_t st, bool overlap);
 cudaError_t launch_rowsum_finalize(int M, int tiles_n, const float* partial, float* out, float scale,
-                                   cudaStream_t st);
+                                   cudaStream_t st, bool overlap);
 cudaError_t launch_rowstat_finalize(int red, int M, int slices, const float* partial, float* out,
-                                    cudaStream_t st);
+                                    cudaStream_t st, bool overlap);
 
 // scalar chains (fp32, and bf16 shapes the tensor-core kernels do not take)
 cudaError_t launch_simt_gemm(int dt, int mode, int act, int M, int N, int K, const void* X,
@@ -68,7 +68,7 @@ cudaError_t launch_groupnorm(int dt, int Nb, int Cout, int groups, long long hw,
 // GroupNorm from the per-tile channel statistics the convolution epilogue wrote (bf16 only)
 cudaError_t launch_groupnorm_apply(int Nb, int Cout, int groups, long long hw, int tiles_per_image,
                                    float eps, const float* stats, const void* gamma,
-                                   const void* beta, void* y, cudaStream_t st);
+                                   const void* beta, void* y, cudaStream_t st, bool overlap);
 
 // GroupNorm over column groups of an fp32 matrix + activation (scalar path of kf_gemm_groupnorm)
 cudaError_t launch_row_groupnorm(int dt, int M, int N, int gs, float eps, const float* A, long long lda,
@@ -80,7 +80,7 @@ cudaError_t launch_row_groupnorm_inplace(int M, int N, int gs, float eps, const 
                                          cudaStream_t st);
 cudaError_t launch_row_groupnorm_apply(int M, int N, int gs, int tiles_n, float eps, const float* stats,
                                        const void* gamma, const void* beta, int act, void* Y,
-                                       long long ldy, cudaStream_t st);
+                                       long long ldy, cudaStream_t st, bool overlap);
 
 // max / average pooling (kernel = stride = pool) of an NCHW tensor
 cudaError_t launch_pool2d(int dt, long long planes, int H, int Wd, int pool, int kind, const void* in,
@@ -88,7 +88,7 @@ cudaError_t launch_pool2d(int dt, long long planes, int H, int Wd, int pool, int
 
 // global average pooling: from the convolution's statistics, or from a stored NCHW tensor
 cudaError_t launch_gap_finalize(int Nb, int Cout, int parts, long long hw, const float* stats, float* out,
-                                cudaStream_t st);
+                                cudaStream_t st, bool overlap);
 cudaError_t launch_plane_mean(int dt, long long rows, long long len, const void* in, float* out,
                               cudaStream_t st);
 

@@ -6,6 +6,32 @@
 
 namespace kf {
 
+// Launch of a second-pass kernel.  With `overlap` it is launched with programmatic stream
+// serialization: it may be scheduled while the kernel before it (which has called
+// griddepcontrol.launch_dependents) is still running, and waits in its first instruction
+// (griddep_wait) until that kernel has completed.  That saves 1.5-2 us when the first pass left
+// SMs idle (a partial wave).  After a first pass that filled every SM it was measured neutral to
+// harmful (the waiting CTAs were released 5-7 us after the first pass ended: 4096x4096x1024
+// row sum 34.3 -> 39.2 us, conv + channel softmax + pool 148 -> 155 us), so callers pass
+// overlap = false there and the launch is an ordinary one.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_after(bool overlap, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                cudaStream_t st, Args... args) {
+  static const bool pdl = getenv("KF_NO_PDL") == nullptr;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = (pdl && overlap) ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
+
 template <typename T>
 static cudaError_t simt_gemm_t(int mode, int act, int M, int N, int K, const void* X,
                                long long ldx, const void* W, long long ldw, const void* bias,
@@ -72,42 +98,37 @@ cudaError_t launch_row_reduce(int red, int M, int N, const float* A, long long l
 }
 
 cudaError_t launch_softmax_finalize(int out_dt, int M, int N, int bn, int tiles_n, const float* partial,
-                                    void* out, long long ldo, int vec_ok, cudaStream_t st) {
+                                    void* out, long long ldo, int vec_ok, cudaStream_t st, bool overlap) {
   int bn_shift = 0;                      // slices are powers of two (half a first-pass tile)
   while ((1 << bn_shift) < bn) ++bn_shift;
   if (tiles_n <= 32) {
     const unsigned grid = static_cast<unsigned>((M + 7) / 8);
     const float2* pw = reinterpret_cast<const float2*>(partial);
     if (out_dt == DT_F32)
-      softmax_finalize_warp_kernel<float><<<grid, 256, 0, st>>>(M, N, bn_shift, tiles_n, pw,
-                                                               static_cast<float*>(out), ldo, vec_ok);
-    else
-      softmax_finalize_warp_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
-          M, N, bn_shift, tiles_n, pw, static_cast<__nv_bfloat16*>(out), ldo, vec_ok);
-    return cudaGetLastError();
+      return launch_after(overlap, softmax_finalize_warp_kernel<float>, dim3(grid), dim3(256), 0, st, M, N, bn_shift,
+                          tiles_n, pw, static_cast<float*>(out), ldo, vec_ok);
+    return launch_after(overlap, softmax_finalize_warp_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, st, M, N,
+                        bn_shift, tiles_n, pw, static_cast<__nv_bfloat16*>(out), ldo, vec_ok);
   }
   const size_t smem = static_cast<size_t>(tiles_n) * sizeof(float);
   const float2* part = reinterpret_cast<const float2*>(partial);
   if (out_dt == DT_F32)
-    softmax_finalize_kernel<float><<<M, 256, smem, st>>>(
-        N, bn_shift, tiles_n, part, static_cast<float*>(out), ldo, vec_ok);
-  else
-    softmax_finalize_kernel<__nv_bfloat16><<<M, 256, smem, st>>>(
-        N, bn_shift, tiles_n, part, static_cast<__nv_bfloat16*>(out), ldo, vec_ok);
-  return cudaGetLastError();
+    return launch_after(overlap, softmax_finalize_kernel<float>, dim3(M), dim3(256), smem, st, N, bn_shift, tiles_n,
+                        part, static_cast<float*>(out), ldo, vec_ok);
+  return launch_after(overlap, softmax_finalize_kernel<__nv_bfloat16>, dim3(M), dim3(256), smem, st, N, bn_shift,
+                      tiles_n, part, static_cast<__nv_bfloat16*>(out), ldo, vec_ok);
 }
 
 cudaError_t launch_rowsum_finalize(int M, int tiles_n, const float* partial, float* out, float scale,
-                                   cudaStream_t st) {
-  rowsum_finalize_kernel<<<(M + 255) / 256, 256, 0, st>>>(M, tiles_n, partial, out, scale);
-  return cudaGetLastError();
+                                   cudaStream_t st, bool overlap) {
+  return launch_after(overlap, rowsum_finalize_kernel, dim3((M + 255) / 256), dim3(256), 0, st, M, tiles_n, partial, out,
+                      scale);
 }
 
 cudaError_t launch_rowstat_finalize(int red, int M, int slices, const float* partial, float* out,
-                                    cudaStream_t st) {
-  rowstat_finalize_kernel<<<(M + 255) / 256, 256, 0, st>>>(
-      M, slices, reinterpret_cast<const float2*>(partial), out, red);
-  return cudaGetLastError();
+                                    cudaStream_t st, bool overlap) {
+  return launch_after(overlap, rowstat_finalize_kernel, dim3((M + 255) / 256), dim3(256), 0, st, M, slices,
+                      reinterpret_cast<const float2*>(partial), out, red);
 }
 
 cudaError_t launch_row_groupnorm(int dt, int M, int N, int gs, float eps, const float* A, long long lda,
@@ -137,12 +158,11 @@ cudaError_t launch_row_groupnorm_inplace(int M, int N, int gs, float eps, const 
 
 cudaError_t launch_row_groupnorm_apply(int M, int N, int gs, int tiles_n, float eps, const float* stats,
                                        const void* gamma, const void* beta, int act, void* Y,
-                                       long long ldy, cudaStream_t st) {
+                                       long long ldy, cudaStream_t st, bool overlap) {
   const size_t smem = static_cast<size_t>(N / gs) * sizeof(float2);
-  row_groupnorm_apply_kernel<<<M, 256, smem, st>>>(
-      N, gs, tiles_n, eps, reinterpret_cast<const float2*>(stats), static_cast<const __nv_bfloat16*>(gamma),
-      static_cast<const __nv_bfloat16*>(beta), act, static_cast<__nv_bfloat16*>(Y), ldy);
-  return cudaGetLastError();
+  return launch_after(overlap, row_groupnorm_apply_kernel, dim3(M), dim3(256), smem, st, N, gs, tiles_n, eps,
+                      reinterpret_cast<const float2*>(stats), static_cast<const __nv_bfloat16*>(gamma),
+                      static_cast<const __nv_bfloat16*>(beta), act, static_cast<__nv_bfloat16*>(Y), ldy);
 }
 
 cudaError_t launch_pool2d(int dt, long long planes, int H, int Wd, int pool, int kind, const void* in,
@@ -161,11 +181,10 @@ cudaError_t launch_pool2d(int dt, long long planes, int H, int Wd, int pool, int
 }
 
 cudaError_t launch_gap_finalize(int Nb, int Cout, int parts, long long hw, const float* stats, float* out,
-                                cudaStream_t st) {
+                                cudaStream_t st, bool overlap) {
   const long long total = static_cast<long long>(Nb) * Cout;
-  gap_finalize_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, st>>>(
-      Nb, Cout, parts, hw, reinterpret_cast<const float2*>(stats), out);
-  return cudaGetLastError();
+  return launch_after(overlap, gap_finalize_kernel, dim3(static_cast<unsigned>((total + 255) / 256)), dim3(256), 0, st, Nb,
+                      Cout, parts, hw, reinterpret_cast<const float2*>(stats), out);
 }
 
 cudaError_t launch_plane_mean(int dt, long long rows, long long len, const void* in, float* out,
@@ -251,13 +270,11 @@ cudaError_t launch_groupnorm(int dt, int Nb, int Cout, int groups, long long hw,
 
 cudaError_t launch_groupnorm_apply(int Nb, int Cout, int groups, long long hw, int tiles_per_image,
                                    float eps, const float* stats, const void* gamma,
-                                   const void* beta, void* y, cudaStream_t st) {
+                                   const void* beta, void* y, cudaStream_t st, bool overlap) {
   const unsigned grid = static_cast<unsigned>(Nb) * static_cast<unsigned>(groups);
-  groupnorm_apply_kernel<<<grid, 512, 0, st>>>(
-      Cout, groups, hw, tiles_per_image, eps, reinterpret_cast<const float2*>(stats),
-      static_cast<const __nv_bfloat16*>(gamma), static_cast<const __nv_bfloat16*>(beta),
-      static_cast<__nv_bfloat16*>(y));
-  return cudaGetLastError();
+  return launch_after(overlap, groupnorm_apply_kernel, dim3(grid), dim3(512), 0, st, Cout, groups, hw, tiles_per_image, eps,
+                      reinterpret_cast<const float2*>(stats), static_cast<const __nv_bfloat16*>(gamma),
+                      static_cast<const __nv_bfloat16*>(beta), static_cast<__nv_bfloat16*>(y));
 }
 
 namespace {
@@ -297,8 +314,7 @@ cudaError_t channel_softmax_pool_typed(int Nb, int C, int H, int Wd, int pool, c
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(kPoolStripBytes * 3 + 8192));
     if (e != cudaSuccess) return e;
-    kern<<<static_cast<unsigned>(blocks), 256, smem, st>>>(Nb, C, H, Wd, tw, a, y);
-    return cudaGetLastError();
+    return launch_after(false, kern, dim3(static_cast<unsigned>(blocks)), dim3(256), smem, st, Nb, C, H, Wd, tw, a, y);
   };
   auto by_pool = [&](auto vec_tag) -> cudaError_t {
     constexpr int V = decltype(vec_tag)::value;

@@ -231,6 +231,7 @@ row_groupnorm_apply_kernel(int N, int gs, int tiles_n, float eps, const float2* 
                            const __nv_bfloat16* __restrict__ gamma,
                            const __nv_bfloat16* __restrict__ beta, int act_code, __nv_bfloat16* Y,
                            long long ldy) {
+  griddep_wait();      // may have been scheduled before the kernel it depends on finished
   extern __shared__ float2 mr[];            // [groups] (mu, rstd)
   const int groups = N / gs, tpg = static_cast<int>(static_cast<long long>(gs) * tiles_n / N);   // entries per group
   const float2* part = stats + static_cast<long long>(blockIdx.x) * tiles_n;
@@ -270,6 +271,7 @@ template <typename OutT>
 __global__ void __launch_bounds__(256)
 softmax_finalize_kernel(int N, int bn_shift, int tiles_n, const float2* __restrict__ partial,
                         OutT* out, long long ldo, int vec_ok) {
+  griddep_wait();      // may have been scheduled before the kernel it depends on finished
   extern __shared__ float fac[];   // [tiles_n]
   __shared__ float scratch[32];
   // The first pass wrote the rows in increasing order, so its last rows are the ones still in
@@ -349,6 +351,7 @@ __global__ void __launch_bounds__(256)
 softmax_finalize_warp_kernel(int M, int N, int bn_shift, int tiles_n,
                              const float2* __restrict__ partial, OutT* out, long long ldo,
                              int vec_ok) {
+  griddep_wait();      // may have been scheduled before the kernel it depends on finished
   const int lane = threadIdx.x & 31;
   // last-written rows first (they are the ones still in L2)
   const long long m = static_cast<long long>(gridDim.x - 1 - blockIdx.x) * 8 + (threadIdx.x >> 5);
@@ -399,6 +402,7 @@ softmax_finalize_warp_kernel(int M, int N, int bn_shift, int tiles_n,
 // Row sum: out[m] = scale * sum_t partial[m,t] in increasing t (scale = 1/N for the mean).
 __global__ void __launch_bounds__(256)
 rowsum_finalize_kernel(int M, int tiles_n, const float* __restrict__ partial, float* out, float scale) {
+  griddep_wait();      // may have been scheduled before the kernel it depends on finished
   const long long m = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (m >= M) return;
   float s = 0.0f;
@@ -410,6 +414,7 @@ rowsum_finalize_kernel(int M, int tiles_n, const float* __restrict__ partial, fl
 // statistics-only mode: mx = max_t mx_t; lse = mx + log sum_t sum_t * exp(mx_t - mx).
 __global__ void __launch_bounds__(256)
 rowstat_finalize_kernel(int M, int slices, const float2* __restrict__ partial, float* out, int red) {
+  griddep_wait();      // may have been scheduled before the kernel it depends on finished
   const long long m = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (m >= M) return;
   const float2* part = partial + m * slices;
@@ -672,6 +677,7 @@ __global__ void __launch_bounds__(512)
 groupnorm_apply_kernel(int Cout, int groups, long long hw, int tiles_per_image, float eps,
                        const float2* __restrict__ stats, const __nv_bfloat16* __restrict__ gamma,
                        const __nv_bfloat16* __restrict__ beta, __nv_bfloat16* y) {
+  griddep_wait();      // may have been scheduled before the kernel it depends on finished
   const int cpg = Cout / groups;
   const long long cnt = static_cast<long long>(cpg) * hw;
   // increasing image order: the convolution wrote the first images last, they are still in L2
@@ -770,6 +776,7 @@ pool2d_kernel(long long planes, int H, int Wd, int pool, int kind, const T* __re
 __global__ void __launch_bounds__(256)
 gap_finalize_kernel(int Nb, int Cout, int parts, long long hw, const float2* __restrict__ stats,
                     float* __restrict__ out) {
+  griddep_wait();      // may have been scheduled before the kernel it depends on finished
   const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (gid >= static_cast<long long>(Nb) * Cout) return;
   const long long n = gid / Cout;
@@ -889,6 +896,7 @@ template <typename T, int VEC, int POOL>
 __global__ void __launch_bounds__(256)
 channel_softmax_pool_tiled_kernel(int Nb, int C, int H, int Wd, int tw, const T* __restrict__ a,
                                   T* __restrict__ y) {
+  griddep_wait();      // may have been scheduled before the kernel it depends on finished
   extern __shared__ __align__(16) unsigned char smem_raw[];
   T* s = reinterpret_cast<T*>(smem_raw);
   const int Ho = H / POOL, Wo = Wd / POOL;

@@ -911,21 +911,41 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           float2* sbuf = reinterpret_cast<float2*>(stg + C::kStaging + C::kBarBytes) + (buf * 2 + grp) * 32;
           float2* inbox = reinterpret_cast<float2*>(stg + C::kStaging + C::kBarBytes + C::kBiasBytes);
           uint8_t* yslab = stg + grp * kPieceBytes;               // the group's staging piece
+          const uint64_t bias2 = f32x2_pack(bias_v, bias_v);
+          uint64_t s1p = f32x2_pack(0.0f, 0.0f), s2p = s1p;
 #pragma unroll 1
           for (int c = 0; c < my_pieces; ++c) {
             uint32_t v[32];
             tmem_ld_32x32(t_acc + c * 32, v);
             tmem_ld_wait();
             const int left = px_valid - (piece0 + c) * 32;
+            if (left >= 32) {
+              // whole piece: bias, sum and sum of squares on packed pairs (even and odd pixels
+              // accumulate separately and are added after the loop)
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + bias_v, p.act_rt);
-              float y1 = act_f<ACT, true>(__uint_as_float(v[2 * j + 1]) + bias_v, p.act_rt);
-              if (2 * j >= left) y0 = 0.0f;
-              if (2 * j + 1 >= left) y1 = 0.0f;
-              s1 += y0 + y1;
-              s2 = fmaf(y0, y0, fmaf(y1, y1, s2));
+              for (int j = 0; j < 16; ++j) {
+                float y0, y1;
+                f32x2_unpack(f32x2_add(f32x2_pack(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])), bias2), y0, y1);
+                const uint64_t y = f32x2_pack(act_f<ACT, true>(y0, p.act_rt), act_f<ACT, true>(y1, p.act_rt));
+                s1p = f32x2_add(s1p, y);
+                s2p = f32x2_fma(y, y, s2p);
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + bias_v, p.act_rt);
+                float y1 = act_f<ACT, true>(__uint_as_float(v[2 * j + 1]) + bias_v, p.act_rt);
+                if (2 * j >= left) y0 = 0.0f;
+                if (2 * j + 1 >= left) y1 = 0.0f;
+                s1 += y0 + y1;
+                s2 = fmaf(y0, y0, fmaf(y1, y1, s2));
+              }
             }
+          }
+          {
+            float e, o;
+            f32x2_unpack(s1p, e, o); s1 += e + o;
+            f32x2_unpack(s2p, e, o); s2 += e + o;
           }
           for (int o = cpg >> 1; o > 0; o >>= 1) {                // the group's channels: adjacent lanes
             s1 += __shfl_xor_sync(0xffffffffu, s1, o);
@@ -961,6 +981,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             sh = fmaf(-mu, sc, be);
           }
           if (my_pieces == 0) release_acc();
+          const uint64_t sc2 = f32x2_pack(sc, sc), sh2 = f32x2_pack(sh, sh);
 #pragma unroll 1
           for (int c = 0; c < my_pieces; ++c) {
             uint32_t v[32];
@@ -970,9 +991,11 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             uint32_t w[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-              const float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + bias_v, p.act_rt);
-              const float y1 = act_f<ACT, true>(__uint_as_float(v[2 * j + 1]) + bias_v, p.act_rt);
-              w[j] = pack_bf16x2(fmaf(y0, sc, sh), fmaf(y1, sc, sh));
+              float y0, y1;
+              f32x2_unpack(f32x2_add(f32x2_pack(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])), bias2), y0, y1);
+              const uint64_t y = f32x2_pack(act_f<ACT, true>(y0, p.act_rt), act_f<ACT, true>(y1, p.act_rt));
+              f32x2_unpack(f32x2_fma(y, sc2, sh2), y0, y1);
+              w[j] = pack_bf16x2(y0, y1);
             }
             bulk_wait_group_read<0>();       // this warp's previous store has let go of the slab
             __syncwarp();

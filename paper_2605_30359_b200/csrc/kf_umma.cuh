@@ -891,6 +891,9 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // left out of the statistics and are not stored
         const int px_valid = static_cast<int>(min(static_cast<long long>(p.tile_px), hw - px0));
         float s1 = 0.0f, s2 = 0.0f;
+        const uint64_t bias2 = f32x2_pack(bias_v, bias_v);
+        uint64_t s1p = f32x2_pack(0.0f, 0.0f), s2p = s1p;   // (even, odd) pixel partial sums
+        const bool want_stats = p.partial != nullptr;
         if constexpr (EPI == EPI_CONV_GN) {
           // GroupNorm without a second kernel.  The CTAs of this cluster hold the tiles of one
           // image, one each.  The accumulator stays in TMEM while (1) each epilogue group adds
@@ -911,8 +914,6 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           float2* sbuf = reinterpret_cast<float2*>(stg + C::kStaging + C::kBarBytes) + (buf * 2 + grp) * 32;
           float2* inbox = reinterpret_cast<float2*>(stg + C::kStaging + C::kBarBytes + C::kBiasBytes);
           uint8_t* yslab = stg + grp * kPieceBytes;               // the group's staging piece
-          const uint64_t bias2 = f32x2_pack(bias_v, bias_v);
-          uint64_t s1p = f32x2_pack(0.0f, 0.0f), s2p = s1p;
 #pragma unroll 1
           for (int c = 0; c < my_pieces; ++c) {
             uint32_t v[32];
@@ -971,6 +972,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           {
             const float2* ib = inbox + buf * 16 * 2 * 32 + row / cpg;
             float g1 = 0.0f, g2 = 0.0f;
+#pragma unroll 4      // loads in flight together; the additions keep their order
             for (int r = 0; r < 2 * csize; ++r) { const float2 q = ib[r * 32]; g1 += q.x; g2 += q.y; }
             const float cnt = static_cast<float>(static_cast<long long>(cpg) * hw);
             const float mu = g1 / cnt;
@@ -1042,10 +1044,13 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
               for (int t = 0; t < 2; ++t) {
                 const int i = 4 * j + 2 * t;
-                const float a00 = act_f<ACT, true>(__uint_as_float(v0[i]) + bias_v, p.act_rt);
-                const float a01 = act_f<ACT, true>(__uint_as_float(v0[i + 1]) + bias_v, p.act_rt);
-                const float a10 = act_f<ACT, true>(__uint_as_float(v1[i]) + bias_v, p.act_rt);
-                const float a11 = act_f<ACT, true>(__uint_as_float(v1[i + 1]) + bias_v, p.act_rt);
+                float a00, a01, a10, a11;
+                f32x2_unpack(f32x2_add(f32x2_pack(__uint_as_float(v0[i]), __uint_as_float(v0[i + 1])), bias2), a00, a01);
+                f32x2_unpack(f32x2_add(f32x2_pack(__uint_as_float(v1[i]), __uint_as_float(v1[i + 1])), bias2), a10, a11);
+                a00 = act_f<ACT, true>(a00, p.act_rt);
+                a01 = act_f<ACT, true>(a01, p.act_rt);
+                a10 = act_f<ACT, true>(a10, p.act_rt);
+                a11 = act_f<ACT, true>(a11, p.act_rt);
                 o[t] = p.pool2 == 1 ? fmaxf(fmaxf(a00, a01), fmaxf(a10, a11))
                                     : 0.25f * ((a00 + a01) + (a10 + a11));
               }
@@ -1076,15 +1081,40 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (c == pieces - 1) release_acc();
           uint32_t w[16];
           const int left = px_valid - c * 32;               // valid pixels from this piece on
+          if (left >= 32) {
+            // whole piece: bias (and the statistics, where a later pass wants them) on packed
+            // pairs; even and odd pixels accumulate separately and are added after the loop
+            if (want_stats) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + bias_v, p.act_rt);
-            float y1 = act_f<ACT, true>(__uint_as_float(v[2 * j + 1]) + bias_v, p.act_rt);
-            w[j] = pack_bf16x2(y0, y1);
-            if (2 * j >= left) y0 = 0.0f;
-            if (2 * j + 1 >= left) y1 = 0.0f;
-            s1 += y0 + y1;
-            s2 = fmaf(y0, y0, fmaf(y1, y1, s2));
+              for (int j = 0; j < 16; ++j) {
+                float y0, y1;
+                f32x2_unpack(f32x2_add(f32x2_pack(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])), bias2), y0, y1);
+                y0 = act_f<ACT, true>(y0, p.act_rt);
+                y1 = act_f<ACT, true>(y1, p.act_rt);
+                w[j] = pack_bf16x2(y0, y1);
+                const uint64_t y = f32x2_pack(y0, y1);
+                s1p = f32x2_add(s1p, y);
+                s2p = f32x2_fma(y, y, s2p);
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                float y0, y1;
+                f32x2_unpack(f32x2_add(f32x2_pack(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])), bias2), y0, y1);
+                w[j] = pack_bf16x2(act_f<ACT, true>(y0, p.act_rt), act_f<ACT, true>(y1, p.act_rt));
+              }
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + bias_v, p.act_rt);
+              float y1 = act_f<ACT, true>(__uint_as_float(v[2 * j + 1]) + bias_v, p.act_rt);
+              w[j] = pack_bf16x2(y0, y1);
+              if (2 * j >= left) y0 = 0.0f;
+              if (2 * j + 1 >= left) y1 = 0.0f;
+              s1 += y0 + y1;
+              s2 = fmaf(y0, y0, fmaf(y1, y1, s2));
+            }
           }
           if (p.stats_only != 0) continue;     // only the per-channel statistics are wanted
           if (staged) {
@@ -1130,7 +1160,10 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             named_barrier_sync(bar_b, kEpiThreads);    // the buffer is free for the next piece
           }
         }
-        if (p.partial != nullptr && ch_ok) {      // one entry per pixel tile and channel
+        if (want_stats && ch_ok) {                // one entry per pixel tile and channel
+          float e, o;
+          f32x2_unpack(s1p, e, o); s1 += e + o;
+          f32x2_unpack(s2p, e, o); s2 += e + o;
           float2* part = reinterpret_cast<float2*>(p.partial);
           part[static_cast<long long>(tn) * p.N + ch] = make_float2(s1, s2);
         }

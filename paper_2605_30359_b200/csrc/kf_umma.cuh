@@ -570,15 +570,30 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 const float u = (__uint_as_float(v[j]) + bs[j] - gn_mu) * gn_rstd;
                 f[j] = p.scale * act_f<ACT, true>(fmaf(u, ga[j], be[j]), p.act_rt);
               }
-            } else {
+            } else if (CTA2 || p.gn_tile_stats) {
+              // (the CTA-pair kernel's epilogue hides behind its MMAs: it keeps the scalar form)
 #pragma unroll
               for (int j = 0; j < 32; ++j) {
                 const float z = __uint_as_float(v[j]) + bs[j];
                 if (p.gn_tile_stats) { ts1 += z; ts2 = fmaf(z, z, ts2); }   // columns past N hold 0
                 f[j] = p.scale * act_f<ACT, true>(z, p.act_rt);
               }
+            } else {
+              // the plain chain on packed pairs: bias, then scale (and residual) in one
+              // instruction per two columns
+              const uint64_t scale2 = f32x2_pack(p.scale, p.scale);
+              const uint32_t* rw = reinterpret_cast<const uint32_t*>(rv);   // 16 bf16 pairs
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                float z0, z1;
+                f32x2_unpack(f32x2_add(f32x2_pack(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])),
+                                       f32x2_pack(bs[2 * j], bs[2 * j + 1])), z0, z1);
+                const uint64_t a2 = f32x2_pack(act_f<ACT, true>(z0, p.act_rt), act_f<ACT, true>(z1, p.act_rt));
+                if (has_r) f32x2_unpack(f32x2_fma(a2, scale2, f32x2_pack(bf16_lo(rw[j]), bf16_hi(rw[j]))), f[2 * j], f[2 * j + 1]);
+                else f32x2_unpack(f32x2_mul(a2, scale2), f[2 * j], f[2 * j + 1]);
+              }
             }
-            if (has_r) {
+            if (has_r && (CTA2 || p.gn_pieces > 0 || p.gn_tile_stats)) {
 #pragma unroll
               for (int q = 0; q < 4; ++q) {
                 f[8 * q + 0] += bf16_lo(rv[q].x); f[8 * q + 1] += bf16_hi(rv[q].x);

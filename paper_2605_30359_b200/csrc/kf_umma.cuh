@@ -699,10 +699,20 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           float bs[32];
           load_sbias32(sbias + c * 32, bs);
           tmem_ld_wait();
+          if (c * 32 + 32 <= n_valid) {          // whole piece: bias on packed pairs, no masks
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
-            if (c * 32 + j < n_valid) mx = fmaxf(mx, z);
+            for (int j = 0; j < 16; ++j) {
+              float z0, z1;
+              f32x2_unpack(f32x2_add(f32x2_pack(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])),
+                                     f32x2_pack(bs[2 * j], bs[2 * j + 1])), z0, z1);
+              mx = fmaxf(mx, fmaxf(act_f<ACT, true>(z0, p.act_rt), act_f<ACT, true>(z1, p.act_rt)));
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
+              if (c * 32 + j < n_valid) mx = fmaxf(mx, z);
+            }
           }
         }
         // A row that lies in this one tile (tiles_n == 1) is finished here: the two groups
@@ -777,11 +787,36 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           tmem_ld_wait();
           if (staged && c == PIECES - 1 && phase != 1) release_acc();
           float f[32];
+          if (c * 32 + 32 <= n_valid) {
+            // whole piece on packed pairs: exp(z - mx) = 2^(z log2(e) - mx log2(e)), one fused
+            // multiply-add per two columns; even and odd columns add up separately
+            constexpr float kLog2e = 1.4426950408889634f;
+            const uint64_t l2e2 = f32x2_pack(kLog2e, kLog2e);
+            const uint64_t off2 = f32x2_pack(-mx * kLog2e, -mx * kLog2e);
+            const uint64_t inv2 = f32x2_pack(inv, inv);
+            uint64_t sum2 = f32x2_pack(0.0f, 0.0f);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
-            f[j] = __expf(z - mx) * inv;
-            if (phase != 2 && c * 32 + j < n_valid) sum += f[j];
+            for (int j = 0; j < 16; ++j) {
+              float z0, z1;
+              f32x2_unpack(f32x2_add(f32x2_pack(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])),
+                                     f32x2_pack(bs[2 * j], bs[2 * j + 1])), z0, z1);
+              f32x2_unpack(f32x2_fma(f32x2_pack(act_f<ACT, true>(z0, p.act_rt), act_f<ACT, true>(z1, p.act_rt)), l2e2, off2),
+                           z0, z1);
+              uint64_t e2 = f32x2_pack(exp2_approx(z0), exp2_approx(z1));
+              if (whole_row) e2 = f32x2_mul(e2, inv2);
+              f32x2_unpack(e2, f[2 * j], f[2 * j + 1]);
+              if (phase != 2) sum2 = f32x2_add(sum2, e2);
+            }
+            float se, so;
+            f32x2_unpack(sum2, se, so);
+            sum += se + so;
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
+              f[j] = __expf(z - mx) * inv;
+              if (phase != 2 && c * 32 + j < n_valid) sum += f[j];
+            }
           }
           if (p.stats_only != 0 || phase == 1) continue;
           if constexpr (sizeof(OutT) == 2) {
@@ -874,10 +909,24 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           load_sbias32(sbias + c * 32, bs);
           tmem_ld_wait();
           float part = 0.0f;
+          if (c * 32 + 32 <= n_valid) {          // whole piece: packed pairs, no masks
+            uint64_t part2 = f32x2_pack(0.0f, 0.0f);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
-            if (c * 32 + j < n_valid) part += z;
+            for (int j = 0; j < 16; ++j) {
+              float z0, z1;
+              f32x2_unpack(f32x2_add(f32x2_pack(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])),
+                                     f32x2_pack(bs[2 * j], bs[2 * j + 1])), z0, z1);
+              part2 = f32x2_add(part2, f32x2_pack(act_f<ACT, true>(z0, p.act_rt), act_f<ACT, true>(z1, p.act_rt)));
+            }
+            float pe, po;
+            f32x2_unpack(part2, pe, po);
+            part = pe + po;
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float z = act_f<ACT, true>(__uint_as_float(v[j]) + bs[j], p.act_rt);
+              if (c * 32 + j < n_valid) part += z;
+            }
           }
           sum += part;
         }

@@ -989,15 +989,19 @@ channel_softmax_pool_tiled_kernel(int Nb, int C, int H, int Wd, int tw, const T*
           m0 = fmaxf(m0, v[0]); m1 = fmaxf(m1, v[1]);
         }
       }
-      const float b0 = -m0 * kLog2e, b1 = -m1 * kLog2e;
-      float s0 = 0.0f, s1 = 0.0f;
+      // both pixels' exponent arguments in one packed multiply-add, both sums in one packed add
+      const uint64_t l2e2 = f32x2_pack(kLog2e, kLog2e), off2 = f32x2_pack(-m0 * kLog2e, -m1 * kLog2e);
+      uint64_t sum2 = f32x2_pack(0.0f, 0.0f);
 #pragma unroll 8
       for (int c = c0; c < c1; ++c) {
         float v[2];
         ld_row<2>(col + c * P, v);
-        s0 += ex2_approx(fmaf(v[0], kLog2e, b0));
-        s1 += ex2_approx(fmaf(v[1], kLog2e, b1));
+        float t0, t1;
+        f32x2_unpack(f32x2_fma(f32x2_pack(v[0], v[1]), l2e2, off2), t0, t1);
+        sum2 = f32x2_add(sum2, f32x2_pack(ex2_approx(t0), ex2_approx(t1)));
       }
+      float s0, s1;
+      f32x2_unpack(sum2, s0, s1);
       if (slices == 1) {
         lse[p] = m0 + __logf(s0);
         lse[p + 1] = m1 + __logf(s1);

@@ -145,8 +145,9 @@ size_t kf_gemm_groupnorm_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dty
  * The reduction is deterministic (no floating-point atomics): repeated calls give identical
  * bits.  The workspace holds per-tile partial statistics.  bf16 softmax: a GEMM kernel that
  * leaves numerators and per-tile (max, sum), then a rescaling kernel; rows that lie in one tile,
- * or in up to 16 tiles of 64 columns (small problems; their CTAs form a cluster and exchange
- * the pairs through distributed shared memory), are finished by the GEMM kernel alone. */
+ * or in up to 16 tiles of 64 columns or up to 8 tiles of 128 columns (small problems; their CTAs
+ * form a cluster and exchange the pairs through distributed shared memory), are finished by the
+ * GEMM kernel alone. */
 kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype,
                             const void* X, int64_t ldx, const void* W, int64_t ldw,
                             const void* bias, kf_act pre_act, kf_rowred red,

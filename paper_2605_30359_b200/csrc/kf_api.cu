@@ -821,11 +821,32 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
         pc.gn_cluster = p.tiles_n;
         pc.num_tiles = p.tiles_m;            // the schedule counts row blocks
         pc.tiles_per_unit = 1;
-        if (launch_umma_softmax_cluster(pre_act, out_dtype, tm, pc, p.tiles_m, st) == cudaSuccess) {
+        if (launch_umma_softmax_cluster(bn, pre_act, out_dtype, tm, pc, p.tiles_m, st) == cudaSuccess) {
           g_launches += 1;
           return KF_OK;
         }
         (void)cudaGetLastError();            // no such cluster can be resident: the two-kernel route
+      }
+      // Rows of 2..8 tiles of 128 columns whose narrow-tile clusters would not all be resident:
+      // the same kernel with 128-column tiles and clusters of at most 8 (15 fit on the GPU).
+      {
+        const int64_t tn128 = (N + 127) / 128;
+        if (bn == kRowReduceNarrowBN && out_dtype == KF_BF16 && p.staged && tn128 >= 2 && tn128 <= 8 &&
+            static_cast<int64_t>(p.tiles_m) * tn128 <= env_int("KF_CL128_MAX_CTAS", 120) &&
+            static_cast<int64_t>(p.tiles_m) * p.tiles_n > 112 && getenv("KF_NO_CLUSTER_SOFTMAX") == nullptr) {
+          UmmaMaps tc = tm;
+          if (!encode_2d(&tc.b, W, N, K, ldw, 128)) return KF_ERR_CUDA;
+          UmmaParams pc = p;
+          pc.tiles_n = static_cast<int>(tn128);
+          pc.gn_cluster = pc.tiles_n;
+          pc.num_tiles = p.tiles_m;
+          pc.tiles_per_unit = 1;
+          if (launch_umma_softmax_cluster(128, pre_act, out_dtype, tc, pc, p.tiles_m, st) == cudaSuccess) {
+            g_launches += 1;
+            return KF_OK;
+          }
+          (void)cudaGetLastError();
+        }
       }
       // a row that lies in one tile is finished in the GEMM epilogue: no second kernel
       p.softmax_fused = (p.tiles_n == 1 && getenv("KF_NO_FUSED_SOFTMAX") == nullptr) ? 1 : 0;

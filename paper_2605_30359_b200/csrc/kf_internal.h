@@ -32,7 +32,7 @@ cudaError_t launch_umma_conv(int bn, int act, const UmmaMaps& tm, const UmmaPara
                              cudaStream_t st);
 // the cluster form with GroupNorm in the epilogue: `images` units, p.gn_cluster CTAs per cluster
 // the cluster softmax: `row_blocks` units, p.gn_cluster (= column tiles per row) CTAs per cluster
-cudaError_t launch_umma_softmax_cluster(int act, int out_dt, const UmmaMaps& tm, const UmmaParams& p,
+cudaError_t launch_umma_softmax_cluster(int bn, int act, int out_dt, const UmmaMaps& tm, const UmmaParams& p,
                                         int row_blocks, cudaStream_t st);
 cudaError_t launch_umma_conv_gn(int bn, int act, const UmmaMaps& tm, const UmmaParams& p, int images,
                                 cudaStream_t st);

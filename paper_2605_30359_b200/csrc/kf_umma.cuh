@@ -144,7 +144,9 @@ struct UmmaCfg {
   // EPI_CONV_GN: statistics arriving from the cluster, [2 buffers][16 CTAs x 2 groups][32 x float2]
   // EPI_SOFTMAX_CL: [2 buffers][16 CTAs x 2 groups][128 rows x float2] arriving, then the
   // [2 buffers][2 groups][128 x float2] it sends
-  static constexpr int kInboxBytes = EPI == EPI_CONV_GN ? 2 * 32 * 256 : (EPI == EPI_SOFTMAX_CL ? 2 * 32 * 1024 + 4 * 1024 : 0);
+  // (EPI_SOFTMAX_CL: clusters of up to 16 CTAs with 64-column tiles, up to 8 with wider ones)
+  static constexpr int kClMax = BN <= 64 ? 16 : 8;
+  static constexpr int kInboxBytes = EPI == EPI_CONV_GN ? 2 * 32 * 256 : (EPI == EPI_SOFTMAX_CL ? 2 * 2 * kClMax * 1024 + 4 * 1024 : 0);
   static constexpr int kFit = (kMaxDynSmem - 1024 - kStaging - kBarBytes - kBiasBytes - kInboxBytes) / kStage;
   static constexpr int kStages = kFit > 8 ? 8 : kFit;
   static constexpr int kRing = kStage * kStages;
@@ -752,14 +754,15 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const int buf = it & 1;
             const int csize = p.gn_cluster;
             float2* inbox = reinterpret_cast<float2*>(stg + C::kStaging + C::kBarBytes + C::kBiasBytes);
-            float2* sbuf = inbox + 2 * 32 * 128 + (buf * 2 + grp) * 128;
+            constexpr int kClMax = C::kClMax;             // inbox slots per buffer: 2 groups x kClMax ranks
+            float2* sbuf = inbox + 2 * 2 * kClMax * 128 + (buf * 2 + grp) * 128;
             sbuf[et] = make_float2(mx, sum);
             fence_proxy_async_smem();
             named_barrier_sync(bar_b, kEpiThreads);
             if (lead_warp) {
               if (elect_one()) {
                 if (grp == 0) mbar_expect_tx(&rbar[buf], static_cast<uint32_t>(csize) * 2u * 1024u);
-                const uint32_t dst = smem_u32(inbox + ((buf * 16 + static_cast<int>(crank)) * 2 + grp) * 128);
+                const uint32_t dst = smem_u32(inbox + ((buf * kClMax + static_cast<int>(crank)) * 2 + grp) * 128);
                 for (int r = 0; r < csize; ++r)
                   bulk_copy_to_peer(mapa_shared(dst, r), smem_u32(sbuf), 1024u, mapa_shared(smem_u32(&rbar[buf]), r));
               }
@@ -768,7 +771,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                                     KF_DEV_TIMEOUT_EPILOGUE);
             all_in = named_barrier_and(bar_a, kEpiThreads, all_in);
             if (!all_in) { alive = false; break; }
-            const float2* ib = inbox + buf * 32 * 128 + et;
+            const float2* ib = inbox + buf * 2 * kClMax * 128 + et;
             float big = -INFINITY;
             for (int r = 0; r < 2 * csize; ++r) big = fmaxf(big, ib[r * 128].x);
             float den = 0.0f;

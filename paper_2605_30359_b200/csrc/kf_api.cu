@@ -317,6 +317,12 @@ int pick_split_k(int64_t M, int64_t N, int64_t K, int sm_count, int* bn_out) {
     int sk = 0;
     if (bn == 256 && kb >= 32 && tiles * 8 <= 64) sk = 8;
     else if (tiles * 4 <= sm_count - sm_count % 4) sk = 4;
+    // 128-column tiles with three stages: two CTAs per SM, so that one CTA's exchange and
+    // epilogue run beside the other's loads.  Pays with long K shares or few live rows
+    // (64x8192x8192 26.9 -> 25.6 us, 32x5120x8192 19.1 -> 18.7, 16x9472x4096 20.8 -> 17.4;
+    // 128x8192x4096 13.8 -> 14.4 us, hence the conditions).
+    else if (bn == 128 && tiles * 4 <= 2 * (sm_count - sm_count % 4) && (kb >= 128 || M <= 32) &&
+             env_int("KF_SPLITK_TWO_PER_SM", 1) != 0) sk = 4;
     else if (bn == 128 && tiles * 2 <= sm_count - sm_count % 2) sk = 2;
     *ctas = tiles * sk;
     return sk;
@@ -537,7 +543,9 @@ kf_status kf_gemm_epilogue(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, c
                 (residual == nullptr || (ldr % 8 == 0 && aligned(residual, 16)))) ? 1 : 0;
     p.bias_vec = aligned(bias, 16) ? 1 : 0;
     p.status = d->status;
-    if (launch_umma_splitk(bn_split, split, act, tm, p, st) != cudaSuccess) return KF_ERR_CUDA;
+    // more clusters than one CTA per SM can hold: the three-stage instance, two CTAs per SM
+    const bool two_per_sm = static_cast<int64_t>(p.num_tiles) * split > d->sm_count;
+    if (launch_umma_splitk(bn_split, split, act, tm, p, st, two_per_sm) != cudaSuccess) return KF_ERR_CUDA;
     g_launches += 1;
     return KF_OK;
   }

@@ -134,7 +134,7 @@ cudaError_t launch_tf32_chain(int bn, const CUtensorMap& ah, const CUtensorMap& 
 
 // split-K cluster kernel of the elementwise chain: bn in {128, 256}, s CTAs per tile
 cudaError_t launch_umma_splitk(int bn, int s, int act, const UmmaMaps& tm, const UmmaParams& p,
-                               cudaStream_t st);
+                               cudaStream_t st, bool two_per_sm = false);
 
 // softmax over channels + pool x pool max-pool of an NCHW tensor (pool <= 4)
 cudaError_t launch_channel_softmax_pool(int dt, int Nb, int C, int H, int Wd, int pool, const void* a,

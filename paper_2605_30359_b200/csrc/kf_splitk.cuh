@@ -18,12 +18,14 @@
 
 namespace kf {
 
-template <int BN, int S>
+// STAGES = 3 with 128-column tiles keeps a CTA under half of the SM's shared memory, so that two
+// CTAs share an SM: one streams its K share while the other exchanges and finishes its slice.
+template <int BN, int S, int STAGES = 4>
 struct SplitKCfg {
   static constexpr int kSlice = BN / S;                          // columns a CTA finishes
   static_assert(kSlice == 32 || kSlice == 64, "a CTA finishes one or two 32-column chunks");
   static constexpr int kStage = kBM * kBK * 2 + BN * kBK * 2;
-  static constexpr int kStages = 4;
+  static constexpr int kStages = STAGES;
   static constexpr int kRing = kStage * kStages;
   static constexpr int kChunk = kBM * 32 * 4;                    // 128 rows x 32 fp32 = 16 KB
   static constexpr int kSlot = (kSlice / 32) * kChunk;           // one peer's partial slice
@@ -64,11 +66,11 @@ __device__ __forceinline__ void apply_act32(int act, float scale, float (&f)[32]
   }
 }
 
-template <int BN, int S>
+template <int BN, int S, int STAGES = 4>
 __global__ void __launch_bounds__(kNumThreads, 1)
 umma_splitk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                    const UmmaParams p, const int act) {
-  using C = SplitKCfg<BN, S>;
+  using C = SplitKCfg<BN, S, STAGES>;
   constexpr int kStages = C::kStages;
   const uint32_t rank = cluster_ctarank();
   const int tile = static_cast<int>(blockIdx.x) / S;
@@ -112,6 +114,9 @@ umma_splitk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   griddep_launch_dependents();
 
   bool have_acc = false;       // epilogue threads: this CTA's accumulator is complete
+  // Rows of the tile that exist (few for skinny problems), rounded up to whole warps: only they
+  // are exchanged, added and stored; the epilogue warps above them only attend the barriers.
+  const int rows32 = (min(kBM, p.M - tm * kBM) + 31) & ~31;
   if (warp == 0) {
     // every lane waits (warp-uniform loop), one elected lane issues
     int s = 0; uint32_t ph = 0;
@@ -152,7 +157,8 @@ umma_splitk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   } else {
     bool ok = true;
     if (threadIdx.x == 64) {
-      mbar_expect_tx(recv_bar, C::kSlots);      // armed before barrier A, i.e. before any peer sends
+      // armed before barrier A, i.e. before any peer sends: per peer and chunk, the live rows
+      mbar_expect_tx(recv_bar, static_cast<uint32_t>((S - 1) * (C::kSlice / 32) * rows32 * 128));
       ok = mbar_wait(tmem_full, 0, abort_flag, p.status, KF_DEV_TIMEOUT_EPILOGUE);
     }
     have_acc = named_barrier_and(1, kEpiThreads, ok);
@@ -165,6 +171,7 @@ umma_splitk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
 
   const int quad = warp & 3;
   const int row = quad * 32 + lane;                       // tile row = TMEM lane (epilogue warps)
+  const bool warp_live = quad * 32 < rows32;              // this warp's rows exist
   const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
   // Partial slices live as [slot][chunk of 32 columns][row][8 x 16 bytes], the 16-byte position
   // xor-ed with the row so that a quarter warp covers all banks.  Outgoing slots first, then
@@ -187,7 +194,7 @@ umma_splitk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       for (int i = 1; i < S; ++i) {
         const uint32_t d = (rank + i) % S;
 #pragma unroll 1
-        for (int ch = 0; ch < C::kSlice / 32; ++ch) {
+        for (int ch = 0; ch < C::kSlice / 32 && warp_live; ++ch) {
           uint32_t v[32];
           tmem_ld_32x32(t_acc + d * C::kSlice + ch * 32, v);
           tmem_ld_wait();
@@ -200,9 +207,10 @@ umma_splitk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         named_barrier_sync(2, kEpiThreads);
         if (threadIdx.x == 64) {
           const int slot = static_cast<int>(rank < d ? rank : rank - 1);
-          bulk_copy_to_peer(mapa_shared(smem_u32(incoming + slot * C::kSlot), d),
-                            smem_u32(ring + (i - 1) * C::kSlot), C::kSlot,
-                            mapa_shared(smem_u32(recv_bar), d));
+          for (int ch = 0; ch < C::kSlice / 32; ++ch)      // a chunk's rows are contiguous: the live prefix
+            bulk_copy_to_peer(mapa_shared(smem_u32(incoming + slot * C::kSlot + ch * C::kChunk), d),
+                              smem_u32(ring + (i - 1) * C::kSlot + ch * C::kChunk),
+                              static_cast<uint32_t>(rows32 * 128), mapa_shared(smem_u32(recv_bar), d));
         }
       }
     }
@@ -224,7 +232,7 @@ umma_splitk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     have_all = named_barrier_and(1, kEpiThreads, ok);
   }
 
-  if (warp >= 2 && have_all) {
+  if (warp >= 2 && have_all && warp_live) {
     __nv_bfloat16* Y = reinterpret_cast<__nv_bfloat16*>(p.out);
     const long long m = m_row;
     const bool row_ok = m < p.M;
@@ -302,11 +310,11 @@ umma_splitk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   }
 }
 
-template <int BN, int S>
+template <int BN, int S, int STAGES = 4>
 inline cudaError_t launch_splitk_instance(const CUtensorMap& tmA, const CUtensorMap& tmB,
                                           const UmmaParams& p, int act, cudaStream_t st) {
-  using C = SplitKCfg<BN, S>;
-  auto kern = umma_splitk_kernel<BN, S>;
+  using C = SplitKCfg<BN, S, STAGES>;
+  auto kern = umma_splitk_kernel<BN, S, STAGES>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kTotal);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};

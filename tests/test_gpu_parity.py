@@ -218,7 +218,10 @@ def test_bf16_gemm_tile_widths_and_unaligned_rows(kf, shape):
                                    (200, 300, 1800),      # 4 tiles x 4 CTAs, ragged M, N, K (28.1 K blocks)
                                    (100, 128, 4096),      # 128-column tile x 4 CTAs
                                    (64, 2000, 2048),      # 8 tiles x 8 CTAs, last tile ragged in N
-                                   (130, 777, 1848)])     # unaligned rows: scalar stores
+                                   (130, 777, 1848),      # unaligned rows: scalar stores
+                                   (16, 5000, 2048),      # 40 tiles x 4 CTAs, two CTAs per SM, 32 live rows
+                                   (40, 4800, 8192),      # ... long K shares, 64 live rows
+                                   (97, 2048, 1920)])     # 128 live rows, one CTA per SM
 def test_bf16_gemm_split_k_cluster_kernel(kf, shape):
     M, N, K = shape
     d = ki.gemm_inputs("c2", seed=31, M=M, N=N, K=K)

@@ -823,8 +823,15 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
       // (only while every row block's cluster is resident at once: 7 clusters of 16, 15 of 8, 33
       // of 4 fit on the GPU; 1024^3, eight row blocks of 16 tiles, took 19.1 us in two rounds
       // against 17.0 us for the two-kernel route)
-      if (bn == kRowReduceNarrowBN && p.tiles_n >= 2 && p.tiles_n <= 16 &&
-          static_cast<int64_t>(p.tiles_m) * p.tiles_n <= 112 && getenv("KF_NO_CLUSTER_SOFTMAX") == nullptr) {
+      // (where the 128-column form below can take the problem, the narrow form keeps only the
+      // small ones, up to 80 CTAs: 1024x768x512 11.8 us in clusters of 12 narrow tiles, 8.7 us
+      // in clusters of 6 wide ones; 512x640x1024 9.5 against 10.3 us)
+      const int64_t tn128 = (N + 127) / 128;
+      const bool cl128_ok = bn == kRowReduceNarrowBN && out_dtype == KF_BF16 && p.staged && tn128 >= 2 &&
+                            tn128 <= 8 && static_cast<int64_t>(p.tiles_m) * tn128 <= env_int("KF_CL128_MAX_CTAS", 120);
+      const bool cl64 = bn == kRowReduceNarrowBN && p.tiles_n >= 2 && p.tiles_n <= 16 &&
+                        static_cast<int64_t>(p.tiles_m) * p.tiles_n <= (cl128_ok ? 80 : 112);
+      if (cl64 && getenv("KF_NO_CLUSTER_SOFTMAX") == nullptr) {
         UmmaParams pc = p;
         pc.gn_cluster = p.tiles_n;
         pc.num_tiles = p.tiles_m;            // the schedule counts row blocks
@@ -838,10 +845,7 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
       // Rows of 2..8 tiles of 128 columns whose narrow-tile clusters would not all be resident:
       // the same kernel with 128-column tiles and clusters of at most 8 (15 fit on the GPU).
       {
-        const int64_t tn128 = (N + 127) / 128;
-        if (bn == kRowReduceNarrowBN && out_dtype == KF_BF16 && p.staged && tn128 >= 2 && tn128 <= 8 &&
-            static_cast<int64_t>(p.tiles_m) * tn128 <= env_int("KF_CL128_MAX_CTAS", 120) &&
-            static_cast<int64_t>(p.tiles_m) * p.tiles_n > 112 && getenv("KF_NO_CLUSTER_SOFTMAX") == nullptr) {
+        if (cl128_ok && !cl64 && getenv("KF_NO_CLUSTER_SOFTMAX") == nullptr) {
           UmmaMaps tc = tm;
           if (!encode_2d(&tc.b, W, N, K, ldw, 128)) return KF_ERR_CUDA;
           UmmaParams pc = p;

@@ -542,7 +542,8 @@ def test_gemm_groupnorm(kf, dtype, shape, groups, monkeypatch):
                                    (128, 1024, 2048),        # clusters of 16 x 32 K blocks
                                    (1024, 1024, 1024),       # 128-column tiles, clusters of 8
                                    (1100, 1000, 64),         # ... ragged last tile and row block
-                                   (1700, 600, 520)])        # ... fourteen row blocks, clusters of 5
+                                   (1700, 600, 520),         # ... fourteen row blocks, clusters of 5
+                                   (1024, 768, 512)])        # 96 narrow CTAs: the 128-column form, clusters of 6
 def test_bf16_softmax_one_kernel(kf, shape, monkeypatch):
     M, N, K = shape
     d = ki.gemm_inputs("c3", seed=41, M=M, N=N, K=K)
@@ -559,10 +560,10 @@ def test_bf16_softmax_one_kernel(kf, shape, monkeypatch):
     # lies in one tile, or in 2..16 narrow tiles (their CTAs form a cluster); else two.
     bn = 64 if ((M + 127) // 128) * ((N + 63) // 64) <= 148 else 256
     tiles = ((M + 127) // 128) * ((N + 63) // 64)
-    # Narrow-tile clusters that would not all be resident (more than 112 CTAs): 128-column tiles
-    # in clusters of at most 8, while those are at most 120 CTAs.
-    cl64 = bn == 64 and (N + 63) // 64 <= 16 and tiles <= 112
-    cl128 = bn == 64 and tiles > 112 and 2 <= (N + 127) // 128 <= 8 and ((M + 127) // 128) * ((N + 127) // 128) <= 120
+    # Narrow-tile clusters of more than 80 CTAs (or that would not all be resident, more than
+    # 112): 128-column tiles in clusters of at most 8, while those are at most 120 CTAs.
+    cl128 = bn == 64 and 2 <= (N + 127) // 128 <= 8 and ((M + 127) // 128) * ((N + 127) // 128) <= 120
+    cl64 = bn == 64 and (N + 63) // 64 <= 16 and tiles <= (80 if cl128 else 112)
     assert launches == (1 if (N <= bn or cl64 or cl128) else 2)
     # the two-kernel route gives the same probabilities up to the rounding of the numerators
     monkeypatch.setenv("KF_NO_FUSED_SOFTMAX", "1")

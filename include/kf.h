@@ -4,9 +4,9 @@
  * pass where a reduction spans tiles), the operator chains the Kernel Foundry paper's search
  * targets: a dense contraction followed by its elementwise and reduction epilogue.  The
  * problem statement mirrored here is the paper's own (Section 3.1 and Appendix A, output
- * requirement 1): a given PyTorch operator chain in, a kernel with "full functional
- * equivalence" out, with every operator computed inside the kernel rather than by an
- * external library call (Section 3.2.2, anti-cheating rule).
+ * requirement 1): a given PyTorch operator chain in, a kernel that computes the same function
+ * out, with every operator computed inside the kernel rather than by an external library
+ * call (Section 3.2.2, anti-cheating rule).
  *
  * Conventions for every entry point
  *   - All tensor pointers are DEVICE pointers on the current CUDA device.  The caller owns
@@ -16,7 +16,9 @@
  *   - Matrices are row-major with a leading dimension in ELEMENTS (ld >= row length).
  *   - dtype KF_F32 = IEEE fp32, KF_BF16 = bfloat16.  bf16 chains accumulate in fp32 on the
  *     tensor cores, apply the epilogue in fp32 and round once (nearest-even) on store.
- *     fp32 chains use fp32 FMA throughout (no TF32).
+ *     fp32 chains never use single-pass TF32: small ones run on fp32 FMA, large ones on the
+ *     tensor cores with every operand split into two TF32 parts (three products per term,
+ *     fp32 running sum), which stays inside the fp32 tolerance.
  *   - bias / gamma / beta vectors have the chain's io dtype.
  *   - Errors are return codes; nothing throws, aborts or prints.  On any code other than
  *     KF_OK no kernel was launched by that call.  Inputs must be finite.
@@ -289,6 +291,17 @@ kf_status kf_selftest_bounded_wait(uint64_t limit_ns, uint64_t* waited_ns, void*
 
 /* Number of kernels the library has launched from this process since load (all streams). */
 int64_t kf_launch_count(void);
+
+/* Host-side state of the call path (no counterpart in the paper: library plumbing).
+ * The dispatch switches (KF_NO_PAIR, KF_NO_SPLITK, KF_NO_FUSED_GN, KF_NO_FUSED_SOFTMAX,
+ * KF_NO_CLUSTER_SOFTMAX, KF_NO_FUSED_POOL, KF_NO_TF32X3) and thresholds (KF_PAIR_MIN_K,
+ * KF_PAIR_MIN_KB_PER_CTA, KF_SPLITK_MIN_KB, KF_SPLITK_TWO_PER_SM, KF_CL128_MAX_CTAS) are read
+ * from the environment once, at the first call; kf_reload_tuning() reads them again (tests
+ * and A/B measurements that force a route).  Encoded TMA tensor maps are cached by (base
+ * pointer, extents, pitches, box, swizzle); kf_tensor_map_cache_stats reports how many
+ * lookups hit and how many had to ask the driver (either pointer may be NULL). */
+void kf_reload_tuning(void);
+void kf_tensor_map_cache_stats(int64_t* hits, int64_t* misses);
 
 const char* kf_status_string(kf_status s);
 int kf_version(void);

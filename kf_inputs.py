@@ -37,11 +37,24 @@ def _u01(key: np.uint64, idx: np.ndarray) -> np.ndarray:
     return (bits >> np.uint64(11)).astype(np.float64) * (1.0 / 9007199254740992.0)
 
 
-def uniform(seed: int, tensor_id: int, shape, lo: float, hi: float) -> np.ndarray:
-    """float64 array of U(lo, hi) draws; element i depends only on (seed, tensor_id, i)."""
+def _element_indices(shape, first):
+    """Flat element indices (uint64) of the slices `first` along axis 0 of a tensor of `shape`."""
+    inner = int(np.prod(shape[1:])) if len(shape) > 1 else 1
+    first = np.asarray(first, dtype=np.uint64).reshape(-1, 1)
+    return (first * np.uint64(inner) + np.arange(inner, dtype=np.uint64).reshape(1, -1)).reshape(-1)
+
+
+def uniform(seed: int, tensor_id: int, shape, lo: float, hi: float, first=None) -> np.ndarray:
+    """float64 array of U(lo, hi) draws; element i depends only on (seed, tensor_id, i).
+
+    ``first`` (indices along axis 0) draws only those slices of the tensor of ``shape``: the
+    values are the ones the full tensor holds there, without generating the rest."""
+    key = _key(seed, tensor_id)
+    if first is not None:
+        u = _u01(key, _element_indices(shape, first))
+        return (lo + (hi - lo) * u).reshape((len(first),) + tuple(shape[1:]))
     n = int(np.prod(shape))
     out = np.empty(n, np.float64)
-    key = _key(seed, tensor_id)
     for s in range(0, n, _CHUNK):
         e = min(n, s + _CHUNK)
         u = _u01(key, np.arange(s, e, dtype=np.uint64))
@@ -49,11 +62,19 @@ def uniform(seed: int, tensor_id: int, shape, lo: float, hi: float) -> np.ndarra
     return out.reshape(shape)
 
 
-def normal(seed: int, tensor_id: int, shape) -> np.ndarray:
-    """float64 array of N(0,1) draws (Box-Muller on two indexed uniforms per element)."""
+def normal(seed: int, tensor_id: int, shape, first=None) -> np.ndarray:
+    """float64 array of N(0,1) draws (Box-Muller on two indexed uniforms per element).
+
+    ``first``: as in uniform()."""
+    key = _key(seed, tensor_id)
+    if first is not None:
+        i = _element_indices(shape, first)
+        u1 = 1.0 - _u01(key, i * np.uint64(2))
+        u2 = _u01(key, i * np.uint64(2) + np.uint64(1))
+        return (np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * math.pi * u2)).reshape(
+            (len(first),) + tuple(shape[1:]))
     n = int(np.prod(shape))
     out = np.empty(n, np.float64)
-    key = _key(seed, tensor_id)
     for s in range(0, n, _CHUNK):
         e = min(n, s + _CHUNK)
         i = np.arange(s, e, dtype=np.uint64)
@@ -121,22 +142,25 @@ def gemm_inputs(name: str, seed: int = 0, M=None, N=None, K=None, dtype=None, ro
     M, N, K = M or M0, N or N0, K or K0
     bound = 1.0 / math.sqrt(K)
     d = {"M": M, "N": N, "K": K, "dtype": dt, "seed": seed, "name": name}
-    Xf = normal(seed, _X, (M, K))
     d["W"] = store(uniform(seed, _W, (N, K), -bound, bound), dt)
     d["b"] = store(uniform(seed, _B, (N,), -bound, bound), dt)
-    Rf = normal(seed, _R, (M, N)) if name == "c2" else None
     if rows is not None:
         rows = np.asarray(rows)
-        Xf = Xf[rows]
-        Rf = Rf[rows] if Rf is not None else None
+        Xf = normal(seed, _X, (M, K), first=rows)
+        Rf = normal(seed, _R, (M, N), first=rows) if name == "c2" else None
         d["M"] = len(rows)
+    else:
+        Xf = normal(seed, _X, (M, K))
+        Rf = normal(seed, _R, (M, N)) if name == "c2" else None
     d["X"] = store(Xf, dt)
     d["R"] = store(Rf, dt) if Rf is not None else None
     return d
 
 
 def conv_inputs(name: str = "c5", seed: int = 0, Nb=None, Cin=None, H=None, W=None, Cout=None,
-                groups=None, dtype=None):
+                groups=None, dtype=None, images=None):
+    """Inputs of the convolution workload.  ``images`` (an index array) returns only those
+    images of x, holding exactly the values the full batch has there (images are independent)."""
     dt, Nb0, Cin0, H0, W0, Cout0, g0 = CONV_CONFIG[name]
     dt = dtype or dt
     Nb, Cin, H, W, Cout = Nb or Nb0, Cin or Cin0, H or H0, W or W0, Cout or Cout0
@@ -145,7 +169,7 @@ def conv_inputs(name: str = "c5", seed: int = 0, Nb=None, Cin=None, H=None, W=No
     return {
         "Nb": Nb, "Cin": Cin, "H": H, "W": W, "Cout": Cout, "groups": groups, "eps": 1e-5,
         "dtype": dt, "seed": seed, "name": name,
-        "x": store(normal(seed, _X, (Nb, Cin, H, W)), dt),
+        "x": store(normal(seed, _X, (Nb, Cin, H, W), first=images), dt),
         "w": store(uniform(seed, _W, (Cout, Cin, 3, 3), -bound, bound), dt),
         "bias": store(uniform(seed, _B, (Cout,), -bound, bound), dt),
     }

@@ -35,7 +35,7 @@ EXPORTS = ["kf_gemm_epilogue", "kf_gemm_rowreduce", "kf_gemm_rowreduce_static",
            "kf_gemm_groupnorm", "kf_gemm_groupnorm_workspace_bytes",
            "kf_gemm_epilogue_workspace_bytes", "kf_gemm_rowreduce_workspace_bytes",
            "kf_conv3x3_workspace_bytes", "kf_device_status", "kf_launch_count",
-           "kf_status_string", "kf_version"]
+           "kf_reload_tuning", "kf_tensor_map_cache_stats", "kf_status_string", "kf_version"]
 
 
 class KfError(RuntimeError):
@@ -98,6 +98,10 @@ def lib() -> ctypes.CDLL:
     L.kf_device_status.argtypes = []
     L.kf_launch_count.restype = i64
     L.kf_launch_count.argtypes = []
+    L.kf_reload_tuning.restype = None
+    L.kf_reload_tuning.argtypes = []
+    L.kf_tensor_map_cache_stats.restype = None
+    L.kf_tensor_map_cache_stats.argtypes = [ctypes.POINTER(i64), ctypes.POINTER(i64)]
     L.kf_status_string.restype = ctypes.c_char_p
     L.kf_status_string.argtypes = [ci]
     L.kf_version.restype = ci
@@ -201,6 +205,18 @@ def kf_device_status() -> int:
 
 def kf_launch_count() -> int:
     return lib().kf_launch_count()
+
+
+def kf_reload_tuning() -> None:
+    """Re-read the KF_* dispatch switches from the environment (they are read once otherwise)."""
+    lib().kf_reload_tuning()
+
+
+def kf_tensor_map_cache_stats():
+    """(hits, misses) of the encoded-tensor-map cache since load."""
+    h, m = ctypes.c_int64(0), ctypes.c_int64(0)
+    lib().kf_tensor_map_cache_stats(ctypes.byref(h), ctypes.byref(m))
+    return int(h.value), int(m.value)
 
 
 def status_string(status: int) -> str:

@@ -14,6 +14,45 @@ using namespace kf;
 
 std::atomic<int64_t> g_launches{0};
 
+// Dispatch switches and thresholds.  They can be overridden from the environment (KF_NO_* to
+// force a route for A/B measurements and for tests that must reach a fallback path, the others
+// to move a threshold); the environment is read ONCE, at the first call, and again only when
+// kf_reload_tuning() is called, so a call on the hot path reads no environment variable.
+struct Tuning {
+  bool no_fused_pool, no_tf32x3, no_splitk, no_pair, no_cluster_softmax, no_fused_softmax, no_fused_gn;
+  int splitk_min_kb, splitk_two_per_sm, pair_min_k, pair_min_kb_per_cta, cl128_max_ctas;
+};
+Tuning g_tune;
+std::atomic<bool> g_tune_loaded{false};
+std::mutex g_tune_mu;
+void load_tuning_locked() {
+  auto flag = [](const char* n) { return getenv(n) != nullptr; };
+  auto num = [](const char* n, int dflt) {
+    const char* v = getenv(n);
+    return (v != nullptr && *v != '\0') ? atoi(v) : dflt;
+  };
+  g_tune.no_fused_pool = flag("KF_NO_FUSED_POOL");
+  g_tune.no_tf32x3 = flag("KF_NO_TF32X3");
+  g_tune.no_splitk = flag("KF_NO_SPLITK");
+  g_tune.no_pair = flag("KF_NO_PAIR");
+  g_tune.no_cluster_softmax = flag("KF_NO_CLUSTER_SOFTMAX");
+  g_tune.no_fused_softmax = flag("KF_NO_FUSED_SOFTMAX");
+  g_tune.no_fused_gn = flag("KF_NO_FUSED_GN");
+  g_tune.splitk_min_kb = num("KF_SPLITK_MIN_KB", 28);
+  g_tune.splitk_two_per_sm = num("KF_SPLITK_TWO_PER_SM", 1);
+  g_tune.pair_min_k = num("KF_PAIR_MIN_K", 2048);
+  g_tune.pair_min_kb_per_cta = num("KF_PAIR_MIN_KB_PER_CTA", 128);
+  g_tune.cl128_max_ctas = num("KF_CL128_MAX_CTAS", 120);
+  g_tune_loaded.store(true, std::memory_order_release);
+}
+inline const Tuning& tune() {
+  if (!g_tune_loaded.load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> lk(g_tune_mu);
+    if (!g_tune_loaded.load(std::memory_order_relaxed)) load_tuning_locked();
+  }
+  return g_tune;
+}
+
 // One status word per device, in static device memory (no allocation on any call path).
 __device__ uint32_t g_dev_status_word;
 
@@ -63,6 +102,56 @@ inline bool valid_dtype(int dt) { return dt == DT_F32 || dt == DT_BF16; }
 inline bool valid_act(int a) { return a >= 0 && a < ACT_COUNT; }
 constexpr int64_t kMaxDim = 2147483647ll;
 
+// Encoded tensor maps are cached: a descriptor depends only on (base, element type, extents,
+// strides, box, swizzle), never on the data, so a call that repeats an earlier call's operands
+// (the normal case: weights, a pre-allocated activation buffer) finds its maps in a small
+// direct-mapped table instead of asking the driver again.  One lock per lookup.
+struct MapKey {
+  const void* base;
+  uint64_t dims[4];
+  uint64_t strides[3];
+  uint32_t box[4];
+  uint32_t rank, dtype, swizzle;
+  bool operator==(const MapKey& o) const { return std::memcmp(this, &o, sizeof(MapKey)) == 0; }
+};
+struct MapSlot {
+  MapKey key;
+  CUtensorMap map;
+  bool used;
+};
+constexpr int kMapSlots = 512;
+std::mutex g_map_mu;
+MapSlot g_map_cache[kMapSlots];
+std::atomic<int64_t> g_map_hits{0}, g_map_misses{0};
+
+bool encode_generic(CUtensorMap* tm, CUtensorMapDataType dt, uint32_t rank, const void* base,
+                    const cuuint64_t* dims, const cuuint64_t* strides, const cuuint32_t* box,
+                    CUtensorMapSwizzle swz) {
+  MapKey k;
+  std::memset(&k, 0, sizeof(k));
+  k.base = base; k.rank = rank; k.dtype = static_cast<uint32_t>(dt); k.swizzle = static_cast<uint32_t>(swz);
+  for (uint32_t i = 0; i < rank; ++i) { k.dims[i] = dims[i]; k.box[i] = box[i]; }
+  for (uint32_t i = 0; i + 1 < rank; ++i) k.strides[i] = strides[i];
+  uint64_t h = 1469598103934665603ull;                       // FNV-1a over the key's words
+  const uint64_t* w = reinterpret_cast<const uint64_t*>(&k);
+  for (size_t i = 0; i < sizeof(MapKey) / 8; ++i) { h ^= w[i]; h *= 1099511628211ull; }
+  MapSlot& slot = g_map_cache[(h ^ (h >> 29)) % kMapSlots];
+  {
+    std::lock_guard<std::mutex> lk(g_map_mu);
+    if (slot.used && slot.key == k) { *tm = slot.map; ++g_map_hits; return true; }
+  }
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  if (g_encode(tm, dt, rank, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  std::lock_guard<std::mutex> lk(g_map_mu);
+  slot.key = k; slot.map = *tm; slot.used = true;
+  ++g_map_misses;
+  return true;
+}
+static_assert(sizeof(MapKey) % 8 == 0, "the key is hashed as 64-bit words");
+
 // bf16 row-major [rows, cols] with leading dimension ld -> boxes of box_rows x box_cols,
 // zero fill outside the tensor on loads, clipping on stores.  Operand tiles use 64 columns with
 // the 128-byte swizzle; epilogue pieces use 32 columns with the 64-byte swizzle.
@@ -72,11 +161,7 @@ bool encode_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, in
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
   const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
   const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
-  const cuuint32_t estr[2] = {1, 1};
-  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides,
-                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
-                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
-         CUDA_SUCCESS;
+  return encode_generic(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, swz);
 }
 // fp32 row-major [rows, cols] with pitch ld (a multiple of 4 elements) -> boxes of box_rows x 16
 // columns (64 bytes) with the 64-byte swizzle, zero fill outside the tensor.
@@ -85,11 +170,8 @@ bool encode_2d_f32(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
   const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 4};
   const cuuint32_t box[2] = {16u, static_cast<cuuint32_t>(box_rows)};
-  const cuuint32_t estr[2] = {1, 1};
-  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides,
-                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
-                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
-         CUDA_SUCCESS;
+  return encode_generic(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box,
+                        CU_TENSOR_MAP_SWIZZLE_64B);
 }
 // NHWC fp32 activations [Nb,H,W,C] (C a multiple of 16) -> boxes of 16 channels x box_w pixels x
 // rows image rows, 64-byte swizzle, zero fill outside the image.
@@ -100,11 +182,8 @@ bool encode_nhwc_f32(CUtensorMap* tm, const void* base, int64_t Nb, int64_t H, i
   const cuuint64_t strides[3] = {static_cast<cuuint64_t>(C) * 4, static_cast<cuuint64_t>(Wd) * C * 4,
                                  static_cast<cuuint64_t>(H) * Wd * C * 4};
   const cuuint32_t box[4] = {16u, static_cast<cuuint32_t>(box_w), static_cast<cuuint32_t>(rows), 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(base), dims, strides,
-                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
-                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
-         CUDA_SUCCESS;
+  return encode_generic(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, base, dims, strides, box,
+                        CU_TENSOR_MAP_SWIZZLE_64B);
 }
 bool encode_piece(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld) {
   return encode_2d(tm, base, rows, cols, ld, kBM, kPieceCols, CU_TENSOR_MAP_SWIZZLE_64B);
@@ -124,11 +203,8 @@ bool encode_nhwc(CUtensorMap* tm, const void* base, int64_t Nb, int64_t H, int64
                                  static_cast<cuuint64_t>(H) * Wd * C * 2};
   const cuuint32_t box[4] = {static_cast<cuuint32_t>(kBK), static_cast<cuuint32_t>(box_w),
                              static_cast<cuuint32_t>(rows), 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides,
-                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
-         CUDA_SUCCESS;
+  return encode_generic(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box,
+                        CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 // NCHW bf16 output seen as [Nb][C][H*W] -> store boxes of 32 pixels x 32 channels of one image
@@ -139,11 +215,8 @@ bool encode_nchw_out(CUtensorMap* tm, const void* base, int64_t Nb, int64_t C, i
   const cuuint64_t strides[2] = {static_cast<cuuint64_t>(hw) * 2,
                                  static_cast<cuuint64_t>(C) * hw * 2};
   const cuuint32_t box[3] = {static_cast<cuuint32_t>(kPieceCols), 32, 1};   // one warp's slab of a piece
-  const cuuint32_t estr[3] = {1, 1, 1};
-  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides,
-                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
-                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
-         CUDA_SUCCESS;
+  return encode_generic(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box,
+                        CU_TENSOR_MAP_SWIZZLE_64B);
 }
 
 // Can the tensor-core GEMM take these operands?  (TMA: 16-byte aligned base and row pitch.)
@@ -186,12 +259,12 @@ bool conv_pool_fused_ok(int dt, int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, 
   (void)Nb; (void)Cin; (void)Cout;
   if (dt != DT_BF16 || pool != 2 || !conv_umma_shape_ok(dt, Cin, H, Wd, Cout)) return false;
   const int rows = conv_rows_per_tile(H, Wd);
-  return Wd % 32 == 0 && Wd <= 256 && rows % 2 == 0 && H % 2 == 0 && getenv("KF_NO_FUSED_POOL") == nullptr;
+  return Wd % 32 == 0 && Wd <= 256 && rows % 2 == 0 && H % 2 == 0 && !tune().no_fused_pool;
 }
 // fp32 convolutions large enough for the tensor cores take the 3xTF32 implicit GEMM
 int64_t conv32_cpad(int64_t Cin) { return (Cin + 15) / 16 * 16; }
 bool conv_tf32_ok(int dt, int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout) {
-  if (dt != DT_F32 || getenv("KF_NO_TF32X3") != nullptr) return false;
+  if (dt != DT_F32 || tune().no_tf32x3) return false;
   return conv_rows_per_tile(H, Wd) > 0 && Nb * H * Wd * Cout * Cin >= (int64_t{1} << 24);
 }
 size_t conv_tf32_ws(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout) {
@@ -283,7 +356,7 @@ bool repack_bf16(int64_t M, int64_t N, int64_t K, const void* X, int64_t ldx, co
 // TF32 hi + lo parts in the workspace); smaller ones stay on the fp32 FMA kernel (measured:
 // 512^3 18.6 us FMA / 35 us tensor, 1024^3 112 / 54 us, 4096^3 6569 / 667 us).
 bool use_tf32x3(int dt, int64_t M, int64_t N, int64_t K) {
-  if (dt != DT_F32 || getenv("KF_NO_TF32X3") != nullptr) return false;
+  if (dt != DT_F32 || tune().no_tf32x3) return false;
   if (M < 64 || N < 64 || K < 64) return false;
   if (M * N * K >= (int64_t{1} << 29)) return true;
   // from 2^28 when there are enough tiles to spread over the SMs (768^3: 49.8 us FMA, 28 us here)
@@ -296,21 +369,15 @@ size_t tf32_ws(int64_t M, int64_t N, int64_t K) {
          2 * round256(static_cast<size_t>(N) * tf32_kp(K) * 4);
 }
 
-// Tuning thresholds can be overridden from the environment (measurement aid).
-int env_int(const char* name, int dflt) {
-  const char* v = getenv(name);
-  return (v != nullptr && *v != '\0') ? atoi(v) : dflt;
-}
-
 // Cluster size of the split-K kernel, or 0.  Measured on B200: a narrow-tile CTA spends about
 // 0.16 us per K block, the cluster exchange costs about 4 us, so splitting pays from about 28 K
 // blocks (K = 1536: 9.9 us split, 8.9 us plain; K = 2048: 9.4 against 10.7 us); clusters of 8 schedule well only while there are few
 // of them (16 clusters of 8 already ran in two waves).
 int pick_split_k(int64_t M, int64_t N, int64_t K, int sm_count, int* bn_out) {
   *bn_out = N <= 128 ? 128 : 256;
-  if (getenv("KF_NO_SPLITK") != nullptr) return 0;
+  if (tune().no_splitk) return 0;
   const int64_t kb = (K + kBK - 1) / kBK;
-  if (kb < env_int("KF_SPLITK_MIN_KB", 28)) return 0;
+  if (kb < tune().splitk_min_kb) return 0;
   // cluster size for tiles of `bn` columns, and the CTAs that gives
   auto split_for = [&](int bn, int64_t* ctas) {
     const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + bn - 1) / bn);
@@ -322,7 +389,7 @@ int pick_split_k(int64_t M, int64_t N, int64_t K, int sm_count, int* bn_out) {
     // (64x8192x8192 26.9 -> 25.6 us, 32x5120x8192 19.1 -> 18.7, 16x9472x4096 20.8 -> 17.4;
     // 128x8192x4096 13.8 -> 14.4 us, hence the conditions).
     else if (bn == 128 && tiles * 4 <= 2 * (sm_count - sm_count % 4) && (kb >= 128 || M <= 32) &&
-             env_int("KF_SPLITK_TWO_PER_SM", 1) != 0) sk = 4;
+             tune().splitk_two_per_sm != 0) sk = 4;
     else if (bn == 128 && tiles * 2 <= sm_count - sm_count % 2) sk = 2;
     *ctas = tiles * sk;
     return sk;
@@ -340,7 +407,7 @@ int pick_split_k(int64_t M, int64_t N, int64_t K, int sm_count, int* bn_out) {
 }
 
 bool use_cta_pairs(int64_t M, int64_t K) {
-  return M > 256 && K >= env_int("KF_PAIR_MIN_K", 2048) && getenv("KF_NO_PAIR") == nullptr;
+  return M > 256 && K >= tune().pair_min_k && !tune().no_pair;
 }
 // The elementwise chain: the pair kernel runs one epilogue group, the single-CTA kernel two, so
 // pairs pay only where a CTA has enough MMA work to hide its epilogues behind: from about 128
@@ -351,7 +418,7 @@ bool use_cta_pairs_chain(int64_t M, int64_t N, int64_t K, int sm_count) {
   if (!use_cta_pairs(M, K)) return false;
   const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + 255) / 256);
   const int64_t kb = (K + kBK - 1) / kBK;
-  return tiles * kb >= static_cast<int64_t>(env_int("KF_PAIR_MIN_KB_PER_CTA", 128)) * sm_count;
+  return tiles * kb >= static_cast<int64_t>(tune().pair_min_kb_per_cta) * sm_count;
 }
 size_t rowreduce_simt_ws(int64_t M, int64_t N) { return round256(static_cast<size_t>(M) * N * 4); }
 
@@ -434,6 +501,16 @@ const char* kf_status_string(kf_status s) {
 int kf_version(void) { return 100; }
 
 int64_t kf_launch_count(void) { return g_launches.load(); }
+
+void kf_reload_tuning(void) {
+  std::lock_guard<std::mutex> lk(g_tune_mu);
+  load_tuning_locked();
+}
+
+void kf_tensor_map_cache_stats(int64_t* hits, int64_t* misses) {
+  if (hits != nullptr) *hits = g_map_hits.load();
+  if (misses != nullptr) *misses = g_map_misses.load();
+}
 
 kf_status kf_device_status(void) {
   DeviceInfo* d = nullptr;
@@ -828,10 +905,10 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
       // in clusters of 6 wide ones; 512x640x1024 9.5 against 10.3 us)
       const int64_t tn128 = (N + 127) / 128;
       const bool cl128_ok = bn == kRowReduceNarrowBN && out_dtype == KF_BF16 && p.staged && tn128 >= 2 &&
-                            tn128 <= 8 && static_cast<int64_t>(p.tiles_m) * tn128 <= env_int("KF_CL128_MAX_CTAS", 120);
+                            tn128 <= 8 && static_cast<int64_t>(p.tiles_m) * tn128 <= tune().cl128_max_ctas;
       const bool cl64 = bn == kRowReduceNarrowBN && p.tiles_n >= 2 && p.tiles_n <= 16 &&
                         static_cast<int64_t>(p.tiles_m) * p.tiles_n <= (cl128_ok ? 80 : 112);
-      if (cl64 && getenv("KF_NO_CLUSTER_SOFTMAX") == nullptr) {
+      if (cl64 && !tune().no_cluster_softmax) {
         UmmaParams pc = p;
         pc.gn_cluster = p.tiles_n;
         pc.num_tiles = p.tiles_m;            // the schedule counts row blocks
@@ -845,7 +922,7 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
       // Rows of 2..8 tiles of 128 columns whose narrow-tile clusters would not all be resident:
       // the same kernel with 128-column tiles and clusters of at most 8 (15 fit on the GPU).
       {
-        if (cl128_ok && !cl64 && getenv("KF_NO_CLUSTER_SOFTMAX") == nullptr) {
+        if (cl128_ok && !cl64 && !tune().no_cluster_softmax) {
           UmmaMaps tc = tm;
           if (!encode_2d(&tc.b, W, N, K, ldw, 128)) return KF_ERR_CUDA;
           UmmaParams pc = p;
@@ -861,7 +938,7 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
         }
       }
       // a row that lies in one tile is finished in the GEMM epilogue: no second kernel
-      p.softmax_fused = (p.tiles_n == 1 && getenv("KF_NO_FUSED_SOFTMAX") == nullptr) ? 1 : 0;
+      p.softmax_fused = (p.tiles_n == 1 && !tune().no_fused_softmax) ? 1 : 0;
       if (launch_umma_softmax(bn, pre_act, out_dtype, pair ? 1 : 0, tm, p, grid, st) != cudaSuccess)
         return KF_ERR_CUDA;
       if (p.softmax_fused) { g_launches += 1; return KF_OK; }
@@ -1038,7 +1115,7 @@ static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
     const bool gn_fused = groups > 0 && p.staged &&
                           tpi >= 1 && (tpi <= 8 || tpi == 16) &&      // 9..15 pack badly into GPCs (56x56: 43.6 us against 41.5)
                           (cpg == 4 || cpg == 8 || cpg == 16 || cpg == 32) &&
-                          getenv("KF_NO_FUSED_GN") == nullptr;
+                          !tune().no_fused_gn;
     if (gn_fused) {
       p.gn_cluster = tpi; p.gn_groups = groups; p.gn_eps = eps;
       p.gn_gamma = static_cast<const __nv_bfloat16*>(gamma);

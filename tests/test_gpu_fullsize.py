@@ -150,10 +150,10 @@ def test_conv_act_pool_full_size_sampled_images(kf):
     assert float(y.float().min()) >= 0.0
 
 
-def test_c5_two_kernel_route_full_size_sampled_images(kf, monkeypatch):
+def test_c5_two_kernel_route_full_size_sampled_images(kf, tuning):
     """Config 5 through the convolution + separate normalisation kernels (the route shapes take
     that do not qualify for the cluster form)."""
-    monkeypatch.setenv("KF_NO_FUSED_GN", "1")
+    tuning.setenv("KF_NO_FUSED_GN", "1")
     d = ki.conv_inputs("c5", seed=0)
     y = kf.conv3x3_epilogue(to_dev(d["x"]), to_dev(d["w"]), to_dev(d["bias"]), "relu", d["groups"], d["eps"])
     check_status()

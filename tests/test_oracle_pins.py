@@ -518,3 +518,125 @@ def test_channel_softmax_pooling():
     # a ragged rim is dropped
     d3 = ki.conv_inputs(Nb=1, Cin=2, H=5, W=7, Cout=3, groups=0, seed=9)
     assert oracle.conv3x3_softmax_pool(d3["x"], d3["w"], None, pool=2).shape == (1, 3, 2, 3)
+
+
+# ------------------------------------------------------------------ stored fixed points
+def test_activation_fixed_points_from_golden_file():
+    """Values of the activation definitions at fixed points, computed once with 40-digit
+    arithmetic by tests/golden/make_activation_fixed_points.py (no oracle, no GPU)."""
+    path = os.path.join(os.path.dirname(__file__), "golden", "activation_fixed_points.txt")
+    n = 0
+    for line in open(path):
+        line = line.split("#")[0].split()
+        if len(line) == 3:
+            name, z, want = line[0], float(line[1]), float(line[2])
+            assert abs(oracle.act(name, z) - want) <= 4e-16 * max(1.0, abs(want)), (name, z)
+            n += 1
+    assert n == 7
+
+
+# ------------------------------------------------------------------ the worked chain's rewrites
+def test_chain95_rewrites_agree():
+    """Appendix C.2 prints four programs for the same post-matmul chain (iterations 15, 20, 25
+    and 30); they differ only in how the same algebra is written.  Each variant is restated
+    here from its description -- clamp by min/max or by two selects, exp(2s) evaluated twice or
+    once, the erf argument inline or as a temporary -- and all of them must agree with each
+    other and with the oracle's chain95 on a grid (values where exp(2s) is finite)."""
+    c = golden()
+
+    def swish(x):
+        return x / (1.0 + math.exp(-x)) if x > -700 else 0.0
+
+    def clamp_minmax(g):
+        return min(max(g, c["hardtanh_lo"]), c["hardtanh_hi"])
+
+    def clamp_select(g):
+        return c["hardtanh_hi"] if g > c["hardtanh_hi"] else (c["hardtanh_lo"] if g < c["hardtanh_lo"] else g)
+
+    def form_a(x):          # exponential written out twice, clamp by min/max
+        s = swish(x)
+        t = (math.exp(c["tanh_exp_factor"] * s) - 1.0) / (math.exp(c["tanh_exp_factor"] * s) + 1.0)
+        return clamp_minmax(t * 0.5 * (1.0 + math.erf(t * c["erf_gelu_inner_scale"])))
+
+    def form_b(x):          # same, clamp by two selects (two of the printed programs share this form)
+        s = swish(x)
+        t = (math.exp(2 * s) - 1) / (math.exp(2 * s) + 1)
+        return clamp_select(t * 0.5 * (1.0 + math.erf(t * c["erf_gelu_inner_scale"])))
+
+    def form_c(x):          # sigmoid reused, one exponential, erf argument as a temporary
+        sg = 1.0 / (1.0 + math.exp(-x)) if x > -700 else 0.0
+        s = sg * x
+        e2 = math.exp(2.0 * s)
+        t = (e2 - 1.0) / (e2 + 1.0)
+        arg = t * c["erf_gelu_inner_scale"]
+        return clamp_select(t * 0.5 * (1.0 + math.erf(arg)))
+
+    zs = np.concatenate([np.linspace(-30.0, 30.0, 1201), [-300.0, -50.0, 50.0, 300.0, 1e-9, -1e-9]])
+    for z in zs:
+        z = float(z)
+        a, b, cc = form_a(z), form_b(z), form_c(z)
+        assert abs(a - b) < 1e-15 and abs(a - cc) < 1e-15, z
+        assert abs(oracle.act("chain95", z) - a) < 1e-14, z
+    # the chain's range: swish >= -0.2785, so tanh >= -0.2716 and gelu(erf) of it >= -0.107; the
+    # upper clamp is reached only in the limit (gelu_erf(1) = 0.8413 < 1): hardtanh never acts
+    vals = np.array([oracle.act("chain95", float(z)) for z in zs])
+    assert vals.min() > -0.11 and vals.max() < 0.8414
+
+
+# ------------------------------------------------------------------ full-size spot checks
+# One sampled row (image) of every full-size benchmark configuration: the oracle's routine on
+# that row against numpy / scipy fp64 on the same stored inputs.  Rows are independent, and the
+# generator is index-addressed, so a row subset holds exactly the full tensor's values there.
+def _rows_for(M):
+    return np.array([0, M // 2 + 1, M - 1])
+
+
+def test_full_size_c2_rows_against_numpy():
+    rows = _rows_for(8192)
+    d = ki.gemm_inputs("c2", seed=0, rows=rows)
+    got = oracle.gemm_epilogue(d["X"], d["W"], d["b"], "gelu_tanh", 0.5, d["R"])
+    z = ki.widen(d["X"]) @ ki.widen(d["W"]).T + ki.widen(d["b"])
+    want = 0.5 * (0.5 * z * (1.0 + np.tanh(math.sqrt(2.0 / math.pi) * (z + 0.044715 * z ** 3)))) + ki.widen(d["R"])
+    assert got.shape == (3, 4096)
+    assert np.abs(got - want).max() < 1e-12
+
+
+def test_full_size_c3_rows_against_scipy():
+    rows = _rows_for(4096)
+    d = ki.gemm_inputs("c3", seed=0, rows=rows)
+    got = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "none", "softmax")
+    z = ki.widen(d["X"]) @ ki.widen(d["W"]).T + ki.widen(d["b"])
+    want = scipy.special.softmax(z, axis=1)
+    assert got.shape == (3, 8192)
+    assert np.abs(got - want).max() < 1e-15 and np.abs(got / want - 1).max() < 1e-11
+
+
+def test_full_size_c4_rows_against_scipy():
+    rows = _rows_for(16384)
+    d = ki.gemm_inputs("c4", seed=0, rows=rows)
+    got = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "sigmoid", "sum").reshape(-1)
+    z = ki.widen(d["X"]) @ ki.widen(d["W"]).T + ki.widen(d["b"])
+    want = scipy.special.expit(z).sum(axis=1)
+    assert np.abs(got - want).max() < 1e-10
+
+
+def test_full_size_c5_image_against_numpy():
+    d = ki.conv_inputs("c5", seed=0, images=[77])
+    got = oracle.conv3x3_gn(d["x"], d["w"], d["bias"], "relu", d["groups"], d["eps"])
+    x, w, b = ki.widen(d["x"])[0], ki.widen(d["w"]), ki.widen(d["bias"])
+    xp = np.pad(x, ((0, 0), (1, 1), (1, 1)))
+    win = np.lib.stride_tricks.sliding_window_view(xp, (3, 3), axis=(1, 2))      # [c, h, w, r, s]
+    y = np.tensordot(w, win, axes=([1, 2, 3], [0, 3, 4])) + b[:, None, None]      # [o, h, w]
+    a = np.maximum(y, 0.0).reshape(d["groups"], -1)
+    want = ((a - a.mean(axis=1, keepdims=True)) / np.sqrt(a.var(axis=1, keepdims=True) + d["eps"])).reshape(y.shape)
+    assert got.shape == (1, 128, 64, 64)
+    assert np.abs(got[0] - want).max() < 1e-11
+
+
+def test_generator_row_subsets_hold_the_full_tensor_values():
+    a = ki.gemm_inputs("c2", seed=3, M=40, N=24, K=16)
+    b = ki.gemm_inputs("c2", seed=3, M=40, N=24, K=16, rows=[3, 39, 0])
+    assert (a["X"][[3, 39, 0]] == b["X"]).all() and (a["R"][[3, 39, 0]] == b["R"]).all()
+    c = ki.conv_inputs(seed=2, Nb=5, Cin=3, H=4, W=6, Cout=2)
+    e = ki.conv_inputs(seed=2, Nb=5, Cin=3, H=4, W=6, Cout=2, images=[4, 1])
+    assert (c["x"][[4, 1]] == e["x"]).all()

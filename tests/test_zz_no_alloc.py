@@ -6,13 +6,14 @@ so the library keeps the per-tile partial statistics in a fixed array of its own
 calls the entry point through the C ABI twice in a row -- the second time on a different,
 smaller problem, so that whatever the first call left in the shared array would show up if it
 were ever read -- and checks each result against kf_gemm_rowreduce with a caller-owned
-workspace.  This file sorts last on purpose: a run that stops at the first failure has then
+workspace (bit for bit) and against the fp64 CPU oracle on the same seeded inputs.  This file sorts last on purpose: a run that stops at the first failure has then
 already run every other test.
 """
 import numpy as np
 import pytest
 
 import kf_inputs as ki
+import oracle
 import paper_2605_30359_b200 as kf
 from gpu_util import assert_close, check_status, to_dev, to_f64
 
@@ -45,6 +46,13 @@ def test_static_scratch_matches_workspace_variant_twice_in_a_row():
         check_status()
         assert_close(to_f64(out), to_f64(ref), 2e-2, 2e-2, "%s %s static vs workspace" % (name, red))
         assert torch.equal(out, ref)                        # same kernels, same order: same bits
+        # and against the definition itself: the fp64 oracle, with the gates the row reductions use
+        want = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], act, red).reshape(to_f64(out).shape)
+        assert_close(to_f64(out), want, 2e-2, 2e-2, "%s %s static vs oracle" % (name, red))
+        if red == "softmax":
+            assert_close(to_f64(out), want, 1e-7, 2e-2, "%s static vs oracle, relative" % name)
+        else:
+            assert_close(to_f64(out), want, 0.0, 1e-3, "%s static vs oracle, relative" % name)
 
 
 def test_static_scratch_rejects_oversized_problems():
@@ -52,7 +60,7 @@ def test_static_scratch_rejects_oversized_problems():
     kf.lib()
     before = kf.kf_launch_count()
     p = 0x10000
-    # softmax partials for 16384 x 8192: 16384 * 32 * 8 bytes = 4 MiB > the 2 MiB array
+    # softmax partials for 16384 x 8192: 16384 rows * 32 tiles * 16 bytes (two float2 per tile) = 8 MiB > the 2 MiB array
     assert kf.kf_gemm_rowreduce_workspace_bytes(16384, 8192, 1024, kf.KF_BF16, 0) > kf.KF_STATIC_SCRATCH_BYTES
     st = kf.kf_gemm_rowreduce_static(16384, 8192, 1024, kf.KF_BF16, p, 1024, p, 1024, None, 0, 0,
                                      p + 4096, 8192, kf.KF_BF16, None)

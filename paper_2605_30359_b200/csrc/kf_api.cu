@@ -19,7 +19,7 @@ std::atomic<int64_t> g_launches{0};
 // to move a threshold); the environment is read ONCE, at the first call, and again only when
 // kf_reload_tuning() is called, so a call on the hot path reads no environment variable.
 struct Tuning {
-  bool no_fused_pool, no_tf32x3, no_splitk, no_pair, no_cluster_softmax, no_fused_softmax, no_fused_gn;
+  bool no_fused_pool, no_tf32x3, no_splitk, no_pair, no_cluster_softmax, no_fused_softmax, no_fused_gn, no_conv_slab;
   int splitk_min_kb, splitk_two_per_sm, pair_min_k, pair_min_kb_per_cta, cl128_max_ctas;
 };
 Tuning g_tune;
@@ -38,6 +38,7 @@ void load_tuning_locked() {
   g_tune.no_cluster_softmax = flag("KF_NO_CLUSTER_SOFTMAX");
   g_tune.no_fused_softmax = flag("KF_NO_FUSED_SOFTMAX");
   g_tune.no_fused_gn = flag("KF_NO_FUSED_GN");
+  g_tune.no_conv_slab = flag("KF_NO_CONV_SLAB");
   g_tune.splitk_min_kb = num("KF_SPLITK_MIN_KB", 28);
   g_tune.splitk_two_per_sm = num("KF_SPLITK_TWO_PER_SM", 1);
   g_tune.pair_min_k = num("KF_PAIR_MIN_K", 2048);
@@ -1103,6 +1104,17 @@ static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
     p.status = d->status;
     p.H = static_cast<int>(H); p.Wd = static_cast<int>(Wd); p.Cin = static_cast<int>(Cp);
     p.rows_per_tile = rows;
+    // Slab mode (see UmmaParams::slab): the pixel window with its halo rows is fetched once per
+    // column shift instead of once per tap, which cuts the pixel traffic from L2 into the SM to
+    // a third.  Needs whole 1024-byte groups per image row of the copy (8 pixels of 128 bytes)
+    // and a copy of at most 48 KB.
+    const int box_w = static_cast<int>(Wd / segs);
+    if (box_w % 8 == 0 && (rows + 2) * box_w <= 384 && rows + 2 <= 256 && !tune().no_conv_slab) {
+      if (!encode_nhwc(&tm.r, xt, Nb, H, Wd, Cp, rows + 2, box_w)) return KF_ERR_CUDA;
+      p.slab = 1;
+      p.slab_bytes = (rows + 2) * box_w * kBK * 2;
+      p.slab_row_bytes = box_w * kBK * 2;
+    }
     // the output pieces travel by TMA when every image plane starts on 16 bytes
     p.staged = (!gap_in_epilogue && aligned(y, 16) && hw % 8 == 0) ? 1 : 0;
     if (pool2 != 0) { p.pool2 = pool2; p.staged = 0; p.vec_ok = aligned(y, 16) ? 1 : 0; }

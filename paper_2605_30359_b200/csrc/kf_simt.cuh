@@ -467,10 +467,12 @@ conv_prep_kernel(int Nb, int Cin, int H, int Wd, int Cout, const __nv_bfloat16* 
   const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   const int wb = Wd / 8, cbk = Cin / 8;
   if (gid < x_blocks) {
-    // gid -> (n, h, cblk, wblk) with wblk fastest: neighbouring lanes read one row of x
-    const int wblk = static_cast<int>(gid % wb);
-    long long t = gid / wb;
-    const int cblk = static_cast<int>(t % cbk); t /= cbk;
+    // gid -> (n, h, wblk, cblk) with cblk fastest: the lanes that hold one pixel's channel blocks
+    // write whole 128-byte stretches of its NHWC row (L2 takes a 16-byte write request as long as
+    // a 128-byte one); the reads still cover 64-byte runs of a row of x
+    const int cblk = static_cast<int>(gid % cbk);
+    long long t = gid / cbk;
+    const int wblk = static_cast<int>(t % wb); t /= wb;
     const int h = static_cast<int>(t % H);
     const long long n = t / H;
     const long long hw = static_cast<long long>(H) * Wd;

@@ -105,6 +105,11 @@ struct UmmaParams {
   int gn_cluster;              // EPI_CONV_GN: CTAs per cluster = pixel tiles per image (1..8 or 16);
                                // EPI_SOFTMAX_CL: CTAs per cluster = column tiles per row (2..16)
   int gn_groups;               // EPI_CONV_GN: GroupNorm groups (channels per group a power of two, 4..32)
+  int slab;                    // convolution: 1 = the producer loads, per column shift, ONE copy of the tile's
+                               // pixel window with its two halo rows ((rows_per_tile + 2) x box_w pixels,
+                               // through tmR) and the three row taps read it at offsets of whole rows
+  int slab_bytes;              // bytes of one such copy (<= 48 KB)
+  int slab_row_bytes;          // bytes of one image row of the copy: box_w * 128, a multiple of 1024
   int pool2;                   // convolution: 0, or 2x2 pooling in the epilogue (1 = max, 2 = mean);
                                // needs w_segs == 1, Wd % 32 == 0, rows_per_tile and H even
 };
@@ -264,6 +269,15 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   uint64_t* rbar = r_full + 8;             // EPI_CONV_GN: [2] statistics from the cluster have arrived
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(rbar + 2);   // r_full: [epilogue warp][2]
   volatile uint32_t* abort_flag = tmem_holder + 1;
+  // Convolution in slab mode: the ring holds two pixel copies of up to 48 KB and six weight slots
+  // of 16 KB; its sixteen barriers are the stage barriers followed by r_full's (which only the
+  // elementwise chain uses): weight slot full [0,6), empty [6,12), copy full [12,14), empty [14,16).
+  [[maybe_unused]] constexpr int kSlabPx = 49152;
+  [[maybe_unused]] constexpr int kSlabW = 6;
+  static_assert(!is_conv(EPI) || (C::kRing >= 2 * kSlabPx + kSlabW * C::kStageA && kStages >= 4), "slab layout");
+  [[maybe_unused]] auto slab_bar = [&](int i) -> uint64_t* {
+    return i < 2 * kStages ? full + i : r_full + (i - 2 * kStages);
+  };
 
   // The warp index comes out of a shuffle so that the compiler knows it is the same in every
   // lane: the producer and issuer loops below then run with warp-uniform control flow, and the
@@ -313,6 +327,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // every lane waits for the stage (so the loop stays warp-uniform); one elected lane issues
     {
       int s = 0; uint32_t ph = 0;
+      [[maybe_unused]] int pb = 0; [[maybe_unused]] uint32_t pph = 0;   // slab mode: pixel-copy buffer and its phase
       for (int it = 0;; ++it) {
         const int tile = tile_at(it);
         if (tile < 0) break;
@@ -327,6 +342,36 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           tm = tile / p.tiles_n; tn = tile % p.tiles_n;
         }
         bool ok = true;
+        if constexpr (is_conv(EPI)) {
+          if (p.slab) {
+            // Per 64-channel block and column shift: one copy of the window with its halo rows
+            // (out-of-image pixels read zeros: the padding), then the three row taps' weights.
+            for (int cs = 0; cs < 3 * p.kb_per_tap && ok; ++cs) {
+              const int cb = cs / 3, sx = cs % 3;
+              ok = mbar_wait(slab_bar(12 + 2 + pb), pph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_PRODUCER);
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+              if (elect_one()) {
+                mbar_expect_tx(slab_bar(12 + pb), static_cast<uint32_t>(p.slab_bytes));
+                tma_load_4d(ring + pb * kSlabPx, &tmR, slab_bar(12 + pb), cb * kBK, x0 + sx - 1, h0 - 1, img);
+              }
+              if (++pb == 2) { pb = 0; pph ^= 1u; }
+              for (int r = 0; r < 3; ++r) {
+                ok = mbar_wait(slab_bar(6 + s), ph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_PRODUCER);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (elect_one()) {
+                  mbar_expect_tx(slab_bar(s), C::kStageA);
+                  tma_load_2d(ring + 2 * kSlabPx + s * C::kStageA, &tmA, slab_bar(s), cb * kBK,
+                              (r * 3 + sx) * p.N + tm * kBM);
+                }
+                if (++s == kSlabW) { s = 0; ph ^= 1u; }
+              }
+            }
+            if (!ok) break;
+            continue;
+          }
+        }
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           ok = mbar_wait(&empty[s], ph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_PRODUCER);
           ok = __all_sync(0xffffffffu, ok);
@@ -371,6 +416,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const uint32_t idesc =
           umma_idesc_bf16_f32(kTileM, is_conv(EPI) ? static_cast<uint32_t>(p.tile_px) : BN);
       int s = 0; uint32_t ph = 0; int a = 0; uint32_t aph = 0;
+      [[maybe_unused]] int pb = 0; [[maybe_unused]] uint32_t pph = 0;   // slab mode: pixel-copy buffer and its phase
       bool ok = true;
       for (int it = 0; ok; ++it) {
         if (tile_at(it) < 0) break;
@@ -379,6 +425,38 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(a * BN);
+        if constexpr (is_conv(EPI)) {
+          if (p.slab) {
+            for (int cs = 0; cs < 3 * p.kb_per_tap && ok; ++cs) {
+              ok = mbar_wait(slab_bar(12 + pb), pph, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+              const uint32_t px = smem_u32(ring + pb * kSlabPx);
+              for (int r = 0; r < 3; ++r) {
+                ok = mbar_wait(slab_bar(s), ph, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint64_t adesc = smem_desc_kmajor_sw128(smem_u32(ring + 2 * kSlabPx + s * C::kStageA));
+                // the window of tap row r starts r image rows (whole 1024-byte groups) into the copy
+                const uint64_t bdesc = smem_desc_kmajor_sw128(px + static_cast<uint32_t>(r * p.slab_row_bytes));
+                if (elect_one()) {
+#pragma unroll
+                  for (int k = 0; k < kBK / kUmmaK; ++k)
+                    umma_f16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (cs | r | k) != 0 ? 1u : 0u);
+                  umma_commit(slab_bar(6 + s));                   // frees the weight slot
+                  if (r == 2) umma_commit(slab_bar(12 + 2 + pb));  // ... and, after the third tap, the copy
+                }
+                if (++s == kSlabW) { s = 0; ph ^= 1u; }
+              }
+              if (++pb == 2) { pb = 0; pph ^= 1u; }
+            }
+            if (!ok) break;
+            if (elect_one()) umma_commit(&tmem_full[a]);
+            if (++a == 2) { a = 0; aph ^= 1u; }
+            continue;
+          }
+        }
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           ok = mbar_wait(&full[s], ph, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
           ok = __all_sync(0xffffffffu, ok);

@@ -54,9 +54,17 @@ def load_peaks():
     return d
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the config-2 kernel, from the ncu
-# capture summarised in profiles/umma_chain_kernel_c2_gelu_residual.md (214.7 MB + 52.8 MB)
-TRAFFIC_C2_BYTES = 267.4e6
+def c2_traffic_bytes():
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the config-2 kernel: the figure the
+    committed ncu summary of that kernel states (a line `dram_bytes_per_launch = N`), or None."""
+    path = os.path.join(ROOT, "profiles", "umma_chain_kernel_c2_gelu_residual.md")
+    try:
+        for line in open(path):
+            if line.strip().startswith("dram_bytes_per_launch"):
+                return float(line.split("=")[1].split()[0])
+    except Exception:
+        pass
+    return None
 
 
 # ------------------------------------------------------------------ clocks during the timed region
@@ -153,11 +161,52 @@ def to_pinned(a):
     return t.pin_memory()
 
 
-def time_calls(fn, iters, warmup, graph_batch=0):
-    """Average device time of fn() in microseconds (CUDA events on the current stream).
+def time_calls_stats(fn, iters, warmup, graph_batch=0, flush=None):
+    """Device time of fn() in microseconds: {"mean", "median", "min", "samples"} over CUDA-event pairs
+    on the current stream, one pair per call (per graph replay when graph_batch > 0).
 
     graph_batch > 0 captures that many calls into a CUDA graph first, so that launch-bound
-    chains are timed on the device rather than at the host's launch rate."""
+    chains are timed on the device rather than at the host's launch rate.  flush: a callable run
+    before every timed sample, outside its event pair (the cold-cache variant writes a buffer
+    larger than L2 there)."""
+    import torch
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    runner, per = fn, 1
+    if graph_batch > 0:
+        try:
+            g = torch.cuda.CUDAGraph()
+            s = torch.cuda.Stream()
+            s.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(s):
+                fn()
+                with torch.cuda.graph(g, stream=s):
+                    for _ in range(graph_batch):
+                        fn()
+            torch.cuda.current_stream().wait_stream(s)
+            torch.cuda.synchronize()
+            runner, per = g.replay, graph_batch
+            runner()
+            torch.cuda.synchronize()
+        except Exception:
+            runner, per = fn, 1
+    reps = max(3, iters // per)
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for e0, e1 in pairs:
+        if flush is not None:
+            flush()
+        e0.record()
+        runner()
+        e1.record()
+    torch.cuda.synchronize()
+    t = np.array([e0.elapsed_time(e1) * 1e3 / per for e0, e1 in pairs])
+    return {"mean": float(t.mean()), "median": float(np.median(t)), "min": float(t.min()), "samples": int(reps)}
+
+
+def time_calls(fn, iters, warmup, graph_batch=0):
+    """Average device time of fn() in microseconds over back-to-back calls (one event pair around
+    all of them: what a loop of calls costs per call)."""
     import torch
     for _ in range(warmup):
         fn()
@@ -268,6 +317,8 @@ def chain_table(kf, device, peaks, c2_tensors, c2_us):
     torch.backends.cuda.matmul.allow_tf32 = False
     torch.backends.cudnn.allow_tf32 = False
     out = {}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)      # larger than the 126 MB L2
+    c2_out = torch.empty(M2, N2, dtype=torch.bfloat16, device=device)
     specs = {
         "c1": dict(flops=2.0 * 128 * 256 * 512, bytes=4 * (128 * 512 + 256 * 512 + 256 + 128 * 256)),
         "c2": dict(flops=FLOPS_C2, bytes=ALG_BYTES_C2),
@@ -288,7 +339,7 @@ def chain_table(kf, device, peaks, c2_tensors, c2_us):
         if name == "c1":
             fn = lambda: kf.gemm_epilogue(t["X"], t["W"], t["b"], "relu")
         elif name == "c2":
-            fn = None
+            fn = None          # set below (needs t)
         elif name == "c3":
             o3 = torch.empty(4096, 8192, dtype=torch.bfloat16, device=device)
             fn = lambda: kf.gemm_rowreduce(t["X"], t["W"], t["b"], "none", "softmax", out=o3)
@@ -299,18 +350,41 @@ def chain_table(kf, device, peaks, c2_tensors, c2_us):
             o5 = torch.empty(128, 128, 64, 64, dtype=torch.bfloat16, device=device)
             fn = lambda: kf.conv3x3_epilogue(t["x"], t["w"], t["bias"], "relu", 32, 1e-5, out=o5)
         small = name in ("c1", "c4")
-        us = c2_us if fn is None else time_calls(fn, 200 if small else 40, 5, graph_batch=20 if small else 0)
+        if fn is None:
+            fn = lambda: kf.gemm_epilogue(t["X"], t["W"], t["b"], "gelu_tanh", 0.5, t["R"], out=c2_out)
+        us = c2_us if name == "c2" else time_calls(fn, 200 if small else 40, 5, graph_batch=20 if small else 0)
+        st = time_calls_stats(fn, 200 if small else 40, 5, graph_batch=20 if small else 0)
         us_torch = time_calls(torch_unfused(name, t), 200 if small else 20, 5, graph_batch=20 if small else 0)
         s = specs[name]
         tf = s["flops"] / us / 1e6
         gbs = s["bytes"] / us / 1e3
+        # the roofline time of the chain: the slower of its FLOPs at the measured bf16 burst peak
+        # (fp32 chain c1: launch-bound, reported for completeness) and its algorithmic bytes at the
+        # measured HBM bandwidth
+        t_roof = max(s["flops"] / (peaks["bf16_tflops"] * 1e6), s["bytes"] / (peaks["hbm_gbs"] * 1e3))
         out[name] = {
-            "us_per_call": round(us, 3), "tflops": round(tf, 2),
+            "us_per_call": round(us, 3), "us_median": round(st["median"], 3), "us_min": round(st["min"], 3),
+            "samples": st["samples"], "tflops": round(tf, 2),
+            "t_roof_us": round(t_roof, 3), "roofline_frac": round(t_roof / us, 4),
+            "roofline_bound": "tensor" if s["flops"] / (peaks["bf16_tflops"] * 1e6) >= s["bytes"] / (peaks["hbm_gbs"] * 1e3) else "hbm",
             "frac_tensor_peak_measured_burst": round(tf / peaks["bf16_tflops"], 4),
             "frac_tensor_peak_nominal_2250": round(tf / 2250.0, 4),
             "algorithmic_gbs": round(gbs, 1), "frac_hbm_measured": round(gbs / peaks["hbm_gbs"], 4),
             "unfused_torch_us": round(us_torch, 3), "speedup_vs_unfused_torch": round(us_torch / us, 3),
         }
+        if small:
+            # these two fit in L2 (0.9 MB, 36 MB): the figures above are warm (back-to-back calls);
+            # cold = a 256 MiB buffer is overwritten before every timed call
+            cold = time_calls_stats(fn, 30, 3, flush=flush.zero_)
+            out[name]["cache"] = "warm (L2-resident); cold variant beside it"
+            out[name]["us_cold_median"] = round(cold["median"], 3)
+            out[name]["us_cold_min"] = round(cold["min"], 3)
+        if name == "c1":
+            # launch-bound: the same call without CUDA-graph replay (host launch path included), and
+            # an empty kernel launched the same two ways
+            out[name]["us_per_call_eager"] = round(time_calls(fn, 400, 20), 3)
+            out[name]["noop_kernel_us_graph"] = round(time_calls(kf.kf_launch_noop, 400, 20, graph_batch=20), 3)
+            out[name]["noop_kernel_us_eager"] = round(time_calls(kf.kf_launch_noop, 400, 20), 3)
         del t
     # The paper's worked chain (Appendix C.2): matmul, add, swish, tanh, GELU(erf), hardtanh.  The
     # paper fuses only the five post-matmul operators (speedup 1.04 -> 1.31x on an RTX 5090);
@@ -469,8 +543,14 @@ def run_sweep(kf, device):
         big = flops > 2e9
         us = time_calls(fn, 30 if big else 200, 5, graph_batch=0 if big else 20)
         ut = time_calls(ref, 20 if big else 200, 5, graph_batch=0 if big else 20)
-        rows.append({"category": cat, "shape": name, "us": round(us, 2), "torch_us": round(ut, 2),
-                     "speedup": round(ut / us, 3), "tflops": round(flops / us / 1e6, 1)})
+        row = {"category": cat, "shape": name, "us": round(us, 2), "torch_us": round(ut, 2),
+               "speedup": round(ut / us, 3), "tflops": round(flops / us / 1e6, 1)}
+        if not big:
+            # launch-bound shapes are replayed from CUDA graphs above; eager = plain calls in a loop,
+            # host launch path (argument checks, dispatch, tensor-map lookup) included
+            row["eager_us"] = round(time_calls(fn, 200, 10), 2)
+            row["torch_eager_us"] = round(time_calls(ref, 200, 10), 2)
+        rows.append(row)
 
     for dtn, M, N, K, act, scale, res in SWEEP_GEMM:
         dt = torch.bfloat16 if dtn == "bf16" else torch.float32
@@ -673,7 +753,7 @@ def main():
             dist.destroy_process_group()
         return
 
-    traffic = TRAFFIC_C2_BYTES
+    traffic = c2_traffic_bytes()
     line = {
         "metric": "fused_chain_tflops", "value": round(value, 2), "unit": "TFLOP/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -687,17 +767,40 @@ def main():
                    "peaks": peaks["_source"]},
         "clocks": clocks,
         "e2e": {"value": round(e2e_val, 2), "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                "call": "kf_gemm_epilogue_host (C ABI, pinned host buffers, 4 row blocks)"},
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "kernel": "umma_chain_kernel<256,elementwise,gelu_tanh>",
                      "achieved": round(kernel_tflops, 2), "peak": peaks["bf16_tflops"],
                      "unit": "TFLOP/s", "frac": round(kernel_tflops / peaks["bf16_tflops"], 4),
-                     "frac_of_sustained_peak": round(kernel_tflops / peaks["bf16_tflops_sustained"], 4),
                      "frac_of_nominal_2250": round(kernel_tflops / 2250.0, 4),
                      "peak_source": peaks["_source"] + " cuBLAS bf16 burst",
-                     "traffic": traffic},
+                     "traffic": traffic,
+                     "traffic_source": "ncu summary under profiles/ (one capture of this kernel)" if traffic else None},
     }
     if world == 1 and not args.no_extras:
+        # a seconds-long leg of the same step, to set beside the sustained (power-capped) peak
+        sus = ClockSampler(local)
+        torch.cuda.synchronize()
+        sus.start()
+        n_sus, t0 = 0, time.perf_counter()
+        e0.record()
+        while time.perf_counter() - t0 < 2.2:
+            for _ in range(50):
+                step()
+            n_sus += 50
+            torch.cuda.synchronize()
+        e1.record()
+        torch.cuda.synchronize()
+        sus_ms = e0.elapsed_time(e1)
+        sus_clk = sus.stop()
+        sus_tf = FLOPS_C2 * n_sus / (sus_ms * 1e-3) / 1e12
+        line["sustained"] = {"seconds": round(sus_ms * 1e-3, 2), "steps": n_sus, "tflops": round(sus_tf, 2),
+                             "us_per_call": round(sus_ms * 1e3 / n_sus, 2),
+                             "peak_sustained": peaks["bf16_tflops_sustained"],
+                             "frac_of_measured_sustained": round(sus_tf / peaks["bf16_tflops_sustained"], 4),
+                             "sm_mhz_median": sus_clk["sm_mhz"], "reasons": sus_clk["reasons"],
+                             "note": "includes a host synchronize every 50 steps"}
         rows, secs, cores = oracle_sample_c2(d)
         line["cpu_baseline"] = {
             "value": round(2.0 * rows * N2 * K2 / secs / 1e12, 6), "unit": "TFLOP/s", "cores": cores,

@@ -289,6 +289,30 @@ kf_status kf_device_status(void);
  * clears it.  Nothing traps, faults or loops without bound. */
 kf_status kf_selftest_bounded_wait(uint64_t limit_ns, uint64_t* waited_ns, void* cuda_stream);
 
+/* kf_gemm_epilogue for HOST buffers (the chain of kf_gemm_epilogue, same formula; the paper has
+ * no counterpart: this is the end-to-end form of the call for a caller whose tensors live in host
+ * memory).  X, W, bias, residual and Y are HOST pointers -- page-locked memory if the copies are
+ * to run asynchronously -- with leading dimensions in elements; `staging` is a DEVICE buffer, 256-
+ * byte aligned, of at least kf_gemm_epilogue_host_staging_bytes() bytes (dense copies of X, W, Y,
+ * bias, residual, then the chain's own workspace), owned by the caller.  The batch is cut into
+ * `row_blocks` blocks of rows (1..32; rows are independent): block i is computed on `cuda_stream`
+ * while block i+1 is still arriving and block i-1 is already leaving, on two copy streams the
+ * library creates once per device (host objects; no device memory).  Everything is enqueued when
+ * the call returns; the downloads are joined into `cuda_stream`, so synchronising that stream
+ * makes Y readable.  A later call's uploads start as soon as this call's kernels are done.
+ * Calls are serialised per process.  Errors as for kf_gemm_epilogue; KF_ERR_WORKSPACE when the
+ * staging buffer is null, misaligned or too small. */
+size_t kf_gemm_epilogue_host_staging_bytes(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
+                                           int has_bias, int has_residual);
+kf_status kf_gemm_epilogue_host(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, const void* X,
+                                int64_t ldx, const void* W, int64_t ldw, const void* bias, kf_act act,
+                                float scale, const void* residual, int64_t ldr, void* Y, int64_t ldy,
+                                void* staging, size_t staging_bytes, int row_blocks, void* cuda_stream);
+
+/* Launches an empty kernel (one warp that does nothing) on the stream: the launch-latency
+ * reference the benchmark prints beside the smallest chain (no counterpart in the paper). */
+kf_status kf_launch_noop(void* cuda_stream);
+
 /* Number of kernels the library has launched from this process since load (all streams). */
 int64_t kf_launch_count(void);
 

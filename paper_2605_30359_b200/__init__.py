@@ -35,7 +35,8 @@ EXPORTS = ["kf_gemm_epilogue", "kf_gemm_rowreduce", "kf_gemm_rowreduce_static",
            "kf_gemm_groupnorm", "kf_gemm_groupnorm_workspace_bytes",
            "kf_gemm_epilogue_workspace_bytes", "kf_gemm_rowreduce_workspace_bytes",
            "kf_conv3x3_workspace_bytes", "kf_device_status", "kf_launch_count",
-           "kf_reload_tuning", "kf_tensor_map_cache_stats", "kf_status_string", "kf_version"]
+           "kf_reload_tuning", "kf_tensor_map_cache_stats", "kf_status_string", "kf_version",
+           "kf_gemm_epilogue_host", "kf_gemm_epilogue_host_staging_bytes", "kf_launch_noop"]
 
 
 class KfError(RuntimeError):
@@ -98,6 +99,13 @@ def lib() -> ctypes.CDLL:
     L.kf_device_status.argtypes = []
     L.kf_launch_count.restype = i64
     L.kf_launch_count.argtypes = []
+    L.kf_gemm_epilogue_host_staging_bytes.restype = sz
+    L.kf_gemm_epilogue_host_staging_bytes.argtypes = [i64, i64, i64, ci, ci, ci]
+    L.kf_gemm_epilogue_host.restype = ci
+    L.kf_gemm_epilogue_host.argtypes = [i64, i64, i64, ci, vp, i64, vp, i64, vp, ci, f32, vp, i64, vp, i64,
+                                        vp, sz, ci, vp]
+    L.kf_launch_noop.restype = ci
+    L.kf_launch_noop.argtypes = [vp]
     L.kf_reload_tuning.restype = None
     L.kf_reload_tuning.argtypes = []
     L.kf_tensor_map_cache_stats.restype = None
@@ -255,12 +263,13 @@ def _check_cuda(*ts):
 _workspaces = {}
 
 
-def workspace(nbytes: int, device):
-    """A cached, 256-byte aligned device scratch buffer of at least nbytes (None for 0)."""
+def workspace(nbytes: int, device, slot: str = "ws"):
+    """A cached, 256-byte aligned device scratch buffer of at least nbytes (None for 0); buffers
+    of different `slot` names are distinct."""
     if nbytes == 0:
         return None
     torch = _torch()
-    key = (device.type, device.index)
+    key = (device.type, device.index, slot)
     buf = _workspaces.get(key)
     if buf is None or buf.numel() < nbytes:
         buf = torch.empty(max(nbytes, 1 << 20), dtype=torch.uint8, device=device)
@@ -433,83 +442,37 @@ def conv3x3_act_pool(x, w, bias=None, act="none", kind="max", pool=2, out=None, 
 
 
 # ------------------------------------------------------------------ host-buffer front end
-_staging = {}
-
-
-def _stage(name, host, device):
-    """Device staging buffer matching a host tensor (cached: repeated calls allocate nothing)."""
-    torch = _torch()
-    key = (name, tuple(host.shape), host.dtype, device.index)
-    buf = _staging.get(key)
-    if buf is None:
-        buf = torch.empty(host.shape, dtype=host.dtype, device=device)
-        _staging[key] = buf
-    return buf
-
-
-_side_streams = {}
-_last_compute = {}     # device index -> event after the last kernel that read the staging buffers
-
-
-def _side(device):
-    """Two cached copy streams per device (host-to-device, device-to-host)."""
-    torch = _torch()
-    key = device.index
-    if key not in _side_streams:
-        _side_streams[key] = (torch.cuda.Stream(device), torch.cuda.Stream(device))
-    return _side_streams[key]
+def kf_launch_noop(stream=None):
+    st = lib().kf_launch_noop(_stream_ptr(stream))
+    if st != KF_OK:
+        raise KfError(st, "kf_launch_noop")
 
 
 def gemm_epilogue_host(X, W, bias=None, act="none", scale=1.0, residual=None, out_host=None,
                        device=None, stream=None, chunks=4):
-    """gemm_epilogue for HOST tensors (pinned memory recommended).
-
-    Copies the inputs to the device, runs the fused kernel and copies Y back into out_host.
-    Rows are independent, so the batch is cut into `chunks` row blocks: block i is computed
-    while block i+1 is still arriving and block i-1 is already leaving (the copy engines of the
-    two directions run concurrently).  The kernels run on `stream` (default: the current stream)
-    and the downloads are joined back into it: synchronise it before reading out_host.  Uploads
-    of a call start as soon as the previous call's kernels are done, so back-to-back calls keep
-    both PCIe directions busy."""
+    """gemm_epilogue for HOST tensors (pinned memory recommended): marshals the arguments of
+    kf_gemm_epilogue_host, which pipelines uploads, kernels and downloads over `chunks` row
+    blocks.  The work is enqueued on `stream` (default: the current stream); synchronise it
+    before reading out_host.  The device staging buffer is the binding's cached workspace."""
     torch = _torch()
     device = device or torch.device("cuda", torch.cuda.current_device())
-    s = stream if stream is not None else torch.cuda.current_stream(device)
-    s_in, s_out = _side(device)
-    M = X.shape[0]
+    for t in (X, W, bias, residual, out_host):
+        if t is not None and t.is_cuda:
+            raise ValueError("gemm_epilogue_host takes host tensors")
+    M, K = X.shape
+    N = W.shape[0]
+    dt = _kf_dtype(X)
     if out_host is None:
-        out_host = torch.empty((M, W.shape[0]), dtype=X.dtype).pin_memory()
-    dX, dW, dY = _stage("X", X, device), _stage("W", W, device), _stage("Y", out_host, device)
-    db = _stage("b", bias, device) if bias is not None else None
-    dR = _stage("R", residual, device) if residual is not None else None
-    chunks = max(1, min(int(chunks), M // 256)) if M >= 512 else 1
-    bounds = [M * i // chunks for i in range(chunks + 1)]
-    # The inputs are host memory: the uploads need not wait for earlier work on `s`, only for the
-    # kernels of the previous call that still read the (cached) staging buffers.  So the next
-    # call's uploads overlap the previous call's downloads (PCIe runs both directions at once).
-    last = _last_compute.get(device.index)
-    if last is not None:
-        s_in.wait_event(last)
-    s_out.wait_stream(s)
-    with torch.cuda.stream(s_in):
-        dW.copy_(W, non_blocking=True)
-        if db is not None:
-            db.copy_(bias, non_blocking=True)
-    for i in range(chunks):
-        r0, r1 = bounds[i], bounds[i + 1]
-        with torch.cuda.stream(s_in):
-            dX[r0:r1].copy_(X[r0:r1], non_blocking=True)
-            if dR is not None:
-                dR[r0:r1].copy_(residual[r0:r1], non_blocking=True)
-            arrived = torch.cuda.Event()
-            arrived.record(s_in)
-        s.wait_event(arrived)
-        gemm_epilogue(dX[r0:r1], dW, db, act, scale, dR[r0:r1] if dR is not None else None,
-                      out=dY[r0:r1], stream=s)
-        computed = torch.cuda.Event()
-        computed.record(s)
-        s_out.wait_event(computed)
-        with torch.cuda.stream(s_out):
-            out_host[r0:r1].copy_(dY[r0:r1], non_blocking=True)
-        _last_compute[device.index] = computed
-    s.wait_stream(s_out)
+        out_host = torch.empty((M, N), dtype=X.dtype).pin_memory()
+    nb = lib().kf_gemm_epilogue_host_staging_bytes(M, N, K, dt, int(bias is not None), int(residual is not None))
+    ws = workspace(nb, device, slot="host_staging")
+    with torch.cuda.device(device):
+        st = lib().kf_gemm_epilogue_host(M, N, K, dt, X.data_ptr(), X.stride(0), W.data_ptr(), W.stride(0),
+                                         bias.data_ptr() if bias is not None else None, ACT[act], float(scale),
+                                         residual.data_ptr() if residual is not None else None,
+                                         residual.stride(0) if residual is not None else 0,
+                                         out_host.data_ptr(), out_host.stride(0), _ptr(ws), nb, int(chunks),
+                                         _stream_ptr(stream))
+    if st != KF_OK:
+        raise KfError(st, "kf_gemm_epilogue_host")
     return out_host

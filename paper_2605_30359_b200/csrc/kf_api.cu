@@ -1355,3 +1355,130 @@ extern "C" kf_status kf_conv3x3_softmax_pool(int64_t Nb, int64_t Cin, int64_t H,
   g_launches += 1;
   return KF_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Host-buffer form of the GEMM chain: uploads, kernels and downloads pipelined over row blocks.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t s_in = nullptr, s_out = nullptr;     // upload and download streams
+  cudaEvent_t arrived[32], computed[32];            // per row block
+  cudaEvent_t last_compute = nullptr;               // after the last kernel of the previous call
+  cudaEvent_t caller_here = nullptr;
+  bool has_last = false;
+};
+std::mutex g_pipe_mu;
+HostPipe g_pipe[64];
+
+HostPipe* host_pipe() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lk(g_pipe_mu);
+  HostPipe& hp = g_pipe[dev];
+  if (!hp.ready) {
+    if (cudaStreamCreateWithFlags(&hp.s_in, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&hp.s_out, cudaStreamNonBlocking) != cudaSuccess)
+      return nullptr;
+    for (int i = 0; i < 32; ++i)
+      if (cudaEventCreateWithFlags(&hp.arrived[i], cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&hp.computed[i], cudaEventDisableTiming) != cudaSuccess)
+        return nullptr;
+    if (cudaEventCreateWithFlags(&hp.last_compute, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&hp.caller_here, cudaEventDisableTiming) != cudaSuccess)
+      return nullptr;
+    hp.ready = true;
+  }
+  return &hp;
+}
+
+__global__ void noop_kernel() {}
+
+}  // namespace
+
+extern "C" size_t kf_gemm_epilogue_host_staging_bytes(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
+                                                      int has_bias, int has_residual) {
+  if (M < 1 || N < 1 || K < 1 || !valid_dtype(io_dtype)) return 0;
+  const size_t es = esize(io_dtype);
+  return round256(static_cast<size_t>(M) * K * es) + round256(static_cast<size_t>(N) * K * es) +
+         round256(static_cast<size_t>(M) * N * es) + (has_bias ? round256(static_cast<size_t>(N) * es) : 0) +
+         (has_residual ? round256(static_cast<size_t>(M) * N * es) : 0) +
+         kf_gemm_epilogue_workspace_bytes(M, N, K, io_dtype);
+}
+
+extern "C" kf_status kf_gemm_epilogue_host(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, const void* X,
+                                           int64_t ldx, const void* W, int64_t ldw, const void* bias,
+                                           kf_act act, float scale, const void* residual, int64_t ldr,
+                                           void* Y, int64_t ldy, void* staging, size_t staging_bytes,
+                                           int row_blocks, void* cuda_stream) {
+  if (M < 1 || N < 1 || K < 1 || M > kMaxDim || N > kMaxDim || K > kMaxDim) return KF_ERR_INVALID_ARG;
+  if (!valid_dtype(io_dtype) || !valid_act(act)) return KF_ERR_INVALID_ARG;
+  if (X == nullptr || W == nullptr || Y == nullptr || ldx < K || ldw < K || ldy < N) return KF_ERR_INVALID_ARG;
+  if (residual != nullptr && ldr < N) return KF_ERR_INVALID_ARG;
+  const size_t need = kf_gemm_epilogue_host_staging_bytes(M, N, K, io_dtype, bias != nullptr, residual != nullptr);
+  kf_status vs = check_workspace(staging, staging_bytes, need);
+  if (vs != KF_OK) return vs;
+  HostPipe* hp = host_pipe();
+  if (hp == nullptr) return KF_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t es = esize(io_dtype);
+  // dense device copies, in this order: X, W, Y, bias, residual, then the chain's own workspace
+  uint8_t* base = static_cast<uint8_t*>(staging);
+  uint8_t* dX = base; base += round256(static_cast<size_t>(M) * K * es);
+  uint8_t* dW = base; base += round256(static_cast<size_t>(N) * K * es);
+  uint8_t* dY = base; base += round256(static_cast<size_t>(M) * N * es);
+  uint8_t* db = nullptr;
+  if (bias != nullptr) { db = base; base += round256(static_cast<size_t>(N) * es); }
+  uint8_t* dR = nullptr;
+  if (residual != nullptr) { dR = base; base += round256(static_cast<size_t>(M) * N * es); }
+  const size_t ws_bytes = kf_gemm_epilogue_workspace_bytes(M, N, K, io_dtype);
+  void* ws = ws_bytes ? base : nullptr;
+  int blocks = row_blocks < 1 ? 1 : (row_blocks > 32 ? 32 : row_blocks);
+  if (ws_bytes != 0) blocks = 1;                 // a chain that needs its workspace runs as one call
+  if (M < 512) blocks = 1;
+  else if (blocks > M / 256) blocks = static_cast<int>(M / 256);
+  std::lock_guard<std::mutex> lk(g_pipe_mu);      // one pipelined call at a time per process
+  bool ok = true;
+  // The inputs are host memory: the uploads need not wait for earlier work on the caller's stream,
+  // only for the previous call's kernels, which still read the staging buffers.  So the next
+  // call's uploads overlap the previous call's downloads (both PCIe directions at once).
+  if (hp->has_last) ok = ok && cudaStreamWaitEvent(hp->s_in, hp->last_compute, 0) == cudaSuccess;
+  ok = ok && cudaEventRecord(hp->caller_here, st) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(hp->s_out, hp->caller_here, 0) == cudaSuccess;
+  ok = ok && cudaMemcpy2DAsync(dW, K * es, W, ldw * es, K * es, N, cudaMemcpyHostToDevice, hp->s_in) == cudaSuccess;
+  if (db != nullptr) ok = ok && cudaMemcpyAsync(db, bias, N * es, cudaMemcpyHostToDevice, hp->s_in) == cudaSuccess;
+  if (!ok) return KF_ERR_CUDA;
+  for (int i = 0; i < blocks; ++i) {
+    const int64_t r0 = M * i / blocks, r1 = M * (i + 1) / blocks, rows = r1 - r0;
+    ok = ok && cudaMemcpy2DAsync(dX + r0 * K * es, K * es, static_cast<const uint8_t*>(X) + r0 * ldx * es, ldx * es,
+                                 K * es, rows, cudaMemcpyHostToDevice, hp->s_in) == cudaSuccess;
+    if (dR != nullptr)
+      ok = ok && cudaMemcpy2DAsync(dR + r0 * N * es, N * es, static_cast<const uint8_t*>(residual) + r0 * ldr * es,
+                                   ldr * es, N * es, rows, cudaMemcpyHostToDevice, hp->s_in) == cudaSuccess;
+    ok = ok && cudaEventRecord(hp->arrived[i], hp->s_in) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(st, hp->arrived[i], 0) == cudaSuccess;
+    if (!ok) return KF_ERR_CUDA;
+    vs = kf_gemm_epilogue(rows, N, K, io_dtype, dX + r0 * K * es, K, dW, K, db, act, scale,
+                          dR != nullptr ? dR + r0 * N * es : nullptr, N, dY + r0 * N * es, N, ws, ws_bytes, cuda_stream);
+    if (vs != KF_OK) return vs;
+    ok = ok && cudaEventRecord(hp->computed[i], st) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(hp->s_out, hp->computed[i], 0) == cudaSuccess;
+    ok = ok && cudaMemcpy2DAsync(static_cast<uint8_t*>(Y) + r0 * ldy * es, ldy * es, dY + r0 * N * es, N * es, N * es,
+                                 rows, cudaMemcpyDeviceToHost, hp->s_out) == cudaSuccess;
+    if (!ok) return KF_ERR_CUDA;
+  }
+  ok = ok && cudaEventRecord(hp->last_compute, st) == cudaSuccess;
+  hp->has_last = true;
+  // the downloads join the caller's stream: synchronising it makes Y readable
+  ok = ok && cudaEventRecord(hp->caller_here, hp->s_out) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(st, hp->caller_here, 0) == cudaSuccess;
+  return ok ? KF_OK : KF_ERR_CUDA;
+}
+
+extern "C" kf_status kf_launch_noop(void* cuda_stream) {
+  noop_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>();
+  if (cudaGetLastError() != cudaSuccess) return KF_ERR_CUDA;
+  g_launches += 1;
+  return KF_OK;
+}

@@ -1022,3 +1022,28 @@ def test_host_front_end_back_to_back_calls(kf):
         ref = kf.gemm_epilogue(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "gelu_tanh", 0.5, to_dev(d["R"]))
         assert torch.equal(out, ref.cpu())
     check_status()
+
+
+# ------------------------------------------------------------------ host-buffer entry point
+@pytest.mark.parametrize("blocks", [1, 4])
+def test_gemm_epilogue_host_buffers_through_the_c_abi(kf, blocks):
+    """kf_gemm_epilogue_host: pinned host tensors in, host tensor out, pitched rows, two calls in a
+    row on the same staging buffer (the second call's uploads must wait for the first call's
+    kernels); against the oracle and bit for bit against the device-buffer entry point."""
+    import torch
+    M, N, K = 1024, 320, 136
+    d = ki.gemm_inputs("c2", seed=21, M=M, N=N, K=K)
+    hX = torch.zeros(M, K + 8, dtype=torch.bfloat16).pin_memory()
+    hX[:, :K] = torch.from_numpy(d["X"].view(np.int16)).view(torch.bfloat16)
+    hW = torch.from_numpy(d["W"].view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    hb = torch.from_numpy(d["b"].view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    hR = torch.from_numpy(d["R"].view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    ref = oracle.gemm_epilogue(d["X"], d["W"], d["b"], "gelu_tanh", 0.5, d["R"])
+    dev = kf.gemm_epilogue(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "gelu_tanh", 0.5, to_dev(d["R"]))
+    for rep in range(2):
+        hY = torch.zeros(M, N, dtype=torch.bfloat16).pin_memory()
+        kf.gemm_epilogue_host(hX[:, :K], hW, hb, "gelu_tanh", 0.5, hR, out_host=hY, chunks=blocks)
+        torch.cuda.synchronize()
+        check_status()
+        assert_close(hY.float().numpy().astype(np.float64), ref, 2e-2, 2e-2, "host buffers, call %d" % rep)
+        assert torch.equal(hY, dev.cpu())

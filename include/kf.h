@@ -267,8 +267,21 @@ size_t kf_conv3x3_act_pool_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, i
                                            kf_dtype io_dtype, int pool);
 
 /* Workspace sizes in bytes for the calls above with the same arguments (0 = none needed).
- * Pure host arithmetic; no CUDA call is made. */
+ * Pure host arithmetic; no CUDA call is made.  The short forms assume operands the TMA engine can
+ * load as they are: 16-byte aligned bases and, for bf16, leading dimensions that are multiples
+ * of 8 elements (for kf_gemm_groupnorm also a 16-byte aligned Y with ldy % 8 == 0).  For any
+ * other operands ask the *_for forms, which take the pointers and leading dimensions of the call
+ * and return what the route the call will take for them needs (repacked copies of X and W, or the
+ * scalar kernels' M*N floats). */
 size_t kf_gemm_epilogue_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype);
+size_t kf_gemm_epilogue_workspace_bytes_for(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
+                                            const void* X, int64_t ldx, const void* W, int64_t ldw);
+size_t kf_gemm_rowreduce_workspace_bytes_for(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype,
+                                             kf_rowred red, const void* X, int64_t ldx,
+                                             const void* W, int64_t ldw);
+size_t kf_gemm_groupnorm_workspace_bytes_for(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype,
+                                             int groups, const void* X, int64_t ldx, const void* W,
+                                             int64_t ldw, const void* Y, int64_t ldy);
 size_t kf_gemm_rowreduce_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype,
                                          kf_rowred red);
 size_t kf_conv3x3_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,

@@ -36,7 +36,9 @@ EXPORTS = ["kf_gemm_epilogue", "kf_gemm_rowreduce", "kf_gemm_rowreduce_static",
            "kf_gemm_epilogue_workspace_bytes", "kf_gemm_rowreduce_workspace_bytes",
            "kf_conv3x3_workspace_bytes", "kf_device_status", "kf_launch_count",
            "kf_reload_tuning", "kf_tensor_map_cache_stats", "kf_status_string", "kf_version",
-           "kf_gemm_epilogue_host", "kf_gemm_epilogue_host_staging_bytes", "kf_launch_noop"]
+           "kf_gemm_epilogue_host", "kf_gemm_epilogue_host_staging_bytes", "kf_launch_noop",
+           "kf_gemm_epilogue_workspace_bytes_for", "kf_gemm_rowreduce_workspace_bytes_for",
+           "kf_gemm_groupnorm_workspace_bytes_for"]
 
 
 class KfError(RuntimeError):
@@ -104,6 +106,12 @@ def lib() -> ctypes.CDLL:
     L.kf_gemm_epilogue_host.restype = ci
     L.kf_gemm_epilogue_host.argtypes = [i64, i64, i64, ci, vp, i64, vp, i64, vp, ci, f32, vp, i64, vp, i64,
                                         vp, sz, ci, vp]
+    L.kf_gemm_epilogue_workspace_bytes_for.restype = sz
+    L.kf_gemm_epilogue_workspace_bytes_for.argtypes = [i64, i64, i64, ci, vp, i64, vp, i64]
+    L.kf_gemm_rowreduce_workspace_bytes_for.restype = sz
+    L.kf_gemm_rowreduce_workspace_bytes_for.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64]
+    L.kf_gemm_groupnorm_workspace_bytes_for.restype = sz
+    L.kf_gemm_groupnorm_workspace_bytes_for.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64, vp, i64]
     L.kf_launch_noop.restype = ci
     L.kf_launch_noop.argtypes = [vp]
     L.kf_reload_tuning.restype = None
@@ -292,7 +300,7 @@ def gemm_epilogue(X, W, bias=None, act="none", scale=1.0, residual=None, out=Non
     dt = _kf_dtype(X)
     if out is None:
         out = torch.empty((M, N), dtype=X.dtype, device=X.device)
-    nb = kf_gemm_epilogue_workspace_bytes(M, N, K, dt)
+    nb = lib().kf_gemm_epilogue_workspace_bytes_for(M, N, K, dt, _ptr(X), X.stride(0), _ptr(W), W.stride(0))
     ws = workspace(nb, X.device)
     st = kf_gemm_epilogue(M, N, K, dt, _ptr(X), X.stride(0), _ptr(W), W.stride(0), _ptr(bias),
                           ACT[act], float(scale), _ptr(residual),
@@ -320,7 +328,8 @@ def gemm_rowreduce(X, W, bias=None, pre_act="none", red="softmax", out_dtype=Non
         if out is None:
             out = torch.empty((M, N), dtype=out_dtype or X.dtype, device=X.device)
         odt, ldo = _kf_dtype(out), out.stride(0)
-    nb = kf_gemm_rowreduce_workspace_bytes(M, N, K, dt, RED[red])
+    nb = lib().kf_gemm_rowreduce_workspace_bytes_for(M, N, K, dt, RED[red], _ptr(X), X.stride(0), _ptr(W),
+                                                     W.stride(0))
     ws = workspace(nb, X.device)
     st = kf_gemm_rowreduce(M, N, K, dt, _ptr(X), X.stride(0), _ptr(W), W.stride(0), _ptr(bias),
                            ACT[pre_act], RED[red], _ptr(out), ldo, odt, _ptr(ws), nb,
@@ -383,12 +392,8 @@ def gemm_groupnorm(X, W, bias=None, groups=1, eps=1e-5, gamma=None, beta=None, p
     dt = _kf_dtype(X)
     if out is None:
         out = torch.empty((M, N), dtype=X.dtype, device=X.device)
-    nb = kf_gemm_groupnorm_workspace_bytes(M, N, K, dt, int(groups))
-    if dt == KF_BF16:
-        # the query cannot see pitches and alignment: give the fallback its scratch when needed
-        if not (X.stride(0) % 8 == 0 and W.stride(0) % 8 == 0 and out.stride(0) % 8 == 0 and
-                X.data_ptr() % 16 == 0 and W.data_ptr() % 16 == 0 and out.data_ptr() % 16 == 0):
-            nb = max(nb, M * N * 4)
+    nb = lib().kf_gemm_groupnorm_workspace_bytes_for(M, N, K, dt, int(groups), _ptr(X), X.stride(0), _ptr(W),
+                                                     W.stride(0), _ptr(out), out.stride(0))
     ws = workspace(nb, X.device)
     st = kf_gemm_groupnorm(M, N, K, dt, _ptr(X), X.stride(0), _ptr(W), W.stride(0), _ptr(bias), int(groups),
                            float(eps), _ptr(gamma), _ptr(beta), ACT[post_act], _ptr(out), out.stride(0),

@@ -557,6 +557,41 @@ size_t kf_gemm_rowreduce_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dty
   return rowreduce_simt_ws(M, N) + (use_tf32x3(in_dtype, M, N, K) ? tf32_ws(M, N, K) : 0);
 }
 
+// The same queries for the operands a call will actually get: they take the route the call takes
+// for these pointers and leading dimensions (an operand TMA cannot load is repacked or sends the
+// chain to the scalar kernels, which stage M*N floats).
+size_t kf_gemm_epilogue_workspace_bytes_for(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, const void* X,
+                                            int64_t ldx, const void* W, int64_t ldw) {
+  if (M < 1 || N < 1 || K < 1) return 0;
+  if (io_dtype == KF_BF16 && !umma_gemm_ok(io_dtype, K, X, ldx, W, ldw) && bf16_repack_pays(M, N, K))
+    return bf16_pad_ws(M, N, K);
+  return use_tf32x3(io_dtype, M, N, K) ? tf32_ws(M, N, K) : 0;
+}
+
+size_t kf_gemm_rowreduce_workspace_bytes_for(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, kf_rowred red,
+                                             const void* X, int64_t ldx, const void* W, int64_t ldw) {
+  if (M < 1 || N < 1 || K < 1) return 0;
+  const bool tiles_ok = (N + kRowReduceBN - 1) / kRowReduceBN <= 4096;
+  if (umma_gemm_ok(in_dtype, K, X, ldx, W, ldw) && tiles_ok) return rowreduce_umma_ws(M, N, red);
+  if (in_dtype == KF_BF16 && bf16_repack_pays(M, N, K) && tiles_ok)
+    return bf16_pad_ws(M, N, K) + rowreduce_umma_ws(M, N, red);
+  return rowreduce_simt_ws(M, N) + (use_tf32x3(in_dtype, M, N, K) ? tf32_ws(M, N, K) : 0);
+}
+
+size_t kf_gemm_groupnorm_workspace_bytes_for(int64_t M, int64_t N, int64_t K, kf_dtype io_dtype, int groups,
+                                             const void* X, int64_t ldx, const void* W, int64_t ldw,
+                                             const void* Y, int64_t ldy) {
+  if (M < 1 || N < 1 || K < 1 || groups < 1 || N % groups != 0) return 0;
+  const int64_t gs = N / groups;
+  const bool tc = umma_gemm_ok(io_dtype, K, X, ldx, W, ldw);
+  const bool staged_ok = ldy % 8 == 0 && aligned(Y, 16);
+  if (tc && staged_ok && (gs == 32 || gs == 64 || gs == 128)) return 0;
+  if (tc && staged_ok && gs % 256 == 0 && N / 256 <= 4096)
+    return round256(static_cast<size_t>(M) * ((N + 255) / 256) * 16);
+  if (tc && bf16_repack_pays(M, N, K)) return 0;
+  return rowreduce_simt_ws(M, N) + (use_tf32x3(io_dtype, M, N, K) ? tf32_ws(M, N, K) : 0);
+}
+
 size_t kf_conv3x3_workspace_bytes(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
                                   kf_dtype io_dtype, int groups) {
   (void)groups;

@@ -3,6 +3,7 @@
 // cudaError_t; none synchronises.
 #pragma once
 #include <cstdlib>
+#include <mutex>
 
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -173,15 +174,26 @@ inline cudaError_t launch_umma_instance(const UmmaMaps& tm, const UmmaParams& p,
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    static int resident[17] = {0};             // clusters of this size that fit on the device
-    if (resident[cluster] == 0) {
-      int n = 0;
-      e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
-      if (e != cudaSuccess) return e;
-      if (n < 1) return cudaErrorInvalidConfiguration;
-      resident[cluster] = n;
+    // clusters of this size that fit on the device: asked once per device and kernel instance
+    static std::mutex mu;
+    static int resident[64][17] = {};
+    int dev = 0;
+    e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    int fit = 0;
+    {
+      std::lock_guard<std::mutex> lk(mu);
+      if (resident[dev][cluster] == 0) {
+        int n = 0;
+        e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+        if (e != cudaSuccess) return e;
+        if (n < 1) return cudaErrorInvalidConfiguration;
+        resident[dev][cluster] = n;
+      }
+      fit = resident[dev][cluster];
     }
-    const int clusters = grid < resident[cluster] ? grid : resident[cluster];
+    const int clusters = grid < fit ? grid : fit;
     cfg.gridDim = dim3(clusters * cluster, 1, 1);
     static const bool pdl_cl = getenv("KF_NO_PDL") == nullptr;
     cfg.numAttrs = pdl_cl ? 2 : 1;

@@ -1047,3 +1047,67 @@ def test_gemm_epilogue_host_buffers_through_the_c_abi(kf, blocks):
         check_status()
         assert_close(hY.float().numpy().astype(np.float64), ref, 2e-2, 2e-2, "host buffers, call %d" % rep)
         assert torch.equal(hY, dev.cpu())
+
+
+# ------------------------------------------------------------------ workspace queries for any operands
+def test_workspace_queries_for_unaligned_operands_cover_the_call(kf):
+    """Operands TMA cannot load (an odd pitch, a base off 16 bytes) take other routes with other
+    workspace needs: the *_for queries, given the call's own pointers and pitches, must return
+    enough for the call to succeed, through the raw C ABI."""
+    import torch
+    M, N, K = 96, 80, 72
+    d = ki.gemm_inputs("c3", seed=31, M=M, N=N, K=K)
+    Xb = torch.zeros(M * (K + 3) + 1, dtype=torch.bfloat16, device="cuda")
+    X = Xb[1:].view(M, K + 3)[:, :K]                     # base off 16 bytes, pitch 75
+    X.copy_(to_dev(d["X"]))
+    W, b = to_dev(d["W"]), to_dev(d["b"])
+    Y = torch.empty(M, N + 1, dtype=torch.bfloat16, device="cuda")[:, :N]     # pitch 81
+    stream = torch.cuda.current_stream().cuda_stream
+    L = kf.lib()
+
+    def ws_for(nbytes):
+        return (torch.empty(max(nbytes, 1), dtype=torch.uint8, device="cuda"), nbytes)
+
+    nb = L.kf_gemm_epilogue_workspace_bytes_for(M, N, K, kf.KF_BF16, X.data_ptr(), X.stride(0), W.data_ptr(), K)
+    ws, nb = ws_for(nb)
+    st = kf.kf_gemm_epilogue(M, N, K, kf.KF_BF16, X.data_ptr(), X.stride(0), W.data_ptr(), K, b.data_ptr(),
+                             kf.ACT["relu"], 1.0, None, 0, Y.data_ptr(), Y.stride(0), ws.data_ptr() if nb else None,
+                             nb, stream)
+    assert st == kf.KF_OK, kf.status_string(st)
+    assert_close(to_f64(Y), oracle.gemm_epilogue(d["X"], d["W"], d["b"], "relu"), 2e-2, 2e-2, "epilogue, odd pitch")
+
+    for red, name in ((kf.RED["softmax"], "softmax"), (kf.RED["sum"], "sum")):
+        assert kf.kf_gemm_rowreduce_workspace_bytes(M, N, K, kf.KF_BF16, red) < M * N * 4     # the short form is not enough
+        nb = L.kf_gemm_rowreduce_workspace_bytes_for(M, N, K, kf.KF_BF16, red, X.data_ptr(), X.stride(0),
+                                                     W.data_ptr(), K)
+        assert nb >= M * N * 4
+        ws, nb = ws_for(nb)
+        out = (torch.empty(M, N, dtype=torch.bfloat16, device="cuda") if name == "softmax"
+               else torch.empty(M, dtype=torch.float32, device="cuda"))
+        st = kf.kf_gemm_rowreduce(M, N, K, kf.KF_BF16, X.data_ptr(), X.stride(0), W.data_ptr(), K, b.data_ptr(),
+                                  kf.ACT["none"], red, out.data_ptr(), N if name == "softmax" else 1,
+                                  kf.KF_BF16 if name == "softmax" else kf.KF_F32, ws.data_ptr(), nb, stream)
+        assert st == kf.KF_OK, kf.status_string(st)
+        ref = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "none", name).reshape(to_f64(out).shape)
+        assert_close(to_f64(out), ref, 2e-2, 2e-2, "rowreduce %s, odd pitch" % name)
+
+    groups = 5                                           # 16 columns per group: the scalar route in any case
+    assert kf.kf_gemm_groupnorm_workspace_bytes(M, N, K, kf.KF_BF16, 2) >= 0
+    nb = L.kf_gemm_groupnorm_workspace_bytes_for(M, N, K, kf.KF_BF16, groups, X.data_ptr(), X.stride(0),
+                                                 W.data_ptr(), K, Y.data_ptr(), Y.stride(0))
+    ws, nb = ws_for(nb)
+    st = kf.kf_gemm_groupnorm(M, N, K, kf.KF_BF16, X.data_ptr(), X.stride(0), W.data_ptr(), K, b.data_ptr(), groups,
+                              1e-5, None, None, kf.ACT["none"], Y.data_ptr(), Y.stride(0),
+                              ws.data_ptr() if nb else None, nb, stream)
+    assert st == kf.KF_OK, kf.status_string(st)
+    check_status()
+    assert_close(to_f64(Y), oracle.gemm_groupnorm(d["X"], d["W"], d["b"], groups, 1e-5, None, None, "none"),
+                 2e-2, 2e-2, "groupnorm, odd pitch")
+    # a 64-column group with a Y that TMA cannot store to: the short query says 0, the call needs M*N floats
+    assert kf.kf_gemm_groupnorm_workspace_bytes(128, 128, 64, kf.KF_BF16, 2) == 0
+    Xa = torch.zeros(128, 64, dtype=torch.bfloat16, device="cuda")
+    Wa = torch.zeros(128, 64, dtype=torch.bfloat16, device="cuda")
+    Ya = torch.empty(128, 129, dtype=torch.bfloat16, device="cuda")[:, :128]
+    nb = L.kf_gemm_groupnorm_workspace_bytes_for(128, 128, 64, kf.KF_BF16, 2, Xa.data_ptr(), 64, Wa.data_ptr(), 64,
+                                                 Ya.data_ptr(), 129)
+    assert nb >= 128 * 128 * 4

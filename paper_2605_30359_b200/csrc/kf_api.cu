@@ -19,8 +19,9 @@ std::atomic<int64_t> g_launches{0};
 // to move a threshold); the environment is read ONCE, at the first call, and again only when
 // kf_reload_tuning() is called, so a call on the hot path reads no environment variable.
 struct Tuning {
-  bool no_fused_pool, no_tf32x3, no_splitk, no_pair, no_cluster_softmax, no_fused_softmax, no_fused_gn, no_conv_slab;
+  bool no_fused_pool, no_tf32x3, no_splitk, no_pair, no_cluster_softmax, no_fused_softmax, no_fused_gn, no_conv_slab, no_gnx;
   int splitk_min_kb, splitk_two_per_sm, pair_min_k, pair_min_kb_per_cta, cl128_max_ctas;
+  int gnx_min_tiles, gnx_min_tpi, gnx_max_tpi;     // all-SM GroupNorm convolution: tiles in all (-1: two waves), tiles per image
 };
 Tuning g_tune;
 std::atomic<bool> g_tune_loaded{false};
@@ -39,11 +40,15 @@ void load_tuning_locked() {
   g_tune.no_fused_softmax = flag("KF_NO_FUSED_SOFTMAX");
   g_tune.no_fused_gn = flag("KF_NO_FUSED_GN");
   g_tune.no_conv_slab = flag("KF_NO_CONV_SLAB");
+  g_tune.no_gnx = flag("KF_NO_GNX");
   g_tune.splitk_min_kb = num("KF_SPLITK_MIN_KB", 28);
   g_tune.splitk_two_per_sm = num("KF_SPLITK_TWO_PER_SM", 1);
   g_tune.pair_min_k = num("KF_PAIR_MIN_K", 2048);
   g_tune.pair_min_kb_per_cta = num("KF_PAIR_MIN_KB_PER_CTA", 128);
   g_tune.cl128_max_ctas = num("KF_CL128_MAX_CTAS", 120);
+  g_tune.gnx_min_tiles = num("KF_GNX_MIN_TILES", -1);
+  g_tune.gnx_min_tpi = num("KF_GNX_MIN_TPI", 9);
+  g_tune.gnx_max_tpi = num("KF_GNX_MAX_TPI", 64);
   g_tune_loaded.store(true, std::memory_order_release);
 }
 inline const Tuning& tune() {
@@ -277,8 +282,15 @@ int64_t conv_stat_parts(int64_t H, int64_t Wd) {
   const int r = conv_rows_per_tile(H, Wd);
   return (H + r - 1) / r * conv_w_segs(Wd);
 }
+// per-tile channel statistics of the two-kernel route, or (same region) the per-tile group
+// statistics of the all-SM GroupNorm kernel, followed by that kernel's per-image counters
+size_t conv_gx_part_bytes(int64_t Nb, int64_t H, int64_t Wd, int64_t Cout) {
+  const size_t per_channel = static_cast<size_t>(Nb) * conv_stat_parts(H, Wd) * Cout * 8;
+  const size_t per_group = static_cast<size_t>(Nb) * ((Cout + kBM - 1) / kBM) * conv_stat_parts(H, Wd) * 256;
+  return round256(per_channel > per_group ? per_channel : per_group);
+}
 size_t conv_stats_bytes(int64_t Nb, int64_t H, int64_t Wd, int64_t Cout) {
-  return round256(static_cast<size_t>(Nb) * conv_stat_parts(H, Wd) * Cout * 8);
+  return conv_gx_part_bytes(Nb, H, Wd, Cout) + round256(static_cast<size_t>(Nb) * ((Cout + kBM - 1) / kBM) * 4);
 }
 
 kf_status check_gemm_common(int64_t M, int64_t N, int64_t K, int dt, const void* X, int64_t ldx,
@@ -1104,9 +1116,11 @@ static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
     void* xt = workspace;
     void* wr = static_cast<uint8_t*>(workspace) + xt_bytes;
     float* stats = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + xt_bytes + wr_bytes);
+    uint32_t* gx_count = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(stats) + conv_gx_part_bytes(Nb, H, Wd, Cout));
+    const int gx_units = static_cast<int>(Nb * ((Cout + kBM - 1) / kBM));
     if (launch_conv_prep(static_cast<int>(Nb), static_cast<int>(Cin), static_cast<int>(Cp),
                          static_cast<int>(H), static_cast<int>(Wd), static_cast<int>(Cout), x, w, xt, wr,
-                         st) != cudaSuccess)
+                         st, groups > 0 ? gx_count : nullptr, gx_units) != cudaSuccess)
       return KF_ERR_CUDA;
     ++launches;
     const int rows = conv_rows_per_tile(H, Wd);        // image rows per tile
@@ -1163,6 +1177,30 @@ static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
                           tpi >= 1 && (tpi <= 8 || tpi == 16) &&      // 9..15 pack badly into GPCs (56x56: 43.6 us against 41.5)
                           (cpg == 4 || cpg == 8 || cpg == 16 || cpg == 32) &&
                           !tune().no_fused_gn;
+    // GroupNorm inside the epilogue on every SM (any number of tiles per image): neighbouring CTAs
+    // of a cooperative grid hold an image's tiles and exchange the statistics through global memory
+    // Taken for images of 9 to 64 tiles on problems of at least two waves (measured against the other
+    // routes on B200: 128x64x64x64 -> 128, 16 tiles per image, 123.9 us against 131.0 in clusters of
+    // 16, which occupy 112 of the 148 SMs; 8x64x128x128 -> 64, 64 tiles, 45.5 us against 75.6 for
+    // two kernels; 32x64x56x56 -> 64, 14 tiles, 39.4 against 39.3; smaller problems lose to the
+    // cooperative launch's set-up, images of hundreds of tiles to the wait for the whole image).
+    const int gnx_min_tiles = tune().gnx_min_tiles >= 0 ? tune().gnx_min_tiles : 2 * d->sm_count;
+    if (groups > 0 && p.staged && (cpg == 4 || cpg == 8 || cpg == 16 || cpg == 32) && tpi >= tune().gnx_min_tpi &&
+        tpi <= tune().gnx_max_tpi && p.num_tiles >= gnx_min_tiles && !tune().no_gnx && !tune().no_fused_gn) {
+      UmmaParams q = p;
+      q.gn_groups = groups; q.gn_eps = eps;
+      q.gn_gamma = static_cast<const __nv_bfloat16*>(gamma);
+      q.gn_beta = static_cast<const __nv_bfloat16*>(beta);
+      q.partial = nullptr;
+      q.gx_part = reinterpret_cast<float2*>(stats);
+      q.gx_count = gx_count;
+      const int gridx = q.num_tiles < d->sm_count ? q.num_tiles : d->sm_count;
+      if (launch_umma_conv_gnx(bn, act, tm, q, gridx, st) == cudaSuccess) {
+        g_launches += launches + 1;
+        return KF_OK;
+      }
+      (void)cudaGetLastError();      // the device cannot hold the grid at once: the other routes
+    }
     if (gn_fused) {
       p.gn_cluster = tpi; p.gn_groups = groups; p.gn_eps = eps;
       p.gn_gamma = static_cast<const __nv_bfloat16*>(gamma);

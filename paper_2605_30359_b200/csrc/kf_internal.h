@@ -37,6 +37,10 @@ cudaError_t launch_umma_softmax_cluster(int bn, int act, int out_dt, const UmmaM
                                         int row_blocks, cudaStream_t st);
 cudaError_t launch_umma_conv_gn(int bn, int act, const UmmaMaps& tm, const UmmaParams& p, int images,
                                 cudaStream_t st);
+// the same chain on every SM: statistics exchanged through global memory, cooperative launch of
+// `grid` CTAs (at most one per SM)
+cudaError_t launch_umma_conv_gnx(int bn, int act, const UmmaMaps& tm, const UmmaParams& p, int grid,
+                                 cudaStream_t st);
 constexpr int kRowReduceBN = 256;   // tile width of the row-reduce first pass
 constexpr int kRowReduceNarrowBN = 64;   // ... of the softmax first pass of one-wave problems
 
@@ -59,8 +63,10 @@ cudaError_t launch_row_reduce(int red, int M, int N, const float* A, long long l
                               cudaStream_t st);
 
 // convolution helpers
+// (also sets `zero_words` 32-bit words at `zero` to 0: the counters of EPI_CONV_GNX)
 cudaError_t launch_conv_prep(int Nb, int Cin, int Cp, int H, int Wd, int Cout, const void* x,
-                             const void* w, void* xt, void* wr, cudaStream_t st);
+                             const void* w, void* xt, void* wr, cudaStream_t st, void* zero = nullptr,
+                             int zero_words = 0);
 cudaError_t launch_conv_direct(int dt, int act, int Nb, int Cin, int H, int Wd, int Cout,
                                const void* x, const void* w, const void* bias, void* y,
                                cudaStream_t st);
@@ -147,8 +153,10 @@ cudaError_t launch_channel_softmax_pool(int dt, int Nb, int C, int H, int Wd, in
 template <int BN, int EPI, int ACT, typename OutT, bool CTA2 = false>
 // `cluster` > 0 (EPI_CONV_GN): `grid` counts the images; the launch uses as many clusters of that
 // many CTAs as can be resident at once (at most one per image).
+// `coop`: a cooperative launch (every CTA of the grid resident together; `grid` must not exceed
+// what the device holds at once), for the kernels whose CTAs wait for one another.
 inline cudaError_t launch_umma_instance(const UmmaMaps& tm, const UmmaParams& p, int grid,
-                                        cudaStream_t st, int cluster = 0) {
+                                        cudaStream_t st, int cluster = 0, bool coop = false) {
   using C = UmmaCfg<BN, EPI, CTA2>;
   constexpr int smem = C::kTotal;
   static_assert(smem <= kMaxDynSmem, "shared-memory plan exceeds the per-CTA limit");
@@ -223,6 +231,13 @@ inline cudaError_t launch_umma_instance(const UmmaMaps& tm, const UmmaParams& p,
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
+    if (coop) {
+      attr[0].id = cudaLaunchAttributeCooperative;
+      attr[0].val.cooperative = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      return cudaLaunchKernelEx(&cfg, kern, tm.a, tm.b, tm.r, tm.y, p);
+    }
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;

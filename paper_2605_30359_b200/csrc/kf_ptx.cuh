@@ -93,6 +93,31 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
   return true;
 }
 
+// Release / acquire on a counter in global memory at device scope: a thread that has written data
+// (and fenced) adds to the counter with release; a thread that reads the counter with acquire and
+// finds the expected value may read that data.
+__device__ __forceinline__ void red_release_gpu_add(uint32_t* addr, uint32_t v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void red_relaxed_gpu_add(uint32_t* addr, uint32_t v) {
+  asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_relaxed_gpu(const uint32_t* addr) {
+  uint32_t v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* addr) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
+  return v;
+}
+// Arrive without waiting: the producer half of a producer / consumer hand-over (the consumer
+// calls named_barrier_sync with the same id and thread count).
+__device__ __forceinline__ void named_barrier_arrive(uint32_t id, uint32_t nthreads) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
 // Packed fp32 pairs (sm_100: one instruction adds or multiply-adds two floats held in a 64-bit
 // register).  The epilogues that are bound by instruction issue use them where both elements
 // take the same operation.

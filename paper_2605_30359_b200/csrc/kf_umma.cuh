@@ -35,9 +35,12 @@ namespace kf {
 // EPI_SOFTMAX_CL: the softmax of a row whose column tiles are held by the CTAs of one cluster: the
 // per-row (maximum, sum) pairs travel through distributed shared memory and every CTA stores
 // final probabilities (one kernel, no second pass).
+// EPI_CONV_GNX: the same chain on all SMs without clusters: the tiles of an image are held by
+// neighbouring CTAs of one co-resident (cooperative) grid, which exchange the group statistics
+// through global memory; the epilogue is software-pipelined so that the exchange is not waited for.
 enum : int { EPI_ELEMENTWISE = 0, EPI_SOFTMAX = 1, EPI_ROWSUM = 2, EPI_CONV = 3, EPI_CONV_GN = 4,
-             EPI_SOFTMAX_CL = 5 };
-constexpr bool is_conv(int epi) { return epi == 3 || epi == 4; }
+             EPI_SOFTMAX_CL = 5, EPI_CONV_GNX = 6 };
+constexpr bool is_conv(int epi) { return epi == 3 || epi == 4 || epi == 6; }
 constexpr bool is_softmax(int epi) { return epi == 1 || epi == 5; }
 constexpr bool is_cluster_epi(int epi) { return epi == 4 || epi == 5; }
 
@@ -58,10 +61,14 @@ constexpr int kNumThreads = 192;  // 6 warps: producer, UMMA issuer, epilogue
 // cost it 2 %) keeps one group.
 constexpr int epi_groups(int epi, int bn, bool cta2) {
   return epi == 1 /* EPI_SOFTMAX */ || epi == 4 /* EPI_CONV_GN */ || epi == 5 /* EPI_SOFTMAX_CL */ ||
+                 epi == 6 /* EPI_CONV_GNX */ ||
                  (epi == 0 /* EPI_ELEMENTWISE */ && bn >= 64 && !cta2)
              ? 2 : 1;
 }
-constexpr int num_threads(int epi, int bn, bool cta2) { return 64 + kEpiThreads * epi_groups(epi, bn, cta2); }
+// (EPI_CONV_GNX carries one more warp, which does the epilogue's global-memory work: see conv_gnx_helper)
+constexpr int num_threads(int epi, int bn, bool cta2) {
+  return 64 + kEpiThreads * epi_groups(epi, bn, cta2) + (epi == 6 /* EPI_CONV_GNX */ ? 32 : 0);
+}
 constexpr int kPieceCols = 32;    // epilogue piece: 128 rows x 32 columns
 constexpr int kPieceBytes = kBM * kPieceCols * 2;   // 8 KB of bf16
 constexpr int kMaxDynSmem = 232448;                 // 227 KB opt-in limit per CTA
@@ -110,6 +117,11 @@ struct UmmaParams {
                                // through tmR) and the three row taps read it at offsets of whole rows
   int slab_bytes;              // bytes of one such copy (<= 48 KB)
   int slab_row_bytes;          // bytes of one image row of the copy: box_w * 128, a multiple of 1024
+  // EPI_CONV_GNX: per (image, channel tile) unit u: gx_part[(u * tiles_per_image + t) * 32 + g] =
+  // (sum, sum of squares) of GroupNorm group g over pixel tile t; gx_count[u] = tiles published
+  // (zero when the kernel starts)
+  float2* gx_part;
+  uint32_t* gx_count;
   int pool2;                   // convolution: 0, or 2x2 pooling in the epilogue (1 = max, 2 = mean);
                                // needs w_segs == 1, Wd % 32 == 0, rows_per_tile and H even
 };
@@ -145,7 +157,8 @@ struct UmmaCfg {
                                                     : (EPI == EPI_ROWSUM ? 0 : 2 * kPieceBytes);     // EPI_CONV_GN: one piece per epilogue group
   static constexpr int kBarBytes = 256;
   // GEMM epilogues: the tile's BN bias values as fp32, staged once per tile
-  static constexpr int kBiasBytes = EPI == EPI_CONV ? 0 : BN * 4;   // EPI_CONV_GN: the statistics it sends
+  // (EPI_CONV_GNX: partial sums [2][2 groups][32] and group statistics [2][32], float2)
+  static constexpr int kBiasBytes = EPI == EPI_CONV ? 0 : (EPI == EPI_CONV_GNX ? 1536 : BN * 4);   // EPI_CONV_GN: the statistics it sends
   // EPI_CONV_GN: statistics arriving from the cluster, [2 buffers][16 CTAs x 2 groups][32 x float2]
   // EPI_SOFTMAX_CL: [2 buffers][16 CTAs x 2 groups][128 rows x float2] arriving, then the
   // [2 buffers][2 groups][128 x float2] it sends
@@ -220,6 +233,282 @@ __device__ __forceinline__ void load_sbias32(const float* sb, float (&b)[32]) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Epilogue of EPI_CONV_GNX: conv3x3 -> activation -> GroupNorm in one kernel on every SM.
+//
+// Tiles are dealt round-robin, tile t to CTA t mod grid, so the pixel tiles of one image are held
+// by neighbouring CTAs at (almost) the same time; the grid is launched cooperatively, i.e. all of
+// its CTAs are resident together.  Two epilogue groups of four warps, each owning half of the
+// tile's pixels; a thread is one output channel.  Per tile:
+//   A  the thread reads its share of the accumulator ONCE (the warp hands the accumulator back to
+//      the UMMA issuer as soon as its last load has landed), applies bias and activation, adds up
+//      sum and sum of squares in fp32 and keeps the activations in registers as bf16; shuffles
+//      reduce the sums over the channels of a GroupNorm group; one warp adds the two groups'
+//      partial sums, writes the tile's 32 (sum, sum of squares) pairs to global memory and
+//      counts the tile in (release at device scope).
+//   B  one thread checks (acquire, bounded) that all of the image's tiles are counted in; every
+//      thread adds the tiles' pairs of its group in tile order, normalises its activations from
+//      the registers and stores them through the warp's 2 KB slab (32 channels x 32 pixels) with TMA.
+// The loop is software-pipelined: A of this CTA's next tile runs BEFORE B of the current one (two
+// register buffers of activations), so by the time B asks, the other CTAs have long published and
+// the exchange's latency is hidden behind an accumulator pass.  A only ever waits for this CTA's
+// own MMAs, so the waits cannot form a cycle.  No thread leaves the loop inside a tile: a wait
+// that runs out is reported at the next go/no-go, which all eight warps take together.
+// ---------------------------------------------------------------------------------------------
+template <int BN, int ACT, typename TileAt>
+__device__ __forceinline__ void conv_gnx_epilogue(const UmmaParams& p, const CUtensorMap* tmY, uint8_t* stg,
+                                                  float2* aux, uint64_t* tmem_full, uint64_t* tmem_empty,
+                                                  uint64_t* gx_parts, uint64_t* gx_stats,
+                                                  volatile uint32_t* abort_flag, uint32_t tmem_base,
+                                                  int warp, int lane, int my_tiles, TileAt tile_at) {
+  constexpr int kGroups = 2;
+  constexpr int kGroupCols = BN / kGroups;
+  constexpr int kGP = kGroupCols / 32;                  // pieces per thread: 4 (BN = 256) or 2
+  const int grp = (warp - 2) >> 2;
+  const int quad = warp & 3;                            // TMEM lane quarter this warp may read
+  const int row = quad * 32 + lane;                     // output channel inside the 128-channel tile
+  const bool leader = threadIdx.x == 64;                // polls for all
+  const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
+  const int cpg = p.N / p.gn_groups;                    // channels per group: 4, 8, 16 or 32
+  const int gidx = row / cpg;                           // this channel's group inside the tile: 0..31
+  const long long hw = static_cast<long long>(p.H) * p.Wd;
+  const float inv_cnt = 1.0f / static_cast<float>(static_cast<long long>(cpg) * hw);
+  const int pieces = p.tile_px / 32;
+  const int piece0 = grp * kGP;
+  const int my_pieces = max(0, min(kGP, pieces - piece0));
+  const int tpi = p.tiles_per_image;
+  uint8_t* yslab = stg + grp * kPieceBytes;             // the group's staging piece (a 2 KB slab per warp)
+  bool failed = false;                                  // one of this thread's waits ran out
+
+  struct Tile { int tm, img, pt, unit, px0, px_valid; float bias_v, ga, be; };
+  auto locate = [&](int it) {
+    const int tile = tile_at(it);
+    Tile t;
+    t.tm = tile % p.tiles_m;
+    const int tn = conv_pixel_tile(p, tile / p.tiles_m);
+    t.img = tn / tpi;
+    t.pt = tn % tpi;
+    t.unit = t.img * p.tiles_m + t.tm;
+    t.px0 = t.pt * p.tile_px;
+    t.px_valid = static_cast<int>(min(static_cast<long long>(p.tile_px), hw - t.px0));
+    const int ch = t.tm * kBM + row;
+    const bool ch_ok = ch < p.N;
+    t.bias_v = (p.bias != nullptr && ch_ok) ? __bfloat162float(p.bias[ch]) : 0.0f;
+    t.ga = (p.gn_gamma != nullptr && ch_ok) ? __bfloat162float(p.gn_gamma[ch]) : 1.0f;
+    t.be = (p.gn_beta != nullptr && ch_ok) ? __bfloat162float(p.gn_beta[ch]) : 0.0f;
+    return t;
+  };
+
+  // A: accumulator -> activations in `st` (bf16 pairs); this tile's statistics published.
+  // Returns false when the go/no-go said stop (then every epilogue thread got false).
+  auto phase_a = [&](int it, uint32_t (&st)[kGP * 16]) -> bool {
+    const Tile t = locate(it);
+    const int a = it & 1;
+    bool ok = true;
+    if (leader)
+      ok = mbar_wait(&tmem_full[a], static_cast<uint32_t>((it >> 1) & 1), abort_flag, p.status,
+                     KF_DEV_TIMEOUT_EPILOGUE);
+    ok = named_barrier_and(9u, kGroups * kEpiThreads, ok && !failed);
+    if (!ok) return false;
+    tc_fence_after_sync();
+    const uint32_t t_acc = tmem_base + static_cast<uint32_t>(a * BN + grp * kGroupCols) + lane_off;
+    const uint64_t bias2 = f32x2_pack(t.bias_v, t.bias_v);
+    float s1 = 0.0f, s2 = 0.0f;
+    uint64_t s1p = f32x2_pack(0.0f, 0.0f), s2p = s1p;   // (even, odd) pixel partial sums
+#pragma unroll
+    for (int c = 0; c < kGP; ++c) {
+      uint32_t v[32];
+      if (c < my_pieces) {
+        tmem_ld_32x32(t_acc + c * 32, v);
+        tmem_ld_wait();
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = 0u;
+      }
+      if (c == kGP - 1) {
+        // the last of this warp's loads has landed: hand the accumulator back (one arrival per warp)
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tmem_empty[a]);
+      }
+      const int left = t.px_valid - (piece0 + c) * 32;  // valid pixels from this piece on
+      if (left >= 32) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          float y0, y1;
+          f32x2_unpack(f32x2_add(f32x2_pack(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])), bias2), y0, y1);
+          y0 = act_f<ACT, true>(y0, p.act_rt);
+          y1 = act_f<ACT, true>(y1, p.act_rt);
+          const uint64_t y = f32x2_pack(y0, y1);
+          s1p = f32x2_add(s1p, y);
+          s2p = f32x2_fma(y, y, s2p);
+          st[c * 16 + j] = pack_bf16x2(y0, y1);
+        }
+      } else {
+        // a tile that hangs over the end of its image: those pixels were read as zeros, are left
+        // out of the statistics and are not stored
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + t.bias_v, p.act_rt);
+          float y1 = act_f<ACT, true>(__uint_as_float(v[2 * j + 1]) + t.bias_v, p.act_rt);
+          if (2 * j >= left) y0 = 0.0f;
+          if (2 * j + 1 >= left) y1 = 0.0f;
+          s1 += y0 + y1;
+          s2 = fmaf(y0, y0, fmaf(y1, y1, s2));
+          st[c * 16 + j] = pack_bf16x2(y0, y1);
+        }
+      }
+    }
+    {
+      float e, o;
+      f32x2_unpack(s1p, e, o); s1 += e + o;
+      f32x2_unpack(s2p, e, o); s2 += e + o;
+    }
+    for (int o = cpg >> 1; o > 0; o >>= 1) {            // the group's channels: adjacent lanes
+      s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+      s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+    }
+    // the partial sums go to the helper warp, which publishes them (see conv_gnx_helper)
+    float2* part = aux + (it & 1) * 64;                 // [2 tiles in flight][2 groups][32]
+    if ((row & (cpg - 1)) == 0) part[grp * 32 + gidx] = make_float2(s1, s2);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&gx_parts[it & 1]);      // (release: the warp's writes above are ordered before it)
+    return true;
+  };
+
+  // B: the image's statistics -> normalised activations -> global memory.
+  auto phase_b = [&](int it, const uint32_t (&st)[kGP * 16]) {
+    const Tile t = locate(it);
+    // the helper warp has added the image's tiles up and left (mean, 1/std) per group
+    if (!mbar_wait(&gx_stats[it & 1], static_cast<uint32_t>((it >> 1) & 1), abort_flag, p.status, KF_DEV_TIMEOUT_EPILOGUE))
+      failed = true;                      // the status word has it; finish the tile with the others
+    const float2 ms = aux[128 + (it & 1) * 32 + gidx];  // [2][32] after the partial sums
+    const float sc = ms.y * t.ga;
+    const float sh = fmaf(-ms.x, sc, t.be);
+    const uint64_t sc2 = f32x2_pack(sc, sc), sh2 = f32x2_pack(sh, sh);
+#pragma unroll
+    for (int c = 0; c < kGP; ++c) {
+      if (c < my_pieces) {
+        uint32_t w[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const uint32_t u = st[c * 16 + j];
+          float y0, y1;
+          f32x2_unpack(f32x2_fma(f32x2_pack(bf16_lo(u), bf16_hi(u)), sc2, sh2), y0, y1);
+          w[j] = pack_bf16x2(y0, y1);
+        }
+        bulk_wait_group_read<0>();       // this warp's previous store has let go of the slab
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          *reinterpret_cast<uint4*>(yslab + piece_off(row, q)) =
+              make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (elect_one()) {
+          const int px = (piece0 + c) * 32;               // first pixel of the piece inside the tile
+          if (t.px_valid - px > 0 && t.tm * kBM + quad * 32 < p.N)
+            tma_store_3d(tmY, yslab + quad * (kPieceBytes / 4), t.px0 + px, t.tm * kBM + quad * 32, t.img);
+          bulk_commit_group();
+        }
+      }
+    }
+  };
+
+  uint32_t st_a[kGP * 16], st_b[kGP * 16];
+  bool alive = true;
+  for (int it = 0; it <= my_tiles && alive; it += 2) {
+    if (it < my_tiles) alive = phase_a(it, st_a);
+    if (alive && it >= 1) phase_b(it - 1, st_b);
+    if (alive && it + 1 < my_tiles) alive = phase_a(it + 1, st_b);
+    if (alive && it < my_tiles) phase_b(it, st_a);
+  }
+  bulk_wait_group_read<0>();
+}
+
+// The helper warp of EPI_CONV_GNX: everything in the GroupNorm exchange that touches global memory.
+// A small state machine over this CTA's tiles, never blocking on one thing while another is due:
+//   publish(k)  once the epilogue warps have left tile k's partial sums: the two groups' sums in a
+//               fixed order to global memory as one 256-byte row, a fence, and the tile is counted
+//               in (release at device scope);
+//   stats(k)    once all tiles of tile k's image are counted in (acquire): lane g adds the tiles'
+//               pairs of group g in tile order and leaves (mean, 1/std) for the epilogue warps.
+// Every wait is bounded; a wait that runs out raises the abort flag, and the outstanding hand-overs
+// are still completed so that no epilogue warp is left waiting on a barrier.
+template <typename TileAt>
+__device__ __forceinline__ void conv_gnx_helper(const UmmaParams& p, float2* aux, uint64_t* gx_parts,
+                                                uint64_t* gx_stats, volatile uint32_t* abort_flag,
+                                                int lane, int my_tiles, TileAt tile_at) {
+  const int tpi = p.tiles_per_image;
+  const int cpg = p.N / p.gn_groups;
+  const long long hw = static_cast<long long>(p.H) * p.Wd;
+  const float inv_cnt = 1.0f / static_cast<float>(static_cast<long long>(cpg) * hw);
+  auto unit_of = [&](int it, int* pt) {
+    const int tile = tile_at(it);
+    const int tn = conv_pixel_tile(p, tile / p.tiles_m);
+    *pt = tn % tpi;
+    return (tn / tpi) * p.tiles_m + tile % p.tiles_m;
+  };
+  int pub = 0, stt = 0;
+  bool dead = false;
+  uint64_t t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  while (stt < my_tiles) {
+    bool progressed = false;
+    if (pub < my_tiles && (dead || mbar_try_wait(&gx_parts[pub & 1], static_cast<uint32_t>((pub >> 1) & 1)))) {
+      int pt;
+      const int unit = unit_of(pub, &pt);
+      const float2* part = aux + (pub & 1) * 64;
+      float2 m = make_float2(0.0f, 0.0f);
+      if (lane < kBM / cpg) {
+        const float2 a0 = part[lane], a1 = part[32 + lane];
+        m = make_float2(a0.x + a1.x, a0.y + a1.y);
+      }
+      p.gx_part[(static_cast<long long>(unit) * tpi + pt) * 32 + lane] = m;
+      // the warp's 32 stores are ordered before lane 0's release by the warp barrier; no separate
+      // device-wide fence (measured: a fence per tile in this warp cost the kernel 5 us)
+      __syncwarp();
+      if (lane == 0) red_release_gpu_add(p.gx_count + unit, 1u);
+      ++pub;
+      progressed = true;
+    }
+    if (stt < pub) {
+      int pt;
+      const int unit = unit_of(stt, &pt);
+      uint32_t cnt = 0;
+      if (lane == 0) cnt = ld_acquire_gpu(p.gx_count + unit);
+      cnt = __shfl_sync(0xffffffffu, cnt, 0);
+      if (dead || cnt >= static_cast<uint32_t>(tpi)) {
+        __syncwarp();
+        const float2* gp = p.gx_part + static_cast<long long>(unit) * tpi * 32 + lane;
+        float g1 = 0.0f, g2 = 0.0f;
+        for (int r0 = 0; r0 < tpi; r0 += 16) {           // all loads in flight, the additions in tile order
+          float2 qv[16];
+#pragma unroll
+          for (int r = 0; r < 16; ++r) qv[r] = (r0 + r < tpi) ? __ldcg(gp + (r0 + r) * 32) : make_float2(0.0f, 0.0f);
+#pragma unroll
+          for (int r = 0; r < 16; ++r) { g1 += qv[r].x; g2 += qv[r].y; }
+        }
+        const float mu = g1 * inv_cnt;
+        aux[128 + (stt & 1) * 32 + lane] = make_float2(mu, rsqrtf(fmaxf(g2 * inv_cnt - mu * mu, 0.0f) + p.gn_eps));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&gx_stats[stt & 1]);
+        ++stt;
+        progressed = true;
+      }
+    }
+    if (progressed) { t0 = globaltimer_ns(); spins = 0; continue; }
+    if ((++spins & 15u) == 0u && !dead) {
+      if (*abort_flag) dead = true;                      // another role gave up: hand over what is owed and leave
+      else if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1u;
+        atomicOr(p.status, KF_DEV_TIMEOUT_EPILOGUE);
+        dead = true;
+      }
+    }
+  }
+}
+
 template <int BN, int EPI, int ACT, typename OutT, bool CTA2>
 __global__ void __launch_bounds__(num_threads(EPI, BN, CTA2), 1)
 umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -267,7 +556,13 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   uint64_t* tmem_empty = tmem_full + 2;
   uint64_t* r_full = tmem_empty + 2;
   uint64_t* rbar = r_full + 8;             // EPI_CONV_GN: [2] statistics from the cluster have arrived
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(rbar + 2);   // r_full: [epilogue warp][2]
+  // EPI_CONV_GNX: gx_parts[2] = the epilogue warps have left a tile's partial sums for the helper
+  // warp; gx_stats[2] = the helper warp has left the image's (mean, 1/std) per group
+  constexpr int kGxBars = EPI == EPI_CONV_GNX ? 4 : 0;
+  [[maybe_unused]] uint64_t* gx_parts = rbar + 2;
+  [[maybe_unused]] uint64_t* gx_stats = rbar + 4;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(rbar + 2 + kGxBars);   // r_full: [epilogue warp][2]
+  static_assert((2 * kStages + 4 + 8 + 2 + kGxBars) * 8 + 8 <= C::kBarBytes, "barrier block overflows");
   volatile uint32_t* abort_flag = tmem_holder + 1;
   // Convolution in slab mode: the ring holds two pixel copies of up to 48 KB and six weight slots
   // of 16 KB; its sixteen barriers are the stage barriers followed by r_full's (which only the
@@ -297,6 +592,10 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       mbar_init(&tmem_full[a], 1);
       mbar_init(&tmem_empty[a], (kEpiThreads / 32) * epi_groups(EPI, BN, CTA2) * (CTA2 ? 2 : 1));
       mbar_init(&rbar[a], 1);
+      if constexpr (EPI == EPI_CONV_GNX) {
+        mbar_init(&gx_parts[a], 2 * kEpiThreads / 32);      // one arrival per epilogue warp
+        mbar_init(&gx_stats[a], 1);
+      }
     }
     if (lane >= 16 && lane < 24) mbar_init(&r_full[lane - 16], 1);       // one per epilogue warp and buffer
     if (lane == 31) {
@@ -488,8 +787,21 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       }
     }
     __syncwarp();
+  } else if (EPI == EPI_CONV_GNX && warp == 2 + 4 * epi_groups(EPI, BN, CTA2)) {
+    // ------------------------------------------------------------ helper warp (EPI_CONV_GNX)
+    if constexpr (EPI == EPI_CONV_GNX) {
+      const int my_tiles = cta < p.num_tiles ? (p.num_tiles - cta + ncta - 1) / ncta : 0;
+      conv_gnx_helper(p, reinterpret_cast<float2*>(stg + C::kStaging + C::kBarBytes), gx_parts, gx_stats, abort_flag,
+                      lane, my_tiles, tile_at);
+    }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5, and 6..9 with two groups)
+    if constexpr (EPI == EPI_CONV_GNX) {
+      const int my_tiles = cta < p.num_tiles ? (p.num_tiles - cta + ncta - 1) / ncta : 0;
+      conv_gnx_epilogue<BN, ACT>(p, &tmY, stg, reinterpret_cast<float2*>(stg + C::kStaging + C::kBarBytes),
+                                 tmem_full, tmem_empty, gx_parts, gx_stats, abort_flag, tmem_base, warp, lane,
+                                 my_tiles, tile_at);
+    } else {
     constexpr int kGroups = epi_groups(EPI, BN, CTA2);
     constexpr int NB = 2 / kGroups;            // elementwise: staging buffers per group (4 pieces in all)
     constexpr int kGroupCols = BN / kGroups;   // columns of the tile one epilogue group owns
@@ -1318,6 +1630,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // every output store has finished reading shared memory (a no-op in lanes that issued none);
     // the writes themselves complete with the kernel, like any store in flight at exit
     bulk_wait_group_read<0>();
+    }   // the epilogues other than EPI_CONV_GNX
   }
 
   // ---------------------------------------------------------------- teardown

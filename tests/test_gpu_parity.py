@@ -788,6 +788,39 @@ def test_conv_groupnorm_cluster_kernel(kf, cfg, tuning):
     assert (np.abs(fused - two) <= 2.0 ** -7 * np.maximum(1.0, np.abs(two))).all()      # two bf16 ulps
 
 
+# The same chain on every SM (no clusters): the tiles of an image sit on neighbouring CTAs of a
+# cooperative grid, the group statistics travel through global memory, the epilogue is pipelined
+# one tile ahead.  Normally taken for 9..64 tiles per image on multi-wave problems; the knobs
+# force it here on small problems, including images that straddle two rounds of the schedule.
+@pytest.mark.parametrize("cfg", [
+    dict(Nb=3, Cin=64, H=64, W=64, Cout=128, groups=32),     # 16 tiles per image, benchmark geometry
+    dict(Nb=11, Cin=32, H=56, W=56, Cout=64, groups=8),      # 14 tiles of 224 pixels, ragged channel rows, 154 tiles: 2 rounds
+    dict(Nb=2, Cin=16, H=128, W=128, Cout=64, groups=4),     # 64 tiles per image
+    dict(Nb=40, Cin=16, H=16, W=16, Cout=160, groups=5),     # one tile per image, two channel tiles (the second ragged)
+    dict(Nb=5, Cin=16, H=30, W=40, Cout=32, groups=8),       # 8 tiles, the last one hangs over the image's end
+    dict(Nb=2, Cin=64, H=8, W=64, Cout=128, groups=32),      # fewer tiles than CTAs: one tile each
+])
+def test_conv_groupnorm_all_sm_kernel(kf, cfg, tuning):
+    d = ki.conv_inputs(seed=23, dtype="bf16", **cfg)
+    gamma = ki.store(ki.uniform(23, 7, (cfg["Cout"],), 0.5, 1.5), "bf16")
+    beta = ki.store(ki.uniform(23, 8, (cfg["Cout"],), -1.0, 1.0), "bf16")
+    tuning.setenv("KF_GNX_MIN_TILES", "1")
+    tuning.setenv("KF_GNX_MIN_TPI", "1")
+    before = kf.kf_launch_count()
+    for act, g_, b_ in (("relu", None, None), ("mish", gamma, beta)):
+        got, ref = run_conv(kf, d, act=act, gamma=g_, beta=b_)
+        assert_close(got, ref, 2e-2, 2e-2, "conv GN all SMs %s %s" % (cfg, act))
+    assert kf.kf_launch_count() - before == 4               # prepass + one kernel per call: the route was taken
+    again, _ = run_conv(kf, d, act="mish", gamma=gamma, beta=beta)
+    assert (again == got).all()                              # fixed summation order: repeat runs are bit-identical
+    # the two-kernel route on the same inputs: same statistics, activations rounded to bf16
+    # before instead of after the normalisation
+    fused, _ = run_conv(kf, d)
+    tuning.setenv("KF_NO_FUSED_GN", "1")
+    two, ref = run_conv(kf, d)
+    assert (np.abs(fused - two) <= 2.0 ** -7 * np.maximum(1.0, np.abs(two))).all()      # two bf16 ulps
+
+
 # ------------------------------------------------------------------ conv -> activation -> global average pool
 @pytest.mark.parametrize("dtype,cfg", [
     ("bf16", dict(Nb=2, Cin=64, H=8, W=64, Cout=128)),      # means from the tensor-core epilogue

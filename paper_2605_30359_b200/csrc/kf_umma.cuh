@@ -498,6 +498,7 @@ __device__ __forceinline__ void conv_gnx_helper(const UmmaParams& p, float2* aux
       }
     }
     if (progressed) { t0 = globaltimer_ns(); spins = 0; continue; }
+    __nanosleep(200);                                    // nothing due: do not compete with the mainloop for shared memory
     if ((++spins & 15u) == 0u && !dead) {
       if (*abort_flag) dead = true;                      // another role gave up: hand over what is owed and leave
       else if (globaltimer_ns() - t0 > kWaitLimitNs) {

@@ -315,24 +315,21 @@ __device__ __forceinline__ void conv_gnx_epilogue(const UmmaParams& p, const CUt
     const uint64_t bias2 = f32x2_pack(t.bias_v, t.bias_v);
     float s1 = 0.0f, s2 = 0.0f;
     uint64_t s1p = f32x2_pack(0.0f, 0.0f), s2p = s1p;   // (even, odd) pixel partial sums
+    // (the whole-tile case and the ragged case are two separate unrolled loops: the hot one stays
+    // contiguous in the instruction stream)
+    const bool whole = t.px_valid >= (piece0 + my_pieces) * 32 && my_pieces == kGP;
+    if (whole) {
 #pragma unroll
-    for (int c = 0; c < kGP; ++c) {
-      uint32_t v[32];
-      if (c < my_pieces) {
+      for (int c = 0; c < kGP; ++c) {
+        uint32_t v[32];
         tmem_ld_32x32(t_acc + c * 32, v);
         tmem_ld_wait();
-      } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = 0u;
-      }
-      if (c == kGP - 1) {
-        // the last of this warp's loads has landed: hand the accumulator back (one arrival per warp)
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&tmem_empty[a]);
-      }
-      const int left = t.px_valid - (piece0 + c) * 32;  // valid pixels from this piece on
-      if (left >= 32) {
+        if (c == kGP - 1) {
+          // the last of this warp's loads has landed: hand the accumulator back (one arrival per warp)
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tmem_empty[a]);
+        }
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
           float y0, y1;
@@ -344,9 +341,26 @@ __device__ __forceinline__ void conv_gnx_epilogue(const UmmaParams& p, const CUt
           s2p = f32x2_fma(y, y, s2p);
           st[c * 16 + j] = pack_bf16x2(y0, y1);
         }
-      } else {
-        // a tile that hangs over the end of its image: those pixels were read as zeros, are left
-        // out of the statistics and are not stored
+      }
+    } else {
+      // a tile that hangs over the end of its image (those pixels were read as zeros, are left out
+      // of the statistics and are not stored), or a group with fewer pieces than it has room for
+#pragma unroll
+      for (int c = 0; c < kGP; ++c) {
+        uint32_t v[32];
+        if (c < my_pieces) {
+          tmem_ld_32x32(t_acc + c * 32, v);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = 0u;
+        }
+        if (c == kGP - 1) {
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tmem_empty[a]);
+        }
+        const int left = t.px_valid - (piece0 + c) * 32;  // valid pixels from this piece on
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
           float y0 = act_f<ACT, true>(__uint_as_float(v[2 * j]) + t.bias_v, p.act_rt);
@@ -415,13 +429,15 @@ __device__ __forceinline__ void conv_gnx_epilogue(const UmmaParams& p, const CUt
     }
   };
 
-  uint32_t st_a[kGP * 16], st_b[kGP * 16];
+  // One copy of each phase's code (the unrolled per-piece loops are long, and instruction fetch was
+  // a visible stall with two): the new tile's activations are moved over to `st_old` after B.
+  uint32_t st_new[kGP * 16], st_old[kGP * 16];
   bool alive = true;
-  for (int it = 0; it <= my_tiles && alive; it += 2) {
-    if (it < my_tiles) alive = phase_a(it, st_a);
-    if (alive && it >= 1) phase_b(it - 1, st_b);
-    if (alive && it + 1 < my_tiles) alive = phase_a(it + 1, st_b);
-    if (alive && it < my_tiles) phase_b(it, st_a);
+  for (int it = 0; it <= my_tiles && alive; ++it) {
+    if (it < my_tiles) alive = phase_a(it, st_new);
+    if (alive && it >= 1) phase_b(it - 1, st_old);
+#pragma unroll
+    for (int j = 0; j < kGP * 16; ++j) st_old[j] = st_new[j];
   }
   bulk_wait_group_read<0>();
 }

@@ -1182,11 +1182,14 @@ static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
     // Taken for images of 9 to 64 tiles on problems of at least two waves (measured against the other
     // routes on B200: 128x64x64x64 -> 128, 16 tiles per image, 123.9 us against 131.0 in clusters of
     // 16, which occupy 112 of the 148 SMs; 8x64x128x128 -> 64, 64 tiles, 45.5 us against 75.6 for
-    // two kernels; 32x64x56x56 -> 64, 14 tiles, 39.4 against 39.3; smaller problems lose to the
-    // cooperative launch's set-up, images of hundreds of tiles to the wait for the whole image).
+    // two kernels; smaller problems lose to the cooperative launch's set-up, images of hundreds of
+    // tiles to the wait for the whole image) whose tiles fill the accumulator (tiles of 224 or 192
+    // pixels leave the two epilogue groups unequal shares and take the ragged loops: 32x64x56x56 ->
+    // 64 43.2 us against 39.3 for two kernels, 16x64x96x96 -> 64 62.4 against 54.3).
     const int gnx_min_tiles = tune().gnx_min_tiles >= 0 ? tune().gnx_min_tiles : 2 * d->sm_count;
     if (groups > 0 && p.staged && (cpg == 4 || cpg == 8 || cpg == 16 || cpg == 32) && tpi >= tune().gnx_min_tpi &&
-        tpi <= tune().gnx_max_tpi && p.num_tiles >= gnx_min_tiles && !tune().no_gnx && !tune().no_fused_gn) {
+        tpi <= tune().gnx_max_tpi && p.num_tiles >= gnx_min_tiles && (tile_px == bn || tune().gnx_min_tiles >= 0) &&
+        !tune().no_gnx && !tune().no_fused_gn) {
       UmmaParams q = p;
       q.gn_groups = groups; q.gn_eps = eps;
       q.gn_gamma = static_cast<const __nv_bfloat16*>(gamma);

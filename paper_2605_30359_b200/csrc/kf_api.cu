@@ -19,8 +19,9 @@ std::atomic<int64_t> g_launches{0};
 // to move a threshold); the environment is read ONCE, at the first call, and again only when
 // kf_reload_tuning() is called, so a call on the hot path reads no environment variable.
 struct Tuning {
-  bool no_fused_pool, no_tf32x3, no_splitk, no_pair, no_cluster_softmax, no_fused_softmax, no_fused_gn, no_conv_slab, no_gnx;
+  bool no_fused_pool, no_tf32x3, no_splitk, no_pair, no_cluster_softmax, no_fused_softmax, no_fused_gn, no_conv_slab, no_gnx, no_softmax_gx;
   int splitk_min_kb, splitk_two_per_sm, pair_min_k, pair_min_kb_per_cta, cl128_max_ctas;
+  int softmax_gx_min_tiles;                        // one-kernel softmax of wide rows: tiles in all (-1: two waves)
   int gnx_min_tiles, gnx_min_tpi, gnx_max_tpi;     // all-SM GroupNorm convolution: tiles in all (-1: two waves), tiles per image
 };
 Tuning g_tune;
@@ -41,6 +42,8 @@ void load_tuning_locked() {
   g_tune.no_fused_gn = flag("KF_NO_FUSED_GN");
   g_tune.no_conv_slab = flag("KF_NO_CONV_SLAB");
   g_tune.no_gnx = flag("KF_NO_GNX");
+  g_tune.no_softmax_gx = flag("KF_NO_SOFTMAX_GX");
+  g_tune.softmax_gx_min_tiles = num("KF_SOFTMAX_GX_MIN_TILES", -1);
   g_tune.splitk_min_kb = num("KF_SPLITK_MIN_KB", 28);
   g_tune.splitk_two_per_sm = num("KF_SPLITK_TWO_PER_SM", 1);
   g_tune.pair_min_k = num("KF_PAIR_MIN_K", 2048);
@@ -321,11 +324,16 @@ int rowreduce_bn(int64_t M, int64_t N, int red) {
   const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + kRowReduceNarrowBN - 1) / kRowReduceNarrowBN);
   return (softmax_like(red) && tiles <= 148) ? kRowReduceNarrowBN : kRowReduceBN;
 }
-size_t rowreduce_umma_ws(int64_t M, int64_t N, int red) {
+size_t rowreduce_part_bytes(int64_t M, int64_t N, int red) {
   const int bn = rowreduce_bn(M, N, red);
   const int64_t tiles_n = (N + bn - 1) / bn;
   // softmax: (max, sum) per row and per half tile (one per epilogue group); row sum: one float
-  return round256(static_cast<size_t>(M) * tiles_n * (softmax_like(red) ? 16 : 4));
+  // (rows rounded up to whole 128-row blocks: the one-kernel softmax lays its pairs out per block)
+  return round256(static_cast<size_t>((M + kBM - 1) / kBM * kBM) * tiles_n * (softmax_like(red) ? 16 : 4));
+}
+size_t rowreduce_umma_ws(int64_t M, int64_t N, int red) {
+  // ... followed, for the softmax, by one counter per 128-row block (the one-kernel form)
+  return rowreduce_part_bytes(M, N, red) + (red == RED_SOFTMAX ? round256(static_cast<size_t>((M + kBM - 1) / kBM) * 4) : 0);
 }
 // CTA pairs (256-row tiles, each CTA loading half of the W tile) pay off when the K loop is
 // long: measured +3.6 % at K = 4096, +3.3 % at K = 2048, -4 % at K = 1024 (fewer, larger tiles
@@ -983,6 +991,33 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
             return KF_OK;
           }
           (void)cudaGetLastError();
+        }
+      }
+      // Rows of 2..64 whole 256-column tiles on problems of at least two waves: one kernel on every
+      // SM; the tiles of a row block sit on neighbouring CTAs of a cooperative grid, exchange per-row
+      // (maximum, sum) through global memory and write final probabilities (no numerators in
+      // memory, no second pass)
+      {
+        const int gx_min = tune().softmax_gx_min_tiles >= 0 ? tune().softmax_gx_min_tiles : 2 * slots;
+        // (only where a tile's MMAs outlast this longer epilogue, K >= 2048: measured 4096x8192x2048
+        // 107.4 us against 110.2 for two kernels and 2048x16384x2048 122.9 / 123.8, but 4096x4096x1024
+        // 50.3 / 41.4 and 4096x8192x512 78.5 / 58.4; the part is power-limited on these shapes, so the
+        // gain is the energy of the numerators' round trip, not the second pass's time)
+        if (bn == kRowReduceBN && out_dtype == KF_BF16 && p.staged && N % kRowReduceBN == 0 && p.tiles_n >= 2 &&
+            p.tiles_n <= 64 && p.num_tiles >= gx_min && (K >= 2048 || tune().softmax_gx_min_tiles >= 0) &&
+            !tune().no_softmax_gx) {
+          uint8_t* cnt = static_cast<uint8_t*>(workspace) + rowreduce_part_bytes(M, N, red);
+          const size_t cnt_bytes = static_cast<size_t>((M + kBM - 1) / kBM) * 4;
+          if (cudaMemsetAsync(cnt, 0, cnt_bytes, st) != cudaSuccess) return KF_ERR_CUDA;
+          UmmaParams q = p;
+          q.gx_part = reinterpret_cast<float2*>(workspace);
+          q.gx_count = reinterpret_cast<uint32_t*>(cnt);
+          q.partial = nullptr;
+          if (launch_umma_softmax_gx(pre_act, pair ? 1 : 0, tm, q, grid, st) == cudaSuccess) {
+            g_launches += 1;
+            return KF_OK;
+          }
+          (void)cudaGetLastError();      // the device cannot hold the grid at once: the two-kernel route
         }
       }
       // a row that lies in one tile is finished in the GEMM epilogue: no second kernel

@@ -27,6 +27,10 @@ cudaError_t launch_umma_softmax(int bn, int act, int out_dt, int pair, const Umm
                                 const UmmaParams& p, int grid, cudaStream_t st);
 cudaError_t launch_umma_softmax_narrow(int act, int out_dt, const UmmaMaps& tm, const UmmaParams& p,
                                        int grid, cudaStream_t st);
+// the one-kernel softmax of wide rows: per-row (maximum, sum) exchanged through global memory,
+// cooperative launch (bf16 out, 256-column tiles)
+cudaError_t launch_umma_softmax_gx(int act, int pair, const UmmaMaps& tm, const UmmaParams& p, int grid,
+                                   cudaStream_t st);
 cudaError_t launch_umma_rowsum(int act, int pair, const UmmaMaps& tm, const UmmaParams& p,
                                int grid, cudaStream_t st);
 cudaError_t launch_umma_conv(int bn, int act, const UmmaMaps& tm, const UmmaParams& p, int grid,
@@ -213,13 +217,15 @@ inline cudaError_t launch_umma_instance(const UmmaMaps& tm, const UmmaParams& p,
     cfg.blockDim = dim3(num_threads(EPI, BN, CTA2), 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeCooperative;
+    attr[1].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = coop ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, kern, tm.a, tm.b, tm.r, tm.y, p);
   } else {
     // programmatic dependent launch: with few CTAs the next launch of the stream starts on the

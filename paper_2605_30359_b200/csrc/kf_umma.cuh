@@ -38,8 +38,11 @@ namespace kf {
 // EPI_CONV_GNX: the same chain on all SMs without clusters: the tiles of an image are held by
 // neighbouring CTAs of one co-resident (cooperative) grid, which exchange the group statistics
 // through global memory; the epilogue is software-pipelined so that the exchange is not waited for.
+// EPI_SOFTMAX_GX: the row softmax of a wide row (several 256-column tiles) in ONE kernel without
+// clusters: the tiles of a row block sit on neighbouring CTAs of a co-resident (cooperative) grid,
+// which exchange per-row (maximum, sum) through global memory; the numerators wait in registers.
 enum : int { EPI_ELEMENTWISE = 0, EPI_SOFTMAX = 1, EPI_ROWSUM = 2, EPI_CONV = 3, EPI_CONV_GN = 4,
-             EPI_SOFTMAX_CL = 5, EPI_CONV_GNX = 6 };
+             EPI_SOFTMAX_CL = 5, EPI_CONV_GNX = 6, EPI_SOFTMAX_GX = 7 };
 constexpr bool is_conv(int epi) { return epi == 3 || epi == 4 || epi == 6; }
 constexpr bool is_softmax(int epi) { return epi == 1 || epi == 5; }
 constexpr bool is_cluster_epi(int epi) { return epi == 4 || epi == 5; }
@@ -61,7 +64,7 @@ constexpr int kNumThreads = 192;  // 6 warps: producer, UMMA issuer, epilogue
 // cost it 2 %) keeps one group.
 constexpr int epi_groups(int epi, int bn, bool cta2) {
   return epi == 1 /* EPI_SOFTMAX */ || epi == 4 /* EPI_CONV_GN */ || epi == 5 /* EPI_SOFTMAX_CL */ ||
-                 epi == 6 /* EPI_CONV_GNX */ ||
+                 epi == 6 /* EPI_CONV_GNX */ || epi == 7 /* EPI_SOFTMAX_GX */ ||
                  (epi == 0 /* EPI_ELEMENTWISE */ && bn >= 64 && !cta2)
              ? 2 : 1;
 }
@@ -153,12 +156,13 @@ struct UmmaCfg {
   // staging: elementwise = 2 output + 2 residual pieces; softmax = 2 output pieces per epilogue
   // group; conv = 2 output pieces
   static constexpr int kStaging =
-      EPI == EPI_ELEMENTWISE || is_softmax(EPI) ? 4 * kPieceBytes
+      EPI == EPI_ELEMENTWISE || is_softmax(EPI) ? 4 * kPieceBytes      // (EPI_SOFTMAX_GX: one piece per group, below)
                                                     : (EPI == EPI_ROWSUM ? 0 : 2 * kPieceBytes);     // EPI_CONV_GN: one piece per epilogue group
   static constexpr int kBarBytes = 256;
   // GEMM epilogues: the tile's BN bias values as fp32, staged once per tile
-  // (EPI_CONV_GNX: partial sums [2][2 groups][32] and group statistics [2][32], float2)
-  static constexpr int kBiasBytes = EPI == EPI_CONV ? 0 : (EPI == EPI_CONV_GNX ? 1536 : BN * 4);   // EPI_CONV_GN: the statistics it sends
+  // (EPI_CONV_GNX: partial sums [2][2 groups][32] and group statistics [2][32], float2;
+  //  EPI_SOFTMAX_GX: the bias, then the groups' per-row (maximum, sum) [2 groups][128 rows] float2)
+  static constexpr int kBiasBytes = EPI == EPI_CONV ? 0 : (EPI == EPI_CONV_GNX ? 1536 : (EPI == EPI_SOFTMAX_GX ? BN * 4 + 2048 : BN * 4));   // EPI_CONV_GN: the statistics it sends
   // EPI_CONV_GN: statistics arriving from the cluster, [2 buffers][16 CTAs x 2 groups][32 x float2]
   // EPI_SOFTMAX_CL: [2 buffers][16 CTAs x 2 groups][128 rows x float2] arriving, then the
   // [2 buffers][2 groups][128 x float2] it sends
@@ -526,6 +530,234 @@ __device__ __forceinline__ void conv_gnx_helper(const UmmaParams& p, float2* aux
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Epilogue of EPI_SOFTMAX_GX: GEMM + bias (+ activation) + softmax over rows of several 256-column
+// tiles in one kernel, probabilities written once (no numerators in memory, no second pass).
+//
+// Tiles are dealt round-robin with the column tile fastest, so the tiles of a block of 128 rows
+// are held by neighbouring CTAs (CTA pairs) of one cooperative grid at (almost) the same time.  Two
+// epilogue groups of four warps, each owning 128 of the tile's columns; a thread is one row.
+//   A  maximum of the row's 128 values (first pass over the accumulator), then numerators
+//      e = exp(a - maximum) and their fp32 sum (second pass); the numerators stay in registers as
+//      bf16, the accumulator goes back to the UMMA issuer; one warp merges the two groups' (maximum,
+//      sum) per row, writes the tile's 128 pairs to global memory and counts the tile in (release
+//      at device scope);
+//   B  one thread checks (acquire, bounded) that all column tiles of the row block are counted in;
+//      a thread reads its row's pairs in tile order, forms the row's maximum M and denominator
+//      S = sum s_t exp(m_t - M), scales its numerators by exp(m - M) / S and stores them through
+//      shared memory and TMA.
+// The loop is software-pipelined: A of this CTA's next tile runs before B of the current one, so
+// the other CTAs have published by the time B asks.  A only waits for this CTA's own MMAs: the
+// waits cannot form a cycle.  A wait that runs out is reported at the next go/no-go, which all
+// eight warps take together.  Whole 256-column tiles only (N a multiple of 256).
+// ---------------------------------------------------------------------------------------------
+template <int BN, int ACT, bool CTA2, typename TileAt>
+__device__ __forceinline__ void softmax_gx_epilogue(const UmmaParams& p, const CUtensorMap* tmY, uint8_t* stg,
+                                                    float* sbias_all, float2* part, uint64_t* tmem_full,
+                                                    uint64_t* tmem_empty, volatile uint32_t* abort_flag,
+                                                    uint32_t tmem_base, uint32_t rank, int warp, int lane,
+                                                    int my_tiles, TileAt tile_at) {
+  constexpr int kGroups = 2;
+  constexpr int kGroupCols = BN / kGroups;              // 128
+  constexpr int PIECES = kGroupCols / 32;               // 4
+  constexpr int kTileM = CTA2 ? 2 * kBM : kBM;
+  constexpr float kLog2e = 1.4426950408889634f;
+  const int grp = (warp - 2) >> 2;
+  const int quad = warp & 3;
+  const int row = quad * 32 + lane;
+  const int et = static_cast<int>(threadIdx.x) - 64 - grp * kEpiThreads;
+  const bool leader = threadIdx.x == 64;
+  const bool grp_leader = et == 0;
+  const uint32_t bar_b = 2u + 2u * grp;
+  const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
+  float* sbias = sbias_all + grp * kGroupCols;
+  uint8_t* ybuf = stg + grp * kPieceBytes;              // the group's staging piece
+  const int tiles_n = p.tiles_n;
+  bool failed = false;
+
+  struct Tile { int tm, tn, m_cta, rb; };
+  auto locate = [&](int it) {
+    const int tile = tile_at(it);
+    Tile t;
+    t.tm = tile / tiles_n; t.tn = tile % tiles_n;
+    t.m_cta = t.tm * kTileM + static_cast<int>(rank) * kBM;
+    t.rb = t.m_cta / kBM;
+    return t;
+  };
+
+  auto phase_a = [&](int it, uint32_t (&st)[PIECES * 16], float& mx_out) -> bool {
+    const Tile t = locate(it);
+    const int a = it & 1;
+    const int n_tile = t.tn * BN + grp * kGroupCols;
+    // this thread's two of the group's bias values, fetched before the wait for the accumulator
+    float2 bpre = make_float2(0.0f, 0.0f);
+    if (p.bias != nullptr && 2 * et < kGroupCols) {
+      bpre.x = __bfloat162float(p.bias[n_tile + 2 * et]);
+      bpre.y = __bfloat162float(p.bias[n_tile + 2 * et + 1]);
+    }
+    bool ok = true;
+    if (leader)
+      ok = mbar_wait(&tmem_full[a], static_cast<uint32_t>((it >> 1) & 1), abort_flag, p.status,
+                     KF_DEV_TIMEOUT_EPILOGUE);
+    ok = named_barrier_and(9u, kGroups * kEpiThreads, ok && !failed);
+    if (!ok) return false;
+    tc_fence_after_sync();
+    if (2 * et < kGroupCols) *reinterpret_cast<float2*>(sbias + 2 * et) = bpre;
+    named_barrier_sync(bar_b, kEpiThreads);
+    const uint32_t t_acc = tmem_base + static_cast<uint32_t>(a * BN + grp * kGroupCols) + lane_off;
+    float mx = -INFINITY;
+#pragma unroll 1
+    for (int c = 0; c < PIECES; ++c) {
+      uint32_t v[32];
+      tmem_ld_32x32(t_acc + c * 32, v);
+      float bs[32];
+      load_sbias32(sbias + c * 32, bs);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        float z0, z1;
+        f32x2_unpack(f32x2_add(f32x2_pack(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])),
+                               f32x2_pack(bs[2 * j], bs[2 * j + 1])), z0, z1);
+        mx = fmaxf(mx, fmaxf(act_f<ACT, true>(z0, p.act_rt), act_f<ACT, true>(z1, p.act_rt)));
+      }
+    }
+    const uint64_t l2e2 = f32x2_pack(kLog2e, kLog2e);
+    const uint64_t off2 = f32x2_pack(-mx * kLog2e, -mx * kLog2e);
+    uint64_t sum2 = f32x2_pack(0.0f, 0.0f);
+#pragma unroll
+    for (int c = 0; c < PIECES; ++c) {
+      uint32_t v[32];
+      tmem_ld_32x32(t_acc + c * 32, v);
+      float bs[32];
+      load_sbias32(sbias + c * 32, bs);
+      tmem_ld_wait();
+      if (c == PIECES - 1) {
+        // the last load has landed: hand the accumulator back (one arrival per warp)
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) {
+          if constexpr (CTA2) mbar_arrive_cluster(mapa_shared(smem_u32(&tmem_empty[a]), 0));
+          else mbar_arrive(&tmem_empty[a]);
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        float z0, z1;
+        f32x2_unpack(f32x2_add(f32x2_pack(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])),
+                               f32x2_pack(bs[2 * j], bs[2 * j + 1])), z0, z1);
+        f32x2_unpack(f32x2_fma(f32x2_pack(act_f<ACT, true>(z0, p.act_rt), act_f<ACT, true>(z1, p.act_rt)), l2e2, off2),
+                     z0, z1);
+        const float e0 = exp2_approx(z0), e1 = exp2_approx(z1);
+        sum2 = f32x2_add(sum2, f32x2_pack(e0, e1));
+        st[c * 16 + j] = pack_bf16x2(e0, e1);
+      }
+    }
+    float se, so;
+    f32x2_unpack(sum2, se, so);
+    mx_out = mx;
+    part[grp * kBM + row] = make_float2(mx, se + so);
+    if (warp == 2) {
+      // the combiner: once all eight warps have arrived, the two groups' pairs merged per row go to
+      // global memory as 128 pairs (four coalesced stores per lane), and the tile is counted in
+      named_barrier_sync(10u, kGroups * kEpiThreads);
+      float2* dst = p.gx_part + (static_cast<long long>(t.rb) * tiles_n + t.tn) * kBM;
+#pragma unroll
+      for (int i = 0; i < kBM / 32; ++i) {
+        const int r = i * 32 + lane;
+        const float2 q0 = part[r], q1 = part[kBM + r];
+        const float m = fmaxf(q0.x, q1.x);
+        dst[r] = make_float2(m, q0.y * exp2_approx((q0.x - m) * kLog2e) + q1.y * exp2_approx((q1.x - m) * kLog2e));
+      }
+      __syncwarp();
+      if (lane == 0) red_release_gpu_add(p.gx_count + t.rb, 1u);
+    } else {
+      __threadfence_block();
+      named_barrier_arrive(10u, kGroups * kEpiThreads);
+    }
+    return true;
+  };
+
+  auto phase_b = [&](int it, const uint32_t (&st)[PIECES * 16], float mx) {
+    const Tile t = locate(it);
+    bool in = true;
+    if (leader) {
+      const uint64_t t0 = globaltimer_ns();
+      uint32_t spins = 0;
+      while (ld_acquire_gpu(p.gx_count + t.rb) < static_cast<uint32_t>(tiles_n)) {
+        __nanosleep(100);
+        if ((++spins & 15u) == 0u) {
+          if (*abort_flag) { in = false; break; }
+          if (globaltimer_ns() - t0 > kWaitLimitNs) {
+            *abort_flag = 1u;
+            atomicOr(p.status, KF_DEV_TIMEOUT_EPILOGUE);
+            in = false;
+            break;
+          }
+        }
+      }
+    }
+    in = named_barrier_and(11u, kGroups * kEpiThreads, in);
+    if (!in) failed = true;                  // the status word has it; finish the tile with the others
+    // the row's maximum and denominator from the tiles' pairs, in tile order (sixteen loads in flight)
+    float M = -INFINITY, S = 0.0f;
+    {
+      const float2* gp = p.gx_part + static_cast<long long>(t.rb) * tiles_n * kBM + row;
+      for (int t0 = 0; t0 < tiles_n; t0 += 16) {
+        float2 q[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          q[i] = (in && t0 + i < tiles_n) ? __ldcg(gp + static_cast<long long>(t0 + i) * kBM) : make_float2(-INFINITY, 0.0f);
+        float bm = M;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) bm = fmaxf(bm, q[i].x);
+        if (bm > -INFINITY) {
+          S *= exp2_approx((M - bm) * kLog2e);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) S += q[i].y * exp2_approx((q[i].x - bm) * kLog2e);
+          M = bm;
+        }
+      }
+    }
+    const float scale = exp2_approx((mx - M) * kLog2e) / S;
+    const uint64_t sc2 = f32x2_pack(scale, scale);
+#pragma unroll
+    for (int c = 0; c < PIECES; ++c) {
+      uint32_t w[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const uint32_t u = st[c * 16 + j];
+        float y0, y1;
+        f32x2_unpack(f32x2_mul(f32x2_pack(bf16_lo(u), bf16_hi(u)), sc2), y0, y1);
+        w[j] = pack_bf16x2(y0, y1);
+      }
+      if (grp_leader) bulk_wait_group_read<0>();     // the previous piece's store has let go of the buffer
+      named_barrier_sync(bar_b, kEpiThreads);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        *reinterpret_cast<uint4*>(ybuf + piece_off(row, q)) =
+            make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+      fence_proxy_async_smem();
+      named_barrier_sync(bar_b, kEpiThreads);
+      if (grp_leader) {
+        tma_store_2d(tmY, ybuf, t.tn * BN + grp * kGroupCols + c * kPieceCols, t.m_cta);   // clipped at M
+        bulk_commit_group();
+      }
+    }
+  };
+
+  uint32_t st_new[PIECES * 16], st_old[PIECES * 16];
+  float mx_new = 0.0f, mx_old = 0.0f;
+  bool alive = true;
+  for (int it = 0; it <= my_tiles && alive; ++it) {
+    if (it < my_tiles) alive = phase_a(it, st_new, mx_new);
+    if (alive && it >= 1) phase_b(it - 1, st_old, mx_old);
+#pragma unroll
+    for (int j = 0; j < PIECES * 16; ++j) st_old[j] = st_new[j];
+    mx_old = mx_new;
+  }
+  bulk_wait_group_read<0>();
+}
+
 template <int BN, int EPI, int ACT, typename OutT, bool CTA2>
 __global__ void __launch_bounds__(num_threads(EPI, BN, CTA2), 1)
 umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -813,7 +1045,12 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     }
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5, and 6..9 with two groups)
-    if constexpr (EPI == EPI_CONV_GNX) {
+    if constexpr (EPI == EPI_SOFTMAX_GX) {
+      const int my_tiles = cta < p.num_tiles ? (p.num_tiles - cta + ncta - 1) / ncta : 0;
+      float* sb = reinterpret_cast<float*>(stg + C::kStaging + C::kBarBytes);
+      softmax_gx_epilogue<BN, ACT, CTA2>(p, &tmY, stg, sb, reinterpret_cast<float2*>(sb + BN), tmem_full, tmem_empty,
+                                         abort_flag, tmem_base, rank, warp, lane, my_tiles, tile_at);
+    } else if constexpr (EPI == EPI_CONV_GNX) {
       const int my_tiles = cta < p.num_tiles ? (p.num_tiles - cta + ncta - 1) / ncta : 0;
       conv_gnx_epilogue<BN, ACT>(p, &tmY, stg, reinterpret_cast<float2*>(stg + C::kStaging + C::kBarBytes),
                                  tmem_full, tmem_empty, gx_parts, gx_stats, abort_flag, tmem_base, warp, lane,

@@ -529,6 +529,36 @@ def test_gemm_groupnorm(kf, dtype, shape, groups, tuning):
     assert np.abs(blk.var(axis=2) - 1.0).max() < (5e-2 if dtype == "bf16" else 1e-3)
 
 
+# Rows of several whole 256-column tiles in ONE kernel on every SM: the tiles of a row block sit on
+# neighbouring CTAs of a cooperative grid, exchange per-row (maximum, sum) through global memory and
+# write final probabilities; the numerators wait in registers.  Normally taken from K = 2048 on
+# problems of two waves; the knob forces it on small ones (single-CTA form below K = 2048, CTA pairs
+# from there).
+@pytest.mark.parametrize("shape,act", [
+    ((1000, 1024, 256), "none"),        # 8 row blocks x 4 tiles, ragged last row block
+    ((640, 2048, 128), "gelu_tanh"),    # a pre-activation; 5 x 8 tiles
+    ((256, 16384, 64), "none"),         # 64 tiles per row: two rounds of the schedule per row block
+    ((40000, 512, 64), "none"),         # 313 row blocks x 2 tiles: many rounds, counters of many blocks
+    ((1536, 1024, 2048), "none"),       # CTA pairs (K = 2048): 256-row tiles, both CTAs publish their own rows
+    ((700, 768, 2112), "relu"),         # CTA pairs, ragged last pair (rows 512..699), 33 K blocks
+])
+def test_bf16_softmax_wide_rows_one_kernel(kf, shape, act, tuning):
+    M, N, K = shape
+    d = ki.gemm_inputs("c3", seed=17, M=M, N=N, K=K)
+    tuning.setenv("KF_SOFTMAX_GX_MIN_TILES", "1")
+    before = kf.kf_launch_count()
+    P = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), act, "softmax")
+    check_status()
+    assert kf.kf_launch_count() - before == 1                # the one-kernel route was taken
+    ref = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], act, "softmax")
+    got = to_f64(P)
+    assert_close(got, ref, 2e-2, 2e-2, "softmax one kernel %s" % (shape,))
+    assert_close(got, ref, 1e-7, 2e-2, "softmax one kernel, relative %s" % (shape,))
+    assert np.abs(got.sum(axis=1) - 1.0).max() < 4e-3
+    P2 = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), act, "softmax")
+    assert (to_f64(P2) == got).all()                          # fixed order of the exchange: bit-identical repeats
+
+
 # Rows that lie in one tile (N <= 256, or <= 64 on the narrow-tile kernel): the softmax is finished
 # inside the GEMM epilogue (maxima and sums exchanged between the two epilogue groups), no second
 # kernel runs.

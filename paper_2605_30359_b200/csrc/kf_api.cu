@@ -286,14 +286,11 @@ int64_t conv_stat_parts(int64_t H, int64_t Wd) {
   return (H + r - 1) / r * conv_w_segs(Wd);
 }
 // per-tile channel statistics of the two-kernel route, or (same region) the per-tile group
-// statistics of the all-SM GroupNorm kernel, followed by that kernel's per-image counters
-size_t conv_gx_part_bytes(int64_t Nb, int64_t H, int64_t Wd, int64_t Cout) {
+// statistics of the all-SM GroupNorm kernel (one 256-byte row per tile)
+size_t conv_stats_bytes(int64_t Nb, int64_t H, int64_t Wd, int64_t Cout) {
   const size_t per_channel = static_cast<size_t>(Nb) * conv_stat_parts(H, Wd) * Cout * 8;
   const size_t per_group = static_cast<size_t>(Nb) * ((Cout + kBM - 1) / kBM) * conv_stat_parts(H, Wd) * 256;
   return round256(per_channel > per_group ? per_channel : per_group);
-}
-size_t conv_stats_bytes(int64_t Nb, int64_t H, int64_t Wd, int64_t Cout) {
-  return conv_gx_part_bytes(Nb, H, Wd, Cout) + round256(static_cast<size_t>(Nb) * ((Cout + kBM - 1) / kBM) * 4);
 }
 
 kf_status check_gemm_common(int64_t M, int64_t N, int64_t K, int dt, const void* X, int64_t ldx,
@@ -1151,13 +1148,6 @@ static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
     void* xt = workspace;
     void* wr = static_cast<uint8_t*>(workspace) + xt_bytes;
     float* stats = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + xt_bytes + wr_bytes);
-    uint32_t* gx_count = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(stats) + conv_gx_part_bytes(Nb, H, Wd, Cout));
-    const int gx_units = static_cast<int>(Nb * ((Cout + kBM - 1) / kBM));
-    if (launch_conv_prep(static_cast<int>(Nb), static_cast<int>(Cin), static_cast<int>(Cp),
-                         static_cast<int>(H), static_cast<int>(Wd), static_cast<int>(Cout), x, w, xt, wr,
-                         st, groups > 0 ? gx_count : nullptr, gx_units) != cudaSuccess)
-      return KF_ERR_CUDA;
-    ++launches;
     const int rows = conv_rows_per_tile(H, Wd);        // image rows per tile
     const int segs = conv_w_segs(Wd);                  // > 1: a tile is one segment of one row
     const int tile_px = static_cast<int>(rows * Wd / segs);   // pixels per tile = UMMA N
@@ -1222,16 +1212,23 @@ static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
     // pixels leave the two epilogue groups unequal shares and take the ragged loops: 32x64x56x56 ->
     // 64 43.2 us against 39.3 for two kernels, 16x64x96x96 -> 64 62.4 against 54.3).
     const int gnx_min_tiles = tune().gnx_min_tiles >= 0 ? tune().gnx_min_tiles : 2 * d->sm_count;
-    if (groups > 0 && p.staged && (cpg == 4 || cpg == 8 || cpg == 16 || cpg == 32) && tpi >= tune().gnx_min_tpi &&
-        tpi <= tune().gnx_max_tpi && p.num_tiles >= gnx_min_tiles && (tile_px == bn || tune().gnx_min_tiles >= 0) &&
-        !tune().no_gnx && !tune().no_fused_gn) {
+    const bool gnx = groups > 0 && p.staged && (cpg == 4 || cpg == 8 || cpg == 16 || cpg == 32) &&
+                     tpi >= tune().gnx_min_tpi && tpi <= tune().gnx_max_tpi && p.num_tiles >= gnx_min_tiles &&
+                     (tile_px == bn || tune().gnx_min_tiles >= 0) && !tune().no_gnx && !tune().no_fused_gn;
+    // the prepass (NHWC copy, weights by tap); with it, for the all-SM GroupNorm kernel, the exchange
+    // buffer is filled with the pattern that means "no pair here yet" (one 256-byte row per tile)
+    if (launch_conv_prep(static_cast<int>(Nb), static_cast<int>(Cin), static_cast<int>(Cp),
+                         static_cast<int>(H), static_cast<int>(Wd), static_cast<int>(Cout), x, w, xt, wr,
+                         st, gnx ? stats : nullptr, gnx ? static_cast<size_t>(p.num_tiles) * 256 : 0) != cudaSuccess)
+      return KF_ERR_CUDA;
+    ++launches;
+    if (gnx) {
       UmmaParams q = p;
       q.gn_groups = groups; q.gn_eps = eps;
       q.gn_gamma = static_cast<const __nv_bfloat16*>(gamma);
       q.gn_beta = static_cast<const __nv_bfloat16*>(beta);
       q.partial = nullptr;
       q.gx_part = reinterpret_cast<float2*>(stats);
-      q.gx_count = gx_count;
       const int gridx = q.num_tiles < d->sm_count ? q.num_tiles : d->sm_count;
       if (launch_umma_conv_gnx(bn, act, tm, q, gridx, st) == cudaSuccess) {
         g_launches += launches + 1;

@@ -67,10 +67,10 @@ cudaError_t launch_row_reduce(int red, int M, int N, const float* A, long long l
                               cudaStream_t st);
 
 // convolution helpers
-// (also sets `zero_words` 32-bit words at `zero` to 0: the counters of EPI_CONV_GNX)
+// (also sets `ones_bytes` bytes at `ones` to 0xff: the empty exchange buffer of EPI_CONV_GNX)
 cudaError_t launch_conv_prep(int Nb, int Cin, int Cp, int H, int Wd, int Cout, const void* x,
-                             const void* w, void* xt, void* wr, cudaStream_t st, void* zero = nullptr,
-                             int zero_words = 0);
+                             const void* w, void* xt, void* wr, cudaStream_t st, void* ones = nullptr,
+                             size_t ones_bytes = 0);
 cudaError_t launch_conv_direct(int dt, int act, int Nb, int Cin, int H, int Wd, int Cout,
                                const void* x, const void* w, const void* bias, void* y,
                                cudaStream_t st);

@@ -72,6 +72,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
+// The same question without waiting at all (try_wait may suspend the thread for a while): for a
+// warp that has something else to look at when the answer is no.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.b32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
 // Bounded wait.  Returns false if the CTA is aborting (another role gave up) or if this wait
 // ran out of time, in which case it raises the CTA's abort flag and the device status word.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
@@ -110,6 +126,17 @@ __device__ __forceinline__ uint32_t ld_relaxed_gpu(const uint32_t* addr) {
 __device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* addr) {
   uint32_t v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
+  return v;
+}
+// A 64-bit word that is its own flag: the producer stores the datum (never the "empty" pattern the
+// buffer was filled with), a consumer that loads anything else has the datum.  Aligned 64-bit
+// accesses are single-copy atomic, so neither side needs a fence or a counter.
+__device__ __forceinline__ void st_relaxed_gpu_b64(uint64_t* addr, uint64_t v) {
+  asm volatile("st.relaxed.gpu.global.b64 [%0], %1;" ::"l"(addr), "l"(v) : "memory");
+}
+__device__ __forceinline__ uint64_t ld_relaxed_gpu_b64(const uint64_t* addr) {
+  uint64_t v;
+  asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(v) : "l"(addr) : "memory");
   return v;
 }
 // Arrive without waiting: the producer half of a producer / consumer hand-over (the consumer

@@ -209,9 +209,8 @@ cudaError_t launch_pad_rows_bf16(long long rows, int K, int kp, const void* in, 
 }
 
 cudaError_t launch_conv_prep(int Nb, int Cin, int Cp, int H, int Wd, int Cout, const void* x,
-                             const void* w, void* xt, void* wr, cudaStream_t st, void* zero, int zero_words) {
-  if (zero != nullptr && zero_words > 0 &&
-      cudaMemsetAsync(zero, 0, static_cast<size_t>(zero_words) * 4, st) != cudaSuccess)
+                             const void* w, void* xt, void* wr, cudaStream_t st, void* ones, size_t ones_bytes) {
+  if (ones != nullptr && ones_bytes > 0 && cudaMemsetAsync(ones, 0xff, ones_bytes, st) != cudaSuccess)
     return cudaGetLastError();
   const __nv_bfloat16* xs = static_cast<const __nv_bfloat16*>(x);
   const __nv_bfloat16* ws = static_cast<const __nv_bfloat16*>(w);

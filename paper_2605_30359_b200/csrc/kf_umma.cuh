@@ -121,8 +121,10 @@ struct UmmaParams {
   int slab_bytes;              // bytes of one such copy (<= 48 KB)
   int slab_row_bytes;          // bytes of one image row of the copy: box_w * 128, a multiple of 1024
   // EPI_CONV_GNX: per (image, channel tile) unit u: gx_part[(u * tiles_per_image + t) * 32 + g] =
-  // (sum, sum of squares) of GroupNorm group g over pixel tile t; gx_count[u] = tiles published
-  // (zero when the kernel starts)
+  // (sum, sum of squares) of GroupNorm group g over pixel tile t; all bits set where no pair has
+  // been stored yet (the state the kernel starts from)
+  // EPI_SOFTMAX_GX: gx_part[(row block * tiles_n + t) * 128 + row] = (maximum, sum) of a row over
+  // column tile t; gx_count[row block] = tiles published (zero when the kernel starts)
   float2* gx_part;
   uint32_t* gx_count;
   int pool2;                   // convolution: 0, or 2x2 pooling in the epilogue (1 = max, 2 = mean);
@@ -152,7 +154,7 @@ template <int BN, int EPI, bool CTA2 = false>
 struct UmmaCfg {
   static constexpr int kStageA = kBM * kBK * 2;
   static constexpr int kStageB = (CTA2 ? BN / 2 : BN) * kBK * 2;
-  static constexpr int kStage = kStageA + kStageB;
+  static constexpr int kStage1 = kStageA + kStageB;          // one 64-wide K block of A and B
   // staging: elementwise = 2 output + 2 residual pieces; softmax = 2 output pieces per epilogue
   // group; conv = 2 output pieces
   static constexpr int kStaging =
@@ -169,7 +171,15 @@ struct UmmaCfg {
   // (EPI_SOFTMAX_CL: clusters of up to 16 CTAs with 64-column tiles, up to 8 with wider ones)
   static constexpr int kClMax = BN <= 64 ? 16 : 8;
   static constexpr int kInboxBytes = EPI == EPI_CONV_GN ? 2 * 32 * 256 : (EPI == EPI_SOFTMAX_CL ? 2 * 2 * kClMax * 1024 + 4 * 1024 : 0);
-  static constexpr int kFit = (kMaxDynSmem - 1024 - kStaging - kBarBytes - kBiasBytes - kInboxBytes) / kStage;
+  // GEMMs: a stage holds two K blocks behind one barrier where three such stages fit.  The UMMA
+  // issuer pays a barrier wait, an election and a commit per stage, each of which waits its turn
+  // behind the operand reads of the MMAs in flight (150 cycles and more): with one block per
+  // stage it needed about 600 cycles per block against the tensor pipe's 512 (256 at 128-column
+  // tiles), and the pipe's short queue ran dry.
+  static constexpr int kBudget = kMaxDynSmem - 1024 - kStaging - kBarBytes - kBiasBytes - kInboxBytes;
+  static constexpr int kKB = (!is_conv(EPI) && kBudget / (2 * kStage1) >= 3) ? 2 : 1;
+  static constexpr int kStage = kKB * kStage1;
+  static constexpr int kFit = kBudget / kStage;
   static constexpr int kStages = kFit > 8 ? 8 : kFit;
   static constexpr int kRing = kStage * kStages;
   static constexpr int kTotal = 1024 /*alignment slack*/ + kRing + kStaging + kBarBytes + kBiasBytes + kInboxBytes;
@@ -247,12 +257,12 @@ __device__ __forceinline__ void load_sbias32(const float* sb, float (&b)[32]) {
 //   A  the thread reads its share of the accumulator ONCE (the warp hands the accumulator back to
 //      the UMMA issuer as soon as its last load has landed), applies bias and activation, adds up
 //      sum and sum of squares in fp32 and keeps the activations in registers as bf16; shuffles
-//      reduce the sums over the channels of a GroupNorm group; one warp adds the two groups'
-//      partial sums, writes the tile's 32 (sum, sum of squares) pairs to global memory and
-//      counts the tile in (release at device scope).
-//   B  one thread checks (acquire, bounded) that all of the image's tiles are counted in; every
-//      thread adds the tiles' pairs of its group in tile order, normalises its activations from
-//      the registers and stores them through the warp's 2 KB slab (32 channels x 32 pixels) with TMA.
+//      reduce the sums over the channels of a GroupNorm group; the helper warp adds the two
+//      groups' partial sums and stores the tile's 32 (sum, sum of squares) pairs to global memory.
+//   B  the helper warp has read the pairs of all of the image's tiles (each 64-bit pair is its own
+//      "present" flag: no counter, no fence), added them up in tile order and left (mean, 1/std)
+//      per group in shared memory; every thread normalises its activations from the registers
+//      and stores them through the warp's 2 KB slab (32 channels x 32 pixels) with TMA.
 // The loop is software-pipelined: A of this CTA's next tile runs BEFORE B of the current one (two
 // register buffers of activations), so by the time B asks, the other CTAs have long published and
 // the exchange's latency is hidden behind an accumulator pass.  A only ever waits for this CTA's
@@ -448,13 +458,19 @@ __device__ __forceinline__ void conv_gnx_epilogue(const UmmaParams& p, const CUt
 
 // The helper warp of EPI_CONV_GNX: everything in the GroupNorm exchange that touches global memory.
 // A small state machine over this CTA's tiles, never blocking on one thing while another is due:
-//   publish(k)  once the epilogue warps have left tile k's partial sums: the two groups' sums in a
-//               fixed order to global memory as one 256-byte row, a fence, and the tile is counted
-//               in (release at device scope);
-//   stats(k)    once all tiles of tile k's image are counted in (acquire): lane g adds the tiles'
-//               pairs of group g in tile order and leaves (mean, 1/std) for the epilogue warps.
+//   publish(k)  once the epilogue warps have left tile k's partial sums (tested, not waited for: a
+//               try_wait may suspend the warp while statistics are due): the two groups' sums in
+//               a fixed order to global memory as one 256-byte row of 64-bit pairs;
+//   stats(k)    lane g loads group g's pair of every tile of tile k's image; once none of them is
+//               the "empty" pattern any more it adds them in tile order and leaves (mean, 1/std)
+//               for the epilogue warps.  (With a counter per image, a release after the stores
+//               and an acquire before the loads, the two fences cost this warp about 3000 cycles
+//               per tile beside the mainloop, and the image's statistics arrived 4000 cycles
+//               after the epilogue asked for them.)
 // Every wait is bounded; a wait that runs out raises the abort flag, and the outstanding hand-overs
 // are still completed so that no epilogue warp is left waiting on a barrier.
+constexpr uint64_t kGxEmpty = ~0ull;   // what the exchange buffer holds before a tile's pair arrives
+
 template <typename TileAt>
 __device__ __forceinline__ void conv_gnx_helper(const UmmaParams& p, float2* aux, uint64_t* gx_parts,
                                                 uint64_t* gx_stats, volatile uint32_t* abort_flag,
@@ -473,9 +489,10 @@ __device__ __forceinline__ void conv_gnx_helper(const UmmaParams& p, float2* aux
   bool dead = false;
   uint64_t t0 = globaltimer_ns();
   uint32_t spins = 0;
+  uint64_t* gx = reinterpret_cast<uint64_t*>(p.gx_part);
   while (stt < my_tiles) {
     bool progressed = false;
-    if (pub < my_tiles && (dead || mbar_try_wait(&gx_parts[pub & 1], static_cast<uint32_t>((pub >> 1) & 1)))) {
+    if (pub < my_tiles && (dead || mbar_test_wait(&gx_parts[pub & 1], static_cast<uint32_t>((pub >> 1) & 1)))) {
       int pt;
       const int unit = unit_of(pub, &pt);
       const float2* part = aux + (pub & 1) * 64;
@@ -484,31 +501,33 @@ __device__ __forceinline__ void conv_gnx_helper(const UmmaParams& p, float2* aux
         const float2 a0 = part[lane], a1 = part[32 + lane];
         m = make_float2(a0.x + a1.x, a0.y + a1.y);
       }
-      p.gx_part[(static_cast<long long>(unit) * tpi + pt) * 32 + lane] = m;
-      // the warp's 32 stores are ordered before lane 0's release by the warp barrier; no separate
-      // device-wide fence (measured: a fence per tile in this warp cost the kernel 5 us)
-      __syncwarp();
-      if (lane == 0) red_release_gpu_add(p.gx_count + unit, 1u);
+      // the pair is its own flag (see st_relaxed_gpu_b64); the one pattern that means "not yet"
+      // (two NaNs of all ones, which no addition produces) is stored as the canonical NaN pair
+      uint64_t bits = (static_cast<uint64_t>(__float_as_uint(m.y)) << 32) | __float_as_uint(m.x);
+      if (bits == kGxEmpty) bits = 0x7fffffff7fffffffull;
+      st_relaxed_gpu_b64(gx + (static_cast<long long>(unit) * tpi + pt) * 32 + lane, bits);
       ++pub;
       progressed = true;
     }
     if (stt < pub) {
       int pt;
       const int unit = unit_of(stt, &pt);
-      uint32_t cnt = 0;
-      if (lane == 0) cnt = ld_acquire_gpu(p.gx_count + unit);
-      cnt = __shfl_sync(0xffffffffu, cnt, 0);
-      if (dead || cnt >= static_cast<uint32_t>(tpi)) {
-        __syncwarp();
-        const float2* gp = p.gx_part + static_cast<long long>(unit) * tpi * 32 + lane;
-        float g1 = 0.0f, g2 = 0.0f;
-        for (int r0 = 0; r0 < tpi; r0 += 16) {           // all loads in flight, the additions in tile order
-          float2 qv[16];
+      const uint64_t* gp = gx + static_cast<long long>(unit) * tpi * 32 + lane;
+      float g1 = 0.0f, g2 = 0.0f;
+      bool all = true;
+      for (int r0 = 0; r0 < tpi; r0 += 16) {             // all loads in flight, the additions in tile order
+        uint64_t qv[16];
 #pragma unroll
-          for (int r = 0; r < 16; ++r) qv[r] = (r0 + r < tpi) ? __ldcg(gp + (r0 + r) * 32) : make_float2(0.0f, 0.0f);
+        for (int r = 0; r < 16; ++r) qv[r] = (r0 + r < tpi) ? ld_relaxed_gpu_b64(gp + (r0 + r) * 32) : 0ull;
 #pragma unroll
-          for (int r = 0; r < 16; ++r) { g1 += qv[r].x; g2 += qv[r].y; }
+        for (int r = 0; r < 16; ++r) {
+          all = all && qv[r] != kGxEmpty;
+          g1 += __uint_as_float(static_cast<uint32_t>(qv[r]));
+          g2 += __uint_as_float(static_cast<uint32_t>(qv[r] >> 32));
         }
+      }
+      all = __all_sync(0xffffffffu, all);
+      if (dead || all) {
         const float mu = g1 * inv_cnt;
         aux[128 + (stt & 1) * 32 + lane] = make_float2(mu, rsqrtf(fmaxf(g2 * inv_cnt - mu * mu, 0.0f) + p.gn_eps));
         __syncwarp();
@@ -814,11 +833,15 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   static_assert((2 * kStages + 4 + 8 + 2 + kGxBars) * 8 + 8 <= C::kBarBytes, "barrier block overflows");
   volatile uint32_t* abort_flag = tmem_holder + 1;
   // Convolution in slab mode: the ring holds two pixel copies of up to 48 KB and six weight slots
-  // of 16 KB; its sixteen barriers are the stage barriers followed by r_full's (which only the
-  // elementwise chain uses): weight slot full [0,6), empty [6,12), copy full [12,14), empty [14,16).
+  // of 16 KB; its barriers are the stage barriers followed by r_full's (which only the
+  // elementwise chain uses).
   [[maybe_unused]] constexpr int kSlabPx = 49152;
-  [[maybe_unused]] constexpr int kSlabW = 6;
-  static_assert(!is_conv(EPI) || (C::kRing >= 2 * kSlabPx + kSlabW * C::kStageA && kStages >= 4), "slab layout");
+  [[maybe_unused]] constexpr int kSlabBufs = 2;     // pixel copies in flight
+  [[maybe_unused]] constexpr int kSlabW = 6;        // weight slots: the three taps of two column shifts
+  // barriers: "this column shift's copy and its three weight blocks have landed" [0,2); weight slot
+  // free [2,8); copy buffer free [8,10)
+  [[maybe_unused]] constexpr int kGFull = 0, kWEmpty = 2, kCEmpty = 8;
+  static_assert(!is_conv(EPI) || (C::kRing >= kSlabBufs * kSlabPx + kSlabW * C::kStageA && kStages >= 4), "slab layout");
   [[maybe_unused]] auto slab_bar = [&](int i) -> uint64_t* {
     return i < 2 * kStages ? full + i : r_full + (i - 2 * kStages);
   };
@@ -896,21 +919,22 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             // (out-of-image pixels read zeros: the padding), then the three row taps' weights.
             for (int cs = 0; cs < 3 * p.kb_per_tap && ok; ++cs) {
               const int cb = cs / 3, sx = cs % 3;
-              ok = mbar_wait(slab_bar(12 + 2 + pb), pph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_PRODUCER);
+              ok = mbar_wait(slab_bar(kCEmpty + pb), pph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_PRODUCER);
               ok = __all_sync(0xffffffffu, ok);
               if (!ok) break;
+              // (one barrier per column shift takes the copy's bytes and the three weight blocks')
+              uint64_t* gfull = slab_bar(kGFull + pb);
               if (elect_one()) {
-                mbar_expect_tx(slab_bar(12 + pb), static_cast<uint32_t>(p.slab_bytes));
-                tma_load_4d(ring + pb * kSlabPx, &tmR, slab_bar(12 + pb), cb * kBK, x0 + sx - 1, h0 - 1, img);
+                mbar_expect_tx(gfull, static_cast<uint32_t>(p.slab_bytes) + 3u * C::kStageA);
+                tma_load_4d(ring + pb * kSlabPx, &tmR, gfull, cb * kBK, x0 + sx - 1, h0 - 1, img);
               }
-              if (++pb == 2) { pb = 0; pph ^= 1u; }
+              if (++pb == kSlabBufs) { pb = 0; pph ^= 1u; }
               for (int r = 0; r < 3; ++r) {
-                ok = mbar_wait(slab_bar(6 + s), ph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_PRODUCER);
+                ok = mbar_wait(slab_bar(kWEmpty + s), ph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_PRODUCER);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (elect_one()) {
-                  mbar_expect_tx(slab_bar(s), C::kStageA);
-                  tma_load_2d(ring + 2 * kSlabPx + s * C::kStageA, &tmA, slab_bar(s), cb * kBK,
+                  tma_load_2d(ring + kSlabBufs * kSlabPx + s * C::kStageA, &tmA, gfull, cb * kBK,
                               (r * 3 + sx) * p.N + tm * kBM);
                 }
                 if (++s == kSlabW) { s = 0; ph ^= 1u; }
@@ -920,18 +944,23 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             continue;
           }
         }
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
+        for (int kb = 0; kb < p.k_blocks; kb += C::kKB) {
           ok = mbar_wait(&empty[s], ph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_PRODUCER);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           uint8_t* sa = ring + s * C::kStage;
           uint8_t* sb = sa + C::kStageA;
+          [[maybe_unused]] const int kbs = min(C::kKB, p.k_blocks - kb);   // K blocks in this stage
           if constexpr (CTA2) {
             if (elect_one()) {
               // both CTAs' bytes complete on rank 0's barrier, which rank 0 arms for the pair
-              if (rank == 0) mbar_expect_tx(&full[s], 2 * C::kStage);
-              tma_load_2d_pair(sa, &tmA, &full[s], kb * kBK, tm * kTileM + static_cast<int>(rank) * kBM);
-              tma_load_2d_pair(sb, &tmB, &full[s], kb * kBK, tn * BN + static_cast<int>(rank) * (BN / 2));
+              if (rank == 0) mbar_expect_tx(&full[s], static_cast<uint32_t>(2 * kbs * C::kStage1));
+              for (int j = 0; j < kbs; ++j) {
+                tma_load_2d_pair(sa + j * C::kStage1, &tmA, &full[s], (kb + j) * kBK,
+                                 tm * kTileM + static_cast<int>(rank) * kBM);
+                tma_load_2d_pair(sb + j * C::kStage1, &tmB, &full[s], (kb + j) * kBK,
+                                 tn * BN + static_cast<int>(rank) * (BN / 2));
+              }
             }
           } else if constexpr (is_conv(EPI)) {
             const int tap = kb / p.kb_per_tap, cb = kb % p.kb_per_tap;
@@ -946,9 +975,11 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
           } else {
             if (elect_one()) {
-              mbar_expect_tx(&full[s], C::kStage);
-              tma_load_2d(sa, &tmA, &full[s], kb * kBK, tm * kBM);
-              tma_load_2d(sb, &tmB, &full[s], kb * kBK, tn * BN);
+              mbar_expect_tx(&full[s], static_cast<uint32_t>(kbs * C::kStage1));
+              for (int j = 0; j < kbs; ++j) {
+                tma_load_2d(sa + j * C::kStage1, &tmA, &full[s], (kb + j) * kBK, tm * kBM);
+                tma_load_2d(sb + j * C::kStage1, &tmB, &full[s], (kb + j) * kBK, tn * BN);
+              }
             }
           }
           if (++s == kStages) { s = 0; ph ^= 1u; }
@@ -966,61 +997,82 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       int s = 0; uint32_t ph = 0; int a = 0; uint32_t aph = 0;
       [[maybe_unused]] int pb = 0; [[maybe_unused]] uint32_t pph = 0;   // slab mode: pixel-copy buffer and its phase
       bool ok = true;
-      for (int it = 0; ok; ++it) {
+      bool slab_done = false;
+      if constexpr (is_conv(EPI)) {
+        if (p.slab) {
+          // Slab mode, all of this CTA's tiles as one sequence of column shifts (three per 64-channel
+          // block of a tile).  Per shift ONE barrier says that its copy and its weight blocks have
+          // landed; one elected lane then issues its twelve MMAs and the commits.  (A barrier
+          // operation waits its turn behind the MMAs' operand reads, 150 cycles and more: with a
+          // wait, an election and a branch per weight block the issuer needed about 600 cycles
+          // per block against the tensor pipe's 512.)
+          int my_tiles = 0;
+          while (tile_at(my_tiles) >= 0) ++my_tiles;
+          const int ncs = 3 * p.kb_per_tap;
+          const int total = my_tiles * ncs;
+          int cs = 0;
+          for (int g = 0; g < total && ok; ++g) {
+            if (cs == 0) ok = mbar_wait(&tmem_empty[a], aph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
+            ok = ok && mbar_wait(slab_bar(kGFull + pb), pph, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(a * BN);
+            const uint32_t px = smem_u32(ring + pb * kSlabPx);
+            const uint32_t wbase = smem_u32(ring + kSlabBufs * kSlabPx);
+            const bool tile_end = cs == ncs - 1;
+            if (elect_one()) {
+#pragma unroll
+              for (int r = 0; r < 3; ++r) {
+                const int slot = s + r;                                // the shift's three blocks: slots s..s+2
+                const uint64_t adesc = smem_desc_kmajor_sw128(wbase + static_cast<uint32_t>(slot * C::kStageA));
+                // the window of tap row r starts r image rows (whole 1024-byte groups) into the copy
+                const uint64_t bdesc = smem_desc_kmajor_sw128(px + static_cast<uint32_t>(r * p.slab_row_bytes));
+#pragma unroll
+                for (int k = 0; k < kBK / kUmmaK; ++k)
+                  umma_f16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (cs | r | k) != 0 ? 1u : 0u);
+                umma_commit(slab_bar(kWEmpty + slot));                  // frees the weight slot
+              }
+              umma_commit(slab_bar(kCEmpty + pb));                  // after the third tap, the copy
+              if (tile_end) umma_commit(&tmem_full[a]);
+            }
+            __syncwarp();
+            s = s == 0 ? 3 : 0;                                     // (slots 0..2 and 3..5 in turn)
+            if (++pb == kSlabBufs) { pb = 0; pph ^= 1u; }
+            if (tile_end) { cs = 0; if (++a == 2) { a = 0; aph ^= 1u; } } else { ++cs; }
+          }
+          slab_done = true;
+        }
+      }
+      for (int it = 0; ok && !slab_done; ++it) {
         if (tile_at(it) < 0) break;
         ok = mbar_wait(&tmem_empty[a], aph ^ 1u, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(a * BN);
-        if constexpr (is_conv(EPI)) {
-          if (p.slab) {
-            for (int cs = 0; cs < 3 * p.kb_per_tap && ok; ++cs) {
-              ok = mbar_wait(slab_bar(12 + pb), pph, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
-              ok = __all_sync(0xffffffffu, ok);
-              if (!ok) break;
-              const uint32_t px = smem_u32(ring + pb * kSlabPx);
-              for (int r = 0; r < 3; ++r) {
-                ok = mbar_wait(slab_bar(s), ph, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                tc_fence_after_sync();
-                const uint64_t adesc = smem_desc_kmajor_sw128(smem_u32(ring + 2 * kSlabPx + s * C::kStageA));
-                // the window of tap row r starts r image rows (whole 1024-byte groups) into the copy
-                const uint64_t bdesc = smem_desc_kmajor_sw128(px + static_cast<uint32_t>(r * p.slab_row_bytes));
-                if (elect_one()) {
-#pragma unroll
-                  for (int k = 0; k < kBK / kUmmaK; ++k)
-                    umma_f16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (cs | r | k) != 0 ? 1u : 0u);
-                  umma_commit(slab_bar(6 + s));                   // frees the weight slot
-                  if (r == 2) umma_commit(slab_bar(12 + 2 + pb));  // ... and, after the third tap, the copy
-                }
-                if (++s == kSlabW) { s = 0; ph ^= 1u; }
-              }
-              if (++pb == 2) { pb = 0; pph ^= 1u; }
-            }
-            if (!ok) break;
-            if (elect_one()) umma_commit(&tmem_full[a]);
-            if (++a == 2) { a = 0; aph ^= 1u; }
-            continue;
-          }
-        }
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
+        for (int kb = 0; kb < p.k_blocks; kb += C::kKB) {
           ok = mbar_wait(&full[s], ph, abort_flag, p.status, KF_DEV_TIMEOUT_MMA);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after_sync();
           const uint32_t sa = smem_u32(ring + s * C::kStage);
-          const uint64_t adesc = smem_desc_kmajor_sw128(sa);
-          const uint64_t bdesc = smem_desc_kmajor_sw128(sa + C::kStageA);
+          const int kbs = min(C::kKB, p.k_blocks - kb);              // K blocks in this stage
           if (elect_one()) {
 #pragma unroll
-            for (int k = 0; k < kBK / kUmmaK; ++k) {
-              // +32 bytes per K step inside the 128-byte swizzled row = +2 in the address field
-              if constexpr (CTA2)
-                umma_f16_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-              else
-                umma_f16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            for (int j = 0; j < C::kKB; ++j) {
+              if (j < kbs) {
+                const uint64_t adesc = smem_desc_kmajor_sw128(sa + static_cast<uint32_t>(j * C::kStage1));
+                const uint64_t bdesc = smem_desc_kmajor_sw128(sa + static_cast<uint32_t>(j * C::kStage1 + C::kStageA));
+#pragma unroll
+                for (int k = 0; k < kBK / kUmmaK; ++k) {
+                  // +32 bytes per K step inside the 128-byte swizzled row = +2 in the address field
+                  if constexpr (CTA2)
+                    umma_f16_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | j | k) != 0 ? 1u : 0u);
+                  else
+                    umma_f16_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | j | k) != 0 ? 1u : 0u);
+                }
+              }
             }
             if constexpr (CTA2) umma_commit_pair(&empty[s], 3);      // frees the stage in both CTAs
             else umma_commit(&empty[s]);

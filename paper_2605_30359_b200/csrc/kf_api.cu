@@ -328,10 +328,7 @@ size_t rowreduce_part_bytes(int64_t M, int64_t N, int red) {
   // (rows rounded up to whole 128-row blocks: the one-kernel softmax lays its pairs out per block)
   return round256(static_cast<size_t>((M + kBM - 1) / kBM * kBM) * tiles_n * (softmax_like(red) ? 16 : 4));
 }
-size_t rowreduce_umma_ws(int64_t M, int64_t N, int red) {
-  // ... followed, for the softmax, by one counter per 128-row block (the one-kernel form)
-  return rowreduce_part_bytes(M, N, red) + (red == RED_SOFTMAX ? round256(static_cast<size_t>((M + kBM - 1) / kBM) * 4) : 0);
-}
+size_t rowreduce_umma_ws(int64_t M, int64_t N, int red) { return rowreduce_part_bytes(M, N, red); }
 // CTA pairs (256-row tiles, each CTA loading half of the W tile) pay off when the K loop is
 // long: measured +3.6 % at K = 4096, +3.3 % at K = 2048, -4 % at K = 1024 (fewer, larger tiles
 // make the last wave's tail longer).  KF_NO_PAIR=1 forces one CTA per tile for A/B runs.
@@ -1003,12 +1000,12 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
         if (bn == kRowReduceBN && out_dtype == KF_BF16 && p.staged && N % kRowReduceBN == 0 && p.tiles_n >= 2 &&
             p.tiles_n <= 64 && p.num_tiles >= gx_min && (K >= 2048 || tune().softmax_gx_min_tiles >= 0) &&
             !tune().no_softmax_gx) {
-          uint8_t* cnt = static_cast<uint8_t*>(workspace) + rowreduce_part_bytes(M, N, red);
-          const size_t cnt_bytes = static_cast<size_t>((M + kBM - 1) / kBM) * 4;
-          if (cudaMemsetAsync(cnt, 0, cnt_bytes, st) != cudaSuccess) return KF_ERR_CUDA;
+          // the exchange buffer, one 64-bit (maximum, sum) pair per row and tile, starts out as
+          // the pattern that means "no pair here yet"
+          const size_t gx_bytes = static_cast<size_t>((M + kBM - 1) / kBM * kBM) * p.tiles_n * 8;
+          if (cudaMemsetAsync(workspace, 0xff, gx_bytes, st) != cudaSuccess) return KF_ERR_CUDA;
           UmmaParams q = p;
           q.gx_part = reinterpret_cast<float2*>(workspace);
-          q.gx_count = reinterpret_cast<uint32_t*>(cnt);
           q.partial = nullptr;
           if (launch_umma_softmax_gx(pre_act, pair ? 1 : 0, tm, q, grid, st) == cudaSuccess) {
             g_launches += 1;

@@ -109,25 +109,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
   return true;
 }
 
-// Release / acquire on a counter in global memory at device scope: a thread that has written data
-// (and fenced) adds to the counter with release; a thread that reads the counter with acquire and
-// finds the expected value may read that data.
-__device__ __forceinline__ void red_release_gpu_add(uint32_t* addr, uint32_t v) {
-  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(addr), "r"(v) : "memory");
-}
-__device__ __forceinline__ void red_relaxed_gpu_add(uint32_t* addr, uint32_t v) {
-  asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(addr), "r"(v) : "memory");
-}
-__device__ __forceinline__ uint32_t ld_relaxed_gpu(const uint32_t* addr) {
-  uint32_t v;
-  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
-  return v;
-}
-__device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* addr) {
-  uint32_t v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
-  return v;
-}
 // A 64-bit word that is its own flag: the producer stores the datum (never the "empty" pattern the
 // buffer was filled with), a consumer that loads anything else has the datum.  Aligned 64-bit
 // accesses are single-copy atomic, so neither side needs a fence or a counter.

@@ -210,25 +210,28 @@ cudaError_t launch_pad_rows_bf16(long long rows, int K, int kp, const void* in, 
 
 cudaError_t launch_conv_prep(int Nb, int Cin, int Cp, int H, int Wd, int Cout, const void* x,
                              const void* w, void* xt, void* wr, cudaStream_t st, void* ones, size_t ones_bytes) {
-  if (ones != nullptr && ones_bytes > 0 && cudaMemsetAsync(ones, 0xff, ones_bytes, st) != cudaSuccess)
-    return cudaGetLastError();
   const __nv_bfloat16* xs = static_cast<const __nv_bfloat16*>(x);
   const __nv_bfloat16* ws = static_cast<const __nv_bfloat16*>(w);
   __nv_bfloat16* xd = static_cast<__nv_bfloat16*>(xt);
   __nv_bfloat16* wd = static_cast<__nv_bfloat16*>(wr);
+  uint4* od = static_cast<uint4*>(ones);                    // (256-byte aligned, a multiple of 256 bytes)
+  const long long ones16 = ones != nullptr ? static_cast<long long>(ones_bytes / 16) : 0;
   if (Cp == Cin && Cin % 8 == 0 && Wd % 8 == 0 && reinterpret_cast<uintptr_t>(x) % 16 == 0) {
     const long long x_blocks = static_cast<long long>(Nb) * H * (Cin / 8) * (Wd / 8);
-    const long long total = x_blocks + 9ll * Cout * Cin;
+    long long total = x_blocks + 9ll * Cout * Cin;
+    if (total < ones16) total = ones16;
     const long long grid = (total + 255) / 256;
+    if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
     conv_prep_kernel<<<static_cast<unsigned>(grid), 256, 0, st>>>(Nb, Cin, H, Wd, Cout, xs, ws, xd, wd,
-                                                                  x_blocks);
+                                                                  x_blocks, od, ones16);
   } else {
     const long long x_items = static_cast<long long>(Nb) * H * Wd * (Cp / 8);
-    const long long total = x_items + 9ll * Cout * Cp;
+    long long total = x_items + 9ll * Cout * Cp;
+    if (total < ones16) total = ones16;
     const long long grid = (total + 255) / 256;
     if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
     conv_prep_general_kernel<<<static_cast<unsigned>(grid), 256, 0, st>>>(Nb, Cin, Cp, H, Wd, Cout, xs, ws,
-                                                                          xd, wd, x_items);
+                                                                          xd, wd, x_items, od, ones16);
   }
   return cudaGetLastError();
 }

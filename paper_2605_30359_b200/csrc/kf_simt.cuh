@@ -463,8 +463,11 @@ pad_rows_bf16_kernel(long long rows, int K, int kp, const __nv_bfloat16* __restr
 __global__ void __launch_bounds__(256)
 conv_prep_kernel(int Nb, int Cin, int H, int Wd, int Cout, const __nv_bfloat16* __restrict__ x,
                  const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ xt,
-                 __nv_bfloat16* __restrict__ wr, long long x_blocks) {
+                 __nv_bfloat16* __restrict__ wr, long long x_blocks, uint4* __restrict__ ones, long long ones16) {
   const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  // (the first ones16 threads also set 16 bytes each of `ones` to all ones: the empty exchange
+  // buffer of the all-SM GroupNorm kernel, which would otherwise cost a memset of its own)
+  if (gid < ones16) ones[gid] = make_uint4(~0u, ~0u, ~0u, ~0u);
   const int wb = Wd / 8, cbk = Cin / 8;
   if (gid < x_blocks) {
     // gid -> (n, h, wblk, cblk) with cblk fastest: the lanes that hold one pixel's channel blocks
@@ -510,8 +513,9 @@ __global__ void __launch_bounds__(256)
 conv_prep_general_kernel(int Nb, int Cin, int Cp, int H, int Wd, int Cout,
                          const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
                          __nv_bfloat16* __restrict__ xt, __nv_bfloat16* __restrict__ wr,
-                         long long x_items) {
+                         long long x_items, uint4* __restrict__ ones, long long ones16) {
   const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (gid < ones16) ones[gid] = make_uint4(~0u, ~0u, ~0u, ~0u);   // (see conv_prep_kernel)
   const long long hw = static_cast<long long>(H) * Wd;
   const int cbk = Cp / 8;
   if (gid < x_items) {

@@ -124,9 +124,8 @@ struct UmmaParams {
   // (sum, sum of squares) of GroupNorm group g over pixel tile t; all bits set where no pair has
   // been stored yet (the state the kernel starts from)
   // EPI_SOFTMAX_GX: gx_part[(row block * tiles_n + t) * 128 + row] = (maximum, sum) of a row over
-  // column tile t; gx_count[row block] = tiles published (zero when the kernel starts)
+  // column tile t, the same convention
   float2* gx_part;
-  uint32_t* gx_count;
   int pool2;                   // convolution: 0, or 2x2 pooling in the epilogue (1 = max, 2 = mean);
                                // needs w_segs == 1, Wd % 32 == 0, rows_per_tile and H even
 };
@@ -559,12 +558,12 @@ __device__ __forceinline__ void conv_gnx_helper(const UmmaParams& p, float2* aux
 //   A  maximum of the row's 128 values (first pass over the accumulator), then numerators
 //      e = exp(a - maximum) and their fp32 sum (second pass); the numerators stay in registers as
 //      bf16, the accumulator goes back to the UMMA issuer; one warp merges the two groups' (maximum,
-//      sum) per row, writes the tile's 128 pairs to global memory and counts the tile in (release
-//      at device scope);
-//   B  one thread checks (acquire, bounded) that all column tiles of the row block are counted in;
-//      a thread reads its row's pairs in tile order, forms the row's maximum M and denominator
-//      S = sum s_t exp(m_t - M), scales its numerators by exp(m - M) / S and stores them through
-//      shared memory and TMA.
+//      sum) per row and stores the tile's 128 pairs to global memory, each 64-bit pair being its
+//      own "present" flag in a buffer that starts out as all ones (no counter, no fence);
+//   B  a thread loads its row's pairs of all column tiles (again, bounded, while one of them is
+//      still the empty pattern), forms the row's maximum M and denominator S = sum s_t exp(m_t - M)
+//      in tile order, scales its numerators by exp(m - M) / S and stores them through shared
+//      memory and TMA.
 // The loop is software-pipelined: A of this CTA's next tile runs before B of the current one, so
 // the other CTAs have published by the time B asks.  A only waits for this CTA's own MMAs: the
 // waits cannot form a cycle.  A wait that runs out is reported at the next go/no-go, which all
@@ -677,18 +676,20 @@ __device__ __forceinline__ void softmax_gx_epilogue(const UmmaParams& p, const C
     part[grp * kBM + row] = make_float2(mx, se + so);
     if (warp == 2) {
       // the combiner: once all eight warps have arrived, the two groups' pairs merged per row go to
-      // global memory as 128 pairs (four coalesced stores per lane), and the tile is counted in
+      // global memory as 128 pairs (four coalesced stores per lane)
       named_barrier_sync(10u, kGroups * kEpiThreads);
-      float2* dst = p.gx_part + (static_cast<long long>(t.rb) * tiles_n + t.tn) * kBM;
+      uint64_t* dst = reinterpret_cast<uint64_t*>(p.gx_part) + (static_cast<long long>(t.rb) * tiles_n + t.tn) * kBM;
 #pragma unroll
       for (int i = 0; i < kBM / 32; ++i) {
         const int r = i * 32 + lane;
         const float2 q0 = part[r], q1 = part[kBM + r];
         const float m = fmaxf(q0.x, q1.x);
-        dst[r] = make_float2(m, q0.y * exp2_approx((q0.x - m) * kLog2e) + q1.y * exp2_approx((q1.x - m) * kLog2e));
+        const float sm = q0.y * exp2_approx((q0.x - m) * kLog2e) + q1.y * exp2_approx((q1.x - m) * kLog2e);
+        // the pair is its own "present" flag (see st_relaxed_gpu_b64): no counter and no fence
+        uint64_t bits = (static_cast<uint64_t>(__float_as_uint(sm)) << 32) | __float_as_uint(m);
+        if (bits == kGxEmpty) bits = 0x7fffffff7fffffffull;
+        st_relaxed_gpu_b64(dst + r, bits);
       }
-      __syncwarp();
-      if (lane == 0) red_release_gpu_add(p.gx_count + t.rb, 1u);
     } else {
       __threadfence_block();
       named_barrier_arrive(10u, kGroups * kEpiThreads);
@@ -698,43 +699,47 @@ __device__ __forceinline__ void softmax_gx_epilogue(const UmmaParams& p, const C
 
   auto phase_b = [&](int it, const uint32_t (&st)[PIECES * 16], float mx) {
     const Tile t = locate(it);
-    bool in = true;
-    if (leader) {
-      const uint64_t t0 = globaltimer_ns();
-      uint32_t spins = 0;
-      while (ld_acquire_gpu(p.gx_count + t.rb) < static_cast<uint32_t>(tiles_n)) {
-        __nanosleep(100);
-        if ((++spins & 15u) == 0u) {
-          if (*abort_flag) { in = false; break; }
-          if (globaltimer_ns() - t0 > kWaitLimitNs) {
-            *abort_flag = 1u;
-            atomicOr(p.status, KF_DEV_TIMEOUT_EPILOGUE);
-            in = false;
-            break;
-          }
-        }
-      }
-    }
-    in = named_barrier_and(11u, kGroups * kEpiThreads, in);
-    if (!in) failed = true;                  // the status word has it; finish the tile with the others
-    // the row's maximum and denominator from the tiles' pairs, in tile order (sixteen loads in flight)
+    // the row's maximum and denominator from the tiles' pairs, in tile order (sixteen loads in
+    // flight); a pair that is still the "empty" pattern sends the thread round again (bounded)
     float M = -INFINITY, S = 0.0f;
     {
-      const float2* gp = p.gx_part + static_cast<long long>(t.rb) * tiles_n * kBM + row;
-      for (int t0 = 0; t0 < tiles_n; t0 += 16) {
-        float2 q[16];
+      const uint64_t* gp = reinterpret_cast<const uint64_t*>(p.gx_part) + static_cast<long long>(t.rb) * tiles_n * kBM + row;
+      uint64_t t_start = 0;
+      uint32_t spins = 0;
+      int t0 = 0;
+      while (t0 < tiles_n) {
+        uint64_t q[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i)
-          q[i] = (in && t0 + i < tiles_n) ? __ldcg(gp + static_cast<long long>(t0 + i) * kBM) : make_float2(-INFINITY, 0.0f);
+          q[i] = (t0 + i < tiles_n) ? ld_relaxed_gpu_b64(gp + static_cast<long long>(t0 + i) * kBM) : 0xff800000ull;   // (-inf, 0)
+        bool all = true;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) all = all && q[i] != kGxEmpty;
+        if (!all && !failed) {
+          __nanosleep(100);
+          if ((++spins & 15u) == 0u) {
+            if (t_start == 0) t_start = globaltimer_ns();
+            if (*abort_flag) failed = true;
+            else if (globaltimer_ns() - t_start > kWaitLimitNs) {
+              *abort_flag = 1u;
+              atomicOr(p.status, KF_DEV_TIMEOUT_EPILOGUE);
+              failed = true;              // the status word has it; finish the tile with the others
+            }
+          }
+          continue;
+        }
         float bm = M;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) bm = fmaxf(bm, q[i].x);
+        for (int i = 0; i < 16; ++i) bm = fmaxf(bm, __uint_as_float(static_cast<uint32_t>(q[i])));
         if (bm > -INFINITY) {
           S *= exp2_approx((M - bm) * kLog2e);
 #pragma unroll
-          for (int i = 0; i < 16; ++i) S += q[i].y * exp2_approx((q[i].x - bm) * kLog2e);
+          for (int i = 0; i < 16; ++i)
+            S += __uint_as_float(static_cast<uint32_t>(q[i] >> 32)) *
+                 exp2_approx((__uint_as_float(static_cast<uint32_t>(q[i])) - bm) * kLog2e);
           M = bm;
         }
+        t0 += 16;
       }
     }
     const float scale = exp2_approx((mx - M) * kLog2e) / S;

@@ -35,7 +35,7 @@ def test_host_queries(lib):
     assert "workspace" in kf.status_string(kf.KF_ERR_WORKSPACE)
     assert kf.kf_gemm_epilogue_workspace_bytes(8192, 4096, 4096, kf.KF_BF16) == 0
     # softmax first pass: (max, sum) per row and 256-column tile
-    assert kf.kf_gemm_rowreduce_workspace_bytes(4096, 8192, 2048, kf.KF_BF16, 0) == 4096 * 64 * 8 + 256   # (max, sum) per half tile + a counter per row block
+    assert kf.kf_gemm_rowreduce_workspace_bytes(4096, 8192, 2048, kf.KF_BF16, 0) == 4096 * 64 * 8   # (max, sum) per half tile
     assert kf.kf_gemm_rowreduce_workspace_bytes(16384, 1024, 1024, kf.KF_BF16, 1) == 16384 * 4 * 4
     # fp32 chains stage the pre-reduction values
     assert kf.kf_gemm_rowreduce_workspace_bytes(128, 256, 512, kf.KF_F32, 0) == 128 * 256 * 4

@@ -176,7 +176,7 @@ struct UmmaCfg {
   // stage it needed about 600 cycles per block against the tensor pipe's 512 (256 at 128-column
   // tiles), and the pipe's short queue ran dry.
   static constexpr int kBudget = kMaxDynSmem - 1024 - kStaging - kBarBytes - kBiasBytes - kInboxBytes;
-  static constexpr int kKB = (!is_conv(EPI) && kBudget / (2 * kStage1) >= 3) ? 2 : 1;
+  static constexpr int kKB = (!is_conv(EPI) && !CTA2 && kBudget / (2 * kStage1) >= 3) ? 2 : 1;
   static constexpr int kStage = kKB * kStage1;
   static constexpr int kFit = kBudget / kStage;
   static constexpr int kStages = kFit > 8 ? 8 : kFit;

@@ -538,7 +538,7 @@ def test_gemm_groupnorm(kf, dtype, shape, groups, tuning):
     ((1000, 1024, 256), "none"),        # 8 row blocks x 4 tiles, ragged last row block
     ((640, 2048, 128), "gelu_tanh"),    # a pre-activation; 5 x 8 tiles
     ((256, 16384, 64), "none"),         # 64 tiles per row: two rounds of the schedule per row block
-    ((40000, 512, 64), "none"),         # 313 row blocks x 2 tiles: many rounds, counters of many blocks
+    ((40000, 512, 64), "none"),         # 313 row blocks x 2 tiles: many rounds, exchange rows of many blocks
     ((1536, 1024, 2048), "none"),       # CTA pairs (K = 2048): 256-row tiles, both CTAs publish their own rows
     ((700, 768, 2112), "relu"),         # CTA pairs, ragged last pair (rows 512..699), 33 K blocks
 ])
@@ -557,6 +557,39 @@ def test_bf16_softmax_wide_rows_one_kernel(kf, shape, act, tuning):
     assert np.abs(got.sum(axis=1) - 1.0).max() < 4e-3
     P2 = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), act, "softmax")
     assert (to_f64(P2) == got).all()                          # fixed order of the exchange: bit-identical repeats
+
+
+def _softmax_gx_fuzz_cases():
+    rng = np.random.default_rng(20261126)
+    cases = []
+    while len(cases) < 6:
+        M = int(rng.integers(100, 9000))
+        N = 256 * int(rng.integers(2, 11))
+        K = 8 * int(rng.integers(8, 280))                  # 64..2232: both the single-CTA form and CTA pairs
+        # (problems of one wave of 256-column tiles take 64-column tiles and another route)
+        if M * N * K > 6e9 or ((M + 127) // 128) * (N // 256) <= 160:
+            continue
+        cases.append((M, N, K))
+    return cases
+
+
+@pytest.mark.parametrize("shape", _softmax_gx_fuzz_cases())
+def test_bf16_softmax_wide_rows_one_kernel_seeded_shapes(kf, shape, tuning):
+    M, N, K = shape
+    d = ki.gemm_inputs("c3", seed=29, M=M, N=N, K=K)
+    tuning.setenv("KF_SOFTMAX_GX_MIN_TILES", "1")
+    before = kf.kf_launch_count()
+    P = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "none", "softmax")
+    check_status()
+    assert kf.kf_launch_count() - before == 1                # the one-kernel route was taken
+    got = to_f64(P)
+    ref = oracle.gemm_rowreduce(d["X"], d["W"], d["b"], "none", "softmax")
+    assert_close(got, ref, 2e-2, 2e-2, "softmax one kernel, seeded shape %s" % (shape,))
+    assert_close(got, ref, 1e-7, 2e-2, "softmax one kernel, seeded shape, relative %s" % (shape,))
+    # the two-kernel route on the same inputs
+    tuning.setenv("KF_NO_SOFTMAX_GX", "1")
+    P2 = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), "none", "softmax")
+    assert_close(to_f64(P2), got, 1e-7, 2e-2, "softmax one kernel against two kernels %s" % (shape,))
 
 
 # Rows that lie in one tile (N <= 256, or <= 64 on the narrow-tile kernel): the softmax is finished
@@ -849,6 +882,38 @@ def test_conv_groupnorm_all_sm_kernel(kf, cfg, tuning):
     tuning.setenv("KF_NO_FUSED_GN", "1")
     two, ref = run_conv(kf, d)
     assert (np.abs(fused - two) <= 2.0 ** -7 * np.maximum(1.0, np.abs(two))).all()      # two bf16 ulps
+
+
+def _gnx_fuzz_cases():
+    # seeded shapes the all-SM kernel accepts when forced: widths whose tiles are whole 32-pixel
+    # pieces, groups of 4 / 8 / 16 / 32 channels, any number of rows, images and channel tiles
+    rng = np.random.default_rng(20261125)
+    cases = []
+    while len(cases) < 10:
+        W = int(rng.choice([16, 32, 64, 128, 8, 24, 40, 56]))
+        H = int(rng.integers(3, 41))
+        Cin = int(rng.choice([16, 32, 64, 128]))
+        cpg = int(rng.choice([4, 8, 16, 32]))
+        groups = int(rng.integers(1, 9))
+        Cout = cpg * groups
+        Nb = int(rng.integers(1, 8))
+        if Nb * H * W * Cout * Cin * 9 > 3e8:
+            continue
+        cases.append(dict(Nb=Nb, Cin=Cin, H=H, W=W, Cout=Cout, groups=groups))
+    return cases
+
+
+@pytest.mark.parametrize("cfg", _gnx_fuzz_cases())
+def test_conv_groupnorm_all_sm_kernel_seeded_shapes(kf, cfg, tuning):
+    d = ki.conv_inputs(seed=41, dtype="bf16", **cfg)
+    tuning.setenv("KF_GNX_MIN_TILES", "1")
+    tuning.setenv("KF_GNX_MIN_TPI", "1")
+    got, ref = run_conv(kf, d, act="swish")
+    assert_close(got, ref, 2e-2, 2e-2, "conv GN all SMs, seeded shape %s" % (cfg,))
+    # the other routes (cluster or two kernels) on the same inputs agree to two bf16 ulps
+    tuning.setenv("KF_NO_GNX", "1")
+    other, _ = run_conv(kf, d, act="swish")
+    assert (np.abs(got - other) <= 2.0 ** -7 * np.maximum(1.0, np.abs(other))).all()
 
 
 # ------------------------------------------------------------------ conv -> activation -> global average pool

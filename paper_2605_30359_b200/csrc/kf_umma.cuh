@@ -1731,7 +1731,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 bulk_copy_to_peer(mapa_shared(dst, r), smem_u32(sbuf), 256u, mapa_shared(smem_u32(&rbar[buf]), r));
             }
           }
-          // every thread waits itself (it reads what the copies wrote), then one verdict for all
+          // every thread waits itself (it reads what the copies wrote), then one decision for all
           bool all_in = mbar_wait(&rbar[buf], static_cast<uint32_t>((it >> 1) & 1), abort_flag, p.status,
                                   KF_DEV_TIMEOUT_EPILOGUE);
           all_in = named_barrier_and(bar_a, kEpiThreads, all_in);

@@ -149,7 +149,11 @@ size_t kf_gemm_groupnorm_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dty
  * leaves numerators and per-tile (max, sum), then a rescaling kernel; rows that lie in one tile,
  * or in up to 16 tiles of 64 columns or up to 8 tiles of 128 columns (small problems; their CTAs
  * form a cluster and exchange the pairs through distributed shared memory), are finished by the
- * GEMM kernel alone. */
+ * GEMM kernel alone.  So are rows of 2..64 whole 256-column tiles on problems of at least two waves
+ * with K >= 2048 (bf16 out, TMA-storable out): the tiles of a row block sit on neighbouring CTAs of
+ * one cooperative launch, which exchange the per-row (max, sum) pairs through the workspace and
+ * write final probabilities; no numerators reach memory.  A device that cannot hold that grid at
+ * once takes the two-kernel route. */
 kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype,
                             const void* X, int64_t ldx, const void* W, int64_t ldw,
                             const void* bias, kf_act pre_act, kf_rowred red,
@@ -206,6 +210,9 @@ kf_status kf_gemm_rowreduce_static(int64_t M, int64_t N, int64_t K, kf_dtype in_
  * (bf16, 16-byte aligned y, H*Wd % 8 == 0) the CTAs of an image (and channel tile) form a
  * cluster, exchange the statistics through distributed shared memory and normalise inside the
  * convolution kernel: one kernel after the NHWC copy, the activations are written once.
+ * Images of 9..64 whole tiles on problems of at least two waves (same conditions otherwise) run
+ * the same chain on every SM: one cooperative launch whose neighbouring CTAs hold an image's
+ * tiles and exchange the group statistics through the workspace.
  * groups must divide Cout. */
 kf_status kf_conv3x3_epilogue(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, int64_t Cout,
                               kf_dtype io_dtype, const void* x, const void* w, const void* bias,

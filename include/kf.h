@@ -338,7 +338,8 @@ int64_t kf_launch_count(void);
 
 /* Host-side state of the call path (no counterpart in the paper: library plumbing).
  * The dispatch switches (KF_NO_PAIR, KF_NO_SPLITK, KF_NO_FUSED_GN, KF_NO_FUSED_SOFTMAX,
- * KF_NO_CLUSTER_SOFTMAX, KF_NO_FUSED_POOL, KF_NO_TF32X3, KF_NO_CONV_SLAB, KF_NO_GNX, KF_NO_SOFTMAX_GX) and thresholds
+ * KF_NO_CLUSTER_SOFTMAX, KF_NO_FUSED_POOL, KF_NO_TF32X3, KF_NO_CONV_SLAB, KF_NO_GNX, KF_NO_SOFTMAX_GX,
+ * KF_NO_WIDE_STORE) and thresholds
  * (KF_PAIR_MIN_K, KF_PAIR_MIN_KB_PER_CTA, KF_SPLITK_MIN_KB, KF_SPLITK_TWO_PER_SM, KF_CL128_MAX_CTAS,
  * KF_GNX_MIN_TILES, KF_GNX_MIN_TPI, KF_GNX_MAX_TPI, KF_SOFTMAX_GX_MIN_TILES) are read
  * from the environment once, at the first call; kf_reload_tuning() reads them again (tests

@@ -19,7 +19,7 @@ std::atomic<int64_t> g_launches{0};
 // to move a threshold); the environment is read ONCE, at the first call, and again only when
 // kf_reload_tuning() is called, so a call on the hot path reads no environment variable.
 struct Tuning {
-  bool no_fused_pool, no_tf32x3, no_splitk, no_pair, no_cluster_softmax, no_fused_softmax, no_fused_gn, no_conv_slab, no_gnx, no_softmax_gx;
+  bool no_fused_pool, no_tf32x3, no_splitk, no_pair, no_cluster_softmax, no_fused_softmax, no_fused_gn, no_conv_slab, no_gnx, no_softmax_gx, no_wide_store;
   int splitk_min_kb, splitk_two_per_sm, pair_min_k, pair_min_kb_per_cta, cl128_max_ctas;
   int softmax_gx_min_tiles;                        // one-kernel softmax of wide rows: tiles in all (-1: two waves)
   int gnx_min_tiles, gnx_min_tpi, gnx_max_tpi;     // all-SM GroupNorm convolution: tiles in all (-1: two waves), tiles per image
@@ -43,6 +43,7 @@ void load_tuning_locked() {
   g_tune.no_conv_slab = flag("KF_NO_CONV_SLAB");
   g_tune.no_gnx = flag("KF_NO_GNX");
   g_tune.no_softmax_gx = flag("KF_NO_SOFTMAX_GX");
+  g_tune.no_wide_store = flag("KF_NO_WIDE_STORE");
   g_tune.softmax_gx_min_tiles = num("KF_SOFTMAX_GX_MIN_TILES", -1);
   g_tune.splitk_min_kb = num("KF_SPLITK_MIN_KB", 28);
   g_tune.splitk_two_per_sm = num("KF_SPLITK_TWO_PER_SM", 1);
@@ -218,6 +219,16 @@ bool encode_nhwc(CUtensorMap* tm, const void* base, int64_t Nb, int64_t H, int64
 
 // NCHW bf16 output seen as [Nb][C][H*W] -> store boxes of 32 pixels x 32 channels of one image
 // (64-byte swizzle like every epilogue piece); channels past C are clipped.
+// ... and boxes of 64 pixels x 32 channels (128-byte rows, 128-byte swizzle)
+bool encode_nchw_out_wide(CUtensorMap* tm, const void* base, int64_t Nb, int64_t C, int64_t hw) {
+  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(hw), static_cast<cuuint64_t>(C),
+                              static_cast<cuuint64_t>(Nb)};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(hw) * 2,
+                                 static_cast<cuuint64_t>(C) * hw * 2};
+  const cuuint32_t box[3] = {64, 32, 1};
+  return encode_generic(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box,
+                        CU_TENSOR_MAP_SWIZZLE_128B);
+}
 bool encode_nchw_out(CUtensorMap* tm, const void* base, int64_t Nb, int64_t C, int64_t hw) {
   const cuuint64_t dims[3] = {static_cast<cuuint64_t>(hw), static_cast<cuuint64_t>(C),
                               static_cast<cuuint64_t>(Nb)};
@@ -1226,8 +1237,13 @@ static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
       q.gn_beta = static_cast<const __nv_bfloat16*>(beta);
       q.partial = nullptr;
       q.gx_part = reinterpret_cast<float2*>(stats);
+      UmmaMaps tq = tm;
+      if (q.slab && !tune().no_wide_store) {       // slab mode does not use the per-tap map: it carries the wide store map
+        if (!encode_nchw_out_wide(&tq.b, y, Nb, Cout, hw)) return KF_ERR_CUDA;
+        q.y_wide = 1;
+      }
       const int gridx = q.num_tiles < d->sm_count ? q.num_tiles : d->sm_count;
-      if (launch_umma_conv_gnx(bn, act, tm, q, gridx, st) == cudaSuccess) {
+      if (launch_umma_conv_gnx(bn, act, tq, q, gridx, st) == cudaSuccess) {
         g_launches += launches + 1;
         return KF_OK;
       }

@@ -126,6 +126,7 @@ struct UmmaParams {
   // EPI_SOFTMAX_GX: gx_part[(row block * tiles_n + t) * 128 + row] = (maximum, sum) of a row over
   // column tile t, the same convention
   float2* gx_part;
+  int y_wide;                  // EPI_CONV_GNX in slab mode: tmB is a store map of 64 pixels x 32 channels (128-byte swizzle)
   int pool2;                   // convolution: 0, or 2x2 pooling in the epilogue (1 = max, 2 = mean);
                                // needs w_segs == 1, Wd % 32 == 0, rows_per_tile and H even
 };
@@ -157,7 +158,7 @@ struct UmmaCfg {
   // staging: elementwise = 2 output + 2 residual pieces; softmax = 2 output pieces per epilogue
   // group; conv = 2 output pieces
   static constexpr int kStaging =
-      EPI == EPI_ELEMENTWISE || is_softmax(EPI) ? 4 * kPieceBytes      // (EPI_SOFTMAX_GX: one piece per group, below)
+      EPI == EPI_ELEMENTWISE || is_softmax(EPI) || EPI == EPI_CONV_GNX ? 4 * kPieceBytes      // (EPI_SOFTMAX_GX: one piece per group, below; EPI_CONV_GNX: a 4 KB slab per epilogue warp)
                                                     : (EPI == EPI_ROWSUM ? 0 : 2 * kPieceBytes);     // EPI_CONV_GN: one piece per epilogue group
   static constexpr int kBarBytes = 256;
   // GEMM epilogues: the tile's BN bias values as fp32, staged once per tile
@@ -269,7 +270,8 @@ __device__ __forceinline__ void load_sbias32(const float* sb, float (&b)[32]) {
 // that runs out is reported at the next go/no-go, which all eight warps take together.
 // ---------------------------------------------------------------------------------------------
 template <int BN, int ACT, typename TileAt>
-__device__ __forceinline__ void conv_gnx_epilogue(const UmmaParams& p, const CUtensorMap* tmY, uint8_t* stg,
+__device__ __forceinline__ void conv_gnx_epilogue(const UmmaParams& p, const CUtensorMap* tmY,
+                                                  const CUtensorMap* tmYw, uint8_t* stg,
                                                   float2* aux, uint64_t* tmem_full, uint64_t* tmem_empty,
                                                   uint64_t* gx_parts, uint64_t* gx_stats,
                                                   volatile uint32_t* abort_flag, uint32_t tmem_base,
@@ -290,7 +292,7 @@ __device__ __forceinline__ void conv_gnx_epilogue(const UmmaParams& p, const CUt
   const int piece0 = grp * kGP;
   const int my_pieces = max(0, min(kGP, pieces - piece0));
   const int tpi = p.tiles_per_image;
-  uint8_t* yslab = stg + grp * kPieceBytes;             // the group's staging piece (a 2 KB slab per warp)
+  uint8_t* wslab = stg + (grp * 4 + quad) * 4096;       // this warp's staging slab (4 KB; the 32-pixel form uses half)
   bool failed = false;                                  // one of this thread's waits ran out
 
   struct Tile { int tm, img, pt, unit, px0, px_valid; float bias_v, ga, be; };
@@ -413,6 +415,35 @@ __device__ __forceinline__ void conv_gnx_epilogue(const UmmaParams& p, const CUt
     const float sc = ms.y * t.ga;
     const float sh = fmaf(-ms.x, sc, t.be);
     const uint64_t sc2 = f32x2_pack(sc, sc), sh2 = f32x2_pack(sh, sh);
+    if (p.y_wide && my_pieces == kGP && t.px_valid >= (piece0 + kGP) * 32) {
+      // whole shares leave in slabs of 64 pixels x 32 channels (128-byte rows, 128-byte swizzle):
+      // half as many waits for the slab, fences and store issues as with 32-pixel slabs
+#pragma unroll
+      for (int c2 = 0; c2 < kGP / 2; ++c2) {
+        uint32_t w[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const uint32_t u = st[c2 * 32 + j];
+          float y0, y1;
+          f32x2_unpack(f32x2_fma(f32x2_pack(bf16_lo(u), bf16_hi(u)), sc2, sh2), y0, y1);
+          w[j] = pack_bf16x2(y0, y1);
+        }
+        bulk_wait_group_read<0>();       // this warp's previous store has let go of the slab
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          *reinterpret_cast<uint4*>(wslab + lane * 128 + ((q ^ (lane & 7)) << 4)) =
+              make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (elect_one()) {
+          if (t.tm * kBM + quad * 32 < p.N)
+            tma_store_3d(tmYw, wslab, t.px0 + (piece0 + 2 * c2) * 32, t.tm * kBM + quad * 32, t.img);
+          bulk_commit_group();
+        }
+      }
+      return;
+    }
 #pragma unroll
     for (int c = 0; c < kGP; ++c) {
       if (c < my_pieces) {
@@ -428,14 +459,14 @@ __device__ __forceinline__ void conv_gnx_epilogue(const UmmaParams& p, const CUt
         __syncwarp();
 #pragma unroll
         for (int q = 0; q < 4; ++q)
-          *reinterpret_cast<uint4*>(yslab + piece_off(row, q)) =
+          *reinterpret_cast<uint4*>(wslab + piece_off(lane, q)) =
               make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
         fence_proxy_async_smem();
         __syncwarp();
         if (elect_one()) {
           const int px = (piece0 + c) * 32;               // first pixel of the piece inside the tile
           if (t.px_valid - px > 0 && t.tm * kBM + quad * 32 < p.N)
-            tma_store_3d(tmY, yslab + quad * (kPieceBytes / 4), t.px0 + px, t.tm * kBM + quad * 32, t.img);
+            tma_store_3d(tmY, wslab, t.px0 + px, t.tm * kBM + quad * 32, t.img);
           bulk_commit_group();
         }
       }
@@ -1109,7 +1140,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                                          abort_flag, tmem_base, rank, warp, lane, my_tiles, tile_at);
     } else if constexpr (EPI == EPI_CONV_GNX) {
       const int my_tiles = cta < p.num_tiles ? (p.num_tiles - cta + ncta - 1) / ncta : 0;
-      conv_gnx_epilogue<BN, ACT>(p, &tmY, stg, reinterpret_cast<float2*>(stg + C::kStaging + C::kBarBytes),
+      conv_gnx_epilogue<BN, ACT>(p, &tmY, &tmB, stg, reinterpret_cast<float2*>(stg + C::kStaging + C::kBarBytes),
                                  tmem_full, tmem_empty, gx_parts, gx_stats, abort_flag, tmem_base, warp, lane,
                                  my_tiles, tile_at);
     } else {

@@ -876,6 +876,12 @@ def test_conv_groupnorm_all_sm_kernel(kf, cfg, tuning):
     assert kf.kf_launch_count() - before == 4               # prepass + one kernel per call: the route was taken
     again, _ = run_conv(kf, d, act="mish", gamma=gamma, beta=beta)
     assert (again == got).all()                              # fixed summation order: repeat runs are bit-identical
+    # whole shares leave in 64-pixel slabs where the mainloop's mode frees a tensor map for them;
+    # the 32-pixel form stores the same bits
+    tuning.setenv("KF_NO_WIDE_STORE", "1")
+    narrow, _ = run_conv(kf, d, act="mish", gamma=gamma, beta=beta)
+    assert (narrow == got).all()
+    tuning.delenv("KF_NO_WIDE_STORE")
     # the two-kernel route on the same inputs: same statistics, activations rounded to bf16
     # before instead of after the normalisation
     fused, _ = run_conv(kf, d)

@@ -1267,6 +1267,10 @@ static kf_status conv3x3_impl(int64_t Nb, int64_t Cin, int64_t H, int64_t Wd, in
       p.num_tiles = p.tiles_m * p.tiles_n;
     }
     const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
+    if (p.slab && p.staged && !tune().no_wide_store) {   // slab mode does not use the per-tap map: it carries the wide store map
+      if (!encode_nchw_out_wide(&tm.b, y, Nb, Cout, hw)) return KF_ERR_CUDA;
+      p.y_wide = 1;
+    }
     if (launch_umma_conv(bn, act, tm, p, grid, st) != cudaSuccess) return KF_ERR_CUDA;
     ++launches;
     if (gap_in_epilogue) {

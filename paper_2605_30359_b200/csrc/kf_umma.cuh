@@ -158,7 +158,7 @@ struct UmmaCfg {
   // staging: elementwise = 2 output + 2 residual pieces; softmax = 2 output pieces per epilogue
   // group; conv = 2 output pieces
   static constexpr int kStaging =
-      EPI == EPI_ELEMENTWISE || is_softmax(EPI) || EPI == EPI_CONV_GNX ? 4 * kPieceBytes      // (EPI_SOFTMAX_GX: one piece per group, below; EPI_CONV_GNX: a 4 KB slab per epilogue warp)
+      EPI == EPI_ELEMENTWISE || is_softmax(EPI) || EPI == EPI_CONV_GNX || EPI == EPI_CONV ? 4 * kPieceBytes      // (EPI_SOFTMAX_GX: one piece per group, below; EPI_CONV_GNX: a 4 KB slab per epilogue warp; EPI_CONV: two)
                                                     : (EPI == EPI_ROWSUM ? 0 : 2 * kPieceBytes);     // EPI_CONV_GN: one piece per epilogue group
   static constexpr int kBarBytes = 256;
   // GEMM epilogues: the tile's BN bias values as fp32, staged once per tile
@@ -1872,8 +1872,54 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (++a == 2) { a = 0; aph ^= 1u; }
           continue;
         }
+        int c = 0;
+        if constexpr (EPI == EPI_CONV) {
+          // whole pairs of pieces leave as slabs of 64 pixels x 32 channels (128-byte rows,
+          // 128-byte swizzle, the store map in tmB, which slab mode does not use): half as many
+          // waits for the slab, fences and store issues
+          if (staged && p.y_wide && p.stats_only == 0) {
 #pragma unroll 1
-        for (int c = 0; c < pieces; ++c, ++g) {
+            for (; c + 2 <= pieces && px_valid - c * 32 >= 64; c += 2, ++g) {
+              uint32_t w[32];
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                uint32_t v[32];
+                tmem_ld_32x32(t_acc + (c + h) * 32, v);
+                tmem_ld_wait();
+                if (h == 1 && c + 2 == pieces) release_acc();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                  float y0, y1;
+                  f32x2_unpack(f32x2_add(f32x2_pack(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])), bias2), y0, y1);
+                  y0 = act_f<ACT, true>(y0, p.act_rt);
+                  y1 = act_f<ACT, true>(y1, p.act_rt);
+                  w[h * 16 + j] = pack_bf16x2(y0, y1);
+                  if (want_stats) {
+                    const uint64_t y = f32x2_pack(y0, y1);
+                    s1p = f32x2_add(s1p, y);
+                    s2p = f32x2_fma(y, y, s2p);
+                  }
+                }
+              }
+              uint8_t* yw = stg + ((static_cast<int>(g & 1)) * 4 + quad) * 4096;
+              bulk_wait_group_read<1>();     // the store from this buffer two slabs ago has let go
+              __syncwarp();
+#pragma unroll
+              for (int q = 0; q < 8; ++q)
+                *reinterpret_cast<uint4*>(yw + lane * 128 + ((q ^ (lane & 7)) << 4)) =
+                    make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+              fence_proxy_async_smem();
+              __syncwarp();
+              if (elect_one()) {
+                if (tm * kBM + quad * 32 < p.N)
+                  tma_store_3d(&tmB, yw, px0 + c * 32, tm * kBM + quad * 32, img);
+                bulk_commit_group();
+              }
+            }
+          }
+        }
+#pragma unroll 1
+        for (; c < pieces; ++c, ++g) {
           uint32_t v[32];
           tmem_ld_32x32(t_acc + c * 32, v);
           tmem_ld_wait();
@@ -1919,20 +1965,22 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (staged) {
             // every warp stages and stores its own 32 channels of the piece (2 KB slab, TMA box
             // of 32 pixels x 32 channels): no barrier between the warps
-            const int b = static_cast<int>(g & 1);
-            uint8_t* yb = ybuf + b * kPieceBytes;
+            // (two buffers of a 4 KB slab per warp, shared with the 64-pixel form above, which
+            // uses all of a slab: the 32-pixel form uses its first half)
+            constexpr int kWarpSlab = EPI == EPI_CONV ? 4096 : 2048;   // (only EPI_CONV has room for the wide form)
+            uint8_t* yb = stg + ((static_cast<int>(g & 1)) * 4 + quad) * kWarpSlab;
             bulk_wait_group_read<1>();       // the store from this buffer two pieces ago has let go
             __syncwarp();
 #pragma unroll
             for (int q = 0; q < 4; ++q)
-              *reinterpret_cast<uint4*>(yb + piece_off(row, q)) =
+              *reinterpret_cast<uint4*>(yb + piece_off(lane, q)) =
                   make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
             fence_proxy_async_smem();
             __syncwarp();
             if (elect_one()) {
               // channels past Cout and pixels past the image are clipped
               if (left > 0 && tm * kBM + quad * 32 < p.N)
-                tma_store_3d(&tmY, yb + quad * (kPieceBytes / 4), px0 + c * 32, tm * kBM + quad * 32, img);
+                tma_store_3d(&tmY, yb, px0 + c * 32, tm * kBM + quad * 32, img);
               bulk_commit_group();
             }
           } else {

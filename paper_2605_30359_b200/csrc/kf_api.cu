@@ -1018,7 +1018,12 @@ kf_status kf_gemm_rowreduce(int64_t M, int64_t N, int64_t K, kf_dtype in_dtype, 
           UmmaParams q = p;
           q.gx_part = reinterpret_cast<float2*>(workspace);
           q.partial = nullptr;
-          if (launch_umma_softmax_gx(pre_act, pair ? 1 : 0, tm, q, grid, st) == cudaSuccess) {
+          UmmaMaps tq = tm;
+          if (!tune().no_wide_store) {       // per-warp store slabs of 32 rows x 32 columns (the residual map's place)
+            if (!encode_warp_piece(&tq.r, out, M, N, ldo)) return KF_ERR_CUDA;
+            q.y_wide = 1;
+          }
+          if (launch_umma_softmax_gx(pre_act, pair ? 1 : 0, tq, q, grid, st) == cudaSuccess) {
             g_launches += 1;
             return KF_OK;
           }

@@ -601,7 +601,8 @@ __device__ __forceinline__ void conv_gnx_helper(const UmmaParams& p, float2* aux
 // eight warps take together.  Whole 256-column tiles only (N a multiple of 256).
 // ---------------------------------------------------------------------------------------------
 template <int BN, int ACT, bool CTA2, typename TileAt>
-__device__ __forceinline__ void softmax_gx_epilogue(const UmmaParams& p, const CUtensorMap* tmY, uint8_t* stg,
+__device__ __forceinline__ void softmax_gx_epilogue(const UmmaParams& p, const CUtensorMap* tmY,
+                                                    const CUtensorMap* tmYw, uint8_t* stg,
                                                     float* sbias_all, float2* part, uint64_t* tmem_full,
                                                     uint64_t* tmem_empty, volatile uint32_t* abort_flag,
                                                     uint32_t tmem_base, uint32_t rank, int warp, int lane,
@@ -775,6 +776,36 @@ __device__ __forceinline__ void softmax_gx_epilogue(const UmmaParams& p, const C
     }
     const float scale = exp2_approx((mx - M) * kLog2e) / S;
     const uint64_t sc2 = f32x2_pack(scale, scale);
+    if (p.y_wide) {
+      // every warp stages and stores its own 32 rows of a piece (2 KB slab, the store map in tmR):
+      // no barrier between the warps of a group
+      uint8_t* wslab = stg + (grp * 4 + quad) * 2048;
+#pragma unroll
+      for (int c = 0; c < PIECES; ++c) {
+        uint32_t w[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const uint32_t u = st[c * 16 + j];
+          float y0, y1;
+          f32x2_unpack(f32x2_mul(f32x2_pack(bf16_lo(u), bf16_hi(u)), sc2), y0, y1);
+          w[j] = pack_bf16x2(y0, y1);
+        }
+        bulk_wait_group_read<0>();       // this warp's previous store has let go of the slab
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          *reinterpret_cast<uint4*>(wslab + piece_off(lane, q)) =
+              make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (elect_one()) {
+          if (t.m_cta + quad * 32 < p.M)
+            tma_store_2d(tmYw, wslab, t.tn * BN + grp * kGroupCols + c * kPieceCols, t.m_cta + quad * 32);   // clipped at M
+          bulk_commit_group();
+        }
+      }
+      return;
+    }
 #pragma unroll
     for (int c = 0; c < PIECES; ++c) {
       uint32_t w[16];
@@ -1136,7 +1167,7 @@ umma_chain_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     if constexpr (EPI == EPI_SOFTMAX_GX) {
       const int my_tiles = cta < p.num_tiles ? (p.num_tiles - cta + ncta - 1) / ncta : 0;
       float* sb = reinterpret_cast<float*>(stg + C::kStaging + C::kBarBytes);
-      softmax_gx_epilogue<BN, ACT, CTA2>(p, &tmY, stg, sb, reinterpret_cast<float2*>(sb + BN), tmem_full, tmem_empty,
+      softmax_gx_epilogue<BN, ACT, CTA2>(p, &tmY, &tmR, stg, sb, reinterpret_cast<float2*>(sb + BN), tmem_full, tmem_empty,
                                          abort_flag, tmem_base, rank, warp, lane, my_tiles, tile_at);
     } else if constexpr (EPI == EPI_CONV_GNX) {
       const int my_tiles = cta < p.num_tiles ? (p.num_tiles - cta + ncta - 1) / ncta : 0;

@@ -557,6 +557,9 @@ def test_bf16_softmax_wide_rows_one_kernel(kf, shape, act, tuning):
     assert np.abs(got.sum(axis=1) - 1.0).max() < 4e-3
     P2 = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), act, "softmax")
     assert (to_f64(P2) == got).all()                          # fixed order of the exchange: bit-identical repeats
+    tuning.setenv("KF_NO_WIDE_STORE", "1")                    # whole pieces behind group barriers instead of per-warp slabs
+    P3 = kf.gemm_rowreduce(to_dev(d["X"]), to_dev(d["W"]), to_dev(d["b"]), act, "softmax")
+    assert (to_f64(P3) == got).all()
 
 
 def _softmax_gx_fuzz_cases():

@@ -352,6 +352,9 @@ def chain_table(kf, device, peaks, c2_tensors, c2_us):
         small = name in ("c1", "c4")
         if fn is None:
             fn = lambda: kf.gemm_epilogue(t["X"], t["W"], t["b"], "gelu_tanh", 0.5, t["R"], out=c2_out)
+        n0 = kf.kf_launch_count()
+        fn()
+        kernels_per_call = int(kf.kf_launch_count() - n0)   # this library's kernels in one call: the route taken
         us = c2_us if name == "c2" else time_calls(fn, 200 if small else 40, 5, graph_batch=20 if small else 0)
         st = time_calls_stats(fn, 200 if small else 40, 5, graph_batch=20 if small else 0)
         us_torch = time_calls(torch_unfused(name, t), 200 if small else 20, 5, graph_batch=20 if small else 0)
@@ -364,7 +367,7 @@ def chain_table(kf, device, peaks, c2_tensors, c2_us):
         t_roof = max(s["flops"] / (peaks["bf16_tflops"] * 1e6), s["bytes"] / (peaks["hbm_gbs"] * 1e3))
         out[name] = {
             "us_per_call": round(us, 3), "us_median": round(st["median"], 3), "us_min": round(st["min"], 3),
-            "samples": st["samples"], "tflops": round(tf, 2),
+            "samples": st["samples"], "kernels_per_call": kernels_per_call, "tflops": round(tf, 2),
             "t_roof_us": round(t_roof, 3), "roofline_frac": round(t_roof / us, 4),
             "roofline_bound": "tensor" if s["flops"] / (peaks["bf16_tflops"] * 1e6) >= s["bytes"] / (peaks["hbm_gbs"] * 1e3) else "hbm",
             "frac_tensor_peak_measured_burst": round(tf / peaks["bf16_tflops"], 4),
@@ -392,6 +395,9 @@ def chain_table(kf, device, peaks, c2_tensors, c2_us):
     import torch.nn.functional as F
     t = c2_tensors
     oc = torch.empty(M2, N2, dtype=torch.bfloat16, device=device)
+    n0 = kf.kf_launch_count()
+    kf.gemm_epilogue(t["X"], t["W"], t["b"], "chain95", out=oc)
+    k95 = int(kf.kf_launch_count() - n0)
     us = time_calls(lambda: kf.gemm_epilogue(t["X"], t["W"], t["b"], "chain95", out=oc), 40, 5)
 
     def torch_chain95():
@@ -403,7 +409,7 @@ def chain_table(kf, device, peaks, c2_tensors, c2_us):
 
     us_torch = time_calls(torch_chain95, 20, 5)
     out["paper_chain_matmul_add_swish_tanh_gelu_hardtanh"] = {
-        "shape": "config 2's X, W, b", "us_per_call": round(us, 3),
+        "shape": "config 2's X, W, b", "us_per_call": round(us, 3), "kernels_per_call": k95,
         "tflops": round(FLOPS_C2 / us / 1e6, 2), "unfused_torch_us": round(us_torch, 3),
         "speedup_vs_unfused_torch": round(us_torch / us, 3), "paper_speedup_rtx5090": 1.31}
     # The 2-D form of the paper's case-study chain (Appendix C.1): conv, softmax over channels,
@@ -411,6 +417,9 @@ def chain_table(kf, device, peaks, c2_tensors, c2_us):
     d = ki.conv_inputs("c5", seed=0)
     t5 = {k: to_dev(d[k], device) for k in ("x", "w", "bias")}
     op = torch.empty(128, 128, 16, 16, dtype=torch.bfloat16, device=device)
+    n0 = kf.kf_launch_count()
+    kf.conv3x3_softmax_pool(t5["x"], t5["w"], t5["bias"], 4, out=op)
+    kpool = int(kf.kf_launch_count() - n0)
     us = time_calls(lambda: kf.conv3x3_softmax_pool(t5["x"], t5["w"], t5["bias"], 4, out=op), 40, 5)
 
     def torch_conv_softmax_pool():
@@ -419,7 +428,7 @@ def chain_table(kf, device, peaks, c2_tensors, c2_us):
 
     us_torch = time_calls(torch_conv_softmax_pool, 20, 5)
     out["paper_chain_conv_softmax_maxpool_maxpool_2d"] = {
-        "shape": "config 5's x, w, bias; pool 2 twice", "us_per_call": round(us, 3),
+        "shape": "config 5's x, w, bias; pool 2 twice", "us_per_call": round(us, 3), "kernels_per_call": kpool,
         "tflops": round(specs["c5"]["flops"] / us / 1e6, 2), "unfused_torch_us": round(us_torch, 3),
         "speedup_vs_unfused_torch": round(us_torch / us, 3)}
     return out
